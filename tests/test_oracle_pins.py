@@ -1,0 +1,293 @@
+"""Pins for the CPU oracle: every check here is fixed by something other than
+the oracle itself (hand-computed values, one-hot probes, numpy's fp64 matmul on
+a dense S built by independent Python code, pure-Python brute force, algebraic
+invariants of the formula)."""
+import itertools
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_36800_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------
+# independent helpers (no oracle code involved)
+# ----------------------------------------------------------------------------
+def bf16(a):
+    return synth.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+
+
+def widen(h):
+    return synth.bf16_bits_to_f32(h).astype(np.float64)
+
+
+def dense_signs_py(bits):
+    """Dense +1/-1 from packed words with explicit Python integer arithmetic."""
+    B, N, Wn = bits.shape
+    S = np.empty((B, N, Wn * 32), dtype=np.float64)
+    for b, n, w in itertools.product(range(B), range(N), range(Wn)):
+        word = int(bits[b, n, w])
+        for j in range(32):
+            S[b, n, 32 * w + j] = 1.0 if (word >> j) & 1 else -1.0
+    return S
+
+
+def dense_signs_np(bits):
+    """Dense +1/-1 via numpy's unpackbits on the little-endian byte view."""
+    B, N, Wn = bits.shape
+    by = bits.astype("<u4").view(np.uint8).reshape(B, N, Wn * 4)
+    b01 = np.unpackbits(by, axis=-1, bitorder="little")
+    return b01.astype(np.float64) * 2.0 - 1.0
+
+
+def reference_np(X, W, bits, alpha, dense=dense_signs_np):
+    x, w, S = widen(X), widen(W), dense(bits)
+    base = np.einsum("btk,nk->btn", x, w)
+    delta = np.einsum("btk,bnk->btn", x, S)
+    return base + alpha.astype(np.float64)[:, None, None] * delta
+
+
+def small_case(B, m, N, K, seed, w_std=0.02):
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, w_std=w_std, seed=seed)
+    return synth.make_inputs(wl)
+
+
+# ----------------------------------------------------------------------------
+# packing
+# ----------------------------------------------------------------------------
+def test_pack_single_positive_element_sets_one_bit():
+    B, N, K = 2, 3, 96
+    for (b, n, k) in [(0, 0, 0), (0, 1, 1), (1, 2, 31), (1, 0, 32), (0, 2, 33), (1, 1, 63), (0, 0, 64), (1, 2, 95)]:
+        S = -np.ones((B, N, K), dtype=np.int8)
+        S[b, n, k] = 1
+        bits = oracle.pack(S)
+        expect = np.zeros((B, N, K // 32), dtype=np.uint32)
+        expect[b, n, k // 32] = np.uint32(1) << np.uint32(k % 32)
+        assert np.array_equal(bits, expect), (b, n, k)
+
+
+def test_pack_hand_word():
+    # first 16 weights +1, last 16 weights -1  ->  0x0000FFFF
+    S = np.concatenate([np.ones(16), -np.ones(16)]).astype(np.int8).reshape(1, 1, 32)
+    assert oracle.pack(S)[0, 0, 0] == 0x0000FFFF
+    # alternating starting with +1 at k=0 -> 0x55555555
+    S = np.tile(np.array([1, -1], dtype=np.int8), 16).reshape(1, 1, 32)
+    assert oracle.pack(S)[0, 0, 0] == 0x55555555
+
+
+def test_pack_zero_and_negative_map_to_clear_bit():
+    S = np.array([0, -1, -128, 1, 127, 2] + [0] * 26, dtype=np.int8).reshape(1, 1, 32)
+    assert oracle.pack(S)[0, 0, 0] == (1 << 3) | (1 << 4) | (1 << 5)
+
+
+def test_pack_matches_numpy_packbits():
+    S = synth.make_signs(3, 17, 160, seed=5)
+    got = oracle.pack(S)
+    by = np.packbits((S > 0).astype(np.uint8), axis=-1, bitorder="little")
+    expect = by.reshape(3, 17, 5, 4).copy().view("<u4").reshape(3, 17, 5)
+    assert np.array_equal(got, expect)
+
+
+def test_pack_unpack_round_trip():
+    S = synth.make_signs(2, 9, 128, seed=11)
+    assert np.array_equal(oracle.unpack(oracle.pack(S)), S)
+    words = np.random.default_rng(3).integers(0, 2**32, size=(2, 5, 7), dtype=np.uint32)
+    assert np.array_equal(oracle.pack(oracle.unpack(words)), words)
+
+
+def test_unpack_matches_independent_decoders():
+    words = np.random.default_rng(4).integers(0, 2**32, size=(2, 3, 2), dtype=np.uint32)
+    S = oracle.unpack(words).astype(np.float64)
+    assert np.array_equal(S, dense_signs_py(words))
+    assert np.array_equal(S, dense_signs_np(words))
+
+
+# ----------------------------------------------------------------------------
+# the fused product
+# ----------------------------------------------------------------------------
+def test_hand_computed_known_answer():
+    # K=32, x_k = k+1, word 0x0000FFFF: (1+..+16) - (17+..+32) = 136 - 392 = -256
+    X = bf16(np.arange(1, 33, dtype=np.float32)).reshape(1, 1, 32)
+    W = np.zeros((1, 32), dtype=np.uint16)
+    bits = np.array([[[0x0000FFFF]]], dtype=np.uint32)
+    Y = oracle.gemm(X, W, bits, np.array([1.0], dtype=np.float32))
+    assert Y[0, 0, 0] == -256.0
+    # with alpha = 0.5 and w = 2 everywhere: 2*528 + 0.5*(-256) = 928
+    W2 = bf16(np.full((1, 32), 2.0))
+    Y = oracle.gemm(X, W2, bits, np.array([0.5], dtype=np.float32))
+    assert Y[0, 0, 0] == 928.0
+
+
+@pytest.mark.parametrize("k", [0, 1, 31, 32, 33, 63, 64, 95])
+def test_one_hot_probe_reads_the_right_bit(k):
+    # X = e_k, W = 0, alpha = 1  =>  Y[n] = s[n,k]
+    B, N, K = 2, 4, 96
+    rng = np.random.default_rng(100 + k)
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    x = np.zeros((B, 1, K), dtype=np.float32)
+    x[:, 0, k] = 1.0
+    Y = oracle.gemm(bf16(x), np.zeros((N, K), dtype=np.uint16), bits, np.ones(B, dtype=np.float32))
+    expect = np.where((bits[:, :, k // 32] >> np.uint32(k % 32)) & np.uint32(1), 1.0, -1.0)
+    assert np.array_equal(Y[:, 0, :], expect)
+
+
+@pytest.mark.parametrize("j", [0, 1, 15, 16, 30, 31])
+def test_single_bit_words(j):
+    # word = 1<<j, x = 1 everywhere: sum = (+1) + 31*(-1) = -30; x = e_j: +1
+    K = 32
+    bits = np.array([[[1 << j]]], dtype=np.uint32)
+    ones = bf16(np.ones((1, 1, K)))
+    Wz = np.zeros((1, K), dtype=np.uint16)
+    a1 = np.ones(1, dtype=np.float32)
+    assert oracle.gemm(ones, Wz, bits, a1)[0, 0, 0] == -30.0
+    e = np.zeros((1, 1, K), dtype=np.float32)
+    e[0, 0, j] = 1.0
+    assert oracle.gemm(bf16(e), Wz, bits, a1)[0, 0, 0] == 1.0
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 5, 64), (1, 1, 7, 96), (3, 2, 4, 32)])
+def test_brute_force_python_loops(shape):
+    B, m, N, K = shape
+    X, W, bits, alpha = small_case(B, m, N, K, seed=sum(shape))
+    got = oracle.gemm(X, W, bits, alpha)
+    x, w = widen(X), widen(W)
+    for b, t, n in itertools.product(range(B), range(m), range(N)):
+        base = 0.0
+        delta = 0.0
+        for k in range(K):
+            s = 1.0 if (int(bits[b, n, k // 32]) >> (k % 32)) & 1 else -1.0
+            base += float(x[b, t, k]) * float(w[n, k])
+            delta += float(x[b, t, k]) * s
+        expect = base + float(np.float64(alpha[b])) * delta
+        assert got[b, t, n] == pytest.approx(expect, rel=1e-13, abs=1e-13)
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 5, 64), (2, 5, 33, 96), (4, 16, 64, 512)])
+def test_matches_numpy_fp64_matmul_on_dense_signs(shape):
+    B, m, N, K = shape
+    X, W, bits, alpha = small_case(B, m, N, K, seed=7 + K)
+    got = oracle.gemm(X, W, bits, alpha)
+    expect = reference_np(X, W, bits, alpha)
+    assert np.max(np.abs(got - expect)) <= 1e-12 * max(1.0, np.max(np.abs(expect)))
+
+
+def test_alpha_zero_is_plain_gemm():
+    X, W, bits, alpha = small_case(2, 4, 24, 128, seed=21)
+    got = oracle.gemm(X, W, bits, np.zeros_like(alpha))
+    expect = np.einsum("btk,nk->btn", widen(X), widen(W))
+    assert np.allclose(got, expect, rtol=1e-13, atol=1e-13)
+
+
+def test_all_bits_set_adds_alpha_times_rowsum():
+    X, W, bits, alpha = small_case(2, 4, 24, 128, seed=22)
+    ones = np.full_like(bits, 0xFFFFFFFF)
+    zeros = np.zeros_like(bits)
+    x, w, a = widen(X), widen(W), alpha.astype(np.float64)
+    expect_p = np.einsum("btk,bnk->btn", x, w[None] + a[:, None, None])
+    expect_m = np.einsum("btk,bnk->btn", x, w[None] - a[:, None, None])
+    assert np.allclose(oracle.gemm(X, W, ones, alpha), expect_p, rtol=1e-12, atol=1e-12)
+    assert np.allclose(oracle.gemm(X, W, zeros, alpha), expect_m, rtol=1e-12, atol=1e-12)
+
+
+def test_flipping_every_bit_negates_the_delta_term():
+    X, W, bits, alpha = small_case(3, 2, 16, 160, seed=23)
+    y1 = oracle.gemm(X, W, bits, alpha)
+    y2 = oracle.gemm(X, W, ~bits, alpha)
+    base = np.einsum("btk,nk->btn", widen(X), widen(W))
+    assert np.allclose(y1 + y2, 2.0 * base, rtol=1e-12, atol=1e-12)
+    assert not np.allclose(y1, y2)
+
+
+def test_delta_is_linear_in_alpha():
+    X, W, bits, alpha = small_case(2, 3, 8, 64, seed=24)
+    y0 = oracle.gemm(X, W, bits, np.zeros_like(alpha))
+    ya = oracle.gemm(X, W, bits, alpha)
+    y2a = oracle.gemm(X, W, bits, (2 * alpha).astype(np.float32))
+    assert np.allclose(y2a - y0, 2.0 * (ya - y0), rtol=1e-11, atol=1e-13)
+
+
+def test_tenants_are_isolated_and_permute():
+    X, W, bits, alpha = small_case(3, 2, 8, 64, seed=25)
+    y = oracle.gemm(X, W, bits, alpha)
+    X2, bits2, alpha2 = X.copy(), bits.copy(), alpha.copy()
+    X2[1] = bf16(np.random.default_rng(1).standard_normal((2, 64)))
+    bits2[1] ^= np.uint32(0xDEADBEEF)
+    alpha2[1] = 0.5
+    y2 = oracle.gemm(X2, W, bits2, alpha2)
+    assert np.array_equal(y[0], y2[0]) and np.array_equal(y[2], y2[2])
+    assert not np.array_equal(y[1], y2[1])
+    perm = [2, 0, 1]
+    yp = oracle.gemm(X[perm], W, bits[perm], alpha[perm])
+    assert np.array_equal(yp, y[perm])
+
+
+def test_transposed_operands_would_be_caught():
+    # N != m and W != W^T: a transposed or mis-strided operand changes the result.
+    X, W, bits, alpha = small_case(1, 3, 5, 64, seed=26)
+    got = oracle.gemm(X, W, bits, alpha)
+    assert got.shape == (1, 3, 5)
+    expect = reference_np(X, W, bits, alpha, dense=dense_signs_py)
+    assert np.allclose(got, expect, rtol=1e-13, atol=1e-13)
+
+
+def test_gemm_at_equals_full_result_and_numpy():
+    X, W, bits, alpha = small_case(3, 4, 40, 256, seed=27)
+    full = oracle.gemm(X, W, bits, alpha)
+    rng = np.random.default_rng(0)
+    idx = np.stack([rng.integers(0, 3, 50), rng.integers(0, 4, 50), rng.integers(0, 40, 50)], axis=1).astype(np.int32)
+    got = oracle.gemm_at(X, W, bits, alpha, idx)
+    assert np.array_equal(got, full[idx[:, 0], idx[:, 1], idx[:, 2]])
+    ref = reference_np(X, W, bits, alpha)
+    assert np.allclose(got, ref[idx[:, 0], idx[:, 1], idx[:, 2]], rtol=1e-12, atol=1e-12)
+
+
+def test_extreme_magnitudes_and_cancellation():
+    # all-equal x with a balanced word: the delta term cancels exactly
+    K = 64
+    X = bf16(np.full((1, 1, K), 3.0))
+    bits = np.array([[[0x0F0F0F0F, 0xF0F0F0F0]]], dtype=np.uint32)
+    W = np.zeros((1, K), dtype=np.uint16)
+    assert oracle.gemm(X, W, bits, np.array([123.0], dtype=np.float32))[0, 0, 0] == 0.0
+    # large and tiny magnitudes stay exact in fp64
+    x = np.zeros((1, 1, K), dtype=np.float32)
+    x[0, 0, 0], x[0, 0, 1] = 2.0**15, 2.0**-20
+    w = np.zeros((1, K), dtype=np.float32)
+    w[0, 0], w[0, 1] = 2.0**-10, 2.0**10
+    y = oracle.gemm(bf16(x), bf16(w), np.zeros((1, 1, 2), dtype=np.uint32), np.array([0.0], dtype=np.float32))
+    assert y[0, 0, 0] == 2.0**5 + 2.0**-10
+
+
+# ----------------------------------------------------------------------------
+# generator determinism + stored seed-0 statistics
+# ----------------------------------------------------------------------------
+def test_bf16_rounding_is_nearest_even():
+    # 1 + 2^-8 is a tie between 1.0 (even) and 1 + 2^-7 -> 1.0; 1 + 3*2^-8 ties up to 1 + 2^-6
+    vals = np.array([1.0, 1.0 + 2.0**-8, 1.0 + 3 * 2.0**-8, 1.0 + 2.0**-8 + 2.0**-20, -2.5], dtype=np.float32)
+    got = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(vals))
+    assert list(got) == [1.0, 1.0, 1.0 + 2.0**-6, 1.0 + 2.0**-7, -2.5]
+    import ml_dtypes
+    r = np.random.default_rng(0).standard_normal(10000).astype(np.float32)
+    assert np.array_equal(synth.f32_to_bf16_bits(r), r.astype(ml_dtypes.bfloat16).view(np.uint16))
+
+
+@pytest.mark.parametrize("name", ["tiny", "decode_attn"])
+def test_seed0_statistics_match_stored_values(name):
+    with open(os.path.join(GOLDEN, "seed0_stats.json")) as f:
+        stats = json.load(f)[name]
+    wl = synth.WORKLOADS_BY_NAME[name]
+    X, W, bits, alpha = synth.make_inputs(wl)
+    assert int(X[0, 0, 0]) == stats["x000_bits"]
+    assert int(W[0, 0]) == stats["w00_bits"]
+    assert int(bits[0, 0, 0]) == stats["bits_first"]
+    assert int(bits[-1, -1, -1]) == stats["bits_last"]
+    Y = oracle.gemm(X, W, bits, alpha)
+    assert Y[0, 0, 0] == pytest.approx(stats["y_first"], rel=1e-10)
+    assert Y[-1, -1, -1] == pytest.approx(stats["y_last"], rel=1e-10)
+    assert np.abs(Y).max() == pytest.approx(stats["y_absmax"], rel=1e-10)
+    assert np.linalg.norm(Y) == pytest.approx(stats["y_fro"], rel=1e-10)
+    assert Y.sum() == pytest.approx(stats["y_sum"], rel=1e-8)
