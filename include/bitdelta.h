@@ -1,0 +1,134 @@
+/*
+ * bitdelta.h -- C ABI of the B200 (sm_100a) BitDelta fused-GEMM library.
+ *
+ * The operation (multi-tenant BitDelta product; the paper's BitDelta paragraph
+ * under "Recently Published Kernels" describes decoding packed binary weights,
+ * s = 2*bit - 1, straight into tensor-core operands; the base-weight term, the
+ * per-tenant scale and the packing order are the task's formula):
+ *
+ *   Y[b,t,n] = sum_k X[b,t,k] * W_base[n,k] + alpha[b] * sum_k X[b,t,k] * S[b,n,k]
+ *
+ * with S in {+1,-1} stored one bit per weight: word w of row (b,n) holds
+ * k = 32w .. 32w+31, bit j (value 1<<j) belongs to k = 32w+j, a set bit means
+ * +1 and a clear bit means -1.
+ *
+ * Conventions for every entry point
+ *   - plain C types only; all arrays dense, row-major, no strides;
+ *   - unless a parameter says "host", pointers are DEVICE pointers that the
+ *     caller owns; the library never frees or reallocates them;
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream);
+ *     work is queued on it and the call returns without synchronising, except
+ *     where stated;
+ *   - the return value is a bitdelta_status; on an argument error nothing is
+ *     launched;
+ *   - only compute capability 10.0 devices are served (BITDELTA_ERR_ARCH
+ *     otherwise); there is no CPU fallback.
+ */
+#ifndef BITDELTA_H_
+#define BITDELTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BITDELTA_OK = 0,
+    BITDELTA_ERR_NULL = 1,      /* a required pointer is NULL                         */
+    BITDELTA_ERR_SHAPE = 2,     /* B, m, N <= 0, K <= 0 or K not a multiple of 32     */
+    BITDELTA_ERR_ALIGN = 3,     /* a pointer is not 16-byte aligned                   */
+    BITDELTA_ERR_WORKSPACE = 4, /* workspace missing or smaller than required         */
+    BITDELTA_ERR_ARCH = 5,      /* current device is not compute capability 10.0      */
+    BITDELTA_ERR_CUDA = 6,      /* a CUDA runtime / driver call failed                */
+    BITDELTA_ERR_TIMEOUT = 7    /* a bounded wait inside a kernel expired             */
+} bitdelta_status;
+
+/*
+ * Packing step (setup, before the GEMM):  bits[b,n,w] = sum_j [S[b,n,32w+j] > 0] << j.
+ * S    : int8  [B,N,K]; any value > 0 packs as +1, zero and negatives as -1.
+ * bits : uint32 [B,N,K/32] (output).  K must be a multiple of 32.
+ * Integer work, bit-exact.  Asynchronous on the stream.
+ */
+int bitdelta_pack(const int8_t* S, uint32_t* bits, int B, int N, int K, void* cuda_stream);
+
+/* Inverse of bitdelta_pack (test aid): S[b,n,k] = +1 if the bit is set, else -1. */
+int bitdelta_unpack(const uint32_t* bits, int8_t* S, int B, int N, int K, void* cuda_stream);
+
+/*
+ * Scratch memory bitdelta_gemm needs for this problem size (may depend on the
+ * shape only, never on the data).  Returns 0 for invalid shapes.
+ */
+size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K);
+
+/*
+ * Prepares a workspace for its first use (clears the arrival counters kept at
+ * its start).  Call once after allocating the workspace; every completed
+ * bitdelta_gemm leaves the workspace ready for the next call, so it need not
+ * be repeated.  Asynchronous on the stream.
+ */
+int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The fused product defined at the top of this file.
+ * X      : bf16 [B,m,K]      activations of B tenants, m tokens each
+ * W_base : bf16 [N,K]        base weight shared by every tenant
+ * bits   : uint32 [B,N,K/32] packed signs of each tenant's delta
+ * alpha  : fp32 [B]          per-tenant scale (device memory)
+ * Y      : bf16 [B,m,N]      output; fp32 accumulation, one round-to-nearest-even
+ *                            conversion at the end
+ * workspace / workspace_bytes : at least bitdelta_gemm_workspace_bytes(B,m,N,K),
+ *          prepared once by bitdelta_workspace_init; calls that may overlap on
+ *          the device must not share a workspace.
+ * m <= 16 selects the streaming (decode) schedule, larger m the tiled (prefill)
+ * schedule; both run on tcgen05 tensor cores with TMEM accumulators.  Shapes
+ * whose K is not a multiple of 128 run on a plain CUDA-core kernel instead.
+ * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.
+ * Asynchronous on the stream; a kernel-side wait that expires is reported by
+ * bitdelta_last_device_status, not here.
+ */
+int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
+                  void* Y, int B, int m, int N, int K,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Diagnostic variant of bitdelta_gemm on plain CUDA cores (one warp per output
+ * row, fp32 accumulation in k order per lane).  Same arguments and result
+ * contract; needs no workspace.  Slow; used to triage the tensor-core path.
+ */
+int bitdelta_gemm_simt(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
+                       void* Y, int B, int m, int N, int K, void* cuda_stream);
+
+/*
+ * End-to-end form for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous).  Copies X, W_base, bits and alpha into the
+ * device arena, runs bitdelta_gemm, copies Y back to Y_host and synchronises
+ * the stream before returning, so Y_host is complete on return.
+ * arena : DEVICE memory of at least bitdelta_gemm_host_arena_bytes(B,m,N,K)
+ *         bytes, 256-byte aligned, owned by the caller.
+ */
+size_t bitdelta_gemm_host_arena_bytes(int B, int m, int N, int K);
+int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32_t* bits_host,
+                       const float* alpha_host, void* Y_host, int B, int m, int N, int K,
+                       void* arena, size_t arena_bytes, void* cuda_stream);
+
+/*
+ * Synchronises the stream, then returns and clears the device-side status of
+ * the current device: BITDELTA_OK, or BITDELTA_ERR_TIMEOUT if a bounded wait in
+ * one of this library's kernels expired since the last query (its output is
+ * then undefined).  `site`, if not NULL (host pointer), receives a code naming
+ * the wait that expired.
+ */
+int bitdelta_last_device_status(void* cuda_stream, int* site);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+unsigned long long bitdelta_kernel_launch_count(void);
+
+/* Static, human-readable text for a status code. */
+const char* bitdelta_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITDELTA_H_ */

@@ -1,0 +1,177 @@
+"""ctypes binding of libbitdelta.so (see include/bitdelta.h).
+
+Argument marshalling only: torch supplies device memory and streams, every
+step of the computation runs in the library's CUDA kernels.  Nothing here falls
+back to the CPU: a missing library or a non-sm_100 device raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libbitdelta.so")
+_lib = None
+
+STATUS_OK = 0
+STATUS_TIMEOUT = 7
+
+EXPORTS = (
+    "bitdelta_pack", "bitdelta_unpack", "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
+    "bitdelta_gemm", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
+    "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
+)
+
+
+class BitDeltaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libbitdelta.so (built in-tree by paper_2609_36800_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2609_36800_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.bitdelta_pack.argtypes = [vp, vp, ci, ci, ci, vp]
+    lib.bitdelta_unpack.argtypes = [vp, vp, ci, ci, ci, vp]
+    lib.bitdelta_gemm_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.bitdelta_gemm_workspace_bytes.restype = sz
+    lib.bitdelta_workspace_init.argtypes = [vp, sz, vp]
+    lib.bitdelta_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
+    lib.bitdelta_gemm_simt.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
+    lib.bitdelta_gemm_host_arena_bytes.argtypes = [ci, ci, ci, ci]
+    lib.bitdelta_gemm_host_arena_bytes.restype = sz
+    lib.bitdelta_gemm_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
+    lib.bitdelta_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.bitdelta_kernel_launch_count.restype = ctypes.c_ulonglong
+    lib.bitdelta_status_string.argtypes = [ci]
+    lib.bitdelta_status_string.restype = ctypes.c_char_p
+    for fn in ("bitdelta_pack", "bitdelta_unpack", "bitdelta_workspace_init", "bitdelta_gemm",
+               "bitdelta_gemm_simt", "bitdelta_gemm_host", "bitdelta_last_device_status"):
+        getattr(lib, fn).restype = ci
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().bitdelta_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != STATUS_OK:
+        raise BitDeltaError(status, where)
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def pack(S, stream=None):
+    """S int8 [B,N,K] (device) -> packed sign words, int32 storage [B,N,K/32] (bit j of word w <-> k = 32w+j)."""
+    import torch
+    B, N, K = S.shape
+    bits = torch.empty((B, N, K // 32), dtype=torch.int32, device=S.device)
+    _check(load_library().bitdelta_pack(_dev(S, torch.int8, "S"), ctypes.c_void_p(bits.data_ptr()),
+                                        B, N, K, _stream_ptr(stream)), "bitdelta_pack")
+    return bits
+
+
+def unpack(bits, stream=None):
+    """Packed sign words [B,N,K/32] (int32 storage, device) -> S int8 [B,N,K] of +1/-1."""
+    import torch
+    B, N, Wn = bits.shape
+    S = torch.empty((B, N, Wn * 32), dtype=torch.int8, device=bits.device)
+    _check(load_library().bitdelta_unpack(_dev(bits, torch.int32, "bits"), ctypes.c_void_p(S.data_ptr()),
+                                          B, N, Wn * 32, _stream_ptr(stream)), "bitdelta_unpack")
+    return S
+
+
+def gemm_workspace_bytes(B: int, m: int, N: int, K: int) -> int:
+    return int(load_library().bitdelta_gemm_workspace_bytes(B, m, N, K))
+
+
+def make_workspace(B: int, m: int, N: int, K: int, device="cuda", stream=None):
+    """Allocate and prepare a workspace for bitdelta_gemm on this shape."""
+    import torch
+    nbytes = gemm_workspace_bytes(B, m, N, K)
+    if nbytes == 0:
+        raise BitDeltaError(2, "bitdelta_gemm_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    _check(load_library().bitdelta_workspace_init(ctypes.c_void_p(ws.data_ptr()), nbytes, _stream_ptr(stream)),
+           "bitdelta_workspace_init")
+    return ws
+
+
+def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bool = False):
+    """Y[b,t,n] = sum_k X W_base + alpha[b] sum_k X S.  X bf16 [B,m,K], W_base bf16 [N,K],
+    bits int32 storage [B,N,K/32], alpha fp32 [B]; returns Y bf16 [B,m,N]."""
+    import torch
+    lib = load_library()
+    B, m, K = X.shape
+    N = W_base.shape[0]
+    if W_base.shape != (N, K) or tuple(bits.shape) != (B, N, K // 32) or tuple(alpha.shape) != (B,):
+        raise ValueError("inconsistent shapes")
+    if out is None:
+        out = torch.empty((B, m, N), dtype=torch.bfloat16, device=X.device)
+    args = [_dev(X, torch.bfloat16, "X"), _dev(W_base, torch.bfloat16, "W_base"), _dev(bits, torch.int32, "bits"),
+            _dev(alpha, torch.float32, "alpha"), _dev(out, torch.bfloat16, "out"), B, m, N, K]
+    if simt:
+        _check(lib.bitdelta_gemm_simt(*args, _stream_ptr(stream)), "bitdelta_gemm_simt")
+        return out
+    if workspace is None:
+        workspace = make_workspace(B, m, N, K, device=X.device, stream=stream)
+    _check(lib.bitdelta_gemm(*args, ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream)),
+           "bitdelta_gemm")
+    return out
+
+
+def gemm_host_arena_bytes(B: int, m: int, N: int, K: int) -> int:
+    return int(load_library().bitdelta_gemm_host_arena_bytes(B, m, N, K))
+
+
+def gemm_host(X, W_base, bits, alpha, out, arena, stream=None):
+    """Host-buffer form: all tensors are CPU tensors (pinned for asynchronous copies), `arena` is a
+    CUDA uint8 tensor of gemm_host_arena_bytes.  Returns `out` (complete on return)."""
+    import torch
+    B, m, K = X.shape
+    N = W_base.shape[0]
+    for t, dt, nm in ((X, torch.bfloat16, "X"), (W_base, torch.bfloat16, "W_base"), (bits, torch.int32, "bits"),
+                      (alpha, torch.float32, "alpha"), (out, torch.bfloat16, "out")):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise TypeError(f"{nm} must be a contiguous CPU tensor of dtype {dt}")
+    _check(load_library().bitdelta_gemm_host(
+        ctypes.c_void_p(X.data_ptr()), ctypes.c_void_p(W_base.data_ptr()), ctypes.c_void_p(bits.data_ptr()),
+        ctypes.c_void_p(alpha.data_ptr()), ctypes.c_void_p(out.data_ptr()), B, m, N, K,
+        ctypes.c_void_p(arena.data_ptr()), arena.numel(), _stream_ptr(stream)), "bitdelta_gemm_host")
+    return out
+
+
+def last_device_status(stream=None):
+    """Synchronise and return (status, site) of the device-side bounded waits."""
+    site = ctypes.c_int(0)
+    st = load_library().bitdelta_last_device_status(_stream_ptr(stream), ctypes.byref(site))
+    return int(st), int(site.value)
+
+
+def kernel_launch_count() -> int:
+    return int(load_library().bitdelta_kernel_launch_count())

@@ -1,0 +1,291 @@
+// extern "C" entry points of libbitdelta.so: argument checks, tensor-map
+// construction and kernel launches.  See include/bitdelta.h for the contract.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/bitdelta.h"
+#include "gemm_tc.h"
+#include "plan.h"
+
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) ==
+                cudaSuccess &&
+            q == cudaDriverEntryPointSuccess) {
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        }
+    });
+    return fn;
+}
+
+struct DeviceInfo {
+    int device = -1;
+    int cc_major = 0, cc_minor = 0, sms = 0;
+};
+
+// Properties of the current device, cached per device id.
+int device_info(DeviceInfo* out) {
+    static DeviceInfo cache[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return BITDELTA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < 0 || dev >= 64) return BITDELTA_ERR_CUDA;
+    if (cache[dev].device != dev) {
+        DeviceInfo d;
+        if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.cc_minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            return BITDELTA_ERR_CUDA;
+        }
+        d.device = dev;
+        cache[dev] = d;
+    }
+    *out = cache[dev];
+    return BITDELTA_OK;
+}
+
+int check_arch(DeviceInfo* d) {
+    int st = device_info(d);
+    if (st != BITDELTA_OK) return st;
+    if (d->cc_major != 10 || d->cc_minor != 0) return BITDELTA_ERR_ARCH;
+    return BITDELTA_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_pack_args(const void* a, const void* b, int B, int N, int K) {
+    if (!a || !b) return BITDELTA_ERR_NULL;
+    if (B <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return BITDELTA_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(b)) return BITDELTA_ERR_ALIGN;
+    return BITDELTA_OK;
+}
+
+int check_gemm_args(const void* X, const void* W, const void* bits, const void* alpha, const void* Y, int B, int m,
+                    int N, int K) {
+    if (!X || !W || !bits || !alpha || !Y) return BITDELTA_ERR_NULL;
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return BITDELTA_ERR_SHAPE;
+    if ((long long)B * m > 0x7FFFFFFFll / 2 || (long long)B * N > 0x7FFFFFFFll) return BITDELTA_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(bits) || !aligned16(Y)) return BITDELTA_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(alpha) & 3u) != 0) return BITDELTA_ERR_ALIGN;
+    return BITDELTA_OK;
+}
+
+// 2-D bf16 [rows, K] row-major, box = 64 columns (128 bytes, swizzled) x box_rows.
+bool encode_bf16_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 3-D uint32 [B, N, K/32], box = 8 words (32 bytes) x 128 rows x tenants.
+bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, uint64_t words, uint32_t tenants) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {words, N, B};
+    cuuint64_t strides[2] = {words * 4, words * 4 * N};
+    cuuint32_t box[3] = {8, 128, tenants};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+int bitdelta_pack(const int8_t* S, uint32_t* bits, int B, int N, int K, void* cuda_stream) {
+    int st = check_pack_args(S, bits, B, N, K);
+    if (st != BITDELTA_OK) return st;
+    DeviceInfo d;
+    st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    const long long words = (long long)B * N * (K / 32);
+    if (bd::launch_pack(S, bits, words, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches++;
+    return BITDELTA_OK;
+}
+
+int bitdelta_unpack(const uint32_t* bits, int8_t* S, int B, int N, int K, void* cuda_stream) {
+    int st = check_pack_args(bits, S, B, N, K);
+    if (st != BITDELTA_OK) return st;
+    DeviceInfo d;
+    st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    const long long words = (long long)B * N * (K / 32);
+    if (bd::launch_unpack(bits, S, words, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches++;
+    return BITDELTA_OK;
+}
+
+size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K) {
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return 0;
+    if ((K % 128) != 0) return 256;   // CUDA-core path: no scratch needed, keep the pointer non-NULL
+    bd::Plan p = bd::make_plan(B, m, N, K, 148);
+    if (!p.ok) return 0;
+    return p.ws_bytes;
+}
+
+int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!workspace) return BITDELTA_ERR_NULL;
+    if (workspace_bytes == 0) return BITDELTA_ERR_WORKSPACE;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    return BITDELTA_OK;
+}
+
+int bitdelta_gemm_simt(const void* X, const void* W_base, const uint32_t* bits, const float* alpha, void* Y, int B,
+                       int m, int N, int K, void* cuda_stream) {
+    int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
+    if (st != BITDELTA_OK) return st;
+    DeviceInfo d;
+    st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    if (bd::launch_gemm_simt(X, W_base, bits, alpha, Y, B, m, N, K, static_cast<cudaStream_t>(cuda_stream)) !=
+        cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches++;
+    return BITDELTA_OK;
+}
+
+int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha, void* Y, int B, int m,
+                  int N, int K, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
+    if (st != BITDELTA_OK) return st;
+    DeviceInfo d;
+    st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    if ((K % 128) != 0) {
+        // Row pitch of the sign words is not a multiple of 16 bytes: no tensor map exists for it.
+        if (bd::launch_gemm_simt(X, W_base, bits, alpha, Y, B, m, N, K, stream) != cudaSuccess)
+            return BITDELTA_ERR_CUDA;
+        g_launches++;
+        return BITDELTA_OK;
+    }
+
+    bd::Plan p = bd::make_plan(B, m, N, K, d.sms);
+    if (!p.ok) return BITDELTA_ERR_SHAPE;
+    if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
+
+    CUtensorMap tmW, tmX, tmBits;
+    if (!encode_bf16_2d(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
+    if (!encode_bf16_2d(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
+    if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB))
+        return BITDELTA_ERR_CUDA;
+
+    bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
+    if (bd::launch_gemm_tc(tmW, tmX, tmBits, args, p.grid, p.smem_bytes, stream) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches++;
+    return BITDELTA_OK;
+}
+
+size_t bitdelta_gemm_host_arena_bytes(int B, int m, int N, int K) {
+    size_t ws = bitdelta_gemm_workspace_bytes(B, m, N, K);
+    if (ws == 0) return 0;
+    size_t total = 0;
+    total += align_up((size_t)B * m * K * 2, 256);
+    total += align_up((size_t)N * K * 2, 256);
+    total += align_up((size_t)B * N * (K / 32) * 4, 256);
+    total += align_up((size_t)B * 4, 256);
+    total += align_up((size_t)B * m * N * 2, 256);
+    total += align_up(ws, 256);
+    return total;
+}
+
+int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32_t* bits_host,
+                       const float* alpha_host, void* Y_host, int B, int m, int N, int K, void* arena,
+                       size_t arena_bytes, void* cuda_stream) {
+    if (!X_host || !W_base_host || !bits_host || !alpha_host || !Y_host || !arena) return BITDELTA_ERR_NULL;
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return BITDELTA_ERR_SHAPE;
+    const size_t need = bitdelta_gemm_host_arena_bytes(B, m, N, K);
+    if (need == 0) return BITDELTA_ERR_SHAPE;
+    if (arena_bytes < need) return BITDELTA_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return BITDELTA_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const size_t xb = (size_t)B * m * K * 2, wb = (size_t)N * K * 2, bb = (size_t)B * N * (K / 32) * 4;
+    const size_t ab = (size_t)B * 4, yb = (size_t)B * m * N * 2;
+    const size_t ws = bitdelta_gemm_workspace_bytes(B, m, N, K);
+    char* p = static_cast<char*>(arena);
+    void* dX = p;      p += align_up(xb, 256);
+    void* dW = p;      p += align_up(wb, 256);
+    void* dBits = p;   p += align_up(bb, 256);
+    void* dAlpha = p;  p += align_up(ab, 256);
+    void* dY = p;      p += align_up(yb, 256);
+    void* dWs = p;
+
+    if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dW, W_base_host, wb, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dBits, bits_host, bb, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dAlpha, alpha_host, ab, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    // Only the arrival counters at the start of the workspace have to be clear.
+    bd::Plan plan = bd::make_plan(B, m, N, K, 148);
+    const size_t header = plan.ok ? plan.ws_header_bytes : (ws < 256 ? ws : 256);
+    if (cudaMemsetAsync(dWs, 0, header, stream) != cudaSuccess) return BITDELTA_ERR_CUDA;
+    int st = bitdelta_gemm(dX, dW, static_cast<const uint32_t*>(dBits), static_cast<const float*>(dAlpha), dY, B, m,
+                           N, K, dWs, ws, cuda_stream);
+    if (st != BITDELTA_OK) return st;
+    if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return BITDELTA_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return BITDELTA_ERR_CUDA;
+    return BITDELTA_OK;
+}
+
+int bitdelta_last_device_status(void* cuda_stream, int* site) {
+    unsigned int st[2] = {0, 0};
+    if (bd::read_device_status(st, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return BITDELTA_ERR_CUDA;
+    if (site) *site = (int)st[1];
+    return st[0] == 0 ? BITDELTA_OK : (int)st[0];
+}
+
+unsigned long long bitdelta_kernel_launch_count(void) { return g_launches.load(); }
+
+const char* bitdelta_status_string(int status) {
+    switch (status) {
+        case BITDELTA_OK: return "ok";
+        case BITDELTA_ERR_NULL: return "null pointer argument";
+        case BITDELTA_ERR_SHAPE: return "invalid shape (B, m, N, K must be positive and K a multiple of 32)";
+        case BITDELTA_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case BITDELTA_ERR_WORKSPACE: return "workspace missing or too small";
+        case BITDELTA_ERR_ARCH: return "device is not compute capability 10.0 (sm_100a required)";
+        case BITDELTA_ERR_CUDA: return "CUDA runtime or driver call failed";
+        case BITDELTA_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,447 @@
+// BitDelta fused GEMM on tcgen05 tensor cores (sm_100a).
+//
+//   Y[b,t,n] = sum_k X[b,t,k] W[n,k] + alpha[b] sum_k X[b,t,k] S[b,n,k]
+//
+// The product is computed transposed: weight rows sit on the MMA's M side (128
+// TMEM lanes), tokens on its N side.  Per 128-wide k step a CTA
+//   * TMA-loads a W_base tile and an X tile into 128B-swizzled shared memory,
+//   * TMA-loads the tile's sign words (32 bytes per weight row and tenant),
+//   * decodes each tenant's signs into packed bf16 +-1 registers with integer
+//     ops and stores them into TENSOR MEMORY as the A operand (no shared-memory
+//     round trip for the 16x expanded weights),
+//   * issues the base MMA (A = W tile from shared memory) into one accumulator
+//     and one delta MMA per tenant (A = decoded signs from tensor memory) into a
+//     second accumulator,
+// and the epilogue forms base + alpha * delta in fp32, rounds once to bf16.
+// Work is a flat list of (tile, k step) items cut evenly across a persistent
+// grid; tiles cut across CTAs are summed through a workspace by the last CTA
+// to arrive, in a fixed order.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "gemm_tc.h"
+#include "ptx.cuh"
+
+namespace bd {
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every spin gives up after 2 s
+constexpr int kThreads = 512;
+constexpr int kWarpProducer = 0;
+constexpr int kWarpMma = 1;
+constexpr int kWarpTmem = 2;
+constexpr int kWarpDecode0 = 4;    // warps 4..11
+constexpr int kWarpEpi0 = 12;      // warps 12..15
+
+__device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] site of the first failure
+
+struct Ctl {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t bfull[kBitSlots];
+    uint64_t bempty[kBitSlots];
+    uint64_t afull[kMaxASlots];
+    uint64_t aempty[kMaxASlots];
+    uint64_t accfull;
+    uint64_t accempty;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t is_last;
+};
+static_assert(sizeof(Ctl) <= kSmemCtrlBytes, "control block too large");
+
+// Bounded wait on an mbarrier phase.  Returns false if the wait was abandoned
+// (limit reached here or in another thread of the CTA).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    const uint64_t t0 = global_timer_ns();
+#pragma unroll 1
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
+            return false;
+        }
+    }
+}
+
+// Walks the k-pair items [lo, hi) of this CTA as segments (unit, p0, p1).
+struct SegIter {
+    long long cur, hi;
+    int P;
+    __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
+        if (cur >= hi) return false;
+        unit = (int)(cur / P);
+        p0 = (int)(cur - (long long)unit * P);
+        long long rem = hi - cur;
+        int len = (rem < (long long)(P - p0)) ? (int)rem : (P - p0);
+        p1 = p0 + len;
+        cur += len;
+        return true;
+    }
+};
+
+struct Unit {
+    int n0;        // first weight row of the tile
+    int tenant0;   // first tenant
+    int nten;      // tenants in this unit
+    int xrow0;     // first row of X (in the [B*m, K] view) staged for this unit
+    int ntok;      // output tokens of this unit (rows xrow0 .. xrow0+ntok-1)
+};
+
+__device__ __forceinline__ Unit unit_info(const GemmArgs& a, int unit) {
+    Unit u;
+    const int nt = unit / a.groups;
+    const int g = unit - nt * a.groups;
+    u.n0 = nt * kTileN;
+    if (a.decode) {
+        u.tenant0 = g * a.TB;
+        u.nten = min(a.TB, a.B - u.tenant0);
+        u.xrow0 = u.tenant0 * a.m;
+        u.ntok = u.nten * a.m;
+    } else {
+        const int b = g / a.m_tiles;
+        const int mt = g - b * a.m_tiles;
+        u.tenant0 = b;
+        u.nten = 1;
+        u.xrow0 = b * a.m + mt * a.tok_tile;
+        u.ntok = min(a.tok_tile, a.m - mt * a.tok_tile);
+    }
+    return u;
+}
+
+// 32 packed sign bits (k = 0..31 of the word, LSB first) -> 16 registers of two
+// bf16 each, register c = {k = 2c (low half), k = 2c+1 (high half)}, +1 for a
+// set bit and -1 for a clear bit.  Only shifts and three-input logic ops: the
+// wanted bits are moved onto the two bf16 sign positions and flip the sign of a
+// packed (-1, -1) constant.
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t* r) {
+    // even bits of the low half stay at 2c, odd bits move to 2c+16 (junk only on odd positions)
+    const uint32_t lo = (w & 0x0000FFFFu) | ((w << 15) & 0xFFFF0000u);
+    const uint32_t hi = (w >> 16) | ((w >> 1) & 0xFFFF0000u);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        r[c] = ((lo << (15 - 2 * c)) & 0x80008000u) ^ 0xBF80BF80u;
+        r[8 + c] = ((hi << (15 - 2 * c)) & 0x80008000u) ^ 0xBF80BF80u;
+    }
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                        const __grid_constant__ CUtensorMap tmBits, const GemmArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t stages_addr = base;
+    const uint32_t bits_addr = base + a.stages * a.stage_bytes;
+    uint8_t* bits_ptr = smem + a.stages * a.stage_bytes;
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + a.stages * a.stage_bytes + kBitSlots * a.bslot_bytes);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int s = 0; s < kBitSlots; ++s) {
+            mbar_init(smem_u32(&ctl->bfull[s]), 1);
+            mbar_init(smem_u32(&ctl->bempty[s]), 8);
+        }
+        for (int s = 0; s < kMaxASlots; ++s) {
+            mbar_init(smem_u32(&ctl->afull[s]), 4);
+            mbar_init(smem_u32(&ctl->aempty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->accfull), 1);
+        mbar_init(smem_u32(&ctl->accempty), 4);
+        ctl->abort_flag = 0;
+        ctl->is_last = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmW);
+        prefetch_tensormap(&tmX);
+        prefetch_tensormap(&tmBits);
+    }
+    if (warp == kWarpTmem) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const long long lo = (long long)blockIdx.x * a.T / gridDim.x;
+    const long long hi = (long long)(blockIdx.x + 1) * a.T / gridDim.x;
+    SegIter it{lo, hi, a.P};
+    int unit, p0, p1;
+
+    if (warp == kWarpProducer) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0, bslot = 0;
+            uint32_t phase = 0, bphase = 0;
+            bool ok = true;
+            while (ok && it.next(unit, p0, p1)) {
+                const Unit u = unit_info(a, unit);
+                for (int p = p0; p < p1 && ok; ++p) {
+                    if (p == p0 || !(p & 1)) {
+                        ok = wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1);
+                        if (!ok) break;
+                        const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
+                        mbar_arrive_expect_tx(bar, a.bslot_bytes);
+                        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+                        if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                    }
+                    ok = wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t dst = stages_addr + stage * a.stage_bytes;
+                    mbar_arrive_expect_tx(bar, a.stage_bytes);
+                    const int k0 = p * kPairK;
+                    tma_load_2d(dst, &tmW, bar, k0, u.n0);
+                    tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+                    tma_load_2d(dst + 2 * a.w_atom_bytes, &tmX, bar, k0, u.xrow0);
+                    tma_load_2d(dst + 2 * a.w_atom_bytes + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
+                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+            const uint32_t idesc_delta = make_idesc_bf16(kTileN, (uint32_t)a.Nd);
+            const uint64_t desc_hi = make_smem_desc_sw128(0) & 0xFFFFFFFF00000000ull;
+            const uint32_t desc_lo_fixed = (uint32_t)(make_smem_desc_sw128(0) & 0xFFFF0000ull);
+            auto desc = [&](uint32_t addr) -> uint64_t {
+                return desc_hi | (uint64_t)(desc_lo_fixed | ((addr >> 4) & 0x3FFFu));
+            };
+            const uint32_t amask = (uint32_t)a.a_slots - 1;
+            const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+            int stage = 0;
+            uint32_t phase = 0, accphase = 0, item = 0;
+            bool ok = true;
+            while (ok && it.next(unit, p0, p1)) {
+                const Unit u = unit_info(a, unit);
+                ok = wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3);
+                if (!ok) break;
+                tc_fence_after();
+                for (int p = p0; p < p1 && ok; ++p) {
+                    ok = wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t wbase = stages_addr + stage * a.stage_bytes;
+                    const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t atom = kk >> 2, k16 = kk & 3;
+                        umma_ss(tmem_base, desc(wbase + atom * a.w_atom_bytes + k16 * 32),
+                                desc(xbase + atom * a.x_atom_bytes + k16 * 32), idesc_base,
+                                (p > p0 || kk > 0) ? 1u : 0u);
+                    }
+                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                        const uint32_t slot = item & amask;
+                        const uint32_t use = item >> ashift;
+                        ok = wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                        const uint32_t a_tmem = tmem_base + a.col_a + slot * kASlotCols;
+                        const uint32_t xwin = xbase + (uint32_t)(j * a.win_rows) * 128u;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t atom = kk >> 2, k16 = kk & 3;
+                            umma_ts(d_tmem, a_tmem + kk * 8, desc(xwin + atom * a.x_atom_bytes + k16 * 32),
+                                    idesc_delta, (p > p0 || kk > 0) ? 1u : 0u);
+                        }
+                        tc_commit(smem_u32(&ctl->aempty[slot]));
+                    }
+                    if (!ok) break;
+                    tc_commit(smem_u32(&ctl->empty[stage]));
+                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctl->accfull));
+                accphase ^= 1;
+            }
+        }
+    } else if (warp >= kWarpDecode0 && warp < kWarpEpi0) {
+        // ------------------------------------------- sign decode -> tensor memory
+        const int grp = (warp - kWarpDecode0) >> 2;
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const uint32_t amask = (uint32_t)a.a_slots - 1;
+        const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+        int bslot = 0;
+        uint32_t bphase = 0, item = 0;
+        bool ok = true;
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            for (int p = p0; p < p1 && ok; ++p) {
+                if (p == p0 || !(p & 1)) {
+                    ok = wait_bar(smem_u32(&ctl->bfull[bslot]), bphase, abort_flag, 6);
+                    if (!ok) break;
+                }
+                const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
+                for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                    if ((int)(item & 1) != grp) continue;
+                    const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
+                    const uint32_t slot = item & amask;
+                    const uint32_t use = item >> ashift;
+                    ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t taddr = lane_taddr + a.col_a + slot * kASlotCols;
+                    uint32_t r[32];
+                    decode_word(w.x, r);
+                    decode_word(w.y, r + 16);
+                    tmem_st32(taddr, r);
+                    decode_word(w.z, r);
+                    decode_word(w.w, r + 16);
+                    tmem_st32(taddr + 32, r);
+                    tc_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                }
+                if (!ok) break;
+                if ((p & 1) || p == p1 - 1) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->bempty[bslot]));
+                    if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                }
+            }
+        }
+    } else if (warp >= kWarpEpi0) {
+        // ---------------------------------------------------------------- epilogue
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int etid = threadIdx.x - kWarpEpi0 * 32;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int first_unit = (int)(lo / a.P);
+        __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
+        uint32_t accphase = 0;
+        bool ok = true;
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            const int n = u.n0 + row;
+            const bool whole = (p0 == 0 && p1 == a.P);
+            float* slotp = nullptr;
+            if (!whole) {
+                const int slot = (unit == first_unit) ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1;
+                slotp = a.partials + (size_t)slot * a.slot_floats;
+            }
+            ok = wait_bar(smem_u32(&ctl->accfull), accphase, abort_flag, 8);
+            if (!ok) break;
+            tc_fence_after();
+            accphase ^= 1;
+            const int nchunks = a.decode ? u.nten : (u.ntok + 15) / 16;
+            for (int i = 0; i < nchunks; ++i) {
+                uint32_t rb[16], rd[16];
+                tmem_ld16(lane_taddr + (uint32_t)(i * a.chunk_rows), rb);
+                tmem_ld16(lane_taddr + a.col_delta + (uint32_t)(i * 16), rd);
+                tc_wait_ld();
+                const float al = __ldg(a.alpha + (a.decode ? u.tenant0 + i : u.tenant0));
+                const int tok0 = i * a.chunk_rows;
+                const int nvalid = a.decode ? a.m : min(16, u.ntok - tok0);
+#pragma unroll
+                for (int t = 0; t < 16; ++t) {
+                    if (t < nvalid) {
+                        const float v = fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t]));
+                        if (whole) {
+                            if (n < a.N) Y[(size_t)(u.xrow0 + tok0 + t) * a.N + n] = __float2bfloat16_rn(v);
+                        } else {
+                            slotp[(size_t)(tok0 + t) * kTileN + row] = v;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
+
+            if (!whole) {
+                // This tile is cut across CTAs: publish the partial, count arrivals, and let
+                // the last CTA to arrive add the partials in CTA order and write Y.
+                const long long first_item = (long long)unit * a.P;
+                const int c0 = (int)(((first_item + 1) * gridDim.x - 1) / a.T);
+                const int c1 = (int)(((first_item + a.P) * (long long)gridDim.x - 1) / a.T);
+                __threadfence();
+                epi_bar_sync();
+                if (etid == 0) {
+                    const unsigned old = atomicAdd(&a.counters[unit], 1u);
+                    ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
+                }
+                epi_bar_sync();
+                if (ctl->is_last) {
+                    __threadfence();
+                    for (int tk = 0; tk < u.ntok; ++tk) {
+                        float sum = 0.f;
+                        for (int c = c0; c <= c1; ++c) {
+                            const int cfirst = (int)(((long long)c * a.T / gridDim.x) / a.P);
+                            const int slot = (unit == cfirst) ? 2 * c : 2 * c + 1;
+                            sum += __ldcg(a.partials + (size_t)slot * a.slot_floats + (size_t)tk * kTileN + row);
+                        }
+                        if (n < a.N) Y[(size_t)(u.xrow0 + tk) * a.N + n] = __float2bfloat16_rn(sum);
+                    }
+                    if (etid == 0) a.counters[unit] = 0u;
+                }
+                epi_bar_sync();   // is_last is rewritten by the next cut tile
+            }
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    __syncthreads();
+    if (*abort_flag) {
+        // A wait was abandoned: give copies and MMAs still in flight a bounded time to land
+        // before shared and tensor memory are released.
+        if (threadIdx.x == 0) {
+            const uint64_t t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 2000000ull) {
+            }
+        }
+        __syncthreads();
+    }
+    tc_fence_after();
+    if (warp == kWarpTmem) {
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmBits,
+                           const GemmArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(bitdelta_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kSmemBudget);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    bitdelta_gemm_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tmW, tmX, tmBits, args);
+    return cudaGetLastError();
+}
+
+cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyFromSymbol(out, g_device_status, sizeof(unsigned int) * 2);
+    if (e != cudaSuccess) return e;
+    if (out[0] != 0) {
+        unsigned int zero[2] = {0, 0};
+        e = cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero));
+    }
+    return e;
+}
+
+}  // namespace bd

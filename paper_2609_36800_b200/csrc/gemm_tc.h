@@ -1,0 +1,56 @@
+// Device-side arguments and launcher of the tcgen05 BitDelta GEMM kernel.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "plan.h"
+
+namespace bd {
+
+struct GemmArgs {
+    int B, m, N, K;
+    int decode, TB, tok_tile, Nb, Nd, win_rows, chunk_rows;
+    int m_tiles, groups, P;
+    long long T;
+    int stages, a_slots;
+    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, bslot_bytes;
+    uint32_t col_delta, col_a;
+    uint32_t slot_floats;
+    const float* alpha;
+    void* Y;
+    unsigned int* counters;
+    float* partials;
+};
+
+inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* workspace) {
+    GemmArgs a{};
+    a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
+    a.decode = p.decode; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
+    a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows;
+    a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = p.T;
+    a.stages = p.stages; a.a_slots = p.a_slots;
+    a.stage_bytes = p.stage_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
+    a.bslot_bytes = p.bslot_bytes;
+    a.col_delta = p.col_delta; a.col_a = p.col_a;
+    a.slot_floats = (uint32_t)p.slot_floats;
+    a.alpha = alpha; a.Y = Y;
+    a.counters = reinterpret_cast<unsigned int*>(workspace);
+    a.partials = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + p.ws_header_bytes);
+    return a;
+}
+
+cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmBits,
+                           const GemmArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream);
+
+// Synchronises the stream, reads {status, site} and clears them if set.
+cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream);
+
+// Plain kernels (pack / unpack / CUDA-core GEMM).
+cudaError_t launch_pack(const int8_t* S, uint32_t* bits, long long words, cudaStream_t stream);
+cudaError_t launch_unpack(const uint32_t* bits, int8_t* S, long long words, cudaStream_t stream);
+cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, void* Y,
+                             int B, int m, int N, int K, cudaStream_t stream);
+
+}  // namespace bd

@@ -1,0 +1,114 @@
+// Host-side schedule of the tcgen05 BitDelta GEMM kernel: tile shapes, shared /
+// tensor memory budget, work decomposition and workspace layout.  Pure integer
+// arithmetic; shared by the launcher and the workspace-size query.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+namespace bd {
+
+constexpr int kTileN = 128;          // weight rows per tile = MMA M = TMEM lanes
+constexpr int kPairK = 128;          // reduction extent of one pipeline stage (two 64-wide swizzle atoms)
+constexpr int kAtomK = 64;           // bf16 elements in one 128-byte swizzled row
+constexpr int kQuadK = 256;          // reduction extent of one sign-word slot (8 words = 32 bytes per row)
+constexpr int kMaxStages = 8;
+constexpr int kBitSlots = 2;
+constexpr int kMaxASlots = 4;
+constexpr int kASlotCols = 64;       // TMEM columns of one decoded operand slot (128 k, two bf16 per column)
+constexpr int kTmemCols = 512;
+constexpr int kMaxCtas = 256;        // upper bound on the grid, sizes the workspace
+constexpr int kDecodeMaxM = 16;      // m <= 16: tenants are grouped into one tile
+constexpr int kSmemBudget = 227 * 1024;
+constexpr int kSmemCtrlBytes = 1024; // barriers, TMEM base, flags
+
+struct Plan {
+    int B, m, N, K;
+    int decode;        // 1: tenants grouped (m <= 16); 0: token tiles of one tenant
+    int TB;            // tenants per unit
+    int tok_tile;      // tokens per unit and tenant in the tiled schedule (0 in decode)
+    int Nb;            // N of the base MMA  (columns of the base accumulator)
+    int Nd;            // N of a delta MMA   (columns of one tenant's delta accumulator)
+    int win_rows;      // X-tile row where tenant j's delta window starts = j * win_rows
+    int chunk_rows;    // epilogue: rows of the X tile between consecutive 16-token chunks
+    int x_rows;        // rows of X staged per stage (TMA box height)
+    int n_tiles, m_tiles, groups, units;
+    int P;             // k-pairs per unit
+    long long T;       // total k-pair work items = units * P
+    int grid;
+    int stages, a_slots;
+    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, bslot_bytes, smem_bytes;
+    uint32_t col_base, col_delta, col_a;
+    size_t slot_floats;   // floats of one partial-result slot: 128 rows x tokens per unit
+    size_t ws_header_bytes;   // arrival counters: one u32 per work unit
+    size_t ws_bytes;
+    bool ok;
+};
+
+inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
+    Plan p{};
+    p.B = B; p.m = m; p.N = N; p.K = K;
+    p.ok = false;
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 128) != 0) return p;
+    p.decode = (m <= kDecodeMaxM) ? 1 : 0;
+    p.n_tiles = (N + kTileN - 1) / kTileN;
+    if (p.decode) {
+        p.TB = B < 8 ? B : 8;
+        p.tok_tile = 0;
+        p.groups = (B + p.TB - 1) / p.TB;
+        p.m_tiles = 1;
+        p.Nb = round_up(p.TB * m, 16);
+        p.Nd = 16;
+        p.win_rows = m;
+        p.chunk_rows = m;
+        int need = (p.TB - 1) * m + 16;
+        p.x_rows = round_up(need > p.Nb ? need : p.Nb, 8);
+        p.slot_floats = (size_t)kTileN * p.TB * m;
+    } else {
+        p.TB = 1;
+        p.tok_tile = m >= 128 ? 128 : round_up(m, 16);
+        p.m_tiles = (m + p.tok_tile - 1) / p.tok_tile;
+        p.groups = B * p.m_tiles;
+        p.Nb = p.tok_tile;
+        p.Nd = p.tok_tile;
+        p.win_rows = 0;
+        p.chunk_rows = 16;
+        p.x_rows = p.tok_tile;
+        p.slot_floats = (size_t)kTileN * p.tok_tile;
+    }
+    p.units = p.n_tiles * p.groups;
+    p.P = (K + kPairK - 1) / kPairK;
+    p.T = (long long)p.units * p.P;
+    int max_grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
+    p.grid = p.T < max_grid ? (int)p.T : max_grid;
+
+    p.w_atom_bytes = kTileN * 128;
+    p.x_atom_bytes = (uint32_t)p.x_rows * 128;
+    p.stage_bytes = 2 * p.w_atom_bytes + 2 * p.x_atom_bytes;
+    p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
+    int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
+    p.stages = avail / (int)p.stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (p.stages < 2) return p;
+    p.smem_bytes = 1024 + p.stages * p.stage_bytes + kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
+    // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
+    if (p.smem_bytes < 120 * 1024) p.smem_bytes = 120 * 1024;
+
+    p.col_base = 0;
+    p.col_delta = (uint32_t)p.Nb;
+    p.col_a = p.col_delta + (uint32_t)(p.TB * p.Nd);
+    int free_cols = kTmemCols - (int)p.col_a;
+    p.a_slots = free_cols / kASlotCols;
+    if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
+    p.a_slots &= ~1;   // the two decode groups alternate slots
+    if (p.a_slots < 2) return p;
+
+    // Workspace: arrival counters, then two partial-result slots per CTA.
+    p.ws_header_bytes = (size_t)round_up(p.units * 4, 1024);
+    p.ws_bytes = p.ws_header_bytes + (size_t)2 * kMaxCtas * p.slot_floats * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+}  // namespace bd

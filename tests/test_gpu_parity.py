@@ -1,0 +1,187 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the fp64 CPU oracle,
+element by element on the same seeded inputs.
+
+Gates: packing bit-exact; GEMM max|Y - Y_ref| <= 2e-2 and relative Frobenius error
+<= 5e-3 against the unrounded fp64 result (the output's own bf16 rounding accounts
+for up to 2^-6 = 1.5625e-2 of the first bound when |Y| is in [4, 8))."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_36800_b200 as bd
+from paper_2609_36800_b200 import synth
+
+from gpu_util import assert_parity, errors, run_gemm, to_device, y_to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ packing
+@pytest.mark.parametrize("shape", [(1, 1, 32), (2, 5, 96), (3, 130, 4096), (1, 11008, 512)])
+def test_pack_unpack_bit_exact(shape):
+    B, N, K = shape
+    S = synth.make_signs(B, N, K, seed=K + N)
+    # non-(+-1) values follow the rule bit = (s > 0)
+    S.reshape(-1)[::7] = 0
+    S.reshape(-1)[::11] = -128
+    S.reshape(-1)[::13] = 127
+    dS = torch.from_numpy(S).cuda()
+    words = bd.pack(dS)
+    torch.cuda.synchronize()
+    got = words.cpu().numpy().view(np.uint32)
+    expect = oracle.pack(S)
+    assert np.array_equal(got, expect)
+    back = bd.unpack(words).cpu().numpy()
+    assert np.array_equal(back, oracle.unpack(expect))
+
+
+# --------------------------------------------------------- layout pins on GPU
+@pytest.mark.parametrize("m", [1, 4, 16, 40])
+def test_one_hot_probe_bit_and_word_order(m):
+    # X = e_k per token, W = 0, alpha = 1  =>  Y[b,t,n] = s[b,n,k_t]: exact in bf16
+    B, N, K = 3, 256, 384
+    rng = np.random.default_rng(m)
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    ks = rng.integers(0, K, size=(B, m))
+    ks[:, 0] = [0, 31, K - 1]
+    x = np.zeros((B, m, K), dtype=np.float32)
+    for b in range(B):
+        for t in range(m):
+            x[b, t, ks[b, t]] = 1.0
+    X = synth.f32_to_bf16_bits(x)
+    W = np.zeros((N, K), dtype=np.uint16)
+    alpha = np.ones(B, dtype=np.float32)
+    Y = run_gemm(X, W, bits, alpha)
+    Yref = oracle.gemm(X, W, bits, alpha)
+    assert np.array_equal(Y, Yref)
+
+
+def test_alpha_zero_and_all_ones_bits():
+    wl = synth.Workload("t", B=2, m=3, K=512, N=384, seed=3)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Yref0 = oracle.gemm(X, W, bits, np.zeros_like(alpha))
+    assert_parity(run_gemm(X, W, bits, np.zeros_like(alpha)), Yref0, "alpha=0")
+    ones = np.full_like(bits, 0xFFFFFFFF)
+    big = (alpha * 10).astype(np.float32)
+    assert_parity(run_gemm(X, W, ones, big), oracle.gemm(X, W, ones, big), "all bits set")
+
+
+# ------------------------------------------------ small shapes, ragged tails
+SMALL = [
+    # B, m, N, K        (several tiles, ragged N, odd tenant counts, every m regime)
+    (1, 1, 128, 128),
+    (1, 16, 512, 512),
+    (2, 1, 200, 256),
+    (3, 2, 384, 640),
+    (5, 3, 130, 384),
+    (8, 1, 1024, 1024),
+    (9, 4, 520, 512),
+    (11, 5, 256, 1152),
+    (16, 8, 384, 768),
+    (17, 15, 136, 256),
+    (3, 16, 264, 384),
+    (2, 17, 256, 384),
+    (1, 64, 384, 512),
+    (2, 100, 300, 640),
+    (3, 127, 128, 256),
+    (2, 128, 256, 1024),
+    (1, 200, 520, 384),
+    (2, 300, 136, 512),
+]
+
+
+@pytest.mark.parametrize("shape", SMALL, ids=lambda s: "B%d_m%d_N%d_K%d" % s)
+def test_small_shapes_match_oracle(shape):
+    B, m, N, K = shape
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B * 1000 + m)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Yref = oracle.gemm(X, W, bits, alpha)
+    Y = run_gemm(X, W, bits, alpha)
+    assert_parity(Y, Yref, str(shape))
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 96, 96), (1, 20, 130, 224), (3, 1, 64, 32)])
+def test_k_not_multiple_of_128_uses_cuda_core_kernel(shape):
+    B, m, N, K = shape
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=5)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    assert_parity(run_gemm(X, W, bits, alpha), oracle.gemm(X, W, bits, alpha), str(shape))
+
+
+@pytest.mark.parametrize("shape", [(2, 4, 256, 512), (2, 40, 256, 512)])
+def test_diagnostic_simt_kernel_matches_oracle(shape):
+    B, m, N, K = shape
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=6)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    assert_parity(run_gemm(X, W, bits, alpha, simt=True), oracle.gemm(X, W, bits, alpha), str(shape))
+
+
+def test_stress_values_large_small_and_cancelling():
+    # magnitudes up to 2^7 and down to 2^-20, exact cancellation in the delta term, signed zeros
+    B, m, N, K = 2, 4, 256, 512
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((B, m, K)).astype(np.float32)
+    x[0, 0, :] = 3.0                      # all-equal row
+    x[0, 1, ::2] = 2.0**7
+    x[0, 1, 1::2] = -(2.0**7)
+    x[1, 0, :] = 2.0**-20
+    x[1, 1, :] = -0.0
+    w = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    w[0, :] = 0.0
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    bits[0, :, :] = 0x0F0F0F0F            # balanced words: delta of the all-equal row is exactly 0
+    alpha = np.array([0.5, 0.001], dtype=np.float32)
+    X, W = synth.f32_to_bf16_bits(x), synth.f32_to_bf16_bits(w)
+    Yref = oracle.gemm(X, W, bits, alpha)
+    Y = run_gemm(X, W, bits, alpha)
+    # relative gate per element here: values reach |Y| ~ 1e3, where bf16 spacing exceeds 2e-2
+    tol = np.maximum(2e-2, np.abs(Yref) * 2.0**-8)
+    assert np.all(np.abs(Y - Yref) <= tol)
+    assert np.all(Y[1, 1] == 0.0)
+
+
+# -------------------------------------------------- the five seeded workloads
+@pytest.mark.parametrize("name", [w.name for w in synth.WORKLOADS])
+def test_workload_matches_oracle(name):
+    wl = synth.WORKLOADS_BY_NAME[name]
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Yref = oracle.gemm(X, W, bits, alpha)
+    Y = run_gemm(X, W, bits, alpha)
+    max_abs, rel_fro = assert_parity(Y, Yref, name)
+    # a correct fp32-accumulate kernel sits on the floor set by the bf16 rounding of Y
+    # (rel. Frobenius ~1.66e-3); far below that would mean comparing against the wrong thing
+    assert rel_fro > 5e-4, f"{name}: rel_fro={rel_fro:.3e} is implausibly small"
+    print(f"{name}: max_abs={max_abs:.4e} rel_fro={rel_fro:.4e}")
+
+
+def test_repeated_calls_are_bit_identical_and_reuse_workspace():
+    wl = synth.WORKLOADS_BY_NAME["decode_attn"]
+    X, W, bits, alpha = synth.make_inputs(wl)
+    dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
+    ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
+    outs = []
+    for _ in range(4):
+        Y = torch.full((wl.B, wl.m, wl.N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        bd.gemm(dX, dW, dbits, dalpha, out=Y, workspace=ws)
+        outs.append(Y)
+    assert bd.last_device_status()[0] == 0
+    ref = outs[0].view(torch.int16)
+    assert not torch.isnan(outs[0]).any()
+    for Y in outs[1:]:
+        assert torch.equal(Y.view(torch.int16), ref)
+
+
+def test_host_entry_point_matches_device_entry_point():
+    wl = synth.Workload("t", B=3, m=2, K=512, N=384, seed=12)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Ydev = run_gemm(X, W, bits, alpha)
+    hX = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hW = torch.from_numpy(W.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hbits = torch.from_numpy(bits.view(np.int32)).pin_memory()
+    halpha = torch.from_numpy(alpha).pin_memory()
+    hY = torch.empty((wl.B, wl.m, wl.N), dtype=torch.bfloat16).pin_memory()
+    arena = torch.empty(bd.gemm_host_arena_bytes(wl.B, wl.m, wl.N, wl.K), dtype=torch.uint8, device="cuda")
+    bd.gemm_host(hX, hW, hbits, halpha, hY, arena)
+    got = synth.bf16_bits_to_f32(hY.view(torch.int16).numpy().view(np.uint16)).astype(np.float64)
+    assert np.array_equal(got, Ydev)
