@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the BitDelta fused GEMM on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all] [--impl reference]
+
+A step is one bitdelta_gemm call (the whole hot path: TMA staging, sign decode,
+both contractions, fused epilogue) on one seeded synthetic batch.  The K timed
+steps are captured in one CUDA graph and cycle through R independent buffer
+sets whose total size exceeds twice the L2, so every launch reads its weights
+from HBM.  Prints one JSON line (rank 0).
+
+--impl reference times the fp64 CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_36800_b200 import synth  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+PAPER_CONTEXT = "paper: 3.34x (standard) / 2.51x (batched) over autotuned Triton 3.6.0 on B200, FP16; no absolute figure"
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernel from the
+# ncu captures summarised under profiles/ ; None where no capture exists yet.
+NCU_TRAFFIC_BYTES = {
+    "decode_attn": None,
+    "decode_mlp_up": None,
+    "prefill": None,
+    "many_tenant_down": None,
+    "tiny": None,
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# --------------------------------------------------------------------------- ours
+def device_sets(wl, X, W, bits, alpha, nsets):
+    import torch
+    sets = []
+    for _ in range(nsets):
+        dX = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
+        dW = torch.from_numpy(W.view(np.int16)).cuda().view(torch.bfloat16)
+        db = torch.from_numpy(bits.view(np.int32)).cuda()
+        da = torch.from_numpy(alpha).cuda()
+        dY = torch.empty((wl.B, wl.m, wl.N), dtype=torch.bfloat16, device="cuda")
+        sets.append((dX, dW, db, da, dY))
+    return sets
+
+
+def time_workload(wl, steps, warmup, dist=None, sampler=None):
+    """Returns (ms_total over `steps` launches, nsets).  Device-timed with CUDA events."""
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    X, W, bits, alpha = synth.make_inputs(wl)
+    nsets = max(2, -(-2 * L2_BYTES // wl.bytes))
+    sets = device_sets(wl, X, W, bits, alpha, nsets)
+    ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, 3)):
+            s = sets[i % nsets]
+            bd.gemm(s[0], s[1], s[2], s[3], out=s[4], workspace=ws)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(steps):
+                s = sets[i % nsets]
+                bd.gemm(s[0], s[1], s[2], s[3], out=s[4], workspace=ws)
+        graph.replay()          # untimed replay: graph upload, clocks up
+        stream.synchronize()
+        st, site = bd.last_device_status()
+        if st != 0:
+            raise RuntimeError(f"device status {st} at site {site}")
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler is not None:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+    return ms, nsets, (X, W, bits, alpha), sets
+
+
+def time_e2e(wl, host_inputs, steps):
+    """Same metric through the host-buffer C-ABI entry point: H2D of every input and D2H of Y
+    inside the timed region, every step."""
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    X, W, bits, alpha = host_inputs
+    hX = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hW = torch.from_numpy(W.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hb = torch.from_numpy(bits.view(np.int32)).pin_memory()
+    ha = torch.from_numpy(alpha).pin_memory()
+    hY = torch.empty((wl.B, wl.m, wl.N), dtype=torch.bfloat16).pin_memory()
+    arena = torch.empty(bd.gemm_host_arena_bytes(wl.B, wl.m, wl.N, wl.K), dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        bd.gemm_host(hX, hW, hb, ha, hY, arena)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        bd.gemm_host(hX, hW, hb, ha, hY, arena)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    h2d = X.nbytes + W.nbytes + bits.nbytes + alpha.nbytes
+    d2h = wl.B * wl.m * wl.N * 2
+    return ms, h2d, d2h
+
+
+def cpu_baseline(wl, host_inputs, budget_s=15.0):
+    """The fp64 oracle, as it stands, on the host cores over a bounded sample of the workload."""
+    import oracle
+    X, W, bits, alpha = host_inputs
+    cores = oracle.num_threads()
+    total = wl.B * wl.m * wl.N
+    rng = np.random.default_rng(123)
+
+    def sample(count):
+        idx = np.stack([rng.integers(0, wl.B, count), rng.integers(0, wl.m, count),
+                        rng.integers(0, wl.N, count)], axis=1).astype(np.int32)
+        t0 = time.perf_counter()
+        oracle.gemm_at(X, W, bits, alpha, idx)
+        return time.perf_counter() - t0
+
+    probe = min(total, 2048)
+    rate = probe / max(sample(probe), 1e-9)          # outputs per second
+    count = int(min(total, max(probe, rate * budget_s)))
+    dt = sample(count)
+    frac = count / total
+    return {
+        "value": wl.bytes * frac / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+        "sample": f"{count} of {total} outputs (b,t,n) drawn uniformly, each a full length-{wl.K} fp64 dot pair; "
+                  f"{dt:.2f} s wall",
+        "tflops": wl.flops * frac / dt / 1e12,
+    }
+
+
+def summarize(wl, ms_total, steps, n_gpus, peaks):
+    sec = ms_total / 1e3 / steps
+    gbs = wl.bytes * n_gpus / sec / 1e9
+    tfl = wl.flops * n_gpus / sec / 1e12
+    hbm_bound = wl.m <= 16
+    per_gpu_gbs, per_gpu_tfl = gbs / n_gpus, tfl / n_gpus
+    if hbm_bound:
+        roof = {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": per_gpu_gbs / peaks["hbm_gbs"]}
+    else:
+        roof = {"bound": "tensor", "achieved": per_gpu_tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": per_gpu_tfl / peaks["bf16_tflops"],
+                "frac_of_sustained": per_gpu_tfl / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])}
+    roof["peak_source"] = peaks["_source"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
+    roof["algorithmic_bytes"] = wl.bytes
+    roof["algorithmic_flops"] = wl.flops
+    roof["kernel"] = "bitdelta_gemm_tc_kernel"
+    roof["us_per_launch"] = sec * 1e6
+    return gbs, tfl, roof
+
+
+def run_ours(args):
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+    bd.load_library()
+    peaks = load_peaks()
+    wl = synth.WORKLOADS_BY_NAME[args.workload]
+
+    sampler = ClockSampler(physical_gpu_index(local_rank)) if rank == 0 else None
+    launches0 = bd.kernel_launch_count()
+    ms, nsets, host_inputs, _sets = time_workload(wl, args.steps, args.warmup, dist, sampler)
+    clocks = sampler.stop() if sampler is not None else None
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    del _sets
+    torch.cuda.empty_cache()
+    gbs, tfl, roof = summarize(wl, ms, args.steps, world, peaks)
+
+    out = None
+    if rank == 0:
+        e2e_steps = max(3, min(args.steps, 20))
+        e_ms, h2d, d2h = time_e2e(wl, host_inputs, e2e_steps)
+        hbm_bound = wl.m <= 16
+        e_val = (wl.bytes if hbm_bound else wl.flops / 1e3) * world / (e_ms / 1e3) / 1e9
+        out = {
+            "metric": "bitdelta_gemm effective HBM GB/s" if hbm_bound else "bitdelta_gemm TFLOP/s",
+            "value": gbs if hbm_bound else tfl,
+            "unit": "GB/s" if hbm_bound else "TFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "m": wl.m, "K": wl.K, "N": wl.N,
+                       "parallelism": "replicas only (no data-path collective)" if world > 1 else "single GPU",
+                       "l2": f"cold: steps cycle through {nsets} buffer sets ({nsets * wl.bytes / 2**20:.0f} MiB > 2x L2)",
+                       "launch": "all timed steps in one CUDA graph"},
+            "tflops": tfl, "gbs": gbs,
+            "roofline": roof,
+            "e2e": {"value": e_val, "unit": "GB/s" if hbm_bound else "TFLOP/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": e2e_steps,
+                    "call": "bitdelta_gemm_host (pinned host buffers, stream synchronised each step)"},
+            "gpu_launches": args.steps,
+            "library_launches_issued": bd.kernel_launch_count() - launches0,
+            "clocks": clocks,
+            "context": PAPER_CONTEXT,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(wl, host_inputs)
+        if args.all:
+            others = {}
+            for w2 in synth.WORKLOADS:
+                if w2.name == wl.name:
+                    continue
+                steps2 = max(20, min(args.steps, int(0.25 / max(w2.bytes / 6.5e12, w2.flops / 1.6e15))))
+                ms2, nsets2, _, s2 = time_workload(w2, steps2, 3)
+                del s2
+                torch.cuda.empty_cache()
+                g2, t2, r2 = summarize(w2, ms2, steps2, 1, peaks)
+                others[w2.name] = {"us_per_launch": ms2 * 1e3 / steps2, "gbs": g2, "tflops": t2, "steps": steps2,
+                                   "buffer_sets": nsets2, "roofline": r2}
+            out["workloads"] = others
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out), flush=True)
+
+
+# ---------------------------------------------------------------------- reference arm
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    wl = synth.WORKLOADS_BY_NAME[args.workload]
+    X, W, bits, alpha = synth.make_inputs(wl)
+    total = wl.B * wl.m * wl.N
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rng = np.random.default_rng(123)
+    nsteps = args.steps + args.warmup
+    probe = min(total, 1024)
+    idx = np.stack([rng.integers(0, wl.B, probe), rng.integers(0, wl.m, probe), rng.integers(0, wl.N, probe)],
+                   axis=1).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.gemm_at(X, W, bits, alpha, idx)
+    rate = probe / max(time.perf_counter() - t0, 1e-9)
+    count = int(max(64, min(total, rate * 90.0 / nsteps)))      # whole run ~90 s
+    idx = np.stack([rng.integers(0, wl.B, count), rng.integers(0, wl.m, count), rng.integers(0, wl.N, count)],
+                   axis=1).astype(np.int32)
+    for _ in range(args.warmup):
+        oracle.gemm_at(X, W, bits, alpha, idx)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.gemm_at(X, W, bits, alpha, idx)
+    dt = (time.perf_counter() - t0) / args.steps
+    frac = count / total
+    hbm_bound = wl.m <= 16
+    val = (wl.bytes * frac / dt / 1e9) if hbm_bound else (wl.flops * frac / dt / 1e12)
+    unit = "GB/s" if hbm_bound else "TFLOP/s"
+    sample = f"{count} of {total} outputs per step, each a full length-{wl.K} fp64 dot pair"
+    out = {
+        "impl": "reference",
+        "metric": "bitdelta_gemm effective HBM GB/s" if hbm_bound else "bitdelta_gemm TFLOP/s",
+        "value": val, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "m": wl.m, "K": wl.K, "N": wl.N},
+        "cpu_baseline": {"value": val, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="decode_attn", choices=sorted(synth.WORKLOADS_BY_NAME))
+    ap.add_argument("--all", action="store_true", help="also time the other workloads (N=1 only)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

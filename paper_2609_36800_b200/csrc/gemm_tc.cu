@@ -24,13 +24,21 @@
 
 namespace bd {
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every spin gives up after 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;   // every spin gives up after 4e9 SM cycles (~2 s)
 constexpr int kThreads = 512;
 constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
 constexpr int kWarpTmem = 2;
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
+
+#ifdef BD_TRACE
+// Debug builds only: per-CTA cycle stamps of the main phases.
+__device__ long long* g_trace_ptr;
+#define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 16 + (idx)] = clock64(); } while (0)
+#else
+#define BD_STAMP(idx) do { } while (0)
+#endif
 
 __device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] site of the first failure
 
@@ -52,16 +60,18 @@ static_assert(sizeof(Ctl) <= kSmemCtrlBytes, "control block too large");
 // Bounded wait on an mbarrier phase.  Returns false if the wait was abandoned
 // (limit reached here or in another thread of the CTA).
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-    }
-    const uint64_t t0 = global_timer_ns();
+    if (mbar_try_wait(bar, parity)) return true;
+    // Slow path: poll, and every 64 polls look at the abort flag and the SM cycle counter
+    // (cheap to read; the limit is ~2 s at 2 GHz, longer at lower clocks).
+    const long long t0 = clock64();
 #pragma unroll 1
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+        }
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (clock64() - t0 > kWaitLimitCycles) {
             *abort_flag = 1;
             if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
             return false;
@@ -147,6 +157,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (warp == 0) BD_STAMP(0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -178,6 +189,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    if (warp == 0) BD_STAMP(1);
 
     const long long lo = (long long)blockIdx.x * a.T / gridDim.x;
     const long long hi = (long long)(blockIdx.x + 1) * a.T / gridDim.x;
@@ -186,23 +198,27 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
     if (warp == kWarpProducer) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0, bslot = 0;
-            uint32_t phase = 0, bphase = 0;
-            bool ok = true;
-            while (ok && it.next(unit, p0, p1)) {
-                const Unit u = unit_info(a, unit);
-                for (int p = p0; p < p1 && ok; ++p) {
-                    if (p == p0 || !(p & 1)) {
-                        ok = wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1);
-                        if (!ok) break;
+        // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
+        int stage = 0, bslot = 0;
+        uint32_t phase = 0, bphase = 0;
+        bool ok = true;
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            for (int p = p0; p < p1 && ok; ++p) {
+                if (p == p0 || !(p & 1)) {
+                    ok = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
+                    if (!ok) break;
+                    if (elect_one()) {
                         const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
                         mbar_arrive_expect_tx(bar, a.bslot_bytes);
                         tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
-                        if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
                     }
-                    ok = wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2);
-                    if (!ok) break;
+                    __syncwarp();
+                    if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                }
+                ok = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
+                if (!ok) break;
+                if (elect_one()) {
                     const uint32_t bar = smem_u32(&ctl->full[stage]);
                     const uint32_t dst = stages_addr + stage * a.stage_bytes;
                     mbar_arrive_expect_tx(bar, a.stage_bytes);
@@ -211,68 +227,83 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
                     tma_load_2d(dst + 2 * a.w_atom_bytes, &tmX, bar, k0, u.xrow0);
                     tma_load_2d(dst + 2 * a.w_atom_bytes + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
-                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
                 }
+                __syncwarp();
+                if (p == p0 && unit == (int)(lo / a.P)) BD_STAMP(2);
+                if (++stage == a.stages) { stage = 0; phase ^= 1; }
             }
         }
+        BD_STAMP(3);
     } else if (warp == kWarpMma) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
-            const uint32_t idesc_delta = make_idesc_bf16(kTileN, (uint32_t)a.Nd);
-            const uint64_t desc_hi = make_smem_desc_sw128(0) & 0xFFFFFFFF00000000ull;
-            const uint32_t desc_lo_fixed = (uint32_t)(make_smem_desc_sw128(0) & 0xFFFF0000ull);
-            auto desc = [&](uint32_t addr) -> uint64_t {
-                return desc_hi | (uint64_t)(desc_lo_fixed | ((addr >> 4) & 0x3FFFu));
-            };
-            const uint32_t amask = (uint32_t)a.a_slots - 1;
-            const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
-            int stage = 0;
-            uint32_t phase = 0, accphase = 0, item = 0;
-            bool ok = true;
-            while (ok && it.next(unit, p0, p1)) {
-                const Unit u = unit_info(a, unit);
-                ok = wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3);
+        // Warp-uniform loop, one elected lane issues: descriptors and predicates then live in
+        // uniform registers, which keeps the issue cost of a tcgen05.mma at its hardware floor.
+        const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+        const uint32_t idesc_delta = make_idesc_bf16(kTileN, (uint32_t)a.Nd);
+        const uint64_t desc_hi = make_smem_desc_sw128(0) & 0xFFFFFFFF00000000ull;
+        const uint32_t desc_lo_fixed = (uint32_t)(make_smem_desc_sw128(0) & 0xFFFF0000ull);
+        auto desc = [&](uint32_t addr) -> uint64_t {
+            return desc_hi | (uint64_t)(desc_lo_fixed | ((addr >> 4) & 0x3FFFu));
+        };
+        const uint32_t amask = (uint32_t)a.a_slots - 1;
+        const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+        int stage = 0;
+        uint32_t phase = 0, accphase = 0, item = 0;
+        bool ok = true;
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            if (!ok) break;
+            tc_fence_after();
+            for (int p = p0; p < p1 && ok; ++p) {
+                ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                 if (!ok) break;
                 tc_fence_after();
-                for (int p = p0; p < p1 && ok; ++p) {
-                    ok = wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t wbase = stages_addr + stage * a.stage_bytes;
-                    const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
+                if (item == 0) BD_STAMP(4);
+                const uint32_t wbase = stages_addr + stage * a.stage_bytes;
+                const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
+                const uint32_t first = (p > p0) ? 1u : 0u;
+                if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t atom = kk >> 2, k16 = kk & 3;
                         umma_ss(tmem_base, desc(wbase + atom * a.w_atom_bytes + k16 * 32),
                                 desc(xbase + atom * a.x_atom_bytes + k16 * 32), idesc_base,
-                                (p > p0 || kk > 0) ? 1u : 0u);
+                                (kk > 0) ? 1u : first);
                     }
-                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
-                        const uint32_t slot = item & amask;
-                        const uint32_t use = item >> ashift;
-                        ok = wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
-                        const uint32_t a_tmem = tmem_base + a.col_a + slot * kASlotCols;
-                        const uint32_t xwin = xbase + (uint32_t)(j * a.win_rows) * 128u;
+                }
+                __syncwarp();
+                for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                    const uint32_t slot = item & amask;
+                    const uint32_t use = item >> ashift;
+                    ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (item == 0) BD_STAMP(5);
+                    const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                    const uint32_t a_tmem = tmem_base + a.col_a + slot * kASlotCols;
+                    const uint32_t xwin = xbase + (uint32_t)(j * a.win_rows) * 128u;
+                    if (elect_one()) {
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t atom = kk >> 2, k16 = kk & 3;
                             umma_ts(d_tmem, a_tmem + kk * 8, desc(xwin + atom * a.x_atom_bytes + k16 * 32),
-                                    idesc_delta, (p > p0 || kk > 0) ? 1u : 0u);
+                                    idesc_delta, (kk > 0) ? 1u : first);
                         }
                         tc_commit(smem_u32(&ctl->aempty[slot]));
                     }
-                    if (!ok) break;
-                    tc_commit(smem_u32(&ctl->empty[stage]));
-                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                    __syncwarp();
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&ctl->accfull));
-                accphase ^= 1;
+                if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
+                __syncwarp();
+                if (++stage == a.stages) { stage = 0; phase ^= 1; }
             }
+            if (!ok) break;
+            if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
+            __syncwarp();
+            accphase ^= 1;
+            BD_STAMP(6);
         }
     } else if (warp >= kWarpDecode0 && warp < kWarpEpi0) {
         // ------------------------------------------- sign decode -> tensor memory
@@ -291,6 +322,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (p == p0 || !(p & 1)) {
                     ok = wait_bar(smem_u32(&ctl->bfull[bslot]), bphase, abort_flag, 6);
                     if (!ok) break;
+                    if (item == 0 && warp == kWarpDecode0) BD_STAMP(14);
                 }
                 const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
                 for (int j = 0; j < u.nten && ok; ++j, ++item) {
@@ -313,6 +345,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                    if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                 }
                 if (!ok) break;
                 if ((p & 1) || p == p1 - 1) {
@@ -345,6 +378,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
+            if (warp == kWarpEpi0) BD_STAMP(7);
             const int nchunks = a.decode ? u.nten : (u.ntok + 15) / 16;
             for (int i = 0; i < nchunks; ++i) {
                 uint32_t rb[16], rd[16];
@@ -369,6 +403,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
+            if (warp == kWarpEpi0) BD_STAMP(8);
 
             if (!whole) {
                 // This tile is cut across CTAs: publish the partial, count arrivals, and let
@@ -383,32 +418,39 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
                 epi_bar_sync();
+                if (warp == kWarpEpi0) BD_STAMP(9);
                 if (ctl->is_last) {
                     __threadfence();
+                    // CTA c0 holds the tile's first item; the tile is its first segment only if its
+                    // range starts exactly there.  Every later CTA starts inside the tile.
+                    const int slot0 = ((long long)c0 * a.T / gridDim.x == first_item) ? 2 * c0 : 2 * c0 + 1;
+                    const float* p0s = a.partials + (size_t)slot0 * a.slot_floats + row;
+                    const float* prest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats + row;
+                    const size_t cstride = 2 * (size_t)a.slot_floats;
                     for (int tk = 0; tk < u.ntok; ++tk) {
-                        float sum = 0.f;
-                        for (int c = c0; c <= c1; ++c) {
-                            const int cfirst = (int)(((long long)c * a.T / gridDim.x) / a.P);
-                            const int slot = (unit == cfirst) ? 2 * c : 2 * c + 1;
-                            sum += __ldcg(a.partials + (size_t)slot * a.slot_floats + (size_t)tk * kTileN + row);
+                        float sum = __ldcg(p0s + (size_t)tk * kTileN);
+                        for (int c = 0; c < c1 - c0; ++c) {
+                            sum += __ldcg(prest + c * cstride + (size_t)tk * kTileN);
                         }
                         if (n < a.N) Y[(size_t)(u.xrow0 + tk) * a.N + n] = __float2bfloat16_rn(sum);
                     }
                     if (etid == 0) a.counters[unit] = 0u;
                 }
                 epi_bar_sync();   // is_last is rewritten by the next cut tile
+                if (warp == kWarpEpi0) BD_STAMP(10);
             }
         }
     }
 
     // ------------------------------------------------------------------ teardown
     __syncthreads();
+    if (warp == 0) BD_STAMP(11);
     if (*abort_flag) {
         // A wait was abandoned: give copies and MMAs still in flight a bounded time to land
         // before shared and tensor memory are released.
         if (threadIdx.x == 0) {
-            const uint64_t t0 = global_timer_ns();
-            while (global_timer_ns() - t0 < 2000000ull) {
+            const long long t0 = clock64();
+            while (clock64() - t0 < 4000000ll) {
             }
         }
         __syncthreads();
@@ -416,8 +458,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     tc_fence_after();
     if (warp == kWarpTmem) {
         tmem_dealloc(tmem_base, kTmemCols);
+        BD_STAMP(12);
     }
 }
+
+#ifdef BD_TRACE
+extern "C" int bitdelta_debug_set_trace(long long* buf) {
+    return (int)cudaMemcpyToSymbol(g_trace_ptr, &buf, sizeof(buf));
+}
+#endif
 
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmBits,
                            const GemmArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
