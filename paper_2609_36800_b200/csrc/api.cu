@@ -103,6 +103,19 @@ bool encode_bf16_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D bytes [rows, K] row-major (e5m2 activation pieces), box = 128 bytes (swizzled) x box_rows.
+bool encode_u8_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 3-D uint32 [B, N, K/32], box = 8 words (32 bytes) x 128 rows x tenants.
 bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, uint64_t words, uint32_t tenants) {
     EncodeTiledFn fn = encode_fn();
@@ -200,14 +213,26 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
     if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
 
-    CUtensorMap tmW, tmX, tmBits;
+    CUtensorMap tmW, tmX, tmX8, tmBits;
     if (!encode_bf16_2d(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
     if (!encode_bf16_2d(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
     if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB))
         return BITDELTA_ERR_CUDA;
+    if (p.decode) {
+        // Decode schedule: split the activations into e5m2 pieces first (tiny), then the GEMM, which
+        // may start prefetching weights while the split is still running.
+        uint8_t* x8 = bd::ws_x8(p, workspace);
+        if (!encode_u8_2d(&tmX8, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, (uint32_t)p.x8_rows))
+            return BITDELTA_ERR_CUDA;
+        if (bd::launch_x_split(X, x8, B, m, K, stream) != cudaSuccess)
+            return BITDELTA_ERR_CUDA;
+        g_launches++;
+    } else {
+        tmX8 = tmX;   // not read by the tiled schedule
+    }
 
     bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
-    if (bd::launch_gemm_tc(tmW, tmX, tmBits, args, p.grid, p.smem_bytes, stream) != cudaSuccess)
+    if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, p.decode != 0, stream) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
     g_launches++;
     return BITDELTA_OK;

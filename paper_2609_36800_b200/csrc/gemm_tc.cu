@@ -35,9 +35,17 @@ constexpr int kWarpEpi0 = 12;      // warps 12..15
 #ifdef BD_TRACE
 // Debug builds only: per-CTA cycle stamps of the main phases.
 __device__ long long* g_trace_ptr;
-#define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 16 + (idx)] = clock64(); } while (0)
+#define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = clock64(); } while (0)
+#define BD_ACC_DECL(name) long long name = 0
+#define BD_ACC_BEGIN(t) const long long t = clock64()
+#define BD_ACC_END(name, t) name += clock64() - t
+#define BD_ACC_STORE(idx, name) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = name; } while (0)
 #else
 #define BD_STAMP(idx) do { } while (0)
+#define BD_ACC_DECL(name) do { } while (0)
+#define BD_ACC_BEGIN(t) do { } while (0)
+#define BD_ACC_END(name, t) do { } while (0)
+#define BD_ACC_STORE(idx, name) do { } while (0)
 #endif
 
 __device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] site of the first failure
@@ -140,11 +148,143 @@ __device__ __forceinline__ void decode_word(uint32_t w, uint32_t* r) {
     }
 }
 
+// ------------------------------------------------------------------- epilogue helpers
+template <int W>
+__device__ __forceinline__ void tmem_ld_w(uint32_t taddr, uint32_t* r) {
+    if constexpr (W == 1) tmem_ld1(taddr, r);
+    else if constexpr (W == 2) tmem_ld2(taddr, r);
+    else if constexpr (W == 4) tmem_ld4(taddr, r);
+    else if constexpr (W == 8) tmem_ld8(taddr, r);
+    else tmem_ld16(taddr, r);
+}
+
+struct EpiOut {
+    __nv_bfloat16* Y;   // output matrix [B*m, N]
+    float* slot;        // partial-result slot, or nullptr when this CTA owns the whole tile
+    int N, n, row, xrow0;
+    __device__ __forceinline__ void put(int tok, float v) const {
+        if (slot) slot[(size_t)tok * kTileN + row] = v;
+        else if (n < N) Y[(size_t)(xrow0 + tok) * N + n] = __float2bfloat16_rn(v);
+    }
+};
+
+// Decode schedule, M tokens per tenant: the base accumulator holds tenant j's tokens in columns
+// j*M .. j*M+M-1; its delta accumulator starts at column N3*j and holds, for piece q of the
+// activation split, token t in column q*M + t.  delta = D0 + D1 + D2 + D3.
+template <int M>
+__device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
+                                                const EpiOut& out) {
+    constexpr int N3 = (kPieces * M + 15) / 16 * 16;
+    constexpr int TPB = (N3 == 16) ? 2 : 1;   // tenants drained per wait
+    for (int j0 = 0; j0 < u.nten; j0 += TPB) {
+        uint32_t rb[16], rd[TPB * N3];
+        tmem_ld16(lane_taddr + (uint32_t)(j0 * M), rb);
+#pragma unroll
+        for (int jj = 0; jj < TPB; ++jj) {
+#pragma unroll
+            for (int c = 0; c < N3; c += 16)
+                tmem_ld16(lane_taddr + a.col_delta + (uint32_t)((j0 + jj) * N3 + c), rd + jj * N3 + c);
+        }
+        tc_wait_ld();
+#pragma unroll
+        for (int jj = 0; jj < TPB; ++jj) {
+            if (j0 + jj < u.nten) {
+                const float al = __ldg(a.alpha + u.tenant0 + j0 + jj);
+#pragma unroll
+                for (int t = 0; t < M; ++t) {
+                    const float lo = __uint_as_float(rd[jj * N3 + 2 * M + t]) + __uint_as_float(rd[jj * N3 + 3 * M + t]);
+                    const float hi = __uint_as_float(rd[jj * N3 + t]) + __uint_as_float(rd[jj * N3 + M + t]);
+                    out.put((j0 + jj) * M + t, fmaf(al, hi + lo, __uint_as_float(rb[jj * M + t])));
+                }
+            }
+        }
+    }
+}
+
+// Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
+__device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
+                                               const EpiOut& out) {
+    const float al = __ldg(a.alpha + u.tenant0);
+    for (int t0 = 0; t0 < u.ntok; t0 += 32) {
+        uint32_t rb[32], rd[32];
+        tmem_ld32(lane_taddr + (uint32_t)t0, rb);
+        tmem_ld32(lane_taddr + a.col_delta + (uint32_t)t0, rd);
+        tc_wait_ld();
+        const int nvalid = min(32, u.ntok - t0);
+#pragma unroll
+        for (int t = 0; t < 32; ++t) {
+            if (t < nvalid) out.put(t0 + t, fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t])));
+        }
+    }
+}
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+
+// Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
+// 128 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+4, ...
+__device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, const float* first,
+                                                const float* rest, size_t cstride, int nrest) {
+    __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
+    const int r4 = (etid & 31) * 4;
+    const int n = u.n0 + r4;
+    const bool vec_ok = ((a.N & 3) == 0) && (n + 3 < a.N);
+    for (int tk = etid >> 5; tk < u.ntok; tk += 16) {
+        float4 acc[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = tk + 4 * q;
+            acc[q] = (t < u.ntok) ? ldcg4(first + (size_t)t * kTileN + r4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int c = 0; c < nrest; ++c) {
+            const float* pc = rest + (size_t)c * cstride;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int t = tk + 4 * q;
+                if (t < u.ntok) {
+                    const float4 v = ldcg4(pc + (size_t)t * kTileN + r4);
+                    acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = tk + 4 * q;
+            if (t < u.ntok) {
+                __nv_bfloat16* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
+                if (vec_ok) {
+                    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc[q].x, acc[q].y);
+                    __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc[q].z, acc[q].w);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+                    pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+                    *reinterpret_cast<uint2*>(dst) = pk;
+                } else {
+                    if (n + 0 < a.N) dst[0] = __float2bfloat16_rn(acc[q].x);
+                    if (n + 1 < a.N) dst[1] = __float2bfloat16_rn(acc[q].y);
+                    if (n + 2 < a.N) dst[2] = __float2bfloat16_rn(acc[q].z);
+                    if (n + 3 < a.N) dst[3] = __float2bfloat16_rn(acc[q].w);
+                }
+            }
+        }
+    }
+}
+
+// 32 packed sign bits -> 8 registers of four e5m2 each (+1 = 0x3C, -1 = 0xBC).  Register c takes
+// bits c, c+8, c+16, c+24 (its bytes 0..3): one shift lands all four on the byte sign positions, one
+// three-input logic op masks them and flips the sign of a packed (-1,-1,-1,-1).  The k order inside
+// the group of 32 is therefore permuted (slot 4c+i holds k = c + 8i); the activation pieces are
+// stored with the same permutation, so the contraction is unchanged.
+__device__ __forceinline__ void decode_word_e5m2(uint32_t w, uint32_t* r) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) r[c] = ((w << (7 - c)) & 0x80808080u) ^ 0xBCBCBCBCu;
+}
+
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                        const __grid_constant__ CUtensorMap tmBits, const GemmArgs a) {
+                        const __grid_constant__ CUtensorMap tmX8, const __grid_constant__ CUtensorMap tmBits,
+                        const GemmArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -158,6 +298,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     if (warp == 0) BD_STAMP(0);
+    if (threadIdx.x == 32) {
+        prefetch_tensormap(&tmW);
+        prefetch_tensormap(&tmX);
+        prefetch_tensormap(&tmBits);
+        if (a.decode) prefetch_tensormap(&tmX8);
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -169,7 +315,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             mbar_init(smem_u32(&ctl->bempty[s]), 8);
         }
         for (int s = 0; s < kMaxASlots; ++s) {
-            mbar_init(smem_u32(&ctl->afull[s]), 4);
+            mbar_init(smem_u32(&ctl->afull[s]), a.decode ? 8 : 4);
             mbar_init(smem_u32(&ctl->aempty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->accfull), 1);
@@ -177,9 +323,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
-        prefetch_tensormap(&tmW);
-        prefetch_tensormap(&tmX);
-        prefetch_tensormap(&tmBits);
     }
     if (warp == kWarpTmem) {
         tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -202,11 +345,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0, bslot = 0;
         uint32_t phase = 0, bphase = 0;
         bool ok = true;
+        BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty);
+        bool dep_waited = false;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             for (int p = p0; p < p1 && ok; ++p) {
                 if (p == p0 || !(p & 1)) {
+                    BD_ACC_BEGIN(tb);
                     ok = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
+                    BD_ACC_END(w_bempty, tb);
                     if (!ok) break;
                     if (elect_one()) {
                         const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
@@ -216,7 +363,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     __syncwarp();
                     if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
                 }
+                BD_ACC_BEGIN(te);
                 ok = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
+                BD_ACC_END(w_empty, te);
                 if (!ok) break;
                 if (elect_one()) {
                     const uint32_t bar = smem_u32(&ctl->full[stage]);
@@ -227,72 +376,125 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
                     tma_load_2d(dst + 2 * a.w_atom_bytes, &tmX, bar, k0, u.xrow0);
                     tma_load_2d(dst + 2 * a.w_atom_bytes + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
+                    if (a.decode) {
+                        // The e5m2 pieces are written by the activation-split kernel queued before this one.
+                        if (!dep_waited) { grid_dependency_wait(); }
+                        tma_load_2d(dst + 2 * a.w_atom_bytes + 2 * a.x_atom_bytes, &tmX8, bar, k0,
+                                    u.tenant0 * kPieces * a.m);
+                    }
                 }
+                dep_waited = true;
                 __syncwarp();
                 if (p == p0 && unit == (int)(lo / a.P)) BD_STAMP(2);
                 if (++stage == a.stages) { stage = 0; phase ^= 1; }
             }
         }
         BD_STAMP(3);
+        BD_ACC_STORE(19, w_empty); BD_ACC_STORE(20, w_bempty);
     } else if (warp == kWarpMma) {
         // -------------------------------------------------------------- MMA issuer
         // Warp-uniform loop, one elected lane issues: descriptors and predicates then live in
         // uniform registers, which keeps the issue cost of a tcgen05.mma at its hardware floor.
+        // Operand buffers in tensor memory are handed over as `items`:
+        //   tiled schedule : one item = one tenant x 128 k of bf16 signs (64 columns, 8 MMAs of K=16)
+        //   decode schedule: one item = all tenants of the unit x 64 k of e5m2 signs (16 columns per
+        //                    tenant, 2 MMAs of K=32 per tenant)
         const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
-        const uint32_t idesc_delta = make_idesc_bf16(kTileN, (uint32_t)a.Nd);
-        const uint64_t desc_hi = make_smem_desc_sw128(0) & 0xFFFFFFFF00000000ull;
-        const uint32_t desc_lo_fixed = (uint32_t)(make_smem_desc_sw128(0) & 0xFFFF0000ull);
-        auto desc = [&](uint32_t addr) -> uint64_t {
-            return desc_hi | (uint64_t)(desc_lo_fixed | ((addr >> 4) & 0x3FFFu));
-        };
+        const uint32_t idesc_delta = a.decode ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
+                                              : make_idesc_bf16(kTileN, (uint32_t)a.Nd);
+        // Descriptor of a tile = descriptor of address 0 plus (address >> 4): addresses stay below
+        // 256 KiB, so the sum never carries out of the 14-bit start-address field.
+        const uint64_t desc0 = make_smem_desc_sw128(0);
+        const uint32_t w_atom16 = a.w_atom_bytes >> 4, x_atom16 = a.x_atom_bytes >> 4;
         const uint32_t amask = (uint32_t)a.a_slots - 1;
         const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
         int stage = 0;
         uint32_t phase = 0, accphase = 0, item = 0;
         bool ok = true;
+        BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id);
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
+            BD_ACC_BEGIN(ta);
             ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            BD_ACC_END(w_acc, ta);
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
+                BD_ACC_BEGIN(tf);
                 ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                BD_ACC_END(w_full, tf);
                 if (!ok) break;
                 tc_fence_after();
                 if (item == 0) BD_STAMP(4);
                 const uint32_t wbase = stages_addr + stage * a.stage_bytes;
                 const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
-                const uint32_t first = (p > p0) ? 1u : 0u;
+                const uint64_t wdesc = desc0 + (wbase >> 4);
+                const uint64_t xdesc = desc0 + (xbase >> 4);
+                const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
+                BD_ACC_BEGIN(tib);
                 if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t atom = kk >> 2, k16 = kk & 3;
-                        umma_ss(tmem_base, desc(wbase + atom * a.w_atom_bytes + k16 * 32),
-                                desc(xbase + atom * a.x_atom_bytes + k16 * 32), idesc_base,
-                                (kk > 0) ? 1u : first);
+                        umma_ss(tmem_base, wdesc + (atom * w_atom16 + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
+                                idesc_base, (kk > 0) ? 1u : first);
                     }
                 }
                 __syncwarp();
-                for (int j = 0; j < u.nten && ok; ++j, ++item) {
-                    const uint32_t slot = item & amask;
-                    const uint32_t use = item >> ashift;
-                    ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (item == 0) BD_STAMP(5);
-                    const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
-                    const uint32_t a_tmem = tmem_base + a.col_a + slot * kASlotCols;
-                    const uint32_t xwin = xbase + (uint32_t)(j * a.win_rows) * 128u;
-                    if (elect_one()) {
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t atom = kk >> 2, k16 = kk & 3;
-                            umma_ts(d_tmem, a_tmem + kk * 8, desc(xwin + atom * a.x_atom_bytes + k16 * 32),
-                                    idesc_delta, (kk > 0) ? 1u : first);
+                BD_ACC_END(w_ib, tib);
+                if (a.decode) {
+                    const uint64_t x8desc = xdesc + 2 * x_atom16;
+                    const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
+                    for (int half = 0; half < 2 && ok; ++half, ++item) {
+                        const uint32_t slot = item & amask;
+                        const uint32_t use = item >> ashift;
+                        BD_ACC_BEGIN(tg);
+                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        BD_ACC_END(w_afull, tg);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (item == 0) BD_STAMP(5);
+                        BD_ACC_BEGIN(tid);
+                        const uint32_t a_buf = tmem_base + a.col_a + slot * (uint32_t)a.aslot_cols;
+                        const uint32_t acc = (half > 0) ? 1u : first;
+                        if (elect_one()) {
+                            for (int j = 0; j < u.nten; ++j) {
+                                const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                                const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
+                                umma_ts_f8(d_tmem, a_buf + j * 16, xj, idesc_delta, acc);
+                                umma_ts_f8(d_tmem, a_buf + j * 16 + 8, xj + 2, idesc_delta, 1u);
+                            }
+                            tc_commit(smem_u32(&ctl->aempty[slot]));
                         }
-                        tc_commit(smem_u32(&ctl->aempty[slot]));
+                        __syncwarp();
+                        BD_ACC_END(w_id, tid);
                     }
-                    __syncwarp();
+                } else {
+                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                        const uint32_t slot = item & amask;
+                        const uint32_t use = item >> ashift;
+                        BD_ACC_BEGIN(tg);
+                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        BD_ACC_END(w_afull, tg);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (item == 0) BD_STAMP(5);
+                        BD_ACC_BEGIN(tid);
+                        const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                        const uint32_t a_tmem = tmem_base + a.col_a + slot * (uint32_t)a.aslot_cols;
+                        const uint64_t xwdesc = xdesc + (uint32_t)(j * a.win_rows) * 8u;   // 128 B per row
+                        if (elect_one()) {
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                const uint32_t atom = kk >> 2, k16 = kk & 3;
+                                umma_ts(d_tmem, a_tmem + kk * 8, xwdesc + (atom * x_atom16 + k16 * 2), idesc_delta,
+                                        (kk > 0) ? 1u : first);
+                            }
+                            tc_commit(smem_u32(&ctl->aempty[slot]));
+                        }
+                        __syncwarp();
+                        BD_ACC_END(w_id, tid);
+                    }
                 }
                 if (!ok) break;
                 if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
@@ -305,9 +507,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             BD_STAMP(6);
         }
+        BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
     } else if (warp >= kWarpDecode0 && warp < kWarpEpi0) {
         // ------------------------------------------- sign decode -> tensor memory
-        const int grp = (warp - kWarpDecode0) >> 2;
+        const int dw = warp - kWarpDecode0;    // 0..7
+        const int grp = dw >> 2;
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -316,36 +520,72 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int bslot = 0;
         uint32_t bphase = 0, item = 0;
         bool ok = true;
+        BD_ACC_DECL(w_bfull); BD_ACC_DECL(w_aempty); BD_ACC_DECL(w_work);
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             for (int p = p0; p < p1 && ok; ++p) {
                 if (p == p0 || !(p & 1)) {
+                    BD_ACC_BEGIN(tb);
                     ok = wait_bar(smem_u32(&ctl->bfull[bslot]), bphase, abort_flag, 6);
+                    BD_ACC_END(w_bfull, tb);
                     if (!ok) break;
                     if (item == 0 && warp == kWarpDecode0) BD_STAMP(14);
                 }
                 const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
-                for (int j = 0; j < u.nten && ok; ++j, ++item) {
-                    if ((int)(item & 1) != grp) continue;
-                    const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
-                    const uint32_t slot = item & amask;
-                    const uint32_t use = item >> ashift;
-                    ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t taddr = lane_taddr + a.col_a + slot * kASlotCols;
-                    uint32_t r[32];
-                    decode_word(w.x, r);
-                    decode_word(w.y, r + 16);
-                    tmem_st32(taddr, r);
-                    decode_word(w.z, r);
-                    decode_word(w.w, r + 16);
-                    tmem_st32(taddr + 32, r);
-                    tc_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
-                    if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
+                if (a.decode) {
+                    // All eight warps fill every buffer: warp (grp, quad) decodes, for its 32 rows,
+                    // the tenants j = grp, grp+2, ... (64 k = two sign words each).
+                    for (int half = 0; half < 2 && ok; ++half, ++item) {
+                        const uint32_t slot = item & amask;
+                        const uint32_t use = item >> ashift;
+                        BD_ACC_BEGIN(tq);
+                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        BD_ACC_END(w_aempty, tq);
+                        if (!ok) break;
+                        tc_fence_after();
+                        BD_ACC_BEGIN(tw);
+                        const uint32_t tbuf = lane_taddr + a.col_a + slot * (uint32_t)a.aslot_cols;
+                        for (int j = grp; j < u.nten; j += 2) {
+                            const uint2 w = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
+                            uint32_t r[16];
+                            decode_word_e5m2(w.x, r);
+                            decode_word_e5m2(w.y, r + 8);
+                            tmem_st16(tbuf + j * 16, r);
+                        }
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                        BD_ACC_END(w_work, tw);
+                        if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
+                    }
+                } else {
+                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                        if ((int)(item & 1) != grp) continue;
+                        const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
+                        const uint32_t slot = item & amask;
+                        const uint32_t use = item >> ashift;
+                        BD_ACC_BEGIN(tq);
+                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        BD_ACC_END(w_aempty, tq);
+                        if (!ok) break;
+                        tc_fence_after();
+                        BD_ACC_BEGIN(tw);
+                        const uint32_t taddr = lane_taddr + a.col_a + slot * (uint32_t)a.aslot_cols;
+                        uint32_t r[32];
+                        decode_word(w.x, r);
+                        decode_word(w.y, r + 16);
+                        tmem_st32(taddr, r);
+                        decode_word(w.z, r);
+                        decode_word(w.w, r + 16);
+                        tmem_st32(taddr + 32, r);
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                        BD_ACC_END(w_work, tw);
+                        if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
+                    }
                 }
                 if (!ok) break;
                 if ((p & 1) || p == p1 - 1) {
@@ -355,6 +595,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
             }
         }
+        if (warp == kWarpDecode0) { BD_ACC_STORE(21, w_bfull); BD_ACC_STORE(22, w_aempty); BD_ACC_STORE(23, w_work); }
+        if (warp == kWarpDecode0 + 4) { BD_ACC_STORE(24, w_bfull); BD_ACC_STORE(25, w_aempty); BD_ACC_STORE(26, w_work); }
     } else if (warp >= kWarpEpi0) {
         // ---------------------------------------------------------------- epilogue
         const int quad = warp & 3;
@@ -379,26 +621,28 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             tc_fence_after();
             accphase ^= 1;
             if (warp == kWarpEpi0) BD_STAMP(7);
-            const int nchunks = a.decode ? u.nten : (u.ntok + 15) / 16;
-            for (int i = 0; i < nchunks; ++i) {
-                uint32_t rb[16], rd[16];
-                tmem_ld16(lane_taddr + (uint32_t)(i * a.chunk_rows), rb);
-                tmem_ld16(lane_taddr + a.col_delta + (uint32_t)(i * 16), rd);
-                tc_wait_ld();
-                const float al = __ldg(a.alpha + (a.decode ? u.tenant0 + i : u.tenant0));
-                const int tok0 = i * a.chunk_rows;
-                const int nvalid = a.decode ? a.m : min(16, u.ntok - tok0);
-#pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    if (t < nvalid) {
-                        const float v = fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t]));
-                        if (whole) {
-                            if (n < a.N) Y[(size_t)(u.xrow0 + tok0 + t) * a.N + n] = __float2bfloat16_rn(v);
-                        } else {
-                            slotp[(size_t)(tok0 + t) * kTileN + row] = v;
-                        }
-                    }
+            EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
+            if (a.decode) {
+                switch (a.m) {
+                    case 1: epilogue_decode<1>(a, u, lane_taddr, out); break;
+                    case 2: epilogue_decode<2>(a, u, lane_taddr, out); break;
+                    case 3: epilogue_decode<3>(a, u, lane_taddr, out); break;
+                    case 4: epilogue_decode<4>(a, u, lane_taddr, out); break;
+                    case 5: epilogue_decode<5>(a, u, lane_taddr, out); break;
+                    case 6: epilogue_decode<6>(a, u, lane_taddr, out); break;
+                    case 7: epilogue_decode<7>(a, u, lane_taddr, out); break;
+                    case 8: epilogue_decode<8>(a, u, lane_taddr, out); break;
+                    case 9: epilogue_decode<9>(a, u, lane_taddr, out); break;
+                    case 10: epilogue_decode<10>(a, u, lane_taddr, out); break;
+                    case 11: epilogue_decode<11>(a, u, lane_taddr, out); break;
+                    case 12: epilogue_decode<12>(a, u, lane_taddr, out); break;
+                    case 13: epilogue_decode<13>(a, u, lane_taddr, out); break;
+                    case 14: epilogue_decode<14>(a, u, lane_taddr, out); break;
+                    case 15: epilogue_decode<15>(a, u, lane_taddr, out); break;
+                    default: epilogue_decode<16>(a, u, lane_taddr, out); break;
                 }
+            } else {
+                epilogue_tiled(a, u, lane_taddr, out);
             }
             tc_fence_before();
             __syncwarp();
@@ -424,16 +668,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
                     // range starts exactly there.  Every later CTA starts inside the tile.
                     const int slot0 = ((long long)c0 * a.T / gridDim.x == first_item) ? 2 * c0 : 2 * c0 + 1;
-                    const float* p0s = a.partials + (size_t)slot0 * a.slot_floats + row;
-                    const float* prest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats + row;
-                    const size_t cstride = 2 * (size_t)a.slot_floats;
-                    for (int tk = 0; tk < u.ntok; ++tk) {
-                        float sum = __ldcg(p0s + (size_t)tk * kTileN);
-                        for (int c = 0; c < c1 - c0; ++c) {
-                            sum += __ldcg(prest + c * cstride + (size_t)tk * kTileN);
-                        }
-                        if (n < a.N) Y[(size_t)(u.xrow0 + tk) * a.N + n] = __float2bfloat16_rn(sum);
-                    }
+                    reduce_partials(a, u, etid, a.partials + (size_t)slot0 * a.slot_floats,
+                                    a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats,
+                                    2 * (size_t)a.slot_floats, c1 - c0);
                     if (etid == 0) a.counters[unit] = 0u;
                 }
                 epi_bar_sync();   // is_last is rewritten by the next cut tile
@@ -468,17 +705,29 @@ extern "C" int bitdelta_debug_set_trace(long long* buf) {
 }
 #endif
 
-cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmBits,
-                           const GemmArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(bitdelta_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kSmemBudget);
+cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
+                           const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
+                           bool after_split, cudaStream_t stream) {
+    static int attr_device = -1;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (attr_device != dev) {
+        e = cudaFuncSetAttribute(bitdelta_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_device = dev;
     }
-    bitdelta_gemm_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tmW, tmX, tmBits, args);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_split ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, bitdelta_gemm_tc_kernel, tmW, tmX, tmX8, tmBits, args);
 }
 
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {

@@ -11,11 +11,11 @@ namespace bd {
 
 struct GemmArgs {
     int B, m, N, K;
-    int decode, TB, tok_tile, Nb, Nd, win_rows, chunk_rows;
+    int decode, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
     int m_tiles, groups, P;
     long long T;
     int stages, a_slots;
-    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, bslot_bytes;
+    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
     const float* alpha;
@@ -28,21 +28,35 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     GemmArgs a{};
     a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
     a.decode = p.decode; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
-    a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows;
+    a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
     a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = p.T;
     a.stages = p.stages; a.a_slots = p.a_slots;
     a.stage_bytes = p.stage_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
+    a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;
     a.col_delta = p.col_delta; a.col_a = p.col_a;
     a.slot_floats = (uint32_t)p.slot_floats;
     a.alpha = alpha; a.Y = Y;
     a.counters = reinterpret_cast<unsigned int*>(workspace);
-    a.partials = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + p.ws_header_bytes);
+    char* ws = reinterpret_cast<char*>(workspace);
+    a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
     return a;
 }
 
-cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmBits,
-                           const GemmArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream);
+// Workspace regions of the decode schedule.
+inline uint8_t* ws_x8(const Plan& p, void* workspace) {
+    return reinterpret_cast<uint8_t*>(workspace) + p.ws_header_bytes + p.ws_partials_bytes;
+}
+
+// tmX8 is only read in the decode schedule; `after_split` launches the kernel so that it may start
+// while the activation-split kernel queued just before it is still running.
+cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
+                           const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
+                           bool after_split, cudaStream_t stream);
+
+// Decode schedule pre-pass: X bf16 [rows, K] -> four e5m2 pieces per element (k permuted inside
+// each group of 32) in X8 [B, 4, m, K].
+cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, cudaStream_t stream);
 
 // Synchronises the stream, reads {status, site} and clears them if set.
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream);

@@ -14,7 +14,7 @@ constexpr int kQuadK = 256;          // reduction extent of one sign-word slot (
 constexpr int kMaxStages = 8;
 constexpr int kBitSlots = 2;
 constexpr int kMaxASlots = 4;
-constexpr int kASlotCols = 64;       // TMEM columns of one decoded operand slot (128 k, two bf16 per column)
+constexpr int kPieces = 4;           // e5m2 pieces an activation is split into for the decode-regime delta MMA
 constexpr int kTmemCols = 512;
 constexpr int kMaxCtas = 256;        // upper bound on the grid, sizes the workspace
 constexpr int kDecodeMaxM = 16;      // m <= 16: tenants are grouped into one tile
@@ -31,15 +31,21 @@ struct Plan {
     int win_rows;      // X-tile row where tenant j's delta window starts = j * win_rows
     int chunk_rows;    // epilogue: rows of the X tile between consecutive 16-token chunks
     int x_rows;        // rows of X staged per stage (TMA box height)
+    int N3;            // decode: columns of one tenant's delta accumulator = round16(4 m) (pieces x tokens)
+    int x8_rows;       // decode: rows of the e5m2 activation pieces staged per stage (0 in the tiled schedule)
+    int aslot_cols;    // TMEM columns of one decoded-operand buffer: decode TB*16 (all tenants x 64 k of e5m2),
+                       // tiled 64 (one tenant x 128 k of bf16)
     int n_tiles, m_tiles, groups, units;
     int P;             // k-pairs per unit
     long long T;       // total k-pair work items = units * P
     int grid;
     int stages, a_slots;
-    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, bslot_bytes, smem_bytes;
+    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
     uint32_t col_base, col_delta, col_a;
     size_t slot_floats;   // floats of one partial-result slot: 128 rows x tokens per unit
     size_t ws_header_bytes;   // arrival counters: one u32 per work unit
+    size_t ws_partials_bytes; // two partial-result slots per CTA
+    size_t ws_x8_bytes;       // decode: e5m2 pieces of X, [B, 4, m, K] bytes
     size_t ws_bytes;
     bool ok;
 };
@@ -54,16 +60,20 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
     p.decode = (m <= kDecodeMaxM) ? 1 : 0;
     p.n_tiles = (N + kTileN - 1) / kTileN;
     if (p.decode) {
-        p.TB = B < 8 ? B : 8;
+        p.N3 = round_up(kPieces * m, 16);
+        const int tb_max = (m <= 4) ? 8 : 4;          // keeps accumulators + two operand buffers within 512 columns
+        p.TB = B < tb_max ? B : tb_max;
         p.tok_tile = 0;
         p.groups = (B + p.TB - 1) / p.TB;
         p.m_tiles = 1;
         p.Nb = round_up(p.TB * m, 16);
-        p.Nd = 16;
+        p.Nd = p.N3;
         p.win_rows = m;
         p.chunk_rows = m;
         int need = (p.TB - 1) * m + 16;
         p.x_rows = round_up(need > p.Nb ? need : p.Nb, 8);
+        p.x8_rows = round_up((p.TB - 1) * kPieces * m + p.N3, 8);
+        p.aslot_cols = p.TB * 16;
         p.slot_floats = (size_t)kTileN * p.TB * m;
     } else {
         p.TB = 1;
@@ -75,6 +85,9 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
         p.win_rows = 0;
         p.chunk_rows = 16;
         p.x_rows = p.tok_tile;
+        p.N3 = 0;
+        p.x8_rows = 0;
+        p.aslot_cols = 64;
         p.slot_floats = (size_t)kTileN * p.tok_tile;
     }
     p.units = p.n_tiles * p.groups;
@@ -85,7 +98,8 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
 
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
-    p.stage_bytes = 2 * p.w_atom_bytes + 2 * p.x_atom_bytes;
+    p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
+    p.stage_bytes = 2 * p.w_atom_bytes + 2 * p.x_atom_bytes + p.x8_atom_bytes;
     p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
     int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
     p.stages = avail / (int)p.stage_bytes;
@@ -99,14 +113,17 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
     p.col_delta = (uint32_t)p.Nb;
     p.col_a = p.col_delta + (uint32_t)(p.TB * p.Nd);
     int free_cols = kTmemCols - (int)p.col_a;
-    p.a_slots = free_cols / kASlotCols;
+    int slots = free_cols / p.aslot_cols;
+    p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
     if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
-    p.a_slots &= ~1;   // the two decode groups alternate slots
     if (p.a_slots < 2) return p;
 
-    // Workspace: arrival counters, then two partial-result slots per CTA.
+    // Workspace: arrival counters, two partial-result slots per CTA, then (decode) the e5m2
+    // pieces of X written by the activation-split kernel.
     p.ws_header_bytes = (size_t)round_up(p.units * 4, 1024);
-    p.ws_bytes = p.ws_header_bytes + (size_t)2 * kMaxCtas * p.slot_floats * sizeof(float);
+    p.ws_partials_bytes = (size_t)2 * kMaxCtas * p.slot_floats * sizeof(float);
+    p.ws_x8_bytes = p.decode ? (((size_t)B * kPieces * m * K + 1023) / 1024 * 1024) : 0;
+    p.ws_bytes = p.ws_header_bytes + p.ws_partials_bytes + p.ws_x8_bytes;
     p.ok = true;
     return p;
 }
