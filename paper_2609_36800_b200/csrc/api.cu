@@ -131,6 +131,17 @@ bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, u
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// BITDELTA_EARLY_START=0 launches the GEMM kernel fully serialised behind its predecessor
+// (for experiments; the default lets it begin its weight prefetch early).
+bool early_start_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = getenv("BITDELTA_EARLY_START");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -218,9 +229,9 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
     if (!encode_bf16_2d(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
     if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB))
         return BITDELTA_ERR_CUDA;
-    if (p.decode) {
-        // Decode schedule: split the activations into e5m2 pieces first (tiny), then the GEMM, which
-        // may start prefetching weights while the split is still running.
+    if (p.decode && !p.convert) {
+        // Decode schedule with many token rows per tile: split the activations into e5m2 pieces first
+        // (tiny), then the GEMM, which may start prefetching weights while the split is still running.
         uint8_t* x8 = bd::ws_x8(p, workspace);
         if (!encode_u8_2d(&tmX8, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, (uint32_t)p.x8_rows))
             return BITDELTA_ERR_CUDA;
@@ -228,11 +239,11 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
             return BITDELTA_ERR_CUDA;
         g_launches++;
     } else {
-        tmX8 = tmX;   // not read by the tiled schedule
+        tmX8 = tmX;   // not read: the kernel splits the activations itself, or runs the tiled schedule
     }
 
     bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
-    if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, p.decode != 0, stream) != cudaSuccess)
+    if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
     g_launches++;
     return BITDELTA_OK;

@@ -17,6 +17,7 @@
 // grid; tiles cut across CTAs are summed through a workspace by the last CTA
 // to arrive, in a fixed order.
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
 #include "gemm_tc.h"
@@ -29,6 +30,7 @@ constexpr int kThreads = 512;
 constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
 constexpr int kWarpTmem = 2;
+constexpr int kWarpConvert0 = 2;   // warps 2..3 split activations in the decode schedule when asked to
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
 
@@ -57,6 +59,7 @@ struct Ctl {
     uint64_t bempty[kBitSlots];
     uint64_t afull[kMaxASlots];
     uint64_t aempty[kMaxASlots];
+    uint64_t x8full[kMaxStages];
     uint64_t accfull;
     uint64_t accempty;
     uint32_t tmem_base;
@@ -269,6 +272,13 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
     }
 }
 
+__device__ __forceinline__ float e5m2_value(uint8_t v) {
+    return __half2float(__half(__nv_cvt_fp8_to_halfraw(v, __NV_E5M2)));
+}
+__device__ __forceinline__ uint8_t e5m2_round(float v) {
+    return (uint8_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
+}
+
 // 32 packed sign bits -> 8 registers of four e5m2 each (+1 = 0x3C, -1 = 0xBC).  Register c takes
 // bits c, c+8, c+16, c+24 (its bytes 0..3): one shift lands all four on the byte sign positions, one
 // three-input logic op masks them and flips the sign of a packed (-1,-1,-1,-1).  The k order inside
@@ -309,6 +319,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
+            mbar_init(smem_u32(&ctl->x8full[s]), 2);
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
@@ -333,6 +344,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     if (warp == 0) BD_STAMP(1);
+    // A kernel queued behind this one with an early start may begin its own prologue and weight
+    // prefetch as soon as SMs free up; it waits for this grid to finish before it touches anything
+    // this grid reads or writes.
+    if (threadIdx.x == 0) grid_launch_dependents();
 
     const long long lo = (long long)blockIdx.x * a.T / gridDim.x;
     const long long hi = (long long)(blockIdx.x + 1) * a.T / gridDim.x;
@@ -342,51 +357,93 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     if (warp == kWarpProducer) {
         // ------------------------------------------------------------ TMA producer
         // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
+        // Weights (W_base, sign words) never depend on the kernel queued before this one, the
+        // activations may: with an early start the first ring of weight loads is issued, then the
+        // grid dependency is awaited, then the activation loads follow.
         int stage = 0, bslot = 0;
         uint32_t phase = 0, bphase = 0;
         bool ok = true;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty);
-        bool dep_waited = false;
+        const bool load_x8 = a.decode && !a.convert;
+        auto issue_weights = [&](const Unit& u, int p, bool first_of_segment) -> bool {
+            if (first_of_segment || !(p & 1)) {
+                BD_ACC_BEGIN(tb);
+                bool good = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
+                BD_ACC_END(w_bempty, tb);
+                if (!good) return false;
+                if (elect_one()) {
+                    const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
+                    mbar_arrive_expect_tx(bar, a.bslot_bytes);
+                    tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+                }
+                __syncwarp();
+                if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+            }
+            BD_ACC_BEGIN(te);
+            bool good = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
+            BD_ACC_END(w_empty, te);
+            if (!good) return false;
+            if (elect_one()) {
+                const uint32_t bar = smem_u32(&ctl->full[stage]);
+                const uint32_t dst = stages_addr + stage * a.stage_bytes;
+                mbar_arrive_expect_tx(bar, load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes);
+                const int k0 = p * kPairK;
+                tma_load_2d(dst, &tmW, bar, k0, u.n0);
+                tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+            }
+            __syncwarp();
+            return true;
+        };
+        auto issue_activations = [&](const Unit& u, int p, int st) {
+            if (elect_one()) {
+                const uint32_t bar = smem_u32(&ctl->full[st]);
+                const uint32_t dst = stages_addr + st * a.stage_bytes + 2 * a.w_atom_bytes;
+                const int k0 = p * kPairK;
+                tma_load_2d(dst, &tmX, bar, k0, u.xrow0);
+                tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
+                if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, u.tenant0 * kPieces * a.m);
+            }
+            __syncwarp();
+        };
+        // Phase 1: weights of the first ring, before the grid dependency is resolved.
+        // Nothing here may block: only as many stages and sign-word slots as exist are used.
+        SegIter ahead = it;
+        int n_ahead = 0;
+        {
+            int u2, q0, q1, slots_used = 0;
+            bool room = true;
+            while (ok && room && n_ahead < a.stages && ahead.next(u2, q0, q1)) {
+                const Unit u = unit_info(a, u2);
+                int q = q0;
+                for (; q < q1 && n_ahead < a.stages && ok; ++q, ++n_ahead) {
+                    if (q == q0 || !(q & 1)) {
+                        if (slots_used == kBitSlots) { room = false; break; }
+                        ++slots_used;
+                    }
+                    ok = issue_weights(u, q, q == q0);
+                    if (!ok) break;
+                    if (n_ahead == 0) BD_STAMP(2);
+                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                }
+                if (q < q1) break;   // ring full in the middle of a segment
+            }
+        }
+        grid_dependency_wait();
+        // Phase 2: the whole schedule; the first n_ahead stages only still need their activations.
+        int done = 0, st2 = 0;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
-            for (int p = p0; p < p1 && ok; ++p) {
-                if (p == p0 || !(p & 1)) {
-                    BD_ACC_BEGIN(tb);
-                    ok = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
-                    BD_ACC_END(w_bempty, tb);
+            for (int p = p0; p < p1 && ok; ++p, ++done) {
+                if (done < n_ahead) {
+                    issue_activations(u, p, st2);
+                    if (++st2 == a.stages) st2 = 0;
+                } else {
+                    const int st = stage;
+                    ok = issue_weights(u, p, p == p0);
                     if (!ok) break;
-                    if (elect_one()) {
-                        const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
-                        mbar_arrive_expect_tx(bar, a.bslot_bytes);
-                        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
-                    }
-                    __syncwarp();
-                    if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                    issue_activations(u, p, st);
+                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
                 }
-                BD_ACC_BEGIN(te);
-                ok = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
-                BD_ACC_END(w_empty, te);
-                if (!ok) break;
-                if (elect_one()) {
-                    const uint32_t bar = smem_u32(&ctl->full[stage]);
-                    const uint32_t dst = stages_addr + stage * a.stage_bytes;
-                    mbar_arrive_expect_tx(bar, a.stage_bytes);
-                    const int k0 = p * kPairK;
-                    tma_load_2d(dst, &tmW, bar, k0, u.n0);
-                    tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
-                    tma_load_2d(dst + 2 * a.w_atom_bytes, &tmX, bar, k0, u.xrow0);
-                    tma_load_2d(dst + 2 * a.w_atom_bytes + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
-                    if (a.decode) {
-                        // The e5m2 pieces are written by the activation-split kernel queued before this one.
-                        if (!dep_waited) { grid_dependency_wait(); }
-                        tma_load_2d(dst + 2 * a.w_atom_bytes + 2 * a.x_atom_bytes, &tmX8, bar, k0,
-                                    u.tenant0 * kPieces * a.m);
-                    }
-                }
-                dep_waited = true;
-                __syncwarp();
-                if (p == p0 && unit == (int)(lo / a.P)) BD_STAMP(2);
-                if (++stage == a.stages) { stage = 0; phase ^= 1; }
             }
         }
         BD_STAMP(3);
@@ -443,6 +500,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if (a.decode) {
+                    if (a.convert) {
+                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 10));
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
                     const uint64_t x8desc = xdesc + 2 * x_atom16;
                     const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
                     for (int half = 0; half < 2 && ok; ++half, ++item) {
@@ -508,6 +570,64 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             BD_STAMP(6);
         }
         BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
+    } else if (warp >= kWarpConvert0 && warp < kWarpConvert0 + 2 && a.convert) {
+        // ----------------------------------------------- activation split (decode, few rows)
+        // Per stage, thread c of these 64 rewrites one group of 32 k of one token row: it reads the
+        // bf16 values from the swizzled X tile and writes the four e5m2 pieces (see the split
+        // kernel for the arithmetic) into the swizzled piece tile of the same stage.
+        const int cid = threadIdx.x - kWarpConvert0 * 32;   // 0..63
+        const int r = cid >> 2, g = cid & 3;                // token row of the unit, 32-k group of the stage
+        const int j = r / a.m, t = r - j * a.m;             // tenant of the unit, token
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            for (int p = p0; p < p1 && ok; ++p) {
+                ok = wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 11);
+                if (!ok) break;
+                if (r < u.ntok) {
+                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
+                    const uint8_t* src = xt + (g >> 1) * a.x_atom_bytes + r * 128;
+                    uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+                    float y[32];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const int chunk = ((g & 1) * 4 + h) ^ (r & 7);
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + chunk * 16);
+                        const uint32_t q4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            y[h * 8 + 2 * i] = __uint_as_float(q4[i] << 16);
+                            y[h * 8 + 2 * i + 1] = __uint_as_float(q4[i] & 0xFFFF0000u);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < kPieces; ++q) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t acc = 0;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const uint8_t pc = e5m2_round(y[c + 8 * i]);
+                                y[c + 8 * i] -= e5m2_value(pc);
+                                acc |= (uint32_t)pc << (8 * i);
+                            }
+                            w[c] = acc;
+                        }
+                        const int r8 = j * (kPieces * a.m) + q * a.m + t;
+                        uint8_t* dst = x8t + r8 * 128;
+                        *reinterpret_cast<uint4*>(dst + (((2 * g) ^ (r8 & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4*>(dst + (((2 * g + 1) ^ (r8 & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    }
+                }
+                fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMA's async-proxy reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->x8full[stage]));
+                if (++stage == a.stages) { stage = 0; phase ^= 1; }
+            }
+        }
     } else if (warp >= kWarpDecode0 && warp < kWarpEpi0) {
         // ------------------------------------------- sign decode -> tensor memory
         const int dw = warp - kWarpDecode0;    // 0..7
@@ -621,6 +741,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             tc_fence_after();
             accphase ^= 1;
             if (warp == kWarpEpi0) BD_STAMP(7);
+            grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
             if (a.decode) {
                 switch (a.m) {
@@ -707,7 +828,7 @@ extern "C" int bitdelta_debug_set_trace(long long* buf) {
 
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
-                           bool after_split, cudaStream_t stream) {
+                           bool early_start, cudaStream_t stream) {
     static int attr_device = -1;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -726,7 +847,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = after_split ? 1 : 0;
+    cfg.numAttrs = early_start ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, bitdelta_gemm_tc_kernel, tmW, tmX, tmX8, tmBits, args);
 }
 

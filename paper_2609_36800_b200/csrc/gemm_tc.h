@@ -11,7 +11,7 @@ namespace bd {
 
 struct GemmArgs {
     int B, m, N, K;
-    int decode, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
+    int decode, convert, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
     int m_tiles, groups, P;
     long long T;
     int stages, a_slots;
@@ -27,7 +27,7 @@ struct GemmArgs {
 inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* workspace) {
     GemmArgs a{};
     a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
-    a.decode = p.decode; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
+    a.decode = p.decode; a.convert = p.convert; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
     a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
     a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = p.T;
     a.stages = p.stages; a.a_slots = p.a_slots;
@@ -48,11 +48,11 @@ inline uint8_t* ws_x8(const Plan& p, void* workspace) {
     return reinterpret_cast<uint8_t*>(workspace) + p.ws_header_bytes + p.ws_partials_bytes;
 }
 
-// tmX8 is only read in the decode schedule; `after_split` launches the kernel so that it may start
-// while the activation-split kernel queued just before it is still running.
+// tmX8 is only read in the decode schedule with a pre-pass split; `early_start` launches the kernel so
+// that it may begin (prologue, weight prefetch) while the kernel queued just before it is still running.
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
-                           bool after_split, cudaStream_t stream);
+                           bool early_start, cudaStream_t stream);
 
 // Decode schedule pre-pass: X bf16 [rows, K] -> four e5m2 pieces per element (k permuted inside
 // each group of 32) in X8 [B, 4, m, K].

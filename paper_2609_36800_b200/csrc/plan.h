@@ -33,6 +33,8 @@ struct Plan {
     int x_rows;        // rows of X staged per stage (TMA box height)
     int N3;            // decode: columns of one tenant's delta accumulator = round16(4 m) (pieces x tokens)
     int x8_rows;       // decode: rows of the e5m2 activation pieces staged per stage (0 in the tiled schedule)
+    int convert;       // decode: 1 = the kernel itself splits the activations (few token rows per unit),
+                       //         0 = a pre-pass kernel writes the pieces to the workspace
     int aslot_cols;    // TMEM columns of one decoded-operand buffer: decode TB*16 (all tenants x 64 k of e5m2),
                        // tiled 64 (one tenant x 128 k of bf16)
     int n_tiles, m_tiles, groups, units;
@@ -74,6 +76,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
         p.x_rows = round_up(need > p.Nb ? need : p.Nb, 8);
         p.x8_rows = round_up((p.TB - 1) * kPieces * m + p.N3, 8);
         p.aslot_cols = p.TB * 16;
+        p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
     } else {
         p.TB = 1;
@@ -86,6 +89,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
         p.chunk_rows = 16;
         p.x_rows = p.tok_tile;
         p.N3 = 0;
+        p.convert = 0;
         p.x8_rows = 0;
         p.aslot_cols = 64;
         p.slot_floats = (size_t)kTileN * p.tok_tile;
