@@ -90,6 +90,27 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
+// Same contract, for the warp on the critical path (the MMA issuer): spins on the non-suspending
+// test so that it reacts within a few cycles of the phase completing, instead of paying the wake-up
+// latency of a suspended try_wait on every hand-over.
+__device__ __forceinline__ bool spin_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i) {
+            if (mbar_test_wait(bar, parity)) return true;
+        }
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
+            return false;
+        }
+    }
+}
+
 // Walks the k-pair items [lo, hi) of this CTA as segments (unit, p0, p1).
 struct SegIter {
     long long cur, hi;
@@ -205,10 +226,11 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
 }
 
 // Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
+// Two warps share each lane quadrant: warp half h drains the 32-token blocks h, h+2, ...
 __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                               const EpiOut& out) {
+                                               const EpiOut& out, int half) {
     const float al = __ldg(a.alpha + u.tenant0);
-    for (int t0 = 0; t0 < u.ntok; t0 += 32) {
+    for (int t0 = 32 * half; t0 < u.ntok; t0 += 64) {
         uint32_t rb[32], rd[32];
         tmem_ld32(lane_taddr + (uint32_t)t0, rb);
         tmem_ld32(lane_taddr + a.col_delta + (uint32_t)t0, rd);
@@ -224,25 +246,25 @@ __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u,
 __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 // Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
-// 128 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+4, ...
-__device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, const float* first,
-                                                const float* rest, size_t cstride, int nrest) {
+// nwarps*32 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+nwarps, ...
+__device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, int nwarps,
+                                                const float* first, const float* rest, size_t cstride, int nrest) {
     __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
     const int r4 = (etid & 31) * 4;
     const int n = u.n0 + r4;
     const bool vec_ok = ((a.N & 3) == 0) && (n + 3 < a.N);
-    for (int tk = etid >> 5; tk < u.ntok; tk += 16) {
+    for (int tk = etid >> 5; tk < u.ntok; tk += 4 * nwarps) {
         float4 acc[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const int t = tk + 4 * q;
+            const int t = tk + nwarps * q;
             acc[q] = (t < u.ntok) ? ldcg4(first + (size_t)t * kTileN + r4) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         for (int c = 0; c < nrest; ++c) {
             const float* pc = rest + (size_t)c * cstride;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const int t = tk + 4 * q;
+                const int t = tk + nwarps * q;
                 if (t < u.ntok) {
                     const float4 v = ldcg4(pc + (size_t)t * kTileN + r4);
                     acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
@@ -251,7 +273,7 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const int t = tk + 4 * q;
+            const int t = tk + nwarps * q;
             if (t < u.ntok) {
                 __nv_bfloat16* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
                 if (vec_ok) {
@@ -289,7 +311,7 @@ __device__ __forceinline__ void decode_word_e5m2(uint32_t w, uint32_t* r) {
     for (int c = 0; c < 8; ++c) r[c] = ((w << (7 - c)) & 0x80808080u) ^ 0xBCBCBCBCu;
 }
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
@@ -307,6 +329,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Tiled schedule: signs need few decode threads, the epilogue many -> warps 8..11 drain accumulators
+    // instead of decoding.
+    const int epi_first_warp = a.decode ? kWarpEpi0 : kWarpEpi0 - 4;
+    const int n_epi_warps = 16 - epi_first_warp;
     if (warp == 0) BD_STAMP(0);
     if (threadIdx.x == 32) {
         prefetch_tensormap(&tmW);
@@ -323,14 +349,14 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
-            mbar_init(smem_u32(&ctl->bempty[s]), 8);
+            mbar_init(smem_u32(&ctl->bempty[s]), a.decode ? 8 : 4);
         }
         for (int s = 0; s < kMaxASlots; ++s) {
             mbar_init(smem_u32(&ctl->afull[s]), a.decode ? 8 : 4);
             mbar_init(smem_u32(&ctl->aempty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->accfull), 1);
-        mbar_init(smem_u32(&ctl->accempty), 4);
+        mbar_init(smem_u32(&ctl->accempty), a.decode ? 4 : 8);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
@@ -472,16 +498,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             BD_ACC_BEGIN(ta);
-            ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            ok = warp_all(spin_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
             BD_ACC_END(w_acc, ta);
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
                 BD_ACC_BEGIN(tf);
-                ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                 BD_ACC_END(w_full, tf);
                 if (!ok) break;
-                tc_fence_after();
                 if (item == 0) BD_STAMP(4);
                 const uint32_t wbase = stages_addr + stage * a.stage_bytes;
                 const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
@@ -501,9 +526,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 BD_ACC_END(w_ib, tib);
                 if (a.decode) {
                     if (a.convert) {
-                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 10));
+                        ok = warp_all(spin_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 10));
                         if (!ok) break;
-                        tc_fence_after();
                     }
                     const uint64_t x8desc = xdesc + 2 * x_atom16;
                     const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
@@ -511,7 +535,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tg);
-                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        ok = warp_all(spin_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
                         BD_ACC_END(w_afull, tg);
                         if (!ok) break;
                         tc_fence_after();
@@ -536,7 +560,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tg);
-                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        ok = warp_all(spin_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
                         BD_ACC_END(w_afull, tg);
                         if (!ok) break;
                         tc_fence_after();
@@ -572,54 +596,60 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
     } else if (warp >= kWarpConvert0 && warp < kWarpConvert0 + 2 && a.convert) {
         // ----------------------------------------------- activation split (decode, few rows)
-        // Per stage, thread c of these 64 rewrites one group of 32 k of one token row: it reads the
-        // bf16 values from the swizzled X tile and writes the four e5m2 pieces (see the split
-        // kernel for the arithmetic) into the swizzled piece tile of the same stage.
+        // Per stage these 64 threads read the bf16 values of the unit's token rows from the swizzled X
+        // tile and write their four e5m2 pieces (same values as the split kernel produces) into the
+        // swizzled piece tile of the same stage.
+        // Task (r, g, h): token row r of the unit, 32-k group g of the stage, half h of the group's
+        // byte slots.  Slot 4c+i holds k = c + 8i, so half h (c = 4h..4h+3) needs, from each of the
+        // group's four 16-byte chunks (i = 0..3), the 8 bytes holding k = 8i+4h .. 8i+4h+3, and
+        // produces one 16-byte chunk per piece.  Arithmetic runs on packed f16 pairs (a bf16 value in
+        // the e5m2 range is exact in f16): p = rn_e5m2(y); y -= p; four times.
         const int cid = threadIdx.x - kWarpConvert0 * 32;   // 0..63
-        const int r = cid >> 2, g = cid & 3;                // token row of the unit, 32-k group of the stage
-        const int j = r / a.m, t = r - j * a.m;             // tenant of the unit, token
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
+            const int ntasks = u.ntok * 8;
             for (int p = p0; p < p1 && ok; ++p) {
                 ok = wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 11);
                 if (!ok) break;
-                if (r < u.ntok) {
-                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
-                    const uint8_t* src = xt + (g >> 1) * a.x_atom_bytes + r * 128;
-                    uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-                    float y[32];
+                uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
+                uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+                for (int task = cid; task < ntasks; task += 64) {
+                    const int r = task >> 3, g = (task >> 1) & 3, h = task & 1;
+                    const int j = r / a.m, t = r - j * a.m;
+                    const uint8_t* src = xt + (g >> 1) * a.x_atom_bytes + r * 128 + h * 8;
+                    __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
 #pragma unroll
-                    for (int h = 0; h < 4; ++h) {
-                        const int chunk = ((g & 1) * 4 + h) ^ (r & 7);
-                        const uint4 v = *reinterpret_cast<const uint4*>(src + chunk * 16);
-                        const uint32_t q4[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            y[h * 8 + 2 * i] = __uint_as_float(q4[i] << 16);
-                            y[h * 8 + 2 * i + 1] = __uint_as_float(q4[i] & 0xFFFF0000u);
-                        }
+                    for (int i = 0; i < 4; ++i) {
+                        const int chunk = ((g & 1) * 4 + i) ^ (r & 7);
+                        const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
+                        y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+                        y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
                     }
 #pragma unroll
                     for (int q = 0; q < kPieces; ++q) {
-                        uint32_t w[8];
+                        uint32_t pk[8];
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t acc = 0;
+                        for (int e = 0; e < 8; ++e) {
+                            const __nv_fp8x2_storage_t pc =
+                                __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
+                            y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
+                            pk[e] = pc;
+                        }
+                        // pk[2i+pc] = {byte for c = 4h+2pc at i (low), byte for c+1 (high)}; word c gathers i = 0..3
+                        uint32_t w[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const uint8_t pc = e5m2_round(y[c + 8 * i]);
-                                y[c + 8 * i] -= e5m2_value(pc);
-                                acc |= (uint32_t)pc << (8 * i);
-                            }
-                            w[c] = acc;
+                        for (int pc = 0; pc < 2; ++pc) {
+                            const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
+                            const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
+                            w[2 * pc] = __byte_perm(r01, r23, 0x6420);
+                            w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
                         }
                         const int r8 = j * (kPieces * a.m) + q * a.m + t;
-                        uint8_t* dst = x8t + r8 * 128;
-                        *reinterpret_cast<uint4*>(dst + (((2 * g) ^ (r8 & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-                        *reinterpret_cast<uint4*>(dst + (((2 * g + 1) ^ (r8 & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+                        *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * g + h) ^ (r8 & 7)) * 16)) =
+                            make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
                 fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMA's async-proxy reads
@@ -628,7 +658,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (++stage == a.stages) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp >= kWarpDecode0 && warp < kWarpEpi0) {
+    } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {
         // ------------------------------------------- sign decode -> tensor memory
         const int dw = warp - kWarpDecode0;    // 0..7
         const int grp = dw >> 2;
@@ -681,7 +711,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     }
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
-                        if ((int)(item & 1) != grp) continue;
                         const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
@@ -717,11 +746,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
         if (warp == kWarpDecode0) { BD_ACC_STORE(21, w_bfull); BD_ACC_STORE(22, w_aempty); BD_ACC_STORE(23, w_work); }
         if (warp == kWarpDecode0 + 4) { BD_ACC_STORE(24, w_bfull); BD_ACC_STORE(25, w_aempty); BD_ACC_STORE(26, w_work); }
-    } else if (warp >= kWarpEpi0) {
+    } else if (warp >= epi_first_warp) {
         // ---------------------------------------------------------------- epilogue
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
-        const int etid = threadIdx.x - kWarpEpi0 * 32;
+        const int etid = threadIdx.x - epi_first_warp * 32;
+        const int ehalf = (warp - epi_first_warp) >> 2;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int first_unit = (int)(lo / a.P);
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
@@ -740,7 +770,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
-            if (warp == kWarpEpi0) BD_STAMP(7);
+            if (warp == epi_first_warp) BD_STAMP(7);
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
             if (a.decode) {
@@ -763,12 +793,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     default: epilogue_decode<16>(a, u, lane_taddr, out); break;
                 }
             } else {
-                epilogue_tiled(a, u, lane_taddr, out);
+                epilogue_tiled(a, u, lane_taddr, out, ehalf);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
-            if (warp == kWarpEpi0) BD_STAMP(8);
+            if (warp == epi_first_warp) BD_STAMP(8);
 
             if (!whole) {
                 // This tile is cut across CTAs: publish the partial, count arrivals, and let
@@ -777,25 +807,25 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const int c0 = (int)(((first_item + 1) * gridDim.x - 1) / a.T);
                 const int c1 = (int)(((first_item + a.P) * (long long)gridDim.x - 1) / a.T);
                 __threadfence();
-                epi_bar_sync();
+                epi_bar_sync(n_epi_warps * 32);
                 if (etid == 0) {
                     const unsigned old = atomicAdd(&a.counters[unit], 1u);
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
-                epi_bar_sync();
-                if (warp == kWarpEpi0) BD_STAMP(9);
+                epi_bar_sync(n_epi_warps * 32);
+                if (warp == epi_first_warp) BD_STAMP(9);
                 if (ctl->is_last) {
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
                     // range starts exactly there.  Every later CTA starts inside the tile.
                     const int slot0 = ((long long)c0 * a.T / gridDim.x == first_item) ? 2 * c0 : 2 * c0 + 1;
-                    reduce_partials(a, u, etid, a.partials + (size_t)slot0 * a.slot_floats,
+                    reduce_partials(a, u, etid, n_epi_warps, a.partials + (size_t)slot0 * a.slot_floats,
                                     a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats,
                                     2 * (size_t)a.slot_floats, c1 - c0);
                     if (etid == 0) a.counters[unit] = 0u;
                 }
-                epi_bar_sync();   // is_last is rewritten by the next cut tile
-                if (warp == kWarpEpi0) BD_STAMP(10);
+                epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
+                if (warp == epi_first_warp) BD_STAMP(10);
             }
         }
     }
