@@ -689,7 +689,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tq);
-                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = spin_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
@@ -715,7 +715,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tq);
-                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = spin_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
