@@ -30,7 +30,8 @@ constexpr int kThreads = 512;
 constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
 constexpr int kWarpTmem = 2;
-constexpr int kWarpConvert0 = 2;   // warps 2..3 split activations in the decode schedule when asked to
+constexpr int kWarpDelta0 = 2;     // decode schedule: warps 2..3 issue the delta MMAs of decode group 0 / 1
+constexpr int kBarAFull0 = 2;      // named barriers 2.. : decode group g, buffer b -> id 2 + g*4 + b
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
 
@@ -57,9 +58,8 @@ struct Ctl {
     uint64_t empty[kMaxStages];
     uint64_t bfull[kBitSlots];
     uint64_t bempty[kBitSlots];
-    uint64_t afull[kMaxASlots];
-    uint64_t aempty[kMaxASlots];
-    uint64_t x8full[kMaxStages];
+    uint64_t afull[kMaxASlots];        // tiled schedule: decoded operand ready (decode warps -> MMA warp)
+    uint64_t aempty[2 * kMaxASlots];   // operand buffer free again (tcgen05.commit); decode: [group][buffer]
     uint64_t accfull;
     uint64_t accempty;
     uint32_t tmem_base;
@@ -344,18 +344,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
-            mbar_init(smem_u32(&ctl->x8full[s]), 2);
+            mbar_init(smem_u32(&ctl->empty[s]), a.decode ? 3 : 1);   // decode: three MMA issuers release a stage
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
             mbar_init(smem_u32(&ctl->bempty[s]), a.decode ? 8 : 4);
         }
-        for (int s = 0; s < kMaxASlots; ++s) {
-            mbar_init(smem_u32(&ctl->afull[s]), a.decode ? 8 : 4);
-            mbar_init(smem_u32(&ctl->aempty[s]), 1);
-        }
-        mbar_init(smem_u32(&ctl->accfull), 1);
+        for (int s = 0; s < kMaxASlots; ++s) mbar_init(smem_u32(&ctl->afull[s]), 4);
+        for (int s = 0; s < 2 * kMaxASlots; ++s) mbar_init(smem_u32(&ctl->aempty[s]), 1);
+        mbar_init(smem_u32(&ctl->accfull), a.decode ? 3 : 1);
         mbar_init(smem_u32(&ctl->accempty), a.decode ? 4 : 8);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
@@ -525,36 +522,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if (a.decode) {
-                    if (a.convert) {
-                        ok = warp_all(spin_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 10));
-                        if (!ok) break;
-                    }
-                    const uint64_t x8desc = xdesc + 2 * x_atom16;
-                    const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
-                    for (int half = 0; half < 2 && ok; ++half, ++item) {
-                        const uint32_t slot = item & amask;
-                        const uint32_t use = item >> ashift;
-                        BD_ACC_BEGIN(tg);
-                        ok = warp_all(spin_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
-                        BD_ACC_END(w_afull, tg);
-                        if (!ok) break;
-                        tc_fence_after();
-                        if (item == 0) BD_STAMP(5);
-                        BD_ACC_BEGIN(tid);
-                        const uint32_t a_buf = tmem_base + a.col_a + slot * (uint32_t)a.aslot_cols;
-                        const uint32_t acc = (half > 0) ? 1u : first;
-                        if (elect_one()) {
-                            for (int j = 0; j < u.nten; ++j) {
-                                const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
-                                const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
-                                umma_ts_f8(d_tmem, a_buf + j * 16, xj, idesc_delta, acc);
-                                umma_ts_f8(d_tmem, a_buf + j * 16 + 8, xj + 2, idesc_delta, 1u);
-                            }
-                            tc_commit(smem_u32(&ctl->aempty[slot]));
-                        }
-                        __syncwarp();
-                        BD_ACC_END(w_id, tid);
-                    }
+                    // Delta MMAs are issued by the two delta-issuer warps.
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
                         const uint32_t slot = item & amask;
@@ -594,68 +562,117 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             BD_STAMP(6);
         }
         BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
-    } else if (warp >= kWarpConvert0 && warp < kWarpConvert0 + 2 && a.convert) {
-        // ----------------------------------------------- activation split (decode, few rows)
-        // Per stage these 64 threads read the bf16 values of the unit's token rows from the swizzled X
-        // tile and write their four e5m2 pieces (same values as the split kernel produces) into the
-        // swizzled piece tile of the same stage.
-        // Task (r, g, h): token row r of the unit, 32-k group g of the stage, half h of the group's
-        // byte slots.  Slot 4c+i holds k = c + 8i, so half h (c = 4h..4h+3) needs, from each of the
-        // group's four 16-byte chunks (i = 0..3), the 8 bytes holding k = 8i+4h .. 8i+4h+3, and
-        // produces one 16-byte chunk per piece.  Arithmetic runs on packed f16 pairs (a bf16 value in
-        // the e5m2 range is exact in f16): p = rn_e5m2(y); y -= p; four times.
-        const int cid = threadIdx.x - kWarpConvert0 * 32;   // 0..63
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        while (ok && it.next(unit, p0, p1)) {
-            const Unit u = unit_info(a, unit);
-            const int ntasks = u.ntok * 8;
-            for (int p = p0; p < p1 && ok; ++p) {
-                ok = wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 11);
+    } else if (warp >= kWarpDelta0 && warp < kWarpDelta0 + 2) {
+        // ------------------------------------------------- delta issuers (decode schedule)
+        // Warp 2+g serves decode group g (tenants j = g, g+2, ... of the unit).  Per 128-k stage it
+        //  * (few token rows per unit) splits those tenants' activations into e5m2 pieces itself,
+        //    reading the bf16 X tile and writing the swizzled piece tile of the stage, and
+        //  * per 64-k half waits, on a named barrier, for the group's decode warps to have filled the
+        //    operand buffer in tensor memory, issues that half's MMAs and commits the buffer's release.
+        // Nothing else writes those tenants' accumulators, so their summation order is fixed.
+        if (a.decode) {
+            const int g = warp - kWarpDelta0;
+            const uint32_t idesc_delta = make_idesc_e5m2(kTileN, (uint32_t)a.Nd);
+            const uint64_t desc0 = make_smem_desc_sw128(0);
+            const uint32_t x_atom16 = a.x_atom_bytes >> 4;
+            const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
+            const uint32_t amask = (uint32_t)a.a_slots - 1;
+            const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+            int stage = 0;
+            uint32_t phase = 0, accphase = 0, item = 0;
+            bool ok = true;
+            while (ok && it.next(unit, p0, p1)) {
+                const Unit u = unit_info(a, unit);
+                ok = warp_all(spin_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
                 if (!ok) break;
-                uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
-                uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-                for (int task = cid; task < ntasks; task += 64) {
-                    const int r = task >> 3, g = (task >> 1) & 3, h = task & 1;
-                    const int j = r / a.m, t = r - j * a.m;
-                    const uint8_t* src = xt + (g >> 1) * a.x_atom_bytes + r * 128 + h * 8;
-                    __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
+                tc_fence_after();
+                for (int p = p0; p < p1 && ok; ++p) {
+                    ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                    if (!ok) break;
+                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
+                    if (a.convert) {
+                        // Task (r, q4, h): token row r (of this group's tenants), 32-k group q4 of the stage,
+                        // half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
+                        // (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the
+                        // group, the 8 bytes holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk
+                        // per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
+                        // exact in f16): p = rn_e5m2(y); y -= p; four times.
+                        uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+                        const int ntasks = u.ntok * 8;
+                        for (int task = lane; task < ntasks; task += 32) {
+                            const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
+                            const int j = r / a.m, t = r - j * a.m;
+                            if ((j & 1) != g) continue;
+                            const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
+                            __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int chunk = ((g & 1) * 4 + i) ^ (r & 7);
-                        const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
-                        y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
-                        y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
-                    }
+                            for (int i = 0; i < 4; ++i) {
+                                const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
+                                const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
+                                y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+                                y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+                            }
 #pragma unroll
-                    for (int q = 0; q < kPieces; ++q) {
-                        uint32_t pk[8];
+                            for (int q = 0; q < kPieces; ++q) {
+                                uint32_t pk[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const __nv_fp8x2_storage_t pc =
-                                __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
-                            y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
-                            pk[e] = pc;
+                                for (int e = 0; e < 8; ++e) {
+                                    const __nv_fp8x2_storage_t pc = __nv_cvt_halfraw2_to_fp8x2(
+                                        static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
+                                    y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
+                                    pk[e] = pc;
+                                }
+                                uint32_t w[4];
+#pragma unroll
+                                for (int pc = 0; pc < 2; ++pc) {
+                                    const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
+                                    const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
+                                    w[2 * pc] = __byte_perm(r01, r23, 0x6420);
+                                    w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
+                                }
+                                const int r8 = j * (kPieces * a.m) + q * a.m + t;
+                                *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) =
+                                    make_uint4(w[0], w[1], w[2], w[3]);
+                            }
                         }
-                        // pk[2i+pc] = {byte for c = 4h+2pc at i (low), byte for c+1 (high)}; word c gathers i = 0..3
-                        uint32_t w[4];
-#pragma unroll
-                        for (int pc = 0; pc < 2; ++pc) {
-                            const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
-                            const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
-                            w[2 * pc] = __byte_perm(r01, r23, 0x6420);
-                            w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
-                        }
-                        const int r8 = j * (kPieces * a.m) + q * a.m + t;
-                        *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * g + h) ^ (r8 & 7)) * 16)) =
-                            make_uint4(w[0], w[1], w[2], w[3]);
+                        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+                        __syncwarp();
                     }
+                    const uint64_t x8desc = desc0 + ((stages_addr + stage * a.stage_bytes + 2 * a.w_atom_bytes) >> 4) +
+                                            2 * x_atom16;
+                    const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
+                    for (int half = 0; half < 2; ++half, ++item) {
+                        const uint32_t slot = item & amask;
+                        if (*abort_flag) { ok = false; break; }
+                        // The group's 128 decode threads arrive here once the buffer is filled (or when they
+                        // give up after an abandoned wait, see the end of the decode role).
+                        named_bar_sync(kBarAFull0 + g * 4 + (int)slot, 160);
+                        if (*abort_flag) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_buf = tmem_base + a.col_a + (uint32_t)(g * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
+                        const uint32_t acc = (half > 0) ? 1u : first;
+                        if (elect_one()) {
+                            for (int j = g; j < u.nten; j += 2) {
+                                const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                                const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
+                                const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 16;
+                                umma_ts_f8(d_tmem, a_j, xj, idesc_delta, acc);
+                                umma_ts_f8(d_tmem, a_j + 8, xj + 2, idesc_delta, 1u);
+                            }
+                            tc_commit(smem_u32(&ctl->aempty[g * kMaxASlots + slot]));
+                        }
+                        __syncwarp();
+                    }
+                    if (!ok) break;
+                    if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
+                    __syncwarp();
+                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
                 }
-                fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMA's async-proxy reads
+                if (!ok) break;
+                if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->x8full[stage]));
-                if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                accphase ^= 1;
+                (void)ashift;
             }
         }
     } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {
@@ -683,29 +700,29 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
                 const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
                 if (a.decode) {
-                    // All eight warps fill every buffer: warp (grp, quad) decodes, for its 32 rows,
-                    // the tenants j = grp, grp+2, ... (64 k = two sign words each).
+                    // Warp (grp, quad) decodes, for its 32 rows, the tenants j = grp, grp+2, ... (64 k = two
+                    // sign words each) into its group's ring of operand buffers, then arrives on the
+                    // buffer's named barrier, on which the group's delta issuer waits.
                     for (int half = 0; half < 2 && ok; ++half, ++item) {
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tq);
-                        ok = spin_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = wait_bar(smem_u32(&ctl->aempty[grp * kMaxASlots + slot]), (use & 1) ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
                         BD_ACC_BEGIN(tw);
-                        const uint32_t tbuf = lane_taddr + a.col_a + slot * (uint32_t)a.aslot_cols;
+                        const uint32_t tbuf = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         for (int j = grp; j < u.nten; j += 2) {
                             const uint2 w = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
                             uint32_t r[16];
                             decode_word_e5m2(w.x, r);
                             decode_word_e5m2(w.y, r + 8);
-                            tmem_st16(tbuf + j * 16, r);
+                            tmem_st16(tbuf + (uint32_t)(j >> 1) * 16, r);
                         }
                         tc_wait_st();
                         tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                        named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
                         BD_ACC_END(w_work, tw);
                         if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
@@ -743,6 +760,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
                 }
             }
+        }
+        if (a.decode && *abort_flag) {
+            // A wait was abandoned somewhere in the CTA.  The group's delta issuer may be blocked on one
+            // of the named barriers (they have no time-out): arrive on all of them so that it wakes up,
+            // sees the abort flag and leaves.
+            __syncwarp();
+            for (int sl = 0; sl < a.a_slots; ++sl) named_bar_arrive(kBarAFull0 + grp * 4 + sl, 160);
         }
         if (warp == kWarpDecode0) { BD_ACC_STORE(21, w_bfull); BD_ACC_STORE(22, w_aempty); BD_ACC_STORE(23, w_work); }
         if (warp == kWarpDecode0 + 4) { BD_ACC_STORE(24, w_bfull); BD_ACC_STORE(25, w_aempty); BD_ACC_STORE(26, w_work); }

@@ -35,8 +35,8 @@ struct Plan {
     int x8_rows;       // decode: rows of the e5m2 activation pieces staged per stage (0 in the tiled schedule)
     int convert;       // decode: 1 = the kernel itself splits the activations (few token rows per unit),
                        //         0 = a pre-pass kernel writes the pieces to the workspace
-    int aslot_cols;    // TMEM columns of one decoded-operand buffer: decode TB*16 (all tenants x 64 k of e5m2),
-                       // tiled 64 (one tenant x 128 k of bf16)
+    int aslot_cols;    // TMEM columns of one decoded-operand buffer: decode ceil(TB/2)*16 (one decode group's
+                       // tenants x 64 k of e5m2; a_slots buffers per group), tiled 64 (one tenant x 128 k of bf16)
     int n_tiles, m_tiles, groups, units;
     int P;             // k-pairs per unit
     long long T;       // total k-pair work items = units * P
@@ -75,7 +75,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
         int need = (p.TB - 1) * m + 16;
         p.x_rows = round_up(need > p.Nb ? need : p.Nb, 8);
         p.x8_rows = round_up((p.TB - 1) * kPieces * m + p.N3, 8);
-        p.aslot_cols = p.TB * 16;
+        p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
     } else {
@@ -118,6 +118,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
     p.col_a = p.col_delta + (uint32_t)(p.TB * p.Nd);
     int free_cols = kTmemCols - (int)p.col_a;
     int slots = free_cols / p.aslot_cols;
+    if (p.decode) slots /= 2;                          // each of the two decode groups has its own ring
     p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
     if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
     if (p.a_slots < 2) return p;
