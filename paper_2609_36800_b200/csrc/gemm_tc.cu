@@ -31,7 +31,8 @@ constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
 constexpr int kWarpTmem = 2;
 constexpr int kWarpDelta0 = 2;     // decode schedule: warps 2..3 issue the delta MMAs of decode group 0 / 1
-constexpr int kBarAFull0 = 2;      // named barriers 2.. : decode group g, buffer b -> id 2 + g*4 + b
+constexpr int kBarAFull0 = 2;      // named barriers 2..9 : decode group g, buffer b -> id 2 + g*4 + b
+constexpr int kBarX8Full0 = 10;    // named barriers 10..13: e5m2 pieces of stage s written (in-kernel split)
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
 
@@ -523,6 +524,55 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 BD_ACC_END(w_ib, tib);
                 if (a.decode) {
                     // Delta MMAs are issued by the two delta-issuer warps.
+                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
+                    if (a.convert) {
+                        // Few token rows per unit: this warp also splits the stage's activations into e5m2 pieces for
+                        // the delta issuers.  Task (r, q4, h): token row r, 32-k group q4 of the stage,
+                        // half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
+                        // (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the
+                        // group, the 8 bytes holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk
+                        // per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
+                        // exact in f16): p = rn_e5m2(y); y -= p; four times.
+                        uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+                        const int ntasks = u.ntok * 8;
+                        for (int task = lane; task < ntasks; task += 32) {
+                            const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
+                            const int j = r / a.m, t = r - j * a.m;
+                            const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
+                            __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
+                                const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
+                                y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+                                y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+                            }
+#pragma unroll
+                            for (int q = 0; q < kPieces; ++q) {
+                                uint32_t pk[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const __nv_fp8x2_storage_t pc = __nv_cvt_halfraw2_to_fp8x2(
+                                        static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
+                                    y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
+                                    pk[e] = pc;
+                                }
+                                uint32_t w[4];
+#pragma unroll
+                                for (int pc = 0; pc < 2; ++pc) {
+                                    const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
+                                    const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
+                                    w[2 * pc] = __byte_perm(r01, r23, 0x6420);
+                                    w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
+                                }
+                                const int r8 = j * (kPieces * a.m) + q * a.m + t;
+                                *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) =
+                                    make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+                        named_bar_arrive(kBarX8Full0 + stage, 96);
+                    }
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
                         const uint32_t slot = item & amask;
@@ -561,6 +611,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             BD_STAMP(6);
         }
+        if (a.decode && a.convert && *abort_flag) {
+            // Abandoned wait somewhere: the delta issuers may be blocked on a piece barrier.
+            __syncwarp();
+            for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
+        }
         BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
     } else if (warp >= kWarpDelta0 && warp < kWarpDelta0 + 2) {
         // ------------------------------------------------- delta issuers (decode schedule)
@@ -589,54 +644,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 for (int p = p0; p < p1 && ok; ++p) {
                     ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                     if (!ok) break;
-                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
                     if (a.convert) {
-                        // Task (r, q4, h): token row r (of this group's tenants), 32-k group q4 of the stage,
-                        // half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
-                        // (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the
-                        // group, the 8 bytes holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk
-                        // per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
-                        // exact in f16): p = rn_e5m2(y); y -= p; four times.
-                        uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-                        const int ntasks = u.ntok * 8;
-                        for (int task = lane; task < ntasks; task += 32) {
-                            const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
-                            const int j = r / a.m, t = r - j * a.m;
-                            if ((j & 1) != g) continue;
-                            const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
-                            __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
-                                const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
-                                y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
-                                y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
-                            }
-#pragma unroll
-                            for (int q = 0; q < kPieces; ++q) {
-                                uint32_t pk[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const __nv_fp8x2_storage_t pc = __nv_cvt_halfraw2_to_fp8x2(
-                                        static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
-                                    y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
-                                    pk[e] = pc;
-                                }
-                                uint32_t w[4];
-#pragma unroll
-                                for (int pc = 0; pc < 2; ++pc) {
-                                    const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
-                                    const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
-                                    w[2 * pc] = __byte_perm(r01, r23, 0x6420);
-                                    w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
-                                }
-                                const int r8 = j * (kPieces * a.m) + q * a.m + t;
-                                *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) =
-                                    make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
-                        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
-                        __syncwarp();
+                        // The base issuer wrote this stage's e5m2 pieces; it arrives when they are visible.
+                        if (*abort_flag) { ok = false; break; }
+                        named_bar_sync(kBarX8Full0 + stage, 96);
+                        if (*abort_flag) { ok = false; break; }
                     }
                     const uint64_t x8desc = desc0 + ((stages_addr + stage * a.stage_bytes + 2 * a.w_atom_bytes) >> 4) +
                                             2 * x_atom16;
@@ -673,6 +685,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 accphase ^= 1;
                 (void)ashift;
+            }
+            if (a.convert && *abort_flag) {
+                // Leave no other issuer blocked on a piece barrier this warp would have joined.
+                __syncwarp();
+                for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
             }
         }
     } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {

@@ -108,6 +108,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
     int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
     p.stages = avail / (int)p.stage_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (p.decode && p.stages > 4) p.stages = 4;   // one named barrier per stage for the in-kernel split
     if (p.stages < 2) return p;
     p.smem_bytes = 1024 + p.stages * p.stage_bytes + kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
     // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
