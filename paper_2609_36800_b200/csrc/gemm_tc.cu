@@ -39,6 +39,11 @@ constexpr int kWarpEpi0 = 12;      // warps 12..15
 #ifdef BD_TRACE
 // Debug builds only: per-CTA cycle stamps of the main phases.
 __device__ long long* g_trace_ptr;
+// What-if switches for timing experiments (results are wrong when any is set):
+// 1 skip sign decode ALU, 2 skip delta MMAs, 4 skip base MMAs, 8 skip sign-word loads, 16 skip W loads,
+// 32 skip activation loads, 64 skip tensor-memory stores of the decode warps, 128 skip the in-kernel split
+__device__ int g_knobs;
+#define BD_KNOB(bit) (g_knobs & (bit))
 #define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = clock64(); } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
@@ -46,6 +51,7 @@ __device__ long long* g_trace_ptr;
 #define BD_ACC_STORE(idx, name) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = name; } while (0)
 #else
 #define BD_STAMP(idx) do { } while (0)
+#define BD_KNOB(bit) 0
 #define BD_ACC_DECL(name) do { } while (0)
 #define BD_ACC_BEGIN(t) do { } while (0)
 #define BD_ACC_END(name, t) do { } while (0)
@@ -397,8 +403,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (!good) return false;
                 if (elect_one()) {
                     const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
-                    mbar_arrive_expect_tx(bar, a.bslot_bytes);
-                    tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+                    if (BD_KNOB(8)) {
+                        mbar_arrive(bar);
+                    } else {
+                        mbar_arrive_expect_tx(bar, a.bslot_bytes);
+                        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+                    }
                 }
                 __syncwarp();
                 if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
@@ -410,16 +420,21 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (elect_one()) {
                 const uint32_t bar = smem_u32(&ctl->full[stage]);
                 const uint32_t dst = stages_addr + stage * a.stage_bytes;
-                mbar_arrive_expect_tx(bar, load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes);
+                uint32_t tx = load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes;
+                if (BD_KNOB(16)) tx -= 2 * a.w_atom_bytes;
+                if (BD_KNOB(32)) tx -= 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0);
+                if (tx) mbar_arrive_expect_tx(bar, tx); else mbar_arrive(bar);
                 const int k0 = p * kPairK;
-                tma_load_2d(dst, &tmW, bar, k0, u.n0);
-                tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+                if (!BD_KNOB(16)) {
+                    tma_load_2d(dst, &tmW, bar, k0, u.n0);
+                    tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+                }
             }
             __syncwarp();
             return true;
         };
         auto issue_activations = [&](const Unit& u, int p, int st) {
-            if (elect_one()) {
+            if (!BD_KNOB(32) && elect_one()) {
                 const uint32_t bar = smem_u32(&ctl->full[st]);
                 const uint32_t dst = stages_addr + st * a.stage_bytes + 2 * a.w_atom_bytes;
                 const int k0 = p * kPairK;
@@ -512,7 +527,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const uint64_t xdesc = desc0 + (xbase >> 4);
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
                 BD_ACC_BEGIN(tib);
-                if (elect_one()) {
+                if (!BD_KNOB(4) && elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t atom = kk >> 2, k16 = kk & 3;
@@ -535,7 +550,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         // exact in f16): p = rn_e5m2(y); y -= p; four times.
                         uint8_t* x8t = xt + 2 * a.x_atom_bytes;
                         const int ntasks = u.ntok * 8;
-                        for (int task = lane; task < ntasks; task += 32) {
+                        for (int task = lane; task < (BD_KNOB(128) ? 0 : ntasks); task += 32) {
                             const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
                             const int j = r / a.m, t = r - j * a.m;
                             const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
@@ -664,7 +679,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t a_buf = tmem_base + a.col_a + (uint32_t)(g * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         const uint32_t acc = (half > 0) ? 1u : first;
                         if (elect_one()) {
-                            for (int j = g; j < u.nten; j += 2) {
+                            for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
                                 const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                                 const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
                                 const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 16;
@@ -733,9 +748,14 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         for (int j = grp; j < u.nten; j += 2) {
                             const uint2 w = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
                             uint32_t r[16];
-                            decode_word_e5m2(w.x, r);
-                            decode_word_e5m2(w.y, r + 8);
-                            tmem_st16(tbuf + (uint32_t)(j >> 1) * 16, r);
+                            if (BD_KNOB(1)) {
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) r[c] = w.x + c;
+                            } else {
+                                decode_word_e5m2(w.x, r);
+                                decode_word_e5m2(w.y, r + 8);
+                            }
+                            if (!BD_KNOB(64)) tmem_st16(tbuf + (uint32_t)(j >> 1) * 16, r);
                         }
                         tc_wait_st();
                         tc_fence_before();
@@ -894,6 +914,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 #ifdef BD_TRACE
 extern "C" int bitdelta_debug_set_trace(long long* buf) {
     return (int)cudaMemcpyToSymbol(g_trace_ptr, &buf, sizeof(buf));
+}
+extern "C" int bitdelta_debug_set_knobs(int knobs) {
+    return (int)cudaMemcpyToSymbol(g_knobs, &knobs, sizeof(knobs));
 }
 #endif
 
