@@ -228,7 +228,16 @@ def cpu_baseline(wl, host_inputs, budget_s=15.0):
     }
 
 
-def summarize(wl, ms_total, steps, n_gpus, peaks):
+def kernels_per_step(wl):
+    """Kernels one bitdelta_gemm call launches: the GEMM kernel, plus the activation-split kernel in the
+    decode schedule when a tile holds more than 16 token rows (otherwise the GEMM kernel splits itself)."""
+    if wl.m > 16:
+        return 1
+    tb = min(wl.B, 8 if wl.m <= 4 else 4)
+    return 1 if tb * wl.m <= 16 else 2
+
+
+def summarize(wl, ms_total, steps, n_gpus, peaks, clocks=None):
     sec = ms_total / 1e3 / steps
     gbs = wl.bytes * n_gpus / sec / 1e9
     tfl = wl.flops * n_gpus / sec / 1e12
@@ -238,9 +247,15 @@ def summarize(wl, ms_total, steps, n_gpus, peaks):
         roof = {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": per_gpu_gbs / peaks["hbm_gbs"]}
     else:
-        roof = {"bound": "tensor", "achieved": per_gpu_tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": per_gpu_tfl / peaks["bf16_tflops"],
-                "frac_of_sustained": per_gpu_tfl / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])}
+        # A kernel timed inside a long, power-capped run is held against the sustained cuBLAS figure,
+        # one timed in a short burst at full clocks against the burst figure; both fractions are printed.
+        capped = bool(clocks and "sw_power_cap" in (clocks.get("reasons") or []))
+        burst = peaks["bf16_tflops"]
+        sustained = peaks.get("bf16_tflops_sustained", burst)
+        peak = sustained if capped else burst
+        roof = {"bound": "tensor", "achieved": per_gpu_tfl, "peak": peak, "unit": "TFLOP/s",
+                "frac": per_gpu_tfl / peak, "peak_kind": "sustained" if capped else "burst",
+                "frac_of_burst": per_gpu_tfl / burst, "frac_of_sustained": per_gpu_tfl / sustained}
     roof["peak_source"] = peaks["_source"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
     roof["algorithmic_bytes"] = wl.bytes
@@ -279,7 +294,7 @@ def run_ours(args):
         ms = float(t.item())
     del _sets
     torch.cuda.empty_cache()
-    gbs, tfl, roof = summarize(wl, ms, args.steps, world, peaks)
+    gbs, tfl, roof = summarize(wl, ms, args.steps, world, peaks, clocks)
 
     out = None
     if rank == 0:
@@ -303,7 +318,7 @@ def run_ours(args):
             "e2e": {"value": e_val, "unit": "GB/s" if hbm_bound else "TFLOP/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": e2e_steps,
                     "call": "bitdelta_gemm_host (pinned host buffers, stream synchronised each step)"},
-            "gpu_launches": args.steps,
+            "gpu_launches": args.steps * kernels_per_step(wl),
             "library_launches_issued": bd.kernel_launch_count() - launches0,
             "clocks": clocks,
             "context": PAPER_CONTEXT,
