@@ -93,6 +93,33 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * bitdelta_gemm for callers that must not allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for the deployment case below.)
+ *
+ * Some hosts of this library may not call cudaMalloc at all: code that runs inside a frozen,
+ * pre-sized memory plan (a serving engine after start-up, a plug-in loaded into a process that owns
+ * every byte of its memory pool, a real-time loop where an allocation can stall or fail).  They
+ * cannot obtain the workspace bitdelta_gemm asks for.  This variant needs none from the caller: its
+ * scratch is a fixed array of BITDELTA_NOALLOC_SCRATCH_BYTES that is part of the library's device
+ * image, so every GPU that loads the library holds it from load until the process exits.  The call
+ * itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine) and needs no
+ * bitdelta_workspace_init.
+ *
+ * Arguments and result are those of bitdelta_gemm, without the workspace pair.
+ *   - Shapes whose workspace (bitdelta_gemm_workspace_bytes) exceeds the array are refused with
+ *     BITDELTA_ERR_WORKSPACE and nothing is launched; use bitdelta_gemm with your own buffer.
+ *   - The first call on each device looks up the array's device address (the current device must be
+ *     the one the call is for); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call first clears, on the stream, the arrival
+ *     counters at its start; the rest keeps whatever the previous call left and is fully rewritten
+ *     before it is read.  Calls that can overlap on the device (issued on different streams) would
+ *     race on it: keep all calls for one device on one stream, or order the streams with events.
+ */
+#define BITDELTA_NOALLOC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int bitdelta_gemm_noalloc(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
+                          void* Y, int B, int m, int N, int K, void* cuda_stream);
+
+/*
  * Diagnostic variant of bitdelta_gemm on plain CUDA cores (one warp per output
  * row, fp32 accumulation in k order per lane).  Same arguments and result
  * contract; needs no workspace.  Slow; used to triage the tensor-core path.

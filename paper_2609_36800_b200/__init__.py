@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     gemm,
     gemm_host,
     gemm_host_arena_bytes,
+    gemm_noalloc,
     gemm_workspace_bytes,
     kernel_launch_count,
     last_device_status,

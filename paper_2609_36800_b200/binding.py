@@ -18,7 +18,7 @@ STATUS_TIMEOUT = 7
 
 EXPORTS = (
     "bitdelta_pack", "bitdelta_unpack", "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
-    "bitdelta_gemm", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
+    "bitdelta_gemm", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
     "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
 )
 
@@ -51,6 +51,7 @@ def load_library():
     lib.bitdelta_workspace_init.argtypes = [vp, sz, vp]
     lib.bitdelta_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
     lib.bitdelta_gemm_simt.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
+    lib.bitdelta_gemm_noalloc.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
     lib.bitdelta_gemm_host_arena_bytes.argtypes = [ci, ci, ci, ci]
     lib.bitdelta_gemm_host_arena_bytes.restype = sz
     lib.bitdelta_gemm_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
@@ -59,7 +60,7 @@ def load_library():
     lib.bitdelta_status_string.argtypes = [ci]
     lib.bitdelta_status_string.restype = ctypes.c_char_p
     for fn in ("bitdelta_pack", "bitdelta_unpack", "bitdelta_workspace_init", "bitdelta_gemm",
-               "bitdelta_gemm_simt", "bitdelta_gemm_host", "bitdelta_last_device_status"):
+               "bitdelta_gemm_simt", "bitdelta_gemm_noalloc", "bitdelta_gemm_host", "bitdelta_last_device_status"):
         getattr(lib, fn).restype = ci
     _lib = lib
     return lib
@@ -142,6 +143,26 @@ def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bo
         workspace = make_workspace(B, m, N, K, device=X.device, stream=stream)
     _check(lib.bitdelta_gemm(*args, ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream)),
            "bitdelta_gemm")
+    return out
+
+
+NOALLOC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def gemm_noalloc(X, W_base, bits, alpha, out, stream=None):
+    """bitdelta_gemm for callers that may not allocate device memory: same arguments as `gemm` with a
+    caller-provided `out`, no workspace.  The scratch is a fixed array inside the library (16 MiB per GPU);
+    shapes needing more raise BitDeltaError(status 4).  Calls that may overlap on the device race on it."""
+    import torch
+    B, m, K = X.shape
+    N = W_base.shape[0]
+    if W_base.shape != (N, K) or tuple(bits.shape) != (B, N, K // 32) or tuple(alpha.shape) != (B,) \
+            or tuple(out.shape) != (B, m, N):
+        raise ValueError("inconsistent shapes")
+    _check(load_library().bitdelta_gemm_noalloc(
+        _dev(X, torch.bfloat16, "X"), _dev(W_base, torch.bfloat16, "W_base"), _dev(bits, torch.int32, "bits"),
+        _dev(alpha, torch.float32, "alpha"), _dev(out, torch.bfloat16, "out"), B, m, N, K, _stream_ptr(stream)),
+        "bitdelta_gemm_noalloc")
     return out
 
 

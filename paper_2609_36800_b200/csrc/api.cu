@@ -14,6 +14,11 @@
 #include "gemm_tc.h"
 #include "plan.h"
 
+// Scratch of bitdelta_gemm_noalloc: lives in the library's device image (zero at load), one copy per GPU
+// that loads the library.  In host code this name is only a handle for cudaGetSymbolAddress, never an
+// address a kernel could use.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[BITDELTA_NOALLOC_SCRATCH_BYTES];
+
 namespace {
 
 std::atomic<unsigned long long> g_launches{0};
@@ -306,6 +311,43 @@ int bitdelta_last_device_status(void* cuda_stream, int* site) {
     if (bd::read_device_status(st, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return BITDELTA_ERR_CUDA;
     if (site) *site = (int)st[1];
     return st[0] == 0 ? BITDELTA_OK : (int)st[0];
+}
+
+int bitdelta_gemm_noalloc(const void* X, const void* W_base, const uint32_t* bits, const float* alpha, void* Y, int B,
+                          int m, int N, int K, void* cuda_stream) {
+    int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
+    if (st != BITDELTA_OK) return st;
+    DeviceInfo d;
+    st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    const size_t need = bitdelta_gemm_workspace_bytes(B, m, N, K);
+    if (need == 0) return BITDELTA_ERR_SHAPE;
+    if (need > (size_t)BITDELTA_NOALLOC_SCRATCH_BYTES) return BITDELTA_ERR_WORKSPACE;
+
+    // Device address of the scratch array, looked up once per device with that device current.
+    static void* scratch_ptr[64] = {};
+    static std::mutex mu;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (d.device < 0 || d.device >= 64) return BITDELTA_ERR_CUDA;
+        if (!scratch_ptr[d.device]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return BITDELTA_ERR_CUDA;
+            scratch_ptr[d.device] = p;
+        }
+        scratch = scratch_ptr[d.device];
+    }
+    // The arrival counters at the start of the scratch have to be zero when the kernel begins; a call
+    // that was cut short could have left them otherwise.
+    if ((K % 128) == 0) {
+        bd::Plan plan = bd::make_plan(B, m, N, K, d.sms);
+        if (!plan.ok) return BITDELTA_ERR_SHAPE;
+        if (cudaMemsetAsync(scratch, 0, plan.ws_header_bytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+            return BITDELTA_ERR_CUDA;
+    }
+    return bitdelta_gemm(X, W_base, bits, alpha, Y, B, m, N, K, scratch, (size_t)BITDELTA_NOALLOC_SCRATCH_BYTES,
+                         cuda_stream);
 }
 
 unsigned long long bitdelta_kernel_launch_count(void) { return g_launches.load(); }
