@@ -289,9 +289,8 @@ def run_ours(args):
     ms, nsets, host_inputs, _sets = time_workload(wl, args.steps, args.warmup, dist, sampler)
     clocks = sampler.stop() if sampler is not None else None
     if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        from paper_2609_36800_b200 import replicas
+        ms = replicas.max_over_ranks(ms, dist, device="cuda")
     del _sets
     torch.cuda.empty_cache()
     gbs, tfl, roof = summarize(wl, ms, args.steps, world, peaks, clocks)
