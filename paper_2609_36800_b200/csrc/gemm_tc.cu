@@ -45,6 +45,9 @@ __device__ long long* g_trace_ptr;
 __device__ int g_knobs;
 #define BD_KNOB(bit) (g_knobs & (bit))
 #define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = clock64(); } while (0)
+// Per-role timelines of CTA 0 and CTA 77: role r's i-th stamp at trace[8192 + cta_sel*1024 + r*128 + i].
+#define BD_TL_DECL int tl_idx = 0
+#define BD_TL(role) do { if (g_trace_ptr && lane == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && tl_idx < 128) { g_trace_ptr[8192 + (blockIdx.x ? 1024 : 0) + (role) * 128 + tl_idx] = clock64(); ++tl_idx; } } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
 #define BD_ACC_END(name, t) name += clock64() - t
@@ -52,6 +55,8 @@ __device__ int g_knobs;
 #else
 #define BD_STAMP(idx) do { } while (0)
 #define BD_KNOB(bit) 0
+#define BD_TL_DECL do { } while (0)
+#define BD_TL(role) do { } while (0)
 #define BD_ACC_DECL(name) do { } while (0)
 #define BD_ACC_BEGIN(t) do { } while (0)
 #define BD_ACC_END(name, t) do { } while (0)
@@ -393,7 +398,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0, bslot = 0;
         uint32_t phase = 0, bphase = 0;
         bool ok = true;
-        BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty);
+        BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
         const bool load_x8 = a.decode && !a.convert;
         auto issue_weights = [&](const Unit& u, int p, bool first_of_segment) -> bool {
             if (first_of_segment || !(p & 1)) {
@@ -431,6 +436,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
             }
             __syncwarp();
+            BD_TL(0);
             return true;
         };
         auto issue_activations = [&](const Unit& u, int p, int st) {
@@ -507,7 +513,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0;
         uint32_t phase = 0, accphase = 0, item = 0;
         bool ok = true;
-        BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id);
+        BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id); BD_TL_DECL;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             BD_ACC_BEGIN(ta);
@@ -521,6 +527,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 BD_ACC_END(w_full, tf);
                 if (!ok) break;
                 if (item == 0) BD_STAMP(4);
+                BD_TL(1);
                 const uint32_t wbase = stages_addr + stage * a.stage_bytes;
                 const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
                 const uint64_t wdesc = desc0 + (wbase >> 4);
@@ -651,6 +658,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             int stage = 0;
             uint32_t phase = 0, accphase = 0, item = 0;
             bool ok = true;
+            BD_TL_DECL;
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
                 ok = warp_all(spin_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
@@ -659,6 +667,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 for (int p = p0; p < p1 && ok; ++p) {
                     ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                     if (!ok) break;
+                    if (g == 0) BD_TL(2);
                     if (a.convert) {
                         // The base issuer wrote this stage's e5m2 pieces; it arrives when they are visible.
                         if (*abort_flag) { ok = false; break; }
@@ -676,6 +685,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         named_bar_sync(kBarAFull0 + g * 4 + (int)slot, 160);
                         if (*abort_flag) { ok = false; break; }
                         tc_fence_after();
+                        if (g == 0) BD_TL(2);
                         const uint32_t a_buf = tmem_base + a.col_a + (uint32_t)(g * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         const uint32_t acc = (half > 0) ? 1u : first;
                         if (elect_one()) {
@@ -719,7 +729,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int bslot = 0;
         uint32_t bphase = 0, item = 0;
         bool ok = true;
-        BD_ACC_DECL(w_bfull); BD_ACC_DECL(w_aempty); BD_ACC_DECL(w_work);
+        BD_ACC_DECL(w_bfull); BD_ACC_DECL(w_aempty); BD_ACC_DECL(w_work); BD_TL_DECL;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             for (int p = p0; p < p1 && ok; ++p) {
@@ -743,6 +753,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
+                        if (warp == kWarpDecode0) BD_TL(3);
                         BD_ACC_BEGIN(tw);
                         const uint32_t tbuf = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         for (int j = grp; j < u.nten; j += 2) {
@@ -761,6 +772,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         tc_fence_before();
                         named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
                         BD_ACC_END(w_work, tw);
+                        if (warp == kWarpDecode0) BD_TL(3);
                         if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
                 } else {
