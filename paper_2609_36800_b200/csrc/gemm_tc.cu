@@ -43,7 +43,11 @@ __device__ long long* g_trace_ptr;
 // 1 skip sign decode ALU, 2 skip delta MMAs, 4 skip base MMAs, 8 skip sign-word loads, 16 skip W loads,
 // 32 skip activation loads, 64 skip tensor-memory stores of the decode warps, 128 skip the in-kernel split
 __device__ int g_knobs;
+#ifdef BD_NO_KNOBS
+#define BD_KNOB(bit) 0
+#else
 #define BD_KNOB(bit) (g_knobs & (bit))
+#endif
 #define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = clock64(); } while (0)
 // Per-role timelines of CTA 0 and CTA 77: role r's i-th stamp at trace[8192 + cta_sel*1024 + r*128 + i].
 #define BD_TL_DECL int tl_idx = 0
@@ -517,13 +521,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             BD_ACC_BEGIN(ta);
-            ok = warp_all(spin_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
             BD_ACC_END(w_acc, ta);
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
                 BD_ACC_BEGIN(tf);
-                ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                 BD_ACC_END(w_full, tf);
                 if (!ok) break;
                 if (item == 0) BD_STAMP(4);
@@ -600,7 +604,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tg);
-                        ok = warp_all(spin_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
                         BD_ACC_END(w_afull, tg);
                         if (!ok) break;
                         tc_fence_after();
@@ -661,11 +665,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             BD_TL_DECL;
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
-                ok = warp_all(spin_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+                ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
                 if (!ok) break;
                 tc_fence_after();
                 for (int p = p0; p < p1 && ok; ++p) {
-                    ok = warp_all(spin_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                    ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                     if (!ok) break;
                     if (g == 0) BD_TL(2);
                     if (a.convert) {
@@ -677,7 +681,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     const uint64_t x8desc = desc0 + ((stages_addr + stage * a.stage_bytes + 2 * a.w_atom_bytes) >> 4) +
                                             2 * x_atom16;
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
-                    for (int half = 0; half < 2; ++half, ++item) {
+                    for (int half = 0; half < a.halves; ++half, ++item) {
                         const uint32_t slot = item & amask;
                         if (*abort_flag) { ok = false; break; }
                         // The group's 128 decode threads arrive here once the buffer is filled (or when they
@@ -687,14 +691,28 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         tc_fence_after();
                         if (g == 0) BD_TL(2);
                         const uint32_t a_buf = tmem_base + a.col_a + (uint32_t)(g * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
-                        const uint32_t acc = (half > 0) ? 1u : first;
                         if (elect_one()) {
-                            for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
-                                const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
-                                const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
-                                const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 16;
-                                umma_ts_f8(d_tmem, a_j, xj, idesc_delta, acc);
-                                umma_ts_f8(d_tmem, a_j + 8, xj + 2, idesc_delta, 1u);
+                            if (a.halves == 2) {
+                                // 64 k per hand-over: two K=32 steps per tenant, 16 operand columns each
+                                const uint32_t acc = (half > 0) ? 1u : first;
+                                for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
+                                    const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                                    const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
+                                    const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 16;
+                                    umma_ts_f8(d_tmem, a_j, xj, idesc_delta, acc);
+                                    umma_ts_f8(d_tmem, a_j + 8, xj + 2, idesc_delta, 1u);
+                                }
+                            } else {
+                                // the whole 128-k stage: four K=32 steps per tenant, 32 operand columns each
+                                for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
+                                    const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                                    const uint64_t xj = x8desc + (uint32_t)j * ten_rows16;
+                                    const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 32;
+                                    umma_ts_f8(d_tmem, a_j, xj, idesc_delta, first);
+                                    umma_ts_f8(d_tmem, a_j + 8, xj + 2, idesc_delta, 1u);
+                                    umma_ts_f8(d_tmem, a_j + 16, xj + 4, idesc_delta, 1u);
+                                    umma_ts_f8(d_tmem, a_j + 24, xj + 6, idesc_delta, 1u);
+                                }
                             }
                             tc_commit(smem_u32(&ctl->aempty[g * kMaxASlots + slot]));
                         }
@@ -745,7 +763,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // Warp (grp, quad) decodes, for its 32 rows, the tenants j = grp, grp+2, ... (64 k = two
                     // sign words each) into its group's ring of operand buffers, then arrives on the
                     // buffer's named barrier, on which the group's delta issuer waits.
-                    for (int half = 0; half < 2 && ok; ++half, ++item) {
+                    for (int half = 0; half < a.halves && ok; ++half, ++item) {
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tq);
@@ -756,19 +774,45 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         if (warp == kWarpDecode0) BD_TL(3);
                         BD_ACC_BEGIN(tw);
                         const uint32_t tbuf = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
-                        for (int j = grp; j < u.nten; j += 2) {
-                            const uint2 w = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
-                            uint32_t r[16];
-                            if (BD_KNOB(1)) {
-#pragma unroll
-                                for (int c = 0; c < 16; ++c) r[c] = w.x + c;
-                            } else {
+                        if (a.halves == 1) {
+                            // whole stage: four sign words (128 k) per tenant, 32 operand columns each
+                            for (int j = grp; j < u.nten; j += 2) {
+                                const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
+                                uint32_t r[32];
                                 decode_word_e5m2(w.x, r);
                                 decode_word_e5m2(w.y, r + 8);
+                                decode_word_e5m2(w.z, r + 16);
+                                decode_word_e5m2(w.w, r + 24);
+                                tmem_st32(tbuf + (uint32_t)(j >> 1) * 32, r);
                             }
-                            if (!BD_KNOB(64)) tmem_st16(tbuf + (uint32_t)(j >> 1) * 16, r);
+                        } else {
+                            // This warp's tenants are j = grp + 2*i, i < 4: fetch all their sign words first, so the
+                            // shared-memory latency is paid once, then decode and store.
+                            uint2 w[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int j = grp + 2 * i;
+                                if (j < u.nten) w[i] = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int j = grp + 2 * i;
+                                if (j < u.nten) {
+                                    uint32_t r[16];
+                                    if (BD_KNOB(1)) {
+#pragma unroll
+                                        for (int c = 0; c < 16; ++c) r[c] = w[i].x + c;
+                                    } else {
+                                        decode_word_e5m2(w[i].x, r);
+                                        decode_word_e5m2(w[i].y, r + 8);
+                                    }
+                                    if (!BD_KNOB(64)) tmem_st16(tbuf + (uint32_t)i * 16, r);
+                                }
+                            }
                         }
+                        if (warp == kWarpDecode0) BD_TL(3);
                         tc_wait_st();
+                        if (warp == kWarpDecode0) BD_TL(3);
                         tc_fence_before();
                         named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
                         BD_ACC_END(w_work, tw);
@@ -781,7 +825,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
                         BD_ACC_BEGIN(tq);
-                        ok = spin_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();

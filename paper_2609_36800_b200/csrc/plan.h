@@ -42,6 +42,7 @@ struct Plan {
     long long T;       // total k-pair work items = units * P
     int grid;
     int stages, a_slots;
+    int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
     uint32_t col_base, col_delta, col_a;
     size_t slot_floats;   // floats of one partial-result slot: 128 rows x tokens per unit
@@ -54,7 +55,7 @@ struct Plan {
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
+inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
@@ -65,6 +66,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
         p.N3 = round_up(kPieces * m, 16);
         const int tb_max = (m <= 4) ? 8 : 4;          // keeps accumulators + two operand buffers within 512 columns
         p.TB = B < tb_max ? B : tb_max;
+        if (tb_override > 0 && tb_override <= tb_max && tb_override <= B) p.TB = tb_override;
         p.tok_tile = 0;
         p.groups = (B + p.TB - 1) / p.TB;
         p.m_tiles = 1;
@@ -118,6 +120,13 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms) {
     p.col_delta = (uint32_t)p.Nb;
     p.col_a = p.col_delta + (uint32_t)(p.TB * p.Nd);
     int free_cols = kTmemCols - (int)p.col_a;
+    p.halves = 2;
+    if (p.decode && free_cols >= 2 * 2 * 2 * p.aslot_cols) {
+        // Room for two whole-stage buffers per decode group: hand over 128 k at a time, which halves
+        // the number of hand-overs (their fixed cost is comparable to the decode work of 64 k).
+        p.halves = 1;
+        p.aslot_cols *= 2;
+    }
     int slots = free_cols / p.aslot_cols;
     if (p.decode) slots /= 2;                          // each of the two decode groups has its own ring
     p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
