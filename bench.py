@@ -34,10 +34,10 @@ PAPER_CONTEXT = "paper: 3.34x (standard) / 2.51x (batched) over autotuned Triton
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernel from the
 # ncu captures summarised under profiles/ ; None where no capture exists yet.
 NCU_TRAFFIC_BYTES = {
-    "decode_attn": None,
-    "decode_mlp_up": None,
-    "prefill": None,
-    "many_tenant_down": None,
+    "decode_attn": 50_497_000,          # 50.49 MB read + 0.01 MB written
+    "decode_mlp_up": 233_000_000,       # 227.2 MB read + 5.8 MB written
+    "prefill": 73_400_000,              # 61.7 MB read + 11.7 MB written
+    "many_tenant_down": 1_305_000_000,  # 1.298 GB read + 7.4 MB written (W_base re-read per tenant group)
     "tiny": None,
 }
 
@@ -217,13 +217,15 @@ def cpu_baseline(wl, host_inputs, budget_s=15.0):
 
     probe = min(total, 2048)
     rate = probe / max(sample(probe), 1e-9)          # outputs per second
-    count = int(min(total, max(probe, rate * budget_s)))
-    dt = sample(count)
-    frac = count / total
+    wall_target = budget_s / max(cores, 1) * 1.5     # ~budget_s CPU-seconds of work
+    count = int(min(total, max(probe, rate * wall_target)))
+    reps = max(1, int(round(wall_target * rate / count)))
+    dt = sum(sample(count) for _ in range(reps))
+    frac = count * reps / total
     return {
         "value": wl.bytes * frac / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-        "sample": f"{count} of {total} outputs (b,t,n) drawn uniformly, each a full length-{wl.K} fp64 dot pair; "
-                  f"{dt:.2f} s wall",
+        "sample": f"{reps} x {count} of {total} outputs (b,t,n) drawn uniformly, each a full length-{wl.K} fp64 "
+                  f"dot pair; {dt:.2f} s wall on {cores} threads",
         "tflops": wl.flops * frac / dt / 1e12,
     }
 
