@@ -131,9 +131,16 @@ __device__ __forceinline__ bool spin_bar(uint32_t bar, uint32_t parity, volatile
 struct SegIter {
     long long cur, hi;
     int P;
+    int stride;   // 0: the CTA owns the items [cur, hi); > 0: whole units cur/P, cur/P + stride, ... (see plan.h)
     __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
         if (cur >= hi) return false;
         unit = (int)(cur / P);
+        if (stride > 0) {
+            p0 = 0;
+            p1 = P;
+            cur += (long long)stride * P;
+            return true;
+        }
         p0 = (int)(cur - (long long)unit * P);
         long long rem = hi - cur;
         int len = (rem < (long long)(P - p0)) ? (int)rem : (P - p0);
@@ -388,9 +395,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     // this grid reads or writes.
     if (threadIdx.x == 0) grid_launch_dependents();
 
-    const long long lo = (long long)blockIdx.x * a.T / gridDim.x;
-    const long long hi = (long long)(blockIdx.x + 1) * a.T / gridDim.x;
-    SegIter it{lo, hi, a.P};
+    // Work: either an even share of the flat item list, or (whole-unit order) units b, b+grid, ...
+    const long long lo = a.whole_units ? (long long)blockIdx.x * a.P : (long long)blockIdx.x * a.T / gridDim.x;
+    const long long hi = a.whole_units ? a.T : (long long)(blockIdx.x + 1) * a.T / gridDim.x;
+    SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
     int unit, p0, p1;
 
     if (warp == kWarpProducer) {

@@ -39,6 +39,7 @@ struct Plan {
                        // tenants x 64 k of e5m2; a_slots buffers per group), tiled 64 (one tenant x 128 k of bf16)
     int n_tiles, m_tiles, groups, units;
     int P;             // k-pairs per unit
+    int whole_units;   // 1: CTAs take whole units round-robin (no tile is cut), 0: even shares of the item list
     long long T;       // total k-pair work items = units * P
     int grid;
     int stages, a_slots;
@@ -55,7 +56,7 @@ struct Plan {
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0) {
+inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
@@ -101,6 +102,17 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.T = (long long)p.units * p.P;
     int max_grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
     p.grid = p.T < max_grid ? (int)p.T : max_grid;
+    // Several tenant groups share each W_base tile.  If every CTA takes whole units in round-robin
+    // order, the groups of a tile run side by side on neighbouring CTAs and sweep k in step, so all
+    // but the first read of a W_base tile hit L2 (cut anywhere, the groups sit at different k and
+    // W_base is fetched from HBM once per group).  Taken when it costs little balance.
+    p.whole_units = 0;
+    if (p.decode && p.groups > 1 && p.units >= max_grid) {
+        const int rounds = (p.units + max_grid - 1) / max_grid;
+        const double balance = (double)p.units / ((double)rounds * max_grid);
+        if (balance >= 0.85 || whole_override == 1) { p.whole_units = 1; p.grid = max_grid; }
+    }
+    if (whole_override == 2) p.whole_units = 0;
 
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
