@@ -317,11 +317,50 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
     }
 }
 
-__device__ __forceinline__ float e5m2_value(uint8_t v) {
-    return __half2float(__half(__nv_cvt_fp8_to_halfraw(v, __NV_E5M2)));
-}
-__device__ __forceinline__ uint8_t e5m2_round(float v) {
-    return (uint8_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
+// In-kernel activation split (decode schedule, few token rows per unit).  Task (r, q4, h): token row r,
+// 32-k group q4 of the stage, half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
+// (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the group, the 8 bytes
+// holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk per piece.  Arithmetic on packed f16
+// pairs (a bf16 value in the e5m2 range is exact in f16): p = rn_e5m2(y); y -= p; four times.
+// `xt` is the stage's X tile (two swizzled 64-k atoms), followed by the piece tile.  Thread `tid` of
+// `nthreads` takes the tasks tid, tid + nthreads, ...
+__device__ __forceinline__ void split_activations(const GemmArgs& a, uint8_t* xt, int ntok, int tid, int nthreads) {
+    uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+    const int ntasks = BD_KNOB(128) ? 0 : ntok * 8;
+    for (int task = tid; task < ntasks; task += nthreads) {
+        const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
+        const int j = r / a.m, t = r - j * a.m;
+        const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
+        __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
+            const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
+            y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+            y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+        }
+#pragma unroll
+        for (int q = 0; q < kPieces; ++q) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const __nv_fp8x2_storage_t pc =
+                    __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
+                y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
+                pk[e] = pc;
+            }
+            uint32_t w[4];
+#pragma unroll
+            for (int pc = 0; pc < 2; ++pc) {
+                const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
+                const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
+                w[2 * pc] = __byte_perm(r01, r23, 0x6420);
+                w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
+            }
+            const int r8 = j * (kPieces * a.m) + q * a.m + t;
+            *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
 }
 
 // 32 packed sign bits -> 8 registers of four e5m2 each (+1 = 0x3C, -1 = 0xBC).  Register c takes
@@ -560,52 +599,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // Delta MMAs are issued by the two delta-issuer warps.
                     uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
                     if (a.convert) {
-                        // Few token rows per unit: this warp also splits the stage's activations into e5m2 pieces for
-                        // the delta issuers.  Task (r, q4, h): token row r, 32-k group q4 of the stage,
-                        // half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
-                        // (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the
-                        // group, the 8 bytes holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk
-                        // per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
-                        // exact in f16): p = rn_e5m2(y); y -= p; four times.
-                        uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-                        const int ntasks = u.ntok * 8;
-                        for (int task = lane; task < (BD_KNOB(128) ? 0 : ntasks); task += 32) {
-                            const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
-                            const int j = r / a.m, t = r - j * a.m;
-                            const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
-                            __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
-                                const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
-                                y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
-                                y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
-                            }
-#pragma unroll
-                            for (int q = 0; q < kPieces; ++q) {
-                                uint32_t pk[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const __nv_fp8x2_storage_t pc = __nv_cvt_halfraw2_to_fp8x2(
-                                        static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
-                                    y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
-                                    pk[e] = pc;
-                                }
-                                uint32_t w[4];
-#pragma unroll
-                                for (int pc = 0; pc < 2; ++pc) {
-                                    const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
-                                    const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
-                                    w[2 * pc] = __byte_perm(r01, r23, 0x6420);
-                                    w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
-                                }
-                                const int r8 = j * (kPieces * a.m) + q * a.m + t;
-                                *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) =
-                                    make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
+                        // Few token rows per unit: the three issuer warps split the stage's activations into
+                        // e5m2 pieces themselves (a third of the rows each) and meet on a named barrier.
+                        split_activations(a, xt, u.ntok, lane, 96);
                         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
-                        named_bar_arrive(kBarX8Full0 + stage, 96);
+                        if (*abort_flag) { ok = false; break; }
+                        named_bar_sync(kBarX8Full0 + stage, 96);
+                        if (*abort_flag) { ok = false; break; }
                     }
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
@@ -681,7 +681,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (!ok) break;
                     if (g == 0) BD_TL(2);
                     if (a.convert) {
-                        // The base issuer wrote this stage's e5m2 pieces; it arrives when they are visible.
+                        // This warp's third of the in-kernel activation split, then the three issuers meet.
+                        split_activations(a, smem + stage * a.stage_bytes + 2 * a.w_atom_bytes, u.ntok, 32 * (g + 1) + lane, 96);
+                        fence_proxy_async_smem();
                         if (*abort_flag) { ok = false; break; }
                         named_bar_sync(kBarX8Full0 + stage, 96);
                         if (*abort_flag) { ok = false; break; }

@@ -88,6 +88,13 @@ SMALL = [
     (2, 128, 256, 1024),
     (1, 200, 520, 384),
     (2, 300, 136, 512),
+    (2, 3, 64, 128),      # tile taller than N: weight rows beyond N are zero-filled by TMA
+    (1, 1, 8, 128),
+    (4, 16, 128, 128),    # m at the decode/tiled boundary, one k step
+    (20, 1, 128, 256),    # three tenant groups, the last one partly filled
+    (7, 9, 256, 256),     # m > 8: groups of four tenants
+    (12, 8, 6400, 256),   # many tiles x several groups: whole-unit work order
+    (33, 2, 1920, 384),   # five groups, whole-unit order with a partly filled last group
 ]
 
 
