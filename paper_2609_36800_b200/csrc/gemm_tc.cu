@@ -501,17 +501,19 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             __syncwarp();
         };
-        // Phase 1: weights of the first ring, before the grid dependency is resolved.
+        // Phase 1: weights of the first stages, before the grid dependency is resolved.
         // Nothing here may block: only as many stages and sign-word slots as exist are used.
+        // a.load_depth > 0 limits the stage loads in flight (default: the whole ring).
+        const int depth = (a.load_depth > 0 && a.load_depth < a.stages) ? a.load_depth : a.stages;
         SegIter ahead = it;
         int n_ahead = 0;
         {
             int u2, q0, q1, slots_used = 0;
             bool room = true;
-            while (ok && room && n_ahead < a.stages && ahead.next(u2, q0, q1)) {
+            while (ok && room && n_ahead < depth && ahead.next(u2, q0, q1)) {
                 const Unit u = unit_info(a, u2);
                 int q = q0;
-                for (; q < q1 && n_ahead < a.stages && ok; ++q, ++n_ahead) {
+                for (; q < q1 && n_ahead < depth && ok; ++q, ++n_ahead) {
                     if (q == q0 || !(q & 1)) {
                         if (slots_used == kBitSlots) { room = false; break; }
                         ++slots_used;
@@ -534,6 +536,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     issue_activations(u, p, st2);
                     if (++st2 == a.stages) st2 = 0;
                 } else {
+                    if (depth < a.stages && done >= depth) {
+                        // load `done - depth` must have landed before load `done` is queued
+                        const int prev = done - depth;
+                        ok = warp_all(wait_bar(smem_u32(&ctl->full[prev % a.stages]), (uint32_t)(prev / a.stages) & 1,
+                                               abort_flag, 9));
+                        if (!ok) break;
+                    }
                     const int st = stage;
                     ok = issue_weights(u, p, p == p0);
                     if (!ok) break;
