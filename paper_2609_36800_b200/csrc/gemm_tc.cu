@@ -45,20 +45,41 @@ __device__ long long* g_trace_ptr;
 __device__ int g_knobs;
 #ifdef BD_NO_KNOBS
 #define BD_KNOB(bit) 0
+#define BD_KNOB_LOAD do { } while (0)
 #else
-#define BD_KNOB(bit) (g_knobs & (bit))
+#define BD_KNOB_LOAD const int bd_knobs = g_knobs
+#define BD_KNOB(bit) (bd_knobs & (bit))
 #endif
-#define BD_STAMP(idx) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = clock64(); } while (0)
-// Per-role timelines of CTA 0 and CTA 77: role r's i-th stamp at trace[8192 + cta_sel*1024 + r*128 + i].
+#define BD_KNOB_G(bit) (g_knobs & (bit))
+// Stamps go to shared memory (behind the control block; the launcher adds 8.5 KB in debug builds) and are
+// copied out at teardown, so that taking one costs a clock read and a shared-memory store.
+// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[8][128]: per-role timelines (CTA 0 and 77 are kept).
+#define BD_TRACE_SETUP \
+    long long* const bd_st = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(ctl) + kSmemCtrlBytes); \
+    long long* const bd_tlb = bd_st + 32; \
+    for (int i = threadIdx.x; i < 32 + 1024; i += kThreads) bd_st[i] = 0; \
+    __syncthreads()
+#define BD_TRACE_FLUSH do { \
+    long long* gp = g_trace_ptr; \
+    if (gp) { \
+        for (int i = threadIdx.x; i < 32; i += kThreads) gp[blockIdx.x * 32 + i] = bd_st[i]; \
+        if (blockIdx.x == 0 || blockIdx.x == 77) \
+            for (int i = threadIdx.x; i < 1024; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + i] = bd_tlb[i]; \
+    } } while (0)
+#define BD_STAMP(idx) do { if (lane == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_TL_DECL int tl_idx = 0
-#define BD_TL(role) do { if (g_trace_ptr && lane == 0 && (blockIdx.x == 0 || blockIdx.x == 77) && tl_idx < 128) { g_trace_ptr[8192 + (blockIdx.x ? 1024 : 0) + (role) * 128 + tl_idx] = clock64(); ++tl_idx; } } while (0)
+#define BD_TL(role) do { if (lane == 0 && tl_idx < 128) { bd_tlb[(role) * 128 + tl_idx] = clock64(); ++tl_idx; } } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
 #define BD_ACC_END(name, t) name += clock64() - t
-#define BD_ACC_STORE(idx, name) do { if (g_trace_ptr && lane == 0) g_trace_ptr[blockIdx.x * 32 + (idx)] = name; } while (0)
+#define BD_ACC_STORE(idx, name) do { if (lane == 0) bd_st[idx] = name; } while (0)
 #else
+#define BD_TRACE_SETUP do { } while (0)
+#define BD_TRACE_FLUSH do { } while (0)
 #define BD_STAMP(idx) do { } while (0)
 #define BD_KNOB(bit) 0
+#define BD_KNOB_G(bit) 0
+#define BD_KNOB_LOAD do { } while (0)
 #define BD_TL_DECL do { } while (0)
 #define BD_TL(role) do { } while (0)
 #define BD_ACC_DECL(name) do { } while (0)
@@ -158,23 +179,24 @@ struct Unit {
     int ntok;      // output tokens of this unit (rows xrow0 .. xrow0+ntok-1)
 };
 
-__device__ __forceinline__ Unit unit_info(const GemmArgs& a, int unit) {
+template <bool kDec>
+__device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am) {
     Unit u;
     const int nt = unit / a.groups;
     const int g = unit - nt * a.groups;
     u.n0 = nt * kTileN;
-    if (a.decode) {
+    if constexpr (kDec) {
         u.tenant0 = g * a.TB;
         u.nten = min(a.TB, a.B - u.tenant0);
-        u.xrow0 = u.tenant0 * a.m;
-        u.ntok = u.nten * a.m;
+        u.xrow0 = u.tenant0 * am;
+        u.ntok = u.nten * am;
     } else {
         const int b = g / a.m_tiles;
         const int mt = g - b * a.m_tiles;
         u.tenant0 = b;
         u.nten = 1;
-        u.xrow0 = b * a.m + mt * a.tok_tile;
-        u.ntok = min(a.tok_tile, a.m - mt * a.tok_tile);
+        u.xrow0 = b * am + mt * a.tok_tile;
+        u.ntok = min(a.tok_tile, am - mt * a.tok_tile);
     }
     return u;
 }
@@ -324,12 +346,12 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
 // pairs (a bf16 value in the e5m2 range is exact in f16): p = rn_e5m2(y); y -= p; four times.
 // `xt` is the stage's X tile (two swizzled 64-k atoms), followed by the piece tile.  Thread `tid` of
 // `nthreads` takes the tasks tid, tid + nthreads, ...
-__device__ __forceinline__ void split_activations(const GemmArgs& a, uint8_t* xt, int ntok, int tid, int nthreads) {
+__device__ __forceinline__ void split_activations(const GemmArgs& a, int am, uint8_t* xt, int ntok, int tid, int nthreads) {
     uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-    const int ntasks = BD_KNOB(128) ? 0 : ntok * 8;
+    const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 8;
     for (int task = tid; task < ntasks; task += nthreads) {
         const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
-        const int j = r / a.m, t = r - j * a.m;
+        const int j = r / am, t = r - j * am;
         const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
         __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
 #pragma unroll
@@ -357,7 +379,7 @@ __device__ __forceinline__ void split_activations(const GemmArgs& a, uint8_t* xt
                 w[2 * pc] = __byte_perm(r01, r23, 0x6420);
                 w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
             }
-            const int r8 = j * (kPieces * a.m) + q * a.m + t;
+            const int r8 = j * (kPieces * am) + q * am + t;
             *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }
@@ -375,6 +397,10 @@ __device__ __forceinline__ void decode_word_e5m2(uint32_t w, uint32_t* r) {
 
 __device__ __forceinline__ void epi_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
+// kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m.
+// One instantiation per mode keeps each launched kernel's code small (the roles' loops then stay in the
+// instruction caches) and turns the schedule switches into compile-time constants.
+template <int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                         const __grid_constant__ CUtensorMap tmX8, const __grid_constant__ CUtensorMap tmBits,
@@ -389,33 +415,39 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + a.stages * a.stage_bytes + kBitSlots * a.bslot_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
+    constexpr bool kDec = kMode != 0;
+    const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
+    const bool convert = (kMode == 1 || kMode == 2) ? true : (kDec && a.convert != 0);
+    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec>(aa, un, am); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    BD_KNOB_LOAD;
+    BD_TRACE_SETUP;
     // Tiled schedule: signs need few decode threads, the epilogue many -> warps 8..11 drain accumulators
     // instead of decoding.
-    const int epi_first_warp = a.decode ? kWarpEpi0 : kWarpEpi0 - 4;
-    const int n_epi_warps = 16 - epi_first_warp;
+    constexpr int epi_first_warp = kDec ? kWarpEpi0 : kWarpEpi0 - 4;
+    constexpr int n_epi_warps = 16 - epi_first_warp;
     if (warp == 0) BD_STAMP(0);
     if (threadIdx.x == 32) {
         prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmX);
         prefetch_tensormap(&tmBits);
-        if (a.decode) prefetch_tensormap(&tmX8);
+        if (kDec) prefetch_tensormap(&tmX8);
     }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), a.decode ? 3 : 1);   // decode: three MMA issuers release a stage
+            mbar_init(smem_u32(&ctl->empty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a stage
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
-            mbar_init(smem_u32(&ctl->bempty[s]), a.decode ? 8 : 4);
+            mbar_init(smem_u32(&ctl->bempty[s]), kDec ? 8 : 4);
         }
         for (int s = 0; s < kMaxASlots; ++s) mbar_init(smem_u32(&ctl->afull[s]), 4);
         for (int s = 0; s < 2 * kMaxASlots; ++s) mbar_init(smem_u32(&ctl->aempty[s]), 1);
-        mbar_init(smem_u32(&ctl->accfull), a.decode ? 3 : 1);
-        mbar_init(smem_u32(&ctl->accempty), a.decode ? 4 : 8);
+        mbar_init(smem_u32(&ctl->accfull), kDec ? 3 : 1);
+        mbar_init(smem_u32(&ctl->accempty), kDec ? 4 : 8);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
@@ -450,7 +482,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint32_t phase = 0, bphase = 0;
         bool ok = true;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
-        const bool load_x8 = a.decode && !a.convert;
+        const bool load_x8 = kDec && !convert;
         auto issue_weights = [&](const Unit& u, int p, bool first_of_segment) -> bool {
             if (first_of_segment || !(p & 1)) {
                 BD_ACC_BEGIN(tb);
@@ -497,7 +529,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const int k0 = p * kPairK;
                 tma_load_2d(dst, &tmX, bar, k0, u.xrow0);
                 tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
-                if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, u.tenant0 * kPieces * a.m);
+                if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, u.tenant0 * kPieces * am);
             }
             __syncwarp();
         };
@@ -562,7 +594,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //   decode schedule: one item = all tenants of the unit x 64 k of e5m2 signs (16 columns per
         //                    tenant, 2 MMAs of K=32 per tenant)
         const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
-        const uint32_t idesc_delta = a.decode ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
+        const uint32_t idesc_delta = kDec ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
                                               : make_idesc_bf16(kTileN, (uint32_t)a.Nd);
         // Descriptor of a tile = descriptor of address 0 plus (address >> 4): addresses stay below
         // 256 KiB, so the sum never carries out of the 14-bit start-address field.
@@ -604,13 +636,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
-                if (a.decode) {
+                if constexpr (kDec) {
                     // Delta MMAs are issued by the two delta-issuer warps.
                     uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
-                    if (a.convert) {
+                    if (convert) {
                         // Few token rows per unit: the three issuer warps split the stage's activations into
                         // e5m2 pieces themselves (a third of the rows each) and meet on a named barrier.
-                        split_activations(a, xt, u.ntok, lane, 96);
+                        split_activations(a, am, xt, u.ntok, lane, 96);
                         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
                         if (*abort_flag) { ok = false; break; }
                         named_bar_sync(kBarX8Full0 + stage, 96);
@@ -654,7 +686,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             BD_STAMP(6);
         }
-        if (a.decode && a.convert && *abort_flag) {
+        if (kDec && convert && *abort_flag) {
             // Abandoned wait somewhere: the delta issuers may be blocked on a piece barrier.
             __syncwarp();
             for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
@@ -668,12 +700,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //  * per 64-k half waits, on a named barrier, for the group's decode warps to have filled the
         //    operand buffer in tensor memory, issues that half's MMAs and commits the buffer's release.
         // Nothing else writes those tenants' accumulators, so their summation order is fixed.
-        if (a.decode) {
+        if constexpr (kDec) {
             const int g = warp - kWarpDelta0;
             const uint32_t idesc_delta = make_idesc_e5m2(kTileN, (uint32_t)a.Nd);
             const uint64_t desc0 = make_smem_desc_sw128(0);
             const uint32_t x_atom16 = a.x_atom_bytes >> 4;
-            const uint32_t ten_rows16 = (uint32_t)(kPieces * a.m) * 8u;   // rows per tenant x 128 B >> 4
+            const uint32_t ten_rows16 = (uint32_t)(kPieces * am) * 8u;   // rows per tenant x 128 B >> 4
             const uint32_t amask = (uint32_t)a.a_slots - 1;
             const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
             int stage = 0;
@@ -689,9 +721,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
                     if (!ok) break;
                     if (g == 0) BD_TL(2);
-                    if (a.convert) {
+                    if (convert) {
                         // This warp's third of the in-kernel activation split, then the three issuers meet.
-                        split_activations(a, smem + stage * a.stage_bytes + 2 * a.w_atom_bytes, u.ntok, 32 * (g + 1) + lane, 96);
+                        split_activations(a, am, smem + stage * a.stage_bytes + 2 * a.w_atom_bytes, u.ntok, 32 * (g + 1) + lane, 96);
                         fence_proxy_async_smem();
                         if (*abort_flag) { ok = false; break; }
                         named_bar_sync(kBarX8Full0 + stage, 96);
@@ -748,7 +780,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 accphase ^= 1;
                 (void)ashift;
             }
-            if (a.convert && *abort_flag) {
+            if (convert && *abort_flag) {
                 // Leave no other issuer blocked on a piece barrier this warp would have joined.
                 __syncwarp();
                 for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
@@ -778,7 +810,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (item == 0 && warp == kWarpDecode0) BD_STAMP(14);
                 }
                 const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
-                if (a.decode) {
+                if constexpr (kDec) {
                     // Warp (grp, quad) decodes, for its 32 rows, the tenants j = grp, grp+2, ... (64 k = two
                     // sign words each) into its group's ring of operand buffers, then arrives on the
                     // buffer's named barrier, on which the group's delta issuer waits.
@@ -873,7 +905,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
             }
         }
-        if (a.decode && *abort_flag) {
+        if (kDec && *abort_flag) {
             // A wait was abandoned somewhere in the CTA.  The group's delta issuer may be blocked on one
             // of the named barriers (they have no time-out): arrive on all of them so that it wakes up,
             // sees the abort flag and leaves.
@@ -893,6 +925,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
         uint32_t accphase = 0;
         bool ok = true;
+        BD_TL_DECL;
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
@@ -906,15 +939,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
-            if (warp == epi_first_warp) BD_STAMP(7);
+            if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
-            if (a.decode) {
-                switch (a.m) {
-                    case 1: epilogue_decode<1>(a, u, lane_taddr, out); break;
-                    case 2: epilogue_decode<2>(a, u, lane_taddr, out); break;
-                    case 3: epilogue_decode<3>(a, u, lane_taddr, out); break;
-                    case 4: epilogue_decode<4>(a, u, lane_taddr, out); break;
+            if constexpr (kMode >= 1 && kMode <= 4) {
+                epilogue_decode<kMode>(a, u, lane_taddr, out);
+            } else if constexpr (kMode == 5) {
+                switch (am) {
                     case 5: epilogue_decode<5>(a, u, lane_taddr, out); break;
                     case 6: epilogue_decode<6>(a, u, lane_taddr, out); break;
                     case 7: epilogue_decode<7>(a, u, lane_taddr, out); break;
@@ -934,7 +965,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
-            if (warp == epi_first_warp) BD_STAMP(8);
+            if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
 
             if (!whole) {
                 // This tile is cut across CTAs: publish the partial, count arrivals, and let
@@ -949,7 +980,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);
-                if (warp == epi_first_warp) BD_STAMP(9);
+                if (warp == epi_first_warp) { BD_STAMP(9); BD_TL(4); }
                 if (ctl->is_last) {
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
@@ -961,7 +992,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (etid == 0) a.counters[unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
-                if (warp == epi_first_warp) BD_STAMP(10);
+                if (warp == epi_first_warp) { BD_STAMP(10); BD_TL(4); }
             }
         }
     }
@@ -984,6 +1015,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         tmem_dealloc(tmem_base, kTmemCols);
         BD_STAMP(12);
     }
+    BD_TRACE_FLUSH;
 }
 
 #ifdef BD_TRACE
@@ -998,26 +1030,34 @@ extern "C" int bitdelta_debug_set_knobs(int knobs) {
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream) {
-    static int attr_device = -1;
+    const int mode = !args.decode ? 0 : (args.m <= 4 ? args.m : 5);
+    using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmArgs);
+    static const KernelFn kernels[6] = {bitdelta_gemm_tc_kernel<0>, bitdelta_gemm_tc_kernel<1>, bitdelta_gemm_tc_kernel<2>,
+                                        bitdelta_gemm_tc_kernel<3>, bitdelta_gemm_tc_kernel<4>, bitdelta_gemm_tc_kernel<5>};
+    static int attr_device[6] = {-1, -1, -1, -1, -1, -1};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (attr_device != dev) {
-        e = cudaFuncSetAttribute(bitdelta_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (attr_device[mode] != dev) {
+        e = cudaFuncSetAttribute(kernels[mode], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (e != cudaSuccess) return e;
-        attr_device = dev;
+        attr_device[mode] = dev;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
+#ifdef BD_TRACE
+    cfg.dynamicSmemBytes = smem_bytes + 8704;   // room for the stamps behind the control block
+#else
     cfg.dynamicSmemBytes = smem_bytes;
+#endif
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = early_start ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, bitdelta_gemm_tc_kernel, tmW, tmX, tmX8, tmBits, args);
+    return cudaLaunchKernelEx(&cfg, kernels[mode], tmW, tmX, tmX8, tmBits, args);
 }
 
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {
