@@ -156,16 +156,6 @@ int whole_override() {
     return v;
 }
 
-// BITDELTA_DEPTH=<n> limits the stage loads in flight (experiments).
-int depth_override() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("BITDELTA_DEPTH");
-        v = e ? atoi(e) : 0;
-    }
-    return v;
-}
-
 // BITDELTA_EARLY_START=0 launches the GEMM kernel fully serialised behind its predecessor
 // (for experiments; the default lets it begin its weight prefetch early).
 bool early_start_enabled() {
@@ -210,7 +200,7 @@ int bitdelta_unpack(const uint32_t* bits, int8_t* S, int B, int N, int K, void* 
 size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K) {
     if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return 0;
     if ((K % 128) != 0) return 256;   // CUDA-core path: no scratch needed, keep the pointer non-NULL
-    bd::Plan p = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override(), depth_override());
+    bd::Plan p = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override());
     if (!p.ok) return 0;
     return p.ws_bytes;
 }
@@ -254,7 +244,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
         return BITDELTA_OK;
     }
 
-    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), depth_override());
+    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
     if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
@@ -325,7 +315,7 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
         cudaMemcpyAsync(dAlpha, alpha_host, ab, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
     // Only the arrival counters at the start of the workspace have to be clear.
-    bd::Plan plan = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override(), depth_override());
+    bd::Plan plan = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override());
     const size_t header = plan.ok ? plan.ws_header_bytes : (ws < 256 ? ws : 256);
     if (cudaMemsetAsync(dWs, 0, header, stream) != cudaSuccess) return BITDELTA_ERR_CUDA;
     int st = bitdelta_gemm(dX, dW, static_cast<const uint32_t*>(dBits), static_cast<const float*>(dAlpha), dY, B, m,
@@ -371,7 +361,7 @@ int bitdelta_gemm_noalloc(const void* X, const void* W_base, const uint32_t* bit
     // The arrival counters at the start of the scratch have to be zero when the kernel begins; a call
     // that was cut short could have left them otherwise.
     if ((K % 128) == 0) {
-        bd::Plan plan = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), depth_override());
+        bd::Plan plan = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override());
         if (!plan.ok) return BITDELTA_ERR_SHAPE;
         if (cudaMemsetAsync(scratch, 0, plan.ws_header_bytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
             return BITDELTA_ERR_CUDA;

@@ -32,7 +32,6 @@ constexpr int kWarpMma = 1;
 constexpr int kWarpTmem = 2;
 constexpr int kWarpDelta0 = 2;     // decode schedule: warps 2..3 issue the delta MMAs of decode group 0 / 1
 constexpr int kBarAFull0 = 2;      // named barriers 2..9 : decode group g, buffer b -> id 2 + g*4 + b
-constexpr int kBarX8Full0 = 10;    // named barriers 10..13: e5m2 pieces of stage s written (in-kernel split)
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
 
@@ -67,8 +66,10 @@ __device__ int g_knobs;
             for (int i = threadIdx.x; i < 1024; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + i] = bd_tlb[i]; \
     } } while (0)
 #define BD_STAMP(idx) do { if (lane == 0) bd_st[idx] = clock64(); } while (0)
+#define BD_STAMP_ONCE(idx) do { if (lane == 0 && bd_st[idx] == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_TL_DECL int tl_idx = 0
 #define BD_TL(role) do { if (lane == 0 && tl_idx < 128) { bd_tlb[(role) * 128 + tl_idx] = clock64(); ++tl_idx; } } while (0)
+#define BD_TL2(role) do { if (lane == 0 && tl_idx2 < 128) { bd_tlb[(role) * 128 + tl_idx2] = clock64(); ++tl_idx2; } } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
 #define BD_ACC_END(name, t) name += clock64() - t
@@ -77,6 +78,7 @@ __device__ int g_knobs;
 #define BD_TRACE_SETUP do { } while (0)
 #define BD_TRACE_FLUSH do { } while (0)
 #define BD_STAMP(idx) do { } while (0)
+#define BD_STAMP_ONCE(idx) do { } while (0)
 #define BD_KNOB(bit) 0
 #define BD_KNOB_G(bit) 0
 #define BD_KNOB_LOAD do { } while (0)
@@ -99,6 +101,8 @@ struct Ctl {
     uint64_t aempty[2 * kMaxASlots];   // operand buffer free again (tcgen05.commit); decode: [group][buffer]
     uint64_t accfull;
     uint64_t accempty;
+    uint64_t x8full[kMaxStages];       // decode, in-kernel split: the stage's e5m2 pieces are written (96 arrivals)
+    uint64_t depready;                 // the grid this launch depends on has completed (activations may be read)
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t is_last;
@@ -106,10 +110,10 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= kSmemCtrlBytes, "control block too large");
 
 // Bounded wait on an mbarrier phase.  Returns false if the wait was abandoned
-// (limit reached here or in another thread of the CTA).
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
-    if (mbar_try_wait(bar, parity)) return true;
-    // Slow path: poll, and every 64 polls look at the abort flag and the SM cycle counter
+// (limit reached here or in another thread of the CTA).  The slow path is kept out of line: it is
+// instantiated at some twenty call sites and would otherwise dominate the kernel's code size.
+__device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+    // Poll, and every 64 polls look at the abort flag and the SM cycle counter
     // (cheap to read; the limit is ~2 s at 2 GHz, longer at lower clocks).
     const long long t0 = clock64();
 #pragma unroll 1
@@ -126,47 +130,55 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         }
     }
 }
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_bar_slow(bar, parity, abort_flag, site);
+}
 
-// Same contract, for the warp on the critical path (the MMA issuer): spins on the non-suspending
-// test so that it reacts within a few cycles of the phase completing, instead of paying the wake-up
-// latency of a suspended try_wait on every hand-over.
-__device__ __forceinline__ bool spin_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
-    if (mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-#pragma unroll 1
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i) {
-            if (mbar_test_wait(bar, parity)) return true;
-        }
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *abort_flag = 1;
-            if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
-            return false;
-        }
-    }
+// Work split.  The T = q*G + r items (T < 2^30) are cut evenly across the G CTAs: CTA b owns
+// [b*q + min(b, r), ...), i.e. the first r CTAs take q+1 items.  32-bit arithmetic only: 64-bit
+// divisions cost several hundred cycles each and sit on the start-up and tail paths.
+__device__ __forceinline__ int cta_first_item(const GemmArgs& a, int b) { return b * a.q + min(b, a.r); }
+__device__ __forceinline__ int cta_of_item(const GemmArgs& a, int i) {
+    const int big = a.r * (a.q + 1);
+    return (i < big) ? (int)((unsigned)i / (unsigned)(a.q + 1)) : a.r + (int)((unsigned)(i - big) / (unsigned)a.q);
 }
 
 // Walks the k-pair items [lo, hi) of this CTA as segments (unit, p0, p1).
 struct SegIter {
-    long long cur, hi;
+    int cur, hi;
     int P;
     int stride;   // 0: the CTA owns the items [cur, hi); > 0: whole units cur/P, cur/P + stride, ... (see plan.h)
     __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
         if (cur >= hi) return false;
-        unit = (int)(cur / P);
+        unit = (int)((unsigned)cur / (unsigned)P);
         if (stride > 0) {
             p0 = 0;
             p1 = P;
-            cur += (long long)stride * P;
+            cur += stride * P;
             return true;
         }
-        p0 = (int)(cur - (long long)unit * P);
-        long long rem = hi - cur;
-        int len = (rem < (long long)(P - p0)) ? (int)rem : (P - p0);
+        p0 = cur - unit * P;
+        const int rem = hi - cur;
+        const int len = (rem < P - p0) ? rem : (P - p0);
         p1 = p0 + len;
         cur += len;
+        return true;
+    }
+};
+
+// The same walk, one (unit, k-pair) item at a time.
+struct ItemIter {
+    SegIter seg;
+    int unit, p, p1;
+    bool first;   // first item of its segment
+    __device__ __forceinline__ explicit ItemIter(const SegIter& s) : seg(s), unit(0), p(0), p1(0), first(false) {}
+    __device__ __forceinline__ bool next() {
+        if (p + 1 < p1) { ++p; first = false; return true; }
+        int p0;
+        if (!seg.next(unit, p0, p1)) { p = 0; p1 = 0; return false; }
+        p = p0;
+        first = true;
         return true;
     }
 };
@@ -417,7 +429,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
     constexpr bool kDec = kMode != 0;
     const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
-    const bool convert = (kMode == 1 || kMode == 2) ? true : (kDec && a.convert != 0);
+    const bool convert = kDec && a.convert != 0;
     auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec>(aa, un, am); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -435,10 +447,52 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         if (kDec) prefetch_tensormap(&tmX8);
     }
 
+    // Work: either an even share of the flat item list, or (whole-unit order) units b, b+grid, ...
+    const int lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
+    const int hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
+    SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
+    int unit, p0, p1;
+    const bool load_x8 = kDec && !convert;
+
+    // Queues the weight loads of one item: its W_base tile into `stage` and, if `with_bits`, the sign words
+    // of its k-pair into sign-word slot `bslot`.  One thread.  The stage's activations follow separately.
+    auto issue_weights_raw = [&](const Unit& u, int p, int stage, int bslot, bool with_bits) {
+        // W_base first: the stage's MMAs need it together with the activations, and the first sign-word
+        // load of a tile is slow (it pulls whole 128-byte lines, i.e. the signs of 1024 k, out of DRAM).
+        const uint32_t bar = smem_u32(&ctl->full[stage]);
+        const uint32_t dst = stages_addr + stage * a.stage_bytes;
+        uint32_t tx = load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes;
+        if (BD_KNOB(16)) tx -= 2 * a.w_atom_bytes;
+        if (BD_KNOB(32)) tx -= 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0);
+        if (tx) mbar_arrive_expect_tx(bar, tx); else mbar_arrive(bar);
+        const int k0 = p * kPairK;
+        if (!BD_KNOB(16)) {
+            tma_load_2d(dst, &tmW, bar, k0, u.n0);
+            tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+        }
+        if (with_bits) {
+            const uint32_t bbar = smem_u32(&ctl->bfull[bslot]);
+            if (BD_KNOB(8)) {
+                mbar_arrive(bbar);
+            } else {
+                mbar_arrive_expect_tx(bbar, a.bslot_bytes);
+                tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (p >> 1) * 8, u.n0, u.tenant0);
+            }
+        }
+    };
+
+    // One issuer thread's share (tasks tid, tid + 96, ...) of the in-kernel activation split of stage `st`.
+    auto do_split = [&](int st, int ntok, int tid) {
+        split_activations(a, am, smem + st * a.stage_bytes + 2 * a.w_atom_bytes, ntok, tid, 96);
+        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+        mbar_arrive(smem_u32(&ctl->x8full[st]));
+    };
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a stage
+            mbar_init(smem_u32(&ctl->x8full[s]), 96);
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
@@ -448,9 +502,17 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         for (int s = 0; s < 2 * kMaxASlots; ++s) mbar_init(smem_u32(&ctl->aempty[s]), 1);
         mbar_init(smem_u32(&ctl->accfull), kDec ? 3 : 1);
         mbar_init(smem_u32(&ctl->accempty), kDec ? 4 : 8);
+        mbar_init(smem_u32(&ctl->depready), 1);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
+        // The first item's weights are requested right here, before the rest of the CTA is set up:
+        // every cycle until the first load is queued is added to the launch's latency.
+        if (lo < hi) {
+            const int unit0 = (int)((unsigned)lo / (unsigned)a.P);
+            issue_weights_raw(unit_info(a, unit0), a.whole_units ? 0 : lo - unit0 * a.P, 0, 0, true);
+        }
+        BD_STAMP(2);
     }
     if (warp == kWarpTmem) {
         tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -466,122 +528,87 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     // this grid reads or writes.
     if (threadIdx.x == 0) grid_launch_dependents();
 
-    // Work: either an even share of the flat item list, or (whole-unit order) units b, b+grid, ...
-    const long long lo = a.whole_units ? (long long)blockIdx.x * a.P : (long long)blockIdx.x * a.T / gridDim.x;
-    const long long hi = a.whole_units ? a.T : (long long)(blockIdx.x + 1) * a.T / gridDim.x;
-    SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
-    int unit, p0, p1;
-
     if (warp == kWarpProducer) {
         // ------------------------------------------------------------ TMA producer
         // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
         // Weights (W_base, sign words) never depend on the kernel queued before this one, the
-        // activations may: with an early start the first ring of weight loads is issued, then the
-        // grid dependency is awaited, then the activation loads follow.
-        int stage = 0, bslot = 0;
+        // activations may.  Weight loads therefore run ahead as far as the rings allow; the activations
+        // of every item whose weights are queued follow as soon as the grid dependency is resolved
+        // (warp 1 waits for it and completes `depready`), so that they are not queued behind a whole
+        // ring of weight traffic when the dependency is already met at launch.
+        ItemIter wi(it), xi(it);
+        int n_w = 0, n_x = 0;            // items whose weights / activations are queued
+        int stage = 0, stage_x = 0, bslot = 0, slots_used = 0;
         uint32_t phase = 0, bphase = 0;
-        bool ok = true;
+        bool ok = true, dep_ok = false;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
-        const bool load_x8 = kDec && !convert;
-        auto issue_weights = [&](const Unit& u, int p, bool first_of_segment) -> bool {
-            if (first_of_segment || !(p & 1)) {
-                BD_ACC_BEGIN(tb);
-                bool good = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
-                BD_ACC_END(w_bempty, tb);
-                if (!good) return false;
-                if (elect_one()) {
-                    const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
-                    if (BD_KNOB(8)) {
-                        mbar_arrive(bar);
-                    } else {
-                        mbar_arrive_expect_tx(bar, a.bslot_bytes);
-                        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
-                    }
+        Unit uw{}, ux{};
+        bool more_w = wi.next();
+        if (more_w) {
+            // queued by thread 0 in the prologue: stage 0, sign-word slot 0
+            n_w = 1; slots_used = 1; bslot = 1 % kBitSlots; bphase = (kBitSlots == 1) ? 1u : 0u;
+            stage = 1 % a.stages; phase = (a.stages == 1) ? 1u : 0u;
+            BD_TL(0);
+            uw = unit_info(a, wi.unit);
+            more_w = wi.next();
+        }
+        const uint32_t depbar = smem_u32(&ctl->depready);
+        for (;;) {
+            const bool need_slot = more_w && (wi.first || !(wi.p & 1));
+            if (!dep_ok) {
+                // Without the activations no stage is ever released: only the first ring may be filled blind.
+                const bool must = !more_w || n_w >= a.stages || (need_slot && slots_used >= kBitSlots);
+                if (must) {
+                    ok = warp_all(wait_bar(depbar, 0, abort_flag, 10));
+                    if (!ok) break;
+                    dep_ok = true;
+                } else {
+                    dep_ok = warp_all(mbar_test_wait(depbar, 0));
                 }
-                __syncwarp();
-                if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+            }
+            if (dep_ok) {
+                while (n_x < n_w) {
+                    xi.next();
+                    if (xi.first) ux = unit_info(a, xi.unit);
+                    if (!BD_KNOB(32) && elect_one()) {
+                        const uint32_t bar = smem_u32(&ctl->full[stage_x]);
+                        const uint32_t dst = stages_addr + stage_x * a.stage_bytes + 2 * a.w_atom_bytes;
+                        const int k0 = xi.p * kPairK;
+                        tma_load_2d(dst, &tmX, bar, k0, ux.xrow0);
+                        tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, ux.xrow0);
+                        if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, ux.tenant0 * kPieces * am);
+                    }
+                    __syncwarp();
+                    BD_STAMP_ONCE(29);
+                    ++n_x;
+                    if (++stage_x == a.stages) stage_x = 0;
+                }
+            }
+            if (!more_w) {
+                if (n_x == n_w) break;
+                continue;
+            }
+            if (wi.first) uw = unit_info(a, wi.unit);
+            if (need_slot) {
+                BD_ACC_BEGIN(tb);
+                ok = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
+                BD_ACC_END(w_bempty, tb);
+                if (!ok) break;
             }
             BD_ACC_BEGIN(te);
-            bool good = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
+            ok = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
             BD_ACC_END(w_empty, te);
-            if (!good) return false;
-            if (elect_one()) {
-                const uint32_t bar = smem_u32(&ctl->full[stage]);
-                const uint32_t dst = stages_addr + stage * a.stage_bytes;
-                uint32_t tx = load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes;
-                if (BD_KNOB(16)) tx -= 2 * a.w_atom_bytes;
-                if (BD_KNOB(32)) tx -= 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0);
-                if (tx) mbar_arrive_expect_tx(bar, tx); else mbar_arrive(bar);
-                const int k0 = p * kPairK;
-                if (!BD_KNOB(16)) {
-                    tma_load_2d(dst, &tmW, bar, k0, u.n0);
-                    tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
-                }
-            }
+            if (!ok) break;
+            if (elect_one()) issue_weights_raw(uw, wi.p, stage, bslot, need_slot);
             __syncwarp();
             BD_TL(0);
-            return true;
-        };
-        auto issue_activations = [&](const Unit& u, int p, int st) {
-            if (!BD_KNOB(32) && elect_one()) {
-                const uint32_t bar = smem_u32(&ctl->full[st]);
-                const uint32_t dst = stages_addr + st * a.stage_bytes + 2 * a.w_atom_bytes;
-                const int k0 = p * kPairK;
-                tma_load_2d(dst, &tmX, bar, k0, u.xrow0);
-                tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, u.xrow0);
-                if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, u.tenant0 * kPieces * am);
+            if (need_slot) {
+                ++slots_used;
+                if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
             }
-            __syncwarp();
-        };
-        // Phase 1: weights of the first stages, before the grid dependency is resolved.
-        // Nothing here may block: only as many stages and sign-word slots as exist are used.
-        // a.load_depth > 0 limits the stage loads in flight (default: the whole ring).
-        const int depth = (a.load_depth > 0 && a.load_depth < a.stages) ? a.load_depth : a.stages;
-        SegIter ahead = it;
-        int n_ahead = 0;
-        {
-            int u2, q0, q1, slots_used = 0;
-            bool room = true;
-            while (ok && room && n_ahead < depth && ahead.next(u2, q0, q1)) {
-                const Unit u = unit_info(a, u2);
-                int q = q0;
-                for (; q < q1 && n_ahead < depth && ok; ++q, ++n_ahead) {
-                    if (q == q0 || !(q & 1)) {
-                        if (slots_used == kBitSlots) { room = false; break; }
-                        ++slots_used;
-                    }
-                    ok = issue_weights(u, q, q == q0);
-                    if (!ok) break;
-                    if (n_ahead == 0) BD_STAMP(2);
-                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
-                }
-                if (q < q1) break;   // ring full in the middle of a segment
-            }
-        }
-        grid_dependency_wait();
-        // Phase 2: the whole schedule; the first n_ahead stages only still need their activations.
-        int done = 0, st2 = 0;
-        while (ok && it.next(unit, p0, p1)) {
-            const Unit u = unit_info(a, unit);
-            for (int p = p0; p < p1 && ok; ++p, ++done) {
-                if (done < n_ahead) {
-                    issue_activations(u, p, st2);
-                    if (++st2 == a.stages) st2 = 0;
-                } else {
-                    if (depth < a.stages && done >= depth) {
-                        // load `done - depth` must have landed before load `done` is queued
-                        const int prev = done - depth;
-                        ok = warp_all(wait_bar(smem_u32(&ctl->full[prev % a.stages]), (uint32_t)(prev / a.stages) & 1,
-                                               abort_flag, 9));
-                        if (!ok) break;
-                    }
-                    const int st = stage;
-                    ok = issue_weights(u, p, p == p0);
-                    if (!ok) break;
-                    issue_activations(u, p, st);
-                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
-                }
-            }
+            ++n_w;
+            if (++stage == a.stages) { stage = 0; phase ^= 1; }
+            more_w = wi.next();
         }
         BD_STAMP(3);
         BD_ACC_STORE(19, w_empty); BD_ACC_STORE(20, w_bempty);
@@ -605,7 +632,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0;
         uint32_t phase = 0, accphase = 0, item = 0;
         bool ok = true;
+        bool split_done = false;   // this warp's share of the current stage's activation split was done ahead
         BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id); BD_TL_DECL;
+        // This warp also tells the producer when the grid this launch depends on has completed.
+        BD_STAMP(30);
+        grid_dependency_wait();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));
+        BD_STAMP(31);
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             BD_ACC_BEGIN(ta);
@@ -614,10 +647,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
-                BD_ACC_BEGIN(tf);
-                ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
-                BD_ACC_END(w_full, tf);
-                if (!ok) break;
+                if (!split_done) {
+                    BD_ACC_BEGIN(tf);
+                    ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                    BD_ACC_END(w_full, tf);
+                    if (!ok) break;
+                }
                 if (item == 0) BD_STAMP(4);
                 BD_TL(1);
                 const uint32_t wbase = stages_addr + stage * a.stage_bytes;
@@ -637,16 +672,21 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if constexpr (kDec) {
-                    // Delta MMAs are issued by the two delta-issuer warps.
-                    uint8_t* xt = smem + stage * a.stage_bytes + 2 * a.w_atom_bytes;
+                    // Delta MMAs are issued by the two delta-issuer warps.  With few token rows per unit the
+                    // three issuer warps split each stage's activations into e5m2 pieces themselves (a third of
+                    // the tasks each, completion counted on x8full[stage]); each warp does its share of the
+                    // NEXT stage as soon as that stage has landed, so the split stays off the critical path.
                     if (convert) {
-                        // Few token rows per unit: the three issuer warps split the stage's activations into
-                        // e5m2 pieces themselves (a third of the rows each) and meet on a named barrier.
-                        split_activations(a, am, xt, u.ntok, lane, 96);
-                        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
-                        if (*abort_flag) { ok = false; break; }
-                        named_bar_sync(kBarX8Full0 + stage, 96);
-                        if (*abort_flag) { ok = false; break; }
+                        if (!split_done) do_split(stage, u.ntok, lane);
+                        split_done = false;
+                        if (p + 1 < p1) {
+                            const int ns = (stage + 1 == a.stages) ? 0 : stage + 1;
+                            const uint32_t nph = (stage + 1 == a.stages) ? phase ^ 1 : phase;
+                            if (warp_all(mbar_test_wait(smem_u32(&ctl->full[ns]), nph))) {
+                                do_split(ns, u.ntok, lane);
+                                split_done = true;
+                            }
+                        }
                     }
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
@@ -686,11 +726,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             BD_STAMP(6);
         }
-        if (kDec && convert && *abort_flag) {
-            // Abandoned wait somewhere: the delta issuers may be blocked on a piece barrier.
-            __syncwarp();
-            for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
-        }
         BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
     } else if (warp >= kWarpDelta0 && warp < kWarpDelta0 + 2) {
         // ------------------------------------------------- delta issuers (decode schedule)
@@ -711,6 +746,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             int stage = 0;
             uint32_t phase = 0, accphase = 0, item = 0;
             bool ok = true;
+            bool split_done = false;   // as in the base issuer
             BD_TL_DECL;
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
@@ -718,16 +754,17 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (!ok) break;
                 tc_fence_after();
                 for (int p = p0; p < p1 && ok; ++p) {
-                    ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
-                    if (!ok) break;
+                    if (!split_done) {
+                        ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                        if (!ok) break;
+                    }
                     if (g == 0) BD_TL(2);
                     if (convert) {
-                        // This warp's third of the in-kernel activation split, then the three issuers meet.
-                        split_activations(a, am, smem + stage * a.stage_bytes + 2 * a.w_atom_bytes, u.ntok, 32 * (g + 1) + lane, 96);
-                        fence_proxy_async_smem();
-                        if (*abort_flag) { ok = false; break; }
-                        named_bar_sync(kBarX8Full0 + stage, 96);
-                        if (*abort_flag) { ok = false; break; }
+                        if (!split_done) do_split(stage, u.ntok, 32 * (g + 1) + lane);
+                        split_done = false;
+                        // all three shares of this stage
+                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 11));
+                        if (!ok) break;
                     }
                     const uint64_t x8desc = desc0 + ((stages_addr + stage * a.stage_bytes + 2 * a.w_atom_bytes) >> 4) +
                                             2 * x_atom16;
@@ -768,6 +805,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                             tc_commit(smem_u32(&ctl->aempty[g * kMaxASlots + slot]));
                         }
                         __syncwarp();
+                        if (half == 0 && convert && p + 1 < p1) {
+                            // idle until the decode warps hand over the next buffer: split the next stage now
+                            const int ns = (stage + 1 == a.stages) ? 0 : stage + 1;
+                            const uint32_t nph = (stage + 1 == a.stages) ? phase ^ 1 : phase;
+                            if (warp_all(mbar_test_wait(smem_u32(&ctl->full[ns]), nph))) {
+                                do_split(ns, u.ntok, 32 * (g + 1) + lane);
+                                split_done = true;
+                            }
+                        }
                     }
                     if (!ok) break;
                     if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
@@ -779,11 +825,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 accphase ^= 1;
                 (void)ashift;
-            }
-            if (convert && *abort_flag) {
-                // Leave no other issuer blocked on a piece barrier this warp would have joined.
-                __syncwarp();
-                for (int st = 0; st < 4; ++st) named_bar_arrive(kBarX8Full0 + st, 96);
             }
         }
     } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {
@@ -798,7 +839,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int bslot = 0;
         uint32_t bphase = 0, item = 0;
         bool ok = true;
+        // shapes with a straight-line decode loop (two operand buffers per group in both)
+        const bool fast8 = kDec && a.TB == 8 && a.halves == 2 && a.a_slots == 2;
+        const bool fast4 = kDec && a.TB == 4 && a.halves == 1 && a.a_slots == 2;
+        const uint32_t aempty_g = smem_u32(&ctl->aempty[grp * kMaxASlots]);
+        const uint32_t tbuf_g = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots) * (uint32_t)a.aslot_cols;
         BD_ACC_DECL(w_bfull); BD_ACC_DECL(w_aempty); BD_ACC_DECL(w_work); BD_TL_DECL;
+#ifdef BD_TRACE
+        int tl_idx2 = 0;
+#endif
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             for (int p = p0; p < p1 && ok; ++p) {
@@ -814,6 +863,74 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // Warp (grp, quad) decodes, for its 32 rows, the tenants j = grp, grp+2, ... (64 k = two
                     // sign words each) into its group's ring of operand buffers, then arrives on the
                     // buffer's named barrier, on which the group's delta issuer waits.
+                    //
+                    // Full units of the two common shapes run as straight-line code: with two warps per
+                    // scheduler nothing hides a warp's own bookkeeping, so every dependent instruction that
+                    // is not decode work costs its full latency.
+                    if (fast8 && u.nten == 8) {
+                        // eight tenants, two 64-k hand-overs per stage into buffers 0 and 1 of the group
+                        const uint8_t* src = bsl + (grp * kTileN + row) * 32;
+                        uint4 wq[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) wq[i] = *reinterpret_cast<const uint4*>(src + i * (2 * kTileN * 32));
+                        const uint32_t par = ((item >> 1) & 1) ^ 1;
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            BD_ACC_BEGIN(tq);
+                            ok = wait_bar(aempty_g + half * 8, par, abort_flag, 7);
+                            BD_ACC_END(w_aempty, tq);
+                            if (!ok) break;
+                            tc_fence_after();
+                            if (warp == kWarpDecode0) BD_TL(3);
+                            BD_ACC_BEGIN(tw);
+                            const uint32_t tbuf = tbuf_g + (uint32_t)half * (uint32_t)a.aslot_cols;
+#pragma unroll
+                            for (int i = 0; i < 4; i += 2) {
+                                uint32_t r[32];
+                                decode_word_e5m2(half ? wq[i].z : wq[i].x, r);
+                                decode_word_e5m2(half ? wq[i].w : wq[i].y, r + 8);
+                                decode_word_e5m2(half ? wq[i + 1].z : wq[i + 1].x, r + 16);
+                                decode_word_e5m2(half ? wq[i + 1].w : wq[i + 1].y, r + 24);
+                                tmem_st32(tbuf + (uint32_t)i * 16, r);
+                            }
+                            if (warp == kWarpDecode0) BD_TL(3);
+                            tc_wait_st();
+                            if (warp == kWarpDecode0) BD_TL(3);
+                            tc_fence_before();
+                            named_bar_arrive(kBarAFull0 + grp * 4 + half, 160);
+                            BD_ACC_END(w_work, tw);
+                            if (warp == kWarpDecode0) BD_TL(3);
+                        }
+                        item += 2;
+                    } else if (fast4 && u.nten == 4) {
+                        // four tenants, one 128-k hand-over per stage, buffers alternate
+                        const uint8_t* src = bsl + (grp * kTileN + row) * 32;
+                        uint4 wq[2];
+                        wq[0] = *reinterpret_cast<const uint4*>(src);
+                        wq[1] = *reinterpret_cast<const uint4*>(src + 2 * kTileN * 32);
+                        const uint32_t slot = item & 1;
+                        BD_ACC_BEGIN(tq);
+                        ok = wait_bar(aempty_g + slot * 8, ((item >> 1) & 1) ^ 1, abort_flag, 7);
+                        BD_ACC_END(w_aempty, tq);
+                        if (!ok) break;
+                        tc_fence_after();
+                        BD_ACC_BEGIN(tw);
+                        const uint32_t tbuf = tbuf_g + slot * (uint32_t)a.aslot_cols;
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            uint32_t r[32];
+                            decode_word_e5m2(wq[i].x, r);
+                            decode_word_e5m2(wq[i].y, r + 8);
+                            decode_word_e5m2(wq[i].z, r + 16);
+                            decode_word_e5m2(wq[i].w, r + 24);
+                            tmem_st32(tbuf + (uint32_t)i * 32, r);
+                        }
+                        tc_wait_st();
+                        tc_fence_before();
+                        named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
+                        BD_ACC_END(w_work, tw);
+                        item += 1;
+                    } else
                     for (int half = 0; half < a.halves && ok; ++half, ++item) {
                         const uint32_t slot = item & amask;
                         const uint32_t use = item >> ashift;
@@ -845,9 +962,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                                 const int j = grp + 2 * i;
                                 if (j < u.nten) w[i] = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
                             }
+#ifdef BD_TRACE
+                            if (warp == kWarpDecode0) { asm volatile("" :: "r"(w[0].x), "r"(w[1].x), "r"(w[2].x), "r"(w[3].x)); BD_TL2(6); }
+#endif
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int j = grp + 2 * i;
+#ifdef BD_TRACE
+                                if (warp == kWarpDecode0 && i > 0) BD_TL2(6);
+#endif
                                 if (j < u.nten) {
                                     uint32_t r[16];
                                     if (BD_KNOB(1)) {
@@ -921,7 +1044,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const int etid = threadIdx.x - epi_first_warp * 32;
         const int ehalf = (warp - epi_first_warp) >> 2;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const int first_unit = (int)(lo / a.P);
+        const int first_unit = (int)((unsigned)lo / (unsigned)a.P);
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
         uint32_t accphase = 0;
         bool ok = true;
@@ -970,9 +1093,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!whole) {
                 // This tile is cut across CTAs: publish the partial, count arrivals, and let
                 // the last CTA to arrive add the partials in CTA order and write Y.
-                const long long first_item = (long long)unit * a.P;
-                const int c0 = (int)(((first_item + 1) * gridDim.x - 1) / a.T);
-                const int c1 = (int)(((first_item + a.P) * (long long)gridDim.x - 1) / a.T);
+                const int first_item = unit * a.P;
+                const int c0 = cta_of_item(a, first_item);
+                const int c1 = cta_of_item(a, first_item + a.P - 1);
                 __threadfence();
                 epi_bar_sync(n_epi_warps * 32);
                 if (etid == 0) {
@@ -985,7 +1108,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
                     // range starts exactly there.  Every later CTA starts inside the tile.
-                    const int slot0 = ((long long)c0 * a.T / gridDim.x == first_item) ? 2 * c0 : 2 * c0 + 1;
+                    const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
                     reduce_partials(a, u, etid, n_epi_warps, a.partials + (size_t)slot0 * a.slot_floats,
                                     a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats,
                                     2 * (size_t)a.slot_floats, c1 - c0);

@@ -13,8 +13,9 @@ struct GemmArgs {
     int B, m, N, K;
     int decode, convert, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
     int m_tiles, groups, P, whole_units;
-    long long T;
-    int stages, a_slots, halves, load_depth;
+    int T;             // work items (< 2^30)
+    int q, r;          // T = q * grid + r
+    int stages, a_slots, halves;
     uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
@@ -29,8 +30,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
     a.decode = p.decode; a.convert = p.convert; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
     a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
-    a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = p.T; a.whole_units = p.whole_units;
-    a.stages = p.stages; a.a_slots = p.a_slots; a.halves = p.halves; a.load_depth = p.load_depth;
+    a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.q = (int)(p.T / p.grid); a.r = (int)(p.T % p.grid); a.whole_units = p.whole_units;
+    a.stages = p.stages; a.a_slots = p.a_slots; a.halves = p.halves;
     a.stage_bytes = p.stage_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;

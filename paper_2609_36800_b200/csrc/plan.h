@@ -43,7 +43,6 @@ struct Plan {
     long long T;       // total k-pair work items = units * P
     int grid;
     int stages, a_slots;
-    int load_depth;    // stage loads kept in flight (0 = as many as the ring holds)
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
     uint32_t col_base, col_delta, col_a;
@@ -57,8 +56,7 @@ struct Plan {
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0,
-                      int depth_override = 0) {
+inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
@@ -102,6 +100,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.units = p.n_tiles * p.groups;
     p.P = (K + kPairK - 1) / kPairK;
     p.T = (long long)p.units * p.P;
+    if (p.T >= (1ll << 30)) return p;   // the kernel's work-split arithmetic is 32-bit
     int max_grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
     p.grid = p.T < max_grid ? (int)p.T : max_grid;
     // Several tenant groups share each W_base tile.  If every CTA takes whole units in round-robin
@@ -134,7 +133,6 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.col_delta = (uint32_t)p.Nb;
     p.col_a = p.col_delta + (uint32_t)(p.TB * p.Nd);
     int free_cols = kTmemCols - (int)p.col_a;
-    p.load_depth = depth_override;
     p.halves = 2;
     if (p.decode && free_cols >= 2 * 2 * 2 * p.aslot_cols) {
         // Room for two whole-stage buffers per decode group: hand over 128 k at a time, which halves
