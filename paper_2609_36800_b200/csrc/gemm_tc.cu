@@ -93,8 +93,10 @@ __device__ int g_knobs;
 __device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] site of the first failure
 
 struct Ctl {
-    uint64_t full[kMaxStages];
-    uint64_t empty[kMaxStages];
+    uint64_t wfull[kMaxStages];        // W_base tile landed
+    uint64_t wempty[kMaxStages];       // ... and was read by the base MMAs (tcgen05.commit)
+    uint64_t xfull[kMaxStages];        // activation tile landed
+    uint64_t xempty[kMaxStages];       // ... and every MMA of its stage has completed
     uint64_t bfull[kBitSlots];
     uint64_t bempty[kBitSlots];
     uint64_t afull[kMaxASlots];        // tiled schedule: decoded operand ready (decode warps -> MMA warp)
@@ -421,10 +423,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t stages_addr = base;
-    const uint32_t bits_addr = base + a.stages * a.stage_bytes;
-    uint8_t* bits_ptr = smem + a.stages * a.stage_bytes;
-    Ctl* ctl = reinterpret_cast<Ctl*>(smem + a.stages * a.stage_bytes + kBitSlots * a.bslot_bytes);
+    const uint32_t w_addr = base;                                        // ring of W_base tiles
+    const uint32_t xr_off = a.n_w * a.w_stage_bytes;                     // ring of activation tiles
+    const uint32_t xr_addr = base + xr_off;
+    const uint32_t bits_off = xr_off + a.n_x * a.xr_bytes;               // sign-word slots
+    const uint32_t bits_addr = base + bits_off;
+    uint8_t* bits_ptr = smem + bits_off;
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + bits_off + kBitSlots * a.bslot_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
     constexpr bool kDec = kMode != 0;
@@ -454,19 +459,20 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     int unit, p0, p1;
     const bool load_x8 = kDec && !convert;
 
-    // Queues the weight loads of one item: its W_base tile into `stage` and, if `with_bits`, the sign words
-    // of its k-pair into sign-word slot `bslot`.  One thread.  The stage's activations follow separately.
+    // Queues the weight loads of one item: its W_base tile into `stage` of the W ring and, if `with_bits`,
+    // the sign words of its k-pair into sign-word slot `bslot`.  One thread.
     auto issue_weights_raw = [&](const Unit& u, int p, int stage, int bslot, bool with_bits) {
         // W_base first: the stage's MMAs need it together with the activations, and the first sign-word
         // load of a tile is slow (it pulls whole 128-byte lines, i.e. the signs of 1024 k, out of DRAM).
-        const uint32_t bar = smem_u32(&ctl->full[stage]);
-        const uint32_t dst = stages_addr + stage * a.stage_bytes;
-        uint32_t tx = load_x8 ? a.stage_bytes : a.stage_bytes - a.x8_atom_bytes;
-        if (BD_KNOB(16)) tx -= 2 * a.w_atom_bytes;
-        if (BD_KNOB(32)) tx -= 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0);
-        if (tx) mbar_arrive_expect_tx(bar, tx); else mbar_arrive(bar);
+        const uint32_t bar = smem_u32(&ctl->wfull[stage]);
+        const uint32_t dst = w_addr + stage * a.w_stage_bytes;
         const int k0 = p * kPairK;
-        if (!BD_KNOB(16)) {
+        if (BD_KNOB(16)) {
+            mbar_arrive(bar);
+        } else {
+            // tiled schedule: the stage's activation tile (same slot index, queued by the activation
+            // stream) completes on this barrier too
+            mbar_arrive_expect_tx(bar, a.w_stage_bytes + ((kDec || BD_KNOB(32)) ? 0u : 2 * a.x_atom_bytes));
             tma_load_2d(dst, &tmW, bar, k0, u.n0);
             tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
         }
@@ -481,17 +487,19 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
     };
 
-    // One issuer thread's share (tasks tid, tid + 96, ...) of the in-kernel activation split of stage `st`.
+    // One issuer thread's share (tasks tid, tid + 96, ...) of the in-kernel activation split of activation slot `st`.
     auto do_split = [&](int st, int ntok, int tid) {
-        split_activations(a, am, smem + st * a.stage_bytes + 2 * a.w_atom_bytes, ntok, tid, 96);
+        split_activations(a, am, smem + xr_off + st * a.xr_bytes, ntok, tid, 96);
         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
         mbar_arrive(smem_u32(&ctl->x8full[st]));
     };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a stage
+            mbar_init(smem_u32(&ctl->wfull[s]), 1);
+            mbar_init(smem_u32(&ctl->wempty[s]), 1);
+            mbar_init(smem_u32(&ctl->xfull[s]), 1);
+            mbar_init(smem_u32(&ctl->xempty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a tile
             mbar_init(smem_u32(&ctl->x8full[s]), 96);
         }
         for (int s = 0; s < kBitSlots; ++s) {
@@ -531,85 +539,97 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     if (warp == kWarpProducer) {
         // ------------------------------------------------------------ TMA producer
         // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
-        // Weights (W_base, sign words) never depend on the kernel queued before this one, the
-        // activations may.  Weight loads therefore run ahead as far as the rings allow; the activations
-        // of every item whose weights are queued follow as soon as the grid dependency is resolved
-        // (warp 1 waits for it and completes `depready`), so that they are not queued behind a whole
-        // ring of weight traffic when the dependency is already met at launch.
+        // Two independent streams over the same item list:
+        //  * weights (W_base tile + sign words) never depend on the kernel queued before this one and
+        //    run ahead as far as their rings allow;
+        //  * activations wait for the grid dependency (warp 1 completes `depready`) and for a free slot
+        //    of their own, shallower ring.
+        // Neither stream may block the other, so the warp polls both rings and sleeps on a short
+        // suspended wait when neither can advance.
         ItemIter wi(it), xi(it);
-        int n_w = 0, n_x = 0;            // items whose weights / activations are queued
-        int stage = 0, stage_x = 0, bslot = 0, slots_used = 0;
-        uint32_t phase = 0, bphase = 0;
+        int stage = 0, xslot = 0, bslot = 0;
+        uint32_t phase = 0, xphase = 0, bphase = 0;
         bool ok = true, dep_ok = false;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
         Unit uw{}, ux{};
         bool more_w = wi.next();
+        bool more_x = xi.next();
+        if (more_x) ux = unit_info(a, xi.unit);
         if (more_w) {
-            // queued by thread 0 in the prologue: stage 0, sign-word slot 0
-            n_w = 1; slots_used = 1; bslot = 1 % kBitSlots; bphase = (kBitSlots == 1) ? 1u : 0u;
-            stage = 1 % a.stages; phase = (a.stages == 1) ? 1u : 0u;
+            // queued by thread 0 in the prologue: W stage 0, sign-word slot 0
+            bslot = 1 % kBitSlots; bphase = (kBitSlots == 1) ? 1u : 0u;
+            stage = 1 % a.n_w; phase = (a.n_w == 1) ? 1u : 0u;
             BD_TL(0);
             uw = unit_info(a, wi.unit);
             more_w = wi.next();
+            if (more_w && wi.first) uw = unit_info(a, wi.unit);
         }
         const uint32_t depbar = smem_u32(&ctl->depready);
-        for (;;) {
-            const bool need_slot = more_w && (wi.first || !(wi.p & 1));
-            if (!dep_ok) {
-                // Without the activations no stage is ever released: only the first ring may be filled blind.
-                const bool must = !more_w || n_w >= a.stages || (need_slot && slots_used >= kBitSlots);
-                if (must) {
-                    ok = warp_all(wait_bar(depbar, 0, abort_flag, 10));
-                    if (!ok) break;
-                    dep_ok = true;
-                } else {
-                    dep_ok = warp_all(mbar_test_wait(depbar, 0));
-                }
-            }
-            if (dep_ok) {
-                while (n_x < n_w) {
-                    xi.next();
-                    if (xi.first) ux = unit_info(a, xi.unit);
-                    if (!BD_KNOB(32) && elect_one()) {
-                        const uint32_t bar = smem_u32(&ctl->full[stage_x]);
-                        const uint32_t dst = stages_addr + stage_x * a.stage_bytes + 2 * a.w_atom_bytes;
+        const uint32_t x_tx = BD_KNOB(32) ? 0u : 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0u);
+        long long t_idle = 0;
+        int idle = 0;
+        while (more_w || more_x) {
+            bool did = false;
+            if (more_x) {
+                if (!dep_ok) dep_ok = warp_all(mbar_test_wait(depbar, 0));
+                const uint32_t xebar = kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot]);
+                if (dep_ok && warp_all(mbar_test_wait(xebar, xphase ^ 1))) {
+                    if (elect_one()) {
+                        const uint32_t bar = kDec ? smem_u32(&ctl->xfull[xslot]) : smem_u32(&ctl->wfull[xslot]);
+                        const uint32_t dst = xr_addr + xslot * a.xr_bytes;
                         const int k0 = xi.p * kPairK;
-                        tma_load_2d(dst, &tmX, bar, k0, ux.xrow0);
-                        tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, ux.xrow0);
-                        if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, ux.tenant0 * kPieces * am);
+                        if (x_tx) {
+                            if (kDec) mbar_arrive_expect_tx(bar, x_tx);
+                            tma_load_2d(dst, &tmX, bar, k0, ux.xrow0);
+                            tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, ux.xrow0);
+                            if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, ux.tenant0 * kPieces * am);
+                        } else if (kDec) {
+                            mbar_arrive(bar);
+                        }
                     }
                     __syncwarp();
-                    BD_STAMP_ONCE(29);
-                    ++n_x;
-                    if (++stage_x == a.stages) stage_x = 0;
+                    if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
+                    more_x = xi.next();
+                    if (more_x && xi.first) ux = unit_info(a, xi.unit);
+                    did = true;
                 }
             }
-            if (!more_w) {
-                if (n_x == n_w) break;
+            if (more_w) {
+                const bool need_slot = wi.first || !(wi.p & 1);
+                if ((!need_slot || warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) &&
+                    warp_all(mbar_test_wait(smem_u32(&ctl->wempty[stage]), phase ^ 1))) {
+                    if (elect_one()) issue_weights_raw(uw, wi.p, stage, bslot, need_slot);
+                    __syncwarp();
+                    BD_TL(0);
+                    if (need_slot && ++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                    if (++stage == a.n_w) { stage = 0; phase ^= 1; }
+                    more_w = wi.next();
+                    if (more_w && wi.first) uw = unit_info(a, wi.unit);
+                    did = true;
+                }
+            }
+            if (did) {
+                idle = 0;
                 continue;
             }
-            if (wi.first) uw = unit_info(a, wi.unit);
-            if (need_slot) {
-                BD_ACC_BEGIN(tb);
-                ok = warp_all(wait_bar(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, abort_flag, 1));
-                BD_ACC_END(w_bempty, tb);
-                if (!ok) break;
-            }
+            // Nothing can advance: a short suspended wait (tens of ns) on one ring, then look at both again.
             BD_ACC_BEGIN(te);
-            ok = warp_all(wait_bar(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, 2));
+            if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 32u);
+            else (void)mbar_try_wait_hint(dep_ok ? (kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot])) : depbar,
+                                          dep_ok ? (xphase ^ 1) : 0u, 32u);
             BD_ACC_END(w_empty, te);
-            if (!ok) break;
-            if (elect_one()) issue_weights_raw(uw, wi.p, stage, bslot, need_slot);
-            __syncwarp();
-            BD_TL(0);
-            if (need_slot) {
-                ++slots_used;
-                if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+            if (idle == 0) t_idle = clock64();
+            if ((++idle & 255) == 0) {
+                if (*abort_flag) { ok = false; break; }
+                if (clock64() - t_idle > kWaitLimitCycles) {
+                    *abort_flag = 1;
+                    if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = 2u;
+                    ok = false;
+                    break;
+                }
             }
-            ++n_w;
-            if (++stage == a.stages) { stage = 0; phase ^= 1; }
-            more_w = wi.next();
         }
+        (void)ok;
         BD_STAMP(3);
         BD_ACC_STORE(19, w_empty); BD_ACC_STORE(20, w_bempty);
     } else if (warp == kWarpMma) {
@@ -629,8 +649,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const uint32_t w_atom16 = a.w_atom_bytes >> 4, x_atom16 = a.x_atom_bytes >> 4;
         const uint32_t amask = (uint32_t)a.a_slots - 1;
         const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
-        int stage = 0;
-        uint32_t phase = 0, accphase = 0, item = 0;
+        int stage = 0, xslot = 0;
+        uint32_t phase = 0, xphase = 0, accphase = 0, item = 0;
         bool ok = true;
         bool split_done = false;   // this warp's share of the current stage's activation split was done ahead
         BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id); BD_TL_DECL;
@@ -647,16 +667,17 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
-                if (!split_done) {
+                {
                     BD_ACC_BEGIN(tf);
-                    ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                    ok = warp_all(wait_bar(smem_u32(&ctl->wfull[stage]), phase, abort_flag, 4));
+                    if (kDec && ok && !split_done) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
                     BD_ACC_END(w_full, tf);
                     if (!ok) break;
                 }
                 if (item == 0) BD_STAMP(4);
                 BD_TL(1);
-                const uint32_t wbase = stages_addr + stage * a.stage_bytes;
-                const uint32_t xbase = wbase + 2 * a.w_atom_bytes;
+                const uint32_t wbase = w_addr + stage * a.w_stage_bytes;
+                const uint32_t xbase = xr_addr + xslot * a.xr_bytes;
                 const uint64_t wdesc = desc0 + (wbase >> 4);
                 const uint64_t xdesc = desc0 + (xbase >> 4);
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
@@ -668,7 +689,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         umma_ss(tmem_base, wdesc + (atom * w_atom16 + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
                                 idesc_base, (kk > 0) ? 1u : first);
                     }
+                    // decode schedule: nothing else reads the W_base tile, hand it back as soon as these MMAs
+                    // have completed
+                    if (kDec) tc_commit(smem_u32(&ctl->wempty[stage]));
                 }
+                if (kDec && BD_KNOB(4) && elect_one()) tc_commit(smem_u32(&ctl->wempty[stage]));
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if constexpr (kDec) {
@@ -677,12 +702,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // the tasks each, completion counted on x8full[stage]); each warp does its share of the
                     // NEXT stage as soon as that stage has landed, so the split stays off the critical path.
                     if (convert) {
-                        if (!split_done) do_split(stage, u.ntok, lane);
+                        if (!split_done) do_split(xslot, u.ntok, lane);
                         split_done = false;
                         if (p + 1 < p1) {
-                            const int ns = (stage + 1 == a.stages) ? 0 : stage + 1;
-                            const uint32_t nph = (stage + 1 == a.stages) ? phase ^ 1 : phase;
-                            if (warp_all(mbar_test_wait(smem_u32(&ctl->full[ns]), nph))) {
+                            const int ns = (xslot + 1 == a.n_x) ? 0 : xslot + 1;
+                            const uint32_t nph = (xslot + 1 == a.n_x) ? xphase ^ 1 : xphase;
+                            if (warp_all(mbar_test_wait(smem_u32(&ctl->xfull[ns]), nph))) {
                                 do_split(ns, u.ntok, lane);
                                 split_done = true;
                             }
@@ -716,9 +741,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     }
                 }
                 if (!ok) break;
-                if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
+                if (elect_one()) tc_commit(kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[stage]));
                 __syncwarp();
-                if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                if (++stage == a.n_w) { stage = 0; phase ^= 1; }
+                if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
             }
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
@@ -743,8 +769,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             const uint32_t ten_rows16 = (uint32_t)(kPieces * am) * 8u;   // rows per tenant x 128 B >> 4
             const uint32_t amask = (uint32_t)a.a_slots - 1;
             const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
-            int stage = 0;
-            uint32_t phase = 0, accphase = 0, item = 0;
+            int xslot = 0;
+            uint32_t xphase = 0, accphase = 0, item = 0;
             bool ok = true;
             bool split_done = false;   // as in the base issuer
             BD_TL_DECL;
@@ -755,19 +781,18 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 tc_fence_after();
                 for (int p = p0; p < p1 && ok; ++p) {
                     if (!split_done) {
-                        ok = warp_all(wait_bar(smem_u32(&ctl->full[stage]), phase, abort_flag, 4));
+                        ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
                         if (!ok) break;
                     }
                     if (g == 0) BD_TL(2);
                     if (convert) {
-                        if (!split_done) do_split(stage, u.ntok, 32 * (g + 1) + lane);
+                        if (!split_done) do_split(xslot, u.ntok, 32 * (g + 1) + lane);
                         split_done = false;
                         // all three shares of this stage
-                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[stage]), phase, abort_flag, 11));
+                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[xslot]), xphase, abort_flag, 11));
                         if (!ok) break;
                     }
-                    const uint64_t x8desc = desc0 + ((stages_addr + stage * a.stage_bytes + 2 * a.w_atom_bytes) >> 4) +
-                                            2 * x_atom16;
+                    const uint64_t x8desc = desc0 + ((xr_addr + xslot * a.xr_bytes) >> 4) + 2 * x_atom16;
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
                     for (int half = 0; half < a.halves; ++half, ++item) {
                         const uint32_t slot = item & amask;
@@ -807,18 +832,18 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         __syncwarp();
                         if (half == 0 && convert && p + 1 < p1) {
                             // idle until the decode warps hand over the next buffer: split the next stage now
-                            const int ns = (stage + 1 == a.stages) ? 0 : stage + 1;
-                            const uint32_t nph = (stage + 1 == a.stages) ? phase ^ 1 : phase;
-                            if (warp_all(mbar_test_wait(smem_u32(&ctl->full[ns]), nph))) {
+                            const int ns = (xslot + 1 == a.n_x) ? 0 : xslot + 1;
+                            const uint32_t nph = (xslot + 1 == a.n_x) ? xphase ^ 1 : xphase;
+                            if (warp_all(mbar_test_wait(smem_u32(&ctl->xfull[ns]), nph))) {
                                 do_split(ns, u.ntok, 32 * (g + 1) + lane);
                                 split_done = true;
                             }
                         }
                     }
                     if (!ok) break;
-                    if (elect_one()) tc_commit(smem_u32(&ctl->empty[stage]));
+                    if (elect_one()) tc_commit(smem_u32(&ctl->xempty[xslot]));
                     __syncwarp();
-                    if (++stage == a.stages) { stage = 0; phase ^= 1; }
+                    if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
                 }
                 if (!ok) break;
                 if (elect_one()) tc_commit(smem_u32(&ctl->accfull));

@@ -42,9 +42,11 @@ struct Plan {
     int whole_units;   // 1: CTAs take whole units round-robin (no tile is cut), 0: even shares of the item list
     long long T;       // total k-pair work items = units * P
     int grid;
-    int stages, a_slots;
+    int n_w;           // ring of W_base tiles (128 rows x 128 k of bf16 each)
+    int n_x;           // ring of activation tiles (X, and in the decode schedule its e5m2 pieces)
+    int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
-    uint32_t stage_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
+    uint32_t w_stage_bytes, xr_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
     uint32_t col_base, col_delta, col_a;
     size_t slot_floats;   // floats of one partial-result slot: 128 rows x tokens per unit
     size_t ws_header_bytes;   // arrival counters: one u32 per work unit
@@ -75,8 +77,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.Nd = p.N3;
         p.win_rows = m;
         p.chunk_rows = m;
-        int need = (p.TB - 1) * m + 16;
-        p.x_rows = round_up(need > p.Nb ? need : p.Nb, 8);
+        p.x_rows = p.Nb;   // the bf16 tile feeds the base MMA (N = Nb) and the in-kernel split only
         p.x8_rows = round_up((p.TB - 1) * kPieces * m + p.N3, 8);
         p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
@@ -118,14 +119,26 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
-    p.stage_bytes = 2 * p.w_atom_bytes + 2 * p.x_atom_bytes + p.x8_atom_bytes;
+    p.w_stage_bytes = 2 * p.w_atom_bytes;
+    p.xr_bytes = 2 * p.x_atom_bytes + p.x8_atom_bytes;
     p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
-    int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
-    p.stages = avail / (int)p.stage_bytes;
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
-    if (p.decode && p.stages > 4) p.stages = 4;   // one named barrier per stage for the in-kernel split
-    if (p.stages < 2) return p;
-    p.smem_bytes = 1024 + p.stages * p.stage_bytes + kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
+    // Shared memory: a ring of W_base tiles, a ring of activation tiles, the sign-word slots.  W_base
+    // comes from DRAM (latency ~1.5 us under load) and a tile is released as soon as the base MMAs have
+    // read it; the activations come from L2 and are small, but a tile stays in use until the last delta
+    // MMA of its stage has completed.  Hence two rings with their own depths in the decode schedule
+    // (few activation slots, every remaining byte to W_base); the tiled schedule keeps them equal.
+    const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
+    if (p.decode) {
+        p.n_x = (p.xr_bytes > 16 * 1024) ? 2 : 3;
+        p.n_w = (avail - p.n_x * (int)p.xr_bytes) / (int)p.w_stage_bytes;
+        if (p.n_w > 6) p.n_w = 6;
+    } else {
+        p.n_w = avail / (int)(p.w_stage_bytes + p.xr_bytes);
+        if (p.n_w > kMaxStages) p.n_w = kMaxStages;
+        p.n_x = p.n_w;
+    }
+    if (p.n_w < 2) return p;
+    p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.xr_bytes + kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
     // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
     if (p.smem_bytes < 120 * 1024) p.smem_bytes = 120 * 1024;
 
