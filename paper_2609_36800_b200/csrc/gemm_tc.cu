@@ -50,26 +50,26 @@ __device__ int g_knobs;
 #define BD_KNOB(bit) (bd_knobs & (bit))
 #endif
 #define BD_KNOB_G(bit) (g_knobs & (bit))
-// Stamps go to shared memory (behind the control block; the launcher adds 8.5 KB in debug builds) and are
+// Stamps go to shared memory (behind the control block; the launcher adds 2.75 KB in debug builds) and are
 // copied out at teardown, so that taking one costs a clock read and a shared-memory store.
-// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[8][128]: per-role timelines (CTA 0 and 77 are kept).
+// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[5][64]: per-role timelines (CTA 0 and 77 are kept).
 #define BD_TRACE_SETUP \
     long long* const bd_st = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(ctl) + kSmemCtrlBytes); \
     long long* const bd_tlb = bd_st + 32; \
-    for (int i = threadIdx.x; i < 32 + 1024; i += kThreads) bd_st[i] = 0; \
+    for (int i = threadIdx.x; i < 32 + 320; i += kThreads) bd_st[i] = 0; \
     __syncthreads()
 #define BD_TRACE_FLUSH do { \
     long long* gp = g_trace_ptr; \
     if (gp) { \
         for (int i = threadIdx.x; i < 32; i += kThreads) gp[blockIdx.x * 32 + i] = bd_st[i]; \
         if (blockIdx.x == 0 || blockIdx.x == 77) \
-            for (int i = threadIdx.x; i < 1024; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + i] = bd_tlb[i]; \
+            for (int i = threadIdx.x; i < 320; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + (i >> 6) * 128 + (i & 63)] = bd_tlb[i]; \
     } } while (0)
 #define BD_STAMP(idx) do { if (lane == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_STAMP_ONCE(idx) do { if (lane == 0 && bd_st[idx] == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_TL_DECL int tl_idx = 0
-#define BD_TL(role) do { if (lane == 0 && tl_idx < 128) { bd_tlb[(role) * 128 + tl_idx] = clock64(); ++tl_idx; } } while (0)
-#define BD_TL2(role) do { if (lane == 0 && tl_idx2 < 128) { bd_tlb[(role) * 128 + tl_idx2] = clock64(); ++tl_idx2; } } while (0)
+#define BD_TL(role) do { if ((role) < 5 && lane == 0 && tl_idx < 64) { bd_tlb[(role) * 64 + tl_idx] = clock64(); ++tl_idx; } } while (0)
+#define BD_TL2(role) do { } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
 #define BD_ACC_END(name, t) name += clock64() - t
@@ -487,9 +487,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
     };
 
-    // One issuer thread's share (tasks tid, tid + 96, ...) of the in-kernel activation split of activation slot `st`.
+    // One epilogue thread's share (tasks tid, tid + 128, ...) of the in-kernel activation split of slot `st`.
     auto do_split = [&](int st, int ntok, int tid) {
-        split_activations(a, am, smem + xr_off + st * a.xr_bytes, ntok, tid, 96);
+        split_activations(a, am, smem + xr_off + st * a.xr_bytes, ntok, tid, 128);
         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
         mbar_arrive(smem_u32(&ctl->x8full[st]));
     };
@@ -500,7 +500,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             mbar_init(smem_u32(&ctl->wempty[s]), 1);
             mbar_init(smem_u32(&ctl->xfull[s]), 1);
             mbar_init(smem_u32(&ctl->xempty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a tile
-            mbar_init(smem_u32(&ctl->x8full[s]), 96);
+            mbar_init(smem_u32(&ctl->x8full[s]), 128);
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
@@ -652,7 +652,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0, xslot = 0;
         uint32_t phase = 0, xphase = 0, accphase = 0, item = 0;
         bool ok = true;
-        bool split_done = false;   // this warp's share of the current stage's activation split was done ahead
         BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id); BD_TL_DECL;
         // This warp also tells the producer when the grid this launch depends on has completed.
         BD_STAMP(30);
@@ -670,7 +669,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 {
                     BD_ACC_BEGIN(tf);
                     ok = warp_all(wait_bar(smem_u32(&ctl->wfull[stage]), phase, abort_flag, 4));
-                    if (kDec && ok && !split_done) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
+                    if (kDec && ok) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
                     BD_ACC_END(w_full, tf);
                     if (!ok) break;
                 }
@@ -697,22 +696,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if constexpr (kDec) {
-                    // Delta MMAs are issued by the two delta-issuer warps.  With few token rows per unit the
-                    // three issuer warps split each stage's activations into e5m2 pieces themselves (a third of
-                    // the tasks each, completion counted on x8full[stage]); each warp does its share of the
-                    // NEXT stage as soon as that stage has landed, so the split stays off the critical path.
-                    if (convert) {
-                        if (!split_done) do_split(xslot, u.ntok, lane);
-                        split_done = false;
-                        if (p + 1 < p1) {
-                            const int ns = (xslot + 1 == a.n_x) ? 0 : xslot + 1;
-                            const uint32_t nph = (xslot + 1 == a.n_x) ? xphase ^ 1 : xphase;
-                            if (warp_all(mbar_test_wait(smem_u32(&ctl->xfull[ns]), nph))) {
-                                do_split(ns, u.ntok, lane);
-                                split_done = true;
-                            }
-                        }
-                    }
+                    // Delta MMAs are issued by the two delta-issuer warps.
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item) {
                         const uint32_t slot = item & amask;
@@ -772,7 +756,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             int xslot = 0;
             uint32_t xphase = 0, accphase = 0, item = 0;
             bool ok = true;
-            bool split_done = false;   // as in the base issuer
             BD_TL_DECL;
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
@@ -780,18 +763,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (!ok) break;
                 tc_fence_after();
                 for (int p = p0; p < p1 && ok; ++p) {
-                    if (!split_done) {
-                        ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
-                        if (!ok) break;
-                    }
+                    // few token rows per unit: the e5m2 pieces are written by the epilogue warps (x8full);
+                    // otherwise they arrive with the activation tile
+                    ok = warp_all(wait_bar(convert ? smem_u32(&ctl->x8full[xslot]) : smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
+                    if (!ok) break;
                     if (g == 0) BD_TL(2);
-                    if (convert) {
-                        if (!split_done) do_split(xslot, u.ntok, 32 * (g + 1) + lane);
-                        split_done = false;
-                        // all three shares of this stage
-                        ok = warp_all(wait_bar(smem_u32(&ctl->x8full[xslot]), xphase, abort_flag, 11));
-                        if (!ok) break;
-                    }
                     const uint64_t x8desc = desc0 + ((xr_addr + xslot * a.xr_bytes) >> 4) + 2 * x_atom16;
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
                     for (int half = 0; half < a.halves; ++half, ++item) {
@@ -830,15 +806,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                             tc_commit(smem_u32(&ctl->aempty[g * kMaxASlots + slot]));
                         }
                         __syncwarp();
-                        if (half == 0 && convert && p + 1 < p1) {
-                            // idle until the decode warps hand over the next buffer: split the next stage now
-                            const int ns = (xslot + 1 == a.n_x) ? 0 : xslot + 1;
-                            const uint32_t nph = (xslot + 1 == a.n_x) ? xphase ^ 1 : xphase;
-                            if (warp_all(mbar_test_wait(smem_u32(&ctl->xfull[ns]), nph))) {
-                                do_split(ns, u.ntok, 32 * (g + 1) + lane);
-                                split_done = true;
-                            }
-                        }
                     }
                     if (!ok) break;
                     if (elect_one()) tc_commit(smem_u32(&ctl->xempty[xslot]));
@@ -1074,10 +1041,45 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint32_t accphase = 0;
         bool ok = true;
         BD_TL_DECL;
+        // Decode schedule with few token rows per unit: these four warps, idle while a tile is being
+        // accumulated, also split every stage's activations into e5m2 pieces (one 16-element task per
+        // thread), as soon as the stage's activation tile has landed.  Each warp walks the items on its
+        // own; x8full[slot] counts all 128 threads.  Items of the current tile are split with blocking
+        // waits (the tile cannot complete without them), later ones whenever there is nothing else to do.
+        const bool splitter = kDec && convert;
+        ItemIter si(it);
+        bool more_s = splitter && si.next();
+        int sslot = 0, n_split = 0, seg_end = 0;
+        uint32_t sphase = 0;
+        Unit us{};
+        if (more_s) us = unit_info(a, si.unit);
+        auto split_next = [&](bool block) -> bool {
+            const uint32_t bar = smem_u32(&ctl->xfull[sslot]);
+            if (block) {
+                if (!wait_bar(bar, sphase, abort_flag, 13)) return false;
+            } else if (!warp_all(mbar_test_wait(bar, sphase))) {
+                return false;
+            }
+            do_split(sslot, us.ntok, etid);
+            if (++sslot == a.n_x) { sslot = 0; sphase ^= 1; }
+            ++n_split;
+            more_s = si.next();
+            if (more_s && si.first) us = unit_info(a, si.unit);
+            return true;
+        };
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
             const bool whole = (p0 == 0 && p1 == a.P);
+            if (splitter) {
+                seg_end += p1 - p0;
+                while (ok && n_split < seg_end) ok = split_next(true);
+                if (!ok) break;
+                // until this tile's accumulators are complete: split ahead whatever has landed
+                while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
+                    if (!split_next(false)) break;
+                }
+            }
             float* slotp = nullptr;
             if (!whole) {
                 const int slot = (unit == first_unit) ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1;
@@ -1114,6 +1116,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
             if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
+            if (splitter) {
+                // the next tile's first stages, before the (slow) fix-up of this one
+                while (more_s && split_next(false)) {
+                }
+            }
 
             if (!whole) {
                 // This tile is cut across CTAs: publish the partial, count arrivals, and let
@@ -1195,7 +1202,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
 #ifdef BD_TRACE
-    cfg.dynamicSmemBytes = smem_bytes + 8704;   // room for the stamps behind the control block
+    cfg.dynamicSmemBytes = smem_bytes + 2816;   // room for the stamps behind the control block
 #else
     cfg.dynamicSmemBytes = smem_bytes;
 #endif
