@@ -268,6 +268,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
     }
 
     bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
+    { static int h = -1; if (h < 0) { const char* e = getenv("BITDELTA_HOLD"); h = (e && e[0] == '0') ? 0 : 1; } args.hold_prefetch = h; }
     if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
     g_launches++;

@@ -256,10 +256,13 @@ struct EpiOut {
 // activation split, token t in column q*M + t.  delta = D0 + D1 + D2 + D3.
 template <int M>
 __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                                const EpiOut& out) {
+                                                const EpiOut& out, const float* alv) {
     constexpr int N3 = (kPieces * M + 15) / 16 * 16;
     constexpr int TPB = (N3 == 16) ? 2 : 1;   // tenants drained per wait
-    for (int j0 = 0; j0 < u.nten; j0 += TPB) {
+    constexpr int kMaxTen = (M <= 4) ? 8 : 4;   // tenants per unit (see the plan)
+#pragma unroll
+    for (int j0 = 0; j0 < kMaxTen; j0 += TPB) {
+        if (j0 >= u.nten) break;
         uint32_t rb[16], rd[TPB * N3];
         tmem_ld16(lane_taddr + (uint32_t)(j0 * M), rb);
 #pragma unroll
@@ -272,7 +275,7 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
 #pragma unroll
         for (int jj = 0; jj < TPB; ++jj) {
             if (j0 + jj < u.nten) {
-                const float al = __ldg(a.alpha + u.tenant0 + j0 + jj);
+                const float al = alv[j0 + jj];
 #pragma unroll
                 for (int t = 0; t < M; ++t) {
                     const float lo = __uint_as_float(rd[jj * N3 + 2 * M + t]) + __uint_as_float(rd[jj * N3 + 3 * M + t]);
@@ -287,8 +290,7 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
 // Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
 // Two warps share each lane quadrant: warp half h drains the 32-token blocks h, h+2, ...
 __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                               const EpiOut& out, int half) {
-    const float al = __ldg(a.alpha + u.tenant0);
+                                               const EpiOut& out, int half, float al) {
     for (int t0 = 32 * half; t0 < u.ntok; t0 += 64) {
         uint32_t rb[32], rd[32];
         tmem_ld32(lane_taddr + (uint32_t)t0, rb);
@@ -550,6 +552,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0, xslot = 0, bslot = 0;
         uint32_t phase = 0, xphase = 0, bphase = 0;
         bool ok = true, dep_ok = false;
+        bool hold = kDec && a.hold_prefetch != 0;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
         Unit uw{}, ux{};
         bool more_w = wi.next();
@@ -594,7 +597,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
-            if (more_w) {
+            if (more_w && hold) {
+                // The first sign-word load of a tile pulls whole 128-byte lines (the signs of 1024 k) out of
+                // DRAM; until it has landed, further weight requests would only queue in front of it.
+                hold = !warp_all(mbar_test_wait(smem_u32(&ctl->bfull[0]), 0));
+            }
+            if (more_w && !hold) {
                 const bool need_slot = wi.first || !(wi.p & 1);
                 if ((!need_slot || warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) &&
                     warp_all(mbar_test_wait(smem_u32(&ctl->wempty[stage]), phase ^ 1))) {
@@ -614,7 +622,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             // Nothing can advance: a short suspended wait (tens of ns) on one ring, then look at both again.
             BD_ACC_BEGIN(te);
-            if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 32u);
+            if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 32u);
+            else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 32u);
             else (void)mbar_try_wait_hint(dep_ok ? (kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot])) : depbar,
                                           dep_ok ? (xphase ^ 1) : 0u, 32u);
             BD_ACC_END(w_empty, te);
@@ -1071,6 +1080,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
             const bool whole = (p0 == 0 && p1 == a.P);
+            // the tenants' scales, requested now so that their latency is not paid after the accumulators complete
+            float alv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
             if (splitter) {
                 seg_end += p1 - p0;
                 while (ok && n_split < seg_end) ok = split_next(true);
@@ -1093,24 +1106,24 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
             if constexpr (kMode >= 1 && kMode <= 4) {
-                epilogue_decode<kMode>(a, u, lane_taddr, out);
+                epilogue_decode<kMode>(a, u, lane_taddr, out, alv);
             } else if constexpr (kMode == 5) {
                 switch (am) {
-                    case 5: epilogue_decode<5>(a, u, lane_taddr, out); break;
-                    case 6: epilogue_decode<6>(a, u, lane_taddr, out); break;
-                    case 7: epilogue_decode<7>(a, u, lane_taddr, out); break;
-                    case 8: epilogue_decode<8>(a, u, lane_taddr, out); break;
-                    case 9: epilogue_decode<9>(a, u, lane_taddr, out); break;
-                    case 10: epilogue_decode<10>(a, u, lane_taddr, out); break;
-                    case 11: epilogue_decode<11>(a, u, lane_taddr, out); break;
-                    case 12: epilogue_decode<12>(a, u, lane_taddr, out); break;
-                    case 13: epilogue_decode<13>(a, u, lane_taddr, out); break;
-                    case 14: epilogue_decode<14>(a, u, lane_taddr, out); break;
-                    case 15: epilogue_decode<15>(a, u, lane_taddr, out); break;
-                    default: epilogue_decode<16>(a, u, lane_taddr, out); break;
+                    case 5: epilogue_decode<5>(a, u, lane_taddr, out, alv); break;
+                    case 6: epilogue_decode<6>(a, u, lane_taddr, out, alv); break;
+                    case 7: epilogue_decode<7>(a, u, lane_taddr, out, alv); break;
+                    case 8: epilogue_decode<8>(a, u, lane_taddr, out, alv); break;
+                    case 9: epilogue_decode<9>(a, u, lane_taddr, out, alv); break;
+                    case 10: epilogue_decode<10>(a, u, lane_taddr, out, alv); break;
+                    case 11: epilogue_decode<11>(a, u, lane_taddr, out, alv); break;
+                    case 12: epilogue_decode<12>(a, u, lane_taddr, out, alv); break;
+                    case 13: epilogue_decode<13>(a, u, lane_taddr, out, alv); break;
+                    case 14: epilogue_decode<14>(a, u, lane_taddr, out, alv); break;
+                    case 15: epilogue_decode<15>(a, u, lane_taddr, out, alv); break;
+                    default: epilogue_decode<16>(a, u, lane_taddr, out, alv); break;
                 }
             } else {
-                epilogue_tiled(a, u, lane_taddr, out, ehalf);
+                epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0]);
             }
             tc_fence_before();
             __syncwarp();
