@@ -355,48 +355,44 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
     }
 }
 
-// In-kernel activation split (decode schedule, few token rows per unit).  Task (r, q4, h): token row r,
-// 32-k group q4 of the stage, half h of the group's byte slots.  Slot 4c+i holds k = c + 8i, so half h
-// (c = 4h..4h+3) needs, from each of the four 16-byte chunks (i = 0..3) of the group, the 8 bytes
-// holding k = 8i+4h .. 8i+4h+3, and produces one 16-byte chunk per piece.  Arithmetic on packed f16
-// pairs (a bf16 value in the e5m2 range is exact in f16): p = rn_e5m2(y); y -= p; four times.
-// `xt` is the stage's X tile (two swizzled 64-k atoms), followed by the piece tile.  Thread `tid` of
-// `nthreads` takes the tasks tid, tid + nthreads, ...
+// In-kernel activation split (decode schedule, few token rows per unit).  Task (r, q4, h, pc): token row
+// r, 32-k group q4 of the stage, half h of the group's byte slots, pair pc of the half's four k classes.
+// Slot 4c+i holds k = c + 8i, so the task's classes c = 4h+2pc, 4h+2pc+1 need, from each of the four
+// 16-byte chunks (i = 0..3) of the group, the 4 bytes holding k = 8i+c, 8i+c+1, and produce 8 bytes
+// (slots 16h+8pc .. +7) per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
+// exact in f16): p = rn_e5m2(y); y -= p; four times.  `xt` is the stage's X tile (two swizzled 64-k
+// atoms), followed by the piece tile.  Thread `tid` of `nthreads` takes the tasks tid, tid + nthreads, ...
+// Small tasks on purpose: 16 per token row spread the work over all four epilogue warps, one warp per
+// scheduler, so that no scheduler's decode warps are slowed more than the others'.
 __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, uint8_t* xt, int ntok, int tid, int nthreads) {
     uint8_t* x8t = xt + 2 * a.x_atom_bytes;
-    const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 8;
+    const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 16;
     for (int task = tid; task < ntasks; task += nthreads) {
-        const int r = task >> 3, q4 = (task >> 1) & 3, h = task & 1;
+        const int r = task >> 4, q4 = (task >> 2) & 3, h = (task >> 1) & 1, pc = task & 1;
         const int j = r / am, t = r - j * am;
-        const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8;
-        __half2 y[8];   // y[2*i + pc]: k = 8i + 4h + 2pc, +1
+        const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8 + pc * 4;
+        __half2 y[4];   // y[i]: k = 8i + 4h + 2pc, +1
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
-            const uint2 v = *reinterpret_cast<const uint2*>(src + chunk * 16);
-            y[2 * i] = __floats2half2_rn(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
-            y[2 * i + 1] = __floats2half2_rn(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(src + chunk * 16);
+            y[i] = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
         }
 #pragma unroll
         for (int q = 0; q < kPieces; ++q) {
-            uint32_t pk[8];
+            uint32_t pk[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const __nv_fp8x2_storage_t pc =
-                    __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[e]), __NV_SATFINITE, __NV_E5M2);
-                y[e] = __hsub2(y[e], __half2(__nv_cvt_fp8x2_to_halfraw2(pc, __NV_E5M2)));
-                pk[e] = pc;
+            for (int i = 0; i < 4; ++i) {
+                const __nv_fp8x2_storage_t p8 =
+                    __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[i]), __NV_SATFINITE, __NV_E5M2);
+                y[i] = __hsub2(y[i], __half2(__nv_cvt_fp8x2_to_halfraw2(p8, __NV_E5M2)));
+                pk[i] = p8;
             }
-            uint32_t w[4];
-#pragma unroll
-            for (int pc = 0; pc < 2; ++pc) {
-                const uint32_t r01 = pk[pc] | (pk[2 + pc] << 16);
-                const uint32_t r23 = pk[4 + pc] | (pk[6 + pc] << 16);
-                w[2 * pc] = __byte_perm(r01, r23, 0x6420);
-                w[2 * pc + 1] = __byte_perm(r01, r23, 0x7531);
-            }
+            const uint32_t r01 = pk[0] | (pk[1] << 16);
+            const uint32_t r23 = pk[2] | (pk[3] << 16);
+            const uint2 w = make_uint2(__byte_perm(r01, r23, 0x6420), __byte_perm(r01, r23, 0x7531));
             const int r8 = j * (kPieces * am) + q * am + t;
-            *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint2*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16) + pc * 8) = w;
         }
     }
 }
