@@ -618,10 +618,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             // Nothing can advance: a short suspended wait (tens of ns) on one ring, then look at both again.
             BD_ACC_BEGIN(te);
-            if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 32u);
-            else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 32u);
+            if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 64u);
+            else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 64u);
             else (void)mbar_try_wait_hint(dep_ok ? (kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot])) : depbar,
-                                          dep_ok ? (xphase ^ 1) : 0u, 32u);
+                                          dep_ok ? (xphase ^ 1) : 0u, 64u);
             BD_ACC_END(w_empty, te);
             if (idle == 0) t_idle = clock64();
             if ((++idle & 255) == 0) {
@@ -1137,9 +1137,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const int first_item = unit * a.P;
                 const int c0 = cta_of_item(a, first_item);
                 const int c1 = cta_of_item(a, first_item + a.P - 1);
-                __threadfence();
+                // All epilogue threads' partial stores, then one thread's fence (cumulative over what the
+                // barrier ordered before it) and the arrival count.
                 epi_bar_sync(n_epi_warps * 32);
                 if (etid == 0) {
+                    __threadfence();
                     const unsigned old = atomicAdd(&a.counters[unit], 1u);
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
