@@ -95,15 +95,18 @@ int check_gemm_args(const void* X, const void* W, const void* bits, const void* 
     return BITDELTA_OK;
 }
 
-// 2-D bf16 [rows, K] row-major, box = 64 columns (128 bytes, swizzled) x box_rows.
-bool encode_bf16_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
+// bf16 [rows, K] row-major, seen as [K/64 atoms][rows][64]: one box = two 64-column atoms (128 bytes per
+// row each, swizzled) x box_rows, i.e. a whole 128-k stage tile in ONE bulk-tensor operation, landing in
+// shared memory atom after atom.  (The number of bulk operations a CTA keeps in flight is what limits
+// its load throughput, not their size.)  Coordinates: (0, first row, k / 64).
+bool encode_bf16_tile(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {K, rows};
-    cuuint64_t strides[1] = {K * 2};
-    cuuint32_t box[2] = {64, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+    cuuint64_t dims[3] = {64, rows, K / 64};
+    cuuint64_t strides[2] = {K * 2, 128};
+    cuuint32_t box[3] = {64, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -250,8 +253,8 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
 
     CUtensorMap tmW, tmX, tmX8, tmBits;
-    if (!encode_bf16_2d(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
-    if (!encode_bf16_2d(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
+    if (!encode_bf16_tile(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
+    if (!encode_bf16_tile(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
     if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB))
         return BITDELTA_ERR_CUDA;
     if (p.decode && !p.convert) {

@@ -50,25 +50,31 @@ __device__ int g_knobs;
 #define BD_KNOB(bit) (bd_knobs & (bit))
 #endif
 #define BD_KNOB_G(bit) (g_knobs & (bit))
-// Stamps go to shared memory (behind the control block; the launcher adds 2.75 KB in debug builds) and are
+#ifndef BD_TLN
+#define BD_TLN 20      // stamps kept per role ...
+#endif
+#ifndef BD_TLSKIP
+#define BD_TLSKIP 0   // ... after skipping this many
+#endif
+// Stamps go to shared memory (behind the control block; the launcher adds about 1 KB in debug builds) and are
 // copied out at teardown, so that taking one costs a clock read and a shared-memory store.
-// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[5][64]: per-role timelines (CTA 0 and 77 are kept).
+// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[5][BD_TLN]: per-role timelines (CTA 0 and 77 are kept).
 #define BD_TRACE_SETUP \
     long long* const bd_st = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(ctl) + kSmemCtrlBytes); \
     long long* const bd_tlb = bd_st + 32; \
-    for (int i = threadIdx.x; i < 32 + 320; i += kThreads) bd_st[i] = 0; \
+    for (int i = threadIdx.x; i < 32 + 5 * BD_TLN; i += kThreads) bd_st[i] = 0; \
     __syncthreads()
 #define BD_TRACE_FLUSH do { \
     long long* gp = g_trace_ptr; \
     if (gp) { \
         for (int i = threadIdx.x; i < 32; i += kThreads) gp[blockIdx.x * 32 + i] = bd_st[i]; \
         if (blockIdx.x == 0 || blockIdx.x == 77) \
-            for (int i = threadIdx.x; i < 320; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + (i >> 6) * 128 + (i & 63)] = bd_tlb[i]; \
+            for (int i = threadIdx.x; i < 5 * BD_TLN; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + (i / BD_TLN) * 128 + (i % BD_TLN)] = bd_tlb[i]; \
     } } while (0)
 #define BD_STAMP(idx) do { if (lane == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_STAMP_ONCE(idx) do { if (lane == 0 && bd_st[idx] == 0) bd_st[idx] = clock64(); } while (0)
 #define BD_TL_DECL int tl_idx = 0
-#define BD_TL(role) do { if ((role) < 5 && lane == 0 && tl_idx < 64) { bd_tlb[(role) * 64 + tl_idx] = clock64(); ++tl_idx; } } while (0)
+#define BD_TL(role) do { if ((role) < 5 && lane == 0 && tl_idx >= BD_TLSKIP && tl_idx < BD_TLSKIP + BD_TLN) { bd_tlb[(role) * BD_TLN + tl_idx - BD_TLSKIP] = clock64(); } ++tl_idx; } while (0)
 #define BD_TL2(role) do { } while (0)
 #define BD_ACC_DECL(name) long long name = 0
 #define BD_ACC_BEGIN(t) const long long t = clock64()
@@ -95,15 +101,16 @@ __device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] s
 struct Ctl {
     uint64_t wfull[kMaxStages];        // W_base tile landed
     uint64_t wempty[kMaxStages];       // ... and was read by the base MMAs (tcgen05.commit)
-    uint64_t xfull[kMaxStages];        // activation tile landed
-    uint64_t xempty[kMaxStages];       // ... and every MMA of its stage has completed
+    uint64_t xfull[kMaxStages];        // bf16 activation tile landed
+    uint64_t xempty[kMaxStages];       // ... and was read by the base MMAs (and by the in-kernel split)
+    uint64_t x8empty[kMaxStages];      // decode: piece tile free again (both delta issuers' MMAs completed)
     uint64_t bfull[kBitSlots];
     uint64_t bempty[kBitSlots];
     uint64_t afull[kMaxASlots];        // tiled schedule: decoded operand ready (decode warps -> MMA warp)
     uint64_t aempty[2 * kMaxASlots];   // operand buffer free again (tcgen05.commit); decode: [group][buffer]
     uint64_t accfull;
     uint64_t accempty;
-    uint64_t x8full[kMaxStages];       // decode, in-kernel split: the stage's e5m2 pieces are written (96 arrivals)
+    uint64_t x8full[kMaxStages];       // decode: the stage's e5m2 pieces are in place (128 splitter threads, or TMA)
     uint64_t depready;                 // the grid this launch depends on has completed (activations may be read)
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -361,11 +368,11 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
 // 16-byte chunks (i = 0..3) of the group, the 4 bytes holding k = 8i+c, 8i+c+1, and produce 8 bytes
 // (slots 16h+8pc .. +7) per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
 // exact in f16): p = rn_e5m2(y); y -= p; four times.  `xt` is the stage's X tile (two swizzled 64-k
-// atoms), followed by the piece tile.  Thread `tid` of `nthreads` takes the tasks tid, tid + nthreads, ...
+// atoms), `x8t` its piece tile.  Thread `tid` of `nthreads` takes the tasks tid, tid + nthreads, ...
 // Small tasks on purpose: 16 per token row spread the work over all four epilogue warps, one warp per
 // scheduler, so that no scheduler's decode warps are slowed more than the others'.
-__device__ __forceinline__ void split_activations(const GemmArgs& a, int am, uint8_t* xt, int ntok, int tid, int nthreads) {
-    uint8_t* x8t = xt + 2 * a.x_atom_bytes;
+__device__ __forceinline__ void split_activations(const GemmArgs& a, int am, const uint8_t* xt, uint8_t* x8t, int ntok, int tid,
+                                                  int nthreads) {
     const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 16;
     for (int task = tid; task < ntasks; task += nthreads) {
         const int r = task >> 4, q4 = (task >> 2) & 3, h = (task >> 1) & 1, pc = task & 1;
@@ -422,9 +429,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     const uint32_t w_addr = base;                                        // ring of W_base tiles
-    const uint32_t xr_off = a.n_w * a.w_stage_bytes;                     // ring of activation tiles
-    const uint32_t xr_addr = base + xr_off;
-    const uint32_t bits_off = xr_off + a.n_x * a.xr_bytes;               // sign-word slots
+    const uint32_t x_off = a.n_w * a.w_stage_bytes;                      // ring of bf16 activation tiles
+    const uint32_t x_addr = base + x_off;
+    const uint32_t x8_off = x_off + a.n_x * a.x_tile_bytes;              // ring of e5m2 piece tiles (decode)
+    const uint32_t x8_addr = base + x8_off;
+    const uint32_t bits_off = x8_off + a.n_x8 * a.x8_atom_bytes;         // sign-word slots
     const uint32_t bits_addr = base + bits_off;
     uint8_t* bits_ptr = smem + bits_off;
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + bits_off + kBitSlots * a.bslot_bytes);
@@ -471,8 +480,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             // tiled schedule: the stage's activation tile (same slot index, queued by the activation
             // stream) completes on this barrier too
             mbar_arrive_expect_tx(bar, a.w_stage_bytes + ((kDec || BD_KNOB(32)) ? 0u : 2 * a.x_atom_bytes));
-            tma_load_2d(dst, &tmW, bar, k0, u.n0);
-            tma_load_2d(dst + a.w_atom_bytes, &tmW, bar, k0 + kAtomK, u.n0);
+            tma_load_3d(dst, &tmW, bar, 0, u.n0, k0 / kAtomK);   // both 64-k atoms of the tile
         }
         if (with_bits) {
             const uint32_t bbar = smem_u32(&ctl->bfull[bslot]);
@@ -485,11 +493,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
     };
 
-    // One epilogue thread's share (tasks tid, tid + 128, ...) of the in-kernel activation split of slot `st`.
-    auto do_split = [&](int st, int ntok, int tid) {
-        split_activations(a, am, smem + xr_off + st * a.xr_bytes, ntok, tid, 128);
+    // One epilogue thread's share (tasks tid, tid + 128, ...) of the in-kernel activation split: bf16 tile
+    // in slot `xs` of its ring -> piece tile in slot `x8s` of its ring.
+    auto do_split = [&](int xs, int x8s, int ntok, int tid) {
+        split_activations(a, am, smem + x_off + xs * a.x_tile_bytes, smem + x8_off + x8s * a.x8_atom_bytes, ntok, tid, 128);
         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
-        mbar_arrive(smem_u32(&ctl->x8full[st]));
+        mbar_arrive(smem_u32(&ctl->x8full[x8s]));
+        mbar_arrive(smem_u32(&ctl->xempty[xs]));   // this thread is done reading the bf16 tile
     };
 
     if (threadIdx.x == 0) {
@@ -497,8 +507,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             mbar_init(smem_u32(&ctl->wfull[s]), 1);
             mbar_init(smem_u32(&ctl->wempty[s]), 1);
             mbar_init(smem_u32(&ctl->xfull[s]), 1);
-            mbar_init(smem_u32(&ctl->xempty[s]), kDec ? 3 : 1);   // decode: three MMA issuers release a tile
-            mbar_init(smem_u32(&ctl->x8full[s]), 128);
+            mbar_init(smem_u32(&ctl->xempty[s]), (kDec && convert) ? 129 : 1);   // base issuer (+ the splitter threads)
+            mbar_init(smem_u32(&ctl->x8full[s]), (kDec && convert) ? 128 : 1);   // splitter threads, or one TMA load
+            mbar_init(smem_u32(&ctl->x8empty[s]), 2);                            // the two delta issuers
         }
         for (int s = 0; s < kBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
@@ -544,9 +555,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //    of their own, shallower ring.
         // Neither stream may block the other, so the warp polls both rings and sleeps on a short
         // suspended wait when neither can advance.
-        ItemIter wi(it), xi(it);
-        int stage = 0, xslot = 0, bslot = 0;
-        uint32_t phase = 0, xphase = 0, bphase = 0;
+        ItemIter wi(it), xi(it), pi(it);
+        int stage = 0, xslot = 0, pslot = 0, bslot = 0;
+        uint32_t phase = 0, xphase = 0, pphase = 0, bphase = 0;
         bool ok = true, dep_ok = false;
         bool hold = kDec && a.hold_prefetch != 0;
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
@@ -554,6 +565,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         bool more_w = wi.next();
         bool more_x = xi.next();
         if (more_x) ux = unit_info(a, xi.unit);
+        // e5m2 piece tiles written by the pre-pass kernel (decode schedule, many token rows per unit)
+        bool more_p = load_x8 && pi.next();
+        Unit up{};
+        if (more_p) up = unit_info(a, pi.unit);
         if (more_w) {
             // queued by thread 0 in the prologue: W stage 0, sign-word slot 0
             bslot = 1 % kBitSlots; bphase = (kBitSlots == 1) ? 1u : 0u;
@@ -564,24 +579,30 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (more_w && wi.first) uw = unit_info(a, wi.unit);
         }
         const uint32_t depbar = smem_u32(&ctl->depready);
-        const uint32_t x_tx = BD_KNOB(32) ? 0u : 2 * a.x_atom_bytes + (load_x8 ? a.x8_atom_bytes : 0u);
+        const uint32_t x_tx = BD_KNOB(32) ? 0u : a.x_tile_bytes;
         long long t_idle = 0;
         int idle = 0;
-        while (more_w || more_x) {
+#ifdef BD_TRACE
+        long long idle_b = 0, idle_w = 0;
+#endif
+        BD_ACC_DECL(t_x); BD_ACC_DECL(t_p); BD_ACC_DECL(t_w); BD_ACC_DECL(n_iter);
+        while (more_w || more_x || more_p) {
             bool did = false;
+#ifdef BD_TRACE
+            ++n_iter;
+#endif
+            BD_ACC_BEGIN(tx0);
             if (more_x) {
                 if (!dep_ok) dep_ok = warp_all(mbar_test_wait(depbar, 0));
                 const uint32_t xebar = kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot]);
                 if (dep_ok && warp_all(mbar_test_wait(xebar, xphase ^ 1))) {
                     if (elect_one()) {
                         const uint32_t bar = kDec ? smem_u32(&ctl->xfull[xslot]) : smem_u32(&ctl->wfull[xslot]);
-                        const uint32_t dst = xr_addr + xslot * a.xr_bytes;
+                        const uint32_t dst = x_addr + xslot * a.x_tile_bytes;
                         const int k0 = xi.p * kPairK;
                         if (x_tx) {
                             if (kDec) mbar_arrive_expect_tx(bar, x_tx);
-                            tma_load_2d(dst, &tmX, bar, k0, ux.xrow0);
-                            tma_load_2d(dst + a.x_atom_bytes, &tmX, bar, k0 + kAtomK, ux.xrow0);
-                            if (load_x8) tma_load_2d(dst + 2 * a.x_atom_bytes, &tmX8, bar, k0, ux.tenant0 * kPieces * am);
+                            tma_load_3d(dst, &tmX, bar, 0, ux.xrow0, k0 / kAtomK);   // both 64-k atoms
                         } else if (kDec) {
                             mbar_arrive(bar);
                         }
@@ -593,6 +614,29 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
+            BD_ACC_END(t_x, tx0);
+            BD_ACC_BEGIN(tp0);
+            if (more_p) {
+                if (!dep_ok) dep_ok = warp_all(mbar_test_wait(depbar, 0));
+                if (dep_ok && warp_all(mbar_test_wait(smem_u32(&ctl->x8empty[pslot]), pphase ^ 1))) {
+                    if (elect_one()) {
+                        const uint32_t bar = smem_u32(&ctl->x8full[pslot]);
+                        if (BD_KNOB(32)) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
+                            tma_load_2d(x8_addr + pslot * a.x8_atom_bytes, &tmX8, bar, pi.p * kPairK, up.tenant0 * kPieces * am);
+                        }
+                    }
+                    __syncwarp();
+                    if (++pslot == a.n_x8) { pslot = 0; pphase ^= 1; }
+                    more_p = pi.next();
+                    if (more_p && pi.first) up = unit_info(a, pi.unit);
+                    did = true;
+                }
+            }
+            BD_ACC_END(t_p, tp0);
+            BD_ACC_BEGIN(tw0);
             if (more_w && hold) {
                 // The first sign-word load of a tile pulls whole 128-byte lines (the signs of 1024 k) out of
                 // DRAM; until it has landed, further weight requests would only queue in front of it.
@@ -602,8 +646,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const bool need_slot = wi.first || !(wi.p & 1);
                 if ((!need_slot || warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) &&
                     warp_all(mbar_test_wait(smem_u32(&ctl->wempty[stage]), phase ^ 1))) {
+                    BD_ACC_BEGIN(ti);
                     if (elect_one()) issue_weights_raw(uw, wi.p, stage, bslot, need_slot);
                     __syncwarp();
+                    BD_ACC_END(w_bempty, ti);
                     BD_TL(0);
                     if (need_slot && ++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
                     if (++stage == a.n_w) { stage = 0; phase ^= 1; }
@@ -612,11 +658,18 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
+            BD_ACC_END(t_w, tw0);
             if (did) {
                 idle = 0;
                 continue;
             }
             // Nothing can advance: a short suspended wait (tens of ns) on one ring, then look at both again.
+#ifdef BD_TRACE
+            if (more_w && !hold) {
+                const bool ns = wi.first || !(wi.p & 1);
+                if (ns && !mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1)) ++idle_b; else ++idle_w;
+            }
+#endif
             BD_ACC_BEGIN(te);
             if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 64u);
             else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 64u);
@@ -637,6 +690,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         (void)ok;
         BD_STAMP(3);
         BD_ACC_STORE(19, w_empty); BD_ACC_STORE(20, w_bempty);
+#ifdef BD_TRACE
+        BD_ACC_STORE(15, idle_b * 1965); BD_ACC_STORE(29, idle_w * 1965);
+        BD_ACC_STORE(4, t_x); BD_ACC_STORE(5, t_p); BD_ACC_STORE(30, t_w); BD_ACC_STORE(31, n_iter * 1965);
+#endif
     } else if (warp == kWarpMma) {
         // -------------------------------------------------------------- MMA issuer
         // Warp-uniform loop, one elected lane issues: descriptors and predicates then live in
@@ -674,14 +731,16 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 {
                     BD_ACC_BEGIN(tf);
                     ok = warp_all(wait_bar(smem_u32(&ctl->wfull[stage]), phase, abort_flag, 4));
-                    if (kDec && ok) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
                     BD_ACC_END(w_full, tf);
+                    BD_ACC_BEGIN(tf2);
+                    if (kDec && ok) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
+                    BD_ACC_END(w_afull, tf2);
                     if (!ok) break;
                 }
                 if (item == 0) BD_STAMP(4);
                 BD_TL(1);
                 const uint32_t wbase = w_addr + stage * a.w_stage_bytes;
-                const uint32_t xbase = xr_addr + xslot * a.xr_bytes;
+                const uint32_t xbase = x_addr + xslot * a.x_tile_bytes;
                 const uint64_t wdesc = desc0 + (wbase >> 4);
                 const uint64_t xdesc = desc0 + (xbase >> 4);
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
@@ -695,9 +754,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     }
                     // decode schedule: nothing else reads the W_base tile, hand it back as soon as these MMAs
                     // have completed
-                    if (kDec) tc_commit(smem_u32(&ctl->wempty[stage]));
+                    if (kDec) {
+                        tc_commit(smem_u32(&ctl->wempty[stage]));
+                        tc_commit(smem_u32(&ctl->xempty[xslot]));
+                    }
                 }
-                if (kDec && BD_KNOB(4) && elect_one()) tc_commit(smem_u32(&ctl->wempty[stage]));
+                if (kDec && BD_KNOB(4) && elect_one()) {
+                    tc_commit(smem_u32(&ctl->wempty[stage]));
+                    tc_commit(smem_u32(&ctl->xempty[xslot]));
+                }
                 __syncwarp();
                 BD_ACC_END(w_ib, tib);
                 if constexpr (kDec) {
@@ -730,8 +795,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     }
                 }
                 if (!ok) break;
-                if (elect_one()) tc_commit(kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[stage]));
-                __syncwarp();
+                if (!kDec) {
+                    if (elect_one()) tc_commit(smem_u32(&ctl->wempty[stage]));
+                    __syncwarp();
+                }
                 if (++stage == a.n_w) { stage = 0; phase ^= 1; }
                 if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
             }
@@ -745,8 +812,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     } else if (warp >= kWarpDelta0 && warp < kWarpDelta0 + 2) {
         // ------------------------------------------------- delta issuers (decode schedule)
         // Warp 2+g serves decode group g (tenants j = g, g+2, ... of the unit).  Per 128-k stage it
-        //  * (few token rows per unit) splits those tenants' activations into e5m2 pieces itself,
-        //    reading the bf16 X tile and writing the swizzled piece tile of the stage, and
+        //  * waits for the stage's e5m2 piece tile, and
         //  * per 64-k half waits, on a named barrier, for the group's decode warps to have filled the
         //    operand buffer in tensor memory, issues that half's MMAs and commits the buffer's release.
         // Nothing else writes those tenants' accumulators, so their summation order is fixed.
@@ -754,33 +820,36 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             const int g = warp - kWarpDelta0;
             const uint32_t idesc_delta = make_idesc_e5m2(kTileN, (uint32_t)a.Nd);
             const uint64_t desc0 = make_smem_desc_sw128(0);
-            const uint32_t x_atom16 = a.x_atom_bytes >> 4;
             const uint32_t ten_rows16 = (uint32_t)(kPieces * am) * 8u;   // rows per tenant x 128 B >> 4
             const uint32_t amask = (uint32_t)a.a_slots - 1;
             const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
             int xslot = 0;
             uint32_t xphase = 0, accphase = 0, item = 0;
             bool ok = true;
-            BD_TL_DECL;
+            BD_TL_DECL; BD_ACC_DECL(d_x8); BD_ACC_DECL(d_nb);
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
                 ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
                 if (!ok) break;
                 tc_fence_after();
                 for (int p = p0; p < p1 && ok; ++p) {
-                    // few token rows per unit: the e5m2 pieces are written by the epilogue warps (x8full);
-                    // otherwise they arrive with the activation tile
-                    ok = warp_all(wait_bar(convert ? smem_u32(&ctl->x8full[xslot]) : smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
+                    // the stage's e5m2 pieces: written by the epilogue warps (few token rows per unit) or loaded
+                    // from the pre-pass kernel's output
+                    BD_ACC_BEGIN(t8);
+                    ok = warp_all(wait_bar(smem_u32(&ctl->x8full[xslot]), xphase, abort_flag, 12));
+                    BD_ACC_END(d_x8, t8);
                     if (!ok) break;
                     if (g == 0) BD_TL(2);
-                    const uint64_t x8desc = desc0 + ((xr_addr + xslot * a.xr_bytes) >> 4) + 2 * x_atom16;
+                    const uint64_t x8desc = desc0 + ((x8_addr + xslot * a.x8_atom_bytes) >> 4);
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
                     for (int half = 0; half < a.halves; ++half, ++item) {
                         const uint32_t slot = item & amask;
                         if (*abort_flag) { ok = false; break; }
                         // The group's 128 decode threads arrive here once the buffer is filled (or when they
                         // give up after an abandoned wait, see the end of the decode role).
+                        BD_ACC_BEGIN(tn);
                         named_bar_sync(kBarAFull0 + g * 4 + (int)slot, 160);
+                        BD_ACC_END(d_nb, tn);
                         if (*abort_flag) { ok = false; break; }
                         tc_fence_after();
                         if (g == 0) BD_TL(2);
@@ -813,9 +882,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         __syncwarp();
                     }
                     if (!ok) break;
-                    if (elect_one()) tc_commit(smem_u32(&ctl->xempty[xslot]));
+                    if (elect_one()) tc_commit(smem_u32(&ctl->x8empty[xslot]));
                     __syncwarp();
-                    if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
+                    if (++xslot == a.n_x8) { xslot = 0; xphase ^= 1; }
                 }
                 if (!ok) break;
                 if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
@@ -823,6 +892,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 accphase ^= 1;
                 (void)ashift;
             }
+            if (g == 0) { BD_ACC_STORE(13, d_x8); BD_ACC_STORE(14, d_nb); }
         }
     } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {
         // ------------------------------------------- sign decode -> tensor memory
@@ -1054,19 +1124,23 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const bool splitter = kDec && convert;
         ItemIter si(it);
         bool more_s = splitter && si.next();
-        int sslot = 0, n_split = 0, seg_end = 0;
-        uint32_t sphase = 0;
+        int sslot = 0, s8slot = 0, n_split = 0, seg_end = 0;
+        uint32_t sphase = 0, s8phase = 0;
         Unit us{};
         if (more_s) us = unit_info(a, si.unit);
         auto split_next = [&](bool block) -> bool {
+            // needs the bf16 tile landed and a free piece tile
             const uint32_t bar = smem_u32(&ctl->xfull[sslot]);
+            const uint32_t bar8 = smem_u32(&ctl->x8empty[s8slot]);
             if (block) {
                 if (!wait_bar(bar, sphase, abort_flag, 13)) return false;
-            } else if (!warp_all(mbar_test_wait(bar, sphase))) {
+                if (!wait_bar(bar8, s8phase ^ 1, abort_flag, 14)) return false;
+            } else if (!warp_all(mbar_test_wait(bar, sphase) && mbar_test_wait(bar8, s8phase ^ 1))) {
                 return false;
             }
-            do_split(sslot, us.ntok, etid);
+            do_split(sslot, s8slot, us.ntok, etid);
             if (++sslot == a.n_x) { sslot = 0; sphase ^= 1; }
+            if (++s8slot == a.n_x8) { s8slot = 0; s8phase ^= 1; }
             ++n_split;
             more_s = si.next();
             if (more_s && si.first) us = unit_info(a, si.unit);
@@ -1213,7 +1287,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
 #ifdef BD_TRACE
-    cfg.dynamicSmemBytes = smem_bytes + 2816;   // room for the stamps behind the control block
+    cfg.dynamicSmemBytes = smem_bytes + 256 + 5 * BD_TLN * 8;   // room for the stamps behind the control block
 #else
     cfg.dynamicSmemBytes = smem_bytes;
 #endif

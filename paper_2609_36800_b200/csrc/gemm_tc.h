@@ -15,9 +15,9 @@ struct GemmArgs {
     int m_tiles, groups, P, whole_units;
     int T;             // work items (< 2^30)
     int q, r;          // T = q * grid + r
-    int n_w, n_x, a_slots, halves;
+    int n_w, n_x, n_x8, a_slots, halves;
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
-    uint32_t w_stage_bytes, xr_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
+    uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
     const float* alpha;
@@ -32,8 +32,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.decode = p.decode; a.convert = p.convert; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
     a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
     a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.q = (int)(p.T / p.grid); a.r = (int)(p.T % p.grid); a.whole_units = p.whole_units;
-    a.n_w = p.n_w; a.n_x = p.n_x; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
-    a.w_stage_bytes = p.w_stage_bytes; a.xr_bytes = p.xr_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
+    a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
+    a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;
     a.col_delta = p.col_delta; a.col_a = p.col_a;

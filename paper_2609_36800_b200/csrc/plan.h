@@ -43,10 +43,11 @@ struct Plan {
     long long T;       // total k-pair work items = units * P
     int grid;
     int n_w;           // ring of W_base tiles (128 rows x 128 k of bf16 each)
-    int n_x;           // ring of activation tiles (X, and in the decode schedule its e5m2 pieces)
+    int n_x;           // ring of bf16 activation tiles
+    int n_x8;          // decode: ring of e5m2 piece tiles
     int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
-    uint32_t w_stage_bytes, xr_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
+    uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
     uint32_t col_base, col_delta, col_a;
     size_t slot_floats;   // floats of one partial-result slot: 128 rows x tokens per unit
     size_t ws_header_bytes;   // arrival counters: one u32 per work unit
@@ -120,25 +121,33 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
     p.w_stage_bytes = 2 * p.w_atom_bytes;
-    p.xr_bytes = 2 * p.x_atom_bytes + p.x8_atom_bytes;
+    p.x_tile_bytes = 2 * p.x_atom_bytes;
     p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
-    // Shared memory: a ring of W_base tiles, a ring of activation tiles, the sign-word slots.  W_base
-    // comes from DRAM (latency ~1.5 us under load) and a tile is released as soon as the base MMAs have
-    // read it; the activations come from L2 and are small, but a tile stays in use until the last delta
-    // MMA of its stage has completed.  Hence two rings with their own depths in the decode schedule
-    // (few activation slots, every remaining byte to W_base); the tiled schedule keeps them equal.
+    // Shared memory: rings of W_base tiles, of bf16 activation tiles and (decode) of e5m2 piece tiles, and
+    // the sign-word slots.  W_base comes from DRAM (latency ~1.5 us under load); it and the bf16
+    // activations are released as soon as the base MMAs have read them.  The piece tiles come from L2 (or
+    // are written in place by the in-kernel split), but stay in use until the last delta MMA of their
+    // stage has completed, which is the longest hold of all: three of them.  Every remaining byte goes to
+    // W_base.  The tiled schedule keeps one ring (activation tile s lives and dies with W_base tile s).
     const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
     if (p.decode) {
-        p.n_x = (p.xr_bytes > 16 * 1024) ? 2 : 3;
-        p.n_w = (avail - p.n_x * (int)p.xr_bytes) / (int)p.w_stage_bytes;
+        p.n_x8 = 3;
+        p.n_x = (p.x_tile_bytes <= 4 * 1024) ? 3 : 2;
+        p.n_w = (avail - p.n_x * (int)p.x_tile_bytes - p.n_x8 * (int)p.x8_atom_bytes) / (int)p.w_stage_bytes;
+        if (p.n_w < 2) {
+            p.n_x8 = 2;
+            p.n_w = (avail - p.n_x * (int)p.x_tile_bytes - p.n_x8 * (int)p.x8_atom_bytes) / (int)p.w_stage_bytes;
+        }
         if (p.n_w > 6) p.n_w = 6;
     } else {
-        p.n_w = avail / (int)(p.w_stage_bytes + p.xr_bytes);
+        p.n_x8 = 0;
+        p.n_w = avail / (int)(p.w_stage_bytes + p.x_tile_bytes);
         if (p.n_w > kMaxStages) p.n_w = kMaxStages;
         p.n_x = p.n_w;
     }
     if (p.n_w < 2) return p;
-    p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.xr_bytes + kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
+    p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
+                   kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
     // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
     if (p.smem_bytes < 120 * 1024) p.smem_bytes = 120 * 1024;
 
