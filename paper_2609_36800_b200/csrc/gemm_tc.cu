@@ -563,10 +563,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
         Unit uw{}, ux{};
         bool more_w = wi.next();
-        bool more_x = xi.next();
+        // (decode schedule, many token rows per unit: the activation tiles are queued by two of the otherwise
+        // idle epilogue warps, so that this warp only serves the weight stream)
+        bool more_x = (!kDec || convert) && xi.next();
         if (more_x) ux = unit_info(a, xi.unit);
         // e5m2 piece tiles written by the pre-pass kernel (decode schedule, many token rows per unit)
-        bool more_p = load_x8 && pi.next();
+        bool more_p = false;
         Unit up{};
         if (more_p) up = unit_info(a, pi.unit);
         if (more_w) {
@@ -1121,14 +1123,55 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         // thread), as soon as the stage's activation tile has landed.  Each warp walks the items on its
         // own; x8full[slot] counts all 128 threads.  Items of the current tile are split with blocking
         // waits (the tile cannot complete without them), later ones whenever there is nothing else to do.
-        const bool splitter = kDec && convert;
+        // With many token rows per unit there is nothing to split (a pre-pass kernel has written the
+        // pieces), but the same walk lets epilogue warp 0 queue the bf16 activation tiles and warp 1 the
+        // piece tiles, each into its own ring, instead of the producer warp.
+        const int ew = warp - epi_first_warp;
+        const bool splitter = kDec && (convert || ew < 2);
         ItemIter si(it);
         bool more_s = splitter && si.next();
+        if (more_s && !convert) grid_dependency_wait();   // activations and pieces come from earlier kernels
         int sslot = 0, s8slot = 0, n_split = 0, seg_end = 0;
         uint32_t sphase = 0, s8phase = 0;
         Unit us{};
         if (more_s) us = unit_info(a, si.unit);
         auto split_next = [&](bool block) -> bool {
+            if (!convert) {
+                // queue one tile load: bf16 activations (warp 0) or pieces (warp 1), when its slot is free
+                const uint32_t ebar = (ew == 0) ? smem_u32(&ctl->xempty[sslot]) : smem_u32(&ctl->x8empty[s8slot]);
+                const uint32_t epar = ((ew == 0) ? sphase : s8phase) ^ 1;
+                if (block) {
+                    if (!warp_all(wait_bar(ebar, epar, abort_flag, 13))) return false;
+                } else if (!warp_all(mbar_test_wait(ebar, epar))) {
+                    return false;
+                }
+                if (elect_one()) {
+                    if (ew == 0) {
+                        const uint32_t bar = smem_u32(&ctl->xfull[sslot]);
+                        if (BD_KNOB(32)) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, a.x_tile_bytes);
+                            tma_load_3d(x_addr + sslot * a.x_tile_bytes, &tmX, bar, 0, us.xrow0, si.p * (kPairK / kAtomK));
+                        }
+                    } else {
+                        const uint32_t bar = smem_u32(&ctl->x8full[s8slot]);
+                        if (BD_KNOB(32)) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
+                            tma_load_2d(x8_addr + s8slot * a.x8_atom_bytes, &tmX8, bar, si.p * kPairK, us.tenant0 * kPieces * am);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (++sslot == a.n_x) { sslot = 0; sphase ^= 1; }
+                if (++s8slot == a.n_x8) { s8slot = 0; s8phase ^= 1; }
+                ++n_split;
+                more_s = si.next();
+                if (more_s && si.first) us = unit_info(a, si.unit);
+                return true;
+            }
             // needs the bf16 tile landed and a free piece tile
             const uint32_t bar = smem_u32(&ctl->xfull[sslot]);
             const uint32_t bar8 = smem_u32(&ctl->x8empty[s8slot]);
