@@ -464,7 +464,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const int hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
     SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
     int unit, p0, p1;
-    const bool load_x8 = kDec && !convert;
 
     // Queues the weight loads of one item: its W_base tile into `stage` of the W ring and, if `with_bits`,
     // the sign words of its k-pair into sign-word slot `bslot`.  One thread.
