@@ -366,11 +366,15 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
 // r, 32-k group q4 of the stage, half h of the group's byte slots, pair pc of the half's four k classes.
 // Slot 4c+i holds k = c + 8i, so the task's classes c = 4h+2pc, 4h+2pc+1 need, from each of the four
 // 16-byte chunks (i = 0..3) of the group, the 4 bytes holding k = 8i+c, 8i+c+1, and produce 8 bytes
-// (slots 16h+8pc .. +7) per piece.  Arithmetic on packed f16 pairs (a bf16 value in the e5m2 range is
-// exact in f16): p = rn_e5m2(y); y -= p; four times.  `xt` is the stage's X tile (two swizzled 64-k
-// atoms), `x8t` its piece tile.  Thread `tid` of `nthreads` takes the tasks tid, tid + nthreads, ...
-// Small tasks on purpose: 16 per token row spread the work over all four epilogue warps, one warp per
-// scheduler, so that no scheduler's decode warps are slowed more than the others'.
+// (slots 16h+8pc .. +7) per piece.
+// The pieces are taken by TRUNCATION on packed f16 pairs (a bf16 value in the e5m2 range is exact in f16,
+// and an e5m2 number is the high byte of an f16 number): p = y with its low byte cleared, y -= p (exact).
+// A bf16 value has 8 significant bits and every piece removes the top three of what is left, so the third
+// piece leaves nothing and the fourth is zero; no conversion instruction is needed (they are slow enough
+// to hold up the decode warps that share a scheduler with the splitting warp).
+// `xt` is the stage's X tile (two swizzled 64-k atoms), `x8t` its piece tile.  Thread `tid` of `nthreads`
+// takes the tasks tid, tid + nthreads, ...  Small tasks on purpose: 16 per token row spread the work over
+// all four epilogue warps, one warp per scheduler.
 __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, const uint8_t* xt, uint8_t* x8t, int ntok, int tid,
                                                   int nthreads) {
     const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 16;
@@ -378,26 +382,29 @@ __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, con
         const int r = task >> 4, q4 = (task >> 2) & 3, h = (task >> 1) & 1, pc = task & 1;
         const int j = r / am, t = r - j * am;
         const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8 + pc * 4;
-        __half2 y[4];   // y[i]: k = 8i + 4h + 2pc, +1
+        uint32_t y[4];   // y[i]: f16 pair, k = 8i + 4h + 2pc, +1
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
             const uint32_t v = *reinterpret_cast<const uint32_t*>(src + chunk * 16);
-            y[i] = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+            const __half2 hv = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+            y[i] = *reinterpret_cast<const uint32_t*>(&hv);
         }
 #pragma unroll
         for (int q = 0; q < kPieces; ++q) {
-            uint32_t pk[4];
+            uint32_t pq[4];   // byte 1 / byte 3: the e5m2 piece of k / k+1
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const __nv_fp8x2_storage_t p8 =
-                    __nv_cvt_halfraw2_to_fp8x2(static_cast<__half2_raw>(y[i]), __NV_SATFINITE, __NV_E5M2);
-                y[i] = __hsub2(y[i], __half2(__nv_cvt_fp8x2_to_halfraw2(p8, __NV_E5M2)));
-                pk[i] = p8;
+                pq[i] = y[i] & 0xFF00FF00u;
+                if (q + 1 < kPieces) {
+                    const __half2 d = __hsub2(*reinterpret_cast<const __half2*>(&y[i]), *reinterpret_cast<const __half2*>(&pq[i]));
+                    y[i] = *reinterpret_cast<const uint32_t*>(&d);
+                }
             }
-            const uint32_t r01 = pk[0] | (pk[1] << 16);
-            const uint32_t r23 = pk[2] | (pk[3] << 16);
-            const uint2 w = make_uint2(__byte_perm(r01, r23, 0x6420), __byte_perm(r01, r23, 0x7531));
+            // bytes (i = 0..3) of element k, then of element k+1
+            const uint32_t t01 = __byte_perm(pq[0], pq[1], 0x7351);   // [p0.b1, p1.b1, p0.b3, p1.b3]
+            const uint32_t t23 = __byte_perm(pq[2], pq[3], 0x7351);
+            const uint2 w = make_uint2(__byte_perm(t01, t23, 0x5410), __byte_perm(t01, t23, 0x7632));
             const int r8 = j * (kPieces * am) + q * am + t;
             *reinterpret_cast<uint2*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16) + pc * 8) = w;
         }

@@ -139,6 +139,16 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             p.n_w = (avail - p.n_x * (int)p.x_tile_bytes - p.n_x8 * (int)p.x8_atom_bytes) / (int)p.w_stage_bytes;
         }
         if (p.n_w > 6) p.n_w = 6;
+        if (p.convert && p.n_w >= 3) {
+            // Few token rows per unit: the activation and piece tiles are small.  Three W_base stages are
+            // enough (deeper rings measured no faster); the rest buys activation slots, so that the epilogue
+            // warps can split several stages ahead -- during the start-up of a launch, when nothing else
+            // runs, they get through most of a short CTA's stages.
+            p.n_w = 3;
+            int n = (avail - p.n_w * (int)p.w_stage_bytes) / (int)(p.x_tile_bytes + p.x8_atom_bytes);
+            if (n > kMaxStages) n = kMaxStages;
+            if (n > p.n_x) { p.n_x = n; p.n_x8 = n; }
+        }
     } else {
         p.n_x8 = 0;
         p.n_w = avail / (int)(p.w_stage_bytes + p.x_tile_bytes);
