@@ -87,6 +87,13 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.
  * Asynchronous on the stream; a kernel-side wait that expires is reported by
  * bitdelta_last_device_status, not here.
+ * Early start: the kernel is queued so that it may begin (prologue, prefetch of
+ * W_base, bits and alpha) while the kernel queued on the stream just before it
+ * is still running; it reads X and writes Y and the workspace only after that
+ * kernel has completed.  W_base, bits and alpha must therefore not be produced
+ * by the kernel queued directly before the call (weights are static in the
+ * intended use); X may be.  BITDELTA_EARLY_START=0 in the environment turns
+ * the early start off.
  */
 int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
                   void* Y, int B, int m, int N, int K,
