@@ -43,6 +43,7 @@ def _load():
         lib.oracle_unpack.argtypes = [p, p, c_int, c_int, c_int]
         lib.oracle_gemm.argtypes = [p, p, p, p, p, c_int, c_int, c_int, c_int]
         lib.oracle_gemm_at.argtypes = [p, p, p, p, p, c_int, p, c_int, c_int, c_int, c_int]
+        lib.oracle_compress.argtypes = [p, p, p, p, c_int, c_int, c_int]
         _lib = lib
     return _lib
 
@@ -84,6 +85,20 @@ def unpack(bits: np.ndarray) -> np.ndarray:
     out = np.empty((B, N, Wn * 32), dtype=np.int8)
     _load().oracle_unpack(_ptr(bits), _ptr(out), B, N, Wn * 32)
     return out
+
+
+def compress(W_fine: np.ndarray, W_base: np.ndarray):
+    """W_fine uint16 [B,N,K] and W_base uint16 [N,K] (bf16 bit patterns) -> (bits uint32 [B,N,K/32],
+    alpha float32 [B]): bit = (W_fine - W_base > 0), alpha = mean |W_fine - W_base| per tenant."""
+    wf = _as(W_fine, np.uint16)
+    wb = _as(W_base, np.uint16)
+    B, N, K = wf.shape
+    if wb.shape != (N, K) or K % 32:
+        raise ValueError("inconsistent shapes, or K not a multiple of 32")
+    bits = np.empty((B, N, K // 32), dtype=np.uint32)
+    alpha = np.empty((B,), dtype=np.float32)
+    _load().oracle_compress(_ptr(wf), _ptr(wb), _ptr(bits), _ptr(alpha), B, N, K)
+    return bits, alpha
 
 
 def _check(X, W, bits, alpha):

@@ -156,3 +156,36 @@ void oracle_gemm_at(const uint16_t *X, const uint16_t *W, const uint32_t *bits,
         out[i] = base + (double)alpha[b] * delta;
     }
 }
+
+/*
+ * compress: the step before the product -- derive a tenant's 1-bit delta from its fine-tuned weights
+ * (the BitDelta method the paper cites in its BitDelta paragraph; the paper itself does not spell it
+ * out, so this is the method's plain definition):
+ *
+ *   delta[b,n,k] = wf[b,n,k] - wb[n,k]                      (bf16 widened exactly to double)
+ *   bit  (k mod 32) of bits[b,n,k div 32] = [delta > 0]     (so zero and negative deltas decode to -1)
+ *   alpha[b] = (1 / (N K)) * sum_{n,k} |delta[b,n,k]|       (double, plain (n,k) order), rounded to fp32
+ *
+ * K must be a multiple of 32.
+ */
+void oracle_compress(const uint16_t *wf, const uint16_t *wb, uint32_t *bits, float *alpha, int B, int N, int K)
+{
+    int words = K / 32;
+    for (int b = 0; b < B; ++b) {
+        double sum_abs = 0.0;
+        for (int n = 0; n < N; ++n) {
+            for (int w = 0; w < words; ++w) {
+                uint32_t word = 0;
+                for (int j = 0; j < 32; ++j) {
+                    int k = 32 * w + j;
+                    double d = bf16_to_double(wf[((long long)b * N + n) * K + k]) - bf16_to_double(wb[(long long)n * K + k]);
+                    if (d > 0.0) word |= (1u << j);
+                    sum_abs += (d < 0.0) ? -d : d;
+                }
+                bits[((long long)b * N + n) * words + w] = word;
+            }
+        }
+        alpha[b] = (float)(sum_abs / ((double)N * (double)K));
+    }
+}
+

@@ -79,3 +79,24 @@ def make_signs(B: int, N: int, K: int, seed: int = 0) -> np.ndarray:
     """Dense S int8 [B,N,K] of +1/-1 (input of the packing step)."""
     rng = np.random.default_rng(seed)
     return (rng.integers(0, 2, size=(B, N, K), dtype=np.int8) * 2 - 1).astype(np.int8)
+
+
+def make_fine_weights(B: int, N: int, K: int, seed: int = 0, w_std: float = 0.02, delta_std: float = 0.004,
+                      zero_frac: float = 0.01):
+    """Inputs of the compress step: (W_fine[B,N,K] u16, W_base[N,K] u16), bf16 bit patterns.
+    W_fine = bf16(W_base + delta) with delta ~ N(0, delta_std) drawn per tenant (a fine-tune moves every
+    weight a little, either way); a fraction `zero_frac` of the positions keeps the base value exactly,
+    so that zero deltas (which must pack as -1) occur.  No arithmetic of the method lives here."""
+    rng = np.random.default_rng(seed)
+    Wf32 = np.float32(w_std) * rng.standard_normal((N, K), dtype=np.float32)
+    W = f32_to_bf16_bits(Wf32)
+    Wb = bf16_bits_to_f32(W)
+    fine = np.empty((B, N, K), dtype=np.uint16)
+    for b in range(B):
+        d = np.float32(delta_std) * rng.standard_normal((N, K), dtype=np.float32)
+        keep = rng.random((N, K)) < zero_frac
+        fb = f32_to_bf16_bits(Wb + d)
+        fb[keep] = W[keep]
+        fine[b] = fb
+    return fine, W
+

@@ -291,3 +291,84 @@ def test_seed0_statistics_match_stored_values(name):
     assert np.abs(Y).max() == pytest.approx(stats["y_absmax"], rel=1e-10)
     assert np.linalg.norm(Y) == pytest.approx(stats["y_fro"], rel=1e-10)
     assert Y.sum() == pytest.approx(stats["y_sum"], rel=1e-8)
+
+
+# ----------------------------------------------------------------------------------------------------
+# compress: bits = [W_fine - W_base > 0], alpha = mean |W_fine - W_base| (the BitDelta method the paper
+# cites in its BitDelta paragraph).  Pins that do not reuse the oracle's code.
+
+def _bf16(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def test_compress_hand_example():
+    # one tenant, one row of 32 weights; deltas chosen by hand (all exactly representable in bf16)
+    base = np.zeros(32, dtype=np.float32)
+    fine = np.zeros(32, dtype=np.float32)
+    base[:4] = [1.0, 2.0, -1.0, 0.5]
+    fine[:4] = [1.5, 1.0, -1.0, 0.75]          # deltas +0.5, -1.0, 0 (packs as 0), +0.25
+    fine[31] = -2.0                            # delta -2.0 at the word's top bit
+    bits, alpha = oracle.compress(_bf16(fine).reshape(1, 1, 32), _bf16(base).reshape(1, 32))
+    assert bits.shape == (1, 1, 1) and bits[0, 0, 0] == (1 << 0) | (1 << 3)
+    assert alpha[0] == np.float32((0.5 + 1.0 + 0.0 + 0.25 + 2.0) / 32)
+
+
+def test_compress_bit_order_and_row_indexing():
+    # a single positive delta at (b, n, k) must set exactly bit k%32 of word k//32 of row (b, n)
+    B, N, K = 2, 3, 96
+    base = np.zeros((N, K), dtype=np.float32)
+    for (b, n, k) in [(0, 0, 0), (1, 2, 95), (0, 1, 37), (1, 0, 64)]:
+        fine = np.zeros((B, N, K), dtype=np.float32)
+        fine[b, n, k] = 3.0
+        bits, alpha = oracle.compress(_bf16(fine), _bf16(base))
+        expect = np.zeros((B, N, K // 32), dtype=np.uint32)
+        expect[b, n, k // 32] = np.uint32(1) << np.uint32(k % 32)
+        assert np.array_equal(bits, expect)
+        expect_alpha = np.zeros(B, dtype=np.float32)
+        expect_alpha[b] = np.float32(3.0 / (N * K))
+        assert np.array_equal(alpha, expect_alpha)
+
+
+@pytest.mark.parametrize("shape", [(1, 4, 32), (3, 5, 64), (2, 16, 256)])
+def test_compress_matches_numpy(shape):
+    # independent statement with numpy: sign through np.packbits, mean through np.mean in float64
+    B, N, K = shape
+    fine, W = synth.make_fine_weights(B, N, K, seed=11)
+    bits, alpha = oracle.compress(fine, W)
+    d = synth.bf16_bits_to_f32(fine).astype(np.float64) - synth.bf16_bits_to_f32(W).astype(np.float64)[None]
+    assert (d == 0).any() and (d > 0).any() and (d < 0).any()
+    packed = np.packbits((d > 0).astype(np.uint8), axis=-1, bitorder="little").view(np.uint32)
+    assert np.array_equal(bits, packed.reshape(B, N, K // 32))
+    ref = np.abs(d).mean(axis=(1, 2))
+    assert np.allclose(alpha.astype(np.float64), ref, rtol=1e-7, atol=0)   # fp32 rounding of an fp64 mean
+
+
+def test_compress_invariants():
+    B, N, K = 2, 8, 64
+    fine, W = synth.make_fine_weights(B, N, K, seed=5)
+    bits, alpha = oracle.compress(fine, W)
+    wf = synth.bf16_bits_to_f32(fine)
+    wb = synth.bf16_bits_to_f32(W)
+    # the pair (W_base = 0, W_fine = delta) has the same signs and the same alpha whenever delta is a bf16 value
+    d = wf - wb[None]
+    d_bits = _bf16(d)
+    exact = synth.bf16_bits_to_f32(d_bits) == d
+    if exact.all():
+        b2, a2 = oracle.compress(d_bits, _bf16(np.zeros((N, K))))
+        assert np.array_equal(b2, bits) and np.array_equal(a2, alpha)
+    # doubling the delta around a zero base doubles alpha and keeps the bits
+    z = _bf16(np.zeros((N, K)))
+    b1, a1 = oracle.compress(_bf16(d), z)
+    b2, a2 = oracle.compress(_bf16(2.0 * synth.bf16_bits_to_f32(_bf16(d))), z)
+    assert np.array_equal(b1, b2) and np.allclose(a2, 2.0 * a1, rtol=1e-7)
+    # negating the delta flips exactly the bits of the non-zero deltas
+    dn = synth.bf16_bits_to_f32(_bf16(d))
+    b3, a3 = oracle.compress(_bf16(-dn), z)
+    nz = np.packbits((dn != 0).astype(np.uint8), axis=-1, bitorder="little").view(np.uint32).reshape(b1.shape)
+    assert np.array_equal(b1 ^ b3, nz) and np.array_equal(a1, a3)
+    # compress followed by unpack gives +1 exactly where the delta is positive
+    S = oracle.unpack(bits)
+    assert np.array_equal(S > 0, d > 0)
+    # tenants are independent
+    b4, a4 = oracle.compress(fine[1:], W)
+    assert np.array_equal(b4[0], bits[1]) and a4[0] == alpha[1]
