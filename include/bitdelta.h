@@ -57,6 +57,22 @@ int bitdelta_pack(const int8_t* S, uint32_t* bits, int B, int N, int K, void* cu
 int bitdelta_unpack(const uint32_t* bits, int8_t* S, int B, int N, int K, void* cuda_stream);
 
 /*
+ * Compress step (setup, before the GEMM; the BitDelta method the paper cites in its BitDelta paragraph):
+ * derives each tenant's 1-bit delta from its fine-tuned weights,
+ *   bits[b,n,w] bit j = [W_fine[b,n,32w+j] - W_base[n,32w+j] > 0]   (zero and negative deltas pack as -1),
+ *   alpha[b]          = mean over (n,k) of |W_fine[b,n,k] - W_base[n,k]|.
+ * W_fine : bf16 [B,N,K]; W_base : bf16 [N,K]; bits : uint32 [B,N,K/32] (output); alpha : fp32 [B] (output).
+ * workspace : at least bitdelta_compress_workspace_bytes(B,N,K) bytes of device memory, 8-byte aligned
+ *             (per-block partial sums; needs no preparation, is fully rewritten).
+ * The signs are exact (compared on the bf16 values); alpha is summed in double in a fixed order, so it is
+ * reproducible bit for bit and within ~1e-7 relative of the exact mean.  K must be a multiple of 32;
+ * W_fine, W_base and bits 16-byte aligned.  Asynchronous on the stream.
+ */
+size_t bitdelta_compress_workspace_bytes(int B, int N, int K);
+int bitdelta_compress(const void* W_fine, const void* W_base, uint32_t* bits, float* alpha, int B, int N, int K,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Scratch memory bitdelta_gemm needs for this problem size (may depend on the
  * shape only, never on the data).  Returns 0 for invalid shapes.
  */

@@ -9,6 +9,7 @@ missing.
 from . import synth  # noqa: F401
 from .binding import (  # noqa: F401
     BitDeltaError,
+    compress,
     gemm,
     gemm_host,
     gemm_host_arena_bytes,

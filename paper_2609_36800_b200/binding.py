@@ -17,7 +17,8 @@ STATUS_OK = 0
 STATUS_TIMEOUT = 7
 
 EXPORTS = (
-    "bitdelta_pack", "bitdelta_unpack", "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
+    "bitdelta_pack", "bitdelta_unpack", "bitdelta_compress_workspace_bytes", "bitdelta_compress",
+    "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
     "bitdelta_gemm", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
     "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
 )
@@ -46,6 +47,9 @@ def load_library():
     vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
     lib.bitdelta_pack.argtypes = [vp, vp, ci, ci, ci, vp]
     lib.bitdelta_unpack.argtypes = [vp, vp, ci, ci, ci, vp]
+    lib.bitdelta_compress_workspace_bytes.argtypes = [ci, ci, ci]
+    lib.bitdelta_compress_workspace_bytes.restype = sz
+    lib.bitdelta_compress.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, sz, vp]
     lib.bitdelta_gemm_workspace_bytes.argtypes = [ci, ci, ci, ci]
     lib.bitdelta_gemm_workspace_bytes.restype = sz
     lib.bitdelta_workspace_init.argtypes = [vp, sz, vp]
@@ -59,7 +63,7 @@ def load_library():
     lib.bitdelta_kernel_launch_count.restype = ctypes.c_ulonglong
     lib.bitdelta_status_string.argtypes = [ci]
     lib.bitdelta_status_string.restype = ctypes.c_char_p
-    for fn in ("bitdelta_pack", "bitdelta_unpack", "bitdelta_workspace_init", "bitdelta_gemm",
+    for fn in ("bitdelta_pack", "bitdelta_unpack", "bitdelta_compress", "bitdelta_workspace_init", "bitdelta_gemm",
                "bitdelta_gemm_simt", "bitdelta_gemm_noalloc", "bitdelta_gemm_host", "bitdelta_last_device_status"):
         getattr(lib, fn).restype = ci
     _lib = lib
@@ -105,6 +109,24 @@ def unpack(bits, stream=None):
     _check(load_library().bitdelta_unpack(_dev(bits, torch.int32, "bits"), ctypes.c_void_p(S.data_ptr()),
                                           B, N, Wn * 32, _stream_ptr(stream)), "bitdelta_unpack")
     return S
+
+
+def compress(W_fine, W_base, stream=None):
+    """Fine-tuned weights bf16 [B,N,K] and base weights bf16 [N,K] (device) -> (bits int32 storage
+    [B,N,K/32], alpha fp32 [B]): bit = (W_fine - W_base > 0), alpha = mean |W_fine - W_base| per tenant."""
+    import torch
+    lib = load_library()
+    B, N, K = W_fine.shape
+    if tuple(W_base.shape) != (N, K) or K % 32:
+        raise ValueError("inconsistent shapes, or K not a multiple of 32")
+    bits = torch.empty((B, N, K // 32), dtype=torch.int32, device=W_fine.device)
+    alpha = torch.empty((B,), dtype=torch.float32, device=W_fine.device)
+    nbytes = int(lib.bitdelta_compress_workspace_bytes(B, N, K))
+    ws = torch.empty(max(nbytes, 8), dtype=torch.uint8, device=W_fine.device)
+    _check(lib.bitdelta_compress(_dev(W_fine, torch.bfloat16, "W_fine"), _dev(W_base, torch.bfloat16, "W_base"),
+                                 ctypes.c_void_p(bits.data_ptr()), ctypes.c_void_p(alpha.data_ptr()), B, N, K,
+                                 ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream_ptr(stream)), "bitdelta_compress")
+    return bits, alpha
 
 
 def gemm_workspace_bytes(B: int, m: int, N: int, K: int) -> int:

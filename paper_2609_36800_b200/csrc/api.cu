@@ -200,6 +200,30 @@ int bitdelta_unpack(const uint32_t* bits, int8_t* S, int B, int N, int K, void* 
     return BITDELTA_OK;
 }
 
+size_t bitdelta_compress_workspace_bytes(int B, int N, int K) {
+    if (B <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return 0;
+    return (size_t)B * (size_t)bd::compress_blocks(N, K) * sizeof(double);
+}
+
+int bitdelta_compress(const void* W_fine, const void* W_base, uint32_t* bits, float* alpha, int B, int N, int K,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!W_fine || !W_base || !bits || !alpha) return BITDELTA_ERR_NULL;
+    if (B <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return BITDELTA_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(W_fine) | reinterpret_cast<uintptr_t>(W_base) | reinterpret_cast<uintptr_t>(bits)) & 15)
+        return BITDELTA_ERR_ALIGN;
+    if (!workspace || workspace_bytes < bitdelta_compress_workspace_bytes(B, N, K) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 7))
+        return BITDELTA_ERR_WORKSPACE;
+    DeviceInfo d;
+    int st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    if (bd::launch_compress(W_fine, W_base, bits, alpha, static_cast<double*>(workspace), B, N, K,
+                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches += 2;
+    return BITDELTA_OK;
+}
+
 size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K) {
     if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0) return 0;
     if ((K % 128) != 0) return 256;   // CUDA-core path: no scratch needed, keep the pointer non-NULL

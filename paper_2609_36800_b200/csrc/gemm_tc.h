@@ -66,6 +66,10 @@ cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream);
 // Plain kernels (pack / unpack / CUDA-core GEMM).
 cudaError_t launch_pack(const int8_t* S, uint32_t* bits, long long words, cudaStream_t stream);
 cudaError_t launch_unpack(const uint32_t* bits, int8_t* S, long long words, cudaStream_t stream);
+// Compress step: signs and per-tenant scale from fine-tuned weights; `partial` holds B x compress_blocks doubles.
+long long compress_blocks(int N, int K);
+cudaError_t launch_compress(const void* Wf, const void* Wb, uint32_t* bits, float* alpha, double* partial, int B, int N,
+                            int K, cudaStream_t stream);
 cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, void* Y,
                              int B, int m, int N, int K, cudaStream_t stream);
 

@@ -153,6 +153,109 @@ cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, cuda
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------- compress
+// The step before the product: bits = [W_fine - W_base > 0], alpha[b] = mean |W_fine - W_base|.
+// A warp owns one weight row and 1024 consecutive k of it (one sign word per lane); it keeps its piece of
+// W_base in registers and walks the tenants, so W_base is read once for all of them.  Per thread and
+// tenant: 64 bytes of W_fine in, one word out.  The comparison is taken on the exact bf16 values (as
+// fp32); |delta| is formed in fp32, four at a time, and summed in double: per thread, then across the
+// warp (shuffles) and the block (fixed order) into one partial per block and tenant; a second kernel adds
+// the partials of a tenant in a fixed order.  Nothing depends on the order in which blocks run.
+constexpr int kCompressWarps = 8;
+constexpr int kCompressTenantChunk = 32;   // tenants whose warp sums are staged in shared memory at once
+
+__device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+__global__ void __launch_bounds__(kCompressWarps * 32)
+compress_kernel(const uint4* __restrict__ Wf, const uint4* __restrict__ Wb, uint32_t* __restrict__ bits,
+                double* __restrict__ partial, int B, int N, int K, int kchunks, long long tiles) {
+    __shared__ double warp_sum[kCompressTenantChunk][kCompressWarps];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long tile = (long long)blockIdx.x * kCompressWarps + warp;
+    const int words = K >> 5;
+    const bool tile_ok = tile < tiles;
+    const int n = tile_ok ? (int)(tile / kchunks) : 0;
+    const int w = tile_ok ? (int)(tile - (long long)n * kchunks) * 32 + lane : words;   // this lane's sign word
+    const bool ok = tile_ok && w < words;
+    uint4 wb[4];
+    if (ok) {
+        const uint4* src = Wb + ((size_t)n * K + (size_t)w * 32) / 8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wb[i] = __ldg(src + i);
+    }
+    for (int b0 = 0; b0 < B; b0 += kCompressTenantChunk) {
+        const int nb = min(kCompressTenantChunk, B - b0);
+        for (int bb = 0; bb < nb; ++bb) {
+            const int b = b0 + bb;
+            double acc = 0.0;
+            if (ok) {
+                const uint4* src = Wf + (((size_t)b * N + n) * K + (size_t)w * 32) / 8;
+                uint4 wf[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) wf[i] = __ldg(src + i);
+                uint32_t word = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t f[4] = {wf[i].x, wf[i].y, wf[i].z, wf[i].w};
+                    const uint32_t g[4] = {wb[i].x, wb[i].y, wb[i].z, wb[i].w};
+                    float s4[2] = {0.f, 0.f};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float f0 = bf16lo(f[q]), f1 = bf16hi(f[q]), g0 = bf16lo(g[q]), g1 = bf16hi(g[q]);
+                        if (f0 > g0) word |= 1u << (i * 8 + q * 2);
+                        if (f1 > g1) word |= 1u << (i * 8 + q * 2 + 1);
+                        s4[q >> 1] += fabsf(f0 - g0) + fabsf(f1 - g1);
+                    }
+                    acc += (double)s4[0] + (double)s4[1];
+                }
+                bits[((size_t)b * N + n) * words + w] = word;
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (lane == 0) warp_sum[bb][warp] = acc;
+        }
+        __syncthreads();
+        for (int bb = threadIdx.x; bb < nb; bb += blockDim.x) {
+            double t = 0.0;
+#pragma unroll
+            for (int i = 0; i < kCompressWarps; ++i) t += warp_sum[bb][i];
+            partial[(size_t)(b0 + bb) * gridDim.x + blockIdx.x] = t;
+        }
+        __syncthreads();
+    }
+}
+
+// alpha[b] = (sum of the tenant's block partials, in a fixed order) / (N K), rounded to fp32.
+__global__ void compress_finish_kernel(const double* __restrict__ partial, float* __restrict__ alpha, int nblocks,
+                                       double inv_count) {
+    const int b = blockIdx.x, lane = threadIdx.x;
+    double t = 0.0;
+    for (int i = lane; i < nblocks; i += 32) t += partial[(size_t)b * nblocks + i];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    if (lane == 0) alpha[b] = (float)(t * inv_count);
+}
+
+long long compress_blocks(int N, int K) {
+    const long long kchunks = (K / 32 + 31) / 32;
+    const long long tiles = (long long)N * kchunks;
+    return (tiles + kCompressWarps - 1) / kCompressWarps;
+}
+
+cudaError_t launch_compress(const void* Wf, const void* Wb, uint32_t* bits, float* alpha, double* partial, int B, int N,
+                            int K, cudaStream_t stream) {
+    const int kchunks = (K / 32 + 31) / 32;
+    const long long tiles = (long long)N * kchunks;
+    const long long blocks = compress_blocks(N, K);
+    compress_kernel<<<(unsigned)blocks, kCompressWarps * 32, 0, stream>>>(
+        reinterpret_cast<const uint4*>(Wf), reinterpret_cast<const uint4*>(Wb), bits, partial, B, N, K, kchunks, tiles);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    compress_finish_kernel<<<(unsigned)B, 32, 0, stream>>>(partial, alpha, (int)blocks, 1.0 / ((double)N * (double)K));
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pack(const int8_t* S, uint32_t* bits, long long words, cudaStream_t stream) {
     const int threads = 256;
     const long long blocks = (words + threads - 1) / threads;
