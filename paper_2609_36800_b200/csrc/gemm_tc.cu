@@ -192,6 +192,16 @@ struct ItemIter {
     }
 };
 
+// Cursor over a ring of n buffers: index of the current buffer and the parity of its use count.
+struct Ring {
+    int idx;
+    uint32_t par;
+    int n;
+    __device__ __forceinline__ void step() {
+        if (++idx == n) { idx = 0; par ^= 1; }
+    }
+};
+
 struct Unit {
     int n0;        // first weight row of the tile
     int tenant0;   // first tenant
@@ -717,8 +727,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         // 256 KiB, so the sum never carries out of the 14-bit start-address field.
         const uint64_t desc0 = make_smem_desc_sw128(0);
         const uint32_t w_atom16 = a.w_atom_bytes >> 4, x_atom16 = a.x_atom_bytes >> 4;
-        const uint32_t amask = (uint32_t)a.a_slots - 1;
-        const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+        Ring ar{0, 0u, a.a_slots};   // operand buffers in tensor memory (tiled schedule)
         int stage = 0, xslot = 0;
         uint32_t phase = 0, xphase = 0, accphase = 0, item = 0;
         bool ok = true;
@@ -776,11 +785,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if constexpr (kDec) {
                     // Delta MMAs are issued by the two delta-issuer warps.
                 } else {
-                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
-                        const uint32_t slot = item & amask;
-                        const uint32_t use = item >> ashift;
+                    for (int j = 0; j < u.nten && ok; ++j, ++item, ar.step()) {
+                        const uint32_t slot = (uint32_t)ar.idx;
                         BD_ACC_BEGIN(tg);
-                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), use & 1, abort_flag, 5));
+                        ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), ar.par, abort_flag, 5));
                         BD_ACC_END(w_afull, tg);
                         if (!ok) break;
                         tc_fence_after();
@@ -829,10 +837,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             const uint32_t idesc_delta = make_idesc_e5m2(kTileN, (uint32_t)a.Nd);
             const uint64_t desc0 = make_smem_desc_sw128(0);
             const uint32_t ten_rows16 = (uint32_t)(kPieces * am) * 8u;   // rows per tenant x 128 B >> 4
-            const uint32_t amask = (uint32_t)a.a_slots - 1;
-            const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+            Ring ar{0, 0u, a.a_slots};   // this group's operand buffers in tensor memory
             int xslot = 0;
-            uint32_t xphase = 0, accphase = 0, item = 0;
+            uint32_t xphase = 0, accphase = 0;
             bool ok = true;
             BD_TL_DECL; BD_ACC_DECL(d_x8); BD_ACC_DECL(d_nb);
             while (ok && it.next(unit, p0, p1)) {
@@ -850,8 +857,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (g == 0) BD_TL(2);
                     const uint64_t x8desc = desc0 + ((x8_addr + xslot * a.x8_atom_bytes) >> 4);
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
-                    for (int half = 0; half < a.halves; ++half, ++item) {
-                        const uint32_t slot = item & amask;
+                    for (int half = 0; half < a.halves; ++half, ar.step()) {
+                        const uint32_t slot = (uint32_t)ar.idx;
                         if (*abort_flag) { ok = false; break; }
                         // The group's 128 decode threads arrive here once the buffer is filled (or when they
                         // give up after an abandoned wait, see the end of the decode role).
@@ -898,7 +905,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
                 __syncwarp();
                 accphase ^= 1;
-                (void)ashift;
             }
             if (g == 0) { BD_ACC_STORE(13, d_x8); BD_ACC_STORE(14, d_nb); }
         }
@@ -909,8 +915,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const uint32_t amask = (uint32_t)a.a_slots - 1;
-        const uint32_t ashift = (a.a_slots == 4) ? 2 : 1;
+        Ring ar{0, 0u, a.a_slots};   // this group's (tiled: the CTA's) operand buffers in tensor memory
         int bslot = 0;
         uint32_t bphase = 0, item = 0;
         bool ok = true;
@@ -948,17 +953,16 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         uint4 wq[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) wq[i] = *reinterpret_cast<const uint4*>(src + i * (2 * kTileN * 32));
-                        const uint32_t par = ((item >> 1) & 1) ^ 1;
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
+                        for (int half = 0; half < 2; ++half, ar.step()) {
                             BD_ACC_BEGIN(tq);
-                            ok = wait_bar(aempty_g + half * 8, par, abort_flag, 7);
+                            ok = wait_bar(aempty_g + (uint32_t)ar.idx * 8, ar.par ^ 1, abort_flag, 7);
                             BD_ACC_END(w_aempty, tq);
                             if (!ok) break;
                             tc_fence_after();
                             if (warp == kWarpDecode0) BD_TL(3);
                             BD_ACC_BEGIN(tw);
-                            const uint32_t tbuf = tbuf_g + (uint32_t)half * (uint32_t)a.aslot_cols;
+                            const uint32_t tbuf = tbuf_g + (uint32_t)ar.idx * (uint32_t)a.aslot_cols;
 #pragma unroll
                             for (int i = 0; i < 4; i += 2) {
                                 uint32_t r[32];
@@ -972,7 +976,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                             tc_wait_st();
                             if (warp == kWarpDecode0) BD_TL(3);
                             tc_fence_before();
-                            named_bar_arrive(kBarAFull0 + grp * 4 + half, 160);
+                            named_bar_arrive(kBarAFull0 + grp * 4 + ar.idx, 160);
                             BD_ACC_END(w_work, tw);
                             if (warp == kWarpDecode0) BD_TL(3);
                         }
@@ -983,9 +987,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         uint4 wq[2];
                         wq[0] = *reinterpret_cast<const uint4*>(src);
                         wq[1] = *reinterpret_cast<const uint4*>(src + 2 * kTileN * 32);
-                        const uint32_t slot = item & 1;
+                        const uint32_t slot = (uint32_t)ar.idx;
                         BD_ACC_BEGIN(tq);
-                        ok = wait_bar(aempty_g + slot * 8, ((item >> 1) & 1) ^ 1, abort_flag, 7);
+                        ok = wait_bar(aempty_g + slot * 8, ar.par ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
@@ -1005,12 +1009,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
                         BD_ACC_END(w_work, tw);
                         item += 1;
+                        ar.step();
                     } else
-                    for (int half = 0; half < a.halves && ok; ++half, ++item) {
-                        const uint32_t slot = item & amask;
-                        const uint32_t use = item >> ashift;
+                    for (int half = 0; half < a.halves && ok; ++half, ++item, ar.step()) {
+                        const uint32_t slot = (uint32_t)ar.idx;
                         BD_ACC_BEGIN(tq);
-                        ok = wait_bar(smem_u32(&ctl->aempty[grp * kMaxASlots + slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = wait_bar(smem_u32(&ctl->aempty[grp * kMaxASlots + slot]), ar.par ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
@@ -1069,12 +1073,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
                 } else {
-                    for (int j = 0; j < u.nten && ok; ++j, ++item) {
+                    for (int j = 0; j < u.nten && ok; ++j, ++item, ar.step()) {
                         const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
-                        const uint32_t slot = item & amask;
-                        const uint32_t use = item >> ashift;
+                        const uint32_t slot = (uint32_t)ar.idx;
                         BD_ACC_BEGIN(tq);
-                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), (use & 1) ^ 1, abort_flag, 7);
+                        ok = wait_bar(smem_u32(&ctl->aempty[slot]), ar.par ^ 1, abort_flag, 7);
                         BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
