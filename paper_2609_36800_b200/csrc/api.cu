@@ -149,7 +149,8 @@ int tb_override() {
     return v;
 }
 
-// BITDELTA_WHOLE=1 forces, =2 forbids the whole-unit work order (experiments).
+// BITDELTA_WHOLE (experiments): 1 forces, 2 forbids the whole-unit work order; 3 forces one team of CTAs per
+// tenant group, 4 forces the plain even cut.
 int whole_override() {
     static int v = -1;
     if (v < 0) {

@@ -13,6 +13,7 @@ struct GemmArgs {
     int B, m, N, K;
     int decode, convert, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
     int m_tiles, groups, P, whole_units;
+    int teams, Tg, cpt, n_tiles;   // work split by teams (see plan.h); q, r then describe one team's cut
     int T;             // work items (< 2^30)
     int q, r;          // T = q * grid + r
     int n_w, n_x, n_x8, a_slots, halves;
@@ -31,7 +32,9 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
     a.decode = p.decode; a.convert = p.convert; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
     a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
-    a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.q = (int)(p.T / p.grid); a.r = (int)(p.T % p.grid); a.whole_units = p.whole_units;
+    a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.whole_units = p.whole_units;
+    a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = p.grid / p.teams; a.n_tiles = p.n_tiles;
+    a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;

@@ -40,6 +40,8 @@ struct Plan {
     int n_tiles, m_tiles, groups, units;
     int P;             // k-pairs per unit
     int whole_units;   // 1: CTAs take whole units round-robin (no tile is cut), 0: even shares of the item list
+    int teams;         // > 1: one team of grid/teams CTAs per tenant group; units are numbered group-major and each
+                       // team cuts its group's items evenly (1: one cut of the whole list, units tile-major)
     long long T;       // total k-pair work items = units * P
     int grid;
     int n_w;           // ring of W_base tiles (128 rows x 128 k of bf16 each)
@@ -105,17 +107,38 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.T >= (1ll << 30)) return p;   // the kernel's work-split arithmetic is 32-bit
     int max_grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
     p.grid = p.T < max_grid ? (int)p.T : max_grid;
-    // Several tenant groups share each W_base tile.  If every CTA takes whole units in round-robin
-    // order, the groups of a tile run side by side on neighbouring CTAs and sweep k in step, so all
-    // but the first read of a W_base tile hit L2 (cut anywhere, the groups sit at different k and
-    // W_base is fetched from HBM once per group).  Taken when it costs little balance.
+    // Several tenant groups share each W_base tile; cut anywhere, the groups of a tile sit at different k at any
+    // moment and W_base is fetched from HBM once per group.  Two work orders keep them in step instead, so
+    // that all but the first read of a W_base tile hit L2:
+    //  * teams: one team of CTAs per tenant group, units numbered group-major, every team cutting its group's
+    //    items (all tiles x all k) the same way: CTA i of every team is at the same (tile, k) at the same
+    //    time.  Costs the CTAs left over when the groups do not divide the SM count.
+    //  * whole units: every CTA takes whole units in round-robin order, the groups of a tile run on
+    //    neighbouring CTAs.  Costs the idle CTAs of the last round.
+    // The one that keeps more of the chip busy is taken if that is at least 85 %; else the plain even cut.
+    // whole_override (experiments): 1 whole units, 3 teams, 2 not whole units, 4 plain cut.
     p.whole_units = 0;
-    if (p.decode && p.groups > 1 && p.units >= max_grid) {
-        const int rounds = (p.units + max_grid - 1) / max_grid;
-        const double balance = (double)p.units / ((double)rounds * max_grid);
-        if (balance >= 0.85 || whole_override == 1) { p.whole_units = 1; p.grid = max_grid; }
+    p.teams = 1;
+    if (p.decode && p.groups > 1) {
+        double s_whole = 0.0, s_teams = 0.0;
+        if (p.units >= max_grid) {
+            const int rounds = (p.units + max_grid - 1) / max_grid;
+            s_whole = (double)p.units / ((double)rounds * max_grid);
+        }
+        const long long Tg = (long long)p.n_tiles * p.P;
+        int cpt = max_grid / p.groups;
+        if (cpt > Tg) cpt = (int)Tg;
+        if (cpt >= 1) s_teams = (double)(cpt * p.groups) / max_grid;
+        int pick = 0;   // 0 plain cut, 1 whole units, 3 teams
+        if (s_teams >= 0.85 && s_teams >= s_whole) pick = 3;
+        else if (s_whole >= 0.85) pick = 1;
+        if (whole_override == 1 && p.units >= max_grid) pick = 1;
+        if (whole_override == 3 && cpt >= 1) pick = 3;
+        if (whole_override == 2 && pick == 1) pick = (s_teams >= 0.85) ? 3 : 0;
+        if (whole_override == 4) pick = 0;
+        if (pick == 1) { p.whole_units = 1; p.grid = max_grid; }
+        if (pick == 3) { p.teams = p.groups; p.grid = cpt * p.groups; }
     }
-    if (whole_override == 2) p.whole_units = 0;
 
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;

@@ -93,8 +93,9 @@ SMALL = [
     (4, 16, 128, 128),    # m at the decode/tiled boundary, one k step
     (20, 1, 128, 256),    # three tenant groups, the last one partly filled
     (7, 9, 256, 256),     # m > 8: groups of four tenants
-    (12, 8, 6400, 256),   # many tiles x several groups: whole-unit work order
-    (33, 2, 1920, 384),   # five groups, whole-unit order with a partly filled last group
+    (12, 8, 6400, 256),   # many tiles x three groups: one team of CTAs per group, tiles cut across CTAs
+    (33, 2, 1920, 384),   # five teams, a partly filled last group
+    (80, 1, 3712, 256),   # ten groups do not divide the SMs well: whole-unit work order
 ]
 
 
