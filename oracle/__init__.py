@@ -25,7 +25,7 @@ def build(force: bool = False) -> str:
     stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if force or stale:
         cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
-               "-fno-fast-math", "-ffp-contract=off", "-o", _LIB, _SRC]
+               "-fno-fast-math", "-ffp-contract=off", "-o", _LIB, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -44,6 +44,8 @@ def _load():
         lib.oracle_gemm.argtypes = [p, p, p, p, p, c_int, c_int, c_int, c_int]
         lib.oracle_gemm_at.argtypes = [p, p, p, p, p, c_int, p, c_int, c_int, c_int, c_int]
         lib.oracle_compress.argtypes = [p, p, p, p, c_int, c_int, c_int]
+        lib.oracle_half_to_double.argtypes = [p, p, ctypes.c_longlong]
+        lib.oracle_gemm_ex.argtypes = [p, p, p, p, p, p, c_int, p, c_int, c_int, c_int, c_int, c_int, c_int]
         _lib = lib
     return _lib
 
@@ -130,4 +132,41 @@ def gemm_at(X, W, bits, alpha, idx) -> np.ndarray:
     out = np.empty((idx.shape[0],), dtype=np.float64)
     _load().oracle_gemm_at(_ptr(X), _ptr(W), _ptr(bits), _ptr(alpha), _ptr(idx),
                            idx.shape[0], _ptr(out), B, m, N, K)
+    return out
+
+
+DTYPES = {"bf16": 0, "f16": 1}
+ACTS = {"none": 0, "silu": 1}
+
+
+def half_to_double(h: np.ndarray) -> np.ndarray:
+    """IEEE binary16 bit patterns (uint16) -> float64, by the format's definition."""
+    h = _as(h, np.uint16)
+    out = np.empty(h.shape, dtype=np.float64)
+    _load().oracle_half_to_double(_ptr(h), _ptr(out), h.size)
+    return out
+
+
+def gemm_ex(X, W, bits, alpha, bias=None, dtype="bf16", act="none", idx=None) -> np.ndarray:
+    """Y = act(sum_k x w + alpha[b] sum_k x s + bias[n]) in fp64.  X, W, bias are 16-bit patterns of
+    `dtype` ("bf16" or "f16"); act is "none" or "silu".  With idx (int32 [count,3] of (b,t,n)) only the
+    listed outputs are computed and returned as a vector."""
+    X, W, bits, alpha, B, m, N, K = _check(X, W, bits, alpha)
+    bp = None
+    if bias is not None:
+        bias = _as(bias, np.uint16)
+        if bias.shape != (N,):
+            raise ValueError("bias must have N entries")
+        bp = _ptr(bias)
+    if idx is not None:
+        idx = _as(idx, np.int32)
+        if idx.ndim != 2 or idx.shape[1] != 3:
+            raise ValueError("idx must be [count,3]")
+        out = np.empty((idx.shape[0],), dtype=np.float64)
+        ip, cnt = _ptr(idx), idx.shape[0]
+    else:
+        out = np.empty((B, m, N), dtype=np.float64)
+        ip, cnt = None, 0
+    _load().oracle_gemm_ex(_ptr(X), _ptr(W), _ptr(bits), _ptr(alpha), bp, ip, cnt, _ptr(out),
+                           B, m, N, K, DTYPES[dtype], ACTS[act])
     return out

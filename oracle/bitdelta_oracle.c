@@ -189,3 +189,75 @@ void oracle_compress(const uint16_t *wf, const uint16_t *wb, uint32_t *bits, flo
     }
 }
 
+
+/*
+ * Extended product (an adjacent variant: the paper's own BitDelta kernel computes in FP16, and its suite
+ * fuses activations into GEMM epilogues; neither is spelled out for this product, so this is the plain
+ * definition):
+ *
+ *   Y[b,t,n] = act( sum_k x w  +  alpha[b] * sum_k x s  +  bias[n] )
+ *
+ * dtype 0: x, w, bias are bf16 bit patterns; dtype 1: IEEE-754 binary16 bit patterns.
+ * bias may be NULL (no bias).  act 0: identity; act 1: SiLU, y * sigmoid(y) = y / (1 + exp(-y)).
+ * Everything is widened exactly to double; sums in double in plain k order; result kept in double.
+ */
+#include <math.h>
+
+/* binary16 -> double by the format's definition: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double half_to_double(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int e = (h >> 10) & 0x1F;
+    int f = h & 0x3FF;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);                 /* zero and subnormals: f * 2^-24 */
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+void oracle_half_to_double(const uint16_t *h, double *out, long long count)
+{
+    for (long long i = 0; i < count; ++i) out[i] = half_to_double(h[i]);
+}
+
+static double widen16(uint16_t v, int dtype)
+{
+    return dtype == 1 ? half_to_double(v) : bf16_to_double(v);
+}
+
+static double finish(double y, double bias, int act)
+{
+    y += bias;
+    if (act == 1) y = y / (1.0 + exp(-y));
+    return y;
+}
+
+/* The extended definition at `count` listed outputs (idx holds count triples b,t,n), or, with idx == NULL,
+ * at every output in (b,t,n) order (count is then ignored and out holds B*m*N values). */
+void oracle_gemm_ex(const uint16_t *X, const uint16_t *W, const uint32_t *bits, const float *alpha,
+                    const uint16_t *bias, const int32_t *idx, int count, double *out,
+                    int B, int m, int N, int K, int dtype, int act)
+{
+    int words = K / 32;
+    long long total = idx ? (long long)count : (long long)B * m * N;
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < total; ++i) {
+        int b, t, n;
+        if (idx) {
+            b = idx[3 * i + 0]; t = idx[3 * i + 1]; n = idx[3 * i + 2];
+        } else {
+            n = (int)(i % N); t = (int)((i / N) % m); b = (int)(i / ((long long)N * m));
+        }
+        const uint16_t *xrow = X + ((size_t)b * m + t) * K;
+        const uint16_t *wrow = W + (size_t)n * K;
+        const uint32_t *row_words = bits + ((size_t)b * N + n) * words;
+        double base = 0.0, delta = 0.0;
+        for (int k = 0; k < K; ++k) {
+            double x = widen16(xrow[k], dtype);
+            base += x * widen16(wrow[k], dtype);
+            delta += x * sign_at(row_words, k);
+        }
+        out[i] = finish(base + (double)alpha[b] * delta, bias ? widen16(bias[n], dtype) : 0.0, act);
+    }
+}

@@ -75,6 +75,24 @@ def make_inputs(wl: Workload, seed: int | None = None):
     return X, W, bits, alpha
 
 
+def make_inputs_f16(wl: Workload, seed: int | None = None, with_bias: bool = True):
+    """The same recipe in IEEE binary16: (X u16, W u16, bits u32, alpha f32, bias[N] u16 or None), the 16-bit
+    arrays being float16 bit patterns (numpy rounds float32 -> float16 to nearest even).  bias ~ N(0, 0.5)."""
+    rng = np.random.default_rng(wl.seed if seed is None else seed)
+    X = rng.standard_normal((wl.B, wl.m, wl.K), dtype=np.float32).astype(np.float16).view(np.uint16)
+    W = (np.float32(wl.w_std) * rng.standard_normal((wl.N, wl.K), dtype=np.float32)).astype(np.float16).view(np.uint16)
+    bits = rng.integers(0, 2**32, size=(wl.B, wl.N, wl.K // 32), dtype=np.uint32)
+    alpha = rng.uniform(wl.alpha_lo, wl.alpha_hi, wl.B).astype(np.float32)
+    bias = (np.float32(0.5) * rng.standard_normal(wl.N, dtype=np.float32)).astype(np.float16).view(np.uint16) if with_bias else None
+    return X, W, bits, alpha, bias
+
+
+def make_bias_bf16(N: int, seed: int = 0) -> np.ndarray:
+    """bias[N] ~ N(0, 0.5) as bf16 bit patterns."""
+    rng = np.random.default_rng(seed)
+    return f32_to_bf16_bits(np.float32(0.5) * rng.standard_normal(N, dtype=np.float32))
+
+
 def make_signs(B: int, N: int, K: int, seed: int = 0) -> np.ndarray:
     """Dense S int8 [B,N,K] of +1/-1 (input of the packing step)."""
     rng = np.random.default_rng(seed)

@@ -372,3 +372,90 @@ def test_compress_invariants():
     # tenants are independent
     b4, a4 = oracle.compress(fine[1:], W)
     assert np.array_equal(b4[0], bits[1]) and a4[0] == alpha[1]
+
+
+# ----------------------------------------------------------------------------
+# extended product: fp16 operands, bias, SiLU
+# ----------------------------------------------------------------------------
+def f16(a):
+    return np.asarray(a, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
+def test_half_decode_matches_numpy_on_every_finite_pattern():
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    finite = ((h >> 10) & 0x1F) != 31
+    got = oracle.half_to_double(h[finite])
+    expect = h[finite].view(np.float16).astype(np.float64)
+    assert np.array_equal(got, expect)
+    assert np.array_equal(np.signbit(got), np.signbit(expect))          # -0.0 keeps its sign
+    assert oracle.half_to_double(np.array([0x3C00, 0xC000, 0x0001, 0x7BFF], dtype=np.uint16)).tolist() == \
+        [1.0, -2.0, 2.0 ** -24, 65504.0]                                 # format constants
+
+
+def test_ex_without_options_is_the_plain_product_bit_for_bit():
+    X, W, bits, alpha = small_case(3, 4, 20, 160, seed=3)
+    assert np.array_equal(oracle.gemm_ex(X, W, bits, alpha), oracle.gemm(X, W, bits, alpha))
+
+
+@pytest.mark.parametrize("shape", [(2, 3, 5, 64), (3, 5, 33, 96)])
+def test_f16_product_matches_numpy_fp64_matmul(shape):
+    B, m, N, K = shape
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=11 + K)
+    X, W, bits, alpha, _ = synth.make_inputs_f16(wl)
+    x = X.view(np.float16).astype(np.float64)
+    w = W.view(np.float16).astype(np.float64)
+    S = dense_signs_py(bits)
+    expect = np.einsum("btk,nk->btn", x, w) + alpha.astype(np.float64)[:, None, None] * np.einsum("btk,bnk->btn", x, S)
+    got = oracle.gemm_ex(X, W, bits, alpha, dtype="f16")
+    assert np.max(np.abs(got - expect)) <= 1e-12 * max(1.0, np.max(np.abs(expect)))
+    # reading the same patterns as bf16 gives something else entirely
+    assert np.max(np.abs(oracle.gemm_ex(X, W, bits, alpha, dtype="bf16") - expect)) > 1e-3
+
+
+def test_bias_is_added_per_output_feature():
+    wl = synth.Workload("t", B=2, m=3, K=64, N=7, seed=5)
+    X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    y0 = oracle.gemm_ex(X, W, bits, alpha, dtype="f16")
+    y1 = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16")
+    b = bias.view(np.float16).astype(np.float64)
+    assert np.max(np.abs((y1 - y0) - b[None, None, :])) <= 1e-13
+    # bf16 bias patterns are read as bf16
+    Xb, Wb, bitsb, alphab = small_case(2, 3, 7, 64, seed=5)
+    bb = synth.make_bias_bf16(7, seed=1)
+    d = oracle.gemm_ex(Xb, Wb, bitsb, alphab, bias=bb) - oracle.gemm(Xb, Wb, bitsb, alphab)
+    assert np.max(np.abs(d - widen(bb)[None, None, :])) <= 1e-13
+
+
+def _probe(y, bias=None, act="none"):
+    """One output whose pre-activation value is exactly y: x = e_0, w[0,0] = y, alpha = 0."""
+    X = np.zeros((1, 1, 32), dtype=np.float32); X[0, 0, 0] = 1.0
+    W = np.zeros((1, 32), dtype=np.float32); W[0, 0] = y
+    bits = np.zeros((1, 1, 1), dtype=np.uint32)
+    alpha = np.zeros(1, dtype=np.float32)
+    b = None if bias is None else f16([bias])
+    return float(oracle.gemm_ex(f16(X), f16(W), bits, alpha, bias=b, dtype="f16", act=act)[0, 0, 0])
+
+
+def test_silu_closed_forms():
+    assert _probe(0.0, act="silu") == 0.0
+    assert _probe(1.0, act="silu") == pytest.approx(0.7310585786300049, rel=1e-15)      # sigmoid(1), textbook value
+    assert _probe(-1.0, act="silu") == pytest.approx(-0.2689414213699951, rel=1e-15)    # -sigmoid(-1)
+    for y in (0.5, 2.0, 7.25):
+        assert _probe(y, act="silu") - _probe(-y, act="silu") == pytest.approx(y, rel=1e-14)   # y (s(y) + s(-y)) = y
+    assert _probe(40.0, act="silu") == pytest.approx(40.0, rel=1e-15)
+    assert abs(_probe(-40.0, act="silu")) < 1e-15
+    assert _probe(3.0, act="none") == 3.0
+
+
+def test_activation_is_applied_after_the_bias():
+    # y = -1, bias = +2: silu(-1 + 2) = sigmoid(1); silu(-1) + 2 would be 1.731...
+    assert _probe(-1.0, bias=2.0, act="silu") == pytest.approx(0.7310585786300049, rel=1e-15)
+
+
+def test_ex_at_listed_outputs_equals_full_result():
+    wl = synth.Workload("t", B=3, m=4, K=96, N=10, seed=9)
+    X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    full = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu")
+    idx = np.array([[0, 0, 0], [2, 3, 9], [1, 2, 5], [2, 0, 7]], dtype=np.int32)
+    at = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu", idx=idx)
+    assert np.array_equal(at, np.array([full[b, t, n] for b, t, n in idx]))
