@@ -42,7 +42,8 @@ typedef enum {
     BITDELTA_ERR_WORKSPACE = 4, /* workspace missing or smaller than required         */
     BITDELTA_ERR_ARCH = 5,      /* current device is not compute capability 10.0      */
     BITDELTA_ERR_CUDA = 6,      /* a CUDA runtime / driver call failed                */
-    BITDELTA_ERR_TIMEOUT = 7    /* a bounded wait inside a kernel expired             */
+    BITDELTA_ERR_TIMEOUT = 7,   /* a bounded wait inside a kernel expired             */
+    BITDELTA_ERR_OPTION = 8     /* unknown data type or activation code               */
 } bitdelta_status;
 
 /*
@@ -114,6 +115,30 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
 int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
                   void* Y, int B, int m, int N, int K,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same product with the paper's own operand type and a fused epilogue (the paper's BitDelta kernel
+ * computes in FP16, and its suite fuses activations into GEMM epilogues, e.g. the fused GEMM-SiLU of
+ * its evaluation; the paper fixes neither for this product, so the definition is the plain one):
+ *
+ *   Y[b,t,n] = act( sum_k X[b,t,k] W_base[n,k] + alpha[b] sum_k X[b,t,k] S[b,n,k] + bias[n] )
+ *
+ * dtype : BITDELTA_DTYPE_BF16 or BITDELTA_DTYPE_F16 (IEEE binary16): the element type of X, W_base,
+ *         bias and Y.  Accumulation is fp32 in both; Y is rounded to nearest even once, after the
+ *         epilogue.  With binary16 the delta term is exact for operands in the normal range (values
+ *         below 2^-14 lose bits below 2^-16, in the delta term only).
+ * bias  : device, [N] values of `dtype`, shared by all tenants, or NULL for none.  2-byte aligned.
+ * act   : BITDELTA_ACT_NONE, or BITDELTA_ACT_SILU: y * sigmoid(y), applied after the bias (fp32,
+ *         hardware exponential: relative error of a few 1e-7, far below the output rounding).
+ * Everything else (shapes, layouts, workspace, stream semantics, errors, tolerance) is as for
+ * bitdelta_gemm, which is this call with BITDELTA_DTYPE_BF16, no bias and no activation.  Unknown
+ * codes return BITDELTA_ERR_OPTION and launch nothing.
+ */
+enum { BITDELTA_DTYPE_BF16 = 0, BITDELTA_DTYPE_F16 = 1 };
+enum { BITDELTA_ACT_NONE = 0, BITDELTA_ACT_SILU = 1 };
+int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
+                     const void* bias, void* Y, int B, int m, int N, int K, int dtype, int act,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * bitdelta_gemm for callers that must not allocate device memory.  (The paper has no counterpart

@@ -19,7 +19,7 @@ STATUS_TIMEOUT = 7
 EXPORTS = (
     "bitdelta_pack", "bitdelta_unpack", "bitdelta_compress_workspace_bytes", "bitdelta_compress",
     "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
-    "bitdelta_gemm", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
+    "bitdelta_gemm", "bitdelta_gemm_ex", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
     "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
 )
 
@@ -54,6 +54,7 @@ def load_library():
     lib.bitdelta_gemm_workspace_bytes.restype = sz
     lib.bitdelta_workspace_init.argtypes = [vp, sz, vp]
     lib.bitdelta_gemm.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
+    lib.bitdelta_gemm_ex.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
     lib.bitdelta_gemm_simt.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
     lib.bitdelta_gemm_noalloc.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp]
     lib.bitdelta_gemm_host_arena_bytes.argtypes = [ci, ci, ci, ci]
@@ -145,26 +146,46 @@ def make_workspace(B: int, m: int, N: int, K: int, device="cuda", stream=None):
     return ws
 
 
-def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bool = False):
-    """Y[b,t,n] = sum_k X W_base + alpha[b] sum_k X S.  X bf16 [B,m,K], W_base bf16 [N,K],
-    bits int32 storage [B,N,K/32], alpha fp32 [B]; returns Y bf16 [B,m,N]."""
+ACTS = {"none": 0, "silu": 1}
+
+
+def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bool = False, bias=None,
+         act: str = "none"):
+    """Y[b,t,n] = act(sum_k X W_base + alpha[b] sum_k X S + bias[n]).  X [B,m,K] and W_base [N,K] in bf16 or
+    (both) fp16, bits int32 storage [B,N,K/32], alpha fp32 [B], optional bias [N] of X's type, act "none" or
+    "silu"; returns Y [B,m,N] of X's type.  (simt=True runs the diagnostic CUDA-core kernel: bf16, no epilogue.)"""
     import torch
     lib = load_library()
     B, m, K = X.shape
     N = W_base.shape[0]
     if W_base.shape != (N, K) or tuple(bits.shape) != (B, N, K // 32) or tuple(alpha.shape) != (B,):
         raise ValueError("inconsistent shapes")
+    io = X.dtype
+    if io not in (torch.bfloat16, torch.float16):
+        raise TypeError("X must be bfloat16 or float16")
+    if act not in ACTS:
+        raise ValueError(f"unknown activation {act!r}")
+    if bias is not None and tuple(bias.shape) != (N,):
+        raise ValueError("bias must have N entries")
     if out is None:
-        out = torch.empty((B, m, N), dtype=torch.bfloat16, device=X.device)
-    args = [_dev(X, torch.bfloat16, "X"), _dev(W_base, torch.bfloat16, "W_base"), _dev(bits, torch.int32, "bits"),
-            _dev(alpha, torch.float32, "alpha"), _dev(out, torch.bfloat16, "out"), B, m, N, K]
+        out = torch.empty((B, m, N), dtype=io, device=X.device)
+    args = [_dev(X, io, "X"), _dev(W_base, io, "W_base"), _dev(bits, torch.int32, "bits"),
+            _dev(alpha, torch.float32, "alpha")]
+    shape = [B, m, N, K]
     if simt:
-        _check(lib.bitdelta_gemm_simt(*args, _stream_ptr(stream)), "bitdelta_gemm_simt")
+        if io != torch.bfloat16 or bias is not None or act != "none":
+            raise ValueError("the diagnostic kernel takes bf16 and has no epilogue")
+        _check(lib.bitdelta_gemm_simt(*args, _dev(out, io, "out"), *shape, _stream_ptr(stream)), "bitdelta_gemm_simt")
         return out
     if workspace is None:
         workspace = make_workspace(B, m, N, K, device=X.device, stream=stream)
-    _check(lib.bitdelta_gemm(*args, ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream)),
-           "bitdelta_gemm")
+    ws = (ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream))
+    if io == torch.bfloat16 and bias is None and act == "none":
+        _check(lib.bitdelta_gemm(*args, _dev(out, io, "out"), *shape, *ws), "bitdelta_gemm")
+    else:
+        bp = _dev(bias, io, "bias") if bias is not None else ctypes.c_void_p(0)
+        _check(lib.bitdelta_gemm_ex(*args, bp, _dev(out, io, "out"), *shape, 1 if io == torch.float16 else 0,
+                                    ACTS[act], *ws), "bitdelta_gemm_ex")
     return out
 
 

@@ -248,8 +248,8 @@ int bitdelta_gemm_simt(const void* X, const void* W_base, const uint32_t* bits, 
     DeviceInfo d;
     st = check_arch(&d);
     if (st != BITDELTA_OK) return st;
-    if (bd::launch_gemm_simt(X, W_base, bits, alpha, Y, B, m, N, K, static_cast<cudaStream_t>(cuda_stream)) !=
-        cudaSuccess)
+    if (bd::launch_gemm_simt(X, W_base, bits, alpha, nullptr, Y, B, m, N, K, 0, 0,
+                             static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
     g_launches++;
     return BITDELTA_OK;
@@ -257,8 +257,19 @@ int bitdelta_gemm_simt(const void* X, const void* W_base, const uint32_t* bits, 
 
 int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha, void* Y, int B, int m,
                   int N, int K, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return bitdelta_gemm_ex(X, W_base, bits, alpha, nullptr, Y, B, m, N, K, BITDELTA_DTYPE_BF16, BITDELTA_ACT_NONE,
+                            workspace, workspace_bytes, cuda_stream);
+}
+
+int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, const float* alpha, const void* bias,
+                     void* Y, int B, int m, int N, int K, int dtype, int act, void* workspace,
+                     size_t workspace_bytes, void* cuda_stream) {
     int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
     if (st != BITDELTA_OK) return st;
+    if ((dtype != BITDELTA_DTYPE_BF16 && dtype != BITDELTA_DTYPE_F16) || (act != BITDELTA_ACT_NONE && act != BITDELTA_ACT_SILU))
+        return BITDELTA_ERR_OPTION;
+    if (bias && (reinterpret_cast<uintptr_t>(bias) & 1)) return BITDELTA_ERR_ALIGN;
+    const int f16 = (dtype == BITDELTA_DTYPE_F16) ? 1 : 0;
     DeviceInfo d;
     st = check_arch(&d);
     if (st != BITDELTA_OK) return st;
@@ -266,7 +277,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
 
     if ((K % 128) != 0) {
         // Row pitch of the sign words is not a multiple of 16 bytes: no tensor map exists for it.
-        if (bd::launch_gemm_simt(X, W_base, bits, alpha, Y, B, m, N, K, stream) != cudaSuccess)
+        if (bd::launch_gemm_simt(X, W_base, bits, alpha, bias, Y, B, m, N, K, f16, act, stream) != cudaSuccess)
             return BITDELTA_ERR_CUDA;
         g_launches++;
         return BITDELTA_OK;
@@ -288,7 +299,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
         uint8_t* x8 = bd::ws_x8(p, workspace);
         if (!encode_u8_2d(&tmX8, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, (uint32_t)p.x8_rows))
             return BITDELTA_ERR_CUDA;
-        if (bd::launch_x_split(X, x8, B, m, K, stream) != cudaSuccess)
+        if (bd::launch_x_split(X, x8, B, m, K, f16, stream) != cudaSuccess)
             return BITDELTA_ERR_CUDA;
         g_launches++;
     } else {
@@ -296,6 +307,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
     }
 
     bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
+    args.f16 = f16; args.act = act; args.bias = bias;
     { static int h = -1; if (h < 0) { const char* e = getenv("BITDELTA_HOLD"); h = (e && e[0] == '0') ? 0 : 1; } args.hold_prefetch = h; }
     if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
@@ -411,6 +423,7 @@ const char* bitdelta_status_string(int status) {
         case BITDELTA_ERR_ARCH: return "device is not compute capability 10.0 (sm_100a required)";
         case BITDELTA_ERR_CUDA: return "CUDA runtime or driver call failed";
         case BITDELTA_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case BITDELTA_ERR_OPTION: return "unknown data type or activation code";
         default: return "unknown status";
     }
 }

@@ -17,6 +17,7 @@
 // grid; tiles cut across CTAs are summed through a workspace by the last CTA
 // to arrive, in a fixed order.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
@@ -257,15 +258,15 @@ __device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am)
 // bf16 each, register c = {k = 2c (low half), k = 2c+1 (high half)}, +1 for a
 // set bit and -1 for a clear bit.  Only shifts and three-input logic ops: the
 // wanted bits are moved onto the two bf16 sign positions and flip the sign of a
-// packed (-1, -1) constant.
-__device__ __forceinline__ void decode_word(uint32_t w, uint32_t* r) {
+// packed (-1, -1) constant (`minus_one2`: 0xBF80BF80 as bf16, 0xBC00BC00 as binary16).
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t* r, uint32_t minus_one2) {
     // even bits of the low half stay at 2c, odd bits move to 2c+16 (junk only on odd positions)
     const uint32_t lo = (w & 0x0000FFFFu) | ((w << 15) & 0xFFFF0000u);
     const uint32_t hi = (w >> 16) | ((w >> 1) & 0xFFFF0000u);
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        r[c] = ((lo << (15 - 2 * c)) & 0x80008000u) ^ 0xBF80BF80u;
-        r[8 + c] = ((hi << (15 - 2 * c)) & 0x80008000u) ^ 0xBF80BF80u;
+        r[c] = ((lo << (15 - 2 * c)) & 0x80008000u) ^ minus_one2;
+        r[8 + c] = ((hi << (15 - 2 * c)) & 0x80008000u) ^ minus_one2;
     }
 }
 
@@ -279,13 +280,28 @@ __device__ __forceinline__ void tmem_ld_w(uint32_t taddr, uint32_t* r) {
     else tmem_ld16(taddr, r);
 }
 
+// Fused epilogue on a finished sum: bias, then the activation, then rounding to the I/O type.
+__device__ __forceinline__ float epi_finish(float v, float bias, int act) {
+    v += bias;
+    if (act == 1) v = v / (1.f + __expf(-v));   // SiLU
+    return v;
+}
+__device__ __forceinline__ uint16_t to_io16(float v, int f16) {
+    return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ float from_io16(uint16_t h, int f16) {
+    return f16 ? __half2float(__ushort_as_half(h)) : __uint_as_float((uint32_t)h << 16);
+}
+
 struct EpiOut {
-    __nv_bfloat16* Y;   // output matrix [B*m, N]
+    uint16_t* Y;        // output matrix [B*m, N], 16-bit values of the I/O type
     float* slot;        // partial-result slot, or nullptr when this CTA owns the whole tile
     int N, n, row, xrow0;
+    float bias;         // of output feature n (0 without a bias)
+    const GemmArgs& a;  // kernel parameters (activation code, I/O type)
     __device__ __forceinline__ void put(int tok, float v) const {
-        if (slot) slot[(size_t)tok * kTileN + row] = v;
-        else if (n < N) Y[(size_t)(xrow0 + tok) * N + n] = __float2bfloat16_rn(v);
+        if (slot) slot[(size_t)tok * kTileN + row] = v;   // partial sums: finished by the CTA that adds them up
+        else if (n < N) Y[(size_t)(xrow0 + tok) * N + n] = to_io16(epi_finish(v, bias, a.act), a.f16);
     }
 };
 
@@ -348,10 +364,16 @@ __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterp
 // nwarps*32 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+nwarps, ...
 __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, int nwarps,
                                                 const float* first, const float* rest, size_t cstride, int nrest) {
-    __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
+    uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
     const int r4 = (etid & 31) * 4;
     const int n = u.n0 + r4;
     const bool vec_ok = ((a.N & 3) == 0) && (n + 3 < a.N);
+    float bias4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (a.bias) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (n + i < a.N) bias4[i] = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n + i), a.f16);
+    }
     for (int tk = etid >> 5; tk < u.ntok; tk += 4 * nwarps) {
         float4 acc[4];
 #pragma unroll
@@ -374,19 +396,18 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
         for (int q = 0; q < 4; ++q) {
             const int t = tk + nwarps * q;
             if (t < u.ntok) {
-                __nv_bfloat16* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
+                uint16_t* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
+                const uint16_t o0 = to_io16(epi_finish(acc[q].x, bias4[0], a.act), a.f16);
+                const uint16_t o1 = to_io16(epi_finish(acc[q].y, bias4[1], a.act), a.f16);
+                const uint16_t o2 = to_io16(epi_finish(acc[q].z, bias4[2], a.act), a.f16);
+                const uint16_t o3 = to_io16(epi_finish(acc[q].w, bias4[3], a.act), a.f16);
                 if (vec_ok) {
-                    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc[q].x, acc[q].y);
-                    __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc[q].z, acc[q].w);
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-                    pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-                    *reinterpret_cast<uint2*>(dst) = pk;
+                    *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)o0 | ((uint32_t)o1 << 16), (uint32_t)o2 | ((uint32_t)o3 << 16));
                 } else {
-                    if (n + 0 < a.N) dst[0] = __float2bfloat16_rn(acc[q].x);
-                    if (n + 1 < a.N) dst[1] = __float2bfloat16_rn(acc[q].y);
-                    if (n + 2 < a.N) dst[2] = __float2bfloat16_rn(acc[q].z);
-                    if (n + 3 < a.N) dst[3] = __float2bfloat16_rn(acc[q].w);
+                    if (n + 0 < a.N) dst[0] = o0;
+                    if (n + 1 < a.N) dst[1] = o1;
+                    if (n + 2 < a.N) dst[2] = o2;
+                    if (n + 3 < a.N) dst[3] = o3;
                 }
             }
         }
@@ -418,8 +439,12 @@ __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, con
         for (int i = 0; i < 4; ++i) {
             const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
             const uint32_t v = *reinterpret_cast<const uint32_t*>(src + chunk * 16);
-            const __half2 hv = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
-            y[i] = *reinterpret_cast<const uint32_t*>(&hv);
+            if (a.f16) {
+                y[i] = v;   // binary16 already: eleven significant bits, the four pieces take 3 + 3 + 3 + 2
+            } else {
+                const __half2 hv = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+                y[i] = *reinterpret_cast<const uint32_t*>(&hv);
+            }
         }
 #pragma unroll
         for (int q = 0; q < kPieces; ++q) {
@@ -741,9 +766,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //   tiled schedule : one item = one tenant x 128 k of bf16 signs (64 columns, 8 MMAs of K=16)
         //   decode schedule: one item = all tenants of the unit x 64 k of e5m2 signs (16 columns per
         //                    tenant, 2 MMAs of K=32 per tenant)
-        const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+        const uint32_t idesc_base = a.f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nb) : make_idesc_bf16(kTileN, (uint32_t)a.Nb);
         const uint32_t idesc_delta = kDec ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
-                                              : make_idesc_bf16(kTileN, (uint32_t)a.Nd);
+                                          : (a.f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nd) : make_idesc_bf16(kTileN, (uint32_t)a.Nd));
         // Descriptor of a tile = descriptor of address 0 plus (address >> 4): addresses stay below
         // 256 KiB, so the sum never carries out of the 14-bit start-address field.
         const uint64_t desc0 = make_smem_desc_sw128(0);
@@ -941,6 +966,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint32_t bphase = 0, item = 0;
         bool ok = true;
         // shapes with a straight-line decode loop (two operand buffers per group in both)
+        const uint32_t minus_one2 = a.f16 ? 0xBC00BC00u : 0xBF80BF80u;   // tiled schedule: packed (-1, -1) in the I/O type
         const bool fast8 = kDec && a.TB == 8 && a.halves == 2 && a.a_slots == 2;
         const bool fast4 = kDec && a.TB == 4 && a.halves == 1 && a.a_slots == 2;
         const uint32_t aempty_g = smem_u32(&ctl->aempty[grp * kMaxASlots]);
@@ -1105,11 +1131,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         BD_ACC_BEGIN(tw);
                         const uint32_t taddr = lane_taddr + a.col_a + slot * (uint32_t)a.aslot_cols;
                         uint32_t r[32];
-                        decode_word(w.x, r);
-                        decode_word(w.y, r + 16);
+                        decode_word(w.x, r, minus_one2);
+                        decode_word(w.y, r + 16, minus_one2);
                         tmem_st32(taddr, r);
-                        decode_word(w.z, r);
-                        decode_word(w.w, r + 16);
+                        decode_word(w.z, r, minus_one2);
+                        decode_word(w.w, r + 16, minus_one2);
                         tmem_st32(taddr + 32, r);
                         tc_wait_st();
                         tc_fence_before();
@@ -1144,7 +1170,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const int ehalf = (warp - epi_first_warp) >> 2;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int first_unit = (int)((unsigned)lo / (unsigned)a.P);
-        __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(a.Y);
+        uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
         uint32_t accphase = 0;
         bool ok = true;
         BD_TL_DECL;
@@ -1227,6 +1253,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             float alv[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
+            const float bias_n = (a.bias && n < a.N) ? from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n), a.f16) : 0.f;
             if (splitter) {
                 seg_end += p1 - p0;
                 while (ok && n_split < seg_end) ok = split_next(true);
@@ -1247,7 +1274,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
-            EpiOut out{Y, slotp, a.N, n, row, u.xrow0};
+            EpiOut out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
             if constexpr (kMode >= 1 && kMode <= 4) {
                 epilogue_decode<kMode>(a, u, lane_taddr, out, alv);
             } else if constexpr (kMode == 5) {

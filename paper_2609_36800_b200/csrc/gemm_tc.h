@@ -12,6 +12,9 @@ namespace bd {
 struct GemmArgs {
     int B, m, N, K;
     int decode, convert, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
+    int f16;             // 0: X, W_base, bias, Y are bf16; 1: IEEE binary16
+    int act;             // fused epilogue: 0 none, 1 SiLU (after the bias)
+    const void* bias;    // [N] values of the I/O type added to every output row, or nullptr
     int m_tiles, groups, P, whole_units;
     int teams, Tg, cpt, n_tiles;   // work split by teams (see plan.h); q, r then describe one team's cut
     int T;             // work items (< 2^30)
@@ -61,7 +64,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
 
 // Decode schedule pre-pass: X bf16 [rows, K] -> four e5m2 pieces per element (k permuted inside
 // each group of 32) in X8 [B, 4, m, K].
-cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, cudaStream_t stream);
+cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream);
 
 // Synchronises the stream, reads {status, site} and clears them if set.
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream);
@@ -73,7 +76,7 @@ cudaError_t launch_unpack(const uint32_t* bits, int8_t* S, long long words, cuda
 long long compress_blocks(int N, int K);
 cudaError_t launch_compress(const void* Wf, const void* Wb, uint32_t* bits, float* alpha, double* partial, int B, int N,
                             int K, cudaStream_t stream);
-cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, void* Y,
-                             int B, int m, int N, int K, cudaStream_t stream);
+cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, const void* bias,
+                             void* Y, int B, int m, int N, int K, int f16, int act, cudaStream_t stream);
 
 }  // namespace bd

@@ -1,5 +1,6 @@
 // Plain CUDA-core kernels: sign packing / unpacking and a diagnostic GEMM.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
@@ -54,9 +55,18 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ bits, int8_t* __restr
 
 // One warp per (tenant, weight row); lanes stride over the sign words, so lane l
 // owns k = 32w .. 32w+31 for w = l, l+32, ...  fp32 accumulation, shuffle reduce.
-__global__ void gemm_simt_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
+// 16-bit values of the I/O type (bf16, or IEEE binary16 when `f16`) <-> fp32.
+__device__ __forceinline__ float io16_to_float(uint16_t h, int f16) {
+    return f16 ? __half2float(__ushort_as_half(h)) : __uint_as_float((uint32_t)h << 16);
+}
+__device__ __forceinline__ uint16_t float_to_io16(float v, int f16) {
+    return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+
+__global__ void gemm_simt_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ W,
                                  const uint32_t* __restrict__ bits, const float* __restrict__ alpha,
-                                 __nv_bfloat16* __restrict__ Y, int B, int m, int N, int K) {
+                                 const uint16_t* __restrict__ bias, uint16_t* __restrict__ Y, int B, int m, int N,
+                                 int K, int f16, int act) {
     const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (gw >= (long long)B * N) return;
@@ -64,17 +74,18 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16* __restrict__ X, const __nv
     const int n = (int)(gw % N);
     const int words = K >> 5;
     const uint32_t* brow = bits + ((size_t)b * N + n) * words;
-    const __nv_bfloat16* wrow = W + (size_t)n * K;
+    const uint16_t* wrow = W + (size_t)n * K;
     const float al = alpha[b];
+    const float bias_n = bias ? io16_to_float(bias[n], f16) : 0.f;
     for (int t = 0; t < m; ++t) {
-        const __nv_bfloat16* xrow = X + ((size_t)b * m + t) * K;
+        const uint16_t* xrow = X + ((size_t)b * m + t) * K;
         float base = 0.f, delta = 0.f;
         for (int w = lane; w < words; w += 32) {
             const uint32_t word = brow[w];
 #pragma unroll 8
             for (int j = 0; j < 32; ++j) {
-                const float x = __bfloat162float(xrow[w * 32 + j]);
-                base = fmaf(x, __bfloat162float(wrow[w * 32 + j]), base);
+                const float x = io16_to_float(xrow[w * 32 + j], f16);
+                base = fmaf(x, io16_to_float(wrow[w * 32 + j], f16), base);
                 delta += ((word >> j) & 1u) ? x : -x;
             }
         }
@@ -83,7 +94,11 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16* __restrict__ X, const __nv
             base += __shfl_xor_sync(0xFFFFFFFFu, base, o);
             delta += __shfl_xor_sync(0xFFFFFFFFu, delta, o);
         }
-        if (lane == 0) Y[((size_t)b * m + t) * N + n] = __float2bfloat16_rn(fmaf(al, delta, base));
+        if (lane == 0) {
+            float v = fmaf(al, delta, base) + bias_n;
+            if (act == 1) v = v / (1.f + __expf(-v));   // SiLU
+            Y[((size_t)b * m + t) * N + n] = float_to_io16(v, f16);
+        }
     }
 }
 
@@ -102,8 +117,8 @@ __device__ __forceinline__ uint8_t e5m2_round(float v) {
     return (uint8_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
 }
 
-__global__ void __launch_bounds__(128) x_split_kernel(const __nv_bfloat16* __restrict__ X, uint8_t* __restrict__ X8,
-                                                      int m, int K, long long total_groups) {
+__global__ void __launch_bounds__(128) x_split_kernel(const uint16_t* __restrict__ X, uint8_t* __restrict__ X8,
+                                                      int m, int K, long long total_groups, int f16) {
     // Let the GEMM kernel queued behind this one start its weight prefetch right away.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -120,8 +135,8 @@ __global__ void __launch_bounds__(128) x_split_kernel(const __nv_bfloat16* __res
         const uint32_t q[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            y[h * 8 + 2 * i] = __uint_as_float(q[i] << 16);
-            y[h * 8 + 2 * i + 1] = __uint_as_float(q[i] & 0xFFFF0000u);
+            y[h * 8 + 2 * i] = io16_to_float((uint16_t)(q[i] & 0xFFFFu), f16);
+            y[h * 8 + 2 * i + 1] = io16_to_float((uint16_t)(q[i] >> 16), f16);
         }
     }
 #pragma unroll
@@ -144,12 +159,11 @@ __global__ void __launch_bounds__(128) x_split_kernel(const __nv_bfloat16* __res
     }
 }
 
-cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, cudaStream_t stream) {
+cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream) {
     const long long total = (long long)B * m * (K >> 5);
     const int threads = 128;
     const long long blocks = (total + threads - 1) / threads;
-    x_split_kernel<<<(unsigned)blocks, threads, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(X), X8, m, K,
-                                                             total);
+    x_split_kernel<<<(unsigned)blocks, threads, 0, stream>>>(reinterpret_cast<const uint16_t*>(X), X8, m, K, total, f16);
     return cudaGetLastError();
 }
 
@@ -270,14 +284,14 @@ cudaError_t launch_unpack(const uint32_t* bits, int8_t* S, long long words, cuda
     return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, void* Y,
-                             int B, int m, int N, int K, cudaStream_t stream) {
+cudaError_t launch_gemm_simt(const void* X, const void* W, const uint32_t* bits, const float* alpha, const void* bias,
+                             void* Y, int B, int m, int N, int K, int f16, int act, cudaStream_t stream) {
     const int threads = 256;
     const long long warps = (long long)B * N;
     const long long blocks = (warps * 32 + threads - 1) / threads;
     gemm_simt_kernel<<<(unsigned)blocks, threads, 0, stream>>>(
-        reinterpret_cast<const __nv_bfloat16*>(X), reinterpret_cast<const __nv_bfloat16*>(W), bits, alpha,
-        reinterpret_cast<__nv_bfloat16*>(Y), B, m, N, K);
+        reinterpret_cast<const uint16_t*>(X), reinterpret_cast<const uint16_t*>(W), bits, alpha,
+        reinterpret_cast<const uint16_t*>(bias), reinterpret_cast<uint16_t*>(Y), B, m, N, K, f16, act);
     return cudaGetLastError();
 }
 

@@ -192,6 +192,10 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N) {
            | ((N >> 3) << 17)   // N / 8
            | ((M >> 4) << 24);  // M / 16
 }
+// The same with binary16 operands (format code 0).
+__host__ __device__ constexpr uint32_t make_idesc_f16(uint32_t M, uint32_t N) {
+    return (1u << 4) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
 
 // Shared-memory matrix descriptor for a K-major tile whose rows are 128 bytes
 // (64 bf16) written with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
