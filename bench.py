@@ -234,6 +234,46 @@ def time_compress(peaks, B=8, N=4096, K=4096, steps=20):
             "steps": steps, "kernels_per_call": 2}
 
 
+def time_gemm_ex(wl, peaks, steps=40):
+    """The extended call (fp16 operands, bias, SiLU fused into the epilogue) on `wl`, timed like the
+    headline: rotating buffer sets larger than L2, all steps in one CUDA graph, CUDA events."""
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    nsets = max(2, -(-2 * L2_BYTES // wl.bytes))
+    f16 = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.float16)
+    sets = [(f16(X), f16(W), torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(alpha).cuda(), f16(bias),
+             torch.empty((wl.B, wl.m, wl.N), dtype=torch.float16, device="cuda")) for _ in range(nsets)]
+    ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
+    stream = torch.cuda.Stream()
+    call = lambda s: bd.gemm(s[0], s[1], s[2], s[3], out=s[5], workspace=ws, bias=s[4], act="silu")
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            call(sets[i % nsets])
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(steps):
+                call(sets[i % nsets])
+        graph.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1)
+    st, site = bd.last_device_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} at site {site}")
+    _, _, roof = summarize(wl, ms, steps, 1, peaks)
+    roof["traffic"] = None                       # not captured separately: same loads as the bf16 call plus N bias values
+    roof["algorithmic_bytes"] = wl.bytes + 2 * wl.N
+    return {"us_per_launch": ms * 1e3 / steps, "steps": steps, "buffer_sets": nsets, "dtype": "f16",
+            "epilogue": "bias+silu", "roofline": roof}
+
+
 def time_e2e(wl, host_inputs, steps):
     """Same metric through the host-buffer C-ABI entry point: H2D of every input and D2H of Y
     inside the timed region, every step."""
@@ -405,6 +445,12 @@ def run_ours(args):
                                    "buffer_sets": nsets2, "roofline": r2}
             out["workloads"] = others
             out["compress"] = time_compress(peaks)
+            out["gemm_ex"] = {}
+            for name in ("decode_attn", "decode_mlp_up", "prefill"):
+                w3 = synth.WORKLOADS_BY_NAME[name]
+                steps3 = max(20, min(args.steps, int(0.25 / max(w3.bytes / 6.5e12, w3.flops / 1.6e15))))
+                out["gemm_ex"][name] = time_gemm_ex(w3, peaks, steps3)
+                torch.cuda.empty_cache()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

@@ -283,16 +283,23 @@ __device__ __forceinline__ void tmem_ld_w(uint32_t taddr, uint32_t* r) {
 // Fused epilogue on a finished sum: bias, then the activation, then rounding to the I/O type.
 __device__ __forceinline__ float epi_finish(float v, float bias, int act) {
     v += bias;
-    if (act == 1) v = v / (1.f + __expf(-v));   // SiLU
+    if (act == 1) v = __fdividef(v, 1.f + __expf(-v));   // SiLU; approximate division (2 ulp) keeps the unrolled epilogues small
     return v;
 }
 __device__ __forceinline__ uint16_t to_io16(float v, int f16) {
     return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
 }
+__device__ __forceinline__ uint16_t finish_io16(float v, float bias, int act, int f16) {
+    return to_io16(epi_finish(v, bias, act), f16);
+}
 __device__ __forceinline__ float from_io16(uint16_t h, int f16) {
     return f16 ? __half2float(__ushort_as_half(h)) : __uint_as_float((uint32_t)h << 16);
 }
 
+// kGen = false: bf16 output, no bias, no activation (the plain product).  The two forms are separate code
+// on purpose: the epilogue runs once per tile, every instruction of it is fetched cold, and the plain
+// product should not pay for the general form's length.
+template <bool kGen>
 struct EpiOut {
     uint16_t* Y;        // output matrix [B*m, N], 16-bit values of the I/O type
     float* slot;        // partial-result slot, or nullptr when this CTA owns the whole tile
@@ -301,22 +308,28 @@ struct EpiOut {
     const GemmArgs& a;  // kernel parameters (activation code, I/O type)
     __device__ __forceinline__ void put(int tok, float v) const {
         if (slot) slot[(size_t)tok * kTileN + row] = v;   // partial sums: finished by the CTA that adds them up
-        else if (n < N) Y[(size_t)(xrow0 + tok) * N + n] = to_io16(epi_finish(v, bias, a.act), a.f16);
+        else if (n < N) {
+            if constexpr (kGen) Y[(size_t)(xrow0 + tok) * N + n] = finish_io16(v, bias, a.act, a.f16);
+            else Y[(size_t)(xrow0 + tok) * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        }
     }
 };
 
 // Decode schedule, M tokens per tenant: the base accumulator holds tenant j's tokens in columns
 // j*M .. j*M+M-1; its delta accumulator starts at column N3*j and holds, for piece q of the
 // activation split, token t in column q*M + t.  delta = D0 + D1 + D2 + D3.
-template <int M>
+// Plain product: the tenant loop is unrolled (the tensor-memory loads of all tenants overlap).  General form
+// with more than four tokens per tenant: a real loop, because its body is long, this code runs once per tile
+// and every instruction of it is fetched cold, so its length is paid in time.
+// `alv[j]`: tenant j's scale (unrolled form); `al_lane`: lane l holds tenant l's scale (loop form).
+template <int M, bool kGen>
 __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                                const EpiOut& out, const float* alv) {
+                                                const EpiOut<kGen>& out, const float* alv, float al_lane) {
     constexpr int N3 = (kPieces * M + 15) / 16 * 16;
     constexpr int TPB = (N3 == 16) ? 2 : 1;   // tenants drained per wait
     constexpr int kMaxTen = (M <= 4) ? 8 : 4;   // tenants per unit (see the plan)
-#pragma unroll
-    for (int j0 = 0; j0 < kMaxTen; j0 += TPB) {
-        if (j0 >= u.nten) break;
+    constexpr bool kLoop = kGen && M > 4;
+    auto drain = [&](int j0) {
         uint32_t rb[16], rd[TPB * N3];
         tmem_ld16(lane_taddr + (uint32_t)(j0 * M), rb);
 #pragma unroll
@@ -328,8 +341,10 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
         tc_wait_ld();
 #pragma unroll
         for (int jj = 0; jj < TPB; ++jj) {
-            if (j0 + jj < u.nten) {
-                const float al = alv[j0 + jj];
+            if (j0 + jj < u.nten) {   // warp-uniform
+                float al;
+                if constexpr (kLoop) al = __shfl_sync(0xFFFFFFFFu, al_lane, j0 + jj);
+                else al = alv[j0 + jj];
 #pragma unroll
                 for (int t = 0; t < M; ++t) {
                     const float lo = __uint_as_float(rd[jj * N3 + 2 * M + t]) + __uint_as_float(rd[jj * N3 + 3 * M + t]);
@@ -338,13 +353,24 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
                 }
             }
         }
+    };
+    if constexpr (kLoop) {
+#pragma unroll 1
+        for (int j0 = 0; j0 < u.nten; j0 += TPB) drain(j0);
+    } else {
+#pragma unroll
+        for (int j0 = 0; j0 < kMaxTen; j0 += TPB) {
+            if (j0 >= u.nten) break;
+            drain(j0);
+        }
     }
 }
 
 // Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
 // Two warps share each lane quadrant: warp half h drains the 32-token blocks h, h+2, ...
+template <class Out>
 __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                               const EpiOut& out, int half, float al) {
+                                               const Out& out, int half, float al) {
     for (int t0 = 32 * half; t0 < u.ntok; t0 += 64) {
         uint32_t rb[32], rd[32];
         tmem_ld32(lane_taddr + (uint32_t)t0, rb);
@@ -362,6 +388,7 @@ __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterp
 
 // Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
 // nwarps*32 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+nwarps, ...
+template <bool kGen>
 __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, int nwarps,
                                                 const float* first, const float* rest, size_t cstride, int nrest) {
     uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
@@ -369,7 +396,7 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
     const int n = u.n0 + r4;
     const bool vec_ok = ((a.N & 3) == 0) && (n + 3 < a.N);
     float bias4[4] = {0.f, 0.f, 0.f, 0.f};
-    if (a.bias) {
+    if (kGen && a.bias) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             if (n + i < a.N) bias4[i] = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n + i), a.f16);
@@ -397,10 +424,18 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
             const int t = tk + nwarps * q;
             if (t < u.ntok) {
                 uint16_t* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
-                const uint16_t o0 = to_io16(epi_finish(acc[q].x, bias4[0], a.act), a.f16);
-                const uint16_t o1 = to_io16(epi_finish(acc[q].y, bias4[1], a.act), a.f16);
-                const uint16_t o2 = to_io16(epi_finish(acc[q].z, bias4[2], a.act), a.f16);
-                const uint16_t o3 = to_io16(epi_finish(acc[q].w, bias4[3], a.act), a.f16);
+                uint16_t o0, o1, o2, o3;
+                if constexpr (kGen) {
+                    o0 = finish_io16(acc[q].x, bias4[0], a.act, a.f16);
+                    o1 = finish_io16(acc[q].y, bias4[1], a.act, a.f16);
+                    o2 = finish_io16(acc[q].z, bias4[2], a.act, a.f16);
+                    o3 = finish_io16(acc[q].w, bias4[3], a.act, a.f16);
+                } else {
+                    o0 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].x));
+                    o1 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].y));
+                    o2 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].z));
+                    o3 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].w));
+                }
                 if (vec_ok) {
                     *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)o0 | ((uint32_t)o1 << 16), (uint32_t)o2 | ((uint32_t)o3 << 16));
                 } else {
@@ -427,6 +462,7 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
 // `xt` is the stage's X tile (two swizzled 64-k atoms), `x8t` its piece tile.  Thread `tid` of `nthreads`
 // takes the tasks tid, tid + nthreads, ...  Small tasks on purpose: 16 per token row spread the work over
 // all four epilogue warps, one warp per scheduler.
+template <bool kF16>
 __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, const uint8_t* xt, uint8_t* x8t, int ntok, int tid,
                                                   int nthreads) {
     const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 16;
@@ -439,7 +475,7 @@ __device__ __forceinline__ void split_activations(const GemmArgs& a, int am, con
         for (int i = 0; i < 4; ++i) {
             const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
             const uint32_t v = *reinterpret_cast<const uint32_t*>(src + chunk * 16);
-            if (a.f16) {
+            if constexpr (kF16) {
                 y[i] = v;   // binary16 already: eleven significant bits, the four pieces take 3 + 3 + 3 + 2
             } else {
                 const __half2 hv = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
@@ -482,7 +518,9 @@ __device__ __forceinline__ void epi_bar_sync(int nthreads) { asm volatile("bar.s
 // kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m.
 // One instantiation per mode keeps each launched kernel's code small (the roles' loops then stay in the
 // instruction caches) and turns the schedule switches into compile-time constants.
-template <int kMode>
+// kGen: the general form (binary16 I/O, bias, activation); false compiles the plain bf16 product alone, whose
+// code is then exactly as short as it can be (the kernel's speed is sensitive to its length).
+template <int kMode, bool kGen>
 __global__ void __launch_bounds__(kThreads, 1)
 bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                         const __grid_constant__ CUtensorMap tmX8, const __grid_constant__ CUtensorMap tmBits,
@@ -505,6 +543,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     constexpr bool kDec = kMode != 0;
     const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
     const bool convert = kDec && a.convert != 0;
+    const bool io_f16 = kGen && a.f16 != 0;
     auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec>(aa, un, am); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -558,7 +597,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     // One epilogue thread's share (tasks tid, tid + 128, ...) of the in-kernel activation split: bf16 tile
     // in slot `xs` of its ring -> piece tile in slot `x8s` of its ring.
     auto do_split = [&](int xs, int x8s, int ntok, int tid) {
-        split_activations(a, am, smem + x_off + xs * a.x_tile_bytes, smem + x8_off + x8s * a.x8_atom_bytes, ntok, tid, 128);
+        // (two instantiations, chosen here: a test of the I/O type inside the split's loops costs the plain
+        // product measurable time)
+        if (io_f16) split_activations<true>(a, am, smem + x_off + xs * a.x_tile_bytes, smem + x8_off + x8s * a.x8_atom_bytes, ntok, tid, 128);
+        else split_activations<false>(a, am, smem + x_off + xs * a.x_tile_bytes, smem + x8_off + x8s * a.x8_atom_bytes, ntok, tid, 128);
         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
         mbar_arrive(smem_u32(&ctl->x8full[x8s]));
         mbar_arrive(smem_u32(&ctl->xempty[xs]));   // this thread is done reading the bf16 tile
@@ -766,9 +808,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //   tiled schedule : one item = one tenant x 128 k of bf16 signs (64 columns, 8 MMAs of K=16)
         //   decode schedule: one item = all tenants of the unit x 64 k of e5m2 signs (16 columns per
         //                    tenant, 2 MMAs of K=32 per tenant)
-        const uint32_t idesc_base = a.f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nb) : make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+        const uint32_t idesc_base = io_f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nb) : make_idesc_bf16(kTileN, (uint32_t)a.Nb);
         const uint32_t idesc_delta = kDec ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
-                                          : (a.f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nd) : make_idesc_bf16(kTileN, (uint32_t)a.Nd));
+                                          : (io_f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nd) : make_idesc_bf16(kTileN, (uint32_t)a.Nd));
         // Descriptor of a tile = descriptor of address 0 plus (address >> 4): addresses stay below
         // 256 KiB, so the sum never carries out of the 14-bit start-address field.
         const uint64_t desc0 = make_smem_desc_sw128(0);
@@ -966,7 +1008,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint32_t bphase = 0, item = 0;
         bool ok = true;
         // shapes with a straight-line decode loop (two operand buffers per group in both)
-        const uint32_t minus_one2 = a.f16 ? 0xBC00BC00u : 0xBF80BF80u;   // tiled schedule: packed (-1, -1) in the I/O type
+        const uint32_t minus_one2 = io_f16 ? 0xBC00BC00u : 0xBF80BF80u;   // tiled schedule: packed (-1, -1) in the I/O type
         const bool fast8 = kDec && a.TB == 8 && a.halves == 2 && a.a_slots == 2;
         const bool fast4 = kDec && a.TB == 4 && a.halves == 1 && a.a_slots == 2;
         const uint32_t aempty_g = smem_u32(&ctl->aempty[grp * kMaxASlots]);
@@ -1253,7 +1295,11 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             float alv[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
-            const float bias_n = (a.bias && n < a.N) ? from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n), a.f16) : 0.f;
+            float al_lane = 0.f, bias_n = 0.f;
+            if constexpr (kGen) {
+                al_lane = (lane < u.nten) ? __ldg(a.alpha + u.tenant0 + lane) : 0.f;   // lane l: tenant l's scale
+                if (a.bias && n < a.N) bias_n = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n), a.f16);
+            }
             if (splitter) {
                 seg_end += p1 - p0;
                 while (ok && n_split < seg_end) ok = split_next(true);
@@ -1274,23 +1320,23 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
-            EpiOut out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
+            const EpiOut<kGen> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
             if constexpr (kMode >= 1 && kMode <= 4) {
-                epilogue_decode<kMode>(a, u, lane_taddr, out, alv);
+                epilogue_decode<kMode>(a, u, lane_taddr, out, alv, al_lane);
             } else if constexpr (kMode == 5) {
                 switch (am) {
-                    case 5: epilogue_decode<5>(a, u, lane_taddr, out, alv); break;
-                    case 6: epilogue_decode<6>(a, u, lane_taddr, out, alv); break;
-                    case 7: epilogue_decode<7>(a, u, lane_taddr, out, alv); break;
-                    case 8: epilogue_decode<8>(a, u, lane_taddr, out, alv); break;
-                    case 9: epilogue_decode<9>(a, u, lane_taddr, out, alv); break;
-                    case 10: epilogue_decode<10>(a, u, lane_taddr, out, alv); break;
-                    case 11: epilogue_decode<11>(a, u, lane_taddr, out, alv); break;
-                    case 12: epilogue_decode<12>(a, u, lane_taddr, out, alv); break;
-                    case 13: epilogue_decode<13>(a, u, lane_taddr, out, alv); break;
-                    case 14: epilogue_decode<14>(a, u, lane_taddr, out, alv); break;
-                    case 15: epilogue_decode<15>(a, u, lane_taddr, out, alv); break;
-                    default: epilogue_decode<16>(a, u, lane_taddr, out, alv); break;
+                    case 5: epilogue_decode<5>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 6: epilogue_decode<6>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 7: epilogue_decode<7>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 8: epilogue_decode<8>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 9: epilogue_decode<9>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 10: epilogue_decode<10>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 11: epilogue_decode<11>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 12: epilogue_decode<12>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 13: epilogue_decode<13>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 14: epilogue_decode<14>(a, u, lane_taddr, out, alv, al_lane); break;
+                    case 15: epilogue_decode<15>(a, u, lane_taddr, out, alv, al_lane); break;
+                    default: epilogue_decode<16>(a, u, lane_taddr, out, alv, al_lane); break;
                 }
             } else {
                 epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0]);
@@ -1326,9 +1372,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
                     // range starts exactly there.  Every later CTA starts inside the tile.
                     const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
-                    reduce_partials(a, u, etid, n_epi_warps, a.partials + (size_t)slot0 * a.slot_floats,
-                                    a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats,
-                                    2 * (size_t)a.slot_floats, c1 - c0);
+                    const float* first = a.partials + (size_t)slot0 * a.slot_floats;
+                    const float* rest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats;
+                    reduce_partials<kGen>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
                     if (etid == 0) a.counters[unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
@@ -1370,11 +1416,16 @@ extern "C" int bitdelta_debug_set_knobs(int knobs) {
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream) {
-    const int mode = !args.decode ? 0 : (args.m <= 4 ? args.m : 5);
+    // the general form only where something beyond the plain bf16 product is asked for
+    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 6 : 0;
+    const int mode = gen + (!args.decode ? 0 : (args.m <= 4 ? args.m : 5));
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmArgs);
-    static const KernelFn kernels[6] = {bitdelta_gemm_tc_kernel<0>, bitdelta_gemm_tc_kernel<1>, bitdelta_gemm_tc_kernel<2>,
-                                        bitdelta_gemm_tc_kernel<3>, bitdelta_gemm_tc_kernel<4>, bitdelta_gemm_tc_kernel<5>};
-    static int attr_device[6] = {-1, -1, -1, -1, -1, -1};
+    static const KernelFn kernels[12] = {
+        bitdelta_gemm_tc_kernel<0, false>, bitdelta_gemm_tc_kernel<1, false>, bitdelta_gemm_tc_kernel<2, false>,
+        bitdelta_gemm_tc_kernel<3, false>, bitdelta_gemm_tc_kernel<4, false>, bitdelta_gemm_tc_kernel<5, false>,
+        bitdelta_gemm_tc_kernel<0, true>,  bitdelta_gemm_tc_kernel<1, true>,  bitdelta_gemm_tc_kernel<2, true>,
+        bitdelta_gemm_tc_kernel<3, true>,  bitdelta_gemm_tc_kernel<4, true>,  bitdelta_gemm_tc_kernel<5, true>};
+    static int attr_device[12] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
