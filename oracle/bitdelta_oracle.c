@@ -20,7 +20,9 @@
  *
  * Parity pins: every function here is pinned by tests that do not reuse it
  * (hand-computed values, one-hot probes, numpy fp64 matmul on a dense S built
- * by independent Python code, brute-force Python loops, algebraic invariants).
+ * by independent Python code, brute-force Python loops, algebraic invariants;
+ * for the extended product at the end of the file also numpy's float16 on
+ * every finite pattern and closed forms of the sigmoid).
  */
 #include <stdint.h>
 #include <stdlib.h>
