@@ -34,10 +34,10 @@ PAPER_CONTEXT = "paper: 3.34x (standard) / 2.51x (batched) over autotuned Triton
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernel from the
 # ncu captures summarised under profiles/ ; None where no capture exists yet.
 NCU_TRAFFIC_BYTES = {
-    "decode_attn": 50_530_000,          # 50.48 MB read + 0.05 MB written
-    "decode_mlp_up": 234_700_000,       # 228.3 MB read + 6.4 MB written (half of W_base read twice)
-    "prefill": 74_100_000,              # 61.7 MB read + 12.4 MB written
-    "many_tenant_down": 405_000_000,    # 400.0 MB read + 4.9 MB written
+    "decode_attn": 50_510_000,          # 50.49 MB read + 0.02 MB written
+    "decode_mlp_up": 219_000_000,       # 213.7 MB read + 5.3 MB written (a third of W_base read twice)
+    "prefill": 74_000_000,              # 62.1 MB read + 12.0 MB written
+    "many_tenant_down": 416_000_000,    # 408.3 MB read + 7.6 MB written
     "tiny": None,
 }
 
