@@ -388,6 +388,18 @@ def run_ours(args):
     peaks = load_peaks()
     wl = synth.WORKLOADS_BY_NAME[args.workload]
 
+    if args.ex_only:
+        if world != 1:
+            raise RuntimeError("--ex-only is a single-GPU run")
+        r = time_gemm_ex(wl, peaks, args.steps)
+        print(json.dumps({"metric": "bitdelta_gemm_ex " + ("effective HBM GB/s" if wl.m <= 16 else "TFLOP/s"),
+                          "value": r["roofline"]["achieved"], "unit": r["roofline"]["unit"], "n_gpus": 1,
+                          "steps": args.steps, "warmup": 3, "ms_per_step": r["us_per_launch"] / 1e3,
+                          "higher_is_better": True, "dtype": "f16", "data": "synthetic",
+                          "config": {"workload": wl.name, "variant": "fp16 operands + bias + SiLU"},
+                          "roofline": r["roofline"], "gpu_launches": args.steps * kernels_per_step(wl)}), flush=True)
+        return
+
     sampler = ClockSampler(physical_gpu_index(local_rank)) if rank == 0 else None
     launches0 = bd.kernel_launch_count()
     ms, nsets, host_inputs, _sets = time_workload(wl, args.steps, args.warmup, dist, sampler)
@@ -514,6 +526,9 @@ def main():
     ap.add_argument("--all", action="store_true", help="also time the other workloads (N=1 only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ex-only", action="store_true",
+                    help="time only the extended call (fp16 operands, bias, SiLU) on --workload and print its "
+                         "line; N=1, no end-to-end or CPU leg (used for profiling that kernel instantiation)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
