@@ -189,6 +189,34 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
                        void* arena, size_t arena_bytes, void* cuda_stream);
 
 /*
+ * Plan queries (host only; no GPU is touched).  They report how bitdelta_gemm would run a shape on a
+ * device with `num_sms` multiprocessors: which schedule, how many thread blocks, and which share of the
+ * work list each block takes.  The work list is the flat list of (unit, k-step) items, unit-major: a unit
+ * is one 128-row tile of W_base for one group of TB tenants (decode schedules) or one tenant's token tile
+ * (tiled schedule), a k-step is 128 k; item = unit * P + k-step.
+ *
+ * bitdelta_gemm_plan fills info[0 .. BITDELTA_PLAN_INFO_INTS-1] (host pointer):
+ *   [0] schedule: 0 tiled, 1 decode with a pre-pass activation split, 2 decode with the in-kernel split,
+ *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then)
+ *   [1] thread blocks   [2] tenants per unit   [3] units   [4] P, k-steps per unit
+ *   [5] work order: 0 one even cut of the list, 1 whole units round-robin (block b: units b, b+blocks, ...),
+ *       2 teams (units numbered group-major, one team of blocks per tenant group, each cutting its
+ *       group's items evenly)
+ *   [6] teams (1 unless order 2)   [7] dynamic shared memory, bytes   [8] W_base ring depth
+ *   [9] activation ring depth   [10] piece ring depth   [11] operand buffers in tensor memory (per decode
+ *   group)   [12] hand-overs per k-step   [13] token tile (tiled schedule)   [14] tenant groups (decode) or
+ *   tenant x token tiles (tiled) per W_base tile   [15] W_base tiles
+ * bitdelta_gemm_plan_cta_items gives block `cta` its items [*first, *end) (orders 0 and 2; for order 1 the
+ * items of its first unit).  bitdelta_gemm_plan_item_cta returns the block that owns `item`, or -1 for a
+ * bad argument.  Errors: BITDELTA_ERR_NULL, BITDELTA_ERR_SHAPE (also: cta out of range, K % 128 != 0 for
+ * the two item queries).
+ */
+#define BITDELTA_PLAN_INFO_INTS 16
+int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info);
+int bitdelta_gemm_plan_cta_items(int B, int m, int N, int K, int num_sms, int cta, int* first, int* end);
+int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int item);
+
+/*
  * Synchronises the stream, then returns and clears the device-side status of
  * the current device: BITDELTA_OK, or BITDELTA_ERR_TIMEOUT if a bounded wait in
  * one of this library's kernels expired since the last query (its output is

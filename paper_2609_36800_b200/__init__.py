@@ -14,6 +14,9 @@ from .binding import (  # noqa: F401
     gemm_host,
     gemm_host_arena_bytes,
     gemm_noalloc,
+    gemm_plan,
+    gemm_plan_cta_items,
+    gemm_plan_item_cta,
     gemm_workspace_bytes,
     kernel_launch_count,
     last_device_status,

@@ -20,6 +20,7 @@ EXPORTS = (
     "bitdelta_pack", "bitdelta_unpack", "bitdelta_compress_workspace_bytes", "bitdelta_compress",
     "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
     "bitdelta_gemm", "bitdelta_gemm_ex", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
+    "bitdelta_gemm_plan", "bitdelta_gemm_plan_cta_items", "bitdelta_gemm_plan_item_cta",
     "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
 )
 
@@ -60,6 +61,9 @@ def load_library():
     lib.bitdelta_gemm_host_arena_bytes.argtypes = [ci, ci, ci, ci]
     lib.bitdelta_gemm_host_arena_bytes.restype = sz
     lib.bitdelta_gemm_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, sz, vp]
+    lib.bitdelta_gemm_plan.argtypes = [ci, ci, ci, ci, ci, ctypes.POINTER(ci)]
+    lib.bitdelta_gemm_plan_cta_items.argtypes = [ci, ci, ci, ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.bitdelta_gemm_plan_item_cta.argtypes = [ci, ci, ci, ci, ci, ci]
     lib.bitdelta_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.bitdelta_kernel_launch_count.restype = ctypes.c_ulonglong
     lib.bitdelta_status_string.argtypes = [ci]
@@ -187,6 +191,30 @@ def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bo
         _check(lib.bitdelta_gemm_ex(*args, bp, _dev(out, io, "out"), *shape, 1 if io == torch.float16 else 0,
                                     ACTS[act], *ws), "bitdelta_gemm_ex")
     return out
+
+
+PLAN_FIELDS = ("schedule", "blocks", "tenants_per_unit", "units", "k_steps", "order", "teams", "smem_bytes",
+               "w_ring", "x_ring", "piece_ring", "operand_buffers", "handovers_per_k_step", "token_tile", "groups",
+               "w_tiles")
+
+
+def gemm_plan(B: int, m: int, N: int, K: int, num_sms: int = 148) -> dict:
+    """How bitdelta_gemm would run this shape (host-only query): schedule, blocks, work order, ring depths."""
+    info = (ctypes.c_int * 16)()
+    _check(load_library().bitdelta_gemm_plan(B, m, N, K, num_sms, info), "bitdelta_gemm_plan")
+    return dict(zip(PLAN_FIELDS, list(info)))
+
+
+def gemm_plan_cta_items(B: int, m: int, N: int, K: int, cta: int, num_sms: int = 148):
+    """Items [first, end) of the flat (unit, k-step) work list that thread block `cta` takes."""
+    first, end = ctypes.c_int(0), ctypes.c_int(0)
+    _check(load_library().bitdelta_gemm_plan_cta_items(B, m, N, K, num_sms, cta, ctypes.byref(first), ctypes.byref(end)),
+           "bitdelta_gemm_plan_cta_items")
+    return first.value, end.value
+
+
+def gemm_plan_item_cta(B: int, m: int, N: int, K: int, item: int, num_sms: int = 148) -> int:
+    return int(load_library().bitdelta_gemm_plan_item_cta(B, m, N, K, num_sms, item))
 
 
 NOALLOC_SCRATCH_BYTES = 16 * 1024 * 1024

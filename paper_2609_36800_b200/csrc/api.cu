@@ -367,6 +367,46 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
     return BITDELTA_OK;
 }
 
+int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
+    if (!info) return BITDELTA_ERR_NULL;
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 32) != 0 || num_sms <= 0) return BITDELTA_ERR_SHAPE;
+    for (int i = 0; i < BITDELTA_PLAN_INFO_INTS; ++i) info[i] = 0;
+    if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
+    bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
+    if (!p.ok) return BITDELTA_ERR_SHAPE;
+    info[0] = !p.decode ? 0 : (p.convert ? 2 : 1);
+    info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
+    info[5] = p.whole_units ? 1 : (p.teams > 1 ? 2 : 0);
+    info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;
+    info[11] = p.a_slots; info[12] = p.halves; info[13] = p.tok_tile; info[14] = p.groups; info[15] = p.n_tiles;
+    return BITDELTA_OK;
+}
+
+int bitdelta_gemm_plan_cta_items(int B, int m, int N, int K, int num_sms, int cta, int* first, int* end) {
+    if (!first || !end) return BITDELTA_ERR_NULL;
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 128) != 0 || num_sms <= 0) return BITDELTA_ERR_SHAPE;
+    bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
+    if (!p.ok || cta < 0 || cta >= p.grid) return BITDELTA_ERR_SHAPE;
+    if (p.whole_units) {
+        *first = cta * p.P;
+        *end = *first + p.P;
+        return BITDELTA_OK;
+    }
+    const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
+    *first = bd::cta_first_item(a, cta);
+    *end = bd::cta_first_item(a, cta + 1);
+    return BITDELTA_OK;
+}
+
+int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int item) {
+    if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 128) != 0 || num_sms <= 0) return -1;
+    bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
+    if (!p.ok || item < 0 || item >= p.T) return -1;
+    if (p.whole_units) return (item / p.P) % p.grid;
+    const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
+    return bd::cta_of_item(a, item);
+}
+
 int bitdelta_last_device_status(void* cuda_stream, int* site) {
     unsigned int st[2] = {0, 0};
     if (bd::read_device_status(st, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return BITDELTA_ERR_CUDA;

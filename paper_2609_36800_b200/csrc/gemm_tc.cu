@@ -145,30 +145,6 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return wait_bar_slow(bar, parity, abort_flag, site);
 }
 
-// Work split.  The T = q*G + r items (T < 2^30) are cut evenly across the G CTAs: CTA b owns
-// [b*q + min(b, r), ...), i.e. the first r CTAs take q+1 items.  32-bit arithmetic only: 64-bit
-// divisions cost several hundred cycles each and sit on the start-up and tail paths.
-// With teams (one per tenant group, cpt CTAs each) the same cut is applied to each team's Tg items.
-__device__ __forceinline__ int cta_first_item(const GemmArgs& a, int b) {
-    int base = 0;
-    if (a.teams > 1) {
-        const int t = (int)((unsigned)b / (unsigned)a.cpt);
-        b -= t * a.cpt;
-        base = t * a.Tg;
-    }
-    return base + b * a.q + min(b, a.r);
-}
-__device__ __forceinline__ int cta_of_item(const GemmArgs& a, int i) {
-    int base = 0;
-    if (a.teams > 1) {
-        const int t = (int)((unsigned)i / (unsigned)a.Tg);
-        i -= t * a.Tg;
-        base = t * a.cpt;
-    }
-    const int big = a.r * (a.q + 1);
-    return base + ((i < big) ? (int)((unsigned)i / (unsigned)(a.q + 1)) : a.r + (int)((unsigned)(i - big) / (unsigned)a.q));
-}
-
 // Walks the k-pair items [lo, hi) of this CTA as segments (unit, p0, p1).
 struct SegIter {
     int cur, hi;

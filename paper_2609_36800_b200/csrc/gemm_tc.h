@@ -51,6 +51,36 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     return a;
 }
 
+#ifdef __CUDACC__
+#define BD_HD __host__ __device__ __forceinline__
+#else
+#define BD_HD inline
+#endif
+// Work split.  The T = q*G + r items (T < 2^30) are cut evenly across the G CTAs: CTA b owns
+// [b*q + min(b, r), ...), i.e. the first r CTAs take q+1 items.  32-bit arithmetic only: 64-bit
+// divisions cost several hundred cycles each and sit on the kernel's start-up and tail paths.
+// With teams (one per tenant group, cpt CTAs each) the same cut is applied to each team's Tg items.
+// (Host and device: the kernel uses them, and the plan queries of the C ABI report them.)
+BD_HD int cta_first_item(const GemmArgs& a, int b) {
+    int base = 0;
+    if (a.teams > 1) {
+        const int t = (int)((unsigned)b / (unsigned)a.cpt);
+        b -= t * a.cpt;
+        base = t * a.Tg;
+    }
+    return base + b * a.q + (b < a.r ? b : a.r);
+}
+BD_HD int cta_of_item(const GemmArgs& a, int i) {
+    int base = 0;
+    if (a.teams > 1) {
+        const int t = (int)((unsigned)i / (unsigned)a.Tg);
+        i -= t * a.Tg;
+        base = t * a.cpt;
+    }
+    const int big = a.r * (a.q + 1);
+    return base + ((i < big) ? (int)((unsigned)i / (unsigned)(a.q + 1)) : a.r + (int)((unsigned)(i - big) / (unsigned)a.q));
+}
+
 // Workspace regions of the decode schedule.
 inline uint8_t* ws_x8(const Plan& p, void* workspace) {
     return reinterpret_cast<uint8_t*>(workspace) + p.ws_header_bytes + p.ws_partials_bytes;
