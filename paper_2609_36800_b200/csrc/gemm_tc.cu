@@ -105,8 +105,8 @@ struct Ctl {
     uint64_t xfull[kMaxStages];        // bf16 activation tile landed
     uint64_t xempty[kMaxStages];       // ... and was read by the base MMAs (and by the in-kernel split)
     uint64_t x8empty[kMaxStages];      // decode: piece tile free again (both delta issuers' MMAs completed)
-    uint64_t bfull[kBitSlots];
-    uint64_t bempty[kBitSlots];
+    uint64_t bfull[kMaxBitSlots];
+    uint64_t bempty[kMaxBitSlots];
     uint64_t afull[kMaxASlots];        // tiled schedule: decoded operand ready (decode warps -> MMA warp)
     uint64_t aempty[2 * kMaxASlots];   // operand buffer free again (tcgen05.commit); decode: [group][buffer]
     uint64_t accfull;
@@ -513,7 +513,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const uint32_t bits_off = x8_off + a.n_x8 * a.x8_atom_bytes;         // sign-word slots
     const uint32_t bits_addr = base + bits_off;
     uint8_t* bits_ptr = smem + bits_off;
-    Ctl* ctl = reinterpret_cast<Ctl*>(smem + bits_off + kBitSlots * a.bslot_bytes);
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + bits_off + a.n_bits * a.bslot_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
     constexpr bool kDec = kMode != 0;
@@ -591,7 +591,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             mbar_init(smem_u32(&ctl->x8full[s]), (kDec && convert) ? 128 : 1);   // splitter threads, or one TMA load
             mbar_init(smem_u32(&ctl->x8empty[s]), 2);                            // the two delta issuers
         }
-        for (int s = 0; s < kBitSlots; ++s) {
+        for (int s = 0; s < kMaxBitSlots; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
             mbar_init(smem_u32(&ctl->bempty[s]), kDec ? 8 : 4);
         }
@@ -651,9 +651,25 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         bool more_p = false;
         Unit up{};
         if (more_p) up = unit_info(a, pi.unit);
+        // Tiled schedule: the sign words are a stream of their own (one small load per k-pair and unit into a
+        // deep ring), so that they run far ahead of the W_base tiles: the decode warps work several stages
+        // ahead of the MMAs.  In the decode schedules they travel with the W_base stream.
+        ItemIter bi(it);
+        bool more_b = !kDec && bi.next();
+        Unit ub{};
+        auto next_pair = [&]() {   // to the next item that starts a k-pair of its segment
+            do {
+                more_b = bi.next();
+            } while (more_b && !bi.first && (bi.p & 1));
+            if (more_b && bi.first) ub = unit_info(a, bi.unit);
+        };
+        if (more_b) {
+            ub = unit_info(a, bi.unit);
+            next_pair();   // the first pair was queued in the prologue
+        }
         if (more_w) {
             // queued by thread 0 in the prologue: W stage 0, sign-word slot 0
-            bslot = 1 % kBitSlots; bphase = (kBitSlots == 1) ? 1u : 0u;
+            bslot = 1; bphase = 0u;   // (at least two sign-word slots)
             stage = 1 % a.n_w; phase = (a.n_w == 1) ? 1u : 0u;
             BD_TL(0);
             uw = unit_info(a, wi.unit);
@@ -668,7 +684,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         long long idle_b = 0, idle_w = 0;
 #endif
         BD_ACC_DECL(t_x); BD_ACC_DECL(t_p); BD_ACC_DECL(t_w); BD_ACC_DECL(n_iter);
-        while (more_w || more_x || more_p) {
+        while (more_w || more_x || more_p || more_b) {
             bool did = false;
 #ifdef BD_TRACE
             ++n_iter;
@@ -718,6 +734,23 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
             }
             BD_ACC_END(t_p, tp0);
+            if (!kDec && more_b) {
+                if (warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) {
+                    if (elect_one()) {
+                        const uint32_t bbar = smem_u32(&ctl->bfull[bslot]);
+                        if (BD_KNOB(8)) {
+                            mbar_arrive(bbar);
+                        } else {
+                            mbar_arrive_expect_tx(bbar, a.bslot_bytes);
+                            tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (bi.p >> 1) * 8, ub.n0, ub.tenant0);
+                        }
+                    }
+                    __syncwarp();
+                    if (++bslot == a.n_bits) { bslot = 0; bphase ^= 1; }
+                    next_pair();
+                    did = true;
+                }
+            }
             BD_ACC_BEGIN(tw0);
             if (more_w && hold) {
                 // The first sign-word load of a tile pulls whole 128-byte lines (the signs of 1024 k) out of
@@ -725,7 +758,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 hold = !warp_all(mbar_test_wait(smem_u32(&ctl->bfull[0]), 0));
             }
             if (more_w && !hold) {
-                const bool need_slot = wi.first || !(wi.p & 1);
+                const bool need_slot = kDec && (wi.first || !(wi.p & 1));
                 if ((!need_slot || warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) &&
                     warp_all(mbar_test_wait(smem_u32(&ctl->wempty[stage]), phase ^ 1))) {
                     BD_ACC_BEGIN(ti);
@@ -733,7 +766,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     __syncwarp();
                     BD_ACC_END(w_bempty, ti);
                     BD_TL(0);
-                    if (need_slot && ++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                    if (need_slot && ++bslot == a.n_bits) { bslot = 0; bphase ^= 1; }
                     if (++stage == a.n_w) { stage = 0; phase ^= 1; }
                     more_w = wi.next();
                     if (more_w && wi.first) uw = unit_info(a, wi.unit);
@@ -755,6 +788,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             BD_ACC_BEGIN(te);
             if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 64u);
             else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 64u);
+            else if (more_b) (void)mbar_try_wait_hint(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, 64u);
             else (void)mbar_try_wait_hint(dep_ok ? (kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot])) : depbar,
                                           dep_ok ? (xphase ^ 1) : 0u, 64u);
             BD_ACC_END(w_empty, te);
@@ -1167,7 +1201,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if ((p & 1) || p == p1 - 1) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl->bempty[bslot]));
-                    if (++bslot == kBitSlots) { bslot = 0; bphase ^= 1; }
+                    if (++bslot == a.n_bits) { bslot = 0; bphase ^= 1; }
                 }
             }
         }

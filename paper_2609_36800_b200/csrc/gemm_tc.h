@@ -19,7 +19,7 @@ struct GemmArgs {
     int teams, Tg, cpt, n_tiles;   // work split by teams (see plan.h); q, r then describe one team's cut
     int T;             // work items (< 2^30)
     int q, r;          // T = q * grid + r
-    int n_w, n_x, n_x8, a_slots, halves;
+    int n_w, n_x, n_x8, n_bits, a_slots, halves;
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
@@ -38,7 +38,7 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.whole_units = p.whole_units;
     a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = p.grid / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
-    a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
+    a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;

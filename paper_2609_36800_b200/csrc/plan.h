@@ -12,7 +12,7 @@ constexpr int kPairK = 128;          // reduction extent of one pipeline stage (
 constexpr int kAtomK = 64;           // bf16 elements in one 128-byte swizzled row
 constexpr int kQuadK = 256;          // reduction extent of one sign-word slot (8 words = 32 bytes per row)
 constexpr int kMaxStages = 8;
-constexpr int kBitSlots = 2;
+constexpr int kMaxBitSlots = 8;   // sign-word slots in shared memory: 2 in the decode schedules, up to 8 (small ones) in the tiled one
 constexpr int kMaxASlots = 4;
 constexpr int kPieces = 4;           // e5m2 pieces an activation is split into for the decode-regime delta MMA
 constexpr int kTmemCols = 512;
@@ -47,6 +47,7 @@ struct Plan {
     int n_w;           // ring of W_base tiles (128 rows x 128 k of bf16 each)
     int n_x;           // ring of bf16 activation tiles
     int n_x8;          // decode: ring of e5m2 piece tiles
+    int n_bits;        // sign-word slots (each holds the signs of one k-pair of one unit)
     int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
@@ -152,7 +153,11 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     // are written in place by the in-kernel split), but stay in use until the last delta MMA of their
     // stage has completed, which is the longest hold of all: three of them.  Every remaining byte goes to
     // W_base.  The tiled schedule keeps one ring (activation tile s lives and dies with W_base tile s).
-    const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - kBitSlots * (int)p.bslot_bytes;
+    // Sign words: two slots in the decode schedules (16-64 KB each; they travel with the W_base stream).  In the
+    // tiled schedule a slot is 4 KB and the words have a stream of their own that runs well ahead of W_base:
+    // the decode warps need them long before the MMAs of their stage (they fill a ring of operand buffers).
+    p.n_bits = p.decode ? 2 : kMaxBitSlots;
+    const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - p.n_bits * (int)p.bslot_bytes;
     if (p.decode) {
         p.n_x8 = 3;
         p.n_x = (p.x_tile_bytes <= 4 * 1024) ? 3 : 2;
@@ -180,7 +185,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     }
     if (p.n_w < 2) return p;
     p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
-                   kBitSlots * p.bslot_bytes + kSmemCtrlBytes;
+                   p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
     // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
     if (p.smem_bytes < 120 * 1024) p.smem_bytes = 120 * 1024;
 
