@@ -198,7 +198,8 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
  * bitdelta_gemm_plan fills info[0 .. BITDELTA_PLAN_INFO_INTS-1] (host pointer):
  *   [0] schedule: 0 tiled, 1 decode with a pre-pass activation split, 2 decode with the in-kernel split,
  *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then)
- *   [1] thread blocks   [2] tenants per unit   [3] units   [4] P, k-steps per unit
+ *   [1] thread blocks   [2] tenants per unit (tiled schedule: more than one in the middle regime,
+ *       16 < m <= 64, where several tenants share a W_base tile)   [3] units   [4] P, k-steps per unit
  *   [5] work order: 0 one even cut of the list, 1 whole units round-robin (block b: units b, b+blocks, ...),
  *       2 teams (units numbered group-major, one team of blocks per tenant group, each cutting its
  *       group's items evenly)

@@ -202,11 +202,11 @@ struct Unit {
     int ntok;      // output tokens of this unit (rows xrow0 .. xrow0+ntok-1)
 };
 
-template <bool kDec>
+template <bool kDec, bool kGrouped>
 __device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am) {
     Unit u;
     int nt, g;
-    if (kDec && a.teams > 1) {   // group-major
+    if ((kDec || kGrouped) && a.teams > 1) {   // group-major (never in the one-tenant tiled schedule)
         g = (int)((unsigned)unit / (unsigned)a.n_tiles);
         nt = unit - g * a.n_tiles;
     } else {
@@ -214,7 +214,7 @@ __device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am)
         g = unit - nt * a.groups;
     }
     u.n0 = nt * kTileN;
-    if constexpr (kDec) {
+    if constexpr (kDec || kGrouped) {   // decode schedules, and the tiled schedule with several tenants per unit
         u.tenant0 = g * a.TB;
         u.nten = min(a.TB, a.B - u.tenant0);
         u.xrow0 = u.tenant0 * am;
@@ -360,6 +360,29 @@ __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u,
     }
 }
 
+// Tiled schedule with several tenants per unit (16 < m <= 64): tenant j's base columns start at j*m, its delta
+// columns at j*Nd; 16-token chunks, dealt alternately to the two warps of a lane quadrant.
+// `al_lane`: lane l holds the scale of the unit's tenant l.
+template <class Out>
+__device__ __forceinline__ void epilogue_tiled_grouped(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, int m,
+                                                       const Out& out, int half, float al_lane) {
+    const int chunks = (m + 15) >> 4;
+#pragma unroll 1
+    for (int c = half; c < u.nten * chunks; c += 2) {
+        const int j = c / chunks, t0 = (c - j * chunks) * 16;
+        uint32_t rb[16], rd[16];
+        tmem_ld16(lane_taddr + (uint32_t)(j * m + t0), rb);
+        tmem_ld16(lane_taddr + a.col_delta + (uint32_t)(j * a.Nd + t0), rd);
+        tc_wait_ld();
+        const float al = __shfl_sync(0xFFFFFFFFu, al_lane, j);
+        const int nvalid = min(16, m - t0);
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+            if (t < nvalid) out.put(j * m + t0 + t, fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t])));
+        }
+    }
+}
+
 __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 // Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
@@ -491,7 +514,8 @@ __device__ __forceinline__ void decode_word_e5m2(uint32_t w, uint32_t* r) {
 
 __device__ __forceinline__ void epi_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
-// kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m.
+// kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m;
+// 6: tiled schedule with several tenants per unit.
 // One instantiation per mode keeps each launched kernel's code small (the roles' loops then stay in the
 // instruction caches) and turns the schedule switches into compile-time constants.
 // kGen: the general form (binary16 I/O, bias, activation); false compiles the plain bf16 product alone, whose
@@ -516,11 +540,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + bits_off + a.n_bits * a.bslot_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
-    constexpr bool kDec = kMode != 0;
+    constexpr bool kGrouped = kMode == 6;   // tiled schedule with several tenants per unit (16 < m <= 64)
+    constexpr bool kDec = kMode != 0 && !kGrouped;
     const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
     const bool convert = kDec && a.convert != 0;
     const bool io_f16 = kGen && a.f16 != 0;
-    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec>(aa, un, am); };
+    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec, kGrouped>(aa, un, am); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     BD_KNOB_LOAD;
@@ -1306,8 +1331,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 #pragma unroll
             for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
             float al_lane = 0.f, bias_n = 0.f;
+            if constexpr (kGen || kGrouped) al_lane = (lane < u.nten) ? __ldg(a.alpha + u.tenant0 + lane) : 0.f;   // lane l: tenant l's scale
             if constexpr (kGen) {
-                al_lane = (lane < u.nten) ? __ldg(a.alpha + u.tenant0 + lane) : 0.f;   // lane l: tenant l's scale
                 if (a.bias && n < a.N) bias_n = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n), a.f16);
             }
             if (splitter) {
@@ -1349,7 +1374,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     default: epilogue_decode<16>(a, u, lane_taddr, out, alv, al_lane); break;
                 }
             } else {
-                epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0]);
+                if constexpr (kGrouped) epilogue_tiled_grouped(a, u, lane_taddr, am, out, ehalf, al_lane);
+                else epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0]);
             }
             tc_fence_before();
             __syncwarp();
@@ -1427,15 +1453,18 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream) {
     // the general form only where something beyond the plain bf16 product is asked for
-    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 6 : 0;
-    const int mode = gen + (!args.decode ? 0 : (args.m <= 4 ? args.m : 5));
+    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 7 : 0;
+    // 0 tiled, 1..4 decode with that many tokens per tenant, 5 decode with 5..16, 6 tiled with several tenants per unit
+    const int mode = gen + (!args.decode ? (args.win_rows > 0 ? 6 : 0) : (args.m <= 4 ? args.m : 5));
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmArgs);
-    static const KernelFn kernels[12] = {
+    static const KernelFn kernels[14] = {
         bitdelta_gemm_tc_kernel<0, false>, bitdelta_gemm_tc_kernel<1, false>, bitdelta_gemm_tc_kernel<2, false>,
         bitdelta_gemm_tc_kernel<3, false>, bitdelta_gemm_tc_kernel<4, false>, bitdelta_gemm_tc_kernel<5, false>,
+        bitdelta_gemm_tc_kernel<6, false>,
         bitdelta_gemm_tc_kernel<0, true>,  bitdelta_gemm_tc_kernel<1, true>,  bitdelta_gemm_tc_kernel<2, true>,
-        bitdelta_gemm_tc_kernel<3, true>,  bitdelta_gemm_tc_kernel<4, true>,  bitdelta_gemm_tc_kernel<5, true>};
-    static int attr_device[12] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
+        bitdelta_gemm_tc_kernel<3, true>,  bitdelta_gemm_tc_kernel<4, true>,  bitdelta_gemm_tc_kernel<5, true>,
+        bitdelta_gemm_tc_kernel<6, true>};
+    static int attr_device[14] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;

@@ -86,6 +86,27 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
+    } else if (m <= 64 && B > 1 && tb_override != 1) {
+        // Tiled schedule, middle regime (16 < m <= 64): a unit holds several tenants, whose tokens share one
+        // W_base tile and one base MMA (N = all their tokens); every tenant keeps its own delta accumulator
+        // (N = m rounded up to 16) and its own operand buffer of decoded signs.  Tenant j's delta MMAs read the
+        // activation rows from j*m on: a window that runs into the next tenant's rows, whose columns are ignored.
+        p.tok_tile = round_up(m, 16);
+        p.m_tiles = 1;
+        p.Nd = p.tok_tile;
+        const int tb_max = 128 / p.Nd;                  // 4 tenants up to m = 32, 2 up to m = 64
+        p.TB = B < tb_max ? B : tb_max;
+        p.groups = (B + p.TB - 1) / p.TB;
+        p.Nb = round_up(p.TB * m, 16);
+        p.win_rows = m;
+        p.chunk_rows = 16;
+        p.x_rows = round_up((p.TB - 1) * m + p.Nd, 8);
+        if (p.x_rows < p.Nb) p.x_rows = p.Nb;
+        p.N3 = 0;
+        p.convert = 0;
+        p.x8_rows = 0;
+        p.aslot_cols = 64;
+        p.slot_floats = (size_t)kTileN * p.TB * m;
     } else {
         p.TB = 1;
         p.tok_tile = m >= 128 ? 128 : round_up(m, 16);
@@ -120,7 +141,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     // whole_override (experiments): 1 whole units, 3 teams, 2 not whole units, 4 plain cut.
     p.whole_units = 0;
     p.teams = 1;
-    if (p.decode && p.groups > 1) {
+    if ((p.decode || p.win_rows > 0) && p.groups > 1) {   // (not the tiled schedule with one tenant per unit)
         double s_whole = 0.0, s_teams = 0.0;
         if (p.units >= max_grid) {
             const int rounds = (p.units + max_grid - 1) / max_grid;
@@ -156,7 +177,12 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     // Sign words: two slots in the decode schedules (16-64 KB each; they travel with the W_base stream).  In the
     // tiled schedule a slot is 4 KB and the words have a stream of their own that runs well ahead of W_base:
     // the decode warps need them long before the MMAs of their stage (they fill a ring of operand buffers).
-    p.n_bits = p.decode ? 2 : kMaxBitSlots;
+    p.n_bits = 2;
+    if (!p.decode) {
+        p.n_bits = (int)(32768u / p.bslot_bytes);
+        if (p.n_bits > kMaxBitSlots) p.n_bits = kMaxBitSlots;
+        if (p.n_bits < 2) p.n_bits = 2;
+    }
     const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - p.n_bits * (int)p.bslot_bytes;
     if (p.decode) {
         p.n_x8 = 3;
@@ -209,7 +235,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     // Workspace: arrival counters, two partial-result slots per CTA, then (decode) the e5m2
     // pieces of X written by the activation-split kernel.
     p.ws_header_bytes = (size_t)round_up(p.units * 4, 1024);
-    p.ws_partials_bytes = (size_t)2 * kMaxCtas * p.slot_floats * sizeof(float);
+    // (sized for the largest grid any device could get, so that the size does not depend on the device;
+    // never more CTAs than items)
+    const long long max_ctas = p.T < kMaxCtas ? p.T : kMaxCtas;
+    p.ws_partials_bytes = (size_t)2 * (size_t)max_ctas * p.slot_floats * sizeof(float);
     p.ws_x8_bytes = p.decode ? (((size_t)B * kPieces * m * K + 1023) / 1024 * 1024) : 0;
     p.ws_bytes = p.ws_header_bytes + p.ws_partials_bytes + p.ws_x8_bytes;
     p.ok = true;

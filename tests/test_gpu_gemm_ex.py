@@ -40,6 +40,8 @@ SHAPES = [
     (7, 9, 256, 256),
     (2, 17, 256, 384),
     (2, 100, 300, 640),
+    (5, 20, 384, 512),
+    (3, 33, 264, 384),
     (1, 200, 520, 384),
     (12, 8, 6400, 256),
     (33, 2, 1920, 384),

@@ -96,6 +96,11 @@ SMALL = [
     (12, 8, 6400, 256),   # many tiles x three groups: one team of CTAs per group, tiles cut across CTAs
     (33, 2, 1920, 384),   # five teams, a partly filled last group
     (80, 1, 3712, 256),   # ten groups do not divide the SMs well: whole-unit work order
+    (5, 20, 384, 512),    # middle regime: four tenants per unit share a W_base tile, last group has one tenant
+    (3, 33, 264, 384),    # two tenants per unit, 48-column delta accumulators, ragged N
+    (4, 64, 256, 512),    # two tenants of 64 tokens fill the 128 base columns
+    (9, 24, 1280, 1024),  # three groups of tenants: teams of CTAs
+    (6, 48, 200, 256),
 ]
 
 

@@ -11,6 +11,7 @@ SHAPES = [(w.B, w.m, w.N, w.K) for w in synth.WORKLOADS] + [
     (1, 1, 128, 128), (2, 1, 200, 256), (20, 1, 128, 256), (12, 8, 6400, 256), (33, 2, 1920, 384),
     (80, 1, 3712, 256), (3, 16, 264, 384), (2, 17, 256, 384), (2, 300, 136, 512), (16, 4, 4096, 8192),
     (5, 3, 130, 384), (64, 2, 512, 1024), (24, 2, 1280, 1024), (7, 9, 256, 256),
+    (5, 20, 384, 512), (9, 24, 1280, 1024), (8, 32, 4096, 4096), (8, 64, 4096, 4096),
 ]
 
 
