@@ -197,7 +197,9 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
  *
  * bitdelta_gemm_plan fills info[0 .. BITDELTA_PLAN_INFO_INTS-1] (host pointer):
  *   [0] schedule: 0 tiled, 1 decode with a pre-pass activation split, 2 decode with the in-kernel split,
- *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then)
+ *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then), 4 tiled on pairs of
+ *       thread blocks (a unit is then two W_base tiles, [3] and the work list count such pairs, and [1] is
+ *       twice the number of pairs that cut the list)
  *   [1] thread blocks   [2] tenants per unit (tiled schedule: more than one in the middle regime,
  *       16 < m <= 64, where several tenants share a W_base tile)   [3] units   [4] P, k-steps per unit
  *   [5] work order: 0 one even cut of the list, 1 whole units round-robin (block b: units b, b+blocks, ...),
@@ -208,8 +210,9 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
  *   group)   [12] hand-overs per k-step   [13] token tile (tiled schedule)   [14] tenant groups (decode) or
  *   tenant x token tiles (tiled) per W_base tile   [15] W_base tiles
  * bitdelta_gemm_plan_cta_items gives block `cta` its items [*first, *end) (orders 0 and 2; for order 1 the
- * items of its first unit).  bitdelta_gemm_plan_item_cta returns the block that owns `item`, or -1 for a
- * bad argument.  Errors: BITDELTA_ERR_NULL, BITDELTA_ERR_SHAPE (also: cta out of range, K % 128 != 0 for
+ * items of its first unit; for schedule 4 both blocks of a pair report the pair's items).
+ * bitdelta_gemm_plan_item_cta returns the block that owns `item` (schedule 4: the first block of the pair), or
+ * -1 for a bad argument.  Errors: BITDELTA_ERR_NULL, BITDELTA_ERR_SHAPE (also: cta out of range, K % 128 != 0 for
  * the two item queries).
  */
 #define BITDELTA_PLAN_INFO_INTS 16

@@ -284,6 +284,14 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     }
 
     bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override());
+    if (p.ok && p.pair) {
+        // The pair schedule wants every pair resident at once (a cluster of two needs two free SMs of one
+        // cluster-capable group); where the device cannot do that, run the one-CTA schedule.  Asked once per device.
+        static int pairs_fit[64] = {};   // 0 unknown, 1 yes, -1 no
+        const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
+        if (pairs_fit[di] == 0) pairs_fit[di] = (2 * bd::max_active_pairs(p.smem_bytes) >= p.grid) ? 1 : -1;
+        if (pairs_fit[di] < 0) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false);
+    }
     if (!p.ok) return BITDELTA_ERR_SHAPE;
     if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
@@ -374,7 +382,7 @@ int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
     if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
-    info[0] = !p.decode ? 0 : (p.convert ? 2 : 1);
+    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.convert ? 2 : 1);
     info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
     info[5] = p.whole_units ? 1 : (p.teams > 1 ? 2 : 0);
     info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;
@@ -393,8 +401,9 @@ int bitdelta_gemm_plan_cta_items(int B, int m, int N, int K, int num_sms, int ct
         return BITDELTA_OK;
     }
     const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
-    *first = bd::cta_first_item(a, cta);
-    *end = bd::cta_first_item(a, cta + 1);
+    const int cutter = p.pair ? cta / 2 : cta;   // both blocks of a pair take the pair's items
+    *first = bd::cta_first_item(a, cutter);
+    *end = bd::cta_first_item(a, cutter + 1);
     return BITDELTA_OK;
 }
 
@@ -404,7 +413,7 @@ int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int ite
     if (!p.ok || item < 0 || item >= p.T) return -1;
     if (p.whole_units) return (item / p.P) % p.grid;
     const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
-    return bd::cta_of_item(a, item);
+    return p.pair ? 2 * bd::cta_of_item(a, item) : bd::cta_of_item(a, item);   // (pairs: the pair's first block)
 }
 
 int bitdelta_last_device_status(void* cuda_stream, int* site) {

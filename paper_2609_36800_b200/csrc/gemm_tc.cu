@@ -202,8 +202,8 @@ struct Unit {
     int ntok;      // output tokens of this unit (rows xrow0 .. xrow0+ntok-1)
 };
 
-template <bool kDec, bool kGrouped>
-__device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am) {
+template <bool kDec, bool kGrouped, bool kPair = false>
+__device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am, int rank = 0) {
     Unit u;
     int nt, g;
     if ((kDec || kGrouped) && a.teams > 1) {   // group-major (never in the one-tenant tiled schedule)
@@ -213,6 +213,7 @@ __device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am)
         nt = unit / a.groups;
         g = unit - nt * a.groups;
     }
+    if constexpr (kPair) nt = 2 * nt + rank;   // the pair's two W_base tiles
     u.n0 = nt * kTileN;
     if constexpr (kDec || kGrouped) {   // decode schedules, and the tiled schedule with several tenants per unit
         u.tenant0 = g * a.TB;
@@ -541,11 +542,16 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
     constexpr bool kGrouped = kMode == 6;   // tiled schedule with several tenants per unit (16 < m <= 64)
-    constexpr bool kDec = kMode != 0 && !kGrouped;
+    constexpr bool kPair = kMode == 7;      // tiled schedule on CTA pairs (cluster of two, 256-row MMAs)
+    constexpr bool kDec = kMode >= 1 && kMode <= 5;
+    // Pair schedule: this CTA's rank in its cluster (0 = leader, issues the MMAs), the leader's view of
+    // the barriers both CTAs signal, and the work share of the CLUSTER.
+    const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+    const int cta_id = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // index into the work split
     const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
     const bool convert = kDec && a.convert != 0;
     const bool io_f16 = kGen && a.f16 != 0;
-    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec, kGrouped>(aa, un, am); };
+    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec, kGrouped, kPair>(aa, un, am, (int)rank); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     BD_KNOB_LOAD;
@@ -563,8 +569,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     }
 
     // Work: either an even share of the flat item list, or (whole-unit order) units b, b+grid, ...
-    const int lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
-    const int hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
+    const int lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, cta_id);
+    const int hi = a.whole_units ? (int)a.T : cta_first_item(a, cta_id + 1);
     SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
     int unit, p0, p1;
 
@@ -576,7 +582,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const uint32_t bar = smem_u32(&ctl->wfull[stage]);
         const uint32_t dst = w_addr + stage * a.w_stage_bytes;
         const int k0 = p * kPairK;
-        if (BD_KNOB(16)) {
+        if constexpr (kPair) {
+            // Both CTAs' tiles of the stage (W_base and half an activation tile each) are counted on the
+            // leader's barrier, which only the leader arms.
+            if (rank == 0) mbar_arrive_expect_tx(bar, 2u * (a.w_stage_bytes + 2 * a.x_atom_bytes));
+            tma_load_3d_pair(dst, &tmW, mapa_shared(bar, 0), 0, u.n0, k0 / kAtomK);
+        } else if (BD_KNOB(16)) {
             mbar_arrive(bar);
         } else {
             // tiled schedule: the stage's activation tile (same slot index, queued by the activation
@@ -620,28 +631,41 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
             mbar_init(smem_u32(&ctl->bempty[s]), kDec ? 8 : 4);
         }
-        for (int s = 0; s < kMaxASlots; ++s) mbar_init(smem_u32(&ctl->afull[s]), 4);
+        for (int s = 0; s < kMaxASlots; ++s) mbar_init(smem_u32(&ctl->afull[s]), kPair ? 8 : 4);   // (pair: both CTAs' decode warps)
         for (int s = 0; s < 2 * kMaxASlots; ++s) mbar_init(smem_u32(&ctl->aempty[s]), 1);
         mbar_init(smem_u32(&ctl->accfull), kDec ? 3 : 1);
-        mbar_init(smem_u32(&ctl->accempty), kDec ? 4 : 8);
+        mbar_init(smem_u32(&ctl->accempty), kDec ? 4 : (kPair ? 16 : 8));
         mbar_init(smem_u32(&ctl->depready), 1);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
         // The first item's weights are requested right here, before the rest of the CTA is set up:
         // every cycle until the first load is queued is added to the launch's latency.
-        if (lo < hi) {
+        // (pair schedule: not before the other CTA's barriers exist, i.e. after the cluster barrier below)
+        if (!kPair && lo < hi) {
             const int unit0 = (int)((unsigned)lo / (unsigned)a.P);
             issue_weights_raw(unit_info(a, unit0), a.whole_units ? 0 : lo - unit0 * a.P, 0, 0, true);
         }
         BD_STAMP(2);
     }
     if (warp == kWarpTmem) {
-        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
-        tmem_relinquish();
+        if constexpr (kPair) {
+            tmem_alloc_pair(smem_u32(&ctl->tmem_base), kTmemCols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) {
+        cluster_sync_all();   // both CTAs' barriers are initialised and both hold their tensor memory
+        if (threadIdx.x == 0 && lo < hi) {
+            const int unit0 = (int)((unsigned)lo / (unsigned)a.P);
+            issue_weights_raw(unit_info(a, unit0), lo - unit0 * a.P, 0, 0, true);
+        }
+    }
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     if (warp == 0) BD_STAMP(1);
@@ -723,7 +747,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint32_t bar = kDec ? smem_u32(&ctl->xfull[xslot]) : smem_u32(&ctl->wfull[xslot]);
                         const uint32_t dst = x_addr + xslot * a.x_tile_bytes;
                         const int k0 = xi.p * kPairK;
-                        if (x_tx) {
+                        if constexpr (kPair) {
+                            // this CTA's half of the token tile, counted on the leader's barrier
+                            tma_load_3d_pair(dst, &tmX, mapa_shared(bar, 0), 0, ux.xrow0 + (int)rank * (a.tok_tile / 2), k0 / kAtomK);
+                        } else if (x_tx) {
                             if (kDec) mbar_arrive_expect_tx(bar, x_tx);
                             tma_load_3d(dst, &tmX, bar, 0, ux.xrow0, k0 / kAtomK);   // both 64-k atoms
                         } else if (kDec) {
@@ -843,9 +870,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         //   tiled schedule : one item = one tenant x 128 k of bf16 signs (64 columns, 8 MMAs of K=16)
         //   decode schedule: one item = all tenants of the unit x 64 k of e5m2 signs (16 columns per
         //                    tenant, 2 MMAs of K=32 per tenant)
-        const uint32_t idesc_base = io_f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nb) : make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+        constexpr uint32_t kM = kPair ? 2 * kTileN : kTileN;   // MMA M: both CTAs' weight rows in the pair schedule
+        const uint32_t idesc_base = io_f16 ? make_idesc_f16(kM, (uint32_t)a.Nb) : make_idesc_bf16(kM, (uint32_t)a.Nb);
         const uint32_t idesc_delta = kDec ? make_idesc_e5m2(kTileN, (uint32_t)a.Nd)
-                                          : (io_f16 ? make_idesc_f16(kTileN, (uint32_t)a.Nd) : make_idesc_bf16(kTileN, (uint32_t)a.Nd));
+                                          : (io_f16 ? make_idesc_f16(kM, (uint32_t)a.Nd) : make_idesc_bf16(kM, (uint32_t)a.Nd));
         // Descriptor of a tile = descriptor of address 0 plus (address >> 4): addresses stay below
         // 256 KiB, so the sum never carries out of the 14-bit start-address field.
         const uint64_t desc0 = make_smem_desc_sw128(0);
@@ -860,7 +888,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         grid_dependency_wait();
         if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));
         BD_STAMP(31);
-        while (ok && it.next(unit, p0, p1)) {
+        // (pair schedule: only the leader's warp issues; its MMAs and commits act on both CTAs)
+        while (ok && (!kPair || rank == 0) && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             BD_ACC_BEGIN(ta);
             ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
@@ -889,8 +918,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t atom = kk >> 2, k16 = kk & 3;
-                        umma_ss(tmem_base, wdesc + (atom * w_atom16 + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
-                                idesc_base, (kk > 0) ? 1u : first);
+                        if constexpr (kPair)
+                            umma_ss_pair(tmem_base, wdesc + (atom * w_atom16 + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
+                                         idesc_base, (kk > 0) ? 1u : first);
+                        else
+                            umma_ss(tmem_base, wdesc + (atom * w_atom16 + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
+                                    idesc_base, (kk > 0) ? 1u : first);
                     }
                     // decode schedule: nothing else reads the W_base tile, hand it back as soon as these MMAs
                     // have completed
@@ -924,10 +957,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk) {
                                 const uint32_t atom = kk >> 2, k16 = kk & 3;
-                                umma_ts(d_tmem, a_tmem + kk * 8, xwdesc + (atom * x_atom16 + k16 * 2), idesc_delta,
-                                        (kk > 0) ? 1u : first);
+                                if constexpr (kPair)
+                                    umma_ts_pair(d_tmem, a_tmem + kk * 8, xwdesc + (atom * x_atom16 + k16 * 2), idesc_delta,
+                                                 (kk > 0) ? 1u : first);
+                                else
+                                    umma_ts(d_tmem, a_tmem + kk * 8, xwdesc + (atom * x_atom16 + k16 * 2), idesc_delta,
+                                            (kk > 0) ? 1u : first);
                             }
-                            tc_commit(smem_u32(&ctl->aempty[slot]));
+                            if constexpr (kPair) tc_commit_pair(smem_u32(&ctl->aempty[slot]), 3);
+                            else tc_commit(smem_u32(&ctl->aempty[slot]));
                         }
                         __syncwarp();
                         BD_ACC_END(w_id, tid);
@@ -935,14 +973,20 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
                 if (!ok) break;
                 if (!kDec) {
-                    if (elect_one()) tc_commit(smem_u32(&ctl->wempty[stage]));
+                    if (elect_one()) {
+                        if constexpr (kPair) tc_commit_pair(smem_u32(&ctl->wempty[stage]), 3);
+                        else tc_commit(smem_u32(&ctl->wempty[stage]));
+                    }
                     __syncwarp();
                 }
                 if (++stage == a.n_w) { stage = 0; phase ^= 1; }
                 if (++xslot == a.n_x) { xslot = 0; xphase ^= 1; }
             }
             if (!ok) break;
-            if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
+            if (elect_one()) {
+                if constexpr (kPair) tc_commit_pair(smem_u32(&ctl->accfull), 3);
+                else tc_commit(smem_u32(&ctl->accfull));
+            }
             __syncwarp();
             accphase ^= 1;
             BD_STAMP(6);
@@ -1217,7 +1261,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         tc_wait_st();
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&ctl->afull[slot]));
+                        if (lane == 0) {
+                            if (kPair && rank != 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctl->afull[slot]), 0));   // the leader's
+                            else mbar_arrive(smem_u32(&ctl->afull[slot]));
+                        }
                         BD_ACC_END(w_work, tw);
                         if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
@@ -1379,7 +1426,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
+            if (lane == 0) {
+                if (kPair && rank != 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctl->accempty), 0));   // the leader's
+                else mbar_arrive(smem_u32(&ctl->accempty));
+            }
             if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
             if (splitter) {
                 // the next tile's first stages, before the (slow) fix-up of this one
@@ -1398,7 +1448,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 epi_bar_sync(n_epi_warps * 32);
                 if (etid == 0) {
                     __threadfence();
-                    const unsigned old = atomicAdd(&a.counters[unit], 1u);
+                    const unsigned old = atomicAdd(&a.counters[kPair ? 2 * unit + (int)rank : unit], 1u);
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);
@@ -1407,11 +1457,14 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
                     // range starts exactly there.  Every later CTA starts inside the tile.
-                    const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
+                    // (pair schedule: c0, c1 count clusters; this CTA adds up the slots of the CTAs of its own rank)
+                    const int b0 = kPair ? 2 * c0 + (int)rank : c0;            // first contributing CTA
+                    const int bstep = kPair ? 2 : 1;                           // CTAs from one contributor to the next
+                    const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * b0 : 2 * b0 + 1;
                     const float* first = a.partials + (size_t)slot0 * a.slot_floats;
-                    const float* rest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats;
-                    reduce_partials<kGen>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
-                    if (etid == 0) a.counters[unit] = 0u;
+                    const float* rest = a.partials + (size_t)(2 * (b0 + bstep)) * a.slot_floats;
+                    reduce_partials<kGen>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)bstep * a.slot_floats, c1 - c0);
+                    if (etid == 0) a.counters[kPair ? 2 * unit + (int)rank : unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
                 if (warp == epi_first_warp) { BD_STAMP(10); BD_TL(4); }
@@ -1433,8 +1486,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         __syncthreads();
     }
     tc_fence_after();
+    if constexpr (kPair) cluster_sync_all();   // neither CTA's shared or tensor memory goes while the other may still signal it
     if (warp == kWarpTmem) {
-        tmem_dealloc(tmem_base, kTmemCols);
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+        else tmem_dealloc(tmem_base, kTmemCols);
         BD_STAMP(12);
     }
     BD_TRACE_FLUSH;
@@ -1453,18 +1508,19 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream) {
     // the general form only where something beyond the plain bf16 product is asked for
-    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 7 : 0;
-    // 0 tiled, 1..4 decode with that many tokens per tenant, 5 decode with 5..16, 6 tiled with several tenants per unit
-    const int mode = gen + (!args.decode ? (args.win_rows > 0 ? 6 : 0) : (args.m <= 4 ? args.m : 5));
+    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 8 : 0;
+    // 0 tiled, 1..4 decode with that many tokens per tenant, 5 decode with 5..16, 6 tiled with several tenants per unit,
+    // 7 tiled on CTA pairs
+    const int mode = gen + (!args.decode ? (args.pair ? 7 : (args.win_rows > 0 ? 6 : 0)) : (args.m <= 4 ? args.m : 5));
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmArgs);
-    static const KernelFn kernels[14] = {
+    static const KernelFn kernels[16] = {
         bitdelta_gemm_tc_kernel<0, false>, bitdelta_gemm_tc_kernel<1, false>, bitdelta_gemm_tc_kernel<2, false>,
         bitdelta_gemm_tc_kernel<3, false>, bitdelta_gemm_tc_kernel<4, false>, bitdelta_gemm_tc_kernel<5, false>,
-        bitdelta_gemm_tc_kernel<6, false>,
+        bitdelta_gemm_tc_kernel<6, false>, bitdelta_gemm_tc_kernel<7, false>,
         bitdelta_gemm_tc_kernel<0, true>,  bitdelta_gemm_tc_kernel<1, true>,  bitdelta_gemm_tc_kernel<2, true>,
         bitdelta_gemm_tc_kernel<3, true>,  bitdelta_gemm_tc_kernel<4, true>,  bitdelta_gemm_tc_kernel<5, true>,
-        bitdelta_gemm_tc_kernel<6, true>};
-    static int attr_device[14] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
+        bitdelta_gemm_tc_kernel<6, true>,  bitdelta_gemm_tc_kernel<7, true>};
+    static int attr_device[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1482,12 +1538,45 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
     cfg.dynamicSmemBytes = smem_bytes;
 #endif
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    if (early_start) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
+    }
+    if (args.pair) {   // clusters of two CTAs
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = early_start ? 1 : 0;
+    cfg.numAttrs = nattr;
     return cudaLaunchKernelEx(&cfg, kernels[mode], tmW, tmX, tmX8, tmBits, args);
+}
+
+int max_active_pairs(uint32_t smem_bytes) {
+    auto kernel = bitdelta_gemm_tc_kernel<7, false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * kMaxCtas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
 }
 
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {

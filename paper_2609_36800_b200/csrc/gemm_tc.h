@@ -12,6 +12,7 @@ namespace bd {
 struct GemmArgs {
     int B, m, N, K;
     int decode, convert, TB, tok_tile, Nb, Nd, win_rows, chunk_rows, aslot_cols;
+    int pair;            // tiled schedule on CTA pairs (see plan.h)
     int f16;             // 0: X, W_base, bias, Y are bf16; 1: IEEE binary16
     int act;             // fused epilogue: 0 none, 1 SiLU (after the bias)
     const void* bias;    // [N] values of the I/O type added to every output row, or nullptr
@@ -36,7 +37,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.decode = p.decode; a.convert = p.convert; a.TB = p.TB; a.tok_tile = p.tok_tile; a.Nb = p.Nb; a.Nd = p.Nd;
     a.win_rows = p.win_rows; a.chunk_rows = p.chunk_rows; a.aslot_cols = p.aslot_cols;
     a.m_tiles = p.m_tiles; a.groups = p.groups; a.P = p.P; a.T = (int)p.T; a.whole_units = p.whole_units;
-    a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = p.grid / p.teams; a.n_tiles = p.n_tiles;
+    a.pair = p.pair;
+    a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = (p.pair ? p.grid / 2 : p.grid) / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
@@ -91,6 +93,10 @@ inline uint8_t* ws_x8(const Plan& p, void* workspace) {
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream);
+
+// Number of CTA pairs (clusters of two) of the pair schedule's kernel that the current device can hold at once
+// with `smem_bytes` of dynamic shared memory each (0 if the query fails).
+int max_active_pairs(uint32_t smem_bytes);
 
 // Decode schedule pre-pass: X bf16 [rows, K] -> four e5m2 pieces per element (k permuted inside
 // each group of 32) in X8 [B, 4, m, K].

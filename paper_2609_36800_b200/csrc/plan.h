@@ -2,6 +2,7 @@
 // tensor memory budget, work decomposition and workspace layout.  Pure integer
 // arithmetic; shared by the launcher and the workspace-size query.
 #pragma once
+#include <cstdlib>
 #include <cstddef>
 #include <cstdint>
 
@@ -48,6 +49,9 @@ struct Plan {
     int n_x;           // ring of bf16 activation tiles
     int n_x8;          // decode: ring of e5m2 piece tiles
     int n_bits;        // sign-word slots (each holds the signs of one k-pair of one unit)
+    int pair;          // tiled schedule on CTA pairs: a unit is two W_base tiles (256 rows), one per CTA of a cluster of
+                       // two; each CTA stages its own weights and half of the activation tile, the pair's leader issues
+                       // 256-row MMAs (tcgen05 cta_group::2)
     int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
@@ -62,7 +66,15 @@ struct Plan {
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0) {
+// The pair schedule is taken where it applies unless BITDELTA_PAIR=0 is set (experiments).
+inline bool pair_enabled() {
+    const char* e = getenv("BITDELTA_PAIR");
+    return !(e && e[0] == '0');
+}
+
+// allow_pair = false: the device cannot hold all the pairs at once (see the launcher), plan without them.
+inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0,
+                      bool allow_pair = true) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
@@ -116,19 +128,21 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.Nd = p.tok_tile;
         p.win_rows = 0;
         p.chunk_rows = 16;
-        p.x_rows = p.tok_tile;
+        p.pair = (allow_pair && pair_enabled() && p.tok_tile == 128 && (p.n_tiles % 2) == 0 && num_sms >= 2) ? 1 : 0;
+        p.x_rows = p.pair ? p.tok_tile / 2 : p.tok_tile;   // a pair's CTAs stage half of the token tile each
         p.N3 = 0;
         p.convert = 0;
         p.x8_rows = 0;
         p.aslot_cols = 64;
         p.slot_floats = (size_t)kTileN * p.tok_tile;
     }
-    p.units = p.n_tiles * p.groups;
+    p.units = (p.pair ? p.n_tiles / 2 : p.n_tiles) * p.groups;
     p.P = (K + kPairK - 1) / kPairK;
     p.T = (long long)p.units * p.P;
     if (p.T >= (1ll << 30)) return p;   // the kernel's work-split arithmetic is 32-bit
     int max_grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
     p.grid = p.T < max_grid ? (int)p.T : max_grid;
+    if (p.pair) p.grid = 2 * (int)(p.T < max_grid / 2 ? p.T : max_grid / 2);   // clusters of two
     // Several tenant groups share each W_base tile; cut anywhere, the groups of a tile sit at different k at any
     // moment and W_base is fetched from HBM once per group.  Two work orders keep them in step instead, so
     // that all but the first read of a W_base tile hit L2:
@@ -234,10 +248,11 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
 
     // Workspace: arrival counters, two partial-result slots per CTA, then (decode) the e5m2
     // pieces of X written by the activation-split kernel.
-    p.ws_header_bytes = (size_t)round_up(p.units * 4, 1024);
+    p.ws_header_bytes = (size_t)round_up(p.n_tiles * p.groups * 4, 1024);   // one arrival counter per W_base tile and group
     // (sized for the largest grid any device could get, so that the size does not depend on the device;
     // never more CTAs than items)
-    const long long max_ctas = p.T < kMaxCtas ? p.T : kMaxCtas;
+    const long long items = p.pair ? 2 * p.T : p.T;
+    const long long max_ctas = items < kMaxCtas ? items : kMaxCtas;
     p.ws_partials_bytes = (size_t)2 * (size_t)max_ctas * p.slot_floats * sizeof(float);
     p.ws_x8_bytes = p.decode ? (((size_t)B * kPieces * m * K + 1023) / 1024 * 1024) : 0;
     p.ws_bytes = p.ws_header_bytes + p.ws_partials_bytes + p.ws_x8_bytes;

@@ -23,7 +23,13 @@ def test_every_item_is_taken_exactly_once(shape, sms):
     blocks, units, P, order, teams = info["blocks"], info["units"], info["k_steps"], info["order"], info["teams"]
     T = units * P
     assert 1 <= blocks <= sms
-    assert P == K // 128 and units == info["w_tiles"] * info["groups"]
+    pair = info["schedule"] == 4     # a unit is two W_base tiles, two thread blocks share every share of the list
+    assert P == K // 128 and units == info["w_tiles"] * info["groups"] // (2 if pair else 1)
+    if pair:
+        assert blocks % 2 == 0 and info["w_tiles"] % 2 == 0 and order == 0
+        for b in range(0, blocks, 2):
+            assert bd.gemm_plan_cta_items(B, m, N, K, b, num_sms=sms) == bd.gemm_plan_cta_items(B, m, N, K, b + 1, num_sms=sms)
+    step = 2 if pair else 1
     if order == 1:
         # whole units round-robin: block b starts at unit b; all units are reached when blocks <= units
         assert blocks <= units
@@ -32,7 +38,7 @@ def test_every_item_is_taken_exactly_once(shape, sms):
         for item in (0, T - 1, T // 2):
             assert bd.gemm_plan_item_cta(B, m, N, K, item, num_sms=sms) == (item // P) % blocks
         return
-    ranges = [bd.gemm_plan_cta_items(B, m, N, K, b, num_sms=sms) for b in range(blocks)]
+    ranges = [bd.gemm_plan_cta_items(B, m, N, K, b, num_sms=sms) for b in range(0, blocks, step)]
     # contiguous, in order, covering [0, T)
     assert ranges[0][0] == 0 and ranges[-1][1] == T
     for (lo, hi), (lo2, _) in zip(ranges, ranges[1:]):
@@ -61,7 +67,7 @@ def test_every_item_is_taken_exactly_once(shape, sms):
     items = range(T) if T <= 4096 else sorted(set(rng.integers(0, T, 2048).tolist()) | {0, T - 1} | {lo for lo, _ in ranges} | {hi - 1 for _, hi in ranges})
     starts = np.array([lo for lo, _ in ranges])
     for item in items:
-        assert bd.gemm_plan_item_cta(B, m, N, K, item, num_sms=sms) == int(np.searchsorted(starts, item, side="right") - 1)
+        assert bd.gemm_plan_item_cta(B, m, N, K, item, num_sms=sms) == step * int(np.searchsorted(starts, item, side="right") - 1)
 
 
 def test_schedules_and_work_orders_of_the_measured_workloads():
@@ -70,7 +76,7 @@ def test_schedules_and_work_orders_of_the_measured_workloads():
     assert got["tiny"]["schedule"] == 2
     assert got["decode_mlp_up"]["schedule"] == 1 and got["decode_mlp_up"]["order"] == 2 and got["decode_mlp_up"]["teams"] == 2
     assert got["many_tenant_down"]["order"] == 2 and got["many_tenant_down"]["teams"] == 8 and got["many_tenant_down"]["blocks"] == 144
-    assert got["prefill"]["schedule"] == 0 and got["prefill"]["order"] == 0
+    assert got["prefill"]["schedule"] == 4 and got["prefill"]["order"] == 0 and got["prefill"]["blocks"] == 148
     for g in got.values():
         assert g["smem_bytes"] <= 227 * 1024 and g["w_ring"] >= 2 and g["operand_buffers"] >= 2
 
