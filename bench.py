@@ -36,7 +36,7 @@ PAPER_CONTEXT = "paper: 3.34x (standard) / 2.51x (batched) over autotuned Triton
 NCU_TRAFFIC_BYTES = {
     "decode_attn": 50_510_000,          # 50.49 MB read + 0.02 MB written
     "decode_mlp_up": 219_000_000,       # 213.7 MB read + 5.3 MB written (a third of W_base read twice)
-    "prefill": 74_000_000,              # 62.1 MB read + 12.0 MB written
+    "prefill": 96_000_000,              # 75 MB read + 21 MB written (pair schedule; 62 + 12 MB with one CTA per tile)
     "many_tenant_down": 416_000_000,    # 408.3 MB read + 7.6 MB written
     "tiny": None,
 }
