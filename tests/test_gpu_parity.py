@@ -101,6 +101,7 @@ SMALL = [
     (4, 64, 256, 512),    # two tenants of 64 tokens fill the 128 base columns
     (9, 24, 1280, 1024),  # three groups of tenants: teams of CTAs
     (6, 48, 200, 256),
+    (3, 256, 512, 640),   # CTA pairs: four W_base tiles, two token tiles per tenant, tiles cut across clusters
 ]
 
 
