@@ -345,14 +345,18 @@ __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u
 
 // Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
 // Two warps share each lane quadrant: warp half h drains the 32-token blocks h, h+2, ...
-template <class Out>
+// `release` hands the accumulators back (this warp's arrival): it is called as soon as the warp's last
+// tensor-memory load has completed, before the values of that load are finished and stored.
+template <class Out, class Release>
 __device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                               const Out& out, int half, float al) {
+                                               const Out& out, int half, float al, const Release& release) {
+    if (32 * half >= u.ntok) release();
     for (int t0 = 32 * half; t0 < u.ntok; t0 += 64) {
         uint32_t rb[32], rd[32];
         tmem_ld32(lane_taddr + (uint32_t)t0, rb);
         tmem_ld32(lane_taddr + a.col_delta + (uint32_t)t0, rd);
         tc_wait_ld();
+        if (t0 + 64 >= u.ntok) release();
         const int nvalid = min(32, u.ntok - t0);
 #pragma unroll
         for (int t = 0; t < 32; ++t) {
@@ -1403,6 +1407,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             const EpiOut<kGen> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
+            // this warp's arrival on the "accumulators drained" barrier (pair schedule: the leader's)
+            auto release_acc = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (kPair && rank != 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctl->accempty), 0));
+                    else mbar_arrive(smem_u32(&ctl->accempty));
+                }
+            };
             if constexpr (kMode >= 1 && kMode <= 4) {
                 epilogue_decode<kMode>(a, u, lane_taddr, out, alv, al_lane);
             } else if constexpr (kMode == 5) {
@@ -1422,14 +1435,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 }
             } else {
                 if constexpr (kGrouped) epilogue_tiled_grouped(a, u, lane_taddr, am, out, ehalf, al_lane);
-                else epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0]);
+                else epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0], release_acc);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (kPair && rank != 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctl->accempty), 0));   // the leader's
-                else mbar_arrive(smem_u32(&ctl->accempty));
-            }
+            if constexpr (kDec || kGrouped) release_acc();
             if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
             if (splitter) {
                 // the next tile's first stages, before the (slow) fix-up of this one
