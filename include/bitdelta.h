@@ -99,7 +99,9 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  *          prepared once by bitdelta_workspace_init; calls that may overlap on
  *          the device must not share a workspace.
  * m <= 16 selects the streaming (decode) schedule, larger m the tiled (prefill)
- * schedule; both run on tcgen05 tensor cores with TMEM accumulators.  Shapes
+ * schedule (several tenants per tile up to m = 64; pairs of thread blocks with
+ * 256-row MMAs for token tiles of 128); all run on tcgen05 tensor cores with TMEM
+ * accumulators, and bitdelta_gemm_plan tells which one a shape gets.  Shapes
  * whose K is not a multiple of 128 run on a plain CUDA-core kernel instead.
  * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.
  * Asynchronous on the stream; a kernel-side wait that expires is reported by
@@ -127,7 +129,9 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
  *         bias and Y.  Accumulation is fp32 in both; Y is rounded to nearest even once, after the
  *         epilogue.  With binary16 the delta term is exact for operands in the normal range (values
  *         below 2^-14 lose bits below 2^-16, in the delta term only).
- * bias  : device, [N] values of `dtype`, shared by all tenants, or NULL for none.  2-byte aligned.
+ * bias  : device, [N] values of `dtype`, shared by all tenants, or NULL for none.  2-byte aligned.  Like
+ *         alpha it is read during the early start (see bitdelta_gemm): it must not be produced by the kernel
+ *         queued directly before the call.
  * act   : BITDELTA_ACT_NONE, or BITDELTA_ACT_SILU: y * sigmoid(y), applied after the bias (fp32,
  *         hardware exponential: relative error of a few 1e-7, far below the output rounding).
  * Everything else (shapes, layouts, workspace, stream semantics, errors, tolerance) is as for
