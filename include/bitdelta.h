@@ -100,7 +100,7 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  *          the device must not share a workspace.
  * m <= 16 selects the streaming (decode) schedule, larger m the tiled (prefill)
  * schedule (several tenants per tile up to m = 64; pairs of thread blocks with
- * 256-row MMAs for token tiles of 128); all run on tcgen05 tensor cores with TMEM
+ * 256-row MMAs for m > 64); all run on tcgen05 tensor cores with TMEM
  * accumulators, and bitdelta_gemm_plan tells which one a shape gets.  Shapes
  * whose K is not a multiple of 128 run on a plain CUDA-core kernel instead.
  * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.

@@ -128,7 +128,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.Nd = p.tok_tile;
         p.win_rows = 0;
         p.chunk_rows = 16;
-        p.pair = (allow_pair && pair_enabled() && p.tok_tile == 128 && (p.n_tiles % 2) == 0 && num_sms >= 2) ? 1 : 0;
+        p.pair = (allow_pair && pair_enabled() && p.tok_tile >= 80 && (p.n_tiles % 2) == 0 && num_sms >= 2) ? 1 : 0;
         p.x_rows = p.pair ? p.tok_tile / 2 : p.tok_tile;   // a pair's CTAs stage half of the token tile each
         p.N3 = 0;
         p.convert = 0;

@@ -41,6 +41,7 @@ SHAPES = [
     (2, 17, 256, 384),
     (2, 100, 300, 640),
     (2, 130, 256, 512),     # token tiles of 128 and two W_base tiles: the schedule on CTA pairs
+    (2, 90, 256, 384),      # CTA pairs, token tile of 96
     (5, 20, 384, 512),
     (3, 33, 264, 384),
     (1, 200, 520, 384),

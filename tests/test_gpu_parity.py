@@ -102,6 +102,9 @@ SMALL = [
     (9, 24, 1280, 1024),  # three groups of tenants: teams of CTAs
     (6, 48, 200, 256),
     (3, 256, 512, 640),   # CTA pairs: four W_base tiles, two token tiles per tenant, tiles cut across clusters
+    (2, 100, 256, 640),   # CTA pairs with a token tile of 112 (56 rows of it per CTA)
+    (3, 72, 512, 384),    # ... of 80
+    (2, 127, 256, 256),
 ]
 
 
