@@ -91,3 +91,14 @@ def test_cuda_core_path_and_bad_arguments():
     assert lib.bitdelta_gemm_plan_item_cta(1, 1, 128, 128, 148, 5) == -1          # only one item
     a, b = ctypes.c_int(), ctypes.c_int()
     assert lib.bitdelta_gemm_plan_cta_items(1, 1, 128, 128, 148, 3, ctypes.byref(a), ctypes.byref(b)) == 2   # one block only
+
+
+def test_work_lists_beyond_the_32_bit_split_arithmetic_are_refused():
+    # 8192 W_base tiles x 512 tenant groups x 256 k-steps = 2^30 items: one too many for the kernel's 32-bit split
+    B, m, N, K = 4096, 1, 1 << 20, 1 << 15
+    assert bd.gemm_workspace_bytes(B, m, N, K) == 0
+    import ctypes
+    info = (ctypes.c_int * 16)()
+    assert bd.load_library().bitdelta_gemm_plan(B, m, N, K, 148, info) == 2
+    # just below the limit the plan exists
+    assert bd.gemm_plan(B, m, N // 2, K)["units"] * bd.gemm_plan(B, m, N // 2, K)["k_steps"] == 1 << 29
