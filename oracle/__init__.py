@@ -136,7 +136,7 @@ def gemm_at(X, W, bits, alpha, idx) -> np.ndarray:
 
 
 DTYPES = {"bf16": 0, "f16": 1}
-ACTS = {"none": 0, "silu": 1}
+ACTS = {"none": 0, "silu": 1, "silu_gate": 2}
 
 
 def half_to_double(h: np.ndarray) -> np.ndarray:
@@ -149,8 +149,9 @@ def half_to_double(h: np.ndarray) -> np.ndarray:
 
 def gemm_ex(X, W, bits, alpha, bias=None, dtype="bf16", act="none", idx=None) -> np.ndarray:
     """Y = act(sum_k x w + alpha[b] sum_k x s + bias[n]) in fp64.  X, W, bias are 16-bit patterns of
-    `dtype` ("bf16" or "f16"); act is "none" or "silu".  With idx (int32 [count,3] of (b,t,n)) only the
-    listed outputs are computed and returned as a vector."""
+    `dtype` ("bf16" or "f16"); act is "none", "silu", or "silu_gate" (rows 2i / 2i+1 of W are the gate / up
+    projections of feature i: Y[b,t,i] = silu(z[2i]) * z[2i+1], N/2 features per token).  With idx (int32
+    [count,3] of (b,t,output feature)) only the listed outputs are computed and returned as a vector."""
     X, W, bits, alpha, B, m, N, K = _check(X, W, bits, alpha)
     bp = None
     if bias is not None:
@@ -165,7 +166,9 @@ def gemm_ex(X, W, bits, alpha, bias=None, dtype="bf16", act="none", idx=None) ->
         out = np.empty((idx.shape[0],), dtype=np.float64)
         ip, cnt = _ptr(idx), idx.shape[0]
     else:
-        out = np.empty((B, m, N), dtype=np.float64)
+        if act == "silu_gate" and N % 2:
+            raise ValueError("silu_gate needs an even N")
+        out = np.empty((B, m, N // 2 if act == "silu_gate" else N), dtype=np.float64)
         ip, cnt = None, 0
     _load().oracle_gemm_ex(_ptr(X), _ptr(W), _ptr(bits), _ptr(alpha), bp, ip, cnt, _ptr(out),
                            B, m, N, K, DTYPES[dtype], ACTS[act])

@@ -201,6 +201,10 @@ void oracle_compress(const uint16_t *wf, const uint16_t *wb, uint32_t *bits, flo
  *
  * dtype 0: x, w, bias are bf16 bit patterns; dtype 1: IEEE-754 binary16 bit patterns.
  * bias may be NULL (no bias).  act 0: identity; act 1: SiLU, y * sigmoid(y) = y / (1 + exp(-y)).
+ * act 2: SiLU gate of a gated MLP whose gate and up projections are interleaved along N: with
+ *   z[b,t,n] = sum_k x w + alpha[b] sum_k x s + bias[n]   (N even),
+ *   Y[b,t,i] = SiLU(z[b,t,2i]) * z[b,t,2i+1],   i < N/2     (row 2i: gate, row 2i+1: up),
+ * so the result has N/2 features per token.
  * Everything is widened exactly to double; sums in double in plain k order; result kept in double.
  */
 #include <math.h>
@@ -228,11 +232,33 @@ static double widen16(uint16_t v, int dtype)
     return dtype == 1 ? half_to_double(v) : bf16_to_double(v);
 }
 
+static double silu(double y)
+{
+    return y / (1.0 + exp(-y));
+}
+
 static double finish(double y, double bias, int act)
 {
     y += bias;
-    if (act == 1) y = y / (1.0 + exp(-y));
+    if (act == 1) y = silu(y);
     return y;
+}
+
+/* z[b,t,n] before any activation */
+static double preact(const uint16_t *X, const uint16_t *W, const uint32_t *bits, const float *alpha,
+                     const uint16_t *bias, int b, int t, int n, int m, int N, int K, int dtype)
+{
+    int words = K / 32;
+    const uint16_t *xrow = X + ((size_t)b * m + t) * K;
+    const uint16_t *wrow = W + (size_t)n * K;
+    const uint32_t *row_words = bits + ((size_t)b * N + n) * words;
+    double base = 0.0, delta = 0.0;
+    for (int k = 0; k < K; ++k) {
+        double x = widen16(xrow[k], dtype);
+        base += x * widen16(wrow[k], dtype);
+        delta += x * sign_at(row_words, k);
+    }
+    return base + (double)alpha[b] * delta + (bias ? widen16(bias[n], dtype) : 0.0);
 }
 
 /* The extended definition at `count` listed outputs (idx holds count triples b,t,n), or, with idx == NULL,
@@ -242,14 +268,21 @@ void oracle_gemm_ex(const uint16_t *X, const uint16_t *W, const uint32_t *bits, 
                     int B, int m, int N, int K, int dtype, int act)
 {
     int words = K / 32;
-    long long total = idx ? (long long)count : (long long)B * m * N;
+    int No = (act == 2) ? N / 2 : N;   /* output features per token */
+    long long total = idx ? (long long)count : (long long)B * m * No;
 #pragma omp parallel for schedule(static)
     for (long long i = 0; i < total; ++i) {
         int b, t, n;
         if (idx) {
             b = idx[3 * i + 0]; t = idx[3 * i + 1]; n = idx[3 * i + 2];
         } else {
-            n = (int)(i % N); t = (int)((i / N) % m); b = (int)(i / ((long long)N * m));
+            n = (int)(i % No); t = (int)((i / No) % m); b = (int)(i / ((long long)No * m));
+        }
+        if (act == 2) {
+            double gate = preact(X, W, bits, alpha, bias, b, t, 2 * n, m, N, K, dtype);
+            double up = preact(X, W, bits, alpha, bias, b, t, 2 * n + 1, m, N, K, dtype);
+            out[i] = silu(gate) * up;
+            continue;
         }
         const uint16_t *xrow = X + ((size_t)b * m + t) * K;
         const uint16_t *wrow = W + (size_t)n * K;

@@ -459,3 +459,40 @@ def test_ex_at_listed_outputs_equals_full_result():
     idx = np.array([[0, 0, 0], [2, 3, 9], [1, 2, 5], [2, 0, 7]], dtype=np.int32)
     at = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu", idx=idx)
     assert np.array_equal(at, np.array([full[b, t, n] for b, t, n in idx]))
+
+
+# ----------------------------------------------------------------------------
+# SiLU gate over interleaved gate / up rows
+# ----------------------------------------------------------------------------
+def _gate_probe(gate, up, bias=None):
+    """Two weight rows with pre-activation values `gate` (row 0) and `up` (row 1): x = e_0, alpha = 0."""
+    X = np.zeros((1, 1, 32), dtype=np.float32); X[0, 0, 0] = 1.0
+    W = np.zeros((2, 32), dtype=np.float32); W[0, 0] = gate; W[1, 0] = up
+    bits = np.zeros((1, 2, 1), dtype=np.uint32)
+    alpha = np.zeros(1, dtype=np.float32)
+    b = None if bias is None else f16(bias)
+    y = oracle.gemm_ex(f16(X), f16(W), bits, alpha, bias=b, dtype="f16", act="silu_gate")
+    assert y.shape == (1, 1, 1)
+    return float(y[0, 0, 0])
+
+
+def test_silu_gate_closed_forms_and_row_roles():
+    assert _gate_probe(1.0, 3.0) == pytest.approx(3.0 * 0.7310585786300049, rel=1e-15)   # sigmoid(1) * 1 * 3
+    assert _gate_probe(3.0, 1.0) == pytest.approx(3.0 / (1.0 + np.exp(-3.0)), rel=1e-15)  # roles are not symmetric
+    assert _gate_probe(0.0, 5.0) == 0.0 and _gate_probe(5.0, 0.0) == 0.0
+    assert _gate_probe(40.0, -2.0) == pytest.approx(-80.0, rel=1e-15)                       # silu(y) -> y for large y
+    # the bias enters both rows before the gate: (-1 + 2, 3 + 0.5)
+    assert _gate_probe(-1.0, 3.0, bias=[2.0, 0.5]) == pytest.approx(3.5 * 0.7310585786300049, rel=1e-15)
+
+
+def test_silu_gate_equals_recombined_plain_outputs():
+    wl = synth.Workload("t", B=2, m=3, K=96, N=12, seed=13)
+    X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    z = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16")               # pinned above
+    expect = (z[:, :, 0::2] / (1.0 + np.exp(-z[:, :, 0::2]))) * z[:, :, 1::2]
+    got = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu_gate")
+    assert got.shape == (2, 3, 6)
+    assert np.max(np.abs(got - expect)) <= 1e-13
+    idx = np.array([[0, 0, 0], [1, 2, 5], [1, 1, 3]], dtype=np.int32)
+    at = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu_gate", idx=idx)
+    assert np.array_equal(at, np.array([got[b, t, i] for b, t, i in idx]))
