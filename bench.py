@@ -234,7 +234,7 @@ def time_compress(peaks, B=8, N=4096, K=4096, steps=20):
             "steps": steps, "kernels_per_call": 2}
 
 
-def time_gemm_ex(wl, peaks, steps=40):
+def time_gemm_ex(wl, peaks, steps=40, act="silu"):
     """The extended call (fp16 operands, bias, SiLU fused into the epilogue) on `wl`, timed like the
     headline: rotating buffer sets larger than L2, all steps in one CUDA graph, CUDA events."""
     import torch
@@ -244,10 +244,11 @@ def time_gemm_ex(wl, peaks, steps=40):
     nsets = max(2, -(-2 * L2_BYTES // wl.bytes))
     f16 = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.float16)
     sets = [(f16(X), f16(W), torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(alpha).cuda(), f16(bias),
-             torch.empty((wl.B, wl.m, wl.N), dtype=torch.float16, device="cuda")) for _ in range(nsets)]
+             torch.empty((wl.B, wl.m, wl.N // 2 if act == "silu_gate" else wl.N), dtype=torch.float16, device="cuda"))
+            for _ in range(nsets)]
     ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
     stream = torch.cuda.Stream()
-    call = lambda s: bd.gemm(s[0], s[1], s[2], s[3], out=s[5], workspace=ws, bias=s[4], act="silu")
+    call = lambda s: bd.gemm(s[0], s[1], s[2], s[3], out=s[5], workspace=ws, bias=s[4], act=act)
     with torch.cuda.stream(stream):
         for i in range(3):
             call(sets[i % nsets])
@@ -271,7 +272,7 @@ def time_gemm_ex(wl, peaks, steps=40):
     roof["traffic"] = None                       # not captured separately: same loads as the bf16 call plus N bias values
     roof["algorithmic_bytes"] = wl.bytes + 2 * wl.N
     return {"us_per_launch": ms * 1e3 / steps, "steps": steps, "buffer_sets": nsets, "dtype": "f16",
-            "epilogue": "bias+silu", "roofline": roof}
+            "epilogue": "bias+" + act, "roofline": roof}
 
 
 def time_e2e(wl, host_inputs, steps):
@@ -463,6 +464,10 @@ def run_ours(args):
                 steps3 = max(20, min(args.steps, int(0.25 / max(w3.bytes / 6.5e12, w3.flops / 1.6e15))))
                 out["gemm_ex"][name] = time_gemm_ex(w3, peaks, steps3)
                 torch.cuda.empty_cache()
+            # the gated-MLP form on the MLP up projection (gate and up rows interleaved along N)
+            w4 = synth.WORKLOADS_BY_NAME["decode_mlp_up"]
+            out["gemm_ex"]["decode_mlp_up_silu_gate"] = time_gemm_ex(w4, peaks, max(20, min(args.steps, 4000)), act="silu_gate")
+            torch.cuda.empty_cache()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

@@ -133,13 +133,18 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
  *         alpha it is read during the early start (see bitdelta_gemm): it must not be produced by the kernel
  *         queued directly before the call.
  * act   : BITDELTA_ACT_NONE, or BITDELTA_ACT_SILU: y * sigmoid(y), applied after the bias (fp32,
- *         hardware exponential: relative error of a few 1e-7, far below the output rounding).
+ *         hardware exponential: relative error of a few 1e-7, far below the output rounding), or
+ *         BITDELTA_ACT_SILU_GATE: the gate of a gated MLP whose gate and up projections are interleaved
+ *         along N (row 2i of W_base, of every tenant's sign matrix and of bias: gate projection of
+ *         feature i; row 2i+1: its up projection).  With z the sum above before any activation,
+ *           Y[b,t,i] = SiLU(z[b,t,2i]) * z[b,t,2i+1],   i < N/2,
+ *         so Y is [B,m,N/2] (N must be even: BITDELTA_ERR_SHAPE otherwise).
  * Everything else (shapes, layouts, workspace, stream semantics, errors, tolerance) is as for
  * bitdelta_gemm, which is this call with BITDELTA_DTYPE_BF16, no bias and no activation.  Unknown
  * codes return BITDELTA_ERR_OPTION and launch nothing.
  */
 enum { BITDELTA_DTYPE_BF16 = 0, BITDELTA_DTYPE_F16 = 1 };
-enum { BITDELTA_ACT_NONE = 0, BITDELTA_ACT_SILU = 1 };
+enum { BITDELTA_ACT_NONE = 0, BITDELTA_ACT_SILU = 1, BITDELTA_ACT_SILU_GATE = 2 };
 int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
                      const void* bias, void* Y, int B, int m, int N, int K, int dtype, int act,
                      void* workspace, size_t workspace_bytes, void* cuda_stream);

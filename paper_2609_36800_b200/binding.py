@@ -150,14 +150,15 @@ def make_workspace(B: int, m: int, N: int, K: int, device="cuda", stream=None):
     return ws
 
 
-ACTS = {"none": 0, "silu": 1}
+ACTS = {"none": 0, "silu": 1, "silu_gate": 2}
 
 
 def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bool = False, bias=None,
          act: str = "none"):
     """Y[b,t,n] = act(sum_k X W_base + alpha[b] sum_k X S + bias[n]).  X [B,m,K] and W_base [N,K] in bf16 or
-    (both) fp16, bits int32 storage [B,N,K/32], alpha fp32 [B], optional bias [N] of X's type, act "none" or
-    "silu"; returns Y [B,m,N] of X's type.  (simt=True runs the diagnostic CUDA-core kernel: bf16, no epilogue.)"""
+    (both) fp16, bits int32 storage [B,N,K/32], alpha fp32 [B], optional bias [N] of X's type, act "none", "silu"
+    or "silu_gate" (rows 2i / 2i+1 are gate / up projections: Y[b,t,i] = silu(z[2i]) * z[2i+1], Y is [B,m,N/2]);
+    returns Y [B,m,N] of X's type.  (simt=True runs the diagnostic CUDA-core kernel: bf16, no epilogue.)"""
     import torch
     lib = load_library()
     B, m, K = X.shape
@@ -171,8 +172,10 @@ def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bo
         raise ValueError(f"unknown activation {act!r}")
     if bias is not None and tuple(bias.shape) != (N,):
         raise ValueError("bias must have N entries")
+    if act == "silu_gate" and N % 2:
+        raise ValueError("silu_gate needs an even N (interleaved gate / up rows)")
     if out is None:
-        out = torch.empty((B, m, N), dtype=io, device=X.device)
+        out = torch.empty((B, m, N // 2 if act == "silu_gate" else N), dtype=io, device=X.device)
     args = [_dev(X, io, "X"), _dev(W_base, io, "W_base"), _dev(bits, torch.int32, "bits"),
             _dev(alpha, torch.float32, "alpha")]
     shape = [B, m, N, K]

@@ -266,8 +266,9 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
                      size_t workspace_bytes, void* cuda_stream) {
     int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
     if (st != BITDELTA_OK) return st;
-    if ((dtype != BITDELTA_DTYPE_BF16 && dtype != BITDELTA_DTYPE_F16) || (act != BITDELTA_ACT_NONE && act != BITDELTA_ACT_SILU))
+    if ((dtype != BITDELTA_DTYPE_BF16 && dtype != BITDELTA_DTYPE_F16) || (act != BITDELTA_ACT_NONE && act != BITDELTA_ACT_SILU && act != BITDELTA_ACT_SILU_GATE))
         return BITDELTA_ERR_OPTION;
+    if (act == BITDELTA_ACT_SILU_GATE && (N % 2) != 0) return BITDELTA_ERR_SHAPE;
     if (bias && (reinterpret_cast<uintptr_t>(bias) & 1)) return BITDELTA_ERR_ALIGN;
     const int f16 = (dtype == BITDELTA_DTYPE_F16) ? 1 : 0;
     DeviceInfo d;

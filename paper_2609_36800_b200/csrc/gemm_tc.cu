@@ -21,6 +21,8 @@
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
+#include <type_traits>
+
 #include "gemm_tc.h"
 #include "ptx.cuh"
 
@@ -276,16 +278,28 @@ __device__ __forceinline__ float from_io16(uint16_t h, int f16) {
 // kGen = false: bf16 output, no bias, no activation (the plain product).  The two forms are separate code
 // on purpose: the epilogue runs once per tile, every instruction of it is fetched cold, and the plain
 // product should not pay for the general form's length.
-template <bool kGen>
+template <bool kGen, bool kGate = false>
 struct EpiOut {
     uint16_t* Y;        // output matrix [B*m, N], 16-bit values of the I/O type
     float* slot;        // partial-result slot, or nullptr when this CTA owns the whole tile
     int N, n, row, xrow0;
     float bias;         // of output feature n (0 without a bias)
     const GemmArgs& a;  // kernel parameters (activation code, I/O type)
+    // (called by all lanes of a warp together: the gated form exchanges values between neighbouring lanes)
     __device__ __forceinline__ void put(int tok, float v) const {
-        if (slot) slot[(size_t)tok * kTileN + row] = v;   // partial sums: finished by the CTA that adds them up
-        else if (n < N) {
+        if (slot) {
+            slot[(size_t)tok * kTileN + row] = v;   // partial sums: finished by the CTA that adds them up
+            return;
+        }
+        if constexpr (kGate) {
+            // SiLU gate: weight rows come in pairs (2i: gate, 2i+1: up), i.e. in neighbouring lanes
+            const float z = v + bias;
+            const float other = __shfl_xor_sync(0xFFFFFFFFu, z, 1);
+            if (!(n & 1) && n < N)
+                Y[(size_t)(xrow0 + tok) * (N >> 1) + (n >> 1)] = to_io16(__fdividef(z, 1.f + __expf(-z)) * other, a.f16);
+            return;
+        }
+        if (n < N) {
             if constexpr (kGen) Y[(size_t)(xrow0 + tok) * N + n] = finish_io16(v, bias, a.act, a.f16);
             else Y[(size_t)(xrow0 + tok) * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
         }
@@ -299,9 +313,9 @@ struct EpiOut {
 // with more than four tokens per tenant: a real loop, because its body is long, this code runs once per tile
 // and every instruction of it is fetched cold, so its length is paid in time.
 // `alv[j]`: tenant j's scale (unrolled form); `al_lane`: lane l holds tenant l's scale (loop form).
-template <int M, bool kGen>
+template <int M, bool kGen, class Out>
 __device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                                const EpiOut<kGen>& out, const float* alv, float al_lane) {
+                                                const Out& out, const float* alv, float al_lane) {
     constexpr int N3 = (kPieces * M + 15) / 16 * 16;
     constexpr int TPB = (N3 == 16) ? 2 : 1;   // tenants drained per wait
     constexpr int kMaxTen = (M <= 4) ? 8 : 4;   // tenants per unit (see the plan)
@@ -392,7 +406,7 @@ __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterp
 
 // Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
 // nwarps*32 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+nwarps, ...
-template <bool kGen>
+template <bool kGen, bool kGate>
 __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, int nwarps,
                                                 const float* first, const float* rest, size_t cstride, int nrest) {
     uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
@@ -427,6 +441,17 @@ __device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u
         for (int q = 0; q < 4; ++q) {
             const int t = tk + nwarps * q;
             if (t < u.ntok) {
+                if constexpr (kGate) {
+                    {
+                        // SiLU gate: rows (n, n+1) and (n+2, n+3) are (gate, up) pairs; N is even and n a multiple of 4
+                        const float g0 = acc[q].x + bias4[0], u0 = acc[q].y + bias4[1];
+                        const float g1 = acc[q].z + bias4[2], u1 = acc[q].w + bias4[3];
+                        uint16_t* dg = Y + (size_t)(u.xrow0 + t) * (a.N >> 1) + (n >> 1);
+                        if (n < a.N) dg[0] = to_io16(__fdividef(g0, 1.f + __expf(-g0)) * u0, a.f16);
+                        if (n + 2 < a.N) dg[1] = to_io16(__fdividef(g1, 1.f + __expf(-g1)) * u1, a.f16);
+                        continue;
+                    }
+                }
                 uint16_t* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
                 uint16_t o0, o1, o2, o3;
                 if constexpr (kGen) {
@@ -1406,7 +1431,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             accphase ^= 1;
             if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
-            const EpiOut<kGen> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
             // this warp's arrival on the "accumulators drained" barrier (pair schedule: the leader's)
             auto release_acc = [&]() {
                 tc_fence_before();
@@ -1416,26 +1440,37 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     else mbar_arrive(smem_u32(&ctl->accempty));
                 }
             };
-            if constexpr (kMode >= 1 && kMode <= 4) {
-                epilogue_decode<kMode>(a, u, lane_taddr, out, alv, al_lane);
-            } else if constexpr (kMode == 5) {
-                switch (am) {
-                    case 5: epilogue_decode<5>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 6: epilogue_decode<6>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 7: epilogue_decode<7>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 8: epilogue_decode<8>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 9: epilogue_decode<9>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 10: epilogue_decode<10>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 11: epilogue_decode<11>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 12: epilogue_decode<12>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 13: epilogue_decode<13>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 14: epilogue_decode<14>(a, u, lane_taddr, out, alv, al_lane); break;
-                    case 15: epilogue_decode<15>(a, u, lane_taddr, out, alv, al_lane); break;
-                    default: epilogue_decode<16>(a, u, lane_taddr, out, alv, al_lane); break;
+            // (the gated form of the general epilogue is separate code, chosen here once per tile)
+            auto drain = [&](auto gate) {
+                constexpr bool kGate = decltype(gate)::value;
+                const EpiOut<kGen, kGate> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
+                if constexpr (kMode >= 1 && kMode <= 4) {
+                    epilogue_decode<kMode, kGen>(a, u, lane_taddr, out, alv, al_lane);
+                } else if constexpr (kMode == 5) {
+                    switch (am) {
+                        case 5: epilogue_decode<5, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 6: epilogue_decode<6, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 7: epilogue_decode<7, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 8: epilogue_decode<8, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 9: epilogue_decode<9, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 10: epilogue_decode<10, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 11: epilogue_decode<11, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 12: epilogue_decode<12, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 13: epilogue_decode<13, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 14: epilogue_decode<14, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        case 15: epilogue_decode<15, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                        default: epilogue_decode<16, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
+                    }
+                } else {
+                    if constexpr (kGrouped) epilogue_tiled_grouped(a, u, lane_taddr, am, out, ehalf, al_lane);
+                    else epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0], release_acc);
                 }
+            };
+            if constexpr (kGen) {
+                if (a.act == 2) drain(std::true_type{});
+                else drain(std::false_type{});
             } else {
-                if constexpr (kGrouped) epilogue_tiled_grouped(a, u, lane_taddr, am, out, ehalf, al_lane);
-                else epilogue_tiled(a, u, lane_taddr, out, ehalf, alv[0], release_acc);
+                drain(std::false_type{});
             }
             if constexpr (kDec || kGrouped) release_acc();
             if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
@@ -1471,7 +1506,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * b0 : 2 * b0 + 1;
                     const float* first = a.partials + (size_t)slot0 * a.slot_floats;
                     const float* rest = a.partials + (size_t)(2 * (b0 + bstep)) * a.slot_floats;
-                    reduce_partials<kGen>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)bstep * a.slot_floats, c1 - c0);
+                    if (kGen && a.act == 2) reduce_partials<kGen, kGen>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)bstep * a.slot_floats, c1 - c0);
+                    else reduce_partials<kGen, false>(a, u, etid, n_epi_warps, first, rest, 2 * (size_t)bstep * a.slot_floats, c1 - c0);
                     if (etid == 0) a.counters[kPair ? 2 * unit + (int)rank : unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile

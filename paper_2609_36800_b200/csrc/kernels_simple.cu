@@ -73,9 +73,39 @@ __global__ void gemm_simt_kernel(const uint16_t* __restrict__ X, const uint16_t*
     const int b = (int)(gw / N);
     const int n = (int)(gw % N);
     const int words = K >> 5;
+    const float al = alpha[b];
+    if (act == 2) {
+        // SiLU gate over interleaved (gate, up) rows: the warp of the gate row computes both rows of its pair
+        if (n & 1) return;
+        for (int t = 0; t < m; ++t) {
+            const uint16_t* xrow = X + ((size_t)b * m + t) * K;
+            float z[2];
+            for (int r = 0; r < 2; ++r) {
+                const uint32_t* brow2 = bits + ((size_t)b * N + n + r) * words;
+                const uint16_t* wrow2 = W + (size_t)(n + r) * K;
+                float base = 0.f, delta = 0.f;
+                for (int w = lane; w < words; w += 32) {
+                    const uint32_t word = brow2[w];
+#pragma unroll 8
+                    for (int j = 0; j < 32; ++j) {
+                        const float x = io16_to_float(xrow[w * 32 + j], f16);
+                        base = fmaf(x, io16_to_float(wrow2[w * 32 + j], f16), base);
+                        delta += ((word >> j) & 1u) ? x : -x;
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    base += __shfl_xor_sync(0xFFFFFFFFu, base, o);
+                    delta += __shfl_xor_sync(0xFFFFFFFFu, delta, o);
+                }
+                z[r] = fmaf(al, delta, base) + (bias ? io16_to_float(bias[n + r], f16) : 0.f);
+            }
+            if (lane == 0) Y[((size_t)b * m + t) * (N >> 1) + (n >> 1)] = float_to_io16(z[0] / (1.f + __expf(-z[0])) * z[1], f16);
+        }
+        return;
+    }
     const uint32_t* brow = bits + ((size_t)b * N + n) * words;
     const uint16_t* wrow = W + (size_t)n * K;
-    const float al = alpha[b];
     const float bias_n = bias ? io16_to_float(bias[n], f16) : 0.f;
     for (int t = 0; t < m; ++t) {
         const uint16_t* xrow = X + ((size_t)b * m + t) * K;

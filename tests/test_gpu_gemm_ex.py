@@ -81,6 +81,32 @@ def test_bf16_epilogues_match_oracle(shape, opts):
     assert_parity(run_ex(X, W, bits, alpha, bias, "bf16", opts[1]), Yref, f"{shape} {opts}")
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "B%d_m%d_N%d_K%d" % s)
+def test_silu_gate_over_interleaved_rows_matches_oracle(shape, dtype):
+    B, m, N, K = shape
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B * 7 + m)
+    if dtype == "f16":
+        X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    else:
+        X, W, bits, alpha = synth.make_inputs(wl)
+        bias = synth.make_bias_bf16(N, seed=2)
+    Yref = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype=dtype, act="silu_gate")
+    Y = run_ex(X, W, bits, alpha, bias, dtype, "silu_gate")
+    assert Y.shape == (B, m, N // 2)
+    assert_parity(Y, Yref, f"{shape} {dtype}")
+
+
+def test_silu_gate_needs_an_even_feature_count():
+    lib = bd.load_library()
+    t = torch.zeros(256 * 128, dtype=torch.bfloat16, device="cuda")
+    bits = torch.zeros(129 * 4, dtype=torch.int32, device="cuda")
+    al = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws = bd.make_workspace(1, 1, 129, 128)
+    p = lambda x: ctypes.c_void_p(x.data_ptr())
+    assert lib.bitdelta_gemm_ex(p(t), p(t), p(bits), p(al), None, p(t), 1, 1, 129, 128, 0, 2, p(ws), ws.numel(), None) == 2
+
+
 def test_f16_delta_term_is_exact_for_full_precision_activations():
     # alpha = 1, W_base = 0, activations with all eleven significant bits set: Y is the exact sum of +-x,
     # and any piece of x lost by the e5m2 split would show at the 2^-10 level.
@@ -117,6 +143,6 @@ def test_unknown_option_codes_are_refused():
     al = torch.zeros(1, dtype=torch.float32, device="cuda")
     ws = bd.make_workspace(1, 1, 128, 128)
     p = lambda x: ctypes.c_void_p(x.data_ptr())
-    for dtype, act in ((2, 0), (0, 2), (-1, 0)):
+    for dtype, act in ((2, 0), (0, 3), (-1, 0)):
         st = lib.bitdelta_gemm_ex(p(t), p(t), p(bits), p(al), None, p(t), 1, 1, 128, 128, dtype, act, p(ws), ws.numel(), None)
         assert st == 8
