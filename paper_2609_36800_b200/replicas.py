@@ -18,3 +18,20 @@ def aggregate_throughput(units_per_rank: float, ms_per_rank: float, dist, device
     ms = max_over_ranks(ms_per_rank, dist, device)
     total = units_per_rank * world
     return total, ms, total / (ms / 1e3)
+
+
+def shard_tenants(B: int, world: int, rank: int):
+    """Tenants [start, start + count) that `rank` of `world` serves: a contiguous, even cut of the B tenants
+    (the first B % world ranks take one more).  W_base is replicated, so a rank needs nothing from the others."""
+    if B < 0 or world <= 0 or not 0 <= rank < world:
+        raise ValueError("bad shard request")
+    q, r = divmod(B, world)
+    start = rank * q + min(rank, r)
+    return start, q + (1 if rank < r else 0)
+
+
+def tenant_shard(X, bits, alpha, world: int, rank: int):
+    """This rank's slices of the per-tenant operands (X [B,m,K], bits [B,N,K/32], alpha [B]): views, no copies.
+    The product of the shard is rows [start, start + count) of the full product."""
+    start, count = shard_tenants(X.shape[0], world, rank)
+    return X[start:start + count], bits[start:start + count], alpha[start:start + count], start
