@@ -10,7 +10,8 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libbitdelta.so")
+# BITDELTA_LIB points at another build of the same library (the trace build made by `build.py --trace`).
+_LIB_PATH = os.environ.get("BITDELTA_LIB") or os.path.join(_HERE, "libbitdelta.so")
 _lib = None
 
 STATUS_OK = 0

@@ -124,13 +124,14 @@ bool encode_u8_2d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 3-D uint32 [B, N, K/32], box = 8 words (32 bytes) x 128 rows x tenants.
-bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, uint64_t words, uint32_t tenants) {
+// 3-D uint32 [B, N, K/32], box = `box_words` words (8: the signs of 256 k, 32 bytes; 4: of 128 k) x 128 rows x tenants.
+bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, uint64_t words, uint32_t tenants,
+                    uint32_t box_words = 8) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {words, N, B};
     cuuint64_t strides[2] = {words * 4, words * 4 * N};
-    cuuint32_t box[3] = {8, 128, tenants};
+    cuuint32_t box[3] = {box_words, 128, tenants};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -299,8 +300,8 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
 
     CUtensorMap tmW, tmX, tmX8, tmBits;
     if (!encode_bf16_tile(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
-    if (!encode_bf16_tile(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
-    if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB))
+    if (!p.stream && !encode_bf16_tile(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
+    if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, p.stream ? 4u : 8u))
         return BITDELTA_ERR_CUDA;
     if (p.decode && !p.convert) {
         // Decode schedule with many token rows per tile: split the activations into e5m2 pieces first
@@ -317,9 +318,18 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
 
     bd::GemmArgs args = bd::make_args(p, alpha, Y, workspace);
     args.f16 = f16; args.act = act; args.bias = bias;
+    args.X = X;
     { static int h = -1; if (h < 0) { const char* e = getenv("BITDELTA_HOLD"); h = (e && e[0] == '0') ? 0 : 1; } args.hold_prefetch = h; }
-    if (bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream) != cudaSuccess)
-        return BITDELTA_ERR_CUDA;
+#ifdef BD_TRACE
+    args.hold_prefetch = (int)(g_launches.load() & 1);   // trace build: alternate halves of the trace buffer
+#endif
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_EARLY_WEIGHTS"); d = (e && e[0] == '0') ? 0 : 1; } args.early_weights = d; }
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_EARLY_GAP"); d = e ? atoi(e) : 2500; } args.early_gap_ns = d; }
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_PREFETCH"); d = e ? atoi(e) : 0; } args.prefetch_steps = d; }
+    const cudaError_t le = p.stream
+        ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream)
+        : bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream);
+    if (le != cudaSuccess) return BITDELTA_ERR_CUDA;
     g_launches++;
     return BITDELTA_OK;
 }
@@ -383,7 +393,7 @@ int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
     if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
-    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.convert ? 2 : 1);
+    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.stream ? 5 : (p.convert ? 2 : 1));
     info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
     info[5] = p.whole_units ? 1 : (p.teams > 1 ? 2 : 0);
     info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;

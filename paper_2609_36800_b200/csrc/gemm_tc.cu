@@ -23,12 +23,12 @@
 
 #include <type_traits>
 
+#include "gemm_common.cuh"
 #include "gemm_tc.h"
 #include "ptx.cuh"
 
 namespace bd {
 
-constexpr long long kWaitLimitCycles = 4000000000ll;   // every spin gives up after 4e9 SM cycles (~2 s)
 constexpr int kThreads = 512;
 constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
@@ -37,69 +37,6 @@ constexpr int kWarpDelta0 = 2;     // decode schedule: warps 2..3 issue the delt
 constexpr int kBarAFull0 = 2;      // named barriers 2..9 : decode group g, buffer b -> id 2 + g*4 + b
 constexpr int kWarpDecode0 = 4;    // warps 4..11
 constexpr int kWarpEpi0 = 12;      // warps 12..15
-
-#ifdef BD_TRACE
-// Debug builds only: per-CTA cycle stamps of the main phases.
-__device__ long long* g_trace_ptr;
-// What-if switches for timing experiments (results are wrong when any is set):
-// 1 skip sign decode ALU, 2 skip delta MMAs, 4 skip base MMAs, 8 skip sign-word loads, 16 skip W loads,
-// 32 skip activation loads, 64 skip tensor-memory stores of the decode warps, 128 skip the in-kernel split
-__device__ int g_knobs;
-#ifdef BD_NO_KNOBS
-#define BD_KNOB(bit) 0
-#define BD_KNOB_LOAD do { } while (0)
-#else
-#define BD_KNOB_LOAD const int bd_knobs = g_knobs
-#define BD_KNOB(bit) (bd_knobs & (bit))
-#endif
-#define BD_KNOB_G(bit) (g_knobs & (bit))
-#ifndef BD_TLN
-#define BD_TLN 20      // stamps kept per role ...
-#endif
-#ifndef BD_TLSKIP
-#define BD_TLSKIP 0   // ... after skipping this many
-#endif
-// Stamps go to shared memory (behind the control block; the launcher adds about 1 KB in debug builds) and are
-// copied out at teardown, so that taking one costs a clock read and a shared-memory store.
-// bd_st[32]: per-CTA phase stamps and accumulators.  bd_tlb[5][BD_TLN]: per-role timelines (CTA 0 and 77 are kept).
-#define BD_TRACE_SETUP \
-    long long* const bd_st = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(ctl) + kSmemCtrlBytes); \
-    long long* const bd_tlb = bd_st + 32; \
-    for (int i = threadIdx.x; i < 32 + 5 * BD_TLN; i += kThreads) bd_st[i] = 0; \
-    __syncthreads()
-#define BD_TRACE_FLUSH do { \
-    long long* gp = g_trace_ptr; \
-    if (gp) { \
-        for (int i = threadIdx.x; i < 32; i += kThreads) gp[blockIdx.x * 32 + i] = bd_st[i]; \
-        if (blockIdx.x == 0 || blockIdx.x == 77) \
-            for (int i = threadIdx.x; i < 5 * BD_TLN; i += kThreads) gp[8192 + (blockIdx.x ? 1024 : 0) + (i / BD_TLN) * 128 + (i % BD_TLN)] = bd_tlb[i]; \
-    } } while (0)
-#define BD_STAMP(idx) do { if (lane == 0) bd_st[idx] = clock64(); } while (0)
-#define BD_STAMP_ONCE(idx) do { if (lane == 0 && bd_st[idx] == 0) bd_st[idx] = clock64(); } while (0)
-#define BD_TL_DECL int tl_idx = 0
-#define BD_TL(role) do { if ((role) < 5 && lane == 0 && tl_idx >= BD_TLSKIP && tl_idx < BD_TLSKIP + BD_TLN) { bd_tlb[(role) * BD_TLN + tl_idx - BD_TLSKIP] = clock64(); } ++tl_idx; } while (0)
-#define BD_TL2(role) do { } while (0)
-#define BD_ACC_DECL(name) long long name = 0
-#define BD_ACC_BEGIN(t) const long long t = clock64()
-#define BD_ACC_END(name, t) name += clock64() - t
-#define BD_ACC_STORE(idx, name) do { if (lane == 0) bd_st[idx] = name; } while (0)
-#else
-#define BD_TRACE_SETUP do { } while (0)
-#define BD_TRACE_FLUSH do { } while (0)
-#define BD_STAMP(idx) do { } while (0)
-#define BD_STAMP_ONCE(idx) do { } while (0)
-#define BD_KNOB(bit) 0
-#define BD_KNOB_G(bit) 0
-#define BD_KNOB_LOAD do { } while (0)
-#define BD_TL_DECL do { } while (0)
-#define BD_TL(role) do { } while (0)
-#define BD_ACC_DECL(name) do { } while (0)
-#define BD_ACC_BEGIN(t) do { } while (0)
-#define BD_ACC_END(name, t) do { } while (0)
-#define BD_ACC_STORE(idx, name) do { } while (0)
-#endif
-
-__device__ unsigned int g_device_status[2];   // [0] status code (0 = ok), [1] site of the first failure
 
 struct Ctl {
     uint64_t wfull[kMaxStages];        // W_base tile landed
@@ -121,428 +58,6 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= kSmemCtrlBytes, "control block too large");
 
-// Bounded wait on an mbarrier phase.  Returns false if the wait was abandoned
-// (limit reached here or in another thread of the CTA).  The slow path is kept out of line: it is
-// instantiated at some twenty call sites and would otherwise dominate the kernel's code size.
-__device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
-    // Poll, and every 64 polls look at the abort flag and the SM cycle counter
-    // (cheap to read; the limit is ~2 s at 2 GHz, longer at lower clocks).
-    const long long t0 = clock64();
-#pragma unroll 1
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i) {
-            if (mbar_try_wait(bar, parity)) return true;
-        }
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *abort_flag = 1;
-            if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_bar_slow(bar, parity, abort_flag, site);
-}
-
-// Walks the k-pair items [lo, hi) of this CTA as segments (unit, p0, p1).
-struct SegIter {
-    int cur, hi;
-    int P;
-    int stride;   // 0: the CTA owns the items [cur, hi); > 0: whole units cur/P, cur/P + stride, ... (see plan.h)
-    __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
-        if (cur >= hi) return false;
-        unit = (int)((unsigned)cur / (unsigned)P);
-        if (stride > 0) {
-            p0 = 0;
-            p1 = P;
-            cur += stride * P;
-            return true;
-        }
-        p0 = cur - unit * P;
-        const int rem = hi - cur;
-        const int len = (rem < P - p0) ? rem : (P - p0);
-        p1 = p0 + len;
-        cur += len;
-        return true;
-    }
-};
-
-// The same walk, one (unit, k-pair) item at a time.
-struct ItemIter {
-    SegIter seg;
-    int unit, p, p1;
-    bool first;   // first item of its segment
-    __device__ __forceinline__ explicit ItemIter(const SegIter& s) : seg(s), unit(0), p(0), p1(0), first(false) {}
-    __device__ __forceinline__ bool next() {
-        if (p + 1 < p1) { ++p; first = false; return true; }
-        int p0;
-        if (!seg.next(unit, p0, p1)) { p = 0; p1 = 0; return false; }
-        p = p0;
-        first = true;
-        return true;
-    }
-};
-
-// Cursor over a ring of n buffers: index of the current buffer and the parity of its use count.
-struct Ring {
-    int idx;
-    uint32_t par;
-    int n;
-    __device__ __forceinline__ void step() {
-        if (++idx == n) { idx = 0; par ^= 1; }
-    }
-};
-
-struct Unit {
-    int n0;        // first weight row of the tile
-    int tenant0;   // first tenant
-    int nten;      // tenants in this unit
-    int xrow0;     // first row of X (in the [B*m, K] view) staged for this unit
-    int ntok;      // output tokens of this unit (rows xrow0 .. xrow0+ntok-1)
-};
-
-template <bool kDec, bool kGrouped, bool kPair = false>
-__device__ __forceinline__ Unit unit_info_t(const GemmArgs& a, int unit, int am, int rank = 0) {
-    Unit u;
-    int nt, g;
-    if ((kDec || kGrouped) && a.teams > 1) {   // group-major (never in the one-tenant tiled schedule)
-        g = (int)((unsigned)unit / (unsigned)a.n_tiles);
-        nt = unit - g * a.n_tiles;
-    } else {
-        nt = unit / a.groups;
-        g = unit - nt * a.groups;
-    }
-    if constexpr (kPair) nt = 2 * nt + rank;   // the pair's two W_base tiles
-    u.n0 = nt * kTileN;
-    if constexpr (kDec || kGrouped) {   // decode schedules, and the tiled schedule with several tenants per unit
-        u.tenant0 = g * a.TB;
-        u.nten = min(a.TB, a.B - u.tenant0);
-        u.xrow0 = u.tenant0 * am;
-        u.ntok = u.nten * am;
-    } else {
-        const int b = g / a.m_tiles;
-        const int mt = g - b * a.m_tiles;
-        u.tenant0 = b;
-        u.nten = 1;
-        u.xrow0 = b * am + mt * a.tok_tile;
-        u.ntok = min(a.tok_tile, am - mt * a.tok_tile);
-    }
-    return u;
-}
-
-// 32 packed sign bits (k = 0..31 of the word, LSB first) -> 16 registers of two
-// bf16 each, register c = {k = 2c (low half), k = 2c+1 (high half)}, +1 for a
-// set bit and -1 for a clear bit.  Only shifts and three-input logic ops: the
-// wanted bits are moved onto the two bf16 sign positions and flip the sign of a
-// packed (-1, -1) constant (`minus_one2`: 0xBF80BF80 as bf16, 0xBC00BC00 as binary16).
-__device__ __forceinline__ void decode_word(uint32_t w, uint32_t* r, uint32_t minus_one2) {
-    // even bits of the low half stay at 2c, odd bits move to 2c+16 (junk only on odd positions)
-    const uint32_t lo = (w & 0x0000FFFFu) | ((w << 15) & 0xFFFF0000u);
-    const uint32_t hi = (w >> 16) | ((w >> 1) & 0xFFFF0000u);
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        r[c] = ((lo << (15 - 2 * c)) & 0x80008000u) ^ minus_one2;
-        r[8 + c] = ((hi << (15 - 2 * c)) & 0x80008000u) ^ minus_one2;
-    }
-}
-
-// ------------------------------------------------------------------- epilogue helpers
-template <int W>
-__device__ __forceinline__ void tmem_ld_w(uint32_t taddr, uint32_t* r) {
-    if constexpr (W == 1) tmem_ld1(taddr, r);
-    else if constexpr (W == 2) tmem_ld2(taddr, r);
-    else if constexpr (W == 4) tmem_ld4(taddr, r);
-    else if constexpr (W == 8) tmem_ld8(taddr, r);
-    else tmem_ld16(taddr, r);
-}
-
-// Fused epilogue on a finished sum: bias, then the activation, then rounding to the I/O type.
-__device__ __forceinline__ float epi_finish(float v, float bias, int act) {
-    v += bias;
-    if (act == 1) v = __fdividef(v, 1.f + __expf(-v));   // SiLU; approximate division (2 ulp) keeps the unrolled epilogues small
-    return v;
-}
-__device__ __forceinline__ uint16_t to_io16(float v, int f16) {
-    return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
-}
-__device__ __forceinline__ uint16_t finish_io16(float v, float bias, int act, int f16) {
-    return to_io16(epi_finish(v, bias, act), f16);
-}
-__device__ __forceinline__ float from_io16(uint16_t h, int f16) {
-    return f16 ? __half2float(__ushort_as_half(h)) : __uint_as_float((uint32_t)h << 16);
-}
-
-// kGen = false: bf16 output, no bias, no activation (the plain product).  The two forms are separate code
-// on purpose: the epilogue runs once per tile, every instruction of it is fetched cold, and the plain
-// product should not pay for the general form's length.
-template <bool kGen, bool kGate = false>
-struct EpiOut {
-    uint16_t* Y;        // output matrix [B*m, N], 16-bit values of the I/O type
-    float* slot;        // partial-result slot, or nullptr when this CTA owns the whole tile
-    int N, n, row, xrow0;
-    float bias;         // of output feature n (0 without a bias)
-    const GemmArgs& a;  // kernel parameters (activation code, I/O type)
-    // (called by all lanes of a warp together: the gated form exchanges values between neighbouring lanes)
-    __device__ __forceinline__ void put(int tok, float v) const {
-        if (slot) {
-            slot[(size_t)tok * kTileN + row] = v;   // partial sums: finished by the CTA that adds them up
-            return;
-        }
-        if constexpr (kGate) {
-            // SiLU gate: weight rows come in pairs (2i: gate, 2i+1: up), i.e. in neighbouring lanes
-            const float z = v + bias;
-            const float other = __shfl_xor_sync(0xFFFFFFFFu, z, 1);
-            if (!(n & 1) && n < N)
-                Y[(size_t)(xrow0 + tok) * (N >> 1) + (n >> 1)] = to_io16(__fdividef(z, 1.f + __expf(-z)) * other, a.f16);
-            return;
-        }
-        if (n < N) {
-            if constexpr (kGen) Y[(size_t)(xrow0 + tok) * N + n] = finish_io16(v, bias, a.act, a.f16);
-            else Y[(size_t)(xrow0 + tok) * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-        }
-    }
-};
-
-// Decode schedule, M tokens per tenant: the base accumulator holds tenant j's tokens in columns
-// j*M .. j*M+M-1; its delta accumulator starts at column N3*j and holds, for piece q of the
-// activation split, token t in column q*M + t.  delta = D0 + D1 + D2 + D3.
-// Plain product: the tenant loop is unrolled (the tensor-memory loads of all tenants overlap).  General form
-// with more than four tokens per tenant: a real loop, because its body is long, this code runs once per tile
-// and every instruction of it is fetched cold, so its length is paid in time.
-// `alv[j]`: tenant j's scale (unrolled form); `al_lane`: lane l holds tenant l's scale (loop form).
-template <int M, bool kGen, class Out>
-__device__ __forceinline__ void epilogue_decode(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                                const Out& out, const float* alv, float al_lane) {
-    constexpr int N3 = (kPieces * M + 15) / 16 * 16;
-    constexpr int TPB = (N3 == 16) ? 2 : 1;   // tenants drained per wait
-    constexpr int kMaxTen = (M <= 4) ? 8 : 4;   // tenants per unit (see the plan)
-    constexpr bool kLoop = kGen && M > 4;
-    auto drain = [&](int j0) {
-        uint32_t rb[16], rd[TPB * N3];
-        tmem_ld16(lane_taddr + (uint32_t)(j0 * M), rb);
-#pragma unroll
-        for (int jj = 0; jj < TPB; ++jj) {
-#pragma unroll
-            for (int c = 0; c < N3; c += 16)
-                tmem_ld16(lane_taddr + a.col_delta + (uint32_t)((j0 + jj) * N3 + c), rd + jj * N3 + c);
-        }
-        tc_wait_ld();
-#pragma unroll
-        for (int jj = 0; jj < TPB; ++jj) {
-            if (j0 + jj < u.nten) {   // warp-uniform
-                float al;
-                if constexpr (kLoop) al = __shfl_sync(0xFFFFFFFFu, al_lane, j0 + jj);
-                else al = alv[j0 + jj];
-#pragma unroll
-                for (int t = 0; t < M; ++t) {
-                    const float lo = __uint_as_float(rd[jj * N3 + 2 * M + t]) + __uint_as_float(rd[jj * N3 + 3 * M + t]);
-                    const float hi = __uint_as_float(rd[jj * N3 + t]) + __uint_as_float(rd[jj * N3 + M + t]);
-                    out.put((j0 + jj) * M + t, fmaf(al, hi + lo, __uint_as_float(rb[jj * M + t])));
-                }
-            }
-        }
-    };
-    if constexpr (kLoop) {
-#pragma unroll 1
-        for (int j0 = 0; j0 < u.nten; j0 += TPB) drain(j0);
-    } else {
-#pragma unroll
-        for (int j0 = 0; j0 < kMaxTen; j0 += TPB) {
-            if (j0 >= u.nten) break;
-            drain(j0);
-        }
-    }
-}
-
-// Tiled schedule: one tenant, tokens in columns 0..ntok-1 of both accumulators.
-// Two warps share each lane quadrant: warp half h drains the 32-token blocks h, h+2, ...
-// `release` hands the accumulators back (this warp's arrival): it is called as soon as the warp's last
-// tensor-memory load has completed, before the values of that load are finished and stored.
-template <class Out, class Release>
-__device__ __forceinline__ void epilogue_tiled(const GemmArgs& a, const Unit& u, uint32_t lane_taddr,
-                                               const Out& out, int half, float al, const Release& release) {
-    if (32 * half >= u.ntok) release();
-    for (int t0 = 32 * half; t0 < u.ntok; t0 += 64) {
-        uint32_t rb[32], rd[32];
-        tmem_ld32(lane_taddr + (uint32_t)t0, rb);
-        tmem_ld32(lane_taddr + a.col_delta + (uint32_t)t0, rd);
-        tc_wait_ld();
-        if (t0 + 64 >= u.ntok) release();
-        const int nvalid = min(32, u.ntok - t0);
-#pragma unroll
-        for (int t = 0; t < 32; ++t) {
-            if (t < nvalid) out.put(t0 + t, fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t])));
-        }
-    }
-}
-
-// Tiled schedule with several tenants per unit (16 < m <= 64): tenant j's base columns start at j*m, its delta
-// columns at j*Nd; 16-token chunks, dealt alternately to the two warps of a lane quadrant.
-// `al_lane`: lane l holds the scale of the unit's tenant l.
-template <class Out>
-__device__ __forceinline__ void epilogue_tiled_grouped(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, int m,
-                                                       const Out& out, int half, float al_lane) {
-    const int chunks = (m + 15) >> 4;
-#pragma unroll 1
-    for (int c = half; c < u.nten * chunks; c += 2) {
-        const int j = c / chunks, t0 = (c - j * chunks) * 16;
-        uint32_t rb[16], rd[16];
-        tmem_ld16(lane_taddr + (uint32_t)(j * m + t0), rb);
-        tmem_ld16(lane_taddr + a.col_delta + (uint32_t)(j * a.Nd + t0), rd);
-        tc_wait_ld();
-        const float al = __shfl_sync(0xFFFFFFFFu, al_lane, j);
-        const int nvalid = min(16, m - t0);
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            if (t < nvalid) out.put(j * m + t0 + t, fmaf(al, __uint_as_float(rd[t]), __uint_as_float(rb[t])));
-        }
-    }
-}
-
-__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
-
-// Sums the partial results of a tile cut across CTAs c0..c1 (in that order) and writes Y.
-// nwarps*32 threads: thread e owns rows 4*(e%32)..+3 of tokens e/32, e/32+nwarps, ...
-template <bool kGen, bool kGate>
-__device__ __forceinline__ void reduce_partials(const GemmArgs& a, const Unit& u, int etid, int nwarps,
-                                                const float* first, const float* rest, size_t cstride, int nrest) {
-    uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
-    const int r4 = (etid & 31) * 4;
-    const int n = u.n0 + r4;
-    const bool vec_ok = ((a.N & 3) == 0) && (n + 3 < a.N);
-    float bias4[4] = {0.f, 0.f, 0.f, 0.f};
-    if (kGen && a.bias) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (n + i < a.N) bias4[i] = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n + i), a.f16);
-    }
-    for (int tk = etid >> 5; tk < u.ntok; tk += 4 * nwarps) {
-        float4 acc[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int t = tk + nwarps * q;
-            acc[q] = (t < u.ntok) ? ldcg4(first + (size_t)t * kTileN + r4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        for (int c = 0; c < nrest; ++c) {
-            const float* pc = rest + (size_t)c * cstride;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int t = tk + nwarps * q;
-                if (t < u.ntok) {
-                    const float4 v = ldcg4(pc + (size_t)t * kTileN + r4);
-                    acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
-                }
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int t = tk + nwarps * q;
-            if (t < u.ntok) {
-                if constexpr (kGate) {
-                    {
-                        // SiLU gate: rows (n, n+1) and (n+2, n+3) are (gate, up) pairs; N is even and n a multiple of 4
-                        const float g0 = acc[q].x + bias4[0], u0 = acc[q].y + bias4[1];
-                        const float g1 = acc[q].z + bias4[2], u1 = acc[q].w + bias4[3];
-                        uint16_t* dg = Y + (size_t)(u.xrow0 + t) * (a.N >> 1) + (n >> 1);
-                        if (n < a.N) dg[0] = to_io16(__fdividef(g0, 1.f + __expf(-g0)) * u0, a.f16);
-                        if (n + 2 < a.N) dg[1] = to_io16(__fdividef(g1, 1.f + __expf(-g1)) * u1, a.f16);
-                        continue;
-                    }
-                }
-                uint16_t* dst = Y + (size_t)(u.xrow0 + t) * a.N + n;
-                uint16_t o0, o1, o2, o3;
-                if constexpr (kGen) {
-                    o0 = finish_io16(acc[q].x, bias4[0], a.act, a.f16);
-                    o1 = finish_io16(acc[q].y, bias4[1], a.act, a.f16);
-                    o2 = finish_io16(acc[q].z, bias4[2], a.act, a.f16);
-                    o3 = finish_io16(acc[q].w, bias4[3], a.act, a.f16);
-                } else {
-                    o0 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].x));
-                    o1 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].y));
-                    o2 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].z));
-                    o3 = __bfloat16_as_ushort(__float2bfloat16_rn(acc[q].w));
-                }
-                if (vec_ok) {
-                    *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)o0 | ((uint32_t)o1 << 16), (uint32_t)o2 | ((uint32_t)o3 << 16));
-                } else {
-                    if (n + 0 < a.N) dst[0] = o0;
-                    if (n + 1 < a.N) dst[1] = o1;
-                    if (n + 2 < a.N) dst[2] = o2;
-                    if (n + 3 < a.N) dst[3] = o3;
-                }
-            }
-        }
-    }
-}
-
-// In-kernel activation split (decode schedule, few token rows per unit).  Task (r, q4, h, pc): token row
-// r, 32-k group q4 of the stage, half h of the group's byte slots, pair pc of the half's four k classes.
-// Slot 4c+i holds k = c + 8i, so the task's classes c = 4h+2pc, 4h+2pc+1 need, from each of the four
-// 16-byte chunks (i = 0..3) of the group, the 4 bytes holding k = 8i+c, 8i+c+1, and produce 8 bytes
-// (slots 16h+8pc .. +7) per piece.
-// The pieces are taken by TRUNCATION on packed f16 pairs (a bf16 value in the e5m2 range is exact in f16,
-// and an e5m2 number is the high byte of an f16 number): p = y with its low byte cleared, y -= p (exact).
-// A bf16 value has 8 significant bits and every piece removes the top three of what is left, so the third
-// piece leaves nothing and the fourth is zero; no conversion instruction is needed (they are slow enough
-// to hold up the decode warps that share a scheduler with the splitting warp).
-// `xt` is the stage's X tile (two swizzled 64-k atoms), `x8t` its piece tile.  Thread `tid` of `nthreads`
-// takes the tasks tid, tid + nthreads, ...  Small tasks on purpose: 16 per token row spread the work over
-// all four epilogue warps, one warp per scheduler.
-template <bool kF16>
-__device__ __forceinline__ void split_activations(const GemmArgs& a, int am, const uint8_t* xt, uint8_t* x8t, int ntok, int tid,
-                                                  int nthreads) {
-    const int ntasks = BD_KNOB_G(128) ? 0 : ntok * 16;
-    for (int task = tid; task < ntasks; task += nthreads) {
-        const int r = task >> 4, q4 = (task >> 2) & 3, h = (task >> 1) & 1, pc = task & 1;
-        const int j = r / am, t = r - j * am;
-        const uint8_t* src = xt + (q4 >> 1) * a.x_atom_bytes + r * 128 + h * 8 + pc * 4;
-        uint32_t y[4];   // y[i]: f16 pair, k = 8i + 4h + 2pc, +1
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int chunk = ((q4 & 1) * 4 + i) ^ (r & 7);
-            const uint32_t v = *reinterpret_cast<const uint32_t*>(src + chunk * 16);
-            if constexpr (kF16) {
-                y[i] = v;   // binary16 already: eleven significant bits, the four pieces take 3 + 3 + 3 + 2
-            } else {
-                const __half2 hv = __floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
-                y[i] = *reinterpret_cast<const uint32_t*>(&hv);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < kPieces; ++q) {
-            uint32_t pq[4];   // byte 1 / byte 3: the e5m2 piece of k / k+1
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                pq[i] = y[i] & 0xFF00FF00u;
-                if (q + 1 < kPieces) {
-                    const __half2 d = __hsub2(*reinterpret_cast<const __half2*>(&y[i]), *reinterpret_cast<const __half2*>(&pq[i]));
-                    y[i] = *reinterpret_cast<const uint32_t*>(&d);
-                }
-            }
-            // bytes (i = 0..3) of element k, then of element k+1
-            const uint32_t t01 = __byte_perm(pq[0], pq[1], 0x7351);   // [p0.b1, p1.b1, p0.b3, p1.b3]
-            const uint32_t t23 = __byte_perm(pq[2], pq[3], 0x7351);
-            const uint2 w = make_uint2(__byte_perm(t01, t23, 0x5410), __byte_perm(t01, t23, 0x7632));
-            const int r8 = j * (kPieces * am) + q * am + t;
-            *reinterpret_cast<uint2*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16) + pc * 8) = w;
-        }
-    }
-}
-
-// 32 packed sign bits -> 8 registers of four e5m2 each (+1 = 0x3C, -1 = 0xBC).  Register c takes
-// bits c, c+8, c+16, c+24 (its bytes 0..3): one shift lands all four on the byte sign positions, one
-// three-input logic op masks them and flips the sign of a packed (-1,-1,-1,-1).  The k order inside
-// the group of 32 is therefore permuted (slot 4c+i holds k = c + 8i); the activation pieces are
-// stored with the same permutation, so the contraction is unchanged.
-__device__ __forceinline__ void decode_word_e5m2(uint32_t w, uint32_t* r) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) r[c] = ((w << (7 - c)) & 0x80808080u) ^ 0xBCBCBCBCu;
-}
-
-__device__ __forceinline__ void epi_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 // kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m;
 // 6: tiled schedule with several tenants per unit.
@@ -583,13 +98,10 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec, kGrouped, kPair>(aa, un, am, (int)rank); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    BD_KNOB_LOAD;
-    BD_TRACE_SETUP;
     // Tiled schedule: signs need few decode threads, the epilogue many -> warps 8..11 drain accumulators
     // instead of decoding.
     constexpr int epi_first_warp = kDec ? kWarpEpi0 : kWarpEpi0 - 4;
     constexpr int n_epi_warps = 16 - epi_first_warp;
-    if (warp == 0) BD_STAMP(0);
     if (threadIdx.x == 32) {
         prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmX);
@@ -616,22 +128,16 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             // leader's barrier, which only the leader arms.
             if (rank == 0) mbar_arrive_expect_tx(bar, 2u * (a.w_stage_bytes + 2 * a.x_atom_bytes));
             tma_load_3d_pair(dst, &tmW, mapa_shared(bar, 0), 0, u.n0, k0 / kAtomK);
-        } else if (BD_KNOB(16)) {
-            mbar_arrive(bar);
         } else {
             // tiled schedule: the stage's activation tile (same slot index, queued by the activation
             // stream) completes on this barrier too
-            mbar_arrive_expect_tx(bar, a.w_stage_bytes + ((kDec || BD_KNOB(32)) ? 0u : 2 * a.x_atom_bytes));
+            mbar_arrive_expect_tx(bar, a.w_stage_bytes + (kDec ? 0u : 2 * a.x_atom_bytes));
             tma_load_3d(dst, &tmW, bar, 0, u.n0, k0 / kAtomK);   // both 64-k atoms of the tile
         }
         if (with_bits) {
             const uint32_t bbar = smem_u32(&ctl->bfull[bslot]);
-            if (BD_KNOB(8)) {
-                mbar_arrive(bbar);
-            } else {
-                mbar_arrive_expect_tx(bbar, a.bslot_bytes);
-                tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (p >> 1) * 8, u.n0, u.tenant0);
-            }
+            mbar_arrive_expect_tx(bbar, a.bslot_bytes);
+            tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (p >> 1) * 8, u.n0, u.tenant0);
         }
     };
 
@@ -675,7 +181,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             const int unit0 = (int)((unsigned)lo / (unsigned)a.P);
             issue_weights_raw(unit_info(a, unit0), a.whole_units ? 0 : lo - unit0 * a.P, 0, 0, true);
         }
-        BD_STAMP(2);
     }
     if (warp == kWarpTmem) {
         if constexpr (kPair) {
@@ -697,7 +202,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     }
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
-    if (warp == 0) BD_STAMP(1);
     // A kernel queued behind this one with an early start may begin its own prologue and weight
     // prefetch as soon as SMs free up; it waits for this grid to finish before it touches anything
     // this grid reads or writes.
@@ -718,7 +222,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint32_t phase = 0, xphase = 0, pphase = 0, bphase = 0;
         bool ok = true, dep_ok = false;
         bool hold = kDec && a.hold_prefetch != 0;
-        BD_ACC_DECL(w_empty); BD_ACC_DECL(w_bempty); BD_TL_DECL;
         Unit uw{}, ux{};
         bool more_w = wi.next();
         // (decode schedule, many token rows per unit: the activation tiles are queued by two of the otherwise
@@ -749,25 +252,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             // queued by thread 0 in the prologue: W stage 0, sign-word slot 0
             bslot = 1; bphase = 0u;   // (at least two sign-word slots)
             stage = 1 % a.n_w; phase = (a.n_w == 1) ? 1u : 0u;
-            BD_TL(0);
             uw = unit_info(a, wi.unit);
             more_w = wi.next();
             if (more_w && wi.first) uw = unit_info(a, wi.unit);
         }
         const uint32_t depbar = smem_u32(&ctl->depready);
-        const uint32_t x_tx = BD_KNOB(32) ? 0u : a.x_tile_bytes;
         long long t_idle = 0;
         int idle = 0;
-#ifdef BD_TRACE
-        long long idle_b = 0, idle_w = 0;
-#endif
-        BD_ACC_DECL(t_x); BD_ACC_DECL(t_p); BD_ACC_DECL(t_w); BD_ACC_DECL(n_iter);
         while (more_w || more_x || more_p || more_b) {
             bool did = false;
-#ifdef BD_TRACE
-            ++n_iter;
-#endif
-            BD_ACC_BEGIN(tx0);
             if (more_x) {
                 if (!dep_ok) dep_ok = warp_all(mbar_test_wait(depbar, 0));
                 const uint32_t xebar = kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot]);
@@ -779,11 +272,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         if constexpr (kPair) {
                             // this CTA's half of the token tile, counted on the leader's barrier
                             tma_load_3d_pair(dst, &tmX, mapa_shared(bar, 0), 0, ux.xrow0 + (int)rank * (a.tok_tile / 2), k0 / kAtomK);
-                        } else if (x_tx) {
-                            if (kDec) mbar_arrive_expect_tx(bar, x_tx);
+                        } else {
+                            if (kDec) mbar_arrive_expect_tx(bar, a.x_tile_bytes);
                             tma_load_3d(dst, &tmX, bar, 0, ux.xrow0, k0 / kAtomK);   // both 64-k atoms
-                        } else if (kDec) {
-                            mbar_arrive(bar);
                         }
                     }
                     __syncwarp();
@@ -793,19 +284,13 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
-            BD_ACC_END(t_x, tx0);
-            BD_ACC_BEGIN(tp0);
             if (more_p) {
                 if (!dep_ok) dep_ok = warp_all(mbar_test_wait(depbar, 0));
                 if (dep_ok && warp_all(mbar_test_wait(smem_u32(&ctl->x8empty[pslot]), pphase ^ 1))) {
                     if (elect_one()) {
                         const uint32_t bar = smem_u32(&ctl->x8full[pslot]);
-                        if (BD_KNOB(32)) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
-                            tma_load_2d(x8_addr + pslot * a.x8_atom_bytes, &tmX8, bar, pi.p * kPairK, up.tenant0 * kPieces * am);
-                        }
+                        mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
+                        tma_load_2d(x8_addr + pslot * a.x8_atom_bytes, &tmX8, bar, pi.p * kPairK, up.tenant0 * kPieces * am);
                     }
                     __syncwarp();
                     if (++pslot == a.n_x8) { pslot = 0; pphase ^= 1; }
@@ -814,17 +299,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
-            BD_ACC_END(t_p, tp0);
             if (!kDec && more_b) {
                 if (warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) {
                     if (elect_one()) {
                         const uint32_t bbar = smem_u32(&ctl->bfull[bslot]);
-                        if (BD_KNOB(8)) {
-                            mbar_arrive(bbar);
-                        } else {
-                            mbar_arrive_expect_tx(bbar, a.bslot_bytes);
-                            tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (bi.p >> 1) * 8, ub.n0, ub.tenant0);
-                        }
+                        mbar_arrive_expect_tx(bbar, a.bslot_bytes);
+                        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bbar, (bi.p >> 1) * 8, ub.n0, ub.tenant0);
                     }
                     __syncwarp();
                     if (++bslot == a.n_bits) { bslot = 0; bphase ^= 1; }
@@ -832,7 +312,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
-            BD_ACC_BEGIN(tw0);
             if (more_w && hold) {
                 // The first sign-word load of a tile pulls whole 128-byte lines (the signs of 1024 k) out of
                 // DRAM; until it has landed, further weight requests would only queue in front of it.
@@ -842,11 +321,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 const bool need_slot = kDec && (wi.first || !(wi.p & 1));
                 if ((!need_slot || warp_all(mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1))) &&
                     warp_all(mbar_test_wait(smem_u32(&ctl->wempty[stage]), phase ^ 1))) {
-                    BD_ACC_BEGIN(ti);
                     if (elect_one()) issue_weights_raw(uw, wi.p, stage, bslot, need_slot);
                     __syncwarp();
-                    BD_ACC_END(w_bempty, ti);
-                    BD_TL(0);
                     if (need_slot && ++bslot == a.n_bits) { bslot = 0; bphase ^= 1; }
                     if (++stage == a.n_w) { stage = 0; phase ^= 1; }
                     more_w = wi.next();
@@ -854,25 +330,16 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     did = true;
                 }
             }
-            BD_ACC_END(t_w, tw0);
             if (did) {
                 idle = 0;
                 continue;
             }
             // Nothing can advance: a short suspended wait (tens of ns) on one ring, then look at both again.
-#ifdef BD_TRACE
-            if (more_w && !hold) {
-                const bool ns = wi.first || !(wi.p & 1);
-                if (ns && !mbar_test_wait(smem_u32(&ctl->bempty[bslot]), bphase ^ 1)) ++idle_b; else ++idle_w;
-            }
-#endif
-            BD_ACC_BEGIN(te);
             if (more_w && hold) (void)mbar_try_wait_hint(smem_u32(&ctl->bfull[0]), 0u, 64u);
             else if (more_w) (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[stage]), phase ^ 1, 64u);
             else if (more_b) (void)mbar_try_wait_hint(smem_u32(&ctl->bempty[bslot]), bphase ^ 1, 64u);
             else (void)mbar_try_wait_hint(dep_ok ? (kDec ? smem_u32(&ctl->xempty[xslot]) : smem_u32(&ctl->wempty[xslot])) : depbar,
                                           dep_ok ? (xphase ^ 1) : 0u, 64u);
-            BD_ACC_END(w_empty, te);
             if (idle == 0) t_idle = clock64();
             if ((++idle & 255) == 0) {
                 if (*abort_flag) { ok = false; break; }
@@ -885,12 +352,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
         }
         (void)ok;
-        BD_STAMP(3);
-        BD_ACC_STORE(19, w_empty); BD_ACC_STORE(20, w_bempty);
-#ifdef BD_TRACE
-        BD_ACC_STORE(15, idle_b * 1965); BD_ACC_STORE(29, idle_w * 1965);
-        BD_ACC_STORE(4, t_x); BD_ACC_STORE(5, t_p); BD_ACC_STORE(30, t_w); BD_ACC_STORE(31, n_iter * 1965);
-#endif
     } else if (warp == kWarpMma) {
         // -------------------------------------------------------------- MMA issuer
         // Warp-uniform loop, one elected lane issues: descriptors and predicates then live in
@@ -911,39 +372,27 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int stage = 0, xslot = 0;
         uint32_t phase = 0, xphase = 0, accphase = 0, item = 0;
         bool ok = true;
-        BD_ACC_DECL(w_full); BD_ACC_DECL(w_afull); BD_ACC_DECL(w_acc); BD_ACC_DECL(w_ib); BD_ACC_DECL(w_id); BD_TL_DECL;
         // This warp also tells the producer when the grid this launch depends on has completed.
-        BD_STAMP(30);
         grid_dependency_wait();
         if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));
-        BD_STAMP(31);
         // (pair schedule: only the leader's warp issues; its MMAs and commits act on both CTAs)
         while (ok && (!kPair || rank == 0) && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
-            BD_ACC_BEGIN(ta);
             ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
-            BD_ACC_END(w_acc, ta);
             if (!ok) break;
             tc_fence_after();
             for (int p = p0; p < p1 && ok; ++p) {
                 {
-                    BD_ACC_BEGIN(tf);
                     ok = warp_all(wait_bar(smem_u32(&ctl->wfull[stage]), phase, abort_flag, 4));
-                    BD_ACC_END(w_full, tf);
-                    BD_ACC_BEGIN(tf2);
                     if (kDec && ok) ok = warp_all(wait_bar(smem_u32(&ctl->xfull[xslot]), xphase, abort_flag, 12));
-                    BD_ACC_END(w_afull, tf2);
                     if (!ok) break;
                 }
-                if (item == 0) BD_STAMP(4);
-                BD_TL(1);
                 const uint32_t wbase = w_addr + stage * a.w_stage_bytes;
                 const uint32_t xbase = x_addr + xslot * a.x_tile_bytes;
                 const uint64_t wdesc = desc0 + (wbase >> 4);
                 const uint64_t xdesc = desc0 + (xbase >> 4);
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
-                BD_ACC_BEGIN(tib);
-                if (!BD_KNOB(4) && elect_one()) {
+                if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t atom = kk >> 2, k16 = kk & 3;
@@ -961,24 +410,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         tc_commit(smem_u32(&ctl->xempty[xslot]));
                     }
                 }
-                if (kDec && BD_KNOB(4) && elect_one()) {
-                    tc_commit(smem_u32(&ctl->wempty[stage]));
-                    tc_commit(smem_u32(&ctl->xempty[xslot]));
-                }
                 __syncwarp();
-                BD_ACC_END(w_ib, tib);
                 if constexpr (kDec) {
                     // Delta MMAs are issued by the two delta-issuer warps.
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item, ar.step()) {
                         const uint32_t slot = (uint32_t)ar.idx;
-                        BD_ACC_BEGIN(tg);
                         ok = warp_all(wait_bar(smem_u32(&ctl->afull[slot]), ar.par, abort_flag, 5));
-                        BD_ACC_END(w_afull, tg);
                         if (!ok) break;
                         tc_fence_after();
-                        if (item == 0) BD_STAMP(5);
-                        BD_ACC_BEGIN(tid);
                         const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                         const uint32_t a_tmem = tmem_base + a.col_a + slot * (uint32_t)a.aslot_cols;
                         const uint64_t xwdesc = xdesc + (uint32_t)(j * a.win_rows) * 8u;   // 128 B per row
@@ -997,7 +437,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                             else tc_commit(smem_u32(&ctl->aempty[slot]));
                         }
                         __syncwarp();
-                        BD_ACC_END(w_id, tid);
                     }
                 }
                 if (!ok) break;
@@ -1018,9 +457,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             }
             __syncwarp();
             accphase ^= 1;
-            BD_STAMP(6);
         }
-        BD_ACC_STORE(16, w_full); BD_ACC_STORE(17, w_afull); BD_ACC_STORE(18, w_acc); BD_ACC_STORE(27, w_ib); BD_ACC_STORE(28, w_id);
     } else if (warp >= kWarpDelta0 && warp < kWarpDelta0 + 2) {
         // ------------------------------------------------- delta issuers (decode schedule)
         // Warp 2+g serves decode group g (tenants j = g, g+2, ... of the unit).  Per 128-k stage it
@@ -1037,7 +474,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             int xslot = 0;
             uint32_t xphase = 0, accphase = 0;
             bool ok = true;
-            BD_TL_DECL; BD_ACC_DECL(d_x8); BD_ACC_DECL(d_nb);
             while (ok && it.next(unit, p0, p1)) {
                 const Unit u = unit_info(a, unit);
                 ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
@@ -1046,11 +482,8 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 for (int p = p0; p < p1 && ok; ++p) {
                     // the stage's e5m2 pieces: written by the epilogue warps (few token rows per unit) or loaded
                     // from the pre-pass kernel's output
-                    BD_ACC_BEGIN(t8);
                     ok = warp_all(wait_bar(smem_u32(&ctl->x8full[xslot]), xphase, abort_flag, 12));
-                    BD_ACC_END(d_x8, t8);
                     if (!ok) break;
-                    if (g == 0) BD_TL(2);
                     const uint64_t x8desc = desc0 + ((x8_addr + xslot * a.x8_atom_bytes) >> 4);
                     const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this stage starts the accumulation
                     for (int half = 0; half < a.halves; ++half, ar.step()) {
@@ -1058,18 +491,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         if (*abort_flag) { ok = false; break; }
                         // The group's 128 decode threads arrive here once the buffer is filled (or when they
                         // give up after an abandoned wait, see the end of the decode role).
-                        BD_ACC_BEGIN(tn);
                         named_bar_sync(kBarAFull0 + g * 4 + (int)slot, 160);
-                        BD_ACC_END(d_nb, tn);
                         if (*abort_flag) { ok = false; break; }
                         tc_fence_after();
-                        if (g == 0) BD_TL(2);
                         const uint32_t a_buf = tmem_base + a.col_a + (uint32_t)(g * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         if (elect_one()) {
                             if (a.halves == 2) {
                                 // 64 k per hand-over: two K=32 steps per tenant, 16 operand columns each
                                 const uint32_t acc = (half > 0) ? 1u : first;
-                                for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
+                                for (int j = g; j < u.nten; j += 2) {
                                     const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                                     const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
                                     const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 16;
@@ -1078,7 +508,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                                 }
                             } else {
                                 // the whole 128-k stage: four K=32 steps per tenant, 32 operand columns each
-                                for (int j = g; j < (BD_KNOB(2) ? 0 : u.nten); j += 2) {
+                                for (int j = g; j < u.nten; j += 2) {
                                     const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                                     const uint64_t xj = x8desc + (uint32_t)j * ten_rows16;
                                     const uint32_t a_j = a_buf + (uint32_t)(j >> 1) * 32;
@@ -1102,7 +532,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 __syncwarp();
                 accphase ^= 1;
             }
-            if (g == 0) { BD_ACC_STORE(13, d_x8); BD_ACC_STORE(14, d_nb); }
         }
     } else if (warp >= kWarpDecode0 && warp < epi_first_warp) {
         // ------------------------------------------- sign decode -> tensor memory
@@ -1121,19 +550,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         const bool fast4 = kDec && a.TB == 4 && a.halves == 1 && a.a_slots == 2;
         const uint32_t aempty_g = smem_u32(&ctl->aempty[grp * kMaxASlots]);
         const uint32_t tbuf_g = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots) * (uint32_t)a.aslot_cols;
-        BD_ACC_DECL(w_bfull); BD_ACC_DECL(w_aempty); BD_ACC_DECL(w_work); BD_TL_DECL;
-#ifdef BD_TRACE
-        int tl_idx2 = 0;
-#endif
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             for (int p = p0; p < p1 && ok; ++p) {
                 if (p == p0 || !(p & 1)) {
-                    BD_ACC_BEGIN(tb);
                     ok = wait_bar(smem_u32(&ctl->bfull[bslot]), bphase, abort_flag, 6);
-                    BD_ACC_END(w_bfull, tb);
                     if (!ok) break;
-                    if (item == 0 && warp == kWarpDecode0) BD_STAMP(14);
                 }
                 const uint8_t* bsl = bits_ptr + bslot * a.bslot_bytes + (p & 1) * 16;
                 if constexpr (kDec) {
@@ -1152,13 +574,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         for (int i = 0; i < 4; ++i) wq[i] = *reinterpret_cast<const uint4*>(src + i * (2 * kTileN * 32));
 #pragma unroll
                         for (int half = 0; half < 2; ++half, ar.step()) {
-                            BD_ACC_BEGIN(tq);
                             ok = wait_bar(aempty_g + (uint32_t)ar.idx * 8, ar.par ^ 1, abort_flag, 7);
-                            BD_ACC_END(w_aempty, tq);
                             if (!ok) break;
                             tc_fence_after();
-                            if (warp == kWarpDecode0) BD_TL(3);
-                            BD_ACC_BEGIN(tw);
                             const uint32_t tbuf = tbuf_g + (uint32_t)ar.idx * (uint32_t)a.aslot_cols;
 #pragma unroll
                             for (int i = 0; i < 4; i += 2) {
@@ -1169,13 +587,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                                 decode_word_e5m2(half ? wq[i + 1].w : wq[i + 1].y, r + 24);
                                 tmem_st32(tbuf + (uint32_t)i * 16, r);
                             }
-                            if (warp == kWarpDecode0) BD_TL(3);
                             tc_wait_st();
-                            if (warp == kWarpDecode0) BD_TL(3);
                             tc_fence_before();
                             named_bar_arrive(kBarAFull0 + grp * 4 + ar.idx, 160);
-                            BD_ACC_END(w_work, tw);
-                            if (warp == kWarpDecode0) BD_TL(3);
                         }
                         item += 2;
                     } else if (fast4 && u.nten == 4) {
@@ -1185,12 +599,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         wq[0] = *reinterpret_cast<const uint4*>(src);
                         wq[1] = *reinterpret_cast<const uint4*>(src + 2 * kTileN * 32);
                         const uint32_t slot = (uint32_t)ar.idx;
-                        BD_ACC_BEGIN(tq);
                         ok = wait_bar(aempty_g + slot * 8, ar.par ^ 1, abort_flag, 7);
-                        BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
-                        BD_ACC_BEGIN(tw);
                         const uint32_t tbuf = tbuf_g + slot * (uint32_t)a.aslot_cols;
 #pragma unroll
                         for (int i = 0; i < 2; ++i) {
@@ -1204,19 +615,14 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         tc_wait_st();
                         tc_fence_before();
                         named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
-                        BD_ACC_END(w_work, tw);
                         item += 1;
                         ar.step();
                     } else
                     for (int half = 0; half < a.halves && ok; ++half, ++item, ar.step()) {
                         const uint32_t slot = (uint32_t)ar.idx;
-                        BD_ACC_BEGIN(tq);
                         ok = wait_bar(smem_u32(&ctl->aempty[grp * kMaxASlots + slot]), ar.par ^ 1, abort_flag, 7);
-                        BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
-                        if (warp == kWarpDecode0) BD_TL(3);
-                        BD_ACC_BEGIN(tw);
                         const uint32_t tbuf = lane_taddr + a.col_a + (uint32_t)(grp * a.a_slots + (int)slot) * (uint32_t)a.aslot_cols;
                         if (a.halves == 1) {
                             // whole stage: four sign words (128 k) per tenant, 32 operand columns each
@@ -1238,47 +644,28 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                                 const int j = grp + 2 * i;
                                 if (j < u.nten) w[i] = *reinterpret_cast<const uint2*>(bsl + (j * kTileN + row) * 32 + half * 8);
                             }
-#ifdef BD_TRACE
-                            if (warp == kWarpDecode0) { asm volatile("" :: "r"(w[0].x), "r"(w[1].x), "r"(w[2].x), "r"(w[3].x)); BD_TL2(6); }
-#endif
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int j = grp + 2 * i;
-#ifdef BD_TRACE
-                                if (warp == kWarpDecode0 && i > 0) BD_TL2(6);
-#endif
                                 if (j < u.nten) {
                                     uint32_t r[16];
-                                    if (BD_KNOB(1)) {
-#pragma unroll
-                                        for (int c = 0; c < 16; ++c) r[c] = w[i].x + c;
-                                    } else {
-                                        decode_word_e5m2(w[i].x, r);
-                                        decode_word_e5m2(w[i].y, r + 8);
-                                    }
-                                    if (!BD_KNOB(64)) tmem_st16(tbuf + (uint32_t)i * 16, r);
+                                    decode_word_e5m2(w[i].x, r);
+                                    decode_word_e5m2(w[i].y, r + 8);
+                                    tmem_st16(tbuf + (uint32_t)i * 16, r);
                                 }
                             }
                         }
-                        if (warp == kWarpDecode0) BD_TL(3);
                         tc_wait_st();
-                        if (warp == kWarpDecode0) BD_TL(3);
                         tc_fence_before();
                         named_bar_arrive(kBarAFull0 + grp * 4 + (int)slot, 160);
-                        BD_ACC_END(w_work, tw);
-                        if (warp == kWarpDecode0) BD_TL(3);
-                        if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
                 } else {
                     for (int j = 0; j < u.nten && ok; ++j, ++item, ar.step()) {
                         const uint4 w = *reinterpret_cast<const uint4*>(bsl + (j * kTileN + row) * 32);
                         const uint32_t slot = (uint32_t)ar.idx;
-                        BD_ACC_BEGIN(tq);
                         ok = wait_bar(smem_u32(&ctl->aempty[slot]), ar.par ^ 1, abort_flag, 7);
-                        BD_ACC_END(w_aempty, tq);
                         if (!ok) break;
                         tc_fence_after();
-                        BD_ACC_BEGIN(tw);
                         const uint32_t taddr = lane_taddr + a.col_a + slot * (uint32_t)a.aslot_cols;
                         uint32_t r[32];
                         decode_word(w.x, r, minus_one2);
@@ -1294,8 +681,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                             if (kPair && rank != 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctl->afull[slot]), 0));   // the leader's
                             else mbar_arrive(smem_u32(&ctl->afull[slot]));
                         }
-                        BD_ACC_END(w_work, tw);
-                        if (item == 0 && warp == kWarpDecode0) BD_STAMP(13);
                     }
                 }
                 if (!ok) break;
@@ -1313,8 +698,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             __syncwarp();
             for (int sl = 0; sl < a.a_slots; ++sl) named_bar_arrive(kBarAFull0 + grp * 4 + sl, 160);
         }
-        if (warp == kWarpDecode0) { BD_ACC_STORE(21, w_bfull); BD_ACC_STORE(22, w_aempty); BD_ACC_STORE(23, w_work); }
-        if (warp == kWarpDecode0 + 4) { BD_ACC_STORE(24, w_bfull); BD_ACC_STORE(25, w_aempty); BD_ACC_STORE(26, w_work); }
     } else if (warp >= epi_first_warp) {
         // ---------------------------------------------------------------- epilogue
         const int quad = warp & 3;
@@ -1326,7 +709,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
         uint32_t accphase = 0;
         bool ok = true;
-        BD_TL_DECL;
         // Decode schedule with few token rows per unit: these four warps, idle while a tile is being
         // accumulated, also split every stage's activations into e5m2 pieces (one 16-element task per
         // thread), as soon as the stage's activation tile has landed.  Each warp walks the items on its
@@ -1357,20 +739,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 if (elect_one()) {
                     if (ew == 0) {
                         const uint32_t bar = smem_u32(&ctl->xfull[sslot]);
-                        if (BD_KNOB(32)) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_arrive_expect_tx(bar, a.x_tile_bytes);
-                            tma_load_3d(x_addr + sslot * a.x_tile_bytes, &tmX, bar, 0, us.xrow0, si.p * (kPairK / kAtomK));
-                        }
+                        mbar_arrive_expect_tx(bar, a.x_tile_bytes);
+                        tma_load_3d(x_addr + sslot * a.x_tile_bytes, &tmX, bar, 0, us.xrow0, si.p * (kPairK / kAtomK));
                     } else {
                         const uint32_t bar = smem_u32(&ctl->x8full[s8slot]);
-                        if (BD_KNOB(32)) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
-                            tma_load_2d(x8_addr + s8slot * a.x8_atom_bytes, &tmX8, bar, si.p * kPairK, us.tenant0 * kPieces * am);
-                        }
+                        mbar_arrive_expect_tx(bar, a.x8_atom_bytes);
+                        tma_load_2d(x8_addr + s8slot * a.x8_atom_bytes, &tmX8, bar, si.p * kPairK, us.tenant0 * kPieces * am);
                     }
                 }
                 __syncwarp();
@@ -1429,7 +803,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
-            if (warp == epi_first_warp) { BD_STAMP(7); BD_TL(4); }
             grid_dependency_wait();   // Y and the workspace may still be in use by the previous kernel
             // this warp's arrival on the "accumulators drained" barrier (pair schedule: the leader's)
             auto release_acc = [&]() {
@@ -1473,7 +846,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 drain(std::false_type{});
             }
             if constexpr (kDec || kGrouped) release_acc();
-            if (warp == epi_first_warp) { BD_STAMP(8); BD_TL(4); }
             if (splitter) {
                 // the next tile's first stages, before the (slow) fix-up of this one
                 while (more_s && split_next(false)) {
@@ -1495,7 +867,6 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);
-                if (warp == epi_first_warp) { BD_STAMP(9); BD_TL(4); }
                 if (ctl->is_last) {
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
@@ -1511,14 +882,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (etid == 0) a.counters[kPair ? 2 * unit + (int)rank : unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
-                if (warp == epi_first_warp) { BD_STAMP(10); BD_TL(4); }
             }
         }
     }
 
     // ------------------------------------------------------------------ teardown
     __syncthreads();
-    if (warp == 0) BD_STAMP(11);
     if (*abort_flag) {
         // A wait was abandoned: give copies and MMAs still in flight a bounded time to land
         // before shared and tensor memory are released.
@@ -1534,19 +903,9 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     if (warp == kWarpTmem) {
         if constexpr (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
         else tmem_dealloc(tmem_base, kTmemCols);
-        BD_STAMP(12);
     }
-    BD_TRACE_FLUSH;
 }
 
-#ifdef BD_TRACE
-extern "C" int bitdelta_debug_set_trace(long long* buf) {
-    return (int)cudaMemcpyToSymbol(g_trace_ptr, &buf, sizeof(buf));
-}
-extern "C" int bitdelta_debug_set_knobs(int knobs) {
-    return (int)cudaMemcpyToSymbol(g_knobs, &knobs, sizeof(knobs));
-}
-#endif
 
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
@@ -1576,11 +935,7 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
-#ifdef BD_TRACE
-    cfg.dynamicSmemBytes = smem_bytes + 256 + 5 * BD_TLN * 8;   // room for the stamps behind the control block
-#else
     cfg.dynamicSmemBytes = smem_bytes;
-#endif
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     int nattr = 0;
@@ -1631,6 +986,20 @@ cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {
     if (out[0] != 0) {
         unsigned int zero[2] = {0, 0};
         e = cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero));
+        if (e != cudaSuccess) return e;
+    }
+    // the other translation units' copies of the status word (all are read, so that all are cleared);
+    // a time-out is reported in preference to a range flag
+    unsigned int other[2][2] = {{0, 0}, {0, 0}};
+    e = read_stream_status(other[0]);
+    if (e != cudaSuccess) return e;
+    e = read_simple_status(other[1]);
+    if (e != cudaSuccess) return e;
+    for (int i = 0; i < 2; ++i) {
+        if (other[i][0] != 0 && (out[0] == 0 || (out[0] != kStatusTimeout && other[i][0] == kStatusTimeout))) {
+            out[0] = other[i][0];
+            out[1] = other[i][1];
+        }
     }
     return e;
 }

@@ -21,11 +21,17 @@ struct GemmArgs {
     int T;             // work items (< 2^30)
     int q, r;          // T = q * grid + r
     int n_w, n_x, n_x8, n_bits, a_slots, halves;
+    int n_sets;          // streaming decode kernel: operand sets in tensor memory
+    int prefetch_steps;  // ... and how many 128-k steps beyond its rings it prefetches into L2 (0: none)
+    int early_weights;   // ... 1: its weight loads start before the grid dependency is resolved (0: experiments)
+    int early_gap_ns;    // ... and are then queued this many nanoseconds apart
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
     const float* alpha;
+    const void* X;       // [B*m, K] activations (16-bit values): the streaming decode kernel reads them with plain
+                         // loads; the other kernels use their tensor map
     void* Y;
     unsigned int* counters;
     float* partials;
@@ -41,6 +47,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = (p.pair ? p.grid / 2 : p.grid) / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
+    a.n_sets = p.n_sets; a.prefetch_steps = 0;
+    a.early_weights = 1; a.early_gap_ns = 2500;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;
@@ -93,6 +101,16 @@ inline uint8_t* ws_x8(const Plan& p, void* workspace) {
 cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const CUtensorMap& tmX8,
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream);
+
+// The streaming decode kernel (plan.stream): tensor maps for W_base and the sign words (args.X is read directly).
+cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes, bool early_start,
+                               cudaStream_t stream);
+// Thread blocks of the streaming kernel one multiprocessor of the current device holds at once (0: query failed).
+int stream_blocks_per_sm(uint32_t smem_bytes);
+// Status word of the streaming kernel's translation unit (read and cleared; the stream must be idle).
+cudaError_t read_stream_status(unsigned int out[2]);
+// ... and of the plain kernels' translation unit (the pre-pass activation split flags out-of-range values there).
+cudaError_t read_simple_status(unsigned int out[2]);
 
 // Number of CTA pairs (clusters of two) of the pair schedule's kernel that the current device can hold at once
 // with `smem_bytes` of dynamic shared memory each (0 if the query fails).

@@ -147,6 +147,10 @@ __device__ __forceinline__ uint8_t e5m2_round(float v) {
     return (uint8_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
 }
 
+// Status word of this translation unit: [0] = 9 (BITDELTA_ERR_RANGE) once the split has met a magnitude of
+// 2^16 or more (it is clamped to 65504, the largest binary16 number, exactly as the GEMM kernels' own split does).
+static __device__ unsigned int g_simple_status[2];
+
 __global__ void __launch_bounds__(128) x_split_kernel(const uint16_t* __restrict__ X, uint8_t* __restrict__ X8,
                                                       int m, int K, long long total_groups, int f16) {
     // Let the GEMM kernel queued behind this one start its weight prefetch right away.
@@ -159,6 +163,7 @@ __global__ void __launch_bounds__(128) x_split_kernel(const uint16_t* __restrict
     const int b = row / m, t = row - b * m;
     const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)row * K + g * 32);
     float y[32];
+    bool out_of_range = false;
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
         const uint4 v = __ldg(src + h);
@@ -167,7 +172,13 @@ __global__ void __launch_bounds__(128) x_split_kernel(const uint16_t* __restrict
         for (int i = 0; i < 4; ++i) {
             y[h * 8 + 2 * i] = io16_to_float((uint16_t)(q[i] & 0xFFFFu), f16);
             y[h * 8 + 2 * i + 1] = io16_to_float((uint16_t)(q[i] >> 16), f16);
+            if (!f16 && (((q[i] & 0x7FFFu) >= 0x4780u) || (((q[i] >> 16) & 0x7FFFu) >= 0x4780u))) out_of_range = true;
         }
+    }
+    if (out_of_range) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) y[i] = fminf(fmaxf(y[i], -65504.f), 65504.f);
+        atomicCAS(&g_simple_status[0], 0u, 9u);
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -187,6 +198,16 @@ __global__ void __launch_bounds__(128) x_split_kernel(const uint16_t* __restrict
         dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
         dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
+}
+
+cudaError_t read_simple_status(unsigned int out[2]) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_simple_status, sizeof(unsigned int) * 2);
+    if (e != cudaSuccess) return e;
+    if (out[0] != 0) {
+        unsigned int zero[2] = {0, 0};
+        e = cudaMemcpyToSymbol(g_simple_status, zero, sizeof(zero));
+    }
+    return e;
 }
 
 cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream) {

@@ -21,6 +21,14 @@ constexpr int kMaxCtas = 256;        // upper bound on the grid, sizes the works
 constexpr int kDecodeMaxM = 16;      // m <= 16: tenants are grouped into one tile
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kSmemCtrlBytes = 1024; // barriers, TMEM base, flags
+// Streaming decode schedule (few token rows per unit; see gemm_stream.cu)
+constexpr int kStreamSmemBudget = 113 * 1024;   // two thread blocks (of consecutive launches) per multiprocessor
+constexpr int kStreamSetCols = 128;             // one operand set in tensor memory: eight tenants x 64 k of e5m2 signs
+constexpr int kStreamMaxSets = 6;
+// Shared memory behind the control block.  The last tenant's delta window (N3 rows starting at row 4m(TB-1) of
+// the last piece tile) reaches up to round8(4m(TB-1) + N3) rows, i.e. whole 8-row swizzle atoms up to 2 KB past
+// the tile: the control block (1 KB) and this pad are what it reads there (ignored accumulator columns).
+constexpr int kStreamTailPad = 1024;
 
 struct Plan {
     int B, m, N, K;
@@ -49,6 +57,9 @@ struct Plan {
     int n_x;           // ring of bf16 activation tiles
     int n_x8;          // decode: ring of e5m2 piece tiles
     int n_bits;        // sign-word slots (each holds the signs of one k-pair of one unit)
+    int stream;        // decode with the in-kernel split: 1 = the streaming kernel (half a multiprocessor per block,
+                       // W_base in 64-k atoms, operand sets handed to one MMA issuer), 0 = the older decode kernel
+    int n_sets;        // streaming kernel: operand sets in tensor memory
     int pair;          // tiled schedule on CTA pairs: a unit is two W_base tiles (256 rows), one per CTA of a cluster of
                        // two; each CTA stages its own weights and half of the activation tile, the pair's leader issues
                        // 256-row MMAs (tcgen05 cta_group::2)
@@ -69,6 +80,12 @@ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 // The pair schedule is taken where it applies unless BITDELTA_PAIR=0 is set (experiments).
 inline bool pair_enabled() {
     const char* e = getenv("BITDELTA_PAIR");
+    return !(e && e[0] == '0');
+}
+
+// The streaming decode kernel is taken where it applies unless BITDELTA_STREAM=0 is set (experiments).
+inline bool stream_enabled() {
+    const char* e = getenv("BITDELTA_STREAM");
     return !(e && e[0] == '0');
 }
 
@@ -98,6 +115,11 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
+        p.stream = (p.convert && stream_enabled()) ? 1 : 0;
+        if (p.stream) {
+            p.x_rows = round_up(p.TB * m, 8);           // (the base MMA's N = 16 may read past it: ignored columns)
+            p.x8_rows = round_up(p.TB * kPieces * m, 8);   // (the last tenants' windows run past it: ignored columns)
+        }
     } else if (m <= 64 && B > 1 && tb_override != 1) {
         // Tiled schedule, middle regime (16 < m <= 64): a unit holds several tenants, whose tokens share one
         // W_base tile and one base MMA (N = all their tokens); every tenant keeps its own delta accumulator
@@ -181,7 +203,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
     p.w_stage_bytes = 2 * p.w_atom_bytes;
     p.x_tile_bytes = 2 * p.x_atom_bytes;
-    p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
+    p.bslot_bytes = (uint32_t)p.TB * kTileN * (p.stream ? 16 : 32);
     // Shared memory: rings of W_base tiles, of bf16 activation tiles and (decode) of e5m2 piece tiles, and
     // the sign-word slots.  W_base comes from DRAM (latency ~1.5 us under load); it and the bf16
     // activations are released as soon as the base MMAs have read them.  The piece tiles come from L2 (or
@@ -198,7 +220,22 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         if (p.n_bits < 2) p.n_bits = 2;
     }
     const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - p.n_bits * (int)p.bslot_bytes;
-    if (p.decode) {
+    if (p.stream) {
+        // Half a multiprocessor: two sign-word slots (128 k each), two activation and two piece tiles, and
+        // every remaining byte for W_base atoms (64 k, 16 KB each).
+        // Two slots of {activation tile, piece tile} (filled together by the splitter threads), two W_base
+        // stages (one 128-k tile each), and two or three sign-word slots.
+        p.n_x = 2;
+        p.n_x8 = 2;
+        p.n_w = 2;
+        const int fixed = 1024 + kSmemCtrlBytes + kStreamTailPad + p.n_w * (int)p.w_stage_bytes +
+                          p.n_x * (int)p.x_tile_bytes + p.n_x8 * (int)p.x8_atom_bytes;
+        p.n_bits = (kStreamSmemBudget - fixed) / (int)p.bslot_bytes;
+        if (p.n_bits < 2) p.n_bits = (kSmemBudget - fixed) / (int)p.bslot_bytes;   // (a whole multiprocessor per block then)
+        if (p.n_bits > 3) p.n_bits = 3;
+        if (p.n_bits < 2) return p;
+        if (p.n_w > kMaxStages) p.n_w = kMaxStages;
+    } else if (p.decode) {
         p.n_x8 = 3;
         p.n_x = (p.x_tile_bytes <= 4 * 1024) ? 3 : 2;
         p.n_w = (avail - p.n_x * (int)p.x_tile_bytes - p.n_x8 * (int)p.x8_atom_bytes) / (int)p.w_stage_bytes;
@@ -226,8 +263,13 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.n_w < 2) return p;
     p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
                    p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
-    // One CTA per SM is assumed by the TMEM allocation: keep the request above half an SM.
-    if (p.smem_bytes < 120 * 1024) p.smem_bytes = 120 * 1024;
+    if (p.stream) {
+        p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
+                       p.n_bits * p.bslot_bytes + kSmemCtrlBytes + kStreamTailPad;
+    } else if (p.smem_bytes < 120 * 1024) {
+        // One CTA per SM is assumed by this kernel's TMEM allocation: keep the request above half an SM.
+        p.smem_bytes = 120 * 1024;
+    }
 
     p.col_base = 0;
     p.col_delta = (uint32_t)p.Nb;
@@ -244,6 +286,13 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.decode) slots /= 2;                          // each of the two decode groups has its own ring
     p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
     if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
+    if (p.stream) {
+        p.halves = 2;
+        p.n_sets = free_cols / kStreamSetCols;
+        if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
+        if (p.n_sets < 2) return p;
+        p.a_slots = 2;
+    }
     if (p.a_slots < 2) return p;
 
     // Workspace: arrival counters, two partial-result slots per CTA, then (decode) the e5m2
