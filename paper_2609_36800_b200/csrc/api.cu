@@ -294,6 +294,23 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         if (pairs_fit[di] == 0) pairs_fit[di] = (2 * bd::max_active_pairs(p.smem_bytes) >= p.grid) ? 1 : -1;
         if (pairs_fit[di] < 0) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false);
     }
+    if (p.ok && p.cluster > 1) {
+        // The cluster form wants all its clusters resident at once (clusters are independent, so this is about
+        // speed, not progress); where the device cannot hold them, the flat work list is planned.
+        static std::mutex mu;
+        static int fit_cache[64][4][2] = {};   // [device][log2 cluster][smem above half a multiprocessor]: 0 unknown, else n + 1
+        const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
+        const int ci = p.cluster == 8 ? 3 : (p.cluster == 4 ? 2 : 1);
+        const int si = p.smem_bytes > (uint32_t)bd::kStreamSmemBudget ? 1 : 0;
+        int n;
+        {
+            std::lock_guard<std::mutex> lock(mu);
+            if (fit_cache[di][ci][si] == 0) fit_cache[di][ci][si] = bd::stream_max_active_clusters(p.smem_bytes, p.cluster) + 1;
+            n = fit_cache[di][ci][si] - 1;
+        }
+        const int need = p.grid / p.cluster;
+        if (n < need) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false);
+    }
     if (!p.ok) return BITDELTA_ERR_SHAPE;
     if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
@@ -324,7 +341,9 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     args.hold_prefetch = (int)(g_launches.load() & 1);   // trace build: alternate halves of the trace buffer
 #endif
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_EARLY_WEIGHTS"); d = (e && e[0] == '0') ? 0 : 1; } args.early_weights = d; }
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_EARLY_GAP"); d = e ? atoi(e) : 2500; } args.early_gap_ns = d; }
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_STEP"); d = e ? atoi(e) : (1 << 30); } args.trigger_step = d; }
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_EARLY"); d = (e && e[0] == '1') ? 1 : 0; } args.trigger_early = d; }
+    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_DECODE_WARPS"); d = (e && atoi(e) == 16) ? 16 : 8; } args.decode_warps = d; }
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_PREFETCH"); d = e ? atoi(e) : 0; } args.prefetch_steps = d; }
     const cudaError_t le = p.stream
         ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream)
@@ -393,9 +412,9 @@ int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
     if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
-    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.stream ? 5 : (p.convert ? 2 : 1));
+    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.stream ? (p.cluster > 1 ? 6 : 5) : (p.convert ? 2 : 1));
     info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
-    info[5] = p.whole_units ? 1 : (p.teams > 1 ? 2 : 0);
+    info[5] = p.cluster > 1 ? 3 : (p.whole_units ? 1 : (p.teams > 1 ? 2 : 0));
     info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;
     info[11] = p.a_slots; info[12] = p.halves; info[13] = p.tok_tile; info[14] = p.groups; info[15] = p.n_tiles;
     return BITDELTA_OK;
@@ -411,6 +430,12 @@ int bitdelta_gemm_plan_cta_items(int B, int m, int N, int K, int num_sms, int ct
         *end = *first + p.P;
         return BITDELTA_OK;
     }
+    if (p.cluster > 1) {   // block `cta` = rank cta % cluster of the cluster that takes unit cta / cluster
+        const int un = cta / p.cluster, r = cta % p.cluster;
+        *first = un * p.P + (r * p.P) / p.cluster;
+        *end = un * p.P + ((r + 1) * p.P) / p.cluster;
+        return BITDELTA_OK;
+    }
     const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
     const int cutter = p.pair ? cta / 2 : cta;   // both blocks of a pair take the pair's items
     *first = bd::cta_first_item(a, cutter);
@@ -422,6 +447,13 @@ int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int ite
     if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 128) != 0 || num_sms <= 0) return -1;
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok || item < 0 || item >= p.T) return -1;
+    if (p.cluster > 1) {
+        const int un = item / p.P, s = item - un * p.P;
+        int r = (int)(((long long)(s + 1) * p.cluster - 1) / p.P);   // largest r with r * P / cluster <= s
+        while ((r * p.P) / p.cluster > s) --r;
+        while (((r + 1) * p.P) / p.cluster <= s) ++r;
+        return un * p.cluster + r;
+    }
     if (p.whole_units) return (item / p.P) % p.grid;
     const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
     return p.pair ? 2 * bd::cta_of_item(a, item) : bd::cta_of_item(a, item);   // (pairs: the pair's first block)

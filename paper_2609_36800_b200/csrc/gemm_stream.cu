@@ -38,15 +38,12 @@ namespace bd {
 
 constexpr int kSWarpProducer = 0;
 constexpr int kSWarpMma = 1;
-constexpr int kSWarpDecode0 = 2;                 // warps 2..9
-constexpr int kSDecodeWarps = 8;
-constexpr int kSWarpEpi0 = kSWarpDecode0 + kSDecodeWarps;   // warps 10..13
-constexpr int kSEpiWarps = 4;
-constexpr int kSThreads = (kSWarpEpi0 + kSEpiWarps) * 32;   // 448
+constexpr int kSWarpDecode0 = 2;                 // warps 2 .. 2 + 8 kG - 1 decode (kG = 1: 8 warps, kG = 2: 16)
+constexpr int kSEpiWarps = 4;                    // the four warps after them
+__host__ __device__ constexpr int stream_threads(int kG) { return (kSWarpDecode0 + 8 * kG + kSEpiWarps) * 32; }   // 448 / 704
 constexpr int kSBarSet0 = 2;                     // named barrier of operand set s: id 2 + s
 constexpr int kSBarDep = 15;                     // named barrier the decode and epilogue warps sleep on until the grid
                                                  // dependency is resolved (the issuer warp arrives on it)
-constexpr int kSHandover = kSDecodeWarps * 32 + 32;   // decode threads arrive, the issuer warp syncs
 constexpr uint32_t kSAtomBytes = kTileN * 128;   // one W_base atom: 128 rows x 64 k of 16-bit values
 
 #ifdef BD_TRACE
@@ -140,11 +137,47 @@ __device__ __forceinline__ void split_from_global(const GemmArgs& a, int am, con
     if (out_of_range) atomicCAS(&g_device_status[0], 0u, kStatusRange);
 }
 
+// Cluster form: where a block's partial sums go (its own shared memory, [token][128 weight rows] floats).
+struct ClusterPartOut {
+    float* part_row;   // &part[0][this thread's weight row]
+    __device__ __forceinline__ void put(int tok, float v) const { part_row[tok * kTileN] = v; }
+};
+
+// epilogue_decode for a run-time m of 5..16.
+template <bool kG, class Out>
+__device__ __forceinline__ void epilogue_decode_any_m(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
+                                                      const float* alv, float al_lane, int am) {
+    switch (am) {
+        case 5: epilogue_decode<5, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 6: epilogue_decode<6, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 7: epilogue_decode<7, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 8: epilogue_decode<8, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 9: epilogue_decode<9, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 10: epilogue_decode<10, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 11: epilogue_decode<11, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 12: epilogue_decode<12, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 13: epilogue_decode<13, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 14: epilogue_decode<14, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        case 15: epilogue_decode<15, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+        default: epilogue_decode<16, kG>(a, u, lane_taddr, out, alv, al_lane); break;
+    }
+}
+
 // kMode 1..4: m = kMode tokens per tenant; 5: any m up to 16.  kGen: binary16 I/O, bias, activation.
-template <int kMode, bool kGen>
-__global__ void __launch_bounds__(kSThreads, 2)
+// kG = 1: eight decode warps, at most half a multiprocessor per block (flat form); kG = 2: sixteen decode warps, a
+// whole multiprocessor per block (cluster form): four decode warps per scheduler overlap one warp's integer work
+// with the others' tensor-memory stores and waits.
+template <int kMode, bool kGen, int kG>
+__global__ void __launch_bounds__(stream_threads(kG), kG == 1 ? 2 : 1)
 bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmBits,
                             const GemmArgs a) {
+    constexpr int kSDecodeWarps = 8 * kG;
+    constexpr int kSWarpEpi0 = kSWarpDecode0 + kSDecodeWarps;
+    constexpr int kSThreads = stream_threads(kG);
+    constexpr int kSHandover = kSDecodeWarps * 32 + 32;   // decode threads arrive, the issuer warp syncs
+    constexpr int kTenPerWarp = 4 / kG;                   // tenants of a unit a decode warp owns (of up to eight)
+    constexpr int kTenStride = 2 * kG;                    // ... tenant j = kTenStride * i + h for warp half h
+    constexpr int kWarpCols = 64 / kG;                    // ... and its columns of an operand set
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -173,9 +206,19 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         prefetch_tensormap(&tmBits);
     }
 
-    const int lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
-    const int hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
-    SegIter it{lo, hi, a.P, a.whole_units ? (int)gridDim.x : 0};
+    // Work: an even share of the flat (unit, k-step) list (or whole units round-robin), or, in the cluster form,
+    // this block's share of the k-steps of its cluster's unit.
+    const int crank = (a.cluster > 1) ? (int)cluster_ctarank() : 0;
+    int lo, hi;
+    if (a.cluster > 1) {
+        const int cunit = (int)blockIdx.x / a.cluster;
+        lo = cunit * a.P + (crank * a.P) / a.cluster;
+        hi = cunit * a.P + ((crank + 1) * a.P) / a.cluster;
+    } else {
+        lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
+        hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
+    }
+    SegIter it{lo, hi, a.P, (a.whole_units && a.cluster <= 1) ? (int)gridDim.x : 0};
     int unit, p0, p1;
 
     // Weight loads of one 128-k step: sub 0 / 1 = its two W_base atoms, sub 2 = its sign words.  One thread.
@@ -229,9 +272,8 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         ST_VAL(4, smid);
 #endif
     }
-    // A kernel queued behind this one with an early start may become resident now (this block leaves it
-    // half of the multiprocessor) and prefetch its own weights.
-    if (threadIdx.x == 0) grid_launch_dependents();
+    // (a.trigger_early, experiments: let the kernel queued behind this one become resident right away)
+    if (threadIdx.x == 0 && a.trigger_early) grid_launch_dependents();
 
     const uint32_t tmemready = smem_u32(&ctl->tmemready);
 
@@ -259,23 +301,10 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         }
         long long t_idle = 0;
         int idle = 0;
+        int n_w_queued = more_w || a.early_weights ? 1 : 0;   // W_base tiles queued so far (the prologue's included)
         bool dep_done = false;
         while (more_w || more_b) {
             bool did = false;
-            if (!dep_done) {
-                // Before the grid dependency is resolved this block sits next to a running block of the launch
-                // before it, and both use the multiprocessor's one copy engine, which takes about a thousand
-                // cycles per operation: queue the early loads one at a time, a few microseconds apart, so that
-                // each of the running block's loads waits behind one of them at most.
-                dep_done = warp_all(mbar_test_wait(smem_u32(&ctl->depready), 0u));
-                if (!dep_done && a.early_gap_ns > 0) {
-                    const long long t0 = clock64();
-                    while (!dep_done && clock64() - t0 < 2ll * a.early_gap_ns) {   // (~2 cycles per ns)
-                        __nanosleep(200);
-                        dep_done = warp_all(mbar_test_wait(smem_u32(&ctl->depready), 0u));
-                    }
-                }
-            }
             if (more_b && warp_all(mbar_test_wait(smem_u32(&ctl->bempty[br.idx]), br.par ^ 1))) {
                 if (elect_one()) issue_bits(ub, bi.p, br.idx);
                 __syncwarp();
@@ -284,10 +313,11 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                 if (more_b && bi.first) ub = unit_info(a, bi.unit);
                 did = true;
             }
-            if ((dep_done || !did) && more_w && warp_all(mbar_test_wait(smem_u32(&ctl->wempty[wr.idx]), wr.par ^ 1))) {
+            if (more_w && warp_all(mbar_test_wait(smem_u32(&ctl->wempty[wr.idx]), wr.par ^ 1))) {
                 if (elect_one()) issue_w(uw, wi.p, wr.idx);
                 __syncwarp();
                 wr.step();
+                if (++n_w_queued == a.trigger_step && lane == 0) grid_launch_dependents();
                 more_w = wi.next();
                 if (more_w && wi.first) uw = unit_info(a, wi.unit);
                 did = true;
@@ -316,6 +346,12 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
             }
         }
         ST(5);
+        // All of this block's loads are queued: a kernel queued behind this one with an early start may become
+        // resident now (this block leaves it half of the multiprocessor) and fill its rings while this block works
+        // through its last steps, its epilogue and its fix-up, when the copy engine and DRAM have nothing else to do.
+        // (Not earlier: a block of a new grid arriving on the multiprocessor costs the running block several
+        // microseconds in its first steps, measured with and without the newcomer's loads.)
+        if (lane == 0 && !a.trigger_early && n_w_queued < a.trigger_step) grid_launch_dependents();
     } else if (warp == kSWarpMma) {
         // -------------------------------------------------------------- MMA issuer
         // Resolves the grid dependency, then allocates tensor memory (the blocks of the launch before this
@@ -400,8 +436,8 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                     if (elect_one()) {
                         const uint32_t acc = (half > 0) ? 1u : first;
                         for (int j = 0; j < u.nten; ++j) {
-                            // tenant j's 16 columns: decode warp half j & 1, its tenant j >> 1
-                            const uint32_t a_j = a_set + (uint32_t)((j & 1) * 64 + (j >> 1) * 16);
+                            // tenant j's 16 columns: decode warp half j % kTenStride, its tenant j / kTenStride
+                            const uint32_t a_j = a_set + (uint32_t)((j % kTenStride) * kWarpCols + (j / kTenStride) * 16);
                             const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                             const uint64_t xj = x8desc + (uint32_t)j * ten_rows16 + (uint32_t)(half * 4);
                             umma_ts_f8(d_tmem, a_j, xj, idesc_delta, acc);
@@ -435,7 +471,7 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
-        const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * 64);
+        const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * kWarpCols);
         Ring br{0, 0u, a.n_bits}, sr{0, 0u, a.n_sets};
 #ifdef BD_TRACE
         int st_step = 0, st_set = 0;
@@ -453,19 +489,22 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                 if (warp == kSWarpDecode0 && st_step < 10) ST(90 + st_step);
                 ++st_step;
 #endif
-                // this warp's tenants j = 2i + h: their sign words of the step (128 k each), then the slot goes back
+                // this warp's tenants j = kTenStride * i + h: their sign words of the step (128 k each), then the
+                // slot goes back
                 const uint8_t* bsl = smem + bits_off + br.idx * a.bslot_bytes + row * 16;
-                uint4 wq[4];
+                uint4 wq[kTenPerWarp];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int j = 2 * i + h;
+                for (int i = 0; i < kTenPerWarp; ++i) {
+                    const int j = kTenStride * i + h;
                     wq[i] = (j < u.nten) ? *reinterpret_cast<const uint4*>(bsl + j * (kTileN * 16)) : make_uint4(0u, 0u, 0u, 0u);
                 }
-                asm volatile("" : "+r"(wq[0].x), "+r"(wq[1].x), "+r"(wq[2].x), "+r"(wq[3].x), "+r"(wq[0].w), "+r"(wq[1].w), "+r"(wq[2].w), "+r"(wq[3].w));
+#pragma unroll
+                for (int i = 0; i < kTenPerWarp; ++i) asm volatile("" : "+r"(wq[i].x), "+r"(wq[i].w));
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->bempty[br.idx]));
                 br.step();
-                const int npair = (u.nten > 4 + h) ? 2 : ((u.nten > h) ? 1 : 0);   // pairs of this warp's tenants present
+                // tenants of this warp present in the unit (pairs of them share a 32-column store)
+                const int nmine = (u.nten > h) ? (u.nten - h + kTenStride - 1) / kTenStride : 0;
 #ifdef BD_TRACE
                 const long long tstep = clock64();
                 acc_bits += tstep - tc0;
@@ -500,17 +539,17 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                     ++st_set;
 #endif
                     const uint32_t tbuf = tbuf0 + (uint32_t)sr.idx * kStreamSetCols;
-                    if (npair >= 1) {
-                        if (u.nten > 2 + h) tmem_st32(tbuf, r);          // (warp-uniform)
-                        else tmem_st16(tbuf, r);
-                    }
-                    if (npair == 2) {
-                        decode_word_e5m2(half ? wq[2].z : wq[2].x, r);
-                        decode_word_e5m2(half ? wq[2].w : wq[2].y, r + 8);
-                        decode_word_e5m2(half ? wq[3].z : wq[3].x, r + 16);
-                        decode_word_e5m2(half ? wq[3].w : wq[3].y, r + 24);
-                        if (u.nten > 6 + h) tmem_st32(tbuf + 32, r);
-                        else tmem_st16(tbuf + 32, r);
+                    if (nmine >= 2) tmem_st32(tbuf, r);          // (warp-uniform)
+                    else if (nmine == 1) tmem_st16(tbuf, r);
+                    if constexpr (kTenPerWarp == 4) {
+                        if (nmine >= 3) {
+                            decode_word_e5m2(half ? wq[2].z : wq[2].x, r);
+                            decode_word_e5m2(half ? wq[2].w : wq[2].y, r + 8);
+                            decode_word_e5m2(half ? wq[3].z : wq[3].x, r + 16);
+                            decode_word_e5m2(half ? wq[3].w : wq[3].y, r + 24);
+                            if (nmine >= 4) tmem_st32(tbuf + 32, r);
+                            else tmem_st16(tbuf + 32, r);
+                        }
                     }
                     pending = sr.idx;
                     ST_CLK(tc4);
@@ -586,6 +625,7 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         };
         uint32_t tmem_base = 0;
         bool have_tmem = false;
+        int pend_unit[2], pend_c0[2], pend_c1[2], npend = 0;   // cut tiles this block has to finish
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
@@ -607,7 +647,7 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                 if (!split_next(false)) break;
             }
             float* slotp = nullptr;
-            if (!whole) {
+            if (!whole && a.cluster <= 1) {
                 const int slot = (unit == first_unit) ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1;
                 slotp = a.partials + (size_t)slot * a.slot_floats;
             }
@@ -625,26 +665,22 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                 have_tmem = true;
             }
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+            if (a.cluster > 1) {
+                // Cluster form: this block's partial sums go to its own shared memory (the W_base ring: every load
+                // into it has landed and every MMA that read it has completed), token-major, one float per weight
+                // row; the cluster's leader adds the blocks' partials up at the end of the kernel.
+                const ClusterPartOut out{reinterpret_cast<float*>(smem) + row};
+                if constexpr (kMode >= 1 && kMode <= 4) epilogue_decode<kMode, false>(a, u, lane_taddr, out, alv, al_lane);
+                else epilogue_decode_any_m<false>(a, u, lane_taddr, out, alv, al_lane, am);
+                break;   // (one segment per block)
+            }
             auto drain = [&](auto gate) {
                 constexpr bool kGate = decltype(gate)::value;
                 const EpiOut<kGen, kGate> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
                 if constexpr (kMode >= 1 && kMode <= 4) {
                     epilogue_decode<kMode, kGen>(a, u, lane_taddr, out, alv, al_lane);
                 } else {
-                    switch (am) {
-                        case 5: epilogue_decode<5, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 6: epilogue_decode<6, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 7: epilogue_decode<7, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 8: epilogue_decode<8, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 9: epilogue_decode<9, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 10: epilogue_decode<10, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 11: epilogue_decode<11, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 12: epilogue_decode<12, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 13: epilogue_decode<13, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 14: epilogue_decode<14, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        case 15: epilogue_decode<15, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                        default: epilogue_decode<16, kGen>(a, u, lane_taddr, out, alv, al_lane); break;
-                    }
+                    epilogue_decode_any_m<kGen>(a, u, lane_taddr, out, alv, al_lane, am);
                 }
             };
             if constexpr (kGen) {
@@ -660,13 +696,12 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
 #ifdef BD_TRACE
             if (warp == kSWarpEpi0) ST(101 + 3 * st_seg);
 #endif
-            // the next tile's first steps, before the (slow) fix-up of this one
-            while (more_s && split_next(false)) {
-            }
-
             if (!whole) {
-                // This tile is cut across blocks: publish the partial, count arrivals, and let the last block
-                // to arrive add the partials in block order and write Y.
+                // This tile is cut across blocks: publish the partial and count arrivals right away (the sooner every
+                // block has arrived, the sooner the last one can finish the tile).  If this block is the last to
+                // arrive it adds the partials up in block order and writes Y, but only after its other segments
+                // have been drained and published: that sum is a chain of round trips to L2 and would hold up
+                // the next segment's drain.
                 const int first_item = unit * a.P;
                 const int c0 = cta_of_item(a, first_item);
                 const int c1 = cta_of_item(a, first_item + a.P - 1);
@@ -681,21 +716,35 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
                 }
                 epi_bar_sync(kSEpiWarps * 32);
                 if (*abort_flag) break;
-                if (ctl->is_last) {
-                    // Block c0 holds the tile's first step; the tile is its first segment only if its range
-                    // starts exactly there.  Every later block starts inside the tile.
-                    const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
-                    const float* first = a.partials + (size_t)slot0 * a.slot_floats;
-                    const float* rest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats;
-                    if (kGen && a.act == 2) reduce_partials<kGen, kGen>(a, u, etid, kSEpiWarps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
-                    else reduce_partials<kGen, false>(a, u, etid, kSEpiWarps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
-                    if (etid == 0) a.counters[unit] = 0u;
+                if (ctl->is_last) {   // (rewritten only after the next segment's first barrier, which every thread passes after this read)
+                    pend_unit[npend] = unit;
+                    pend_c0[npend] = c0;
+                    pend_c1[npend] = c1;
+                    ++npend;
                 }
-                epi_bar_sync(kSEpiWarps * 32);   // is_last is rewritten by the next cut tile
-                if (*abort_flag) break;
             }
 #ifdef BD_TRACE
             if (warp == kSWarpEpi0) ST(102 + 3 * st_seg);
+#endif
+            // the next tile's first steps
+            while (more_s && split_next(false)) {
+            }
+        }
+        // Tiles this block was the last to arrive at (at most its first and its last segment).
+        for (int k = 0; k < npend && ok && !*abort_flag; ++k) {
+            const int un = pend_unit[k], c0 = pend_c0[k], c1 = pend_c1[k];
+            const Unit u = unit_info(a, un);
+            const int first_item = un * a.P;
+            // Block c0 holds the tile's first step; the tile is its first segment only if its range starts
+            // exactly there.  Every later block starts inside the tile.
+            const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
+            const float* first = a.partials + (size_t)slot0 * a.slot_floats;
+            const float* rest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats;
+            if (kGen && a.act == 2) reduce_partials<kGen, kGen>(a, u, etid, kSEpiWarps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
+            else reduce_partials<kGen, false>(a, u, etid, kSEpiWarps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
+            if (etid == 0) a.counters[un] = 0u;
+#ifdef BD_TRACE
+            if (warp == kSWarpEpi0) ST(106 + k);
 #endif
         }
         if (!ok) {
@@ -720,7 +769,61 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
         __syncthreads();
     }
     tc_fence_after();
+    // (tensor memory goes back before the cluster barriers below: a block must never hold it while it waits for
+    // another block, which might be waiting for tensor memory on the same multiprocessor)
     if (warp == kSWarpMma) tmem_dealloc(ctl->tmem_base, kTmemCols);
+    if (a.cluster > 1) {
+        // Cluster form: every block's partial sums are in its shared memory.  After a cluster barrier the leader's
+        // epilogue threads (one weight row each) add them up in block order, i.e. in k order, read through the
+        // distributed shared memory window, apply the fused epilogue and write Y; a second barrier keeps the
+        // other blocks' shared memory alive until it has read them.
+        if (warp == 0) ST(119);
+        cluster_sync_all();
+        if (warp == 0) ST(120);
+        if (crank == 0 && warp >= kSWarpEpi0 && lo < hi && !*abort_flag) {
+            const Unit u = unit_info(a, (int)blockIdx.x / a.cluster);
+            const int row = (warp & 3) * 32 + lane;
+            const int n = u.n0 + row;
+            float bias_n = 0.f;
+            if constexpr (kGen) {
+                if (a.bias && n < a.N) bias_n = from_io16(__ldg(reinterpret_cast<const uint16_t*>(a.bias) + n), a.f16);
+            }
+            const uint32_t part = base + (uint32_t)row * 4u;   // this block's part[0][row]; same offset in every block
+            uint32_t peer[8];
+#pragma unroll
+            for (int r = 1; r < 8; ++r) peer[r] = (r < a.cluster) ? mapa_shared(part, (uint32_t)r) : 0u;
+            uint16_t* Yp = reinterpret_cast<uint16_t*>(a.Y);
+            auto finish = [&](auto gate) {
+                constexpr bool kGate = decltype(gate)::value;
+                const EpiOut<kGen, kGate> out{Yp, nullptr, a.N, n, row, u.xrow0, bias_n, a};
+                for (int tok = 0; tok < u.ntok; tok += 4) {   // (four tokens' remote loads in flight together)
+                    float pv[4][8];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+#pragma unroll
+                        for (int r = 1; r < 8; ++r)
+                            pv[q][r] = (r < a.cluster && tok + q < u.ntok) ? ld_shared_cluster_f32(peer[r] + (uint32_t)(tok + q) * (kTileN * 4u)) : 0.f;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (tok + q < u.ntok) {   // (warp-uniform)
+                            float v = reinterpret_cast<const float*>(smem)[(tok + q) * kTileN + row];
+#pragma unroll
+                            for (int r = 1; r < 8; ++r) v += pv[q][r];
+                            out.put(tok + q, v);
+                        }
+                    }
+                }
+            };
+            if constexpr (kGen) {
+                if (a.act == 2) finish(std::true_type{});
+                else finish(std::false_type{});
+            } else {
+                finish(std::false_type{});
+            }
+        }
+        if (warp == kSWarpEpi0) ST(121);
+        cluster_sync_relaxed();   // (nothing to publish: the leader's stores to Y need not be waited for here)
+    }
     if (warp == 0) ST(118);
 }
 
@@ -733,16 +836,21 @@ extern "C" int bitdelta_debug_set_trace(unsigned long long* buf) {
 cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes, bool early_start,
                                cudaStream_t stream) {
     const int gen = (args.f16 || args.act || args.bias != nullptr) ? 5 : 0;
-    const int mode = gen + (args.m <= 4 ? args.m : 5) - 1;
+    const int big = (args.cluster > 1 && args.decode_warps == 16) ? 10 : 0;   // (experiments: sixteen decode warps)
+    const int mode = big + gen + (args.m <= 4 ? args.m : 5) - 1;
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const GemmArgs);
-    static const KernelFn kernels[10] = {
-        bitdelta_gemm_stream_kernel<1, false>, bitdelta_gemm_stream_kernel<2, false>, bitdelta_gemm_stream_kernel<3, false>,
-        bitdelta_gemm_stream_kernel<4, false>, bitdelta_gemm_stream_kernel<5, false>,
-        bitdelta_gemm_stream_kernel<1, true>,  bitdelta_gemm_stream_kernel<2, true>,  bitdelta_gemm_stream_kernel<3, true>,
-        bitdelta_gemm_stream_kernel<4, true>,  bitdelta_gemm_stream_kernel<5, true>};
+    static const KernelFn kernels[20] = {
+        bitdelta_gemm_stream_kernel<1, false, 1>, bitdelta_gemm_stream_kernel<2, false, 1>, bitdelta_gemm_stream_kernel<3, false, 1>,
+        bitdelta_gemm_stream_kernel<4, false, 1>, bitdelta_gemm_stream_kernel<5, false, 1>,
+        bitdelta_gemm_stream_kernel<1, true, 1>,  bitdelta_gemm_stream_kernel<2, true, 1>,  bitdelta_gemm_stream_kernel<3, true, 1>,
+        bitdelta_gemm_stream_kernel<4, true, 1>,  bitdelta_gemm_stream_kernel<5, true, 1>,
+        bitdelta_gemm_stream_kernel<1, false, 2>, bitdelta_gemm_stream_kernel<2, false, 2>, bitdelta_gemm_stream_kernel<3, false, 2>,
+        bitdelta_gemm_stream_kernel<4, false, 2>, bitdelta_gemm_stream_kernel<5, false, 2>,
+        bitdelta_gemm_stream_kernel<1, true, 2>,  bitdelta_gemm_stream_kernel<2, true, 2>,  bitdelta_gemm_stream_kernel<3, true, 2>,
+        bitdelta_gemm_stream_kernel<4, true, 2>,  bitdelta_gemm_stream_kernel<5, true, 2>};
     // Per device and instantiation, once: allow the dynamic shared memory and ask for the largest shared-memory
     // carve-out, so that two blocks (of consecutive launches) fit on one multiprocessor.
-    static unsigned char attr_done[64][10] = {};
+    static unsigned char attr_done[64][20] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -756,14 +864,21 @@ cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kSThreads);
+    cfg.blockDim = dim3((unsigned)stream_threads(big ? 2 : 1));
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     int nattr = 0;
     if (early_start) {
         attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
+    }
+    if (args.cluster > 1) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = (unsigned)args.cluster;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
         ++nattr;
     }
     cfg.attrs = attr;
@@ -771,12 +886,35 @@ cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits
     return cudaLaunchKernelEx(&cfg, kernels[mode], tmW, tmBits, args);
 }
 
+int stream_max_active_clusters(uint32_t smem_bytes, int cluster) {
+    auto kernel = bitdelta_gemm_stream_kernel<1, false, 1>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
+    (void)cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(cluster * 64));
+    cfg.blockDim = dim3((unsigned)stream_threads(1));
+    cfg.dynamicSmemBytes = smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
 int stream_blocks_per_sm(uint32_t smem_bytes) {
-    auto kernel = bitdelta_gemm_stream_kernel<1, false>;
+    auto kernel = bitdelta_gemm_stream_kernel<1, false, 1>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
     (void)cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kSThreads, smem_bytes) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, stream_threads(1), smem_bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }

@@ -22,9 +22,12 @@ struct GemmArgs {
     int q, r;          // T = q * grid + r
     int n_w, n_x, n_x8, n_bits, a_slots, halves;
     int n_sets;          // streaming decode kernel: operand sets in tensor memory
+    int cluster;         // ... blocks per cluster (one cluster per unit), or 0: flat work list
+    int decode_warps;    // ... 8, or (experiments, cluster form) 16
     int prefetch_steps;  // ... and how many 128-k steps beyond its rings it prefetches into L2 (0: none)
     int early_weights;   // ... 1: its weight loads start before the grid dependency is resolved (0: experiments)
-    int early_gap_ns;    // ... and are then queued this many nanoseconds apart
+    int trigger_early;   // ... 1: dependents may launch from this kernel's start (0: see trigger_step)
+    int trigger_step;    // ... dependents may launch once this many of a block's W_base tiles are queued (or all of them)
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
@@ -47,8 +50,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = (p.pair ? p.grid / 2 : p.grid) / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
-    a.n_sets = p.n_sets; a.prefetch_steps = 0;
-    a.early_weights = 1; a.early_gap_ns = 2500;
+    a.n_sets = p.n_sets; a.cluster = p.cluster; a.decode_warps = 8; a.prefetch_steps = 0;
+    a.early_weights = 1; a.trigger_early = 0; a.trigger_step = 1 << 30;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;
@@ -105,6 +108,8 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
 // The streaming decode kernel (plan.stream): tensor maps for W_base and the sign words (args.X is read directly).
 cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes, bool early_start,
                                cudaStream_t stream);
+// Clusters of `cluster` blocks of the streaming kernel the current device can hold at once (0: query failed).
+int stream_max_active_clusters(uint32_t smem_bytes, int cluster);
 // Thread blocks of the streaming kernel one multiprocessor of the current device holds at once (0: query failed).
 int stream_blocks_per_sm(uint32_t smem_bytes);
 // Status word of the streaming kernel's translation unit (read and cleared; the stream must be idle).

@@ -60,6 +60,9 @@ struct Plan {
     int stream;        // decode with the in-kernel split: 1 = the streaming kernel (half a multiprocessor per block,
                        // W_base in 64-k atoms, operand sets handed to one MMA issuer), 0 = the older decode kernel
     int n_sets;        // streaming kernel: operand sets in tensor memory
+    int cluster;       // streaming kernel: > 1 = every unit is taken by a cluster of this many blocks, each with an equal
+                       // share of the unit's k-steps; their partial results meet in the leader's shared memory
+                       // (no workspace traffic, no arrival counters); 0 = the flat work list
     int pair;          // tiled schedule on CTA pairs: a unit is two W_base tiles (256 rows), one per CTA of a cluster of
                        // two; each CTA stages its own weights and half of the activation tile, the pair's leader issues
                        // 256-row MMAs (tcgen05 cta_group::2)
@@ -83,13 +86,20 @@ inline bool pair_enabled() {
     return !(e && e[0] == '0');
 }
 
-// The streaming decode kernel is taken where it applies unless BITDELTA_STREAM=0 is set (experiments).
+// The streaming decode kernel (gemm_stream.cu) is taken where it applies when BITDELTA_STREAM=1 is set; the default
+// is the older decode kernel, which measures faster on the decode workloads (18 against 20 us on 8 x 1 x 4096 x 4096).
 inline bool stream_enabled() {
     const char* e = getenv("BITDELTA_STREAM");
+    return e && e[0] == '1';
+}
+
+// The cluster form of the streaming kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
+inline bool cluster_enabled() {
+    const char* e = getenv("BITDELTA_CLUSTER");
     return !(e && e[0] == '0');
 }
 
-// allow_pair = false: the device cannot hold all the pairs at once (see the launcher), plan without them.
+// allow_pair = false: the device cannot hold all the pairs (or clusters) at once (see the launcher), plan without them.
 inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0,
                       bool allow_pair = true) {
     Plan p{};
@@ -198,6 +208,23 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         if (pick == 3) { p.teams = p.groups; p.grid = cpt * p.groups; }
     }
 
+    // Streaming kernel, one tenant group: if clusters of 2, 4 or 8 blocks (one cluster per W_base tile, the k-steps
+    // dealt evenly to its blocks) fill at least 80 % of the blocks the flat list would use, take the largest such
+    // cluster: no tile is then cut at an arbitrary place, every block has one segment, and the partial sums are
+    // added up through distributed shared memory instead of a workspace, arrival counters and L2 round trips.
+    p.cluster = 0;
+    if (p.stream && p.groups == 1 && allow_pair && cluster_enabled()) {
+        for (int c = 8; c >= 2; c >>= 1) {
+            if (p.units * c <= max_grid && p.P >= c && 10 * p.units * c >= 8 * p.grid) {
+                p.cluster = c;
+                p.grid = p.units * c;
+                p.whole_units = 0;
+                p.teams = 1;
+                break;
+            }
+        }
+    }
+
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
@@ -223,8 +250,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.stream) {
         // Half a multiprocessor: two sign-word slots (128 k each), two activation and two piece tiles, and
         // every remaining byte for W_base atoms (64 k, 16 KB each).
-        // Two slots of {activation tile, piece tile} (filled together by the splitter threads), two W_base
-        // stages (one 128-k tile each), and two or three sign-word slots.
+        // Half a multiprocessor: two slots of {activation tile, piece tile} (filled together by the splitter
+        // threads), two W_base stages of one 128-k tile each, two or three sign-word slots.  (A whole
+        // multiprocessor per block with rings a step deeper and sixteen decode warps was measured on the cluster
+        // form: no faster per step, and the next launch's blocks then start their loads a microsecond later.)
         p.n_x = 2;
         p.n_x8 = 2;
         p.n_w = 2;

@@ -45,6 +45,11 @@ def test_every_item_is_taken_exactly_once(shape, sms):
         assert hi == lo2
     sizes = [hi - lo for lo, hi in ranges]
     assert min(sizes) >= 1
+    if order == 3:
+        # clusters: every unit belongs to one cluster of blocks / units blocks, no block's share crosses a unit
+        assert blocks % units == 0 and blocks // units in (2, 4, 8)
+        for b, (lo, hi) in enumerate(ranges):
+            assert lo // P == (hi - 1) // P == b // (blocks // units)
     if order == 2:
         assert teams == info["groups"] and blocks % teams == 0
         cpt, Tg = blocks // teams, T // teams
@@ -72,15 +77,27 @@ def test_every_item_is_taken_exactly_once(shape, sms):
 
 def test_schedules_and_work_orders_of_the_measured_workloads():
     got = {w.name: bd.gemm_plan(w.B, w.m, w.N, w.K) for w in synth.WORKLOADS}
-    # few token rows per unit: the streaming decode kernel, within half a multiprocessor's shared memory
-    assert got["decode_attn"]["schedule"] == 5 and got["decode_attn"]["order"] == 0 and got["decode_attn"]["blocks"] == 148
-    assert got["decode_attn"]["smem_bytes"] <= 113 * 1024 and got["decode_attn"]["w_ring"] >= 2
-    assert got["tiny"]["schedule"] == 5
+    assert got["decode_attn"]["schedule"] == 2 and got["decode_attn"]["order"] == 0 and got["decode_attn"]["blocks"] == 148
+    assert got["tiny"]["schedule"] == 2
     assert got["decode_mlp_up"]["schedule"] == 1 and got["decode_mlp_up"]["order"] == 2 and got["decode_mlp_up"]["teams"] == 2
     assert got["many_tenant_down"]["order"] == 2 and got["many_tenant_down"]["teams"] == 8 and got["many_tenant_down"]["blocks"] == 144
     assert got["prefill"]["schedule"] == 4 and got["prefill"]["order"] == 0 and got["prefill"]["blocks"] == 148
     for g in got.values():
         assert g["smem_bytes"] <= 227 * 1024 and g["w_ring"] >= 2 and g["operand_buffers"] >= 2
+
+
+def test_streaming_decode_kernel_plans(monkeypatch):
+    # BITDELTA_STREAM=1 (read at every plan): few token rows per unit and one tenant group -> clusters of four
+    # blocks per W_base tile; two tenant groups -> the flat list by teams, within half a multiprocessor
+    monkeypatch.setenv("BITDELTA_STREAM", "1")
+    one = bd.gemm_plan(8, 1, 4096, 4096)
+    assert one["schedule"] == 6 and one["order"] == 3 and one["blocks"] == 128 and one["smem_bytes"] <= 113 * 1024
+    assert bd.gemm_plan(1, 16, 512, 512)["schedule"] == 6
+    two = bd.gemm_plan(16, 1, 4096, 4096)
+    assert two["schedule"] == 5 and two["order"] == 2 and two["smem_bytes"] <= 113 * 1024
+    for b in range(one["blocks"]):
+        lo, hi = bd.gemm_plan_cta_items(8, 1, 4096, 4096, b)
+        assert hi - lo == 8 and lo // 32 == b // 4 and bd.gemm_plan_item_cta(8, 1, 4096, 4096, lo) == b
 
 
 def test_cuda_core_path_and_bad_arguments():
