@@ -43,7 +43,9 @@ typedef enum {
     BITDELTA_ERR_ARCH = 5,      /* current device is not compute capability 10.0      */
     BITDELTA_ERR_CUDA = 6,      /* a CUDA runtime / driver call failed                */
     BITDELTA_ERR_TIMEOUT = 7,   /* a bounded wait inside a kernel expired             */
-    BITDELTA_ERR_OPTION = 8     /* unknown data type or activation code               */
+    BITDELTA_ERR_OPTION = 8,    /* unknown data type or activation code               */
+    BITDELTA_ERR_RANGE = 9      /* an activation beyond the decode schedules' range (reported by
+                                   bitdelta_last_device_status, see bitdelta_gemm)    */
 } bitdelta_status;
 
 /*
@@ -106,6 +108,17 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.
  * Asynchronous on the stream; a kernel-side wait that expires is reported by
  * bitdelta_last_device_status, not here.
+ * Range of X in the decode schedules (m <= 16): there the delta term runs on the
+ * 8-bit float tensor path, with every activation rewritten exactly as a sum of
+ * e5m2 numbers, which have binary16's exponent range.  Finite bf16 activations
+ * with |x| < 2^16 are exact down to 2^-16 (smaller parts of x, at most 2^-16 per
+ * element, are dropped from the DELTA term only; the base term always uses the
+ * bf16 value).  An activation with |x| >= 2^16 (or an infinity / NaN) is clamped
+ * to +-65504 in the delta term, in every decode schedule alike, and the call is
+ * flagged: bitdelta_last_device_status then returns BITDELTA_ERR_RANGE.  Inputs
+ * like that need bitdelta_gemm_ex with BITDELTA_DTYPE_WIDE_RANGE, which runs any
+ * m on the tiled schedule (bf16 operands for both terms: exact for every finite
+ * input).  The tiled schedules (m > 16) have no such limit.
  * Early start: the kernel is queued so that it may begin (prologue, prefetch of
  * W_base, bits and alpha) while the kernel queued on the stream just before it
  * is still running; it reads X and writes Y and the workspace only after that
@@ -126,7 +139,8 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
  *   Y[b,t,n] = act( sum_k X[b,t,k] W_base[n,k] + alpha[b] sum_k X[b,t,k] S[b,n,k] + bias[n] )
  *
  * dtype : BITDELTA_DTYPE_BF16 or BITDELTA_DTYPE_F16 (IEEE binary16): the element type of X, W_base,
- *         bias and Y.  Accumulation is fp32 in both; Y is rounded to nearest even once, after the
+ *         bias and Y; optionally OR-ed with BITDELTA_DTYPE_WIDE_RANGE, which plans every m on the tiled
+ *         schedule (no 8-bit float operands: see the range note of bitdelta_gemm; slower for m <= 16).  Accumulation is fp32 in both; Y is rounded to nearest even once, after the
  *         epilogue.  With binary16 the delta term is exact for operands in the normal range (values
  *         below 2^-14 lose bits below 2^-16, in the delta term only).
  * bias  : device, [N] values of `dtype`, shared by all tenants, or NULL for none.  2-byte aligned.  Like
@@ -143,7 +157,7 @@ int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const
  * bitdelta_gemm, which is this call with BITDELTA_DTYPE_BF16, no bias and no activation.  Unknown
  * codes return BITDELTA_ERR_OPTION and launch nothing.
  */
-enum { BITDELTA_DTYPE_BF16 = 0, BITDELTA_DTYPE_F16 = 1 };
+enum { BITDELTA_DTYPE_BF16 = 0, BITDELTA_DTYPE_F16 = 1, BITDELTA_DTYPE_WIDE_RANGE = 0x100 };
 enum { BITDELTA_ACT_NONE = 0, BITDELTA_ACT_SILU = 1, BITDELTA_ACT_SILU_GATE = 2 };
 int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
                      const void* bias, void* Y, int B, int m, int N, int K, int dtype, int act,
@@ -231,10 +245,13 @@ int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int ite
 
 /*
  * Synchronises the stream, then returns and clears the device-side status of
- * the current device: BITDELTA_OK, or BITDELTA_ERR_TIMEOUT if a bounded wait in
+ * the current device: BITDELTA_OK; BITDELTA_ERR_TIMEOUT if a bounded wait in
  * one of this library's kernels expired since the last query (its output is
- * then undefined).  `site`, if not NULL (host pointer), receives a code naming
- * the wait that expired.
+ * then undefined, and a workspace it used must be prepared again with
+ * bitdelta_workspace_init: arrival counters may have been left non-zero); or
+ * BITDELTA_ERR_RANGE if a decode-schedule call met an activation of magnitude
+ * 2^16 or more (see bitdelta_gemm; a time-out takes precedence).  `site`, if not
+ * NULL (host pointer), receives a code naming the wait that expired.
  */
 int bitdelta_last_device_status(void* cuda_stream, int* site);
 

@@ -8,6 +8,8 @@ missing.
 """
 from . import synth  # noqa: F401
 from .binding import (  # noqa: F401
+    STATUS_RANGE,
+    STATUS_TIMEOUT,
     BitDeltaError,
     compress,
     gemm,

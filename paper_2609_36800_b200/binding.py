@@ -16,6 +16,8 @@ _lib = None
 
 STATUS_OK = 0
 STATUS_TIMEOUT = 7
+STATUS_RANGE = 9
+DTYPE_WIDE_RANGE = 0x100
 
 EXPORTS = (
     "bitdelta_pack", "bitdelta_unpack", "bitdelta_compress_workspace_bytes", "bitdelta_compress",
@@ -155,11 +157,13 @@ ACTS = {"none": 0, "silu": 1, "silu_gate": 2}
 
 
 def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bool = False, bias=None,
-         act: str = "none"):
+         act: str = "none", wide_range: bool = False):
     """Y[b,t,n] = act(sum_k X W_base + alpha[b] sum_k X S + bias[n]).  X [B,m,K] and W_base [N,K] in bf16 or
     (both) fp16, bits int32 storage [B,N,K/32], alpha fp32 [B], optional bias [N] of X's type, act "none", "silu"
     or "silu_gate" (rows 2i / 2i+1 are gate / up projections: Y[b,t,i] = silu(z[2i]) * z[2i+1], Y is [B,m,N/2]);
-    returns Y [B,m,N] of X's type.  (simt=True runs the diagnostic CUDA-core kernel: bf16, no epilogue.)"""
+    returns Y [B,m,N] of X's type.  wide_range=True plans every m on the tiled schedule (for activations of
+    magnitude 2^16 or more, which the decode schedules clamp and flag).  (simt=True runs the diagnostic
+    CUDA-core kernel: bf16, no epilogue.)"""
     import torch
     lib = load_library()
     B, m, K = X.shape
@@ -188,11 +192,12 @@ def gemm(X, W_base, bits, alpha, out=None, workspace=None, stream=None, simt: bo
     if workspace is None:
         workspace = make_workspace(B, m, N, K, device=X.device, stream=stream)
     ws = (ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream_ptr(stream))
-    if io == torch.bfloat16 and bias is None and act == "none":
+    if io == torch.bfloat16 and bias is None and act == "none" and not wide_range:
         _check(lib.bitdelta_gemm(*args, _dev(out, io, "out"), *shape, *ws), "bitdelta_gemm")
     else:
         bp = _dev(bias, io, "bias") if bias is not None else ctypes.c_void_p(0)
-        _check(lib.bitdelta_gemm_ex(*args, bp, _dev(out, io, "out"), *shape, 1 if io == torch.float16 else 0,
+        _check(lib.bitdelta_gemm_ex(*args, bp, _dev(out, io, "out"), *shape,
+                                    (1 if io == torch.float16 else 0) | (DTYPE_WIDE_RANGE if wide_range else 0),
                                     ACTS[act], *ws), "bitdelta_gemm_ex")
     return out
 

@@ -231,7 +231,12 @@ size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K) {
     if ((K % 128) != 0) return 256;   // CUDA-core path: no scratch needed, keep the pointer non-NULL
     bd::Plan p = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override());
     if (!p.ok) return 0;
-    return p.ws_bytes;
+    size_t need = p.ws_bytes;
+    if (p.decode) {   // the same shape on the tiled schedule (BITDELTA_DTYPE_WIDE_RANGE) may need more
+        bd::Plan w = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override(), true, true);
+        if (w.ok && w.ws_bytes > need) need = w.ws_bytes;
+    }
+    return need;
 }
 
 int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
@@ -267,6 +272,8 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
                      size_t workspace_bytes, void* cuda_stream) {
     int st = check_gemm_args(X, W_base, bits, alpha, Y, B, m, N, K);
     if (st != BITDELTA_OK) return st;
+    const bool wide = (dtype & BITDELTA_DTYPE_WIDE_RANGE) != 0;
+    dtype &= ~BITDELTA_DTYPE_WIDE_RANGE;
     if ((dtype != BITDELTA_DTYPE_BF16 && dtype != BITDELTA_DTYPE_F16) || (act != BITDELTA_ACT_NONE && act != BITDELTA_ACT_SILU && act != BITDELTA_ACT_SILU_GATE))
         return BITDELTA_ERR_OPTION;
     if (act == BITDELTA_ACT_SILU_GATE && (N % 2) != 0) return BITDELTA_ERR_SHAPE;
@@ -285,14 +292,14 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         return BITDELTA_OK;
     }
 
-    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override());
+    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), true, wide);
     if (p.ok && p.pair) {
         // The pair schedule wants every pair resident at once (a cluster of two needs two free SMs of one
         // cluster-capable group); where the device cannot do that, run the one-CTA schedule.  Asked once per device.
         static int pairs_fit[64] = {};   // 0 unknown, 1 yes, -1 no
         const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
         if (pairs_fit[di] == 0) pairs_fit[di] = (2 * bd::max_active_pairs(p.smem_bytes) >= p.grid) ? 1 : -1;
-        if (pairs_fit[di] < 0) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false);
+        if (pairs_fit[di] < 0) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, wide);
     }
     if (p.ok && p.cluster > 1) {
         // The cluster form wants all its clusters resident at once (clusters are independent, so this is about
@@ -516,6 +523,7 @@ const char* bitdelta_status_string(int status) {
         case BITDELTA_ERR_CUDA: return "CUDA runtime or driver call failed";
         case BITDELTA_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
         case BITDELTA_ERR_OPTION: return "unknown data type or activation code";
+        case BITDELTA_ERR_RANGE: return "an activation of magnitude 2^16 or more was clamped in a decode schedule's delta term";
         default: return "unknown status";
     }
 }

@@ -100,13 +100,14 @@ inline bool cluster_enabled() {
 }
 
 // allow_pair = false: the device cannot hold all the pairs (or clusters) at once (see the launcher), plan without them.
+// force_tiled: plan the tiled schedule whatever m is (bf16 / binary16 operands for both terms).
 inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0,
-                      bool allow_pair = true) {
+                      bool allow_pair = true, bool force_tiled = false) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
     if (B <= 0 || m <= 0 || N <= 0 || K <= 0 || (K % 128) != 0) return p;
-    p.decode = (m <= kDecodeMaxM) ? 1 : 0;
+    p.decode = (m <= kDecodeMaxM && !force_tiled) ? 1 : 0;
     p.n_tiles = (N + kTileN - 1) / kTileN;
     if (p.decode) {
         p.N3 = round_up(kPieces * m, 16);

@@ -33,7 +33,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    for code in range(0, 9):
+    for code in range(0, 10):
         assert bd.status_string(code) != "unknown status"
     assert bd.status_string(99) == "unknown status"
 
