@@ -124,8 +124,10 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * is still running; it reads X and writes Y and the workspace only after that
  * kernel has completed.  W_base, bits and alpha must therefore not be produced
  * by the kernel queued directly before the call (weights are static in the
- * intended use); X may be.  BITDELTA_EARLY_START=0 in the environment turns
- * the early start off.
+ * intended use); X may be.  The library's own producers are covered: the
+ * first bitdelta_gemm call after a bitdelta_pack or bitdelta_compress call is
+ * launched without the early start.  BITDELTA_EARLY_START=0 in the environment
+ * turns the early start off altogether.
  */
 int bitdelta_gemm(const void* X, const void* W_base, const uint32_t* bits, const float* alpha,
                   void* Y, int B, int m, int N, int K,
@@ -180,7 +182,9 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
  *   - Shapes whose workspace (bitdelta_gemm_workspace_bytes) exceeds the array are refused with
  *     BITDELTA_ERR_WORKSPACE and nothing is launched; use bitdelta_gemm with your own buffer.
  *   - The first call on each device looks up the array's device address (the current device must be
- *     the one the call is for); make that first call outside any stream capture.
+ *     the one the call is for) and may be the moment the CUDA runtime binds this library's device image,
+ *     array included, to that device: make that first call at start-up, before the memory plan is
+ *     frozen and outside any stream capture.  Later calls allocate nothing.
  *   - All calls on a device share the one array.  Each call first clears, on the stream, the arrival
  *     counters at its start; the rest keeps whatever the previous call left and is fully rewritten
  *     before it is read.  Calls that can overlap on the device (issued on different streams) would
@@ -254,6 +258,16 @@ int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int ite
  * NULL (host pointer), receives a code naming the wait that expired.
  */
 int bitdelta_last_device_status(void* cuda_stream, int* site);
+
+/*
+ * Self-test of the time-out reporting (test aid; the paper's verifier section lists hangs on mbarrier phases
+ * among the hazards of asynchronous kernels, and every wait in this library's kernels is bounded): queues a
+ * one-warp kernel that waits, with the kernels' own bounded wait, on a barrier nobody signals, for
+ * `limit_cycles` SM cycles (1e3 .. 2e9), then gives up and returns normally.  Afterwards
+ * bitdelta_last_device_status returns BITDELTA_ERR_TIMEOUT with *site = `site`, once; the device and the
+ * library stay usable.  Nothing else is touched.  Asynchronous on the stream.
+ */
+int bitdelta_selftest_timeout(long long limit_cycles, int site, void* cuda_stream);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 unsigned long long bitdelta_kernel_launch_count(void);

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     load_library,
     make_workspace,
     pack,
+    selftest_timeout,
     status_string,
     unpack,
 )

@@ -24,7 +24,7 @@ EXPORTS = (
     "bitdelta_gemm_workspace_bytes", "bitdelta_workspace_init",
     "bitdelta_gemm", "bitdelta_gemm_ex", "bitdelta_gemm_noalloc", "bitdelta_gemm_simt", "bitdelta_gemm_host_arena_bytes", "bitdelta_gemm_host",
     "bitdelta_gemm_plan", "bitdelta_gemm_plan_cta_items", "bitdelta_gemm_plan_item_cta",
-    "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string",
+    "bitdelta_last_device_status", "bitdelta_kernel_launch_count", "bitdelta_status_string", "bitdelta_selftest_timeout",
 )
 
 
@@ -69,6 +69,7 @@ def load_library():
     lib.bitdelta_gemm_plan_item_cta.argtypes = [ci, ci, ci, ci, ci, ci]
     lib.bitdelta_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.bitdelta_kernel_launch_count.restype = ctypes.c_ulonglong
+    lib.bitdelta_selftest_timeout.argtypes = [ctypes.c_longlong, ci, vp]
     lib.bitdelta_status_string.argtypes = [ci]
     lib.bitdelta_status_string.restype = ctypes.c_char_p
     for fn in ("bitdelta_pack", "bitdelta_unpack", "bitdelta_compress", "bitdelta_workspace_init", "bitdelta_gemm",
@@ -76,6 +77,12 @@ def load_library():
         getattr(lib, fn).restype = ci
     _lib = lib
     return lib
+
+
+def selftest_timeout(limit_cycles: int = 1_000_000, site: int = 99, stream=None) -> None:
+    """Queues the one-warp kernel whose bounded wait expires after `limit_cycles`; last_device_status() then
+    reports (STATUS_TIMEOUT, site) once."""
+    _check(load_library().bitdelta_selftest_timeout(int(limit_cycles), int(site), _stream_ptr(stream)), "bitdelta_selftest_timeout")
 
 
 def status_string(status: int) -> str:
@@ -119,20 +126,25 @@ def unpack(bits, stream=None):
     return S
 
 
-def compress(W_fine, W_base, stream=None):
+def compress(W_fine, W_base, stream=None, bits=None, alpha=None):
     """Fine-tuned weights bf16 [B,N,K] and base weights bf16 [N,K] (device) -> (bits int32 storage
-    [B,N,K/32], alpha fp32 [B]): bit = (W_fine - W_base > 0), alpha = mean |W_fine - W_base| per tenant."""
+    [B,N,K/32], alpha fp32 [B]): bit = (W_fine - W_base > 0), alpha = mean |W_fine - W_base| per tenant.
+    `bits` / `alpha`: caller's output tensors (allocated here if omitted)."""
     import torch
     lib = load_library()
     B, N, K = W_fine.shape
     if tuple(W_base.shape) != (N, K) or K % 32:
         raise ValueError("inconsistent shapes, or K not a multiple of 32")
-    bits = torch.empty((B, N, K // 32), dtype=torch.int32, device=W_fine.device)
-    alpha = torch.empty((B,), dtype=torch.float32, device=W_fine.device)
+    if bits is None:
+        bits = torch.empty((B, N, K // 32), dtype=torch.int32, device=W_fine.device)
+    if alpha is None:
+        alpha = torch.empty((B,), dtype=torch.float32, device=W_fine.device)
+    if tuple(bits.shape) != (B, N, K // 32) or tuple(alpha.shape) != (B,):
+        raise ValueError("inconsistent output shapes")
     nbytes = int(lib.bitdelta_compress_workspace_bytes(B, N, K))
     ws = torch.empty(max(nbytes, 8), dtype=torch.uint8, device=W_fine.device)
     _check(lib.bitdelta_compress(_dev(W_fine, torch.bfloat16, "W_fine"), _dev(W_base, torch.bfloat16, "W_base"),
-                                 ctypes.c_void_p(bits.data_ptr()), ctypes.c_void_p(alpha.data_ptr()), B, N, K,
+                                 _dev(bits, torch.int32, "bits"), _dev(alpha, torch.float32, "alpha"), B, N, K,
                                  ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream_ptr(stream)), "bitdelta_compress")
     return bits, alpha
 

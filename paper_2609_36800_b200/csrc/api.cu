@@ -22,6 +22,9 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[BITDELTA_NOALLO
 namespace {
 
 std::atomic<unsigned long long> g_launches{0};
+// Set by the entry points that PRODUCE what the GEMM prefetches before its grid dependency is resolved (sign words,
+// alpha: bitdelta_pack, bitdelta_compress); the next GEMM call then launches fully serialised, once.
+std::atomic<int> g_weights_just_written{0};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -185,6 +188,7 @@ int bitdelta_pack(const int8_t* S, uint32_t* bits, int B, int N, int K, void* cu
     const long long words = (long long)B * N * (K / 32);
     if (bd::launch_pack(S, bits, words, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
+    g_weights_just_written.store(1);
     g_launches++;
     return BITDELTA_OK;
 }
@@ -222,6 +226,7 @@ int bitdelta_compress(const void* W_fine, const void* W_base, uint32_t* bits, fl
     if (bd::launch_compress(W_fine, W_base, bits, alpha, static_cast<double*>(workspace), B, N, K,
                             static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return BITDELTA_ERR_CUDA;
+    g_weights_just_written.store(1);
     g_launches += 2;
     return BITDELTA_OK;
 }
@@ -296,10 +301,19 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     if (p.ok && p.pair) {
         // The pair schedule wants every pair resident at once (a cluster of two needs two free SMs of one
         // cluster-capable group); where the device cannot do that, run the one-CTA schedule.  Asked once per device.
-        static int pairs_fit[64] = {};   // 0 unknown, 1 yes, -1 no
+        static std::mutex mu_pairs;
+        static int pairs_cache[64][2] = {};   // [device]: {shared memory bytes asked with, pairs that fit + 1}
         const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
-        if (pairs_fit[di] == 0) pairs_fit[di] = (2 * bd::max_active_pairs(p.smem_bytes) >= p.grid) ? 1 : -1;
-        if (pairs_fit[di] < 0) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, wide);
+        int fit;
+        {
+            std::lock_guard<std::mutex> lock(mu_pairs);
+            if (pairs_cache[di][1] == 0 || pairs_cache[di][0] != (int)p.smem_bytes) {
+                pairs_cache[di][0] = (int)p.smem_bytes;
+                pairs_cache[di][1] = bd::max_active_pairs(p.smem_bytes) + 1;
+            }
+            fit = pairs_cache[di][1] - 1;
+        }
+        if (2 * fit < p.grid) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, wide);
     }
     if (p.ok && p.cluster > 1) {
         // The cluster form wants all its clusters resident at once (clusters are independent, so this is about
@@ -352,9 +366,11 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_EARLY"); d = (e && e[0] == '1') ? 1 : 0; } args.trigger_early = d; }
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_DECODE_WARPS"); d = (e && atoi(e) == 16) ? 16 : 8; } args.decode_warps = d; }
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_PREFETCH"); d = e ? atoi(e) : 0; } args.prefetch_steps = d; }
+    // (a GEMM queued right behind the library's own pack / compress must not prefetch what they are still writing)
+    const bool early = early_start_enabled() && g_weights_just_written.exchange(0) == 0;
     const cudaError_t le = p.stream
-        ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream)
-        : bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early_start_enabled(), stream);
+        ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early, stream)
+        : bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early, stream);
     if (le != cudaSuccess) return BITDELTA_ERR_CUDA;
     g_launches++;
     return BITDELTA_OK;
@@ -464,6 +480,17 @@ int bitdelta_gemm_plan_item_cta(int B, int m, int N, int K, int num_sms, int ite
     if (p.whole_units) return (item / p.P) % p.grid;
     const bd::GemmArgs a = bd::make_args(p, nullptr, nullptr, nullptr);
     return p.pair ? 2 * bd::cta_of_item(a, item) : bd::cta_of_item(a, item);   // (pairs: the pair's first block)
+}
+
+int bitdelta_selftest_timeout(long long limit_cycles, int site, void* cuda_stream) {
+    if (limit_cycles < 1000 || limit_cycles > 2000000000ll || site < 0) return BITDELTA_ERR_SHAPE;
+    DeviceInfo d;
+    int st = check_arch(&d);
+    if (st != BITDELTA_OK) return st;
+    if (bd::launch_selftest_timeout(limit_cycles, site, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return BITDELTA_ERR_CUDA;
+    g_launches++;
+    return BITDELTA_OK;
 }
 
 int bitdelta_last_device_status(void* cuda_stream, int* site) {

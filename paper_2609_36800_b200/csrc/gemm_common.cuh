@@ -22,9 +22,10 @@ constexpr unsigned int kStatusRange = 9u;     // BITDELTA_ERR_RANGE: an activati
 // Bounded wait on an mbarrier phase.  Returns false if the wait was abandoned
 // (limit reached here or in another thread of the CTA).  The slow path is kept out of line: it is
 // instantiated at some twenty call sites and would otherwise dominate the kernel's code size.
-static __device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+static __device__ __noinline__ bool wait_bar_limited(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site,
+                                                     long long limit_cycles) {
     // Poll, and every 64 polls look at the abort flag and the SM cycle counter
-    // (cheap to read; the limit is ~2 s at 2 GHz, longer at lower clocks).
+    // (cheap to read; the default limit is ~2 s at 2 GHz, longer at lower clocks).
     const long long t0 = clock64();
 #pragma unroll 1
     for (;;) {
@@ -33,12 +34,15 @@ static __device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity,
             if (mbar_try_wait(bar, parity)) return true;
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
-            if (atomicCAS(&g_device_status[0], 0u, 7u) == 0u) g_device_status[1] = (unsigned)site;
+            if (atomicCAS(&g_device_status[0], 0u, kStatusTimeout) == 0u) g_device_status[1] = (unsigned)site;
             return false;
         }
     }
+}
+static __device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
+    return wait_bar_limited(bar, parity, abort_flag, site, kWaitLimitCycles);
 }
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int site) {
     if (mbar_try_wait(bar, parity)) return true;

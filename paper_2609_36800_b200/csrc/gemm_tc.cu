@@ -861,12 +861,14 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                 // All epilogue threads' partial stores, then one thread's fence (cumulative over what the
                 // barrier ordered before it) and the arrival count.
                 epi_bar_sync(n_epi_warps * 32);
+                if (*abort_flag) break;   // (a sibling left on an abandoned wait and released this barrier once)
                 if (etid == 0) {
                     __threadfence();
                     const unsigned old = atomicAdd(&a.counters[kPair ? 2 * unit + (int)rank : unit], 1u);
                     ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);
+                if (*abort_flag) break;   // (a sibling left on an abandoned wait and released this barrier once)
                 if (ctl->is_last) {
                     __threadfence();
                     // CTA c0 holds the tile's first item; the tile is its first segment only if its
@@ -882,7 +884,15 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                     if (etid == 0) a.counters[kPair ? 2 * unit + (int)rank : unit] = 0u;
                 }
                 epi_bar_sync(n_epi_warps * 32);   // is_last is rewritten by the next cut tile
+                if (*abort_flag) break;   // (a sibling left on an abandoned wait and released this barrier once)
             }
+        }
+        if (!ok) {
+            // This warp left on an abandoned wait; a sibling that passed the same wait a moment earlier may be
+            // waiting on the epilogue barrier (which has no time-out): release it once.  It then sees the abort
+            // flag and leaves too.
+            __syncwarp();
+            named_bar_arrive(1, n_epi_warps * 32);
         }
     }
 
@@ -976,6 +986,26 @@ int max_active_pairs(uint32_t smem_bytes) {
         return 0;
     }
     return n;
+}
+
+// Self-test of the time-out path: one warp waits, with the kernels' own bounded wait, on an mbarrier nobody
+// arrives on; the wait gives up after `limit_cycles`, records {time-out, site} in the status word and the
+// kernel returns normally.  No tensor memory, no named or cluster barriers, nothing else in flight.
+__global__ void __launch_bounds__(32, 1) selftest_timeout_kernel(long long limit_cycles, int site) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncwarp();
+    (void)wait_bar_limited(smem_u32(&bar), 0u, &abort_flag, site, limit_cycles);
+}
+
+cudaError_t launch_selftest_timeout(long long limit_cycles, int site, cudaStream_t stream) {
+    selftest_timeout_kernel<<<1, 32, 0, stream>>>(limit_cycles, site);
+    return cudaGetLastError();
 }
 
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {

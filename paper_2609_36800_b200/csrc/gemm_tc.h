@@ -125,6 +125,9 @@ int max_active_pairs(uint32_t smem_bytes);
 // each group of 32) in X8 [B, 4, m, K].
 cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream);
 
+// One warp that lets a bounded wait expire after `limit_cycles` (see bitdelta_selftest_timeout).
+cudaError_t launch_selftest_timeout(long long limit_cycles, int site, cudaStream_t stream);
+
 // Synchronises the stream, reads {status, site} and clears them if set.
 cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream);
 

@@ -60,3 +60,36 @@ def test_compress_is_deterministic_and_feeds_the_gemm():
     Yg = synth.bf16_bits_to_f32(Y.view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
     assert np.max(np.abs(Yg - Yref)) <= 2e-2
     assert np.linalg.norm(Yg - Yref) / np.linalg.norm(Yref) <= 5e-3
+
+
+def test_gemm_queued_directly_behind_compress_reads_the_new_signs():
+    # compress and gemm back to back on one stream, workspace made beforehand, nothing in between: the GEMM's early
+    # weight prefetch must not run ahead of the compress kernels that are still writing the sign words and alpha.
+    # Three rounds into the SAME device buffers with different fine-tuned weights: stale signs would be the
+    # previous round's and miss the gate by far.
+    import torch
+    import paper_2609_36800_b200 as bd
+    B, N, K, m = 8, 1024, 2048, 1
+    rng = np.random.default_rng(4)
+    X = synth.f32_to_bf16_bits(rng.standard_normal((B, m, K), dtype=np.float32))
+    dX = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
+    ws = bd.make_workspace(B, m, N, K)
+    d_fine = torch.empty((B, N, K), dtype=torch.bfloat16, device="cuda")
+    d_W = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    d_bits = torch.empty((B, N, K // 32), dtype=torch.int32, device="cuda")
+    d_alpha = torch.empty((B,), dtype=torch.float32, device="cuda")
+    Y = torch.empty((B, m, N), dtype=torch.bfloat16, device="cuda")
+    for rnd in range(3):
+        fine, W = synth.make_fine_weights(B, N, K, seed=100 + rnd)
+        d_fine.copy_(torch.from_numpy(fine.view(np.int16)).view(torch.bfloat16))
+        d_W.copy_(torch.from_numpy(W.view(np.int16)).view(torch.bfloat16))
+        torch.cuda.synchronize()
+        bd.compress(d_fine, d_W, bits=d_bits, alpha=d_alpha)
+        bd.gemm(dX, d_W, d_bits, d_alpha, out=Y, workspace=ws)
+        torch.cuda.synchronize()
+        ref_bits, ref_alpha = oracle.compress(fine, W)
+        assert np.array_equal(d_bits.cpu().numpy().view(np.uint32), ref_bits)
+        Yref = oracle.gemm(X, W, ref_bits, ref_alpha)
+        Yg = synth.bf16_bits_to_f32(Y.view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+        assert np.max(np.abs(Yg - Yref)) <= 2e-2, rnd
+        assert np.linalg.norm(Yg - Yref) / np.linalg.norm(Yref) <= 5e-3, rnd

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2609_36800_b200 as bd
 from paper_2609_36800_b200 import synth
 
@@ -27,7 +28,7 @@ def _both(wl):
     bd.gemm_noalloc(dX, dW, dbits, dalpha, out)                # new entry point, library-held scratch
     st, site = bd.last_device_status()
     assert st == 0, (st, site)
-    return y_to_f64(out), y_to_f64(ref)
+    return y_to_f64(out), y_to_f64(ref), oracle.gemm(X, W, bits, alpha)
 
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point():
@@ -35,12 +36,32 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     for wl in (synth.Workload("a", B=8, m=1, K=2048, N=1024, seed=31),
                synth.Workload("b", B=2, m=40, K=512, N=384, seed=32),
                synth.Workload("a2", B=8, m=1, K=2048, N=1024, seed=33)):
-        got, ref = _both(wl)
+        got, ref, exact = _both(wl)
         assert not np.isnan(got).any()
         max_abs, rel_fro = errors(got, ref)
         assert max_abs <= MAX_ABS_TOL and rel_fro <= REL_FRO_TOL, (wl.name, max_abs, rel_fro)
         # same kernels, same schedule: in fact identical
         assert np.array_equal(got, ref), wl.name
+        # ... and both are the product itself: the fp64 CPU oracle at the parity gates
+        max_abs, rel_fro = errors(got, exact)
+        assert max_abs <= MAX_ABS_TOL and rel_fro <= REL_FRO_TOL, (wl.name, max_abs, rel_fro)
+
+
+def test_a_warm_call_allocates_no_device_memory():
+    # the entry point's defining property: once the first call on the device has been made, a call leaves the
+    # device's free memory exactly as it found it (inputs and output are the caller's, made beforehand)
+    wl = synth.Workload("c", B=8, m=1, K=2048, N=1024, seed=34)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
+    out = torch.empty((wl.B, wl.m, wl.N), dtype=torch.bfloat16, device="cuda")
+    bd.gemm_noalloc(dX, dW, dbits, dalpha, out)                # first call on this device (if no test ran before)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        bd.gemm_noalloc(dX, dW, dbits, dalpha, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
 
 
 def test_shapes_beyond_the_fixed_scratch_are_refused_without_a_launch():
