@@ -31,15 +31,17 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 PAPER_CONTEXT = "paper: 3.34x (standard) / 2.51x (batched) over autotuned Triton 3.6.0 on B200, FP16; no absolute figure"
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernel from the
-# ncu captures summarised under profiles/ ; None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {
-    "decode_attn": 50_510_000,          # 50.49 MB read + 0.02 MB written
-    "decode_mlp_up": 219_000_000,       # 213.7 MB read + 5.3 MB written (a third of W_base read twice)
-    "prefill": 96_000_000,              # 75 MB read + 21 MB written (pair schedule; 62 + 12 MB with one CTA per tile)
-    "many_tenant_down": 416_000_000,    # 408.3 MB read + 7.6 MB written
-    "tiny": None,
-}
+def load_traffic():
+    """DRAM bytes per launch of the GEMM kernel from the ncu captures summarised under profiles/."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        with open(path) as f:
+            return {k: v for k, v in json.load(f).items() if not k.startswith("_")}
+    except Exception:
+        return {}
+
+
+NCU_TRAFFIC_BYTES = load_traffic()
 
 
 def load_peaks():
@@ -130,12 +132,13 @@ def device_sets(wl, X, W, bits, alpha, nsets):
     return sets
 
 
-def time_workload(wl, steps, warmup, dist=None, sampler=None):
-    """Returns (ms_total over `steps` launches, nsets).  Device-timed with CUDA events."""
+def time_workload(wl, steps, warmup, dist=None, sampler=None, inputs=None):
+    """Returns (ms_total over `steps` launches, nsets).  Device-timed with CUDA events.  `inputs`: host arrays to
+    use instead of the workload's own seeded draw (a tenant shard of a larger workload)."""
     import torch
     import paper_2609_36800_b200 as bd
 
-    X, W, bits, alpha = synth.make_inputs(wl)
+    X, W, bits, alpha = inputs if inputs is not None else synth.make_inputs(wl)
     nsets = max(2, -(-2 * L2_BYTES // wl.bytes))
     sets = device_sets(wl, X, W, bits, alpha, nsets)
     ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
@@ -205,6 +208,63 @@ def batch_stats(wl, sets, batches=20):
                           "launches_per_batch": len(order), "batches": batches}
     out["warm_l2"]["note"] = "one buffer set reused: inputs up to the L2 size stay resident; not a roofline number"
     return out
+
+
+def host_call_cost(wl, sets, calls=200):
+    """Host time of one eager bitdelta_gemm call (argument checks, plan, tensor-map look-up, launch; the ctypes
+    marshalling of this binding included), in microseconds: what a caller outside a CUDA graph pays per call."""
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
+    s = sets[0]
+    for _ in range(10):
+        bd.gemm(s[0], s[1], s[2], s[3], out=s[4], workspace=ws)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        bd.gemm(s[0], s[1], s[2], s[3], out=s[4], workspace=ws)
+    dt = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    return dt / calls * 1e6
+
+
+def time_serialized(wl, sets, launches=24):
+    """The same launches without the early start (BITDELTA_EARLY_START=0): every kernel begins only when the one
+    before it has completed, so nothing of a call hides behind its predecessor.  Cold L2, one CUDA graph."""
+    import torch
+    import paper_2609_36800_b200 as bd
+
+    nsets = len(sets)
+    ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
+    stream = torch.cuda.Stream()
+    old = os.environ.get("BITDELTA_EARLY_START")
+    os.environ["BITDELTA_EARLY_START"] = "0"
+    try:
+        with torch.cuda.stream(stream):
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(launches):
+                    s = sets[i % nsets]
+                    bd.gemm(s[0], s[1], s[2], s[3], out=s[4], workspace=ws)
+            graph.replay()
+            stream.synchronize()
+            times = []
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                graph.replay()
+                e1.record(stream)
+                stream.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3 / launches)
+    finally:
+        if old is None:
+            os.environ.pop("BITDELTA_EARLY_START", None)
+        else:
+            os.environ["BITDELTA_EARLY_START"] = old
+    times.sort()
+    return {"us_per_launch_median": times[len(times) // 2], "us_per_launch_min": times[0], "launches": launches,
+            "note": "early start off: launch latency, prologue and first loads of every call are exposed"}
 
 
 def time_compress(peaks, B=8, N=4096, K=4096, steps=20):
@@ -401,17 +461,42 @@ def run_ours(args):
                           "roofline": r["roofline"], "gpu_launches": args.steps * kernels_per_step(wl)}), flush=True)
         return
 
+    # What this rank runs: the whole workload (replicas: every GPU serves its own copy of all tenants), or with
+    # --shard-tenants its contiguous share of the workload's tenants (W_base replicated, nothing exchanged).
+    full_wl = wl
+    shard_inputs = None
+    shard_note = None
+    if args.shard_tenants and world > 1:
+        from paper_2609_36800_b200 import replicas
+        Xf, Wf, bitsf, alphaf = synth.make_inputs(wl)
+        Xs, bs, als, start = replicas.tenant_shard(Xf, bitsf, alphaf, world, rank)
+        if Xs.shape[0] == 0:
+            raise RuntimeError(f"--shard-tenants: {wl.B} tenants cannot be cut over {world} GPUs")
+        wl = synth.Workload(wl.name, B=int(Xs.shape[0]), m=wl.m, K=wl.K, N=wl.N, w_std=wl.w_std, alpha_lo=wl.alpha_lo,
+                            alpha_hi=wl.alpha_hi, seed=wl.seed)
+        shard_inputs = (np.ascontiguousarray(Xs), Wf, np.ascontiguousarray(bs), np.ascontiguousarray(als))
+        shard_note = f"tenants [{start}, {start + wl.B}) of {full_wl.B} on rank {rank}"
+
     sampler = ClockSampler(physical_gpu_index(local_rank)) if rank == 0 else None
     launches0 = bd.kernel_launch_count()
-    ms, nsets, host_inputs, _sets = time_workload(wl, args.steps, args.warmup, dist, sampler)
+    ms, nsets, host_inputs, _sets = time_workload(wl, args.steps, args.warmup, dist, sampler, inputs=shard_inputs)
     clocks = sampler.stop() if sampler is not None else None
+    job_bytes, job_flops = float(wl.bytes * world), float(wl.flops * world)
     if dist is not None:
         from paper_2609_36800_b200 import replicas
         ms = replicas.max_over_ranks(ms, dist, device="cuda")
+        if shard_inputs is not None:   # ranks may hold different numbers of tenants: add the work up
+            tot = torch.tensor([float(wl.bytes), float(wl.flops)], dtype=torch.float64, device="cuda")
+            dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+            job_bytes, job_flops = float(tot[0].item()), float(tot[1].item())
     stats = batch_stats(wl, _sets) if (rank == 0 and world == 1) else None
+    host_cost = host_call_cost(wl, _sets) if (rank == 0 and world == 1) else None
+    serial = time_serialized(wl, _sets) if (rank == 0 and world == 1) else None
     del _sets
     torch.cuda.empty_cache()
-    gbs, tfl, roof = summarize(wl, ms, args.steps, world, peaks, clocks)
+    gbs, tfl, roof = summarize(wl, ms, args.steps, 1, peaks, clocks)      # this rank's kernel against one GPU's roofline
+    sec_per_step = ms / 1e3 / args.steps
+    gbs, tfl = job_bytes / sec_per_step / 1e9, job_flops / sec_per_step / 1e12   # whole job: all ranks' work over the slowest rank's time
 
     out = None
     if rank == 0:
@@ -424,10 +509,13 @@ def run_ours(args):
             "value": gbs if hbm_bound else tfl,
             "unit": "GB/s" if hbm_bound else "TFLOP/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong" if shard_inputs is not None else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "m": wl.m, "K": wl.K, "N": wl.N,
-                       "parallelism": "replicas only (no data-path collective)" if world > 1 else "single GPU",
+            "config": {"workload": full_wl.name, "B": full_wl.B, "m": full_wl.m, "K": full_wl.K, "N": full_wl.N,
+                       "parallelism": ("single GPU" if world == 1 else
+                                       (f"tenants sharded over {world} GPUs, W_base replicated, no data-path collective ({shard_note})"
+                                        if shard_inputs is not None else f"{world} replicas (no data-path collective)")),
                        "l2": f"cold: steps cycle through {nsets} buffer sets ({nsets * wl.bytes / 2**20:.0f} MiB > 2x L2)",
                        "launch": "all timed steps in one CUDA graph"},
             "tflops": tfl, "gbs": gbs,
@@ -442,22 +530,34 @@ def run_ours(args):
         }
         if stats is not None:
             out["batches"] = stats
+        if host_cost is not None:
+            out["host_us_per_call"] = host_cost
+        if serial is not None:
+            out["serialized_launches"] = serial
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(wl, host_inputs)
-        if args.all:
+        if world == 1 and not args.no_workloads:
+            # The other four workloads and the compress step, timed the same way (cold L2, one CUDA graph), short:
+            # every configuration's roofline fraction comes out of the one default command.
             others = {}
             for w2 in synth.WORKLOADS:
                 if w2.name == wl.name:
                     continue
-                steps2 = max(20, min(args.steps, int(0.25 / max(w2.bytes / 6.5e12, w2.flops / 1.6e15))))
+                steps2 = max(20, min(args.steps, int(0.25 / max(w2.bytes / 6.5e12, w2.flops / 1.6e15)))) if args.all else 20
                 ms2, nsets2, _, s2 = time_workload(w2, steps2, 3)
                 del s2
                 torch.cuda.empty_cache()
                 g2, t2, r2 = summarize(w2, ms2, steps2, 1, peaks)
-                others[w2.name] = {"us_per_launch": ms2 * 1e3 / steps2, "gbs": g2, "tflops": t2, "steps": steps2,
-                                   "buffer_sets": nsets2, "roofline": r2}
+                if args.all:
+                    others[w2.name] = {"us_per_launch": ms2 * 1e3 / steps2, "gbs": g2, "tflops": t2, "steps": steps2,
+                                       "buffer_sets": nsets2, "roofline": r2}
+                else:
+                    others[w2.name] = {"us_per_launch": ms2 * 1e3 / steps2, "steps": steps2, "buffer_sets": nsets2,
+                                       "bound": r2["bound"], "achieved": r2["achieved"], "unit": r2["unit"],
+                                       "peak": r2["peak"], "frac": r2["frac"], "traffic": r2["traffic"]}
             out["workloads"] = others
             out["compress"] = time_compress(peaks)
+        if args.all:
             out["gemm_ex"] = {}
             for name in ("decode_attn", "decode_mlp_up", "prefill"):
                 w3 = synth.WORKLOADS_BY_NAME[name]
@@ -531,14 +631,33 @@ def main():
     ap.add_argument("--all", action="store_true", help="also time the other workloads (N=1 only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="skip the short timings of the other workloads and of the compress step (N=1)")
+    ap.add_argument("--shard-tenants", action="store_true",
+                    help="N > 1: every GPU serves its share of the workload's tenants (strong scaling) instead of "
+                         "a full replica (weak scaling)")
     ap.add_argument("--ex-only", action="store_true",
                     help="time only the extended call (fp16 operands, bias, SiLU) on --workload and print its "
                          "line; N=1, no end-to-end or CPU leg (used for profiling that kernel instantiation)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # Started as a plain `python bench.py --gpus N`: become N processes, one per GPU, under torchrun
+        # (NCCL is used for the barrier and the MAX of the per-rank times only).
+        import socket
+        import subprocess
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.run(cmd).returncode)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != max(args.gpus, 1):
+        print(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}; running {world} rank(s)", file=sys.stderr)
+    run_ours(args)
 
 
 if __name__ == "__main__":

@@ -143,36 +143,72 @@ bool encode_bits_3d(CUtensorMap* map, const void* ptr, uint64_t B, uint64_t N, u
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// BITDELTA_TB=<n> overrides the tenants per decode tile (experiments).
+// BITDELTA_TB=<n> overrides the tenants per decode tile (experiments); read once.
 int tb_override() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("BITDELTA_TB");
-        v = e ? atoi(e) : 0;
-    }
+    static int v = 0;
+    static std::once_flag once;
+    std::call_once(once, [] { const char* e = getenv("BITDELTA_TB"); v = e ? atoi(e) : 0; });
     return v;
 }
 
-// BITDELTA_WHOLE (experiments): 1 forces, 2 forbids the whole-unit work order; 3 forces one team of CTAs per
-// tenant group, 4 forces the plain even cut.
+// BITDELTA_WHOLE (experiments, read once): 1 forces, 2 forbids the whole-unit work order; 3 forces one team of CTAs
+// per tenant group, 4 forces the plain even cut.
 int whole_override() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("BITDELTA_WHOLE");
-        v = e ? atoi(e) : 0;
-    }
+    static int v = 0;
+    static std::once_flag once;
+    std::call_once(once, [] { const char* e = getenv("BITDELTA_WHOLE"); v = e ? atoi(e) : 0; });
     return v;
 }
 
 // BITDELTA_EARLY_START=0 launches the GEMM kernel fully serialised behind its predecessor
 // (for experiments; the default lets it begin its weight prefetch early).
 bool early_start_enabled() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("BITDELTA_EARLY_START");
-        v = (e && e[0] == '0') ? 0 : 1;
+    const char* e = getenv("BITDELTA_EARLY_START");   // (read at every call: bench.py times both settings in one process)
+    return !(e && e[0] == '0');
+}
+
+// Encoded tensor maps, kept per (kind, pointer, shape, box): encoding one costs a microsecond or two of host time,
+// a GEMM call needs three or four, and a serving loop calls with the same few weight and activation buffers.
+struct MapKey {
+    int kind;
+    const void* ptr;
+    uint64_t d0, d1, d2;
+    uint32_t b0, b1;
+    bool operator==(const MapKey& o) const {
+        return kind == o.kind && ptr == o.ptr && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b0 == o.b0 && b1 == o.b1;
     }
-    return v != 0;
+};
+constexpr int kMapCacheSize = 64;
+struct MapCache {
+    std::mutex mu;
+    MapKey keys[kMapCacheSize];
+    CUtensorMap maps[kMapCacheSize];
+    bool used[kMapCacheSize] = {};
+    int next = 0;
+};
+MapCache& map_cache() {
+    static MapCache c;
+    return c;
+}
+template <class Encode>
+bool cached_map(CUtensorMap* out, const MapKey& key, Encode encode) {
+    MapCache& c = map_cache();
+    {
+        std::lock_guard<std::mutex> lock(c.mu);
+        for (int i = 0; i < kMapCacheSize; ++i)
+            if (c.used[i] && c.keys[i] == key) {
+                *out = c.maps[i];
+                return true;
+            }
+    }
+    if (!encode(out)) return false;
+    std::lock_guard<std::mutex> lock(c.mu);
+    const int i = c.next;
+    c.next = (c.next + 1) % kMapCacheSize;
+    c.keys[i] = key;
+    c.maps[i] = *out;
+    c.used[i] = true;
+    return true;
 }
 
 }  // namespace
@@ -337,15 +373,22 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     if (!aligned16(workspace)) return BITDELTA_ERR_ALIGN;
 
     CUtensorMap tmW, tmX, tmX8, tmBits;
-    if (!encode_bf16_tile(&tmW, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN)) return BITDELTA_ERR_CUDA;
-    if (!p.stream && !encode_bf16_tile(&tmX, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows)) return BITDELTA_ERR_CUDA;
-    if (!encode_bits_3d(&tmBits, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, p.stream ? 4u : 8u))
+    if (!cached_map(&tmW, MapKey{0, W_base, (uint64_t)N, (uint64_t)K, 0, (uint32_t)bd::kTileN, 0u},
+                    [&](CUtensorMap* mp) { return encode_bf16_tile(mp, W_base, (uint64_t)N, (uint64_t)K, bd::kTileN); }))
+        return BITDELTA_ERR_CUDA;
+    if (!p.stream && !cached_map(&tmX, MapKey{0, X, (uint64_t)B * m, (uint64_t)K, 0, (uint32_t)p.x_rows, 0u},
+                                 [&](CUtensorMap* mp) { return encode_bf16_tile(mp, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows); }))
+        return BITDELTA_ERR_CUDA;
+    const uint32_t box_words = p.stream ? 4u : 8u;
+    if (!cached_map(&tmBits, MapKey{1, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words},
+                    [&](CUtensorMap* mp) { return encode_bits_3d(mp, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words); }))
         return BITDELTA_ERR_CUDA;
     if (p.decode && !p.convert) {
         // Decode schedule with many token rows per tile: split the activations into e5m2 pieces first
         // (tiny), then the GEMM, which may start prefetching weights while the split is still running.
         uint8_t* x8 = bd::ws_x8(p, workspace);
-        if (!encode_u8_2d(&tmX8, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, (uint32_t)p.x8_rows))
+        if (!cached_map(&tmX8, MapKey{2, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, 0, (uint32_t)p.x8_rows, 0u},
+                        [&](CUtensorMap* mp) { return encode_u8_2d(mp, x8, (uint64_t)B * bd::kPieces * m, (uint64_t)K, (uint32_t)p.x8_rows); }))
             return BITDELTA_ERR_CUDA;
         if (bd::launch_x_split(X, x8, B, m, K, f16, stream) != cudaSuccess)
             return BITDELTA_ERR_CUDA;

@@ -28,6 +28,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <type_traits>
 
 #include "gemm_common.cuh"
@@ -850,17 +851,17 @@ cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits
         bitdelta_gemm_stream_kernel<4, true, 2>,  bitdelta_gemm_stream_kernel<5, true, 2>};
     // Per device and instantiation, once: allow the dynamic shared memory and ask for the largest shared-memory
     // carve-out, so that two blocks (of consecutive launches) fit on one multiprocessor.
-    static unsigned char attr_done[64][20] = {};
+    static std::atomic<unsigned char> attr_done[64][20];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!attr_done[dev][mode]) {
+    if (!attr_done[dev][mode].load()) {
         e = cudaFuncSetAttribute(kernels[mode], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(kernels[mode], cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        attr_done[dev][mode] = 1;
+        attr_done[dev][mode].store(1);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
