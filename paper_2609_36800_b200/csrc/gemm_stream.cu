@@ -39,9 +39,9 @@ namespace bd {
 
 constexpr int kSWarpProducer = 0;
 constexpr int kSWarpMma = 1;
-constexpr int kSWarpDecode0 = 2;                 // warps 2 .. 2 + 8 kG - 1 decode (kG = 1: 8 warps, kG = 2: 16)
+constexpr int kSWarpDecode0 = 2;                 // warps 2 .. 9 decode
 constexpr int kSEpiWarps = 4;                    // the four warps after them
-__host__ __device__ constexpr int stream_threads(int kG) { return (kSWarpDecode0 + 8 * kG + kSEpiWarps) * 32; }   // 448 / 704
+__host__ __device__ constexpr int stream_threads(int /*kG*/) { return (kSWarpDecode0 + 8 + kSEpiWarps) * 32; }   // 448
 constexpr int kSBarSet0 = 2;                     // named barrier of operand set s: id 2 + s
 constexpr int kSBarDep = 15;                     // named barrier the decode and epilogue warps sleep on until the grid
                                                  // dependency is resolved (the issuer warp arrives on it)
@@ -138,6 +138,67 @@ __device__ __forceinline__ void split_from_global(const GemmArgs& a, int am, con
     if (out_of_range) atomicCAS(&g_device_status[0], 0u, kStatusRange);
 }
 
+// The same split for more than eight token rows per unit: a task is a whole 32-k group of one row (64 bytes, four
+// 16-byte loads requested together, so a step costs one round trip to L2 per thread), 16-byte shared stores.
+template <bool kF16>
+__device__ __forceinline__ void split_from_global_wide(const GemmArgs& a, int am, const uint16_t* __restrict__ xg, uint8_t* xt,
+                                                       uint8_t* x8t, int ntok, int tid, int nthreads) {
+    const int ntasks = ntok * 4;
+    bool out_of_range = false;
+    for (int task = tid; task < ntasks; task += nthreads) {
+        const int r = task >> 2, q4 = task & 3;
+        const int j = r / am, t = r - j * am;
+        const uint4* src = reinterpret_cast<const uint4*>(xg + (size_t)r * a.K + q4 * 32);
+        uint4 L[4];   // L[i]: k = 8i .. 8i+7 of the group as four pairs
+#pragma unroll
+        for (int i = 0; i < 4; ++i) L[i] = __ldcg(src + i);
+        uint8_t* xrow = xt + (q4 >> 1) * a.x_atom_bytes + r * 128;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(xrow + ((((q4 & 1) * 4 + i) ^ (r & 7)) * 16)) = L[i];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint2 w[kPieces][2];   // [piece][pc]
+#pragma unroll
+            for (int pc = 0; pc < 2; ++pc) {
+                uint32_t y[4];   // the pair k = 8i + 4h + 2pc as an f16 pair
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t v = (h == 0) ? (pc == 0 ? L[i].x : L[i].y) : (pc == 0 ? L[i].z : L[i].w);
+                    if constexpr (kF16) {
+                        y[i] = v;
+                    } else {
+                        if (((v & 0x7FFFu) >= 0x4780u) || (((v >> 16) & 0x7FFFu) >= 0x4780u)) out_of_range = true;
+                        const __half2 lim = __floats2half2_rn(65504.f, 65504.f);
+                        const __half2 hv = __hmax2(__hmin2(__floats2half2_rn(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u)), lim), __hneg2(lim));
+                        y[i] = *reinterpret_cast<const uint32_t*>(&hv);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kPieces; ++q) {
+                    uint32_t pq[4];   // byte 1 / byte 3: the e5m2 piece of k / k+1
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        pq[i] = y[i] & 0xFF00FF00u;
+                        if (q + 1 < kPieces) {
+                            const __half2 d = __hsub2(*reinterpret_cast<const __half2*>(&y[i]), *reinterpret_cast<const __half2*>(&pq[i]));
+                            y[i] = *reinterpret_cast<const uint32_t*>(&d);
+                        }
+                    }
+                    const uint32_t t01 = __byte_perm(pq[0], pq[1], 0x7351);
+                    const uint32_t t23 = __byte_perm(pq[2], pq[3], 0x7351);
+                    w[q][pc] = make_uint2(__byte_perm(t01, t23, 0x5410), __byte_perm(t01, t23, 0x7632));
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < kPieces; ++q) {
+                const int r8 = j * (kPieces * am) + q * am + t;
+                *reinterpret_cast<uint4*>(x8t + r8 * 128 + (((2 * q4 + h) ^ (r8 & 7)) * 16)) = make_uint4(w[q][0].x, w[q][0].y, w[q][1].x, w[q][1].y);
+            }
+        }
+    }
+    if (out_of_range) atomicCAS(&g_device_status[0], 0u, kStatusRange);
+}
+
 // Cluster form: where a block's partial sums go (its own shared memory, [token][128 weight rows] floats).
 struct ClusterPartOut {
     float* part_row;   // &part[0][this thread's weight row]
@@ -165,20 +226,19 @@ __device__ __forceinline__ void epilogue_decode_any_m(const GemmArgs& a, const U
 }
 
 // kMode 1..4: m = kMode tokens per tenant; 5: any m up to 16.  kGen: binary16 I/O, bias, activation.
-// kG = 1: eight decode warps, at most half a multiprocessor per block (flat form); kG = 2: sixteen decode warps, a
-// whole multiprocessor per block (cluster form): four decode warps per scheduler overlap one warp's integer work
-// with the others' tensor-memory stores and waits.
+// kG = 1: at most half a multiprocessor per block (72 registers per thread), units of up to 16 token rows; kG = 2: a
+// whole multiprocessor per block (its rings need more than half of the shared memory), units of up to 32 token rows.
 template <int kMode, bool kGen, int kG>
 __global__ void __launch_bounds__(stream_threads(kG), kG == 1 ? 2 : 1)
 bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmBits,
                             const GemmArgs a) {
-    constexpr int kSDecodeWarps = 8 * kG;
+    constexpr int kSDecodeWarps = 8;
     constexpr int kSWarpEpi0 = kSWarpDecode0 + kSDecodeWarps;
     constexpr int kSThreads = stream_threads(kG);
     constexpr int kSHandover = kSDecodeWarps * 32 + 32;   // decode threads arrive, the issuer warp syncs
-    constexpr int kTenPerWarp = 4 / kG;                   // tenants of a unit a decode warp owns (of up to eight)
-    constexpr int kTenStride = 2 * kG;                    // ... tenant j = kTenStride * i + h for warp half h
-    constexpr int kWarpCols = 64 / kG;                    // ... and its columns of an operand set
+    constexpr int kTenPerWarp = 4;                        // tenants of a unit a decode warp owns (of up to eight)
+    constexpr int kTenStride = 2;                         // ... tenant j = kTenStride * i + h for warp half h
+    constexpr int kWarpCols = 64;                         // ... and its columns of an operand set
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -614,7 +674,10 @@ bitdelta_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW, const __gri
             const uint16_t* xg = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
             uint8_t* xt = smem + x_off + pr.idx * a.x_tile_bytes;
             uint8_t* x8t = smem + x8_off + pr.idx * a.x8_atom_bytes;
-            if (io_f16) split_from_global<true>(a, am, xg, xt, x8t, us.ntok, etid, kSEpiWarps * 32);
+            if (kG == 2 && us.ntok > 8) {
+                if (io_f16) split_from_global_wide<true>(a, am, xg, xt, x8t, us.ntok, etid, kSEpiWarps * 32);
+                else split_from_global_wide<false>(a, am, xg, xt, x8t, us.ntok, etid, kSEpiWarps * 32);
+            } else if (io_f16) split_from_global<true>(a, am, xg, xt, x8t, us.ntok, etid, kSEpiWarps * 32);
             else split_from_global<false>(a, am, xg, xt, x8t, us.ntok, etid, kSEpiWarps * 32);
             fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
             mbar_arrive(smem_u32(&ctl->pfull[pr.idx]));
@@ -837,7 +900,7 @@ extern "C" int bitdelta_debug_set_trace(unsigned long long* buf) {
 cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes, bool early_start,
                                cudaStream_t stream) {
     const int gen = (args.f16 || args.act || args.bias != nullptr) ? 5 : 0;
-    const int big = (args.cluster > 1 && args.decode_warps == 16) ? 10 : 0;   // (experiments: sixteen decode warps)
+    const int big = (smem_bytes > (uint32_t)kStreamSmemBudget) ? 10 : 0;   // one block per multiprocessor: the instantiation with the larger register budget
     const int mode = big + gen + (args.m <= 4 ? args.m : 5) - 1;
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const GemmArgs);
     static const KernelFn kernels[20] = {

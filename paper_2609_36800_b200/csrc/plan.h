@@ -88,10 +88,12 @@ inline bool pair_enabled() {
 
 // The streaming decode kernel (gemm_stream.cu) is taken where it applies when BITDELTA_STREAM=1 is set; the default
 // is the older decode kernel, which measures faster on the decode workloads (18 against 20 us on 8 x 1 x 4096 x 4096).
-inline bool stream_enabled() {
+// BITDELTA_STREAM=2: also for units of up to 32 token rows (which otherwise take the pre-pass split).
+inline int stream_mode() {
     const char* e = getenv("BITDELTA_STREAM");
-    return e && e[0] == '1';
+    return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
 }
+inline bool stream_enabled() { return stream_mode() != 0; }
 
 // The cluster form of the streaming kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
 inline bool cluster_enabled() {
@@ -126,8 +128,9 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
-        p.stream = (p.convert && stream_enabled()) ? 1 : 0;
+        p.stream = (stream_mode() != 0 && p.TB * m <= (stream_mode() == 2 ? 32 : 16)) ? 1 : 0;
         if (p.stream) {
+            p.convert = 1;                              // the splitter threads read X themselves: no pre-pass
             p.x_rows = round_up(p.TB * m, 8);           // (the base MMA's N = 16 may read past it: ignored columns)
             p.x8_rows = round_up(p.TB * kPieces * m, 8);   // (the last tenants' windows run past it: ignored columns)
         }

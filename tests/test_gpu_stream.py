@@ -95,3 +95,21 @@ def test_stream_kernel_general_form_fp16_bias_silu():
     ref = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu")
     max_abs, rel_fro = errors(got, ref)
     assert max_abs <= 2e-2 and rel_fro <= 5e-3, (max_abs, rel_fro)
+
+
+WIDE_SHAPES = [
+    # units of 17..32 token rows: taken by the streaming kernel only with BITDELTA_STREAM=2 (a whole multiprocessor per
+    # block, whole 32-k groups per splitter thread)
+    ((8, 4, 512, 512), 6), ((16, 4, 1024, 1024), 5), ((4, 8, 512, 1024), 6), ((32, 8, 256, 1024), 5),
+    ((8, 3, 640, 384), 5), ((5, 6, 384, 512), 5), ((3, 8, 256, 256), 6), ((2, 16, 384, 512), 6),
+]
+
+
+@pytest.mark.parametrize("shape,schedule", WIDE_SHAPES, ids=[f"B{s[0]}_m{s[1]}_N{s[2]}_K{s[3]}" for s, _ in WIDE_SHAPES])
+def test_stream_kernel_up_to_32_token_rows_per_unit(shape, schedule, monkeypatch):
+    monkeypatch.setenv("BITDELTA_STREAM", "2")
+    B, m, N, K = shape
+    assert bd.gemm_plan(B, m, N, K)["schedule"] == schedule
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B * 1000 + m * 100 + N + K)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    assert_parity(run_gemm(X, W, bits, alpha), oracle.gemm(X, W, bits, alpha), str(shape))
