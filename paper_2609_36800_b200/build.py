@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(HERE, "libbitdelta.so")
-SOURCES = ["api.cu", "gemm_tc.cu", "gemm_stream.cu", "kernels_simple.cu"]
+SOURCES = ["api.cu", "gemm_tc.cu", "gemm_stream.cu", "gemm_fp4.cu", "kernels_simple.cu"]
 HEADERS = ["ptx.cuh", "plan.h", "gemm_tc.h", "gemm_common.cuh", os.path.join("..", "..", "include", "bitdelta.h")]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 

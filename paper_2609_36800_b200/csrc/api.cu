@@ -276,6 +276,9 @@ size_t bitdelta_gemm_workspace_bytes(int B, int m, int N, int K) {
     if (p.decode) {   // the same shape on the tiled schedule (BITDELTA_DTYPE_WIDE_RANGE) may need more
         bd::Plan w = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override(), true, true);
         if (w.ok && w.ws_bytes > need) need = w.ws_bytes;
+        // ... and a call with options (binary16, bias, activation) never takes the 4-bit decode kernel
+        bd::Plan o = bd::make_plan(B, m, N, K, 148, tb_override(), whole_override(), true, false, false);
+        if (o.ok && o.ws_bytes > need) need = o.ws_bytes;
     }
     return need;
 }
@@ -333,7 +336,8 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         return BITDELTA_OK;
     }
 
-    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), true, wide);
+    const bool plain = !f16 && act == BITDELTA_ACT_NONE && bias == nullptr;   // (the 4-bit decode kernel takes no options)
+    bd::Plan p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), true, wide, plain);
     if (p.ok && p.pair) {
         // The pair schedule wants every pair resident at once (a cluster of two needs two free SMs of one
         // cluster-capable group); where the device cannot do that, run the one-CTA schedule.  Asked once per device.
@@ -349,24 +353,25 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
             }
             fit = pairs_cache[di][1] - 1;
         }
-        if (2 * fit < p.grid) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, wide);
+        if (2 * fit < p.grid) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, wide, plain);
     }
     if (p.ok && p.cluster > 1) {
         // The cluster form wants all its clusters resident at once (clusters are independent, so this is about
         // speed, not progress); where the device cannot hold them, the flat work list is planned.
         static std::mutex mu;
-        static int fit_cache[64][4][2] = {};   // [device][log2 cluster][smem above half a multiprocessor]: 0 unknown, else n + 1
+        static int fit_cache[64][4][3] = {};   // [device][log2 cluster][smem above half a multiprocessor; 2: the 4-bit kernel]: 0 unknown, else n + 1
         const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
         const int ci = p.cluster == 8 ? 3 : (p.cluster == 4 ? 2 : 1);
-        const int si = p.smem_bytes > (uint32_t)bd::kStreamSmemBudget ? 1 : 0;
+        const int si = p.fp4 ? 2 : (p.smem_bytes > (uint32_t)bd::kStreamSmemBudget ? 1 : 0);
         int n;
         {
             std::lock_guard<std::mutex> lock(mu);
-            if (fit_cache[di][ci][si] == 0) fit_cache[di][ci][si] = bd::stream_max_active_clusters(p.smem_bytes, p.cluster) + 1;
+            if (fit_cache[di][ci][si] == 0)
+                fit_cache[di][ci][si] = (p.fp4 ? bd::fp4_max_active_clusters(p.smem_bytes, p.cluster) : bd::stream_max_active_clusters(p.smem_bytes, p.cluster)) + 1;
             n = fit_cache[di][ci][si] - 1;
         }
         const int need = p.grid / p.cluster;
-        if (n < need) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false);
+        if (n < need) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, false, plain);
     }
     if (!p.ok) return BITDELTA_ERR_SHAPE;
     if (!workspace || workspace_bytes < p.ws_bytes) return BITDELTA_ERR_WORKSPACE;
@@ -379,11 +384,21 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     if (!p.stream && !cached_map(&tmX, MapKey{0, X, (uint64_t)B * m, (uint64_t)K, 0, (uint32_t)p.x_rows, 0u},
                                  [&](CUtensorMap* mp) { return encode_bf16_tile(mp, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows); }))
         return BITDELTA_ERR_CUDA;
-    const uint32_t box_words = p.stream ? 4u : 8u;
+    const uint32_t box_words = (p.stream && !p.fp4) ? 4u : 8u;
     if (!cached_map(&tmBits, MapKey{1, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words},
                     [&](CUtensorMap* mp) { return encode_bits_3d(mp, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words); }))
         return BITDELTA_ERR_CUDA;
-    if (p.decode && !p.convert) {
+    if (p.fp4) {
+        // 4-bit decode kernel: the activation operands of every (tenant group, 128-k step) as shared-memory images, and
+        // the token rows' fixed-point units; then the GEMM, which prefetches weights while this is still running.
+        uint8_t* img = bd::ws_x8(p, workspace);
+        static const bool skip_prepass = getenv("BITDELTA_FP4_SKIP_PREPASS") != nullptr;   // WHATIF (timing experiments)
+        // (its early start is always safe: it waits for its predecessor before it touches anything)
+        if (!skip_prepass && !p.convert && bd::launch_x_split_fp4(X, img, reinterpret_cast<float*>(img + p.ws_scale_off), p, early_start_enabled(), stream) != cudaSuccess)
+            return BITDELTA_ERR_CUDA;
+        if (!p.convert) g_launches++;
+        tmX8 = tmW;   // not read
+    } else if (p.decode && !p.convert) {
         // Decode schedule with many token rows per tile: split the activations into e5m2 pieces first
         // (tiny), then the GEMM, which may start prefetching weights while the split is still running.
         uint8_t* x8 = bd::ws_x8(p, workspace);
@@ -411,7 +426,9 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_PREFETCH"); d = e ? atoi(e) : 0; } args.prefetch_steps = d; }
     // (a GEMM queued right behind the library's own pack / compress must not prefetch what they are still writing)
     const bool early = early_start_enabled() && g_weights_just_written.exchange(0) == 0;
-    const cudaError_t le = p.stream
+    const cudaError_t le = p.fp4
+        ? bd::launch_gemm_fp4(tmW, tmBits, args, p.grid, p.smem_bytes, early, stream)
+        : p.stream
         ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early, stream)
         : bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early, stream);
     if (le != cudaSuccess) return BITDELTA_ERR_CUDA;
@@ -478,7 +495,7 @@ int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
     if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
-    info[0] = !p.decode ? (p.pair ? 4 : 0) : (p.stream ? (p.cluster > 1 ? 6 : 5) : (p.convert ? 2 : 1));
+    info[0] = !p.decode ? (p.pair ? 4 : 0) : p.fp4 ? (p.cluster > 1 ? 8 : 7) : (p.stream ? (p.cluster > 1 ? 6 : 5) : (p.convert ? 2 : 1));
     info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
     info[5] = p.cluster > 1 ? 3 : (p.whole_units ? 1 : (p.teams > 1 ? 2 : 0));
     info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;

@@ -1,0 +1,969 @@
+// BitDelta fused GEMM, 4-bit decode schedule (few token rows per unit) on tcgen05 tensor cores.
+//
+//   Y[b,t,n] = sum_k X[b,t,k] W[n,k] + alpha[b] sum_k X[b,t,k] S[b,n,k]
+//
+// Same orientation, roles and work split as the streaming decode kernel (gemm_stream.cu), but the delta term
+// runs on the block-scaled 4-bit tensor path (tcgen05.mma kind::mxf4, K = 64 per instruction):
+//   * Signs are decoded to e2m1 (+1 = 0x2, -1 = 0xA), EIGHT per 32-bit register: per sign word three shifts and four
+//     logic operations, four tensor-memory columns.  That is half the integer work and half the tensor-memory store
+//     traffic of the 8-bit form, the two things that bound the decode schedules, and half the MMA instructions.
+//     Register c of a word holds in nibble i the sign of k = 4i + c.
+//   * Activations: a token row's values are written as 16-bit fixed point relative to the row's largest exponent E
+//     (|x| = v * 2^(E-142), v < 2^16: every value within 8 binades of the row's largest is exact, smaller ones are
+//     truncated below 2^-16 of it) and v as eight radix-4 digits 0..3; a digit d goes into the operand as the e2m1
+//     value d/2, whose 4-bit code is d itself, with the value's sign in the code's sign bit.  Digit q of all tokens
+//     forms row block q of the MMA's B operand; its weight 4^q is the B-side SCALE FACTOR of those rows (ue8m0
+//     127 + 2q, the same for every k: written to tensor memory once per launch), the A-side scale is 1, so a
+//     tenant's delta is the plain sum of its eight accumulator column groups times the row's unit 2^(E-141), which
+//     the epilogue applies together with alpha.  No value of the 16-bit input range saturates or is flagged.  (E is
+//     taken over the whole row by the pre-pass, over a block's k range when the kernel splits the activations.)
+//   * Units of more than 16 token rows: a pre-pass kernel writes, per tenant group and 128-k step, the
+//     shared-memory IMAGE of both activation operands (16-bit tile of the base MMA with its 128-byte swizzle, digit
+//     rows with the 64-byte swizzle); the producer fetches an image with one plain bulk copy.  Units of up to 16 token
+//     rows: the four epilogue warps write the same image straight into shared memory from X.
+// One block per multiprocessor (it needs most of the shared memory), 16 warps: producer, THREE MMA issuers (base; delta
+// of the even and of the odd tenants), eight decode warps, four epilogue warps.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <type_traits>
+
+#include "gemm_common.cuh"
+#include "gemm_tc.h"
+#include "ptx.cuh"
+
+namespace bd {
+
+constexpr int kFWarpProducer = 0;
+constexpr int kFWarpMma = 1;                     // base MMAs (A = W_base tile in shared memory)
+constexpr int kFWarpDelta0 = 2;                  // warps 2, 3: delta MMAs of the even / odd tenants (A = signs in tensor memory)
+constexpr int kFWarpDecode0 = 4;                 // warps 4 .. 11 decode
+constexpr int kFDecodeWarps = 8;
+constexpr int kFWarpEpi0 = kFWarpDecode0 + kFDecodeWarps;
+constexpr int kFEpiWarps = 4;
+constexpr int kFThreads = (kFWarpEpi0 + kFEpiWarps) * 32;   // 512
+constexpr int kFHandover = kFDecodeWarps / 2 * 32 + 32;      // the four decode warps of a tenant half arrive, its issuer warp syncs
+constexpr int kFBarSet0 = 2;                     // named barrier of operand set s, tenant half h: id 2 + 2 s + h
+constexpr int kFBarDep = 15;                     // the decode and epilogue warps sleep on it until the grid dependency resolves
+
+#ifdef BD_TRACE
+// Trace build: per block 32 accumulators (cycles) written at the end of each role; see bitdelta_debug_set_trace_fp4.
+__device__ long long* g_fp4_trace = nullptr;
+#define FT_DECL(n) long long ft_acc[n] = {}; long long ft_t0 = clock64()
+#define FT_ADD(i) do { const long long ft_t1 = clock64(); ft_acc[i] += ft_t1 - ft_t0; ft_t0 = ft_t1; } while (0)
+#define FT_OUT(base, n) do { if (g_fp4_trace && lane == 0) for (int ft_i = 0; ft_i < (n); ++ft_i) g_fp4_trace[(size_t)blockIdx.x * 32 + (base) + ft_i] = ft_acc[ft_i]; } while (0)
+#else
+#define FT_DECL(n) do { } while (0)
+#define FT_ADD(i) do { } while (0)
+#define FT_OUT(base, n) do { } while (0)
+#endif
+
+struct FCtl {
+    uint64_t wfull[kMaxStages];     // W_base tile landed
+    uint64_t wempty[kMaxStages];    // ... and was read by its base MMAs
+    uint64_t bfull[4];              // sign words of two 128-k steps landed
+    uint64_t bempty[4];             // ... and are in the decode warps' registers (8 arrivals)
+    uint64_t pfull[4];              // a step's activation image landed
+    uint64_t pempty[4];             // ... and was read by the step's MMAs
+    uint64_t opfree[2][kStreamMaxSets];   // tenant half h's columns of an operand set in tensor memory free again
+    uint64_t accfull;               // all MMAs of a segment have completed
+    uint64_t accempty;              // the accumulators were drained (4 epilogue warps)
+    uint64_t depready;              // the grid this launch depends on has completed
+    uint64_t tmemready;             // tensor memory is allocated (its base address is in tmem_base)
+    uint64_t sfready;               // the scale factors are in tensor memory (4 epilogue warps)
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t is_last;
+    float xs[64];                   // fixed-point units of the token rows: four segments in flight x 16 rows (the kernel
+                                    // splits), or two x 32 rows (pre-pass)
+    uint32_t emax[4][16];           // the kernel splits: the rows' largest magnitudes (16-bit patterns) of those segments
+};
+static_assert(sizeof(FCtl) <= kSmemCtrlBytes, "control block too large");
+
+// Eight signs per register: register c, nibble i <- bit 4i + c of the word (1 -> +1.0 = 0x2, 0 -> -1.0 = 0xA).
+__device__ __forceinline__ void decode_word_e2m1(uint32_t w, uint32_t* r) {
+    r[0] = ((w << 3) & 0x88888888u) ^ 0xAAAAAAAAu;
+    r[1] = ((w << 2) & 0x88888888u) ^ 0xAAAAAAAAu;
+    r[2] = ((w << 1) & 0x88888888u) ^ 0xAAAAAAAAu;
+    r[3] = (w & 0x88888888u) ^ 0xAAAAAAAAu;
+}
+
+// Eight 16-bit values hv[i] of one token row (k = k0 + 4i) -> for every digit q the register R[q] whose nibble i is
+// the operand code of value i: sign << 3 | digit q of its 16-bit fixed-point magnitude (E: the row's exponent).
+__device__ __forceinline__ void fp4_digits8(const uint32_t* hv, int E, uint32_t* R) {
+    uint32_t T[8];   // T[i]: nibble q = code of digit q of value i
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int ex = (int)((hv[i] >> 7) & 0xFFu);
+        const uint32_t m8 = (hv[i] & 0x7Fu) | (ex ? 0x80u : 0u);
+        uint32_t t = (m8 << 8) >> min(E - max(ex, 1), 31);
+        t = (t | (t << 8)) & 0x00FF00FFu;    // 8 bits per 16-bit lane
+        t = (t | (t << 4)) & 0x0F0F0F0Fu;    // 4 bits per byte
+        t = (t | (t << 2)) & 0x33333333u;    // 2 bits per nibble
+        T[i] = t | ((hv[i] & 0x8000u) ? 0x88888888u : 0u);
+    }
+    // 8 x 8 nibble transpose: 16-bit halves between registers i, i+4; bytes between i, i+2; nibbles between i, i+1
+    uint32_t A[8], Bv[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        A[i] = __byte_perm(T[i], T[i + 4], 0x5410);
+        A[i + 4] = __byte_perm(T[i], T[i + 4], 0x7632);
+    }
+#pragma unroll
+    for (int g = 0; g < 8; g += 4) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            Bv[g + i] = __byte_perm(A[g + i], A[g + i + 2], 0x6240);
+            Bv[g + i + 2] = __byte_perm(A[g + i], A[g + i + 2], 0x7351);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < 8; g += 2) {
+        R[g] = (Bv[g] & 0x0F0F0F0Fu) | ((Bv[g + 1] & 0x0F0F0F0Fu) << 4);
+        R[g + 1] = ((Bv[g] >> 4) & 0x0F0F0F0Fu) | (Bv[g + 1] & 0xF0F0F0F0u);
+    }
+}
+
+// One task of the activation split: of token row `xrow` (row r_local = j*m + t of its unit) the 16-byte chunk `tk`
+// of a 128-k step (k = 8 tk .. 8 tk + 7) goes to the 16-bit tile, and the eight values k = 32 wd + 4i + c (wd = tk / 4,
+// c = tk % 4) to the digit rows j*8m + q*m + t: register c of word wd, the order in which decode_word_e2m1 lays out
+// the signs.  `xstep`: the row's first value of the step; `im`: the step's image (global or shared memory).
+__device__ __forceinline__ void fp4_split_task(const uint16_t* __restrict__ xstep, uint8_t* im, int tk, int r_local, int j, int t,
+                                               int m, int E, uint32_t x_atom_bytes, uint32_t x_tile_bytes) {
+    const uint4 chunk = __ldcg(reinterpret_cast<const uint4*>(xstep) + tk);
+    *reinterpret_cast<uint4*>(im + (tk >> 3) * x_atom_bytes + r_local * 128 + (((tk & 7) ^ (r_local & 7)) * 16)) = chunk;
+    const int wd = tk >> 2, c = tk & 3;
+    uint32_t hv[8], R[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) hv[i] = __ldcg(xstep + 32 * wd + 4 * i + c);
+    fp4_digits8(hv, E, R);
+#pragma unroll
+    for (int q = 0; q < kFp4Pieces; ++q) {
+        const int n = j * (kFp4Pieces * m) + q * m + t;
+        *reinterpret_cast<uint32_t*>(im + x_tile_bytes + n * 64 + ((wd ^ ((n >> 1) & 3)) * 16) + 4 * c) = R[q];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- pre-pass
+// One block per token row.  Phase 1: the row's largest exponent E (biased, subnormals as 1); its fixed-point unit
+// 2^(E-141) goes to xscale.  Phase 2: the row's share of every step's image.
+__global__ void __launch_bounds__(256) x_split_fp4_kernel(const uint16_t* __restrict__ X, uint8_t* __restrict__ img,
+                                                          float* __restrict__ xscale, int m, int K, int TB, int P,
+                                                          uint32_t img_bytes, uint32_t x_atom_bytes, uint32_t x_tile_bytes) {
+    __shared__ uint32_t red[8];
+    // Launched with an early start: the GEMM queued behind this kernel may become resident at once (it prefetches
+    // weights and waits for this kernel before it reads an image); this kernel itself reads X and overwrites the
+    // images only after the kernel before it (possibly the previous GEMM, still reading them) has completed.
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int row = blockIdx.x;
+    const int b = row / m, t = row - b * m;
+    const int g = b / TB, j = b - g * TB;
+    const int r_local = j * m + t;
+    const uint16_t* x = X + (size_t)row * K;
+    const uint4* x4 = reinterpret_cast<const uint4*>(x);
+    uint32_t mx2 = 0;
+    for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
+        const uint4 v = __ldcg(x4 + i);
+        mx2 = __vmaxu2(mx2, __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)));
+    }
+    uint32_t mx = max(mx2 & 0xFFFFu, mx2 >> 16);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) mx = max(mx, red[w]);
+    const int E = max((int)(mx >> 7), 1);
+    if (threadIdx.x == 0) xscale[row] = ldexpf(1.f, E - 141);
+
+    uint8_t* img_g = img + (size_t)g * P * img_bytes;
+    for (int task = threadIdx.x; task < K / 8; task += blockDim.x) {
+        const int p = task >> 4;
+        fp4_split_task(x + (size_t)p * kPairK, img_g + (size_t)p * img_bytes, task & 15, r_local, j, t, m, E, x_atom_bytes, x_tile_bytes);
+    }
+}
+
+cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, float* xscale, const Plan& p, bool early_start, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.B * p.m));
+    cfg.blockDim = dim3(256u);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early_start ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, x_split_fp4_kernel, reinterpret_cast<const uint16_t*>(X), img, xscale, p.m, p.K, p.TB, p.P,
+                              p.img_bytes, p.x_atom_bytes, p.x_tile_bytes);
+}
+
+// Epilogue of one segment, M tokens per tenant: base accumulator columns j*M + t, tenant j's delta accumulator from
+// column 8M*j, digit q of token t in column q*M + t (already weighted 4^q by its scale factor).
+//   out(j*M + t) = base + alpha_j * (xs[j*M + t] * sum_q D[q*M + t])
+template <int M, class Out>
+__device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
+                                             const float* alv, const float* xs_smem) {
+    constexpr int ND = kFp4Pieces * M;
+    uint32_t rb[32];
+    if (a.Nb <= 16) tmem_ld16(lane_taddr, rb);
+    else tmem_ld32(lane_taddr, rb);
+#pragma unroll 1
+    for (int j = 0; j < u.nten; ++j) {
+        uint32_t rd[ND];
+        const uint32_t col = lane_taddr + a.col_delta + (uint32_t)(j * ND);
+        if constexpr (ND >= 32) {
+#pragma unroll
+            for (int c = 0; c + 32 <= ND; c += 32) tmem_ld32(col + c, rd + c);
+        }
+        if constexpr (ND % 32 >= 16) tmem_ld16(col + ND / 32 * 32, rd + ND / 32 * 32);
+        if constexpr (ND % 16 >= 8) tmem_ld8(col + ND / 16 * 16, rd + ND / 16 * 16);
+        tc_wait_ld();
+        const float al = alv[j];
+#pragma unroll
+        for (int t = 0; t < M; ++t) {
+            float d = 0.f;
+#pragma unroll
+            for (int q = 0; q < kFp4Pieces; ++q) d += __uint_as_float(rd[q * M + t]);
+            // (rb is indexed with a run-time tenant: select, do not index, so that it stays in registers)
+            float base = 0.f;
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+                if (c == j * M + t) base = __uint_as_float(rb[c]);
+            out.put(j * M + t, fmaf(al, d * xs_smem[j * M + t], base));
+        }
+    }
+}
+
+template <class Out>
+__device__ __forceinline__ void epilogue_fp4_any_m(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
+                                                   const float* alv, const float* xs_smem, int am) {
+    switch (am) {
+        case 1: epilogue_fp4<1>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 2: epilogue_fp4<2>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 3: epilogue_fp4<3>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 4: epilogue_fp4<4>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 5: epilogue_fp4<5>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 6: epilogue_fp4<6>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 7: epilogue_fp4<7>(a, u, lane_taddr, out, alv, xs_smem); break;
+        default: epilogue_fp4<8>(a, u, lane_taddr, out, alv, xs_smem); break;
+    }
+}
+
+// Cluster form: where a block's partial sums go (its own shared memory, [token][128 weight rows] floats).
+struct FClusterPartOut {
+    float* part_row;   // &part[0][this thread's weight row]
+    __device__ __forceinline__ void put(int tok, float v) const { part_row[tok * kTileN] = v; }
+};
+
+// kTB8: units of up to eight tenants (m <= 4): two operand sets per 128-k step, a set = all tenants x 64 k; else up to
+// four tenants (m <= 8): one set per step, a set = all tenants x 128 k.  Either way a decode warp stores 32 columns per
+// set: warp (quad, h) owns the weight rows of lane quadrant `quad` and the tenants j = 2i + h.
+template <bool kTB8>
+__global__ void __launch_bounds__(kFThreads, 1)
+bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmBits, const GemmArgs a) {
+    constexpr int kSetsPerStep = kTB8 ? 2 : 1;
+    constexpr int kTenPerWarp = kTB8 ? 4 : 2;
+    constexpr int kTenCols = kTB8 ? 8 : 16;            // columns of one tenant in a set
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t w_addr = base;                                          // ring of W_base tiles
+    const uint32_t bits_off = a.n_w * a.w_stage_bytes;                     // sign-word slots (two steps each)
+    const uint32_t bits_addr = base + bits_off;
+    const uint32_t img_off = bits_off + a.n_bits * a.bslot_bytes;          // ring of activation images
+    const uint32_t img_addr = base + img_off;
+    FCtl* ctl = reinterpret_cast<FCtl*>(smem + img_off + a.n_img * a.img_bytes);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const int am = a.m;
+    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<true, false, false>(aa, un, am, 0); };
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 32) {
+        prefetch_tensormap(&tmW);
+        prefetch_tensormap(&tmBits);
+    }
+
+    // Work: an even share of the flat (unit, k-step) list (or whole units round-robin), or, in the cluster form,
+    // this block's share of the k-steps of its cluster's unit.
+    const int crank = (a.cluster > 1) ? (int)cluster_ctarank() : 0;
+    int lo, hi;
+    if (a.cluster > 1) {
+        const int cunit = (int)blockIdx.x / a.cluster;
+        lo = cunit * a.P + (crank * a.P) / a.cluster;
+        hi = cunit * a.P + ((crank + 1) * a.P) / a.cluster;
+    } else {
+        lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
+        hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
+    }
+    SegIter it{lo, hi, a.P, (a.whole_units && a.cluster <= 1) ? (int)gridDim.x : 0};
+    int unit, p0, p1;
+
+    // The W_base tile of a step (128 rows x 128 k: both 64-k atoms) in one bulk-tensor copy.  One thread.
+    auto issue_w = [&](const Unit& u, int p, int stage) {
+        const uint32_t bar = smem_u32(&ctl->wfull[stage]);
+        if (a.prefetch_steps & 4) { mbar_arrive(bar); return; }   // WHATIF
+        mbar_arrive_expect_tx(bar, a.w_stage_bytes);
+        tma_load_3d(w_addr + stage * a.w_stage_bytes, &tmW, bar, 0, u.n0, p * (kPairK / kAtomK));
+    };
+    // The sign words of the two steps 2*(p/2), 2*(p/2)+1 for all the unit's tenants: one bulk-tensor copy (rows of
+    // 32 bytes).  One thread.
+    auto issue_bits = [&](const Unit& u, int p, int bslot) {
+        const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
+        if (a.prefetch_steps & 2) { mbar_arrive(bar); return; }   // WHATIF
+        mbar_arrive_expect_tx(bar, a.bslot_bytes);
+        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+    };
+    // The activation image of a step (written by the pre-pass kernel): one plain bulk copy.  One thread.
+    auto issue_img = [&](const Unit& u, int p, int slot) {
+        const uint32_t bar = smem_u32(&ctl->pfull[slot]);
+        if (a.prefetch_steps & 1) { mbar_arrive(bar); return; }   // WHATIF
+        mbar_arrive_expect_tx(bar, a.img_bytes);
+        const int g = (int)((unsigned)u.tenant0 / (unsigned)a.TB);
+        bulk_load(img_addr + slot * a.img_bytes, a.img + ((size_t)g * a.P + p) * a.img_bytes, a.img_bytes, bar);
+    };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&ctl->wfull[s]), 1);
+            mbar_init(smem_u32(&ctl->wempty[s]), 1);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&ctl->bfull[s]), 1);
+            mbar_init(smem_u32(&ctl->bempty[s]), kFDecodeWarps);
+            mbar_init(smem_u32(&ctl->pfull[s]), a.convert ? kFEpiWarps * 32 : 1);   // splitter threads, or one bulk copy
+            mbar_init(smem_u32(&ctl->pempty[s]), 3);   // (the three issuers)
+        }
+        for (int s = 0; s < kStreamMaxSets; ++s) {
+            mbar_init(smem_u32(&ctl->opfree[0][s]), 1);
+            mbar_init(smem_u32(&ctl->opfree[1][s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->accfull), 3);   // (the three issuers)
+        mbar_init(smem_u32(&ctl->accempty), kFEpiWarps);
+        mbar_init(smem_u32(&ctl->depready), 1);
+        mbar_init(smem_u32(&ctl->tmemready), 1);
+        mbar_init(smem_u32(&ctl->sfready), kFEpiWarps);
+        ctl->abort_flag = 0;
+        ctl->is_last = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    const uint32_t tmemready = smem_u32(&ctl->tmemready);
+
+    if (warp == kFWarpProducer) {
+        // ------------------------------------------------------------ producer
+        // Walks the block's steps three times over, once per stream: W_base tiles and sign words (never written by
+        // another kernel: queued before the grid dependency is resolved, as far as their rings allow) and activation
+        // images (written by the pre-pass kernel queued before this one: only afterwards).
+        ItemIter wi(it), bi(it), xi(it);
+        Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, a.n_img};
+        Unit uw{}, ub{}, ux{};
+        bool more_w = wi.next(), more_b = bi.next(), more_x = !a.convert && xi.next();   // (convert: the epilogue warps write the images)
+        if (more_w) { uw = unit_info(a, wi.unit); ub = uw; ux = uw; }
+        long long t_idle = 0;
+        int idle = 0;
+        bool dep_done = false;
+        while (more_w || more_b || more_x) {
+            bool did = false;
+            if (more_b && warp_all(mbar_test_wait(smem_u32(&ctl->bempty[br.idx]), br.par ^ 1))) {
+                if (elect_one()) issue_bits(ub, bi.p, br.idx);
+                __syncwarp();
+                br.step();
+                // the slot also covers the next step if that is the odd step of the same pair and of the same segment
+                const bool odd_next = ((bi.p & 1) == 0) && (bi.p + 1 < bi.p1);
+                more_b = bi.next();
+                if (more_b && odd_next) more_b = bi.next();
+                if (more_b && bi.first) ub = unit_info(a, bi.unit);
+                did = true;
+            }
+            if (more_w && warp_all(mbar_test_wait(smem_u32(&ctl->wempty[wr.idx]), wr.par ^ 1))) {
+                if (elect_one()) issue_w(uw, wi.p, wr.idx);
+                __syncwarp();
+                wr.step();
+                more_w = wi.next();
+                if (more_w && wi.first) uw = unit_info(a, wi.unit);
+                did = true;
+            }
+            if (dep_done && more_x && warp_all(mbar_test_wait(smem_u32(&ctl->pempty[xr.idx]), xr.par ^ 1))) {
+                if (elect_one()) issue_img(ux, xi.p, xr.idx);
+                __syncwarp();
+                xr.step();
+                more_x = xi.next();
+                if (more_x && xi.first) ux = unit_info(a, xi.unit);
+                did = true;
+            }
+            if (did) {
+                idle = 0;
+                continue;
+            }
+            if (!dep_done) {
+                // the weight rings are full and stay full until the grid dependency resolves: sleep until then
+                dep_done = warp_all(mbar_try_wait_hint(smem_u32(&ctl->depready), 0u, 20000u));
+                continue;
+            }
+            if (more_x) (void)mbar_try_wait_hint(smem_u32(&ctl->pempty[xr.idx]), xr.par ^ 1, 64u);
+            else if (more_b) (void)mbar_try_wait_hint(smem_u32(&ctl->bempty[br.idx]), br.par ^ 1, 64u);
+            else (void)mbar_try_wait_hint(smem_u32(&ctl->wempty[wr.idx]), wr.par ^ 1, 64u);
+            if (idle == 0) t_idle = clock64();
+            if ((++idle & 255) == 0) {
+                if (*abort_flag) break;
+                if (clock64() - t_idle > kWaitLimitCycles) {
+                    *abort_flag = 1;
+                    if (atomicCAS(&g_device_status[0], 0u, kStatusTimeout) == 0u) g_device_status[1] = 2u;
+                    break;
+                }
+            }
+        }
+        // All of this block's loads are queued: a kernel queued behind this one with an early start may become resident.
+        if (lane == 0) grid_launch_dependents();
+    } else if (warp == kFWarpMma) {
+        // -------------------------------------------------------------- MMA issuer
+        grid_dependency_wait();
+        named_bar_arrive(kFBarDep, kFThreads - 32);   // wakes the decode and epilogue warps
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));   // ... and the producer
+        tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+        tmem_relinquish();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tmemready);
+        (void)wait_bar(tmemready, 0, abort_flag, 20);
+        tc_fence_after();
+        const uint32_t tmem_base = ctl->tmem_base;
+        bool ok = true;
+
+        const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
+        const uint64_t desc128 = make_smem_desc_sw128(0);
+        const uint32_t x_atom16 = a.x_atom_bytes >> 4;
+        Ring wr{0, 0u, a.n_w}, pr{0, 0u, a.n_img};
+        uint32_t accphase = 0;
+        FT_DECL(8);
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            FT_ADD(0);
+            ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            FT_ADD(1);
+            if (!ok) break;
+            tc_fence_after();
+            for (int p = p0; p < p1 && ok; ++p) {
+                const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this step starts the accumulation
+                FT_ADD(0);
+                ok = warp_all(wait_bar(smem_u32(&ctl->pfull[pr.idx]), pr.par, abort_flag, 13));
+                FT_ADD(2);
+                if (!ok) break;
+                const uint32_t img_s = img_addr + pr.idx * a.img_bytes;
+                const uint64_t xdesc = desc128 + (img_s >> 4);
+                ok = warp_all(wait_bar(smem_u32(&ctl->wfull[wr.idx]), wr.par, abort_flag, 4));
+                FT_ADD(3);
+                if (!ok) break;
+                {
+                    const uint64_t wdesc = desc128 + ((w_addr + wr.idx * a.w_stage_bytes) >> 4);
+                    if (elect_one()) {
+                        if (!(a.prefetch_steps & 32))   // WHATIF
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t atom = kk >> 2, k16 = kk & 3;
+                            umma_ss(tmem_base, wdesc + (atom * (a.w_atom_bytes >> 4) + k16 * 2), xdesc + (atom * x_atom16 + k16 * 2),
+                                    idesc_base, (kk > 0) ? 1u : first);
+                        }
+                        tc_commit(smem_u32(&ctl->wempty[wr.idx]));
+                    }
+                    __syncwarp();
+                    wr.step();
+                }
+                if (!ok) break;
+                if (elect_one()) tc_commit(smem_u32(&ctl->pempty[pr.idx]));
+                __syncwarp();
+                pr.step();
+            }
+            if (!ok) break;
+            if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
+            __syncwarp();
+            accphase ^= 1;
+        }
+        FT_ADD(0);
+        FT_OUT(0, 8);
+    } else if (warp < kFWarpDecode0) {
+        // -------------------------------------------------------------- delta MMA issuers
+        // Warp 2 + h issues the delta MMAs of the tenants j = 2i + h (A = their decoded signs, filled by the four decode
+        // warps of half h).  One thread issues a tcgen05 instruction every ~50 cycles whatever its size, so three
+        // issuing threads (this pair and the base issuer) are what keeps the per-step instruction count off the
+        // critical path.
+        const int h = warp - kFWarpDelta0;
+        named_bar_sync(kFBarDep, kFThreads - 32);
+        bool ok = warp_all(wait_bar(tmemready, 0, abort_flag, 20));
+        tc_fence_after();
+        const uint32_t tmem_base = ctl->tmem_base;
+        ok = ok && warp_all(wait_bar(smem_u32(&ctl->sfready), 0, abort_flag, 22));   // scale factors written
+        tc_fence_after();
+        const uint32_t idesc_delta = make_idesc_mxf4(kTileN, (uint32_t)a.Nd);
+        const uint64_t desc64 = make_smem_desc_sw64(0);
+        const uint32_t ten_rows16 = (uint32_t)a.Nd * 4u;      // a tenant's digit rows x 64 B >> 4
+        const uint32_t sfa = tmem_base + a.col_sf, sfb = sfa + 4u;
+        Ring pr{0, 0u, a.n_img}, sr{0, 0u, a.n_sets};
+        uint32_t accphase = 0;
+        FT_DECL(8);
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            FT_ADD(0);
+            ok = warp_all(wait_bar(smem_u32(&ctl->accempty), accphase ^ 1, abort_flag, 3));
+            FT_ADD(1);
+            if (!ok) break;
+            tc_fence_after();
+            for (int p = p0; p < p1 && ok; ++p) {
+                const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this step starts the accumulation
+                FT_ADD(0);
+                ok = warp_all(wait_bar(smem_u32(&ctl->pfull[pr.idx]), pr.par, abort_flag, 13));
+                FT_ADD(2);
+                if (!ok) break;
+                const uint64_t x4desc = desc64 + ((img_addr + pr.idx * a.img_bytes + a.x_tile_bytes) >> 4);
+#pragma unroll
+                for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
+                    // The 128 decode threads of this half arrive here once their columns of the set are filled (or when
+                    // they give up after an abandoned wait, see the end of the decode role).
+                    FT_ADD(0);
+                    named_bar_sync(kFBarSet0 + 2 * sr.idx + h, kFHandover);
+                    FT_ADD(4);
+                    if (*abort_flag) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_set = tmem_base + a.col_a + (uint32_t)sr.idx * kFp4SetCols + (uint32_t)(h * 32);
+                    if (elect_one()) {
+                        for (int j = h; j < u.nten; j += 2) {
+                            const uint32_t a_j = a_set + (uint32_t)((j >> 1) * kTenCols);
+                            const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
+                            const uint64_t xj = x4desc + (uint32_t)j * ten_rows16;
+                            if constexpr (kTB8) {
+                                umma_ts_mxf4(d_tmem, a_j, xj + (uint32_t)(s * 2), idesc_delta, sfa, sfb, (s > 0) ? 1u : first);
+                            } else {
+                                umma_ts_mxf4(d_tmem, a_j, xj, idesc_delta, sfa, sfb, first);
+                                umma_ts_mxf4(d_tmem, a_j + 8, xj + 2, idesc_delta, sfa, sfb, 1u);
+                            }
+                        }
+                        tc_commit(smem_u32(&ctl->opfree[h][sr.idx]));
+                    }
+                    __syncwarp();
+                }
+                if (!ok) break;
+                if (elect_one()) tc_commit(smem_u32(&ctl->pempty[pr.idx]));
+                __syncwarp();
+                pr.step();
+            }
+            if (!ok) break;
+            if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
+            __syncwarp();
+            accphase ^= 1;
+        }
+        FT_ADD(0);
+        if (h == 0) FT_OUT(24, 8);
+    } else if (warp < kFWarpEpi0) {
+        // ------------------------------------------- sign decode -> tensor memory
+        const int h = (warp - kFWarpDecode0) >> 2;
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        named_bar_sync(kFBarDep, kFThreads - 32);   // (sleeps while the launch before this one is still running)
+        bool ok = wait_bar(tmemready, 0, abort_flag, 20);
+        tc_fence_after();
+        const uint32_t tmem_base = ctl->tmem_base;
+        const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * 32);
+        Ring br{0, 0u, a.n_bits}, sr{0, 0u, a.n_sets};
+        int pending = -1;
+        FT_DECL(8);
+        while (ok && it.next(unit, p0, p1)) {
+            for (int p = p0; p < p1 && ok; ++p) {
+                // a slot holds the steps 2*(p/2) and 2*(p/2)+1: waited for at the first step of it that this segment takes
+                if (p == p0 || (p & 1) == 0) {
+                    FT_ADD(0);
+                    ok = wait_bar(smem_u32(&ctl->bfull[br.idx]), br.par, abort_flag, 6);
+                    FT_ADD(1);
+                    if (!ok) break;
+                }
+                // this warp's tenants j = 2i + h: their sign words of the step (128 k each)
+                const uint8_t* bsl = smem + bits_off + br.idx * a.bslot_bytes + row * 32 + (p & 1) * 16;
+                uint4 wq[kTenPerWarp];
+#pragma unroll
+                for (int i = 0; i < kTenPerWarp; ++i) wq[i] = *reinterpret_cast<const uint4*>(bsl + (2 * i + h) * (kTileN * 32));
+#pragma unroll
+                for (int i = 0; i < kTenPerWarp; ++i) asm volatile("" : "+r"(wq[i].x), "+r"(wq[i].w));
+                if ((p & 1) == 1 || p + 1 == p1) {   // the slot's last step in this segment: it goes back
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->bempty[br.idx]));
+                    br.step();
+                }
+#pragma unroll
+                for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
+                    uint32_t r[32];
+                    if constexpr (kTB8) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            decode_word_e2m1(s ? wq[i].z : wq[i].x, r + 8 * i);
+                            decode_word_e2m1(s ? wq[i].w : wq[i].y, r + 8 * i + 4);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            decode_word_e2m1(wq[i].x, r + 16 * i);
+                            decode_word_e2m1(wq[i].y, r + 16 * i + 4);
+                            decode_word_e2m1(wq[i].z, r + 16 * i + 8);
+                            decode_word_e2m1(wq[i].w, r + 16 * i + 12);
+                        }
+                    }
+                    // (keeps the decode arithmetic above the waits: the compiler would otherwise sink it to the store)
+                    asm volatile("" : "+r"(r[0]), "+r"(r[7]), "+r"(r[8]), "+r"(r[15]), "+r"(r[16]), "+r"(r[23]), "+r"(r[24]), "+r"(r[31]));
+                    // the previous set's stores complete, the set is handed over; then this set's buffer must be free
+                    FT_ADD(0);
+                    if (pending >= 0) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        named_bar_arrive(kFBarSet0 + 2 * pending + h, kFHandover);
+                    }
+                    FT_ADD(2);
+                    ok = wait_bar(smem_u32(&ctl->opfree[h][sr.idx]), sr.par ^ 1, abort_flag, 7);
+                    FT_ADD(3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (!(a.prefetch_steps & 8)) tmem_st32(tbuf0 + (uint32_t)sr.idx * kFp4SetCols, r);   // WHATIF
+                    pending = sr.idx;
+                }
+            }
+        }
+        if (ok && pending >= 0) {
+            tc_wait_st();
+            tc_fence_before();
+            named_bar_arrive(kFBarSet0 + 2 * pending + h, kFHandover);
+        }
+        FT_ADD(0);
+        if (warp == kFWarpDecode0) FT_OUT(8, 8);
+        if (*abort_flag) {
+            // A wait was abandoned somewhere in the block: the issuer may be blocked on one of the named barriers (they
+            // have no time-out); arrive on all of them so that it wakes up, sees the flag and leaves.
+            __syncwarp();
+            for (int s = 0; s < a.n_sets; ++s) named_bar_arrive(kFBarSet0 + 2 * s + h, kFHandover);
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int etid = threadIdx.x - kFWarpEpi0 * 32;
+        const int first_unit = (int)((unsigned)lo / (unsigned)a.P);
+        uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
+        uint32_t accphase = 0;
+        named_bar_sync(kFBarDep, kFThreads - 32);   // nothing to do before the grid dependency is resolved; sleep until then
+        grid_dependency_wait();                     // (returns at once: orders this thread's accesses behind the previous kernel's)
+        bool ok = wait_bar(tmemready, 0, abort_flag, 20);
+        tc_fence_after();
+        const uint32_t tmem_base = ctl->tmem_base;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        {
+            // Scale factors, once per launch, in this warp's lane quadrant (every quadrant of the tensor core reads its
+            // own copy).  A side (four columns: weight rows 32c + lane): 2^0.  B side: row n of a tenant's digit rows is
+            // digit n / m, weight 4^(n / m); four bytes per column = the four 32-k blocks of a step, all alike.
+            uint32_t sf[8];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) sf[c] = 0x7F7F7F7Fu;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int n = lane + 32 * c;
+                const uint32_t byte = (n < a.Nd) ? (uint32_t)(127 + 2 * (n / am)) : 127u;
+                sf[4 + c] = byte * 0x01010101u;
+            }
+            tmem_st8(lane_taddr + a.col_sf, sf);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->sfready));
+        }
+        int pend_unit[2], pend_c0[2], pend_c1[2], npend = 0;   // cut tiles this block has to finish
+        // Units of up to 16 token rows (a.convert): while a tile is being accumulated these four warps write every
+        // step's activation image.  Entering a segment they first take, per token row, the largest magnitude over the
+        // segment's k range (the row's exponent E for this block; one of four slots, since the images run at most
+        // three steps, i.e. three segments, ahead of the MMAs); then one task per thread and step (fp4_split_task).
+        // Steps of the current tile are written with blocking waits (the tile cannot complete without them), later
+        // ones whenever their image slot is free.
+        ItemIter si(it);
+        bool more_s = a.convert && si.next();
+        Ring xr{0, 0u, a.n_img};
+        int n_split = 0, seg_end = 0, split_seg = -1, seg = -1;
+        Unit us{};
+        auto split_next = [&](bool block) -> bool {
+            const uint32_t bar = smem_u32(&ctl->pempty[xr.idx]);
+            if (block) {
+                if (!wait_bar(bar, xr.par ^ 1, abort_flag, 14)) return false;
+            } else if (!warp_all(mbar_test_wait(bar, xr.par ^ 1))) {
+                return false;
+            }
+            if (si.first) {
+                // a new segment: its rows' largest magnitudes over [si.p, si.p1) x 128 k
+                us = unit_info(a, si.unit);
+                ++split_seg;
+                uint32_t* em = ctl->emax[split_seg & 3];
+                epi_bar_sync(kFEpiWarps * 32);
+                if (etid < 16) em[etid] = 0u;
+                epi_bar_sync(kFEpiWarps * 32);
+                const int cpr = (si.p1 - si.p) * 16;   // 16-byte chunks per row
+                const uint16_t* xg = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
+                // (four chunks per thread requested together: the scan costs one round trip to L2 per 512 chunks)
+                const int total = us.ntok * cpr;
+                for (int idx0 = etid; idx0 < total; idx0 += 4 * kFEpiWarps * 32) {
+                    uint4 v[4];
+                    int rr[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int idx = idx0 + q * kFEpiWarps * 32;
+                        rr[q] = (int)((unsigned)idx / (unsigned)cpr);
+                        v[q] = (idx < total) ? __ldcg(reinterpret_cast<const uint4*>(xg + (size_t)rr[q] * a.K) + (idx - rr[q] * cpr)) : make_uint4(0u, 0u, 0u, 0u);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t mx2 = __vmaxu2(__vmaxu2(v[q].x & 0x7FFF7FFFu, v[q].y & 0x7FFF7FFFu), __vmaxu2(v[q].z & 0x7FFF7FFFu, v[q].w & 0x7FFF7FFFu));
+                        const uint32_t mx = max(mx2 & 0xFFFFu, mx2 >> 16);
+                        if (mx && idx0 + q * kFEpiWarps * 32 < total) atomicMax(em + rr[q], mx);
+                    }
+                }
+                epi_bar_sync(kFEpiWarps * 32);
+                if (etid < 16) ctl->xs[(split_seg & 3) * 16 + etid] = ldexpf(1.f, max((int)(em[etid] >> 7), 1) - 141);
+            }
+            const uint32_t* em = ctl->emax[split_seg & 3];
+            const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
+            uint8_t* im = smem + img_off + xr.idx * a.img_bytes;
+            for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
+                const int r = task >> 4;
+                const int j = r / am, t = r - j * am;
+                fp4_split_task(xstep + (size_t)r * a.K, im, task & 15, r, j, t, am, max((int)(em[r] >> 7), 1), a.x_atom_bytes, a.x_tile_bytes);
+            }
+            fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+            mbar_arrive(smem_u32(&ctl->pfull[xr.idx]));
+            xr.step();
+            ++n_split;
+            more_s = si.next();
+            return true;
+        };
+        FT_DECL(8);
+        while (ok && it.next(unit, p0, p1)) {
+            const Unit u = unit_info(a, unit);
+            const int n = u.n0 + row;
+            const bool whole = (p0 == 0 && p1 == a.P);
+            ++seg;
+            float alv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
+            const float* xs_s = a.convert ? ctl->xs + (seg & 3) * 16 : ctl->xs + (seg & 1) * 32;
+            if (a.convert) {
+                seg_end += p1 - p0;
+                while (ok && n_split < seg_end) ok = split_next(true);
+                if (!ok) break;
+                // until this tile's accumulators are complete: write ahead whatever image slot is free
+                while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
+                    if (!split_next(false)) break;
+                }
+            } else {
+                // the token rows' fixed-point units (written by the pre-pass kernel)
+                epi_bar_sync(kFEpiWarps * 32);   // (the readers of this slot, two segments ago, are long done)
+                if (etid < 32) ctl->xs[(seg & 1) * 32 + etid] = (etid < u.ntok) ? __ldcg(a.xscale + u.xrow0 + etid) : 0.f;
+                epi_bar_sync(kFEpiWarps * 32);
+            }
+            float* slotp = nullptr;
+            if (!whole && a.cluster <= 1) {
+                const int slot = (unit == first_unit) ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1;
+                slotp = a.partials + (size_t)slot * a.slot_floats;
+            }
+            FT_ADD(0);
+            ok = wait_bar(smem_u32(&ctl->accfull), accphase, abort_flag, 8);
+            FT_ADD(1);
+            if (!ok) break;
+            tc_fence_after();
+            accphase ^= 1;
+            if (a.cluster > 1) {
+                // Cluster form: this block's partial sums go to its own shared memory (the W_base ring: every load
+                // into it has landed and every MMA that read it has completed), token-major, one float per weight
+                // row; the cluster's leader adds the blocks' partials up at the end of the kernel.
+                const FClusterPartOut out{reinterpret_cast<float*>(smem) + row};
+                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, xs_s, am);
+                break;   // (one segment per block)
+            }
+            {
+                const EpiOut<false, false> out{Y, slotp, a.N, n, row, u.xrow0, 0.f, a};
+                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, xs_s, am);
+            }
+            // this warp's arrival on the "accumulators drained" barrier
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->accempty));
+            FT_ADD(2);
+            if (!whole) {
+                // This tile is cut across blocks: publish the partial and count arrivals right away.  If this block is
+                // the last to arrive it adds the partials up in block order and writes Y, after its other segments.
+                const int first_item = unit * a.P;
+                const int c0 = cta_of_item(a, first_item);
+                const int c1 = cta_of_item(a, first_item + a.P - 1);
+                epi_bar_sync(kFEpiWarps * 32);
+                if (*abort_flag) break;
+                if (etid == 0) {
+                    unsigned old;
+                    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(a.counters + unit) : "memory");
+                    ctl->is_last = (old == (unsigned)(c1 - c0)) ? 1u : 0u;
+                }
+                epi_bar_sync(kFEpiWarps * 32);
+                if (*abort_flag) break;
+                if (ctl->is_last) {
+                    pend_unit[npend] = unit;
+                    pend_c0[npend] = c0;
+                    pend_c1[npend] = c1;
+                    ++npend;
+                }
+                FT_ADD(3);
+            }
+        }
+        // Tiles this block was the last to arrive at (at most its first and its last segment).
+        for (int k = 0; k < npend && ok && !*abort_flag; ++k) {
+            const int un = pend_unit[k], c0 = pend_c0[k], c1 = pend_c1[k];
+            const Unit u = unit_info(a, un);
+            const int first_item = un * a.P;
+            const int slot0 = (cta_first_item(a, c0) == first_item) ? 2 * c0 : 2 * c0 + 1;
+            const float* first = a.partials + (size_t)slot0 * a.slot_floats;
+            const float* rest = a.partials + (size_t)(2 * (c0 + 1)) * a.slot_floats;
+            reduce_partials<false, false>(a, u, etid, kFEpiWarps, first, rest, 2 * (size_t)a.slot_floats, c1 - c0);
+            if (etid == 0) a.counters[un] = 0u;
+        }
+        FT_ADD(4);
+        if (warp == kFWarpEpi0) FT_OUT(16, 8);
+        if (!ok) {
+            // This warp left on an abandoned wait; a sibling that passed the same wait a moment earlier may be
+            // waiting on the epilogue barrier: release it once (it then sees the flag and leaves too).
+            __syncwarp();
+            named_bar_arrive(1, kFEpiWarps * 32);
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    __syncthreads();
+    if (*abort_flag) {
+        // A wait was abandoned: give copies and MMAs still in flight a bounded time to land before shared
+        // and tensor memory are released.
+        if (threadIdx.x == 0) {
+            const long long t0 = clock64();
+            while (clock64() - t0 < 4000000ll) {
+            }
+        }
+        __syncthreads();
+    }
+    tc_fence_after();
+    if (warp == kFWarpMma) tmem_dealloc(ctl->tmem_base, kTmemCols);
+    if (a.cluster > 1) {
+        // Cluster form: after a cluster barrier the leader's epilogue threads (one weight row each) add the blocks'
+        // partial sums in block order, i.e. in k order, through the distributed shared memory window and write Y; a
+        // second barrier keeps the other blocks' shared memory alive until it has read them.
+        cluster_sync_all();
+        if (crank == 0 && warp >= kFWarpEpi0 && lo < hi && !*abort_flag) {
+            const Unit u = unit_info(a, (int)blockIdx.x / a.cluster);
+            const int row = (warp & 3) * 32 + lane;
+            const int n = u.n0 + row;
+            const uint32_t part = base + (uint32_t)row * 4u;   // this block's part[0][row]; same offset in every block
+            uint32_t peer[8];
+#pragma unroll
+            for (int r = 1; r < 8; ++r) peer[r] = (r < a.cluster) ? mapa_shared(part, (uint32_t)r) : 0u;
+            const EpiOut<false, false> out{reinterpret_cast<uint16_t*>(a.Y), nullptr, a.N, n, row, u.xrow0, 0.f, a};
+            for (int tok = 0; tok < u.ntok; tok += 4) {   // (four tokens' remote loads in flight together)
+                float pv[4][8];
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int r = 1; r < 8; ++r)
+                        pv[q][r] = (r < a.cluster && tok + q < u.ntok) ? ld_shared_cluster_f32(peer[r] + (uint32_t)(tok + q) * (kTileN * 4u)) : 0.f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (tok + q < u.ntok) {   // (warp-uniform)
+                        float v = reinterpret_cast<const float*>(smem)[(tok + q) * kTileN + row];
+#pragma unroll
+                        for (int r = 1; r < 8; ++r) v += pv[q][r];
+                        out.put(tok + q, v);
+                    }
+                }
+            }
+        }
+        cluster_sync_relaxed();
+    }
+}
+
+#ifdef BD_TRACE
+extern "C" int bitdelta_debug_set_trace_fp4(long long* buf) {
+    return (int)cudaMemcpyToSymbol(g_fp4_trace, &buf, sizeof(buf));
+}
+#endif
+
+static void* fp4_kernel(int tb8) {
+    return tb8 ? reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true>) : reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false>);
+}
+
+cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
+                            bool early_start, cudaStream_t stream) {
+    const int mode = args.sets_per_step == 2 ? 1 : 0;
+    static std::atomic<unsigned char> attr_done[64][2];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_done[dev][mode].load()) {
+        e = cudaFuncSetAttribute(fp4_kernel(mode), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (e != cudaSuccess) return e;
+        attr_done[dev][mode].store(1);
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)kFThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    if (early_start) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
+    }
+    if (args.cluster > 1) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = (unsigned)args.cluster;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = nattr;
+    if (mode) return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true>, tmW, tmBits, args);
+    return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false>, tmW, tmBits, args);
+}
+
+int fp4_max_active_clusters(uint32_t smem_bytes, int cluster) {
+    if (cudaFuncSetAttribute(fp4_kernel(1), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(cluster * 16));
+    cfg.blockDim = dim3((unsigned)kFThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, bitdelta_gemm_fp4_kernel<true>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+cudaError_t read_fp4_status(unsigned int out[2]) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_device_status, sizeof(unsigned int) * 2);
+    if (e != cudaSuccess) return e;
+    if (out[0] != 0u) {
+        const unsigned int zero[2] = {0u, 0u};
+        e = cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero));
+    }
+    return e;
+}
+
+}  // namespace bd

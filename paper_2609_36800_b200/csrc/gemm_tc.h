@@ -29,6 +29,13 @@ struct GemmArgs {
     int trigger_early;   // ... 1: dependents may launch from this kernel's start (0: see trigger_step)
     int trigger_step;    // ... dependents may launch once this many of a block's W_base tiles are queued (or all of them)
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
+    int fp4;             // 4-bit decode kernel (gemm_fp4.cu) ...
+    int n_img;           // ... ring of activation operand images
+    int sets_per_step;   // ... operand sets per 128-k step
+    uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
+    uint32_t col_sf;     // ... first scale-factor column in tensor memory
+    const uint8_t* img;  // ... images written by the pre-pass: [group][step][img_bytes]
+    const float* xscale; // ... [B*m] value of one unit of a token row's fixed-point activations
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
@@ -61,6 +68,9 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.counters = reinterpret_cast<unsigned int*>(workspace);
     char* ws = reinterpret_cast<char*>(workspace);
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
+    a.fp4 = p.fp4; a.n_img = p.n_img; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
+    a.img = reinterpret_cast<const uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
+    a.xscale = reinterpret_cast<const float*>(ws + p.ws_header_bytes + p.ws_partials_bytes + p.ws_scale_off);
     return a;
 }
 
@@ -124,6 +134,14 @@ int max_active_pairs(uint32_t smem_bytes);
 // Decode schedule pre-pass: X bf16 [rows, K] -> four e5m2 pieces per element (k permuted inside
 // each group of 32) in X8 [B, 4, m, K].
 cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream);
+
+// The 4-bit decode kernel (plan.fp4).  Pre-pass: per token row its fixed-point unit (xscale) and, per tenant group and
+// 128-k step, the shared-memory image of the activation operands (16-bit tile + eight e2m1 digit rows per token).
+cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, float* xscale, const Plan& p, bool early_start, cudaStream_t stream);
+cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
+                            bool early_start, cudaStream_t stream);
+int fp4_max_active_clusters(uint32_t smem_bytes, int cluster);
+cudaError_t read_fp4_status(unsigned int out[2]);
 
 // One warp that lets a bounded wait expire after `limit_cycles` (see bitdelta_selftest_timeout).
 cudaError_t launch_selftest_timeout(long long limit_cycles, int site, cudaStream_t stream);

@@ -29,6 +29,10 @@ constexpr int kStreamMaxSets = 6;
 // the last piece tile) reaches up to round8(4m(TB-1) + N3) rows, i.e. whole 8-row swizzle atoms up to 2 KB past
 // the tile: the control block (1 KB) and this pad are what it reads there (ignored accumulator columns).
 constexpr int kStreamTailPad = 1024;
+// 4-bit decode schedule (see gemm_fp4.cu): signs and activation pieces as e2m1, block-scaled MMA with constant scales.
+constexpr int kFp4Pieces = 8;        // radix-4 digits of a 16-bit fixed-point activation magnitude
+constexpr int kFp4MaxM = 8;          // tokens per tenant
+constexpr int kFp4SetCols = 64;      // one operand set in tensor memory: 8 tenants x 64 k, or 4 tenants x 128 k
 
 struct Plan {
     int B, m, N, K;
@@ -66,6 +70,12 @@ struct Plan {
     int pair;          // tiled schedule on CTA pairs: a unit is two W_base tiles (256 rows), one per CTA of a cluster of
                        // two; each CTA stages its own weights and half of the activation tile, the pair's leader issues
                        // 256-row MMAs (tcgen05 cta_group::2)
+    int fp4;           // 1: the 4-bit decode kernel (gemm_fp4.cu; a pre-pass writes the activation operands)
+    int n_img;         // ... ring of activation operand images in shared memory
+    int sets_per_step; // ... operand sets per 128-k step (2: eight tenants per unit, 1: four)
+    uint32_t img_bytes;   // ... one image: 16-bit activation tile (two atoms) + e2m1 piece tile (64 bytes per row)
+    uint32_t col_sf;      // ... first scale-factor column in tensor memory (4 for the A side, then the B side's)
+    size_t ws_scale_off;  // ... offset of the per-token scales behind the images in the activation region
     int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
@@ -94,6 +104,11 @@ inline int stream_mode() {
     return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
 }
 inline bool stream_enabled() { return stream_mode() != 0; }
+// BITDELTA_FP4=1: the 4-bit decode kernel where it applies (m <= 8).
+inline bool fp4_enabled() {
+    const char* e = getenv("BITDELTA_FP4");
+    return e && e[0] == '1';
+}
 
 // The cluster form of the streaming kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
 inline bool cluster_enabled() {
@@ -103,8 +118,9 @@ inline bool cluster_enabled() {
 
 // allow_pair = false: the device cannot hold all the pairs (or clusters) at once (see the launcher), plan without them.
 // force_tiled: plan the tiled schedule whatever m is (bf16 / binary16 operands for both terms).
+// allow_fp4 = false: the call has options the 4-bit decode kernel does not take (binary16, bias, activation).
 inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override = 0, int whole_override = 0,
-                      bool allow_pair = true, bool force_tiled = false) {
+                      bool allow_pair = true, bool force_tiled = false, bool allow_fp4 = true) {
     Plan p{};
     p.B = B; p.m = m; p.N = N; p.K = K;
     p.ok = false;
@@ -129,7 +145,20 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
         p.stream = (stream_mode() != 0 && p.TB * m <= (stream_mode() == 2 ? 32 : 16)) ? 1 : 0;
-        if (p.stream) {
+        p.fp4 = (allow_fp4 && fp4_enabled() && m <= kFp4MaxM) ? 1 : 0;
+        if (p.fp4) {
+            // 4-bit operands: eight e2m1 pieces per token stacked along N (tenant j's rows start at 8 m j), written by
+            // a pre-pass together with the 16-bit tile of the base MMA as one image per (tenant group, 128-k step).
+            p.stream = 1;
+            // (BITDELTA_FP4_INKERNEL=1, experiments: with few token rows the kernel's epilogue warps write the images themselves;
+            // measured slower than the pre-pass: every block of a tile column repeats the split)
+            p.convert = (p.TB * m <= 16 && getenv("BITDELTA_FP4_INKERNEL") != nullptr) ? 1 : 0;
+            p.Nd = kFp4Pieces * m;
+            p.N3 = p.Nd;
+            p.x_rows = p.Nb;
+            p.x8_rows = p.TB * kFp4Pieces * m;
+            p.sets_per_step = (p.TB > 4) ? 2 : 1;
+        } else if (p.stream) {
             p.convert = 1;                              // the splitter threads read X themselves: no pre-pass
             p.x_rows = round_up(p.TB * m, 8);           // (the base MMA's N = 16 may read past it: ignored columns)
             p.x8_rows = round_up(p.TB * kPieces * m, 8);   // (the last tenants' windows run past it: ignored columns)
@@ -234,7 +263,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
     p.w_stage_bytes = 2 * p.w_atom_bytes;
     p.x_tile_bytes = 2 * p.x_atom_bytes;
-    p.bslot_bytes = (uint32_t)p.TB * kTileN * (p.stream ? 16 : 32);
+    p.bslot_bytes = (uint32_t)p.TB * kTileN * ((p.stream && !p.fp4) ? 16 : 32);
     // Shared memory: rings of W_base tiles, of bf16 activation tiles and (decode) of e5m2 piece tiles, and
     // the sign-word slots.  W_base comes from DRAM (latency ~1.5 us under load); it and the bf16
     // activations are released as soon as the base MMAs have read them.  The piece tiles come from L2 (or
@@ -251,7 +280,22 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         if (p.n_bits < 2) p.n_bits = 2;
     }
     const int avail = kSmemBudget - 1024 /*alignment slack*/ - kSmemCtrlBytes - p.n_bits * (int)p.bslot_bytes;
-    if (p.stream) {
+    if (p.fp4) {
+        // A whole multiprocessor per block: two sign-word slots (256 k each, 32-byte rows: a copy-engine operation costs
+        // about a cycle per row whatever its width), three activation images if they fit, the rest for W_base tiles.
+        p.img_bytes = (uint32_t)round_up((int)p.x_tile_bytes + p.x8_rows * 64, 1024);
+        p.n_bits = 2;
+        const int fixed = 1024 + kSmemCtrlBytes + p.n_bits * (int)p.bslot_bytes;
+        p.n_img = 3;
+        p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
+        if (p.n_w < 3) {
+            p.n_img = 2;
+            p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
+        }
+        if (p.n_w > 4) p.n_w = 4;
+        p.n_x = p.n_img;
+        p.n_x8 = p.n_img;
+    } else if (p.stream) {
         // Half a multiprocessor: two sign-word slots (128 k each), two activation and two piece tiles, and
         // every remaining byte for W_base atoms (64 k, 16 KB each).
         // Half a multiprocessor: two slots of {activation tile, piece tile} (filled together by the splitter
@@ -296,7 +340,9 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.n_w < 2) return p;
     p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
                    p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
-    if (p.stream) {
+    if (p.fp4) {
+        p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_img * p.img_bytes + p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
+    } else if (p.stream) {
         p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
                        p.n_bits * p.bslot_bytes + kSmemCtrlBytes + kStreamTailPad;
     } else if (p.smem_bytes < 120 * 1024) {
@@ -319,7 +365,16 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.decode) slots /= 2;                          // each of the two decode groups has its own ring
     p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
     if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
-    if (p.stream) {
+    if (p.fp4) {
+        // [base | delta accumulators | 4 + ceil(Nd / 32) scale-factor columns | operand sets of 64 columns]
+        p.col_sf = p.col_a;
+        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + (p.Nd + 31) / 32, 32);
+        p.halves = 2;
+        p.n_sets = (kTmemCols - (int)p.col_a) / kFp4SetCols;
+        if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
+        if (p.n_sets < 2) return p;
+        p.a_slots = 2;
+    } else if (p.stream) {
         p.halves = 2;
         p.n_sets = free_cols / kStreamSetCols;
         if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
@@ -337,6 +392,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     const long long max_ctas = items < kMaxCtas ? items : kMaxCtas;
     p.ws_partials_bytes = (size_t)2 * (size_t)max_ctas * p.slot_floats * sizeof(float);
     p.ws_x8_bytes = p.decode ? (((size_t)B * kPieces * m * K + 1023) / 1024 * 1024) : 0;
+    if (p.fp4) {   // one image per (tenant group, 128-k step), then one scale per token row
+        p.ws_scale_off = (size_t)p.groups * p.P * p.img_bytes;
+        p.ws_x8_bytes = p.ws_scale_off + (((size_t)B * m * sizeof(float) + 1023) / 1024 * 1024);
+    }
     p.ws_bytes = p.ws_header_bytes + p.ws_partials_bytes + p.ws_x8_bytes;
     p.ok = true;
     return p;

@@ -190,6 +190,24 @@ __device__ __forceinline__ void umma_ts_f8(uint32_t d_tmem, uint32_t a_tmem, uin
         : "memory");
 }
 
+// D[tmem] (+)= A[tmem] * B[smem]^T ; e2m1 inputs (eight per TMEM column, K = 64), one ue8m0 scale per row and 32 k
+// on either side (scale_A / scale_B: tensor-memory columns, see gemm_fp4.cu), fp32 accumulate.
+__device__ __forceinline__ void umma_ts_mxf4(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t scale_a_tmem, uint32_t scale_b_tmem, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], [%1], %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(scale_a_tmem), "r"(scale_b_tmem)
+        : "memory");
+}
+
+// Plain bulk copy global -> shared (sizes and addresses multiples of 16 bytes), completion counted on an mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 // ------------------------------------------------- CTA pairs (cluster of two, tcgen05 cta_group::2)
 // One MMA instruction of the pair's leader (rank 0) multiplies a 256-row A (128 rows from each CTA's shared or
 // tensor memory, same offsets in both) by a B whose N rows are split half / half over the two CTAs' shared
@@ -280,6 +298,15 @@ __host__ __device__ constexpr uint32_t make_idesc_e5m2(uint32_t M, uint32_t N) {
            | ((M >> 4) << 24);  // M / 16
 }
 
+// Instruction descriptor, kind::mxf4 (block-scaled): e2m1 x e2m1 -> fp32, ue8m0 scales, scale ids 0, both K-major.
+__host__ __device__ constexpr uint32_t make_idesc_mxf4(uint32_t M, uint32_t N) {
+    return (1u << 7)            // A format: e2m1
+           | (1u << 10)         // B format: e2m1
+           | ((N >> 3) << 17)   // N / 8
+           | (1u << 23)         // scale format: ue8m0
+           | ((M >> 4) << 24);  // M / 16
+}
+
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N) {
     return (1u << 4)            // D format: fp32
@@ -302,6 +329,18 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr) {
     d |= static_cast<uint64_t>(1024 >> 4) << 32;                    // stride byte offset = 1024 B
     d |= static_cast<uint64_t>(1) << 46;                            // descriptor version (sm_100)
     d |= static_cast<uint64_t>(2) << 61;                            // layout: 128-byte swizzle
+    return d;
+}
+
+// The same for rows of 64 bytes with the 64-byte swizzle (16-byte chunk c of row r at chunk c ^ ((r >> 1) & 3)):
+// eight rows are 512 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(1) << 16;
+    d |= static_cast<uint64_t>(512 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(4) << 61;                            // layout: 64-byte swizzle
     return d;
 }
 
@@ -352,6 +391,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                  : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
