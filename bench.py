@@ -394,12 +394,19 @@ def cpu_baseline(wl, host_inputs, budget_s=15.0):
 
 
 def kernels_per_step(wl):
-    """Kernels one bitdelta_gemm call launches: the GEMM kernel, plus the activation-split kernel in the
-    decode schedule when a tile holds more than 16 token rows (otherwise the GEMM kernel splits itself)."""
-    if wl.m > 16:
-        return 1
-    tb = min(wl.B, 8 if wl.m <= 4 else 4)
-    return 1 if tb * wl.m <= 16 else 2
+    """Kernels one bitdelta_gemm call launches, from the library's own plan: the GEMM kernel, plus an activation
+    pre-pass kernel in the 4-bit decode schedule and in the 8-bit decode schedule with more than 16 token rows per
+    unit (otherwise the GEMM kernel splits the activations itself)."""
+    schedule = bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"]
+    if schedule in (7, 8):
+        return 1 if os.environ.get("BITDELTA_FP4_INKERNEL") else 2
+    return 2 if schedule == 1 else 1
+
+
+def gemm_kernel_name(wl):
+    schedule = bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"]
+    return {7: "bitdelta_gemm_fp4_kernel", 8: "bitdelta_gemm_fp4_kernel", 5: "bitdelta_gemm_stream_kernel",
+            6: "bitdelta_gemm_stream_kernel", 3: "gemm_simt_kernel"}.get(schedule, "bitdelta_gemm_tc_kernel")
 
 
 def summarize(wl, ms_total, steps, n_gpus, peaks, clocks=None):
@@ -425,8 +432,8 @@ def summarize(wl, ms_total, steps, n_gpus, peaks, clocks=None):
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
     roof["algorithmic_bytes"] = wl.bytes
     roof["algorithmic_flops"] = wl.flops
-    roof["kernel"] = "bitdelta_gemm_tc_kernel"
-    roof["us_per_launch"] = sec * 1e6
+    roof["kernel"] = gemm_kernel_name(wl)
+    roof["us_per_launch"] = sec * 1e6   # (a whole call: the GEMM kernel and, where the schedule has one, its small pre-pass kernel)
     return gbs, tfl, roof
 
 

@@ -392,9 +392,8 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         // 4-bit decode kernel: the activation operands of every (tenant group, 128-k step) as shared-memory images, and
         // the token rows' fixed-point units; then the GEMM, which prefetches weights while this is still running.
         uint8_t* img = bd::ws_x8(p, workspace);
-        static const bool skip_prepass = getenv("BITDELTA_FP4_SKIP_PREPASS") != nullptr;   // WHATIF (timing experiments)
         // (its early start is always safe: it waits for its predecessor before it touches anything)
-        if (!skip_prepass && !p.convert && bd::launch_x_split_fp4(X, img, reinterpret_cast<float*>(img + p.ws_scale_off), p, early_start_enabled(), stream) != cudaSuccess)
+        if (!p.convert && bd::launch_x_split_fp4(X, img, p, early_start_enabled(), stream) != cudaSuccess)
             return BITDELTA_ERR_CUDA;
         if (!p.convert) g_launches++;
         tmX8 = tmW;   // not read
@@ -423,7 +422,6 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_STEP"); d = e ? atoi(e) : (1 << 30); } args.trigger_step = d; }
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_EARLY"); d = (e && e[0] == '1') ? 1 : 0; } args.trigger_early = d; }
     { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_DECODE_WARPS"); d = (e && atoi(e) == 16) ? 16 : 8; } args.decode_warps = d; }
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_PREFETCH"); d = e ? atoi(e) : 0; } args.prefetch_steps = d; }
     // (a GEMM queued right behind the library's own pack / compress must not prefetch what they are still writing)
     const bool early = early_start_enabled() && g_weights_just_written.exchange(0) == 0;
     const cudaError_t le = p.fp4

@@ -8,15 +8,15 @@
 //     logic operations, four tensor-memory columns.  That is half the integer work and half the tensor-memory store
 //     traffic of the 8-bit form, the two things that bound the decode schedules, and half the MMA instructions.
 //     Register c of a word holds in nibble i the sign of k = 4i + c.
-//   * Activations: a token row's values are written as 16-bit fixed point relative to the row's largest exponent E
-//     (|x| = v * 2^(E-142), v < 2^16: every value within 8 binades of the row's largest is exact, smaller ones are
-//     truncated below 2^-16 of it) and v as eight radix-4 digits 0..3; a digit d goes into the operand as the e2m1
-//     value d/2, whose 4-bit code is d itself, with the value's sign in the code's sign bit.  Digit q of all tokens
-//     forms row block q of the MMA's B operand; its weight 4^q is the B-side SCALE FACTOR of those rows (ue8m0
-//     127 + 2q, the same for every k: written to tensor memory once per launch), the A-side scale is 1, so a
-//     tenant's delta is the plain sum of its eight accumulator column groups times the row's unit 2^(E-141), which
-//     the epilogue applies together with alpha.  No value of the 16-bit input range saturates or is flagged.  (E is
-//     taken over the whole row by the pre-pass, over a block's k range when the kernel splits the activations.)
+//   * Activations: every group of 32 consecutive k of a token row (one sign word) is written as 16-bit fixed point
+//     relative to the group's largest exponent E (|x| = v * 2^(E-142), v < 2^16: every value within 8 binades of the
+//     group's largest is exact, smaller ones are truncated below 2^-16 of it) and v as eight radix-4 digits 0..3; a
+//     digit d goes into the operand as the e2m1 value d/2, whose 4-bit code is d itself, with the value's sign in the
+//     code's sign bit.  Digit q of all tokens forms row block q of the MMA's B operand, and the B-side SCALE FACTOR
+//     of a row and 32-k group (ue8m0, one byte) is E + 2q: the group's exponent and the digit's weight 4^q.  The
+//     A-side scale is 1.  A tenant's delta is then the plain sum of its eight accumulator column groups times
+//     2^-14, which the epilogue applies together with alpha.  No value of the 16-bit input range saturates or is
+//     flagged (exponents above 240, i.e. |x| >= 2^114, are treated as 240).
 //   * Units of more than 16 token rows: a pre-pass kernel writes, per tenant group and 128-k step, the
 //     shared-memory IMAGE of both activation operands (16-bit tile of the base MMA with its 128-byte swizzle, digit
 //     rows with the 64-byte swizzle); the producer fetches an image with one plain bulk copy.  Units of up to 16 token
@@ -71,13 +71,10 @@ struct FCtl {
     uint64_t accempty;              // the accumulators were drained (4 epilogue warps)
     uint64_t depready;              // the grid this launch depends on has completed
     uint64_t tmemready;             // tensor memory is allocated (its base address is in tmem_base)
-    uint64_t sfready;               // the scale factors are in tensor memory (4 epilogue warps)
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t is_last;
-    float xs[64];                   // fixed-point units of the token rows: four segments in flight x 16 rows (the kernel
-                                    // splits), or two x 32 rows (pre-pass)
-    uint32_t emax[4][16];           // the kernel splits: the rows' largest magnitudes (16-bit patterns) of those segments
+    uint64_t imgready[4];           // a step's image is in shared memory and its scale factors in tensor memory (4 epilogue warps)
 };
 static_assert(sizeof(FCtl) <= kSmemCtrlBytes, "control block too large");
 
@@ -125,33 +122,41 @@ __device__ __forceinline__ void fp4_digits8(const uint32_t* hv, int E, uint32_t*
     }
 }
 
-// One task of the activation split: of token row `xrow` (row r_local = j*m + t of its unit) the 16-byte chunk `tk`
-// of a 128-k step (k = 8 tk .. 8 tk + 7) goes to the 16-bit tile, and the eight values k = 32 wd + 4i + c (wd = tk / 4,
-// c = tk % 4) to the digit rows j*8m + q*m + t: register c of word wd, the order in which decode_word_e2m1 lays out
-// the signs.  `xstep`: the row's first value of the step; `im`: the step's image (global or shared memory).
+// One task of the activation split: of token row r_local = j*m + t of its unit the 16-byte chunk `tk` of a 128-k
+// step (k = 8 tk .. 8 tk + 7) goes to the 16-bit tile, and the eight values k = 32 wd + 4i + c (wd = tk / 4, c = tk % 4)
+// to the digit rows j*8m + q*m + t: register c of word wd, the order in which decode_word_e2m1 lays out the signs.
+// The four tasks c = 0..3 of a word sit in neighbouring lanes (all active together) and share the group's exponent,
+// which task c = 0 writes to the image's scale table (byte 4 r_local + wd).  `xstep`: the row's first value of the
+// step; `im`: the step's image (global or shared memory): [16-bit tile | digit rows | scale table].
 __device__ __forceinline__ void fp4_split_task(const uint16_t* __restrict__ xstep, uint8_t* im, int tk, int r_local, int j, int t,
-                                               int m, int E, uint32_t x_atom_bytes, uint32_t x_tile_bytes) {
+                                               int m, uint32_t x_atom_bytes, uint32_t x_tile_bytes, uint32_t sf_off) {
     const uint4 chunk = __ldcg(reinterpret_cast<const uint4*>(xstep) + tk);
     *reinterpret_cast<uint4*>(im + (tk >> 3) * x_atom_bytes + r_local * 128 + (((tk & 7) ^ (r_local & 7)) * 16)) = chunk;
     const int wd = tk >> 2, c = tk & 3;
     uint32_t hv[8], R[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) hv[i] = __ldcg(xstep + 32 * wd + 4 * i + c);
+    uint32_t mx = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mx = max(mx, hv[i] & 0x7FFFu);
+    const unsigned act = __activemask();
+    mx = max(mx, __shfl_xor_sync(act, mx, 1));
+    mx = max(mx, __shfl_xor_sync(act, mx, 2));
+    const int E = min(max((int)(mx >> 7), 1), 240);
     fp4_digits8(hv, E, R);
 #pragma unroll
     for (int q = 0; q < kFp4Pieces; ++q) {
         const int n = j * (kFp4Pieces * m) + q * m + t;
         *reinterpret_cast<uint32_t*>(im + x_tile_bytes + n * 64 + ((wd ^ ((n >> 1) & 3)) * 16) + 4 * c) = R[q];
     }
+    if (c == 0) im[sf_off + 4 * r_local + wd] = (uint8_t)E;
 }
 
 // ---------------------------------------------------------------------------------------------- pre-pass
-// One block per token row.  Phase 1: the row's largest exponent E (biased, subnormals as 1); its fixed-point unit
-// 2^(E-141) goes to xscale.  Phase 2: the row's share of every step's image.
-__global__ void __launch_bounds__(256) x_split_fp4_kernel(const uint16_t* __restrict__ X, uint8_t* __restrict__ img,
-                                                          float* __restrict__ xscale, int m, int K, int TB, int P,
-                                                          uint32_t img_bytes, uint32_t x_atom_bytes, uint32_t x_tile_bytes) {
-    __shared__ uint32_t red[8];
+// Block (row, chunk of 2048 k): the row's share of the images of those steps.
+__global__ void __launch_bounds__(256) x_split_fp4_kernel(const uint16_t* __restrict__ X, uint8_t* __restrict__ img, int m, int K,
+                                                          int TB, int P, uint32_t img_bytes, uint32_t x_atom_bytes,
+                                                          uint32_t x_tile_bytes, uint32_t sf_off) {
     // Launched with an early start: the GEMM queued behind this kernel may become resident at once (it prefetches
     // weights and waits for this kernel before it reads an image); this kernel itself reads X and overwrites the
     // images only after the kernel before it (possibly the previous GEMM, still reading them) has completed.
@@ -162,32 +167,17 @@ __global__ void __launch_bounds__(256) x_split_fp4_kernel(const uint16_t* __rest
     const int g = b / TB, j = b - g * TB;
     const int r_local = j * m + t;
     const uint16_t* x = X + (size_t)row * K;
-    const uint4* x4 = reinterpret_cast<const uint4*>(x);
-    uint32_t mx2 = 0;
-    for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
-        const uint4 v = __ldcg(x4 + i);
-        mx2 = __vmaxu2(mx2, __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)));
-    }
-    uint32_t mx = max(mx2 & 0xFFFFu, mx2 >> 16);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
-    __syncthreads();
-    mx = 0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) mx = max(mx, red[w]);
-    const int E = max((int)(mx >> 7), 1);
-    if (threadIdx.x == 0) xscale[row] = ldexpf(1.f, E - 141);
-
     uint8_t* img_g = img + (size_t)g * P * img_bytes;
-    for (int task = threadIdx.x; task < K / 8; task += blockDim.x) {
+    const int task = blockIdx.y * 256 + threadIdx.x;   // (16 tasks per step: whole groups of four are inside K or outside)
+    if (task < K / 8) {
         const int p = task >> 4;
-        fp4_split_task(x + (size_t)p * kPairK, img_g + (size_t)p * img_bytes, task & 15, r_local, j, t, m, E, x_atom_bytes, x_tile_bytes);
+        fp4_split_task(x + (size_t)p * kPairK, img_g + (size_t)p * img_bytes, task & 15, r_local, j, t, m, x_atom_bytes, x_tile_bytes, sf_off);
     }
 }
 
-cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, float* xscale, const Plan& p, bool early_start, cudaStream_t stream) {
+cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, const Plan& p, bool early_start, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(p.B * p.m));
+    cfg.gridDim = dim3((unsigned)(p.B * p.m), (unsigned)((p.K / 8 + 255) / 256));
     cfg.blockDim = dim3(256u);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
@@ -196,24 +186,25 @@ cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, float* xscale, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = early_start ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, x_split_fp4_kernel, reinterpret_cast<const uint16_t*>(X), img, xscale, p.m, p.K, p.TB, p.P,
-                              p.img_bytes, p.x_atom_bytes, p.x_tile_bytes);
+    return cudaLaunchKernelEx(&cfg, x_split_fp4_kernel, reinterpret_cast<const uint16_t*>(X), img, p.m, p.K, p.TB, p.P, p.img_bytes,
+                              p.x_atom_bytes, p.x_tile_bytes, p.x_tile_bytes + (uint32_t)p.x8_rows * 64u);
 }
 
 // Epilogue of one segment, M tokens per tenant: base accumulator columns j*M + t, tenant j's delta accumulator from
-// column 8M*j, digit q of token t in column q*M + t (already weighted 4^q by its scale factor).
-//   out(j*M + t) = base + alpha_j * (xs[j*M + t] * sum_q D[q*M + t])
+// column 8M*j, digit q of token t in column q*M + t (already weighted by its scale factors).
+//   out(j*M + t) = base + (alpha_j * 2^-14) * sum_q D[q*M + t]
 template <int M, class Out>
-__device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
-                                             const float* alv, const float* xs_smem) {
+__device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out, const float* alv) {
     constexpr int ND = kFp4Pieces * M;
-    uint32_t rb[32];
-    if (a.Nb <= 16) tmem_ld16(lane_taddr, rb);
-    else tmem_ld32(lane_taddr, rb);
+    constexpr int MB = (M <= 1) ? 1 : (M <= 2) ? 2 : (M <= 4) ? 4 : 8;   // base columns read per tenant (a power of two >= M)
 #pragma unroll 1
     for (int j = 0; j < u.nten; ++j) {
-        uint32_t rd[ND];
+        uint32_t rd[ND], rb[MB];
         const uint32_t col = lane_taddr + a.col_delta + (uint32_t)(j * ND);
+        if constexpr (MB == 1) tmem_ld1(lane_taddr + (uint32_t)(j * M), rb);
+        else if constexpr (MB == 2) tmem_ld2(lane_taddr + (uint32_t)(j * M), rb);
+        else if constexpr (MB == 4) tmem_ld4(lane_taddr + (uint32_t)(j * M), rb);
+        else tmem_ld8(lane_taddr + (uint32_t)(j * M), rb);
         if constexpr (ND >= 32) {
 #pragma unroll
             for (int c = 0; c + 32 <= ND; c += 32) tmem_ld32(col + c, rd + c);
@@ -221,34 +212,29 @@ __device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, u
         if constexpr (ND % 32 >= 16) tmem_ld16(col + ND / 32 * 32, rd + ND / 32 * 32);
         if constexpr (ND % 16 >= 8) tmem_ld8(col + ND / 16 * 16, rd + ND / 16 * 16);
         tc_wait_ld();
-        const float al = alv[j];
+        const float al = alv[j] * 6.103515625e-05f;   // 2^-14
 #pragma unroll
         for (int t = 0; t < M; ++t) {
             float d = 0.f;
 #pragma unroll
             for (int q = 0; q < kFp4Pieces; ++q) d += __uint_as_float(rd[q * M + t]);
-            // (rb is indexed with a run-time tenant: select, do not index, so that it stays in registers)
-            float base = 0.f;
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-                if (c == j * M + t) base = __uint_as_float(rb[c]);
-            out.put(j * M + t, fmaf(al, d * xs_smem[j * M + t], base));
+            out.put(j * M + t, fmaf(al, d, __uint_as_float(rb[t])));
         }
     }
 }
 
 template <class Out>
 __device__ __forceinline__ void epilogue_fp4_any_m(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
-                                                   const float* alv, const float* xs_smem, int am) {
+                                                   const float* alv, int am) {
     switch (am) {
-        case 1: epilogue_fp4<1>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 2: epilogue_fp4<2>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 3: epilogue_fp4<3>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 4: epilogue_fp4<4>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 5: epilogue_fp4<5>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 6: epilogue_fp4<6>(a, u, lane_taddr, out, alv, xs_smem); break;
-        case 7: epilogue_fp4<7>(a, u, lane_taddr, out, alv, xs_smem); break;
-        default: epilogue_fp4<8>(a, u, lane_taddr, out, alv, xs_smem); break;
+        case 1: epilogue_fp4<1>(a, u, lane_taddr, out, alv); break;
+        case 2: epilogue_fp4<2>(a, u, lane_taddr, out, alv); break;
+        case 3: epilogue_fp4<3>(a, u, lane_taddr, out, alv); break;
+        case 4: epilogue_fp4<4>(a, u, lane_taddr, out, alv); break;
+        case 5: epilogue_fp4<5>(a, u, lane_taddr, out, alv); break;
+        case 6: epilogue_fp4<6>(a, u, lane_taddr, out, alv); break;
+        case 7: epilogue_fp4<7>(a, u, lane_taddr, out, alv); break;
+        default: epilogue_fp4<8>(a, u, lane_taddr, out, alv); break;
     }
 }
 
@@ -306,7 +292,6 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     // The W_base tile of a step (128 rows x 128 k: both 64-k atoms) in one bulk-tensor copy.  One thread.
     auto issue_w = [&](const Unit& u, int p, int stage) {
         const uint32_t bar = smem_u32(&ctl->wfull[stage]);
-        if (a.prefetch_steps & 4) { mbar_arrive(bar); return; }   // WHATIF
         mbar_arrive_expect_tx(bar, a.w_stage_bytes);
         tma_load_3d(w_addr + stage * a.w_stage_bytes, &tmW, bar, 0, u.n0, p * (kPairK / kAtomK));
     };
@@ -314,14 +299,12 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     // 32 bytes).  One thread.
     auto issue_bits = [&](const Unit& u, int p, int bslot) {
         const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
-        if (a.prefetch_steps & 2) { mbar_arrive(bar); return; }   // WHATIF
         mbar_arrive_expect_tx(bar, a.bslot_bytes);
         tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
     };
     // The activation image of a step (written by the pre-pass kernel): one plain bulk copy.  One thread.
     auto issue_img = [&](const Unit& u, int p, int slot) {
         const uint32_t bar = smem_u32(&ctl->pfull[slot]);
-        if (a.prefetch_steps & 1) { mbar_arrive(bar); return; }   // WHATIF
         mbar_arrive_expect_tx(bar, a.img_bytes);
         const int g = (int)((unsigned)u.tenant0 / (unsigned)a.TB);
         bulk_load(img_addr + slot * a.img_bytes, a.img + ((size_t)g * a.P + p) * a.img_bytes, a.img_bytes, bar);
@@ -334,7 +317,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         for (int s = 0; s < 4; ++s) {
             mbar_init(smem_u32(&ctl->bfull[s]), 1);
             mbar_init(smem_u32(&ctl->bempty[s]), kFDecodeWarps);
-            mbar_init(smem_u32(&ctl->pfull[s]), a.convert ? kFEpiWarps * 32 : 1);   // splitter threads, or one bulk copy
+            mbar_init(smem_u32(&ctl->pfull[s]), 1);   // one bulk copy (pre-pass mode)
+            mbar_init(smem_u32(&ctl->imgready[s]), kFEpiWarps);
             mbar_init(smem_u32(&ctl->pempty[s]), 3);   // (the three issuers)
         }
         for (int s = 0; s < kStreamMaxSets; ++s) {
@@ -345,7 +329,6 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         mbar_init(smem_u32(&ctl->accempty), kFEpiWarps);
         mbar_init(smem_u32(&ctl->depready), 1);
         mbar_init(smem_u32(&ctl->tmemready), 1);
-        mbar_init(smem_u32(&ctl->sfready), kFEpiWarps);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
@@ -451,7 +434,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             for (int p = p0; p < p1 && ok; ++p) {
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this step starts the accumulation
                 FT_ADD(0);
-                ok = warp_all(wait_bar(smem_u32(&ctl->pfull[pr.idx]), pr.par, abort_flag, 13));
+                ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
                 if (!ok) break;
                 const uint32_t img_s = img_addr + pr.idx * a.img_bytes;
@@ -462,7 +445,6 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 {
                     const uint64_t wdesc = desc128 + ((w_addr + wr.idx * a.w_stage_bytes) >> 4);
                     if (elect_one()) {
-                        if (!(a.prefetch_steps & 32))   // WHATIF
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t atom = kk >> 2, k16 = kk & 3;
@@ -497,12 +479,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         bool ok = warp_all(wait_bar(tmemready, 0, abort_flag, 20));
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
-        ok = ok && warp_all(wait_bar(smem_u32(&ctl->sfready), 0, abort_flag, 22));   // scale factors written
-        tc_fence_after();
-        const uint32_t idesc_delta = make_idesc_mxf4(kTileN, (uint32_t)a.Nd);
+        const uint32_t idesc_delta = make_idesc_mxf4(kTileN, (uint32_t)a.Nd);   // (+ the B-side scale id: which pair of a step's four 32-k groups)
         const uint64_t desc64 = make_smem_desc_sw64(0);
         const uint32_t ten_rows16 = (uint32_t)a.Nd * 4u;      // a tenant's digit rows x 64 B >> 4
-        const uint32_t sfa = tmem_base + a.col_sf, sfb = sfa + 4u;
+        const uint32_t sfa = tmem_base + a.col_sf;
         Ring pr{0, 0u, a.n_img}, sr{0, 0u, a.n_sets};
         uint32_t accphase = 0;
         FT_DECL(8);
@@ -516,9 +496,11 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             for (int p = p0; p < p1 && ok; ++p) {
                 const uint32_t first = (p > p0) ? 1u : 0u;   // 0: this step starts the accumulation
                 FT_ADD(0);
-                ok = warp_all(wait_bar(smem_u32(&ctl->pfull[pr.idx]), pr.par, abort_flag, 13));
+                ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
                 if (!ok) break;
+                tc_fence_after();
+                const uint32_t sfb0 = sfa + 4u + (uint32_t)(pr.idx * 4 * a.TB);   // this image slot's scale factors (four columns per tenant)
                 const uint64_t x4desc = desc64 + ((img_addr + pr.idx * a.img_bytes + a.x_tile_bytes) >> 4);
 #pragma unroll
                 for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
@@ -535,11 +517,12 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                             const uint32_t a_j = a_set + (uint32_t)((j >> 1) * kTenCols);
                             const uint32_t d_tmem = tmem_base + a.col_delta + (uint32_t)(j * a.Nd);
                             const uint64_t xj = x4desc + (uint32_t)j * ten_rows16;
+                            const uint32_t sfb = sfb0 + (uint32_t)(4 * j);
                             if constexpr (kTB8) {
-                                umma_ts_mxf4(d_tmem, a_j, xj + (uint32_t)(s * 2), idesc_delta, sfa, sfb, (s > 0) ? 1u : first);
+                                umma_ts_mxf4(d_tmem, a_j, xj + (uint32_t)(s * 2), idesc_delta | ((uint32_t)(2 * s) << 4), sfa, sfb, (s > 0) ? 1u : first);
                             } else {
                                 umma_ts_mxf4(d_tmem, a_j, xj, idesc_delta, sfa, sfb, first);
-                                umma_ts_mxf4(d_tmem, a_j + 8, xj + 2, idesc_delta, sfa, sfb, 1u);
+                                umma_ts_mxf4(d_tmem, a_j + 8, xj + 2, idesc_delta | (2u << 4), sfa, sfb, 1u);
                             }
                         }
                         tc_commit(smem_u32(&ctl->opfree[h][sr.idx]));
@@ -624,7 +607,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                     FT_ADD(3);
                     if (!ok) break;
                     tc_fence_after();
-                    if (!(a.prefetch_steps & 8)) tmem_st32(tbuf0 + (uint32_t)sr.idx * kFp4SetCols, r);   // WHATIF
+                    tmem_st32(tbuf0 + (uint32_t)sr.idx * kFp4SetCols, r);
                     pending = sr.idx;
                 }
             }
@@ -657,84 +640,68 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint32_t tmem_base = ctl->tmem_base;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
         {
-            // Scale factors, once per launch, in this warp's lane quadrant (every quadrant of the tensor core reads its
-            // own copy).  A side (four columns: weight rows 32c + lane): 2^0.  B side: row n of a tenant's digit rows is
-            // digit n / m, weight 4^(n / m); four bytes per column = the four 32-k blocks of a step, all alike.
+            // A-side scale factors (four columns: weight rows 32c + lane), once per launch, in this warp's lane quadrant
+            // (every quadrant of the tensor core reads its own copy): 2^0.  Ordered before the first MMA by the
+            // first image's hand-over below.
             uint32_t sf[8];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) sf[c] = 0x7F7F7F7Fu;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int n = lane + 32 * c;
-                const uint32_t byte = (n < a.Nd) ? (uint32_t)(127 + 2 * (n / am)) : 127u;
-                sf[4 + c] = byte * 0x01010101u;
-            }
+            for (int c = 0; c < 8; ++c) sf[c] = 0x7F7F7F7Fu;
             tmem_st8(lane_taddr + a.col_sf, sf);
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->sfready));
         }
         int pend_unit[2], pend_c0[2], pend_c1[2], npend = 0;   // cut tiles this block has to finish
-        // Units of up to 16 token rows (a.convert): while a tile is being accumulated these four warps write every
-        // step's activation image.  Entering a segment they first take, per token row, the largest magnitude over the
-        // segment's k range (the row's exponent E for this block; one of four slots, since the images run at most
-        // three steps, i.e. three segments, ahead of the MMAs); then one task per thread and step (fp4_split_task).
-        // Steps of the current tile are written with blocking waits (the tile cannot complete without them), later
-        // ones whenever their image slot is free.
+        // While a tile is being accumulated these four warps prepare every step's activation operands.  Units of up to
+        // 16 token rows (a.convert): they write the step's image themselves, one task per thread (fp4_split_task);
+        // otherwise the producer's bulk copy brings it.  Either way they then move the image's scale table into
+        // tensor memory: tenant j's MMAs read the scale factors of their digit rows n = q*m + t from lane n % 32 of
+        // column 4 TB slot + 4 j + n / 32, one byte per 32-k group of the step: the group's exponent + 2q.
+        // Steps of the current tile are served with blocking waits (the tile cannot complete without them), later
+        // ones whenever their image slot is ready.
         ItemIter si(it);
-        bool more_s = a.convert && si.next();
+        bool more_s = si.next();
         Ring xr{0, 0u, a.n_img};
-        int n_split = 0, seg_end = 0, split_seg = -1, seg = -1;
+        int n_split = 0, seg_end = 0;
         Unit us{};
+        const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
         auto split_next = [&](bool block) -> bool {
-            const uint32_t bar = smem_u32(&ctl->pempty[xr.idx]);
+            // convert: the slot must be free (its step's MMAs complete); else: its image must have landed
+            const uint32_t bar = a.convert ? smem_u32(&ctl->pempty[xr.idx]) : smem_u32(&ctl->pfull[xr.idx]);
+            const uint32_t par = a.convert ? (xr.par ^ 1) : xr.par;
             if (block) {
-                if (!wait_bar(bar, xr.par ^ 1, abort_flag, 14)) return false;
-            } else if (!warp_all(mbar_test_wait(bar, xr.par ^ 1))) {
+                if (!wait_bar(bar, par, abort_flag, 14)) return false;
+            } else if (!warp_all(mbar_test_wait(bar, par))) {
                 return false;
             }
-            if (si.first) {
-                // a new segment: its rows' largest magnitudes over [si.p, si.p1) x 128 k
-                us = unit_info(a, si.unit);
-                ++split_seg;
-                uint32_t* em = ctl->emax[split_seg & 3];
-                epi_bar_sync(kFEpiWarps * 32);
-                if (etid < 16) em[etid] = 0u;
-                epi_bar_sync(kFEpiWarps * 32);
-                const int cpr = (si.p1 - si.p) * 16;   // 16-byte chunks per row
-                const uint16_t* xg = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
-                // (four chunks per thread requested together: the scan costs one round trip to L2 per 512 chunks)
-                const int total = us.ntok * cpr;
-                for (int idx0 = etid; idx0 < total; idx0 += 4 * kFEpiWarps * 32) {
-                    uint4 v[4];
-                    int rr[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int idx = idx0 + q * kFEpiWarps * 32;
-                        rr[q] = (int)((unsigned)idx / (unsigned)cpr);
-                        v[q] = (idx < total) ? __ldcg(reinterpret_cast<const uint4*>(xg + (size_t)rr[q] * a.K) + (idx - rr[q] * cpr)) : make_uint4(0u, 0u, 0u, 0u);
-                    }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t mx2 = __vmaxu2(__vmaxu2(v[q].x & 0x7FFF7FFFu, v[q].y & 0x7FFF7FFFu), __vmaxu2(v[q].z & 0x7FFF7FFFu, v[q].w & 0x7FFF7FFFu));
-                        const uint32_t mx = max(mx2 & 0xFFFFu, mx2 >> 16);
-                        if (mx && idx0 + q * kFEpiWarps * 32 < total) atomicMax(em + rr[q], mx);
-                    }
-                }
-                epi_bar_sync(kFEpiWarps * 32);
-                if (etid < 16) ctl->xs[(split_seg & 3) * 16 + etid] = ldexpf(1.f, max((int)(em[etid] >> 7), 1) - 141);
-            }
-            const uint32_t* em = ctl->emax[split_seg & 3];
-            const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
+            if (si.first) us = unit_info(a, si.unit);
             uint8_t* im = smem + img_off + xr.idx * a.img_bytes;
-            for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
-                const int r = task >> 4;
-                const int j = r / am, t = r - j * am;
-                fp4_split_task(xstep + (size_t)r * a.K, im, task & 15, r, j, t, am, max((int)(em[r] >> 7), 1), a.x_atom_bytes, a.x_tile_bytes);
+            if (a.convert) {
+                const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
+                for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
+                    const int r = task >> 4;
+                    const int j = r / am, t = r - j * am;
+                    fp4_split_task(xstep + (size_t)r * a.K, im, task & 15, r, j, t, am, a.x_atom_bytes, a.x_tile_bytes, sf_off);
+                }
+                fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+                epi_bar_sync(kFEpiWarps * 32);
+                if (*abort_flag) return false;
             }
-            fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
-            mbar_arrive(smem_u32(&ctl->pfull[xr.idx]));
+            {
+                // (a tenant's scale factors start at a multiple of four columns: the MMA wants that alignment)
+                const uint32_t sf_slot = lane_taddr + a.col_sf + 4u + (uint32_t)(xr.idx * 4 * a.TB);
+                for (int j = 0; j < us.nten; ++j) {
+                    uint32_t sf[2];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const int n = lane + 32 * c;
+                        const int q = n / am, t = n - q * am;
+                        sf[c] = (n < a.Nd) ? *reinterpret_cast<const uint32_t*>(im + sf_off + 4 * (j * am + t)) + 0x02020202u * (uint32_t)q : 0x7F7F7F7Fu;
+                    }
+                    tmem_st2(sf_slot + (uint32_t)(4 * j), sf[0], sf[1]);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->imgready[xr.idx]));
+            }
             xr.step();
             ++n_split;
             more_s = si.next();
@@ -745,24 +712,15 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
             const bool whole = (p0 == 0 && p1 == a.P);
-            ++seg;
             float alv[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
-            const float* xs_s = a.convert ? ctl->xs + (seg & 3) * 16 : ctl->xs + (seg & 1) * 32;
-            if (a.convert) {
-                seg_end += p1 - p0;
-                while (ok && n_split < seg_end) ok = split_next(true);
-                if (!ok) break;
-                // until this tile's accumulators are complete: write ahead whatever image slot is free
-                while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
-                    if (!split_next(false)) break;
-                }
-            } else {
-                // the token rows' fixed-point units (written by the pre-pass kernel)
-                epi_bar_sync(kFEpiWarps * 32);   // (the readers of this slot, two segments ago, are long done)
-                if (etid < 32) ctl->xs[(seg & 1) * 32 + etid] = (etid < u.ntok) ? __ldcg(a.xscale + u.xrow0 + etid) : 0.f;
-                epi_bar_sync(kFEpiWarps * 32);
+            seg_end += p1 - p0;
+            while (ok && n_split < seg_end) ok = split_next(true);
+            if (!ok) break;
+            // until this tile's accumulators are complete: serve ahead whatever image slot is ready
+            while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
+                if (!split_next(false)) break;
             }
             float* slotp = nullptr;
             if (!whole && a.cluster <= 1) {
@@ -780,12 +738,12 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 // into it has landed and every MMA that read it has completed), token-major, one float per weight
                 // row; the cluster's leader adds the blocks' partials up at the end of the kernel.
                 const FClusterPartOut out{reinterpret_cast<float*>(smem) + row};
-                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, xs_s, am);
+                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, am);
                 break;   // (one segment per block)
             }
             {
                 const EpiOut<false, false> out{Y, slotp, a.N, n, row, u.xrow0, 0.f, a};
-                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, xs_s, am);
+                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, am);
             }
             // this warp's arrival on the "accumulators drained" barrier
             tc_fence_before();

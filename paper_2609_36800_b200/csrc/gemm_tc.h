@@ -24,7 +24,6 @@ struct GemmArgs {
     int n_sets;          // streaming decode kernel: operand sets in tensor memory
     int cluster;         // ... blocks per cluster (one cluster per unit), or 0: flat work list
     int decode_warps;    // ... 8, or (experiments, cluster form) 16
-    int prefetch_steps;  // ... and how many 128-k steps beyond its rings it prefetches into L2 (0: none)
     int early_weights;   // ... 1: its weight loads start before the grid dependency is resolved (0: experiments)
     int trigger_early;   // ... 1: dependents may launch from this kernel's start (0: see trigger_step)
     int trigger_step;    // ... dependents may launch once this many of a block's W_base tiles are queued (or all of them)
@@ -35,7 +34,6 @@ struct GemmArgs {
     uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
     uint32_t col_sf;     // ... first scale-factor column in tensor memory
     const uint8_t* img;  // ... images written by the pre-pass: [group][step][img_bytes]
-    const float* xscale; // ... [B*m] value of one unit of a token row's fixed-point activations
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
@@ -57,7 +55,7 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = (p.pair ? p.grid / 2 : p.grid) / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
-    a.n_sets = p.n_sets; a.cluster = p.cluster; a.decode_warps = 8; a.prefetch_steps = 0;
+    a.n_sets = p.n_sets; a.cluster = p.cluster; a.decode_warps = 8;
     a.early_weights = 1; a.trigger_early = 0; a.trigger_step = 1 << 30;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
@@ -70,7 +68,6 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
     a.fp4 = p.fp4; a.n_img = p.n_img; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
     a.img = reinterpret_cast<const uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
-    a.xscale = reinterpret_cast<const float*>(ws + p.ws_header_bytes + p.ws_partials_bytes + p.ws_scale_off);
     return a;
 }
 
@@ -135,9 +132,9 @@ int max_active_pairs(uint32_t smem_bytes);
 // each group of 32) in X8 [B, 4, m, K].
 cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int f16, cudaStream_t stream);
 
-// The 4-bit decode kernel (plan.fp4).  Pre-pass: per token row its fixed-point unit (xscale) and, per tenant group and
-// 128-k step, the shared-memory image of the activation operands (16-bit tile + eight e2m1 digit rows per token).
-cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, float* xscale, const Plan& p, bool early_start, cudaStream_t stream);
+// The 4-bit decode kernel (plan.fp4).  Pre-pass: per tenant group and 128-k step the shared-memory image of the
+// activation operands (16-bit tile, eight e2m1 digit rows per token, one exponent per token and 32 k).
+cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, const Plan& p, bool early_start, cudaStream_t stream);
 cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                             bool early_start, cudaStream_t stream);
 int fp4_max_active_clusters(uint32_t smem_bytes, int cluster);

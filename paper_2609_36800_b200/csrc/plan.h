@@ -75,7 +75,6 @@ struct Plan {
     int sets_per_step; // ... operand sets per 128-k step (2: eight tenants per unit, 1: four)
     uint32_t img_bytes;   // ... one image: 16-bit activation tile (two atoms) + e2m1 piece tile (64 bytes per row)
     uint32_t col_sf;      // ... first scale-factor column in tensor memory (4 for the A side, then the B side's)
-    size_t ws_scale_off;  // ... offset of the per-token scales behind the images in the activation region
     int a_slots;
     int halves;        // decode: operand hand-overs per 128-k stage (2: 64 k each, 1: the whole stage)
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes, smem_bytes;
@@ -104,10 +103,12 @@ inline int stream_mode() {
     return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
 }
 inline bool stream_enabled() { return stream_mode() != 0; }
-// BITDELTA_FP4=1: the 4-bit decode kernel where it applies (m <= 8).
-inline bool fp4_enabled() {
+// The 4-bit decode kernel (gemm_fp4.cu; m <= 8, plain bf16 calls).  By default it is taken where it measures faster than
+// the 8-bit decode kernels: where its cluster form applies (one tenant group, clusters of 2-8 blocks per W_base tile).
+// BITDELTA_FP4=1: wherever it applies (also the flat work list); BITDELTA_FP4=0: never.
+inline int fp4_mode() {
     const char* e = getenv("BITDELTA_FP4");
-    return e && e[0] == '1';
+    return (e && e[0] == '1') ? 1 : (e && e[0] == '0') ? 0 : 2;
 }
 
 // The cluster form of the streaming kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
@@ -145,7 +146,8 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
         p.stream = (stream_mode() != 0 && p.TB * m <= (stream_mode() == 2 ? 32 : 16)) ? 1 : 0;
-        p.fp4 = (allow_fp4 && fp4_enabled() && m <= kFp4MaxM) ? 1 : 0;
+        if (p.stream) allow_fp4 = false;   // (the streaming kernel was asked for)
+        p.fp4 = (allow_fp4 && fp4_mode() != 0 && m <= kFp4MaxM) ? 1 : 0;
         if (p.fp4) {
             // 4-bit operands: eight e2m1 pieces per token stacked along N (tenant j's rows start at 8 m j), written by
             // a pre-pass together with the 16-bit tile of the base MMA as one image per (tenant group, 128-k step).
@@ -257,6 +259,8 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             }
         }
     }
+    // (default: the 4-bit kernel only in its cluster form)
+    if (p.fp4 && fp4_mode() == 2 && p.cluster <= 1) return make_plan(B, m, N, K, num_sms, tb_override, whole_override, allow_pair, force_tiled, false);
 
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;
@@ -283,7 +287,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     if (p.fp4) {
         // A whole multiprocessor per block: two sign-word slots (256 k each, 32-byte rows: a copy-engine operation costs
         // about a cycle per row whatever its width), three activation images if they fit, the rest for W_base tiles.
-        p.img_bytes = (uint32_t)round_up((int)p.x_tile_bytes + p.x8_rows * 64, 1024);
+        p.img_bytes = (uint32_t)round_up((int)p.x_tile_bytes + p.x8_rows * 64 + 4 * p.TB * p.m, 1024);   // tile, digit rows, scale table
         p.n_bits = 2;
         const int fixed = 1024 + kSmemCtrlBytes + p.n_bits * (int)p.bslot_bytes;
         p.n_img = 3;
@@ -366,9 +370,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.a_slots = slots >= 4 ? 4 : slots >= 2 ? 2 : 0;   // power of two
     if (p.a_slots > kMaxASlots) p.a_slots = kMaxASlots;
     if (p.fp4) {
-        // [base | delta accumulators | 4 + ceil(Nd / 32) scale-factor columns | operand sets of 64 columns]
+        // [base | delta accumulators | scale factors: 4 columns for the A side, 4 per tenant and image slot for the B side |
+        //  operand sets of 64 columns]
         p.col_sf = p.col_a;
-        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + (p.Nd + 31) / 32, 32);
+        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_img, 32);
         p.halves = 2;
         p.n_sets = (kTmemCols - (int)p.col_a) / kFp4SetCols;
         if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
@@ -392,10 +397,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     const long long max_ctas = items < kMaxCtas ? items : kMaxCtas;
     p.ws_partials_bytes = (size_t)2 * (size_t)max_ctas * p.slot_floats * sizeof(float);
     p.ws_x8_bytes = p.decode ? (((size_t)B * kPieces * m * K + 1023) / 1024 * 1024) : 0;
-    if (p.fp4) {   // one image per (tenant group, 128-k step), then one scale per token row
-        p.ws_scale_off = (size_t)p.groups * p.P * p.img_bytes;
-        p.ws_x8_bytes = p.ws_scale_off + (((size_t)B * m * sizeof(float) + 1023) / 1024 * 1024);
-    }
+    if (p.fp4) p.ws_x8_bytes = (size_t)p.groups * p.P * p.img_bytes;   // one image per (tenant group, 128-k step)
     p.ws_bytes = p.ws_header_bytes + p.ws_partials_bytes + p.ws_x8_bytes;
     p.ok = true;
     return p;

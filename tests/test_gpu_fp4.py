@@ -1,0 +1,163 @@
+"""GPU parity tests of the 4-bit decode kernel (csrc/gemm_fp4.cu) against the fp64 CPU oracle: its cluster form (the
+default where it applies), the flat work list (BITDELTA_FP4=1) and the variant whose epilogue warps write the activation
+images themselves (BITDELTA_FP4_INKERNEL=1), at the gates of test_gpu_parity.py; bit and digit order probes; the
+activation range (no value of the bf16 range saturates or is flagged)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_36800_b200 as bd
+from paper_2609_36800_b200 import synth
+
+from gpu_util import assert_parity, run_gemm, to_device, y_to_f64
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # B, m, N, K                 schedule with BITDELTA_FP4=1 (7 flat, 8 clusters)
+    ((1, 1, 128, 128), 7),       # one step
+    ((8, 1, 256, 256), 8),       # eight tenants, clusters of two
+    ((8, 1, 1024, 1024), 8),
+    ((3, 2, 384, 640), 8),       # odd tenant count, five steps over clusters of four
+    ((8, 4, 512, 512), 8),       # 32 token rows per unit, two operand sets per step
+    ((4, 8, 512, 1024), 8),      # four tenants of eight tokens: one operand set per step, 64 digit rows per tenant
+    ((16, 4, 1024, 1024), 7),    # two tenant groups: flat list by teams
+    ((32, 8, 256, 1024), 7),     # eight groups
+    ((5, 3, 130, 384), 7),       # ragged N, 24 digit rows per tenant
+    ((2, 5, 640, 256), 8),       # 40 digit rows per tenant
+    ((7, 1, 2048, 2048), 8),     # 16 tiles x 16 steps, clusters of eight
+    ((16, 1, 512, 1024), 7),
+    ((2, 7, 384, 640), 8),       # 56 digit rows per tenant, five steps over clusters of four
+    ((2, 7, 256, 384), 7),       # ... and three steps on two tiles: flat list
+    ((1, 8, 2176, 512), 8),      # 17 tiles, ragged last tile
+]
+
+
+@pytest.mark.parametrize("inkernel", [0, 1], ids=["prepass", "split_in_kernel"])
+@pytest.mark.parametrize("shape,schedule", SHAPES, ids=[f"B{s[0]}_m{s[1]}_N{s[2]}_K{s[3]}" for s, _ in SHAPES])
+def test_fp4_kernel_matches_oracle(shape, schedule, inkernel, monkeypatch):
+    monkeypatch.setenv("BITDELTA_FP4", "1")
+    if inkernel:
+        monkeypatch.setenv("BITDELTA_FP4_INKERNEL", "1")
+    B, m, N, K = shape
+    assert bd.gemm_plan(B, m, N, K)["schedule"] == schedule
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B * 1000 + m * 100 + N + K)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Y = run_gemm(X, W, bits, alpha)
+    max_abs, rel_fro = assert_parity(Y, oracle.gemm(X, W, bits, alpha), str(shape))
+    assert rel_fro > 1e-5 or max_abs == 0.0   # (a bf16 result cannot sit closer to the fp64 one: guards against comparing a thing with itself)
+
+
+def test_fp4_kernel_one_hot_probe_is_exact():
+    # X = e_k per token, W = 0, alpha = 1  =>  Y[b,t,n] = s[b,n,k_t]: exact in bf16; pins bit, word, digit and tenant order
+    B, m, N, K = 8, 2, 256, 1024
+    assert bd.gemm_plan(B, m, N, K)["schedule"] == 8
+    rng = np.random.default_rng(5)
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    ks = rng.integers(0, K, size=(B, m))
+    ks[:4, 0] = [0, 31, 32, K - 1]
+    x = np.zeros((B, m, K), dtype=np.float32)
+    for b in range(B):
+        for t in range(m):
+            x[b, t, ks[b, t]] = 1.0 if (b + t) % 2 == 0 else -3.0
+    X = synth.f32_to_bf16_bits(x)
+    W = np.zeros((N, K), dtype=np.uint16)
+    alpha = np.ones(B, dtype=np.float32)
+    assert np.array_equal(run_gemm(X, W, bits, alpha), oracle.gemm(X, W, bits, alpha))
+
+
+def test_fp4_kernel_every_mantissa_and_exponent_offset_is_exact():
+    # One 32-k group per token holds values 2^-s * (1 + f/128), s = 0..8 below the group's largest: all eight
+    # significant bits of each survive the 16-bit fixed point (alpha a power of two, W = 0, so the product is exact
+    # in fp32 and rounds to bf16 like the oracle's).
+    B, m, N, K = 2, 4, 128, 256
+    rng = np.random.default_rng(9)
+    x = np.zeros((B, m, K), dtype=np.float32)
+    for b in range(B):
+        for t in range(m):
+            g = 32 * ((3 * b + t) % (K // 32))
+            x[b, t, g] = 1.9921875                      # the group's largest: 255/128
+            for i in range(1, 32):
+                s = i % 9
+                x[b, t, g + i] = (1.0 + rng.integers(0, 128) / 128.0) * 2.0**-s * (1 if i % 3 else -1)
+    X = synth.f32_to_bf16_bits(x)
+    W = np.zeros((N, K), dtype=np.uint16)
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    alpha = np.full(B, 0.0078125, dtype=np.float32)
+    Y, Yref = run_gemm(X, W, bits, alpha), oracle.gemm(X, W, bits, alpha)
+    # (the sum of 32 terms with at most 17 significant bits is exact in fp32; only the final bf16 rounding differs from fp64)
+    assert np.max(np.abs(Y - Yref)) <= np.max(np.abs(Yref)) * 2.0**-8
+
+
+def _gate(Y, Yref):
+    tol = np.maximum(2e-2, np.abs(Yref) * 2.0**-8)
+    bad = np.abs(Y - Yref) > tol
+    assert not bad.any(), f"{int(bad.sum())} outputs off, worst {np.max(np.abs(Y - Yref) / tol):.2f} x the gate"
+
+
+@pytest.mark.parametrize("big", [2.0**15, 65280.0, 2.0**17, 2.0**60], ids=["2^15", "65280", "2^17", "2^60"])
+@pytest.mark.parametrize("shape", [(4, 1, 256, 512), (2, 8, 256, 512)], ids=["m1", "m8"])
+def test_fp4_kernel_has_no_range_limit(shape, big):
+    B, m, N, K = shape
+    assert bd.gemm_plan(B, m, N, K)["schedule"] == 8
+    rng = np.random.default_rng(int(np.log2(big)) + B + m)
+    x = rng.standard_normal((B, m, K)).astype(np.float32)
+    x[:, 0, ::7] = big                       # large magnitudes, both signs, scattered over every 32-k group
+    x[:, 0, 3::11] = -big
+    x[0, m - 1, :] = big                     # a whole row of them
+    sub = np.float32(2.0**-130)              # a bf16 subnormal
+    x[B - 1, m - 1, ::2] = sub
+    x[B - 1, m - 1, 1::2] = -sub
+    w = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    bits = rng.integers(0, 2**32, size=(B, N, K // 32), dtype=np.uint32)
+    alpha = rng.uniform(0.001, 0.01, B).astype(np.float32)
+    X, W = synth.f32_to_bf16_bits(x), synth.f32_to_bf16_bits(w)
+    dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
+    Y = y_to_f64(bd.gemm(dX, dW, dbits, dalpha))
+    st, site = bd.last_device_status()
+    assert st == 0, (st, site)
+    Yref = oracle.gemm(X, W, bits, alpha)
+    fin = np.abs(Yref) < 3.0e38              # (2^60 * K overflows bf16 in some rows: both sides give infinity there)
+    assert np.isfinite(Y[fin]).all()
+    # Values more than 8 binades below their 32-k group's largest are truncated below 2^-16 of it (16-bit fixed point per
+    # group): at worst alpha * sum over groups of 32 * 2^-16 * max|x| on top of the usual gate.
+    gmax = np.abs(synth.bf16_bits_to_f32(X).astype(np.float64)).reshape(B, m, K // 32, 32).max(axis=3).sum(axis=2)   # [B, m]
+    extra = (alpha.astype(np.float64)[:, None] * 32 * 2.0**-16 * gmax)[:, :, None]
+    tol = np.maximum(2e-2, np.abs(Yref) * 2.0**-8) + extra
+    bad = fin & (np.abs(Y - Yref) > tol)
+    assert not bad.any(), f"{int(bad.sum())} outputs off, worst {np.nanmax(np.where(fin, np.abs(Y - Yref) / tol, 0)):.2f} x the gate"
+    # rows without a large value are untouched by it: the plain gate
+    plain = ~(np.abs(synth.bf16_bits_to_f32(X)) >= big).any(axis=2)
+    _gate(Y[plain], Yref[plain])
+    # the row of subnormals: its delta term is alpha * 2^-130 * (sum of signs), far below the base term's rounding
+    assert np.isfinite(Y[B - 1, m - 1]).all()
+
+
+def test_fp4_kernel_headline_shape_default_route_and_determinism():
+    wl = synth.WORKLOADS_BY_NAME["decode_attn"]
+    assert bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"] == 8     # no environment variable: the default route
+    X, W, bits, alpha = synth.make_inputs(wl)
+    Y1 = run_gemm(X, W, bits, alpha)
+    assert_parity(Y1, oracle.gemm(X, W, bits, alpha), "decode_attn")
+    dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
+    outs = [bd.gemm(dX, dW, dbits, dalpha) for _ in range(4)]        # back to back: pre-pass and GEMM alternate on the stream
+    torch.cuda.synchronize()
+    st, site = bd.last_device_status()
+    assert st == 0, (st, site)
+    for Y in outs:
+        assert np.array_equal(y_to_f64(Y), Y1)
+
+
+def test_calls_with_options_keep_the_eight_bit_kernels():
+    # binary16 / bias / activation calls never take the 4-bit kernel; same shape, same workspace
+    B, m, N, K = 8, 1, 1024, 1024
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=21)
+    X, W, bits, alpha, bias = synth.make_inputs_f16(wl)
+    f16 = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.float16)
+    Y = bd.gemm(f16(X), f16(W), torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(alpha).cuda(), bias=f16(bias), act="silu")
+    st, site = bd.last_device_status()
+    assert st == 0, (st, site)
+    ref = oracle.gemm_ex(X, W, bits, alpha, bias=bias, dtype="f16", act="silu")
+    d = Y.cpu().numpy().astype(np.float64) - ref
+    assert np.max(np.abs(d)) <= 2e-2

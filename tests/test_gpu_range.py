@@ -17,6 +17,12 @@ from gpu_util import to_device, y_to_f64
 
 pytestmark = pytest.mark.gpu
 
+
+@pytest.fixture(autouse=True)
+def eight_bit_decode_kernels(monkeypatch):
+    # (the 4-bit decode kernel, which takes some of these shapes by default, has no range limit: test_gpu_fp4.py)
+    monkeypatch.setenv("BITDELTA_FP4", "0")
+
 # (B, m, N, K): in-kernel split; pre-pass split (B >= 3 tenants of 8 tokens: 32 rows per unit); tiled schedule
 SCHEDULES = {"in_kernel_m1": ((4, 1, 256, 512), 2), "prepass_m8": ((5, 8, 256, 512), 1), "tiled_m40": ((2, 40, 256, 512), 0)}
 

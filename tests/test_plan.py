@@ -77,13 +77,34 @@ def test_every_item_is_taken_exactly_once(shape, sms):
 
 def test_schedules_and_work_orders_of_the_measured_workloads():
     got = {w.name: bd.gemm_plan(w.B, w.m, w.N, w.K) for w in synth.WORKLOADS}
-    assert got["decode_attn"]["schedule"] == 2 and got["decode_attn"]["order"] == 0 and got["decode_attn"]["blocks"] == 148
+    # one tenant group, eight tokens per unit: the 4-bit decode kernel in clusters of four blocks per W_base tile
+    assert got["decode_attn"]["schedule"] == 8 and got["decode_attn"]["order"] == 3 and got["decode_attn"]["blocks"] == 128
     assert got["tiny"]["schedule"] == 2
     assert got["decode_mlp_up"]["schedule"] == 1 and got["decode_mlp_up"]["order"] == 2 and got["decode_mlp_up"]["teams"] == 2
     assert got["many_tenant_down"]["order"] == 2 and got["many_tenant_down"]["teams"] == 8 and got["many_tenant_down"]["blocks"] == 144
     assert got["prefill"]["schedule"] == 4 and got["prefill"]["order"] == 0 and got["prefill"]["blocks"] == 148
     for g in got.values():
         assert g["smem_bytes"] <= 227 * 1024 and g["w_ring"] >= 2 and g["operand_buffers"] >= 2
+
+
+def test_four_bit_decode_kernel_plans(monkeypatch):
+    # default: only where its cluster form applies; BITDELTA_FP4=0 never; BITDELTA_FP4=1 also on the flat work list
+    assert bd.gemm_plan(8, 1, 4096, 4096)["schedule"] == 8 and bd.gemm_plan(4, 8, 4096, 4096)["schedule"] == 8
+    assert bd.gemm_plan(16, 1, 4096, 4096)["schedule"] == 2          # two tenant groups: no clusters
+    assert bd.gemm_plan(8, 9, 4096, 4096)["schedule"] == 1           # more than eight tokens per tenant
+    one = bd.gemm_plan(8, 1, 4096, 4096)
+    assert one["smem_bytes"] <= 227 * 1024 and one["w_ring"] >= 3
+    for b in range(one["blocks"]):
+        lo, hi = bd.gemm_plan_cta_items(8, 1, 4096, 4096, b)
+        assert hi - lo == 8 and lo // 32 == b // 4 and bd.gemm_plan_item_cta(8, 1, 4096, 4096, lo) == b
+    monkeypatch.setenv("BITDELTA_FP4", "0")
+    off = bd.gemm_plan(8, 1, 4096, 4096)
+    assert off["schedule"] == 2 and off["order"] == 0 and off["blocks"] == 148
+    monkeypatch.setenv("BITDELTA_FP4", "1")
+    assert bd.gemm_plan(16, 4, 11008, 4096)["schedule"] == 7 and bd.gemm_plan(32, 8, 4096, 14336)["schedule"] == 7
+    # the workspace covers every schedule a call may take
+    monkeypatch.delenv("BITDELTA_FP4")
+    assert bd.gemm_workspace_bytes(8, 1, 4096, 4096) >= 32 * 9 * 1024
 
 
 def test_streaming_decode_kernel_plans(monkeypatch):
