@@ -397,6 +397,7 @@ def kernels_per_step(wl):
     """Kernels one bitdelta_gemm call launches, from the library's own plan: the GEMM kernel, plus an activation
     pre-pass kernel in the 4-bit decode schedule and in the 8-bit decode schedule with more than 16 token rows per
     unit (otherwise the GEMM kernel splits the activations itself)."""
+    import paper_2609_36800_b200 as bd
     schedule = bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"]
     if schedule in (7, 8):
         return 1 if os.environ.get("BITDELTA_FP4_INKERNEL") else 2
@@ -404,6 +405,7 @@ def kernels_per_step(wl):
 
 
 def gemm_kernel_name(wl):
+    import paper_2609_36800_b200 as bd
     schedule = bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"]
     return {7: "bitdelta_gemm_fp4_kernel", 8: "bitdelta_gemm_fp4_kernel", 5: "bitdelta_gemm_stream_kernel",
             6: "bitdelta_gemm_stream_kernel", 3: "gemm_simt_kernel"}.get(schedule, "bitdelta_gemm_tc_kernel")
