@@ -108,9 +108,15 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * X, W_base, bits and Y must be 16-byte aligned; K a multiple of 32.
  * Asynchronous on the stream; a kernel-side wait that expires is reported by
  * bitdelta_last_device_status, not here.
- * Range of X in the decode schedules (m <= 16): there the delta term runs on the
- * 8-bit float tensor path, with every activation rewritten exactly as a sum of
- * e5m2 numbers, which have binary16's exponent range.  Finite bf16 activations
+ * Precision of X in the decode schedules (m <= 16): there the delta term runs on
+ * a narrow-float tensor path.  bitdelta_gemm_plan tells which of two a shape gets.
+ * 4-bit schedules (plan codes 7, 8; m <= 8, calls without options): every group
+ * of 32 consecutive k of a token row is held as 16-bit fixed point relative to the
+ * group's largest magnitude.  Values within a factor 2^8 of it are exact; smaller
+ * ones lose what lies below 2^-16 of it (DELTA term only; the base term always
+ * uses the bf16 value).  Nothing is clamped or flagged, whatever the magnitude.
+ * 8-bit schedules (plan codes 1, 2, 5, 6): every activation is rewritten exactly
+ * as a sum of e5m2 numbers, which have binary16's exponent range.  Finite bf16 activations
  * with |x| < 2^16 are exact down to 2^-16 (smaller parts of x, at most 2^-16 per
  * element, are dropped from the DELTA term only; the base term always uses the
  * bf16 value).  An activation with |x| >= 2^16 (or an infinity / NaN) is clamped
@@ -118,7 +124,8 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * flagged: bitdelta_last_device_status then returns BITDELTA_ERR_RANGE.  Inputs
  * like that need bitdelta_gemm_ex with BITDELTA_DTYPE_WIDE_RANGE, which runs any
  * m on the tiled schedule (bf16 operands for both terms: exact for every finite
- * input).  The tiled schedules (m > 16) have no such limit.
+ * input, and the route to take when neither narrow form is wanted).  The tiled
+ * schedules (m > 16) have no such limit.
  * Early start: the kernel is queued so that it may begin (prologue, prefetch of
  * W_base, bits and alpha) while the kernel queued on the stream just before it
  * is still running; it reads X and writes Y and the workspace only after that
@@ -226,7 +233,10 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
  *   [0] schedule: 0 tiled, 1 decode with a pre-pass activation split, 2 decode with the in-kernel split,
  *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then), 4 tiled on pairs of
  *       thread blocks (a unit is then two W_base tiles, [3] and the work list count such pairs, and [1] is
- *       twice the number of pairs that cut the list)
+ *       twice the number of pairs that cut the list), 5 / 6 the streaming 8-bit decode kernel on the flat work
+ *       list / in clusters (only with BITDELTA_STREAM set in the environment), 7 / 8 the 4-bit decode kernel on
+ *       the flat work list / in clusters (8 is the default wherever it applies: m <= 8, one tenant group,
+ *       2-8 blocks per W_base tile; BITDELTA_FP4=0 in the environment turns it off, =1 also takes 7)
  *   [1] thread blocks   [2] tenants per unit (tiled schedule: more than one in the middle regime,
  *       16 < m <= 64, where several tenants share a W_base tile)   [3] units   [4] P, k-steps per unit
  *   [5] work order: 0 one even cut of the list, 1 whole units round-robin (block b: units b, b+blocks, ...),
