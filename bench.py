@@ -407,8 +407,7 @@ def kernels_per_step(wl):
 def gemm_kernel_name(wl):
     import paper_2609_36800_b200 as bd
     schedule = bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"]
-    return {7: "bitdelta_gemm_fp4_kernel", 8: "bitdelta_gemm_fp4_kernel", 5: "bitdelta_gemm_stream_kernel",
-            6: "bitdelta_gemm_stream_kernel", 3: "gemm_simt_kernel"}.get(schedule, "bitdelta_gemm_tc_kernel")
+    return {7: "bitdelta_gemm_fp4_kernel", 8: "bitdelta_gemm_fp4_kernel", 3: "gemm_simt_kernel"}.get(schedule, "bitdelta_gemm_tc_kernel")
 
 
 def summarize(wl, ms_total, steps, n_gpus, peaks, clocks=None):

@@ -100,7 +100,7 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * workspace / workspace_bytes : at least bitdelta_gemm_workspace_bytes(B,m,N,K),
  *          prepared once by bitdelta_workspace_init; calls that may overlap on
  *          the device must not share a workspace.
- * m <= 16 selects the streaming (decode) schedule, larger m the tiled (prefill)
+ * m <= 16 selects a decode schedule, larger m the tiled (prefill)
  * schedule (several tenants per tile up to m = 64; pairs of thread blocks with
  * 256-row MMAs for m > 64); all run on tcgen05 tensor cores with TMEM
  * accumulators, and bitdelta_gemm_plan tells which one a shape gets.  Shapes
@@ -115,7 +115,7 @@ int bitdelta_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_
  * group's largest magnitude.  Values within a factor 2^8 of it are exact; smaller
  * ones lose what lies below 2^-16 of it (DELTA term only; the base term always
  * uses the bf16 value).  Nothing is clamped or flagged, whatever the magnitude.
- * 8-bit schedules (plan codes 1, 2, 5, 6): every activation is rewritten exactly
+ * 8-bit schedules (plan codes 1, 2): every activation is rewritten exactly
  * as a sum of e5m2 numbers, which have binary16's exponent range.  Finite bf16 activations
  * with |x| < 2^16 are exact down to 2^-16 (smaller parts of x, at most 2^-16 per
  * element, are dropped from the DELTA term only; the base term always uses the
@@ -233,8 +233,7 @@ int bitdelta_gemm_host(const void* X_host, const void* W_base_host, const uint32
  *   [0] schedule: 0 tiled, 1 decode with a pre-pass activation split, 2 decode with the in-kernel split,
  *       3 CUDA-core kernel (K not a multiple of 128; all other entries are 0 then), 4 tiled on pairs of
  *       thread blocks (a unit is then two W_base tiles, [3] and the work list count such pairs, and [1] is
- *       twice the number of pairs that cut the list), 5 / 6 the streaming 8-bit decode kernel on the flat work
- *       list / in clusters (only with BITDELTA_STREAM set in the environment), 7 / 8 the 4-bit decode kernel on
+ *       twice the number of pairs that cut the list), 7 / 8 the 4-bit decode kernel on
  *       the flat work list / in clusters (8 is the default wherever it applies: m <= 8, one tenant group,
  *       2-8 blocks per W_base tile; BITDELTA_FP4=0 in the environment turns it off, =1 also takes 7)
  *   [1] thread blocks   [2] tenants per unit (tiled schedule: more than one in the middle regime,

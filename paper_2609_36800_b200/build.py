@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(HERE, "libbitdelta.so")
-SOURCES = ["api.cu", "gemm_tc.cu", "gemm_stream.cu", "gemm_fp4.cu", "kernels_simple.cu"]
+SOURCES = ["api.cu", "gemm_tc.cu", "gemm_fp4.cu", "kernels_simple.cu"]
 HEADERS = ["ptx.cuh", "plan.h", "gemm_tc.h", "gemm_common.cuh", os.path.join("..", "..", "include", "bitdelta.h")]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
@@ -62,9 +62,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 def build_trace() -> str:
-    """The same library with -DBD_TRACE as libbitdelta_trace.so: the streaming decode kernel then stamps a
-    per-block timeline into a buffer set with bitdelta_debug_set_trace (see csrc/gemm_stream.cu).  Load it by
-    pointing BITDELTA_LIB at it.  Never the default build: the stamps cost time."""
+    """The same library with -DBD_TRACE as libbitdelta_trace.so: the 4-bit decode kernel then adds up, per block and
+    role, the cycles spent in each kind of wait into a buffer set with bitdelta_debug_set_trace_fp4 (see
+    csrc/gemm_fp4.cu).  Load it by pointing BITDELTA_LIB at it.  Never the default build: the stamps cost time."""
     os.makedirs(OBJ, exist_ok=True)
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
         objs = list(pool.map(lambda s: _compile(s, True, False, trace=True), SOURCES))

@@ -359,16 +359,14 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         // The cluster form wants all its clusters resident at once (clusters are independent, so this is about
         // speed, not progress); where the device cannot hold them, the flat work list is planned.
         static std::mutex mu;
-        static int fit_cache[64][4][3] = {};   // [device][log2 cluster][smem above half a multiprocessor; 2: the 4-bit kernel]: 0 unknown, else n + 1
+        static int fit_cache[64][4] = {};   // [device][log2 cluster]: 0 unknown, else clusters that fit + 1
         const int di = (d.device >= 0 && d.device < 64) ? d.device : 0;
         const int ci = p.cluster == 8 ? 3 : (p.cluster == 4 ? 2 : 1);
-        const int si = p.fp4 ? 2 : (p.smem_bytes > (uint32_t)bd::kStreamSmemBudget ? 1 : 0);
         int n;
         {
             std::lock_guard<std::mutex> lock(mu);
-            if (fit_cache[di][ci][si] == 0)
-                fit_cache[di][ci][si] = (p.fp4 ? bd::fp4_max_active_clusters(p.smem_bytes, p.cluster) : bd::stream_max_active_clusters(p.smem_bytes, p.cluster)) + 1;
-            n = fit_cache[di][ci][si] - 1;
+            if (fit_cache[di][ci] == 0) fit_cache[di][ci] = bd::fp4_max_active_clusters(p.smem_bytes, p.cluster) + 1;
+            n = fit_cache[di][ci] - 1;
         }
         const int need = p.grid / p.cluster;
         if (n < need) p = bd::make_plan(B, m, N, K, d.sms, tb_override(), whole_override(), false, false, plain);
@@ -384,7 +382,7 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     if (!p.stream && !cached_map(&tmX, MapKey{0, X, (uint64_t)B * m, (uint64_t)K, 0, (uint32_t)p.x_rows, 0u},
                                  [&](CUtensorMap* mp) { return encode_bf16_tile(mp, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows); }))
         return BITDELTA_ERR_CUDA;
-    const uint32_t box_words = (p.stream && !p.fp4) ? 4u : 8u;
+    const uint32_t box_words = 8u;
     if (!cached_map(&tmBits, MapKey{1, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words},
                     [&](CUtensorMap* mp) { return encode_bits_3d(mp, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words); }))
         return BITDELTA_ERR_CUDA;
@@ -415,19 +413,10 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     args.f16 = f16; args.act = act; args.bias = bias;
     args.X = X;
     { static int h = -1; if (h < 0) { const char* e = getenv("BITDELTA_HOLD"); h = (e && e[0] == '0') ? 0 : 1; } args.hold_prefetch = h; }
-#ifdef BD_TRACE
-    args.hold_prefetch = (int)(g_launches.load() & 1);   // trace build: alternate halves of the trace buffer
-#endif
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_EARLY_WEIGHTS"); d = (e && e[0] == '0') ? 0 : 1; } args.early_weights = d; }
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_STEP"); d = e ? atoi(e) : (1 << 30); } args.trigger_step = d; }
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_TRIGGER_EARLY"); d = (e && e[0] == '1') ? 1 : 0; } args.trigger_early = d; }
-    { static int d = -1; if (d < 0) { const char* e = getenv("BITDELTA_DECODE_WARPS"); d = (e && atoi(e) == 16) ? 16 : 8; } args.decode_warps = d; }
     // (a GEMM queued right behind the library's own pack / compress must not prefetch what they are still writing)
     const bool early = early_start_enabled() && g_weights_just_written.exchange(0) == 0;
     const cudaError_t le = p.fp4
         ? bd::launch_gemm_fp4(tmW, tmBits, args, p.grid, p.smem_bytes, early, stream)
-        : p.stream
-        ? bd::launch_gemm_stream(tmW, tmBits, args, p.grid, p.smem_bytes, early, stream)
         : bd::launch_gemm_tc(tmW, tmX, tmX8, tmBits, args, p.grid, p.smem_bytes, early, stream);
     if (le != cudaSuccess) return BITDELTA_ERR_CUDA;
     g_launches++;
@@ -493,7 +482,7 @@ int bitdelta_gemm_plan(int B, int m, int N, int K, int num_sms, int* info) {
     if ((K % 128) != 0) { info[0] = 3; return BITDELTA_OK; }
     bd::Plan p = bd::make_plan(B, m, N, K, num_sms, tb_override(), whole_override());
     if (!p.ok) return BITDELTA_ERR_SHAPE;
-    info[0] = !p.decode ? (p.pair ? 4 : 0) : p.fp4 ? (p.cluster > 1 ? 8 : 7) : (p.stream ? (p.cluster > 1 ? 6 : 5) : (p.convert ? 2 : 1));
+    info[0] = !p.decode ? (p.pair ? 4 : 0) : p.fp4 ? (p.cluster > 1 ? 8 : 7) : (p.convert ? 2 : 1);
     info[1] = p.grid; info[2] = p.TB; info[3] = p.units; info[4] = p.P;
     info[5] = p.cluster > 1 ? 3 : (p.whole_units ? 1 : (p.teams > 1 ? 2 : 0));
     info[6] = p.teams; info[7] = (int)p.smem_bytes; info[8] = p.n_w; info[9] = p.n_x; info[10] = p.n_x8;

@@ -1,5 +1,5 @@
 // Device-side helpers shared by the tcgen05 BitDelta GEMM kernels (the tiled / grouped schedules in
-// gemm_tc.cu and the streaming decode schedule in gemm_stream.cu): bounded mbarrier waits, the walk over a
+// gemm_tc.cu and the 4-bit decode kernel in gemm_fp4.cu): bounded mbarrier waits, the walk over a
 // thread block's share of the work list, sign decode, the fused epilogues, the split-K fix-up and the
 // in-kernel activation split.  Every translation unit that includes this file gets its own copy of the
 // device status word; read_device_status() looks at all of them.

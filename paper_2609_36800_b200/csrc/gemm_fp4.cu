@@ -2,8 +2,9 @@
 //
 //   Y[b,t,n] = sum_k X[b,t,k] W[n,k] + alpha[b] sum_k X[b,t,k] S[b,n,k]
 //
-// Same orientation, roles and work split as the streaming decode kernel (gemm_stream.cu), but the delta term
-// runs on the block-scaled 4-bit tensor path (tcgen05.mma kind::mxf4, K = 64 per instruction):
+// Same orientation as the other kernels (weight rows on the MMA's M side, tokens on its N side, decoded signs written
+// to tensor memory as the A operand), work split and split-K fix-up as in gemm_tc.cu; the delta term runs on the
+// block-scaled 4-bit tensor path (tcgen05.mma kind::mxf4, K = 64 per instruction):
 //   * Signs are decoded to e2m1 (+1 = 0x2, -1 = 0xA), EIGHT per 32-bit register: per sign word three shifts and four
 //     logic operations, four tensor-memory columns.  That is half the integer work and half the tensor-memory store
 //     traffic of the 8-bit form, the two things that bound the decode schedules, and half the MMA instructions.
@@ -46,6 +47,7 @@ constexpr int kFThreads = (kFWarpEpi0 + kFEpiWarps) * 32;   // 512
 constexpr int kFHandover = kFDecodeWarps / 2 * 32 + 32;      // the four decode warps of a tenant half arrive, its issuer warp syncs
 constexpr int kFBarSet0 = 2;                     // named barrier of operand set s, tenant half h: id 2 + 2 s + h
 constexpr int kFBarDep = 15;                     // the decode and epilogue warps sleep on it until the grid dependency resolves
+constexpr int kFBarImg = 14;                     // resident form: all warps but the producer have written their share of the images
 
 #ifdef BD_TRACE
 // Trace build: per block 32 accumulators (cycles) written at the end of each role; see bitdelta_debug_set_trace_fp4.
@@ -66,7 +68,7 @@ struct FCtl {
     uint64_t bempty[4];             // ... and are in the decode warps' registers (8 arrivals)
     uint64_t pfull[4];              // a step's activation image landed
     uint64_t pempty[4];             // ... and was read by the step's MMAs
-    uint64_t opfree[2][kStreamMaxSets];   // tenant half h's columns of an operand set in tensor memory free again
+    uint64_t opfree[2][kFp4MaxSets];   // tenant half h's columns of an operand set in tensor memory free again
     uint64_t accfull;               // all MMAs of a segment have completed
     uint64_t accempty;              // the accumulators were drained (4 epilogue warps)
     uint64_t depready;              // the grid this launch depends on has completed
@@ -128,28 +130,42 @@ __device__ __forceinline__ void fp4_digits8(const uint32_t* hv, int E, uint32_t*
 // The four tasks c = 0..3 of a word sit in neighbouring lanes (all active together) and share the group's exponent,
 // which task c = 0 writes to the image's scale table (byte 4 r_local + wd).  `xstep`: the row's first value of the
 // step; `im`: the step's image (global or shared memory): [16-bit tile | digit rows | scale table].
-__device__ __forceinline__ void fp4_split_task(const uint16_t* __restrict__ xstep, uint8_t* im, int tk, int r_local, int j, int t,
-                                               int m, uint32_t x_atom_bytes, uint32_t x_tile_bytes, uint32_t sf_off) {
-    const uint4 chunk = __ldcg(reinterpret_cast<const uint4*>(xstep) + tk);
-    *reinterpret_cast<uint4*>(im + (tk >> 3) * x_atom_bytes + r_local * 128 + (((tk & 7) ^ (r_local & 7)) * 16)) = chunk;
+struct Fp4TaskData {
+    uint4 chunk;       // the task's 16-byte chunk of the 16-bit tile
+    uint32_t hv[8];    // the eight values k = 32 wd + 4i + c
+};
+__device__ __forceinline__ void fp4_task_load(const uint16_t* __restrict__ xstep, int tk, Fp4TaskData& d) {
+    // (through L1: the four tasks of a word read the same 64 bytes, and X is not written while this kernel may read it)
+    d.chunk = __ldg(reinterpret_cast<const uint4*>(xstep) + tk);
     const int wd = tk >> 2, c = tk & 3;
-    uint32_t hv[8], R[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) hv[i] = __ldcg(xstep + 32 * wd + 4 * i + c);
+    for (int i = 0; i < 8; ++i) d.hv[i] = __ldg(xstep + 32 * wd + 4 * i + c);
+}
+__device__ __forceinline__ void fp4_task_finish(const Fp4TaskData& d, uint8_t* im, int tk, int r_local, int j, int t, int m,
+                                                uint32_t x_atom_bytes, uint32_t x_tile_bytes, uint32_t sf_off) {
+    *reinterpret_cast<uint4*>(im + (tk >> 3) * x_atom_bytes + r_local * 128 + (((tk & 7) ^ (r_local & 7)) * 16)) = d.chunk;
+    const int wd = tk >> 2, c = tk & 3;
+    uint32_t R[8];
     uint32_t mx = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mx = max(mx, hv[i] & 0x7FFFu);
+    for (int i = 0; i < 8; ++i) mx = max(mx, d.hv[i] & 0x7FFFu);
     const unsigned act = __activemask();
     mx = max(mx, __shfl_xor_sync(act, mx, 1));
     mx = max(mx, __shfl_xor_sync(act, mx, 2));
     const int E = min(max((int)(mx >> 7), 1), 240);
-    fp4_digits8(hv, E, R);
+    fp4_digits8(d.hv, E, R);
 #pragma unroll
     for (int q = 0; q < kFp4Pieces; ++q) {
         const int n = j * (kFp4Pieces * m) + q * m + t;
         *reinterpret_cast<uint32_t*>(im + x_tile_bytes + n * 64 + ((wd ^ ((n >> 1) & 3)) * 16) + 4 * c) = R[q];
     }
     if (c == 0) im[sf_off + 4 * r_local + wd] = (uint8_t)E;
+}
+__device__ __forceinline__ void fp4_split_task(const uint16_t* __restrict__ xstep, uint8_t* im, int tk, int r_local, int j, int t,
+                                               int m, uint32_t x_atom_bytes, uint32_t x_tile_bytes, uint32_t sf_off) {
+    Fp4TaskData d;
+    fp4_task_load(xstep, tk, d);
+    fp4_task_finish(d, im, tk, r_local, j, t, m, x_atom_bytes, x_tile_bytes, sf_off);
 }
 
 // ---------------------------------------------------------------------------------------------- pre-pass
@@ -321,7 +337,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             mbar_init(smem_u32(&ctl->imgready[s]), kFEpiWarps);
             mbar_init(smem_u32(&ctl->pempty[s]), 3);   // (the three issuers)
         }
-        for (int s = 0; s < kStreamMaxSets; ++s) {
+        for (int s = 0; s < kFp4MaxSets; ++s) {
             mbar_init(smem_u32(&ctl->opfree[0][s]), 1);
             mbar_init(smem_u32(&ctl->opfree[1][s]), 1);
         }
@@ -336,6 +352,42 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     __syncthreads();
 
     const uint32_t tmemready = smem_u32(&ctl->tmemready);
+    // Resident form (cluster form, one segment per block): once the grid dependency has resolved, all warps but the
+    // producer write the images of all the block's steps, one task per thread and (token row, 16-byte chunk, step).
+    auto write_resident_images = [&]() {
+        const int cunit = (int)blockIdx.x / a.cluster;
+        const Unit u = unit_info(a, cunit);
+        const int q0 = lo - cunit * a.P, nsteps = hi - lo;
+        const int tid = (int)threadIdx.x - 32;
+        const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
+        const int per_step = u.ntok * 16;
+        // (three tasks per thread requested together: the whole split costs one round trip to X per 1440 tasks)
+        for (int task0 = tid; task0 < nsteps * per_step; task0 += 3 * (kFThreads - 32)) {
+            Fp4TaskData d[3];
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                const int task = task0 + q * (kFThreads - 32);
+                if (task < nsteps * per_step) {
+                    const int st = (int)((unsigned)task / (unsigned)per_step);
+                    const int rem = task - st * per_step;
+                    fp4_task_load(reinterpret_cast<const uint16_t*>(a.X) + (size_t)(u.xrow0 + (rem >> 4)) * a.K + (size_t)(q0 + st) * kPairK, rem & 15, d[q]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                const int task = task0 + q * (kFThreads - 32);
+                if (task < nsteps * per_step) {
+                    const int st = (int)((unsigned)task / (unsigned)per_step);
+                    const int rem = task - st * per_step;
+                    const int r = rem >> 4;
+                    const int j = r / am, t = r - j * am;
+                    fp4_task_finish(d[q], smem + img_off + st * a.img_bytes, rem & 15, r, j, t, am, a.x_atom_bytes, a.x_tile_bytes, sf_off);
+                }
+            }
+        }
+        fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
+        named_bar_sync(kFBarImg, kFThreads - 32);
+    };
 
     if (warp == kFWarpProducer) {
         // ------------------------------------------------------------ producer
@@ -343,7 +395,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // another kernel: queued before the grid dependency is resolved, as far as their rings allow) and activation
         // images (written by the pre-pass kernel queued before this one: only afterwards).
         ItemIter wi(it), bi(it), xi(it);
-        Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, a.n_img};
+        Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, a.n_sf};
         Unit uw{}, ub{}, ux{};
         bool more_w = wi.next(), more_b = bi.next(), more_x = !a.convert && xi.next();   // (convert: the epilogue warps write the images)
         if (more_w) { uw = unit_info(a, wi.unit); ub = uw; ux = uw; }
@@ -417,11 +469,15 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
         bool ok = true;
+        if (a.resident) {
+            grid_dependency_wait();   // (returns at once: orders this thread's reads of X behind the previous kernel)
+            write_resident_images();
+        }
 
         const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
         const uint64_t desc128 = make_smem_desc_sw128(0);
         const uint32_t x_atom16 = a.x_atom_bytes >> 4;
-        Ring wr{0, 0u, a.n_w}, pr{0, 0u, a.n_img};
+        Ring wr{0, 0u, a.n_w}, pr{0, 0u, a.n_sf};
         uint32_t accphase = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
@@ -437,7 +493,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
                 if (!ok) break;
-                const uint32_t img_s = img_addr + pr.idx * a.img_bytes;
+                const uint32_t img_s = img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes;
                 const uint64_t xdesc = desc128 + (img_s >> 4);
                 ok = warp_all(wait_bar(smem_u32(&ctl->wfull[wr.idx]), wr.par, abort_flag, 4));
                 FT_ADD(3);
@@ -479,11 +535,15 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         bool ok = warp_all(wait_bar(tmemready, 0, abort_flag, 20));
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
+        if (a.resident) {
+            grid_dependency_wait();
+            write_resident_images();
+        }
         const uint32_t idesc_delta = make_idesc_mxf4(kTileN, (uint32_t)a.Nd);   // (+ the B-side scale id: which pair of a step's four 32-k groups)
         const uint64_t desc64 = make_smem_desc_sw64(0);
         const uint32_t ten_rows16 = (uint32_t)a.Nd * 4u;      // a tenant's digit rows x 64 B >> 4
         const uint32_t sfa = tmem_base + a.col_sf;
-        Ring pr{0, 0u, a.n_img}, sr{0, 0u, a.n_sets};
+        Ring pr{0, 0u, a.n_sf}, sr{0, 0u, a.n_sets};
         uint32_t accphase = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
@@ -501,7 +561,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sfb0 = sfa + 4u + (uint32_t)(pr.idx * 4 * a.TB);   // this image slot's scale factors (four columns per tenant)
-                const uint64_t x4desc = desc64 + ((img_addr + pr.idx * a.img_bytes + a.x_tile_bytes) >> 4);
+                const uint64_t x4desc = desc64 + ((img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes + a.x_tile_bytes) >> 4);
 #pragma unroll
                 for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
                     // The 128 decode threads of this half arrive here once their columns of the set are filled (or when
@@ -550,6 +610,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
+        if (a.resident) {
+            grid_dependency_wait();
+            write_resident_images();
+        }
         const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * 32);
         Ring br{0, 0u, a.n_bits}, sr{0, 0u, a.n_sets};
         int pending = -1;
@@ -648,6 +712,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             for (int c = 0; c < 8; ++c) sf[c] = 0x7F7F7F7Fu;
             tmem_st8(lane_taddr + a.col_sf, sf);
         }
+        if (a.resident) write_resident_images();
         int pend_unit[2], pend_c0[2], pend_c1[2], npend = 0;   // cut tiles this block has to finish
         // While a tile is being accumulated these four warps prepare every step's activation operands.  Units of up to
         // 16 token rows (a.convert): they write the step's image themselves, one task per thread (fp4_split_task);
@@ -658,8 +723,9 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // ones whenever their image slot is ready.
         ItemIter si(it);
         bool more_s = si.next();
-        Ring xr{0, 0u, a.n_img};
+        Ring xr{0, 0u, a.n_sf};
         int n_split = 0, seg_end = 0;
+        const int p_first = lo - (int)((unsigned)lo / (unsigned)a.P) * a.P;   // (resident form: the block's first step)
         Unit us{};
         const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
         auto split_next = [&](bool block) -> bool {
@@ -672,8 +738,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 return false;
             }
             if (si.first) us = unit_info(a, si.unit);
-            uint8_t* im = smem + img_off + xr.idx * a.img_bytes;
-            if (a.convert) {
+            uint8_t* im = smem + img_off + (a.resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
+            if (a.convert == 1) {
                 const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
                 for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
                     const int r = task >> 4;

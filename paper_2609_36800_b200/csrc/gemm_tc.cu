@@ -1023,14 +1023,12 @@ cudaError_t read_device_status(unsigned int out[2], cudaStream_t stream) {
     }
     // the other translation units' copies of the status word (all are read, so that all are cleared);
     // a time-out is reported in preference to a range flag
-    unsigned int other[3][2] = {{0, 0}, {0, 0}, {0, 0}};
-    e = read_stream_status(other[0]);
+    unsigned int other[2][2] = {{0, 0}, {0, 0}};
+    e = read_simple_status(other[0]);
     if (e != cudaSuccess) return e;
-    e = read_simple_status(other[1]);
+    e = read_fp4_status(other[1]);
     if (e != cudaSuccess) return e;
-    e = read_fp4_status(other[2]);
-    if (e != cudaSuccess) return e;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 2; ++i) {
         if (other[i][0] != 0 && (out[0] == 0 || (out[0] != kStatusTimeout && other[i][0] == kStatusTimeout))) {
             out[0] = other[i][0];
             out[1] = other[i][1];

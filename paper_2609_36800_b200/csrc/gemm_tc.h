@@ -21,15 +21,13 @@ struct GemmArgs {
     int T;             // work items (< 2^30)
     int q, r;          // T = q * grid + r
     int n_w, n_x, n_x8, n_bits, a_slots, halves;
-    int n_sets;          // streaming decode kernel: operand sets in tensor memory
+    int n_sets;          // 4-bit decode kernel: operand sets in tensor memory
     int cluster;         // ... blocks per cluster (one cluster per unit), or 0: flat work list
-    int decode_warps;    // ... 8, or (experiments, cluster form) 16
-    int early_weights;   // ... 1: its weight loads start before the grid dependency is resolved (0: experiments)
-    int trigger_early;   // ... 1: dependents may launch from this kernel's start (0: see trigger_step)
-    int trigger_step;    // ... dependents may launch once this many of a block's W_base tiles are queued (or all of them)
     int hold_prefetch;   // decode: hold further weight loads until the first sign words have landed
     int fp4;             // 4-bit decode kernel (gemm_fp4.cu) ...
-    int n_img;           // ... ring of activation operand images
+    int n_img;           // ... ring of activation operand images (resident form: one per step of a block)
+    int n_sf;            // ... slots of B-side scale factors in tensor memory
+    int resident;        // ... the block writes the images of all its steps itself, once, before its main loop
     int sets_per_step;   // ... operand sets per 128-k step
     uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
     uint32_t col_sf;     // ... first scale-factor column in tensor memory
@@ -38,8 +36,8 @@ struct GemmArgs {
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
     const float* alpha;
-    const void* X;       // [B*m, K] activations (16-bit values): the streaming decode kernel reads them with plain
-                         // loads; the other kernels use their tensor map
+    const void* X;       // [B*m, K] activations (16-bit values): the 4-bit decode kernel's in-kernel split reads them with
+                         // plain loads; the other kernels use their tensor map
     void* Y;
     unsigned int* counters;
     float* partials;
@@ -55,8 +53,7 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.teams = p.teams; a.Tg = (int)(p.T / p.teams); a.cpt = (p.pair ? p.grid / 2 : p.grid) / p.teams; a.n_tiles = p.n_tiles;
     a.q = a.Tg / a.cpt; a.r = a.Tg % a.cpt;
     a.n_w = p.n_w; a.n_x = p.n_x; a.n_x8 = p.n_x8; a.n_bits = p.n_bits; a.a_slots = p.a_slots; a.hold_prefetch = 1; a.halves = p.halves;
-    a.n_sets = p.n_sets; a.cluster = p.cluster; a.decode_warps = 8;
-    a.early_weights = 1; a.trigger_early = 0; a.trigger_step = 1 << 30;
+    a.n_sets = p.n_sets; a.cluster = p.cluster;
     a.w_stage_bytes = p.w_stage_bytes; a.x_tile_bytes = p.x_tile_bytes; a.w_atom_bytes = p.w_atom_bytes; a.x_atom_bytes = p.x_atom_bytes;
     a.x8_atom_bytes = p.x8_atom_bytes;
     a.bslot_bytes = p.bslot_bytes;
@@ -66,7 +63,7 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.counters = reinterpret_cast<unsigned int*>(workspace);
     char* ws = reinterpret_cast<char*>(workspace);
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
-    a.fp4 = p.fp4; a.n_img = p.n_img; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
+    a.fp4 = p.fp4; a.n_img = p.n_img; a.n_sf = p.n_sf; a.resident = p.resident; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
     a.img = reinterpret_cast<const uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
     return a;
 }
@@ -112,16 +109,8 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream);
 
-// The streaming decode kernel (plan.stream): tensor maps for W_base and the sign words (args.X is read directly).
-cudaError_t launch_gemm_stream(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes, bool early_start,
-                               cudaStream_t stream);
-// Clusters of `cluster` blocks of the streaming kernel the current device can hold at once (0: query failed).
-int stream_max_active_clusters(uint32_t smem_bytes, int cluster);
-// Thread blocks of the streaming kernel one multiprocessor of the current device holds at once (0: query failed).
-int stream_blocks_per_sm(uint32_t smem_bytes);
-// Status word of the streaming kernel's translation unit (read and cleared; the stream must be idle).
-cudaError_t read_stream_status(unsigned int out[2]);
-// ... and of the plain kernels' translation unit (the pre-pass activation split flags out-of-range values there).
+// Status word of the plain kernels' translation unit (read and cleared; the stream must be idle): the pre-pass
+// activation split of the 8-bit decode schedule flags out-of-range values there.
 cudaError_t read_simple_status(unsigned int out[2]);
 
 // Number of CTA pairs (clusters of two) of the pair schedule's kernel that the current device can hold at once

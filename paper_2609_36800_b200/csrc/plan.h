@@ -21,14 +21,7 @@ constexpr int kMaxCtas = 256;        // upper bound on the grid, sizes the works
 constexpr int kDecodeMaxM = 16;      // m <= 16: tenants are grouped into one tile
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kSmemCtrlBytes = 1024; // barriers, TMEM base, flags
-// Streaming decode schedule (few token rows per unit; see gemm_stream.cu)
-constexpr int kStreamSmemBudget = 113 * 1024;   // two thread blocks (of consecutive launches) per multiprocessor
-constexpr int kStreamSetCols = 128;             // one operand set in tensor memory: eight tenants x 64 k of e5m2 signs
-constexpr int kStreamMaxSets = 6;
-// Shared memory behind the control block.  The last tenant's delta window (N3 rows starting at row 4m(TB-1) of
-// the last piece tile) reaches up to round8(4m(TB-1) + N3) rows, i.e. whole 8-row swizzle atoms up to 2 KB past
-// the tile: the control block (1 KB) and this pad are what it reads there (ignored accumulator columns).
-constexpr int kStreamTailPad = 1024;
+constexpr int kFp4MaxSets = 6;      // operand sets of the 4-bit decode kernel in tensor memory, at most
 // 4-bit decode schedule (see gemm_fp4.cu): signs and activation pieces as e2m1, block-scaled MMA with constant scales.
 constexpr int kFp4Pieces = 8;        // radix-4 digits of a 16-bit fixed-point activation magnitude
 constexpr int kFp4MaxM = 8;          // tokens per tenant
@@ -61,17 +54,19 @@ struct Plan {
     int n_x;           // ring of bf16 activation tiles
     int n_x8;          // decode: ring of e5m2 piece tiles
     int n_bits;        // sign-word slots (each holds the signs of one k-pair of one unit)
-    int stream;        // decode with the in-kernel split: 1 = the streaming kernel (half a multiprocessor per block,
-                       // W_base in 64-k atoms, operand sets handed to one MMA issuer), 0 = the older decode kernel
-    int n_sets;        // streaming kernel: operand sets in tensor memory
-    int cluster;       // streaming kernel: > 1 = every unit is taken by a cluster of this many blocks, each with an equal
+    int stream;        // 1 = planned for the 4-bit decode kernel (operand sets handed to issuer warps, clusters or the flat list)
+    int n_sets;        // 4-bit decode kernel: operand sets in tensor memory
+    int cluster;       // 4-bit decode kernel: > 1 = every unit is taken by a cluster of this many blocks, each with an equal
                        // share of the unit's k-steps; their partial results meet in the leader's shared memory
                        // (no workspace traffic, no arrival counters); 0 = the flat work list
     int pair;          // tiled schedule on CTA pairs: a unit is two W_base tiles (256 rows), one per CTA of a cluster of
                        // two; each CTA stages its own weights and half of the activation tile, the pair's leader issues
                        // 256-row MMAs (tcgen05 cta_group::2)
     int fp4;           // 1: the 4-bit decode kernel (gemm_fp4.cu; a pre-pass writes the activation operands)
-    int n_img;         // ... ring of activation operand images in shared memory
+    int n_img;         // ... ring of activation operand images in shared memory (resident form: one image per step of a block)
+    int n_sf;          // ... slots of B-side scale factors in tensor memory (= n_img unless the images are resident)
+    int resident;      // ... 1: cluster form with few steps per block and few token rows: every block writes the images of all
+                       //     its steps into shared memory itself, right after the grid dependency resolves (no pre-pass kernel)
     int sets_per_step; // ... operand sets per 128-k step (2: eight tenants per unit, 1: four)
     uint32_t img_bytes;   // ... one image: 16-bit activation tile (two atoms) + e2m1 piece tile (64 bytes per row)
     uint32_t col_sf;      // ... first scale-factor column in tensor memory (4 for the A side, then the B side's)
@@ -95,14 +90,6 @@ inline bool pair_enabled() {
     return !(e && e[0] == '0');
 }
 
-// The streaming decode kernel (gemm_stream.cu) is taken where it applies when BITDELTA_STREAM=1 is set; the default
-// is the older decode kernel, which measures faster on the decode workloads (18 against 20 us on 8 x 1 x 4096 x 4096).
-// BITDELTA_STREAM=2: also for units of up to 32 token rows (which otherwise take the pre-pass split).
-inline int stream_mode() {
-    const char* e = getenv("BITDELTA_STREAM");
-    return (e && e[0] == '1') ? 1 : (e && e[0] == '2') ? 2 : 0;
-}
-inline bool stream_enabled() { return stream_mode() != 0; }
 // The 4-bit decode kernel (gemm_fp4.cu; m <= 8, plain bf16 calls).  By default it is taken where it measures faster than
 // the 8-bit decode kernels: where its cluster form applies (one tenant group, clusters of 2-8 blocks per W_base tile).
 // BITDELTA_FP4=1: wherever it applies (also the flat work list); BITDELTA_FP4=0: never.
@@ -111,7 +98,7 @@ inline int fp4_mode() {
     return (e && e[0] == '1') ? 1 : (e && e[0] == '0') ? 0 : 2;
 }
 
-// The cluster form of the streaming kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
+// The cluster form of the 4-bit decode kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
 inline bool cluster_enabled() {
     const char* e = getenv("BITDELTA_CLUSTER");
     return !(e && e[0] == '0');
@@ -145,8 +132,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.aslot_cols = ((p.TB + 1) / 2) * 16;
         p.convert = (p.TB * m <= 16) ? 1 : 0;   // 64 converter threads, one 32-k group of one row each
         p.slot_floats = (size_t)kTileN * p.TB * m;
-        p.stream = (stream_mode() != 0 && p.TB * m <= (stream_mode() == 2 ? 32 : 16)) ? 1 : 0;
-        if (p.stream) allow_fp4 = false;   // (the streaming kernel was asked for)
+        p.stream = 0;
         p.fp4 = (allow_fp4 && fp4_mode() != 0 && m <= kFp4MaxM) ? 1 : 0;
         if (p.fp4) {
             // 4-bit operands: eight e2m1 pieces per token stacked along N (tenant j's rows start at 8 m j), written by
@@ -157,13 +143,9 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             p.convert = (p.TB * m <= 16 && getenv("BITDELTA_FP4_INKERNEL") != nullptr) ? 1 : 0;
             p.Nd = kFp4Pieces * m;
             p.N3 = p.Nd;
-            p.x_rows = p.Nb;
+            p.x_rows = round_up(p.TB * m, 8);        // (the base MMA's N = Nb may read past the tile's rows: ignored columns)
             p.x8_rows = p.TB * kFp4Pieces * m;
             p.sets_per_step = (p.TB > 4) ? 2 : 1;
-        } else if (p.stream) {
-            p.convert = 1;                              // the splitter threads read X themselves: no pre-pass
-            p.x_rows = round_up(p.TB * m, 8);           // (the base MMA's N = 16 may read past it: ignored columns)
-            p.x8_rows = round_up(p.TB * kPieces * m, 8);   // (the last tenants' windows run past it: ignored columns)
         }
     } else if (m <= 64 && B > 1 && tb_override != 1) {
         // Tiled schedule, middle regime (16 < m <= 64): a unit holds several tenants, whose tokens share one
@@ -267,7 +249,7 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
     p.x8_atom_bytes = (uint32_t)p.x8_rows * 128;
     p.w_stage_bytes = 2 * p.w_atom_bytes;
     p.x_tile_bytes = 2 * p.x_atom_bytes;
-    p.bslot_bytes = (uint32_t)p.TB * kTileN * ((p.stream && !p.fp4) ? 16 : 32);
+    p.bslot_bytes = (uint32_t)p.TB * kTileN * 32;
     // Shared memory: rings of W_base tiles, of bf16 activation tiles and (decode) of e5m2 piece tiles, and
     // the sign-word slots.  W_base comes from DRAM (latency ~1.5 us under load); it and the bf16
     // activations are released as soon as the base MMAs have read them.  The piece tiles come from L2 (or
@@ -297,25 +279,24 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
         }
         if (p.n_w > 4) p.n_w = 4;
+        p.n_sf = p.n_img;
+        p.resident = 0;
+        if (p.cluster > 1 && p.TB * m <= 16 && p.convert == 0 && getenv("BITDELTA_FP4_RESIDENT") != nullptr) {
+            // (experiments) Resident images: all the steps of a block ((P + cluster - 1) / cluster of them) if that leaves three
+            // W_base stages.  Measured slower than the pre-pass (22.6 vs 18.0 us on 8 x 1 x 4096 x 4096): every block repeats
+            // the split of its k range, ~250 instructions per eight values, before its main loop can start.
+            const int steps = (p.P + p.cluster - 1) / p.cluster;
+            const int nw = (kSmemBudget - fixed - steps * (int)p.img_bytes) / (int)p.w_stage_bytes;
+            if (nw >= 3) {
+                p.resident = 1;
+                p.convert = 2;
+                p.n_img = steps;
+                p.n_sf = 3;
+                p.n_w = nw > 4 ? 4 : nw;
+            }
+        }
         p.n_x = p.n_img;
         p.n_x8 = p.n_img;
-    } else if (p.stream) {
-        // Half a multiprocessor: two sign-word slots (128 k each), two activation and two piece tiles, and
-        // every remaining byte for W_base atoms (64 k, 16 KB each).
-        // Half a multiprocessor: two slots of {activation tile, piece tile} (filled together by the splitter
-        // threads), two W_base stages of one 128-k tile each, two or three sign-word slots.  (A whole
-        // multiprocessor per block with rings a step deeper and sixteen decode warps was measured on the cluster
-        // form: no faster per step, and the next launch's blocks then start their loads a microsecond later.)
-        p.n_x = 2;
-        p.n_x8 = 2;
-        p.n_w = 2;
-        const int fixed = 1024 + kSmemCtrlBytes + kStreamTailPad + p.n_w * (int)p.w_stage_bytes +
-                          p.n_x * (int)p.x_tile_bytes + p.n_x8 * (int)p.x8_atom_bytes;
-        p.n_bits = (kStreamSmemBudget - fixed) / (int)p.bslot_bytes;
-        if (p.n_bits < 2) p.n_bits = (kSmemBudget - fixed) / (int)p.bslot_bytes;   // (a whole multiprocessor per block then)
-        if (p.n_bits > 3) p.n_bits = 3;
-        if (p.n_bits < 2) return p;
-        if (p.n_w > kMaxStages) p.n_w = kMaxStages;
     } else if (p.decode) {
         p.n_x8 = 3;
         p.n_x = (p.x_tile_bytes <= 4 * 1024) ? 3 : 2;
@@ -346,9 +327,6 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
                    p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
     if (p.fp4) {
         p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_img * p.img_bytes + p.n_bits * p.bslot_bytes + kSmemCtrlBytes;
-    } else if (p.stream) {
-        p.smem_bytes = 1024 + p.n_w * p.w_stage_bytes + p.n_x * p.x_tile_bytes + p.n_x8 * p.x8_atom_bytes +
-                       p.n_bits * p.bslot_bytes + kSmemCtrlBytes + kStreamTailPad;
     } else if (p.smem_bytes < 120 * 1024) {
         // One CTA per SM is assumed by this kernel's TMEM allocation: keep the request above half an SM.
         p.smem_bytes = 120 * 1024;
@@ -373,16 +351,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         // [base | delta accumulators | scale factors: 4 columns for the A side, 4 per tenant and image slot for the B side |
         //  operand sets of 64 columns]
         p.col_sf = p.col_a;
-        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_img, 32);
+        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_sf, 32);
         p.halves = 2;
         p.n_sets = (kTmemCols - (int)p.col_a) / kFp4SetCols;
-        if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
-        if (p.n_sets < 2) return p;
-        p.a_slots = 2;
-    } else if (p.stream) {
-        p.halves = 2;
-        p.n_sets = free_cols / kStreamSetCols;
-        if (p.n_sets > kStreamMaxSets) p.n_sets = kStreamMaxSets;
+        if (p.n_sets > kFp4MaxSets) p.n_sets = kFp4MaxSets;
         if (p.n_sets < 2) return p;
         p.a_slots = 2;
     }

@@ -39,6 +39,12 @@ def errors(Y, Yref):
 
 def assert_parity(Y, Yref, what=""):
     max_abs, rel_fro = errors(Y, Yref)
-    assert max_abs <= MAX_ABS_TOL and rel_fro <= REL_FRO_TOL, \
-        f"{what}: max_abs={max_abs:.3e} (tol {MAX_ABS_TOL}), rel_fro={rel_fro:.3e} (tol {REL_FRO_TOL})"
+    if not (max_abs <= MAX_ABS_TOL and rel_fro <= REL_FRO_TOL):
+        # where the outputs beyond the gate sit ([B, m, N]: tenant, token, weight row): points at the tile / role at fault
+        d = np.argwhere(np.abs(Y - Yref) > MAX_ABS_TOL)
+        where = ""
+        if len(d):
+            where = (f"; {len(d)} outputs off: tenants {sorted(set(d[:, 0].tolist()))[:8]}, tokens {sorted(set(d[:, 1].tolist()))[:8]}, "
+                     f"128-row tiles {sorted(set((d[:, 2] // 128).tolist()))[:12]}, rows in tile {sorted(set((d[:, 2] % 128).tolist()))[:12]}")
+        raise AssertionError(f"{what}: max_abs={max_abs:.3e} (tol {MAX_ABS_TOL}), rel_fro={rel_fro:.3e} (tol {REL_FRO_TOL}){where}")
     return max_abs, rel_fro

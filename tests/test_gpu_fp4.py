@@ -49,6 +49,21 @@ def test_fp4_kernel_matches_oracle(shape, schedule, inkernel, monkeypatch):
     assert rel_fro > 1e-5 or max_abs == 0.0   # (a bf16 result cannot sit closer to the fp64 one: guards against comparing a thing with itself)
 
 
+@pytest.mark.parametrize("shape", [(8, 1, 1024, 1024), (3, 2, 384, 640), (1, 1, 2048, 1024), (8, 1, 4096, 4096)], ids=str)
+def test_fp4_kernel_resident_images_variant(shape, monkeypatch):
+    # BITDELTA_FP4_RESIDENT=1: every block writes the images of all its steps into shared memory itself (no pre-pass kernel)
+    monkeypatch.setenv("BITDELTA_FP4_RESIDENT", "1")
+    B, m, N, K = shape
+    g = bd.gemm_plan(B, m, N, K)
+    assert g["schedule"] == 8 and g["piece_ring"] == -(-g["k_steps"] // (g["blocks"] // g["units"]))   # one image per step of a block
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B + m + N + K)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    n0 = bd.kernel_launch_count()
+    Y = run_gemm(X, W, bits, alpha)
+    assert bd.kernel_launch_count() - n0 == 1
+    assert_parity(Y, oracle.gemm(X, W, bits, alpha), str(shape))
+
+
 def test_fp4_kernel_one_hot_probe_is_exact():
     # X = e_k per token, W = 0, alpha = 1  =>  Y[b,t,n] = s[b,n,k_t]: exact in bf16; pins bit, word, digit and tenant order
     B, m, N, K = 8, 2, 256, 1024

@@ -107,20 +107,6 @@ def test_four_bit_decode_kernel_plans(monkeypatch):
     assert bd.gemm_workspace_bytes(8, 1, 4096, 4096) >= 32 * 9 * 1024
 
 
-def test_streaming_decode_kernel_plans(monkeypatch):
-    # BITDELTA_STREAM=1 (read at every plan): few token rows per unit and one tenant group -> clusters of four
-    # blocks per W_base tile; two tenant groups -> the flat list by teams, within half a multiprocessor
-    monkeypatch.setenv("BITDELTA_STREAM", "1")
-    one = bd.gemm_plan(8, 1, 4096, 4096)
-    assert one["schedule"] == 6 and one["order"] == 3 and one["blocks"] == 128 and one["smem_bytes"] <= 113 * 1024
-    assert bd.gemm_plan(1, 16, 512, 512)["schedule"] == 6
-    two = bd.gemm_plan(16, 1, 4096, 4096)
-    assert two["schedule"] == 5 and two["order"] == 2 and two["smem_bytes"] <= 113 * 1024
-    for b in range(one["blocks"]):
-        lo, hi = bd.gemm_plan_cta_items(8, 1, 4096, 4096, b)
-        assert hi - lo == 8 and lo // 32 == b // 4 and bd.gemm_plan_item_cta(8, 1, 4096, 4096, lo) == b
-
-
 def test_cuda_core_path_and_bad_arguments():
     assert bd.gemm_plan(2, 3, 96, 96)["schedule"] == 3
     lib = bd.load_library()
