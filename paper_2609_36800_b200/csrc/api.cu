@@ -391,9 +391,9 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
         // the token rows' fixed-point units; then the GEMM, which prefetches weights while this is still running.
         uint8_t* img = bd::ws_x8(p, workspace);
         // (its early start is always safe: it waits for its predecessor before it touches anything)
-        if (!p.convert && bd::launch_x_split_fp4(X, img, p, early_start_enabled(), stream) != cudaSuccess)
+        if (!p.convert && !p.coop && bd::launch_x_split_fp4(X, img, p, early_start_enabled(), stream) != cudaSuccess)
             return BITDELTA_ERR_CUDA;
-        if (!p.convert) g_launches++;
+        if (!p.convert && !p.coop) g_launches++;
         tmX8 = tmW;   // not read
     } else if (p.decode && !p.convert) {
         // Decode schedule with many token rows per tile: split the activations into e5m2 pieces first

@@ -55,7 +55,10 @@ __device__ long long* g_fp4_trace = nullptr;
 #define FT_DECL(n) long long ft_acc[n] = {}; long long ft_t0 = clock64()
 #define FT_ADD(i) do { const long long ft_t1 = clock64(); ft_acc[i] += ft_t1 - ft_t0; ft_t0 = ft_t1; } while (0)
 #define FT_OUT(base, n) do { if (g_fp4_trace && lane == 0) for (int ft_i = 0; ft_i < (n); ++ft_i) g_fp4_trace[(size_t)blockIdx.x * 32 + (base) + ft_i] = ft_acc[ft_i]; } while (0)
+// ... and 16 timestamps (ns, %globaltimer) per block in a second buffer half: [16 .. 31] of the block's second row
+#define FT_STAMP(i) do { if (g_fp4_trace && lane == 0) g_fp4_trace[(size_t)(256 + blockIdx.x) * 32 + (i)] = (long long)global_timer_ns(); } while (0)
 #else
+#define FT_STAMP(i) do { } while (0)
 #define FT_DECL(n) do { } while (0)
 #define FT_ADD(i) do { } while (0)
 #define FT_OUT(base, n) do { } while (0)
@@ -77,6 +80,8 @@ struct FCtl {
     uint32_t abort_flag;
     uint32_t is_last;
     uint64_t imgready[4];           // a step's image is in shared memory and its scale factors in tensor memory (4 epilogue warps)
+    uint64_t cntready;              // cooperative image pass: this block has counted itself; img_target is set
+    uint32_t img_target;            // ... value of the launch-wide counter at which every block's share is written
 };
 static_assert(sizeof(FCtl) <= kSmemCtrlBytes, "control block too large");
 
@@ -285,6 +290,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<true, false, false>(aa, un, am, 0); };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (warp == 0) FT_STAMP(0);   // block start
     if (threadIdx.x == 32) {
         prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmBits);
@@ -345,6 +351,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         mbar_init(smem_u32(&ctl->accempty), kFEpiWarps);
         mbar_init(smem_u32(&ctl->depready), 1);
         mbar_init(smem_u32(&ctl->tmemready), 1);
+        mbar_init(smem_u32(&ctl->cntready), 1);
         ctl->abort_flag = 0;
         ctl->is_last = 0;
         fence_barrier_init();
@@ -438,6 +445,25 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             if (!dep_done) {
                 // the weight rings are full and stay full until the grid dependency resolves: sleep until then
                 dep_done = warp_all(mbar_try_wait_hint(smem_u32(&ctl->depready), 0u, 20000u));
+                if (dep_done && a.coop) {
+                    // Cooperative image pass: every block of the launch writes its share of the activation images to
+                    // the workspace and counts itself; the images may be fetched once all have (all blocks of a
+                    // cluster-form launch are resident together, one per multiprocessor).  Bounded like every wait.
+                    bool ok = warp_all(wait_bar(smem_u32(&ctl->cntready), 0u, abort_flag, 23));
+                    const unsigned int target = ctl->img_target;
+                    const long long t0 = clock64();
+                    while (ok && (int)(ld_acquire_gpu_u32(a.img_counter) - target) < 0) {
+                        if (*abort_flag) ok = false;
+                        if (clock64() - t0 > kWaitLimitCycles) {
+                            *abort_flag = 1;
+                            if (atomicCAS(&g_device_status[0], 0u, kStatusTimeout) == 0u) g_device_status[1] = 24u;
+                            ok = false;
+                        }
+                    }
+                    FT_STAMP(14);   // every block's share is written
+                    fence_proxy_async_all();   // the other blocks' generic-proxy stores -> this warp's bulk copies
+                    if (!ok) break;
+                }
                 continue;
             }
             if (more_x) (void)mbar_try_wait_hint(smem_u32(&ctl->pempty[xr.idx]), xr.par ^ 1, 64u);
@@ -454,10 +480,12 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             }
         }
         // All of this block's loads are queued: a kernel queued behind this one with an early start may become resident.
+        FT_STAMP(2);   // all loads queued
         if (lane == 0) grid_launch_dependents();
     } else if (warp == kFWarpMma) {
         // -------------------------------------------------------------- MMA issuer
         grid_dependency_wait();
+        FT_STAMP(1);   // dependency resolved
         named_bar_arrive(kFBarDep, kFThreads - 32);   // wakes the decode and epilogue warps
         if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));   // ... and the producer
         tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -492,11 +520,14 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 FT_ADD(0);
                 ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
+                if (p == p0) FT_STAMP(3);   // first image ready (base issuer)
                 if (!ok) break;
                 const uint32_t img_s = img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes;
                 const uint64_t xdesc = desc128 + (img_s >> 4);
                 ok = warp_all(wait_bar(smem_u32(&ctl->wfull[wr.idx]), wr.par, abort_flag, 4));
                 FT_ADD(3);
+                if (p == p0) FT_STAMP(4);   // first W_base tile landed
+                if (p == p1 - 1) FT_STAMP(5);   // last W_base tile landed
                 if (!ok) break;
                 {
                     const uint64_t wdesc = desc128 + ((w_addr + wr.idx * a.w_stage_bytes) >> 4);
@@ -713,6 +744,30 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             tmem_st8(lane_taddr + a.col_sf, sf);
         }
         if (a.resident) write_resident_images();
+        if (warp == kFWarpEpi0) FT_STAMP(11);   // epilogue warps awake, tensor memory ready
+        if (a.coop) {
+            // This block's share of the launch's activation images (one tenant group): task = (step, token row, chunk).
+            const Unit u0 = unit_info(a, 0);
+            const uint32_t sf_off0 = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
+            const int per_step = u0.ntok * 16;
+            for (int task = (int)blockIdx.x * (kFEpiWarps * 32) + etid; task < a.P * per_step; task += (int)gridDim.x * (kFEpiWarps * 32)) {
+                const int p = (int)((unsigned)task / (unsigned)per_step);
+                const int rem = task - p * per_step;
+                const int r = rem >> 4;
+                const int j = r / am, t = r - j * am;
+                fp4_split_task(reinterpret_cast<const uint16_t*>(a.X) + (size_t)(u0.xrow0 + r) * a.K + (size_t)p * kPairK,
+                               a.img + (size_t)p * a.img_bytes, rem & 15, r, j, t, am, a.x_atom_bytes, a.x_tile_bytes, sf_off0);
+            }
+            if (warp == kFWarpEpi0) FT_STAMP(12);   // this block's share written
+            __threadfence();
+            epi_bar_sync(kFEpiWarps * 32);
+            if (etid == 0) {
+                const unsigned int old = atomicAdd(a.img_counter, 1u);
+                ctl->img_target = (old / gridDim.x + 1u) * gridDim.x;   // (the launches of a stream take their turns: whole rounds)
+                mbar_arrive(smem_u32(&ctl->cntready));
+            }
+            if (warp == kFWarpEpi0) FT_STAMP(13);   // counted
+        }
         int pend_unit[2], pend_c0[2], pend_c1[2], npend = 0;   // cut tiles this block has to finish
         // While a tile is being accumulated these four warps prepare every step's activation operands.  Units of up to
         // 16 token rows (a.convert): they write the step's image themselves, one task per thread (fp4_split_task);
@@ -796,6 +851,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             FT_ADD(0);
             ok = wait_bar(smem_u32(&ctl->accfull), accphase, abort_flag, 8);
             FT_ADD(1);
+            if (warp == kFWarpEpi0) FT_STAMP(6);   // accumulators complete
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
@@ -863,6 +919,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
 
     // ------------------------------------------------------------------ teardown
     __syncthreads();
+    if (warp == 0) FT_STAMP(7);   // all roles done
     if (*abort_flag) {
         // A wait was abandoned: give copies and MMAs still in flight a bounded time to land before shared
         // and tensor memory are released.
@@ -880,6 +937,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // partial sums in block order, i.e. in k order, through the distributed shared memory window and write Y; a
         // second barrier keeps the other blocks' shared memory alive until it has read them.
         cluster_sync_all();
+        if (warp == 0) FT_STAMP(8);   // cluster barrier passed
         if (crank == 0 && warp >= kFWarpEpi0 && lo < hi && !*abort_flag) {
             const Unit u = unit_info(a, (int)blockIdx.x / a.cluster);
             const int row = (warp & 3) * 32 + lane;
@@ -907,8 +965,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 }
             }
         }
+        if (warp == kFWarpEpi0) FT_STAMP(9);   // leader's sum stored
         cluster_sync_relaxed();
     }
+    if (warp == 0) FT_STAMP(10);   // exit
 }
 
 #ifdef BD_TRACE

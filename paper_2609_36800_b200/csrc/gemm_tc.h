@@ -28,10 +28,12 @@ struct GemmArgs {
     int n_img;           // ... ring of activation operand images (resident form: one per step of a block)
     int n_sf;            // ... slots of B-side scale factors in tensor memory
     int resident;        // ... the block writes the images of all its steps itself, once, before its main loop
+    int coop;            // ... the launch's blocks write the images together into the workspace (no pre-pass kernel)
+    unsigned int* img_counter;   // ... and count themselves here when their share is written
     int sets_per_step;   // ... operand sets per 128-k step
     uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
     uint32_t col_sf;     // ... first scale-factor column in tensor memory
-    const uint8_t* img;  // ... images written by the pre-pass: [group][step][img_bytes]
+    uint8_t* img;        // ... images written by the pre-pass (or by the launch itself, coop): [group][step][img_bytes]
     uint32_t w_stage_bytes, x_tile_bytes, w_atom_bytes, x_atom_bytes, x8_atom_bytes, bslot_bytes;
     uint32_t col_delta, col_a;
     uint32_t slot_floats;
@@ -63,8 +65,9 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     a.counters = reinterpret_cast<unsigned int*>(workspace);
     char* ws = reinterpret_cast<char*>(workspace);
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
-    a.fp4 = p.fp4; a.n_img = p.n_img; a.n_sf = p.n_sf; a.resident = p.resident; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
-    a.img = reinterpret_cast<const uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
+    a.fp4 = p.fp4; a.n_img = p.n_img; a.n_sf = p.n_sf; a.resident = p.resident; a.coop = p.coop;
+    a.img_counter = reinterpret_cast<unsigned int*>(ws + p.ws_header_bytes) - 1; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
+    a.img = reinterpret_cast<uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
     return a;
 }
 

@@ -65,6 +65,8 @@ struct Plan {
     int fp4;           // 1: the 4-bit decode kernel (gemm_fp4.cu; a pre-pass writes the activation operands)
     int n_img;         // ... ring of activation operand images in shared memory (resident form: one image per step of a block)
     int n_sf;          // ... slots of B-side scale factors in tensor memory (= n_img unless the images are resident)
+    int coop;          // ... 1: cluster form: the launch's blocks write the activation images together, each a share of them, into
+                       //     the workspace before their main loops (no pre-pass kernel); 0: a pre-pass kernel writes them
     int resident;      // ... 1: cluster form with few steps per block and few token rows: every block writes the images of all
                        //     its steps into shared memory itself, right after the grid dependency resolves (no pre-pass kernel)
     int sets_per_step; // ... operand sets per 128-k step (2: eight tenants per unit, 1: four)
@@ -295,6 +297,11 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
                 p.n_w = nw > 4 ? 4 : nw;
             }
         }
+        // (experiments, BITDELTA_FP4_COOP=1) Cluster form, every block of the launch resident at once: the blocks write the
+        // images together, each a share, and count themselves in the workspace; no pre-pass kernel.  Measured slower than
+        // the pre-pass (20.5 vs 18.3 us on 8 x 1 x 4096 x 4096): shares written 1.7 us after the grid dependency resolves,
+        // but fence + count + the slowest block + the fetch add up to 9.5 us before the first MMA (pre-pass chain: 9.3).
+        p.coop = (p.cluster > 1 && !p.resident && p.convert == 0 && getenv("BITDELTA_FP4_COOP") != nullptr) ? 1 : 0;
         p.n_x = p.n_img;
         p.n_x8 = p.n_img;
     } else if (p.decode) {
@@ -362,7 +369,8 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
 
     // Workspace: arrival counters, two partial-result slots per CTA, then (decode) the e5m2
     // pieces of X written by the activation-split kernel.
-    p.ws_header_bytes = (size_t)round_up(p.n_tiles * p.groups * 4, 1024);   // one arrival counter per W_base tile and group
+    p.ws_header_bytes = (size_t)round_up((p.n_tiles * p.groups + 1) * 4, 1024);   // one arrival counter per W_base tile and group,
+                                                                                  // and (last word) the activation-image counter of the 4-bit kernel
     // (sized for the largest grid any device could get, so that the size does not depend on the device;
     // never more CTAs than items)
     const long long items = p.pair ? 2 * p.T : p.T;

@@ -202,6 +202,15 @@ __device__ __forceinline__ void umma_ts_mxf4(uint32_t d_tmem, uint32_t a_tmem, u
         : "memory");
 }
 
+// Generic-proxy writes (of any thread, made visible to this one by an acquire) -> visible to this thread's later
+// async-proxy reads (bulk copies).
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ unsigned int ld_acquire_gpu_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // Plain bulk copy global -> shared (sizes and addresses multiples of 16 bytes), completion counted on an mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -64,6 +64,28 @@ def test_fp4_kernel_resident_images_variant(shape, monkeypatch):
     assert_parity(Y, oracle.gemm(X, W, bits, alpha), str(shape))
 
 
+@pytest.mark.parametrize("shape", [(8, 1, 1024, 1024), (3, 2, 384, 640), (4, 8, 512, 1024), (8, 1, 4096, 4096)], ids=str)
+def test_fp4_kernel_cooperative_image_pass_variant(shape, monkeypatch):
+    # BITDELTA_FP4_COOP=1: the launch's blocks write the activation images together into the workspace (no pre-pass kernel);
+    # called three times on one workspace: the launch-wide counter advances by whole rounds
+    monkeypatch.setenv("BITDELTA_FP4_COOP", "1")
+    B, m, N, K = shape
+    assert bd.gemm_plan(B, m, N, K)["schedule"] == 8
+    wl = synth.Workload("t", B=B, m=m, K=K, N=N, seed=B + m + N + K)
+    X, W, bits, alpha = synth.make_inputs(wl)
+    ref = oracle.gemm(X, W, bits, alpha)
+    dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
+    ws = bd.make_workspace(B, m, N, K)
+    n0 = bd.kernel_launch_count()
+    outs = [bd.gemm(dX, dW, dbits, dalpha, workspace=ws) for _ in range(3)]
+    torch.cuda.synchronize()
+    assert bd.kernel_launch_count() - n0 == 3
+    st, site = bd.last_device_status()
+    assert st == 0, (st, site)
+    for Y in outs:
+        assert_parity(y_to_f64(Y), ref, str(shape))
+
+
 def test_fp4_kernel_one_hot_probe_is_exact():
     # X = e_k per token, W = 0, alpha = 1  =>  Y[b,t,n] = s[b,n,k_t]: exact in bf16; pins bit, word, digit and tenant order
     B, m, N, K = 8, 2, 256, 1024
