@@ -53,7 +53,11 @@ constexpr int kFBarImg = 14;                     // resident form: all warps but
 // Trace build: per block 32 accumulators (cycles) written at the end of each role; see bitdelta_debug_set_trace_fp4.
 __device__ long long* g_fp4_trace = nullptr;
 #define FT_DECL(n) long long ft_acc[n] = {}; long long ft_t0 = clock64()
+#ifdef BD_TRACE_TIMELINE_ONLY   /* (the accumulators' clock reads cost time themselves: leave only the timeline stamps) */
+#define FT_ADD(i) do { } while (0)
+#else
 #define FT_ADD(i) do { const long long ft_t1 = clock64(); ft_acc[i] += ft_t1 - ft_t0; ft_t0 = ft_t1; } while (0)
+#endif
 #define FT_OUT(base, n) do { if (g_fp4_trace && lane == 0) for (int ft_i = 0; ft_i < (n); ++ft_i) g_fp4_trace[(size_t)blockIdx.x * 32 + (base) + ft_i] = ft_acc[ft_i]; } while (0)
 // ... and 16 timestamps (ns, %globaltimer) per block in a second buffer half: [16 .. 31] of the block's second row
 #define FT_STAMP(i) do { if (g_fp4_trace && lane == 0) g_fp4_trace[(size_t)(256 + blockIdx.x) * 32 + (i)] = (long long)global_timer_ns(); } while (0)
