@@ -363,7 +363,7 @@ def time_e2e(wl, host_inputs, steps):
     return ms, h2d, d2h
 
 
-def cpu_baseline(wl, host_inputs, budget_s=15.0):
+def cpu_baseline(wl, host_inputs, cpu_seconds=15.0):
     """The fp64 oracle, as it stands, on the host cores over a bounded sample of the workload."""
     import oracle
     X, W, bits, alpha = host_inputs
@@ -380,7 +380,7 @@ def cpu_baseline(wl, host_inputs, budget_s=15.0):
 
     probe = min(total, 2048)
     rate = probe / max(sample(probe), 1e-9)          # outputs per second
-    wall_target = budget_s / max(cores, 1) * 1.5     # ~budget_s CPU-seconds of work
+    wall_target = cpu_seconds / max(cores, 1) * 1.5     # ~cpu_seconds CPU-seconds of work
     count = int(min(total, max(probe, rate * wall_target)))
     reps = max(1, int(round(wall_target * rate / count)))
     dt = sum(sample(count) for _ in range(reps))
