@@ -150,9 +150,16 @@ __device__ __forceinline__ void fp4_task_load(const uint16_t* __restrict__ xstep
 #pragma unroll
     for (int i = 0; i < 8; ++i) d.hv[i] = __ldg(xstep + 32 * wd + 4 * i + c);
 }
+__device__ __forceinline__ void fp4_task_digits(const Fp4TaskData& d, uint8_t* im, int tk, int r_local, int j, int t, int m,
+                                                uint32_t x_tile_bytes, uint32_t sf_off);
 __device__ __forceinline__ void fp4_task_finish(const Fp4TaskData& d, uint8_t* im, int tk, int r_local, int j, int t, int m,
                                                 uint32_t x_atom_bytes, uint32_t x_tile_bytes, uint32_t sf_off) {
     *reinterpret_cast<uint4*>(im + (tk >> 3) * x_atom_bytes + r_local * 128 + (((tk & 7) ^ (r_local & 7)) * 16)) = d.chunk;
+    fp4_task_digits(d, im, tk, r_local, j, t, m, x_tile_bytes, sf_off);
+}
+// ... its second half: the digit rows and the scale table entry from the eight values d.hv
+__device__ __forceinline__ void fp4_task_digits(const Fp4TaskData& d, uint8_t* im, int tk, int r_local, int j, int t, int m,
+                                                uint32_t x_tile_bytes, uint32_t sf_off) {
     const int wd = tk >> 2, c = tk & 3;
     uint32_t R[8];
     uint32_t mx = 0;
@@ -372,16 +379,18 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int tid = (int)threadIdx.x - 32;
         const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
         const int per_step = u.ntok * 16;
-        // (three tasks per thread requested together: the whole split costs one round trip to X per 1440 tasks)
+        // Phase A: the 16-bit tiles, one 16-byte chunk per task (three tasks per thread requested together: one round
+        // trip to X).  Phase B: the digit rows, from the tiles in shared memory (eight 2-byte shared loads per task instead of
+        // eight global ones).
         for (int task0 = tid; task0 < nsteps * per_step; task0 += 3 * (kFThreads - 32)) {
-            Fp4TaskData d[3];
+            uint4 ch[3];
 #pragma unroll
             for (int q = 0; q < 3; ++q) {
                 const int task = task0 + q * (kFThreads - 32);
                 if (task < nsteps * per_step) {
                     const int st = (int)((unsigned)task / (unsigned)per_step);
                     const int rem = task - st * per_step;
-                    fp4_task_load(reinterpret_cast<const uint16_t*>(a.X) + (size_t)(u.xrow0 + (rem >> 4)) * a.K + (size_t)(q0 + st) * kPairK, rem & 15, d[q]);
+                    ch[q] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(a.X) + (size_t)(u.xrow0 + (rem >> 4)) * a.K + (size_t)(q0 + st) * kPairK) + (rem & 15));
                 }
             }
 #pragma unroll
@@ -390,11 +399,27 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (task < nsteps * per_step) {
                     const int st = (int)((unsigned)task / (unsigned)per_step);
                     const int rem = task - st * per_step;
-                    const int r = rem >> 4;
-                    const int j = r / am, t = r - j * am;
-                    fp4_task_finish(d[q], smem + img_off + st * a.img_bytes, rem & 15, r, j, t, am, a.x_atom_bytes, a.x_tile_bytes, sf_off);
+                    const int r = rem >> 4, tk = rem & 15;
+                    *reinterpret_cast<uint4*>(smem + img_off + st * a.img_bytes + (tk >> 3) * a.x_atom_bytes + r * 128 + (((tk & 7) ^ (r & 7)) * 16)) = ch[q];
                 }
             }
+        }
+        named_bar_sync(kFBarImg, kFThreads - 32);
+        for (int task = tid; task < nsteps * per_step; task += kFThreads - 32) {
+            const int st = (int)((unsigned)task / (unsigned)per_step);
+            const int rem = task - st * per_step;
+            const int r = rem >> 4, tk = rem & 15;
+            const int j = r / am, t = r - j * am;
+            uint8_t* im = smem + img_off + st * a.img_bytes;
+            const int wd = tk >> 2, c = tk & 3;
+            Fp4TaskData d;
+            d.chunk = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int kk = 32 * wd + 4 * i + c;   // value k of the step: atom kk / 64, chunk (kk % 64) / 8, element kk % 8
+                d.hv[i] = *reinterpret_cast<const uint16_t*>(im + (kk >> 6) * a.x_atom_bytes + r * 128 + ((((kk & 63) >> 3) ^ (r & 7)) * 16) + (kk & 7) * 2);
+            }
+            fp4_task_digits(d, im, tk, r, j, t, am, a.x_tile_bytes, sf_off);
         }
         fence_proxy_async_smem();   // generic-proxy writes -> visible to the MMAs' async-proxy reads
         named_bar_sync(kFBarImg, kFThreads - 32);

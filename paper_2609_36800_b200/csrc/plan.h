@@ -285,8 +285,9 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         p.resident = 0;
         if (p.cluster > 1 && p.TB * m <= 16 && p.convert == 0 && getenv("BITDELTA_FP4_RESIDENT") != nullptr) {
             // (experiments) Resident images: all the steps of a block ((P + cluster - 1) / cluster of them) if that leaves three
-            // W_base stages.  Measured slower than the pre-pass (22.6 vs 18.0 us on 8 x 1 x 4096 x 4096): every block repeats
-            // the split of its k range, ~250 instructions per eight values, before its main loop can start.
+            // W_base stages.  Measured slower than the pre-pass (20.6 vs 17.7 us on 8 x 1 x 4096 x 4096, no faster with the inputs
+            // resident in L2): every block repeats the split of its k range, ~250 integer instructions per eight values,
+            // before its main loop can start.
             const int steps = (p.P + p.cluster - 1) / p.cluster;
             const int nw = (kSmemBudget - fixed - steps * (int)p.img_bytes) / (int)p.w_stage_bytes;
             if (nw >= 3) {
