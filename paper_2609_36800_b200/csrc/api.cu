@@ -382,7 +382,7 @@ int bitdelta_gemm_ex(const void* X, const void* W_base, const uint32_t* bits, co
     if (!p.stream && !cached_map(&tmX, MapKey{0, X, (uint64_t)B * m, (uint64_t)K, 0, (uint32_t)p.x_rows, 0u},
                                  [&](CUtensorMap* mp) { return encode_bf16_tile(mp, X, (uint64_t)B * m, (uint64_t)K, (uint32_t)p.x_rows); }))
         return BITDELTA_ERR_CUDA;
-    const uint32_t box_words = 8u;
+    const uint32_t box_words = (p.fp4 && p.bits_row == 16) ? 4u : 8u;
     if (!cached_map(&tmBits, MapKey{1, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words},
                     [&](CUtensorMap* mp) { return encode_bits_3d(mp, bits, (uint64_t)B, (uint64_t)N, (uint64_t)(K / 32), (uint32_t)p.TB, box_words); }))
         return BITDELTA_ERR_CUDA;

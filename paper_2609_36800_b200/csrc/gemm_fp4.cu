@@ -293,6 +293,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     const uint32_t bits_off = a.n_w * a.w_stage_bytes;                     // sign-word slots (two steps each)
     const uint32_t bits_addr = base + bits_off;
     const uint32_t img_off = bits_off + a.n_bits * a.bslot_bytes;          // ring of activation images
+    const int n_ring = a.resident ? a.n_sf : a.n_img;                      // ... its slots (resident images: the scale-factor slots)
     const uint32_t img_addr = base + img_off;
     FCtl* ctl = reinterpret_cast<FCtl*>(smem + img_off + a.n_img * a.img_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
@@ -333,7 +334,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     auto issue_bits = [&](const Unit& u, int p, int bslot) {
         const uint32_t bar = smem_u32(&ctl->bfull[bslot]);
         mbar_arrive_expect_tx(bar, a.bslot_bytes);
-        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, (p >> 1) * 8, u.n0, u.tenant0);
+        tma_load_3d(bits_addr + bslot * a.bslot_bytes, &tmBits, bar, a.bits_row == 32 ? (p >> 1) * 8 : p * 4, u.n0, u.tenant0);
     };
     // The activation image of a step (written by the pre-pass kernel): one plain bulk copy.  One thread.
     auto issue_img = [&](const Unit& u, int p, int slot) {
@@ -431,7 +432,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // another kernel: queued before the grid dependency is resolved, as far as their rings allow) and activation
         // images (written by the pre-pass kernel queued before this one: only afterwards).
         ItemIter wi(it), bi(it), xi(it);
-        Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, a.n_sf};
+        Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, n_ring};
         Unit uw{}, ub{}, ux{};
         bool more_w = wi.next(), more_b = bi.next(), more_x = !a.convert && xi.next();   // (convert: the epilogue warps write the images)
         if (more_w) { uw = unit_info(a, wi.unit); ub = uw; ux = uw; }
@@ -445,7 +446,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 __syncwarp();
                 br.step();
                 // the slot also covers the next step if that is the odd step of the same pair and of the same segment
-                const bool odd_next = ((bi.p & 1) == 0) && (bi.p + 1 < bi.p1);
+                const bool odd_next = a.bits_row == 32 && ((bi.p & 1) == 0) && (bi.p + 1 < bi.p1);
                 more_b = bi.next();
                 if (more_b && odd_next) more_b = bi.next();
                 if (more_b && bi.first) ub = unit_info(a, bi.unit);
@@ -534,7 +535,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint32_t idesc_base = make_idesc_bf16(kTileN, (uint32_t)a.Nb);
         const uint64_t desc128 = make_smem_desc_sw128(0);
         const uint32_t x_atom16 = a.x_atom_bytes >> 4;
-        Ring wr{0, 0u, a.n_w}, pr{0, 0u, a.n_sf};
+        Ring wr{0, 0u, a.n_w}, pr{0, 0u, n_ring};
         uint32_t accphase = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
@@ -603,7 +604,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint64_t desc64 = make_smem_desc_sw64(0);
         const uint32_t ten_rows16 = (uint32_t)a.Nd * 4u;      // a tenant's digit rows x 64 B >> 4
         const uint32_t sfa = tmem_base + a.col_sf;
-        Ring pr{0, 0u, a.n_sf}, sr{0, 0u, a.n_sets};
+        Ring pr{0, 0u, n_ring}, fr{0, 0u, a.n_sf}, sr{0, 0u, a.n_sets};
         uint32_t accphase = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
@@ -620,7 +621,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 FT_ADD(2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t sfb0 = sfa + 4u + (uint32_t)(pr.idx * 4 * a.TB);   // this image slot's scale factors (four columns per tenant)
+                const uint32_t sfb0 = sfa + 4u + (uint32_t)(fr.idx * 4 * a.TB);   // this step's scale factors (four columns per tenant)
                 const uint64_t x4desc = desc64 + ((img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes + a.x_tile_bytes) >> 4);
 #pragma unroll
                 for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
@@ -653,6 +654,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (elect_one()) tc_commit(smem_u32(&ctl->pempty[pr.idx]));
                 __syncwarp();
                 pr.step();
+                fr.step();
             }
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
@@ -676,25 +678,28 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         }
         const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * 32);
         Ring br{0, 0u, a.n_bits}, sr{0, 0u, a.n_sets};
+        const int bits_row = a.bits_row;
+        const bool pair_slots = bits_row == 32;
         int pending = -1;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
             for (int p = p0; p < p1 && ok; ++p) {
-                // a slot holds the steps 2*(p/2) and 2*(p/2)+1: waited for at the first step of it that this segment takes
-                if (p == p0 || (p & 1) == 0) {
+                // 32-byte rows: a slot holds the steps 2*(p/2) and 2*(p/2)+1 and is waited for at the first step of it that
+                // this segment takes; 16-byte rows: a slot per step
+                if (!pair_slots || p == p0 || (p & 1) == 0) {
                     FT_ADD(0);
                     ok = wait_bar(smem_u32(&ctl->bfull[br.idx]), br.par, abort_flag, 6);
                     FT_ADD(1);
                     if (!ok) break;
                 }
                 // this warp's tenants j = 2i + h: their sign words of the step (128 k each)
-                const uint8_t* bsl = smem + bits_off + br.idx * a.bslot_bytes + row * 32 + (p & 1) * 16;
+                const uint8_t* bsl = smem + bits_off + br.idx * a.bslot_bytes + row * bits_row + (pair_slots ? (p & 1) * 16 : 0);
                 uint4 wq[kTenPerWarp];
 #pragma unroll
-                for (int i = 0; i < kTenPerWarp; ++i) wq[i] = *reinterpret_cast<const uint4*>(bsl + (2 * i + h) * (kTileN * 32));
+                for (int i = 0; i < kTenPerWarp; ++i) wq[i] = *reinterpret_cast<const uint4*>(bsl + (2 * i + h) * (kTileN * bits_row));
 #pragma unroll
                 for (int i = 0; i < kTenPerWarp; ++i) asm volatile("" : "+r"(wq[i].x), "+r"(wq[i].w));
-                if ((p & 1) == 1 || p + 1 == p1) {   // the slot's last step in this segment: it goes back
+                if (!pair_slots || (p & 1) == 1 || p + 1 == p1) {   // the slot's last step in this segment: it goes back
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl->bempty[br.idx]));
                     br.step();
@@ -807,7 +812,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // ones whenever their image slot is ready.
         ItemIter si(it);
         bool more_s = si.next();
-        Ring xr{0, 0u, a.n_sf};
+        Ring xr{0, 0u, n_ring}, fr{0, 0u, a.n_sf};
         int n_split = 0, seg_end = 0;
         const int p_first = lo - (int)((unsigned)lo / (unsigned)a.P) * a.P;   // (resident form: the block's first step)
         Unit us{};
@@ -820,6 +825,19 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (!wait_bar(bar, par, abort_flag, 14)) return false;
             } else if (!warp_all(mbar_test_wait(bar, par))) {
                 return false;
+            }
+            if (a.n_sf < n_ring && n_split >= a.n_sf) {
+                // Fewer scale-factor slots in tensor memory than images in shared memory: this step's slot is the one of
+                // the step n_sf before it, whose MMAs must be complete (the issuers' commits on that step's image slot).
+                const int prev = n_split - a.n_sf;
+                const uint32_t pbar = smem_u32(&ctl->pempty[prev % n_ring]);
+                const uint32_t ppar = (uint32_t)(prev / n_ring) & 1u;
+                if (block) {
+                    if (!wait_bar(pbar, ppar, abort_flag, 15)) return false;
+                } else if (!warp_all(mbar_test_wait(pbar, ppar))) {
+                    return false;
+                }
+                tc_fence_after();
             }
             if (si.first) us = unit_info(a, si.unit);
             uint8_t* im = smem + img_off + (a.resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
@@ -836,7 +854,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             }
             {
                 // (a tenant's scale factors start at a multiple of four columns: the MMA wants that alignment)
-                const uint32_t sf_slot = lane_taddr + a.col_sf + 4u + (uint32_t)(xr.idx * 4 * a.TB);
+                const uint32_t sf_slot = lane_taddr + a.col_sf + 4u + (uint32_t)(fr.idx * 4 * a.TB);
                 for (int j = 0; j < us.nten; ++j) {
                     uint32_t sf[2];
 #pragma unroll
@@ -853,6 +871,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->imgready[xr.idx]));
             }
             xr.step();
+            fr.step();
             ++n_split;
             more_s = si.next();
             return true;

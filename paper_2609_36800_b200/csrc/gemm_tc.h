@@ -31,6 +31,7 @@ struct GemmArgs {
     int coop;            // ... the launch's blocks write the images together into the workspace (no pre-pass kernel)
     unsigned int* img_counter;   // ... and count themselves here when their share is written
     int sets_per_step;   // ... operand sets per 128-k step
+    int bits_row;        // ... bytes per row of a sign-word slot: 32 (a slot per two steps) or 16 (a slot per step)
     uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
     uint32_t col_sf;     // ... first scale-factor column in tensor memory
     uint8_t* img;        // ... images written by the pre-pass (or by the launch itself, coop): [group][step][img_bytes]
@@ -66,7 +67,7 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     char* ws = reinterpret_cast<char*>(workspace);
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
     a.fp4 = p.fp4; a.n_img = p.n_img; a.n_sf = p.n_sf; a.resident = p.resident; a.coop = p.coop;
-    a.img_counter = reinterpret_cast<unsigned int*>(ws + p.ws_header_bytes) - 1; a.sets_per_step = p.sets_per_step; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
+    a.img_counter = reinterpret_cast<unsigned int*>(ws + p.ws_header_bytes) - 1; a.sets_per_step = p.sets_per_step; a.bits_row = p.bits_row; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
     a.img = reinterpret_cast<uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
     return a;
 }

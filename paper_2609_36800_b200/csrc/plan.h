@@ -64,11 +64,12 @@ struct Plan {
                        // 256-row MMAs (tcgen05 cta_group::2)
     int fp4;           // 1: the 4-bit decode kernel (gemm_fp4.cu; a pre-pass writes the activation operands)
     int n_img;         // ... ring of activation operand images in shared memory (resident form: one image per step of a block)
-    int n_sf;          // ... slots of B-side scale factors in tensor memory (= n_img unless the images are resident)
+    int n_sf;          // ... slots of B-side scale factors in tensor memory (<= n_img unless the images are resident)
     int coop;          // ... 1: cluster form: the launch's blocks write the activation images together, each a share of them, into
                        //     the workspace before their main loops (no pre-pass kernel); 0: a pre-pass kernel writes them
     int resident;      // ... 1: cluster form with few steps per block and few token rows: every block writes the images of all
                        //     its steps into shared memory itself, right after the grid dependency resolves (no pre-pass kernel)
+    int bits_row;      // ... bytes per row of a sign-word slot: 32 = one slot per two 128-k steps, 16 = one per step
     int sets_per_step; // ... operand sets per 128-k step (2: eight tenants per unit, 1: four)
     uint32_t img_bytes;   // ... one image: 16-bit activation tile (two atoms) + e2m1 piece tile (64 bytes per row)
     uint32_t col_sf;      // ... first scale-factor column in tensor memory (4 for the A side, then the B side's)
@@ -101,6 +102,11 @@ inline int fp4_mode() {
 }
 
 // The cluster form of the 4-bit decode kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
+// (experiments) BITDELTA_FP4_BITS16=0: never the one-step sign-word slots of the 4-bit decode kernel.
+inline bool fp4_bits16_enabled() {
+    const char* e = getenv("BITDELTA_FP4_BITS16");
+    return !(e && e[0] == '0');
+}
 inline bool cluster_enabled() {
     const char* e = getenv("BITDELTA_CLUSTER");
     return !(e && e[0] == '0');
@@ -276,6 +282,19 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         const int fixed = 1024 + kSmemCtrlBytes + p.n_bits * (int)p.bslot_bytes;
         p.n_img = 3;
         p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
+        p.bits_row = 32;
+        if (p.n_w < 3 && fp4_bits16_enabled()) {
+            // Three images do not fit next to three W_base stages: three sign-word slots of one step each (16-byte rows,
+            // the same depth in steps on average) free a quarter of the sign-word memory for the third image.
+            const uint32_t half = p.bslot_bytes / 2;
+            const int nw = (kSmemBudget - 1024 - kSmemCtrlBytes - 3 * (int)half - 3 * (int)p.img_bytes) / (int)p.w_stage_bytes;
+            if (nw >= 3) {
+                p.bits_row = 16;
+                p.bslot_bytes = half;
+                p.n_bits = 3;
+                p.n_w = nw;
+            }
+        }
         if (p.n_w < 3) {
             p.n_img = 2;
             p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
@@ -359,6 +378,13 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         // [base | delta accumulators | scale factors: 4 columns for the A side, 4 per tenant and image slot for the B side |
         //  operand sets of 64 columns]
         p.col_sf = p.col_a;
+        // (the pre-pass form may keep fewer scale-factor slots than images: two are enough to run, and with wide
+        // accumulators the columns are worth more as operand sets)
+        for (;;) {
+            const int col_a = round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_sf, 32);
+            if (p.n_sf <= 2 || p.convert != 0 || p.resident || (kTmemCols - col_a) / kFp4SetCols >= 4) break;
+            --p.n_sf;
+        }
         p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_sf, 32);
         p.halves = 2;
         p.n_sets = (kTmemCols - (int)p.col_a) / kFp4SetCols;
