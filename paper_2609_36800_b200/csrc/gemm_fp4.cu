@@ -61,8 +61,18 @@ __device__ long long* g_fp4_trace = nullptr;
 #define FT_OUT(base, n) do { if (g_fp4_trace && lane == 0) for (int ft_i = 0; ft_i < (n); ++ft_i) g_fp4_trace[(size_t)blockIdx.x * 32 + (base) + ft_i] = ft_acc[ft_i]; } while (0)
 // ... and 16 timestamps (ns, %globaltimer) per block in a second buffer half: [16 .. 31] of the block's second row
 #define FT_STAMP(i) do { if (g_fp4_trace && lane == 0) g_fp4_trace[(size_t)(256 + blockIdx.x) * 32 + (i)] = (long long)global_timer_ns(); } while (0)
+#ifdef BD_TRACE_STEPS   /* per-step event log behind the 512 x 32 words above: [block][step mod 64][16 events], nanoseconds */
+#define FT_EVL(ev, n) do { if (g_fp4_trace) g_fp4_trace[512 * 32 + ((size_t)blockIdx.x * 64 + ((n) & 63)) * 16 + (ev)] = (long long)global_timer_ns(); } while (0)
+#else
+#define FT_EVL(ev, n) do { } while (0)
+#endif
+#define FT_EV(ev, n) do { if (lane == 0) FT_EVL(ev, n); } while (0)
+#define FT_STAMPL(i) do { if (g_fp4_trace) g_fp4_trace[(size_t)(256 + blockIdx.x) * 32 + (i)] = (long long)global_timer_ns(); } while (0)
 #else
 #define FT_STAMP(i) do { } while (0)
+#define FT_STAMPL(i) do { } while (0)
+#define FT_EV(ev, n) do { } while (0)
+#define FT_EVL(ev, n) do { } while (0)
 #define FT_DECL(n) do { } while (0)
 #define FT_ADD(i) do { } while (0)
 #define FT_OUT(base, n) do { } while (0)
@@ -537,6 +547,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint32_t x_atom16 = a.x_atom_bytes >> 4;
         Ring wr{0, 0u, a.n_w}, pr{0, 0u, n_ring};
         uint32_t accphase = 0;
+        [[maybe_unused]] int ev_n = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
@@ -551,12 +562,14 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
                 if (p == p0) FT_STAMP(3);   // first image ready (base issuer)
+                FT_EV(3, ev_n);
                 if (!ok) break;
                 const uint32_t img_s = img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes;
                 const uint64_t xdesc = desc128 + (img_s >> 4);
                 ok = warp_all(wait_bar(smem_u32(&ctl->wfull[wr.idx]), wr.par, abort_flag, 4));
                 FT_ADD(3);
                 if (p == p0) FT_STAMP(4);   // first W_base tile landed
+                FT_EV(4, ev_n);
                 if (p == p1 - 1) FT_STAMP(5);   // last W_base tile landed
                 if (!ok) break;
                 {
@@ -577,6 +590,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (elect_one()) tc_commit(smem_u32(&ctl->pempty[pr.idx]));
                 __syncwarp();
                 pr.step();
+                FT_EV(5, ev_n); ++ev_n;
             }
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
@@ -606,6 +620,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint32_t sfa = tmem_base + a.col_sf;
         Ring pr{0, 0u, n_ring}, fr{0, 0u, a.n_sf}, sr{0, 0u, a.n_sets};
         uint32_t accphase = 0;
+        [[maybe_unused]] int ev_n = 0;
         FT_DECL(8);
         while (ok && it.next(unit, p0, p1)) {
             const Unit u = unit_info(a, unit);
@@ -619,9 +634,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 FT_ADD(0);
                 ok = warp_all(wait_bar(smem_u32(&ctl->imgready[pr.idx]), pr.par, abort_flag, 13));
                 FT_ADD(2);
+                if (h == 0) FT_EV(6, ev_n);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t sfb0 = sfa + 4u + (uint32_t)(fr.idx * 4 * a.TB);   // this step's scale factors (four columns per tenant)
+                const uint32_t sfb0 = sfa + 4u + (uint32_t)(fr.idx * (kTB8 ? 32 : 16));   // this step's scale factors (four columns per tenant)
                 const uint64_t x4desc = desc64 + ((img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes + a.x_tile_bytes) >> 4);
 #pragma unroll
                 for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
@@ -630,6 +646,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                     FT_ADD(0);
                     named_bar_sync(kFBarSet0 + 2 * sr.idx + h, kFHandover);
                     FT_ADD(4);
+                    if (h == 0) FT_EV(7 + s, ev_n);
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_set = tmem_base + a.col_a + (uint32_t)sr.idx * kFp4SetCols + (uint32_t)(h * 32);
@@ -655,6 +672,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 __syncwarp();
                 pr.step();
                 fr.step();
+                if (h == 0) FT_EV(9, ev_n);
+                ++ev_n;
             }
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&ctl->accfull));
@@ -679,6 +698,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const uint32_t tbuf0 = tmem_base + ((uint32_t)(quad * 32) << 16) + a.col_a + (uint32_t)(h * 32);
         Ring br{0, 0u, a.n_bits}, sr{0, 0u, a.n_sets};
         const int bits_row = a.bits_row;
+        [[maybe_unused]] int ev_n = 0;
         const bool pair_slots = bits_row == 32;
         int pending = -1;
         FT_DECL(8);
@@ -692,11 +712,13 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                     FT_ADD(1);
                     if (!ok) break;
                 }
+                if (warp == kFWarpDecode0) FT_EV(10, ev_n);
                 // this warp's tenants j = 2i + h: their sign words of the step (128 k each)
                 const uint8_t* bsl = smem + bits_off + br.idx * a.bslot_bytes + row * bits_row + (pair_slots ? (p & 1) * 16 : 0);
                 uint4 wq[kTenPerWarp];
 #pragma unroll
-                for (int i = 0; i < kTenPerWarp; ++i) wq[i] = *reinterpret_cast<const uint4*>(bsl + (2 * i + h) * (kTileN * bits_row));
+                for (int i = 0; i < kTenPerWarp; ++i)   // (tenants past the unit's own have no words in the slot: nothing is read for them)
+                    wq[i] = (2 * i + h < a.TB) ? *reinterpret_cast<const uint4*>(bsl + (2 * i + h) * (kTileN * bits_row)) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                 for (int i = 0; i < kTenPerWarp; ++i) asm volatile("" : "+r"(wq[i].x), "+r"(wq[i].w));
                 if (!pair_slots || (p & 1) == 1 || p + 1 == p1) {   // the slot's last step in this segment: it goes back
@@ -734,11 +756,13 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                     FT_ADD(2);
                     ok = wait_bar(smem_u32(&ctl->opfree[h][sr.idx]), sr.par ^ 1, abort_flag, 7);
                     FT_ADD(3);
+                    if (warp == kFWarpDecode0) FT_EV(11 + s, ev_n);
                     if (!ok) break;
                     tc_fence_after();
                     tmem_st32(tbuf0 + (uint32_t)sr.idx * kFp4SetCols, r);
                     pending = sr.idx;
                 }
+                ++ev_n;
             }
         }
         if (ok && pending >= 0) {
@@ -817,6 +841,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int p_first = lo - (int)((unsigned)lo / (unsigned)a.P) * a.P;   // (resident form: the block's first step)
         Unit us{};
         const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
+        // (digit row n = q*m + t of a tenant: this lane serves n = lane and n = lane + 32)
+        const int sf_t0 = lane % am, sf_t1 = (lane + 32) % am;
+        const uint32_t sf_q0 = 0x02020202u * (uint32_t)(lane / am), sf_q1 = 0x02020202u * (uint32_t)((lane + 32) / am);
+        const bool sf_v0 = lane < a.Nd, sf_v1 = lane + 32 < a.Nd;
         auto split_next = [&](bool block) -> bool {
             // convert: the slot must be free (its step's MMAs complete); else: its image must have landed
             const uint32_t bar = a.convert ? smem_u32(&ctl->pempty[xr.idx]) : smem_u32(&ctl->pfull[xr.idx]);
@@ -839,6 +867,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 }
                 tc_fence_after();
             }
+            if (warp == kFWarpEpi0) FT_EV(13, n_split);
             if (si.first) us = unit_info(a, si.unit);
             uint8_t* im = smem + img_off + (a.resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
             if (a.convert == 1) {
@@ -853,22 +882,26 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (*abort_flag) return false;
             }
             {
-                // (a tenant's scale factors start at a multiple of four columns: the MMA wants that alignment)
-                const uint32_t sf_slot = lane_taddr + a.col_sf + 4u + (uint32_t)(fr.idx * 4 * a.TB);
-                for (int j = 0; j < us.nten; ++j) {
-                    uint32_t sf[2];
+                // (a tenant's scale factors start at a multiple of four columns: the MMA wants that alignment; all the
+                // tenants' columns of the slot go out in one store, the unused ones with a neutral exponent)
+                const uint32_t sf_slot = lane_taddr + a.col_sf + 4u + (uint32_t)(fr.idx * (kTB8 ? 32 : 16));
+                const uint8_t* tab = im + sf_off;
+                uint32_t r[kTB8 ? 32 : 16];
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int n = lane + 32 * c;
-                        const int q = n / am, t = n - q * am;
-                        sf[c] = (n < a.Nd) ? *reinterpret_cast<const uint32_t*>(im + sf_off + 4 * (j * am + t)) + 0x02020202u * (uint32_t)q : 0x7F7F7F7Fu;
-                    }
-                    tmem_st2(sf_slot + (uint32_t)(4 * j), sf[0], sf[1]);
+                for (int j = 0; j < (kTB8 ? 8 : 4); ++j) {
+                    const bool live = j < us.nten;
+                    r[4 * j] = (live && sf_v0) ? *reinterpret_cast<const uint32_t*>(tab + 4 * (j * am + sf_t0)) + sf_q0 : 0x7F7F7F7Fu;
+                    r[4 * j + 1] = (live && sf_v1) ? *reinterpret_cast<const uint32_t*>(tab + 4 * (j * am + sf_t1)) + sf_q1 : 0x7F7F7F7Fu;
+                    r[4 * j + 2] = 0x7F7F7F7Fu;
+                    r[4 * j + 3] = 0x7F7F7F7Fu;
                 }
+                if constexpr (kTB8) tmem_st32(sf_slot, r);
+                else tmem_st16(sf_slot, r);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->imgready[xr.idx]));
+                if (warp == kFWarpEpi0) FT_EV(14, n_split);
             }
             xr.step();
             fr.step();

@@ -103,6 +103,8 @@ inline int fp4_mode() {
 
 // The cluster form of the 4-bit decode kernel is taken where it applies unless BITDELTA_CLUSTER=0 is set (experiments).
 // (experiments) BITDELTA_FP4_BITS16=0: never the one-step sign-word slots of the 4-bit decode kernel.
+// Columns of one scale-factor slot of the 4-bit decode kernel: four per tenant, written with one store of 16 or 32 columns.
+inline int fp4_sf_slot_cols(int TB) { return TB > 4 ? 32 : 16; }
 inline bool fp4_bits16_enabled() {
     const char* e = getenv("BITDELTA_FP4_BITS16");
     return !(e && e[0] == '0');
@@ -381,11 +383,11 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
         // (the pre-pass form may keep fewer scale-factor slots than images: two are enough to run, and with wide
         // accumulators the columns are worth more as operand sets)
         for (;;) {
-            const int col_a = round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_sf, 32);
+            const int col_a = round_up((int)p.col_sf + 4 + fp4_sf_slot_cols(p.TB) * p.n_sf, 32);
             if (p.n_sf <= 2 || p.convert != 0 || p.resident || (kTmemCols - col_a) / kFp4SetCols >= 4) break;
             --p.n_sf;
         }
-        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + 4 * p.TB * p.n_sf, 32);
+        p.col_a = (uint32_t)round_up((int)p.col_sf + 4 + fp4_sf_slot_cols(p.TB) * p.n_sf, 32);
         p.halves = 2;
         p.n_sets = (kTmemCols - (int)p.col_a) / kFp4SetCols;
         if (p.n_sets > kFp4MaxSets) p.n_sets = kFp4MaxSets;

@@ -31,6 +31,8 @@ SHAPES = [
     ((2, 7, 384, 640), 8),       # 56 digit rows per tenant, five steps over clusters of four
     ((2, 7, 256, 384), 7),       # ... and three steps on two tiles: flat list
     ((1, 8, 2176, 512), 8),      # 17 tiles, ragged last tile
+    ((1, 1, 4096, 4096), 8),     # one tenant, eight steps per block: both sign-word slots in use with three tenant columns of a warp unused
+    ((5, 1, 2048, 4096), 8),     # five of eight tenant columns in use, four steps per block
 ]
 
 
