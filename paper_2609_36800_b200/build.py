@@ -36,8 +36,8 @@ def is_stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
-def _compile(src: str, force: bool, verbose: bool, trace: bool = False) -> str:
-    obj = os.path.join(OBJ, os.path.splitext(src)[0] + (".trace.o" if trace else ".o"))
+def _compile(src: str, force: bool, verbose: bool, trace: bool = False, steps: bool = False) -> str:
+    obj = os.path.join(OBJ, os.path.splitext(src)[0] + (".steps.o" if steps else ".trace.o" if trace else ".o"))
     path = os.path.join(CSRC, src)
     if (not force and os.path.exists(obj) and os.path.getmtime(obj) > os.path.getmtime(path)
             and os.path.getmtime(obj) > _newest_header()):
@@ -47,6 +47,8 @@ def _compile(src: str, force: bool, verbose: bool, trace: bool = False) -> str:
         cmd += ["-Xptxas", "-v"]
     if trace:
         cmd += ["-DBD_TRACE"]
+    if steps:
+        cmd += ["-DBD_TRACE_TIMELINE_ONLY", "-DBD_TRACE_STEPS"]
     subprocess.run(cmd, check=True)
     return obj
 
@@ -61,20 +63,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-def build_trace() -> str:
+def build_trace(steps: bool = False) -> str:
     """The same library with -DBD_TRACE as libbitdelta_trace.so: the 4-bit decode kernel then adds up, per block and
     role, the cycles spent in each kind of wait into a buffer set with bitdelta_debug_set_trace_fp4 (see
-    csrc/gemm_fp4.cu).  Load it by pointing BITDELTA_LIB at it.  Never the default build: the stamps cost time."""
+    csrc/gemm_fp4.cu).  steps=True (libbitdelta_steps.so): no accumulators, but a time stamp per block, step and event
+    behind the first 512 x 32 words of that buffer ([block][step mod 64][16 events]; the buffer must hold them).
+    Load either by pointing BITDELTA_LIB at it.  Never the default build: the stamps cost time."""
     os.makedirs(OBJ, exist_ok=True)
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
-        objs = list(pool.map(lambda s: _compile(s, True, False, trace=True), SOURCES))
-    lib = os.path.join(HERE, "libbitdelta_trace.so")
+        objs = list(pool.map(lambda s: _compile(s, True, False, trace=True, steps=steps), SOURCES))
+    lib = os.path.join(HERE, "libbitdelta_steps.so" if steps else "libbitdelta_trace.so")
     subprocess.run([_nvcc(), *ARCH, "-shared", "-cudart", "shared", "-o", lib, *objs], check=True)
     return lib
 
 
 if __name__ == "__main__":
-    if "--trace" in sys.argv:
+    if "--trace-steps" in sys.argv:
+        print(build_trace(steps=True))
+    elif "--trace" in sys.argv:
         print(build_trace())
     else:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
