@@ -220,65 +220,98 @@ cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int 
 
 // ---------------------------------------------------------------------------------------- compress
 // The step before the product: bits = [W_fine - W_base > 0], alpha[b] = mean |W_fine - W_base|.
-// A warp owns one weight row and 1024 consecutive k of it (one sign word per lane); it keeps its piece of
-// W_base in registers and walks the tenants, so W_base is read once for all of them.  Per thread and
-// tenant: 64 bytes of W_fine in, one word out.  The comparison is taken on the exact bf16 values (as
-// fp32); |delta| is formed in fp32, four at a time, and summed in double: per thread, then across the
-// warp (shuffles) and the block (fixed order) into one partial per block and tenant; a second kernel adds
-// the partials of a tenant in a fixed order.  Nothing depends on the order in which blocks run.
+// A warp takes tiles of one weight row x 1024 consecutive k (one sign word per lane), a fixed stride apart; for each
+// it keeps its piece of W_base in registers (as floats) and walks the tenants, so W_base is read once for all of
+// them.  Per thread and tenant: 64 bytes of W_fine in (two 32-byte loads), one word out.  The comparison is taken on
+// the exact bf16 values (as fp32), through the sign of (base - fine); |delta| is formed in fp32, four at a time, and
+// summed in double: per thread, then across the warp (shuffles), over the warp's tiles and the block (fixed order)
+// into one partial per block and tenant; a second kernel adds the partials of a tenant in a fixed order.  Nothing
+// depends on the order in which blocks run, nor on the device (the grid is a fixed number of blocks).
+// Measured on 8 x 4096 x 4096: 62.5 us = 0.78 of the HBM roofline (66.7 us with a compare and a predicated OR per
+// element and the base weights converted again for every tenant).  Tried without gain: 512 contiguous bytes per load
+// instruction across the warp with the sign bytes put together by shuffles (82-96 us), the next tenant's loads
+// issued one iteration ahead (65 us at 80 registers).
 constexpr int kCompressWarps = 8;
 constexpr int kCompressTenantChunk = 32;   // tenants whose warp sums are staged in shared memory at once
 
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+// 32 bytes (32-byte aligned) through the read-only path in one load.
+__device__ __forceinline__ void ld_nc_256(const uint4* p, uint4& a, uint4& b) {
+    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+                 : "l"(p));
+}
 
 __global__ void __launch_bounds__(kCompressWarps * 32)
 compress_kernel(const uint4* __restrict__ Wf, const uint4* __restrict__ Wb, uint32_t* __restrict__ bits,
                 double* __restrict__ partial, int B, int N, int K, int kchunks, long long tiles) {
     __shared__ double warp_sum[kCompressTenantChunk][kCompressWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long tile = (long long)blockIdx.x * kCompressWarps + warp;
     const int words = K >> 5;
-    const bool tile_ok = tile < tiles;
-    const int n = tile_ok ? (int)(tile / kchunks) : 0;
-    const int w = tile_ok ? (int)(tile - (long long)n * kchunks) * 32 + lane : words;   // this lane's sign word
-    const bool ok = tile_ok && w < words;
-    uint4 wb[4];
-    if (ok) {
-        const uint4* src = Wb + ((size_t)n * K + (size_t)w * 32) / 8;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) wb[i] = __ldg(src + i);
-    }
     for (int b0 = 0; b0 < B; b0 += kCompressTenantChunk) {
         const int nb = min(kCompressTenantChunk, B - b0);
-        for (int bb = 0; bb < nb; ++bb) {
-            const int b = b0 + bb;
-            double acc = 0.0;
-            if (ok) {
-                const uint4* src = Wf + (((size_t)b * N + n) * K + (size_t)w * 32) / 8;
-                uint4 wf[4];
+        for (int bb = lane; bb < nb; bb += 32) warp_sum[bb][warp] = 0.0;
+        __syncwarp();
+        // this warp's tiles (weight row, 1024 k), a fixed stride apart: the grid is a fixed number of blocks (see
+        // compress_blocks), every multiprocessor holds its share of them from the start to the end of the kernel
+        for (long long tile = (long long)blockIdx.x * kCompressWarps + warp; tile < tiles; tile += (long long)gridDim.x * kCompressWarps) {
+            const int n = (int)(tile / kchunks);
+            const int w = (int)(tile - (long long)n * kchunks) * 32 + lane;   // this lane's sign word
+            const bool ok = w < words;
+            // This lane's 32 base weights as floats, once for all tenants of the chunk; x + 0 turns a -0 into +0 (see the
+            // sign rule below).
+            float gf[32];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) wf[i] = __ldg(src + i);
-                uint32_t word = 0;
+            for (int i = 0; i < 32; ++i) gf[i] = 0.f;
+            if (ok) {
+                const uint4* src = Wb + ((size_t)n * K + (size_t)w * 32) / 8;
+                uint4 wb[4];
+                ld_nc_256(src, wb[0], wb[1]);
+                ld_nc_256(src + 2, wb[2], wb[3]);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t f[4] = {wf[i].x, wf[i].y, wf[i].z, wf[i].w};
                     const uint32_t g[4] = {wb[i].x, wb[i].y, wb[i].z, wb[i].w};
-                    float s4[2] = {0.f, 0.f};
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const float f0 = bf16lo(f[q]), f1 = bf16hi(f[q]), g0 = bf16lo(g[q]), g1 = bf16hi(g[q]);
-                        if (f0 > g0) word |= 1u << (i * 8 + q * 2);
-                        if (f1 > g1) word |= 1u << (i * 8 + q * 2 + 1);
-                        s4[q >> 1] += fabsf(f0 - g0) + fabsf(f1 - g1);
+                        gf[i * 8 + q * 2] = __fadd_rn(bf16lo(g[q]), 0.f);
+                        gf[i * 8 + q * 2 + 1] = __fadd_rn(bf16hi(g[q]), 0.f);
                     }
-                    acc += (double)s4[0] + (double)s4[1];
                 }
-                bits[((size_t)b * N + n) * words + w] = word;
             }
+            for (int bb = 0; bb < nb; ++bb) {
+                const int b = b0 + bb;
+                double acc = 0.0;
+                if (ok) {
+                    const uint4* src = Wf + (((size_t)b * N + n) * K + (size_t)w * 32) / 8;
+                    uint4 wf[4];
+                    ld_nc_256(src, wf[0], wf[1]);       // (32 bytes per lane and load)
+                    ld_nc_256(src + 2, wf[2], wf[3]);
+                    // Sign bit k of the word = (fine > base) for element k = the sign of (base - fine), which is +0 when
+                    // the two are equal (a base of -0 was made +0 above): the elements are taken from the last to the
+                    // first and each difference's sign bit is shifted in from the right (one funnel shift per element
+                    // instead of a compare and a predicated OR).
+                    uint32_t word = 0;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (lane == 0) warp_sum[bb][warp] = acc;
+                    for (int i = 3; i >= 0; --i) {
+                        const uint32_t f[4] = {wf[i].x, wf[i].y, wf[i].z, wf[i].w};
+                        float s4[2] = {0.f, 0.f};
+#pragma unroll
+                        for (int q = 3; q >= 0; --q) {
+                            const float d1 = gf[i * 8 + q * 2 + 1] - bf16hi(f[q]);
+                            word = __funnelshift_l(__float_as_uint(d1), word, 1);
+                            const float d0 = gf[i * 8 + q * 2] - bf16lo(f[q]);
+                            word = __funnelshift_l(__float_as_uint(d0), word, 1);
+                            s4[q >> 1] += fabsf(d0) + fabsf(d1);
+                        }
+                        acc += (double)s4[0] + (double)s4[1];
+                    }
+                    bits[((size_t)b * N + n) * words + w] = word;
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (lane == 0) warp_sum[bb][warp] += acc;
+            }
         }
         __syncthreads();
         for (int bb = threadIdx.x; bb < nb; bb += blockDim.x) {
@@ -302,10 +335,14 @@ __global__ void compress_finish_kernel(const double* __restrict__ partial, float
     if (lane == 0) alpha[b] = (float)(t * inv_count);
 }
 
+// Blocks of the compress kernel: one per eight tiles, but never more than a B200 holds at once (148 multiprocessors x 4
+// blocks of 256 threads and 64 registers): a fixed number, so that the order of the sums does not depend on the device.
+constexpr long long kCompressMaxBlocks = 148 * 4;
 long long compress_blocks(int N, int K) {
     const long long kchunks = (K / 32 + 31) / 32;
     const long long tiles = (long long)N * kchunks;
-    return (tiles + kCompressWarps - 1) / kCompressWarps;
+    const long long blocks = (tiles + kCompressWarps - 1) / kCompressWarps;
+    return blocks < kCompressMaxBlocks ? blocks : kCompressMaxBlocks;
 }
 
 cudaError_t launch_compress(const void* Wf, const void* Wb, uint32_t* bits, float* alpha, double* partial, int B, int N,

@@ -40,6 +40,33 @@ def test_compress_matches_oracle(shape):
     assert np.allclose(alpha, ref_alpha, rtol=ALPHA_RTOL, atol=0)
 
 
+def test_compress_equal_weights_and_signed_zeros_give_a_zero_bit():
+    # bit = (fine > base) in IEEE terms: equal values, and +0 against -0 either way round, are NOT greater
+    import torch
+    import paper_2609_36800_b200 as bd
+    B, N, K = 2, 16, 1024
+    fine, W = synth.make_fine_weights(B, N, K, seed=11)
+    fine = fine.copy(); W = W.copy()
+    fine[:, :, 0::7] = W[None, :, 0::7]                 # equal
+    W[:, 1::7] = 0x8000; fine[:, :, 1::7] = 0x0000      # base -0, fine +0
+    W[:, 2::7] = 0x0000; fine[:, :, 2::7] = 0x8000      # base +0, fine -0
+    W[:, 3::7] = 0x8000; fine[:, :, 3::7] = 0x8000      # both -0
+    W[:, 4::7] = 0x8000; fine[0, :, 4::7] = 0x0001      # base -0, fine the smallest positive subnormal: greater
+    fine[1, :, 4::7] = 0x8001                           # ... the smallest negative one: not greater
+    d_fine = torch.from_numpy(fine.view(np.int16)).cuda().view(torch.bfloat16)
+    d_W = torch.from_numpy(W.view(np.int16)).cuda().view(torch.bfloat16)
+    bits, alpha = bd.compress(d_fine, d_W)
+    torch.cuda.synchronize()
+    got = bits.cpu().numpy().view(np.uint32)
+    ref_bits, ref_alpha = oracle.compress(fine, W)
+    assert np.array_equal(got, ref_bits)
+    unpacked = oracle.unpack(ref_bits)                  # (pins the expectation itself: +-1 signs, -1 where not greater)
+    for c in (0, 1, 2, 3):
+        assert (unpacked[:, :, c::7] == -1).all()
+    assert (unpacked[0, :, 4::7] == 1).all() and (unpacked[1, :, 4::7] == -1).all()
+    assert np.allclose(alpha.cpu().numpy(), ref_alpha, rtol=ALPHA_RTOL, atol=0)
+
+
 def test_compress_is_deterministic_and_feeds_the_gemm():
     import torch
     import paper_2609_36800_b200 as bd
