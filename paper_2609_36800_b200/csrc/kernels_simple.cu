@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include "gemm_tc.h"
+#include "ptx.cuh"
 
 namespace bd {
 
@@ -227,10 +228,10 @@ cudaError_t launch_x_split(const void* X, uint8_t* X8, int B, int m, int K, int 
 // summed in double: per thread, then across the warp (shuffles), over the warp's tiles and the block (fixed order)
 // into one partial per block and tenant; a second kernel adds the partials of a tenant in a fixed order.  Nothing
 // depends on the order in which blocks run, nor on the device (the grid is a fixed number of blocks).
-// Measured on 8 x 4096 x 4096: 62.5 us = 0.78 of the HBM roofline (66.7 us with a compare and a predicated OR per
-// element and the base weights converted again for every tenant).  Tried without gain: 512 contiguous bytes per load
-// instruction across the warp with the sign bytes put together by shuffles (82-96 us), the next tenant's loads
-// issued one iteration ahead (65 us at 80 registers).
+// Measured on 8 x 4096 x 4096: 61.4 us per call (0.79 of the HBM roofline), the main kernel alone 60 us: bound by memory
+// latency at half occupancy (eight warps waiting on loads per issued instruction, issue slots 54 % busy).  Tried
+// without gain: 512 contiguous bytes per load instruction across the warp with the sign bytes put together by
+// shuffles (82-96 us), the next tenant's loads issued one iteration ahead (65 us at 80 registers).
 constexpr int kCompressWarps = 8;
 constexpr int kCompressTenantChunk = 32;   // tenants whose warp sums are staged in shared memory at once
 
@@ -249,6 +250,7 @@ compress_kernel(const uint4* __restrict__ Wf, const uint4* __restrict__ Wb, uint
     __shared__ double warp_sum[kCompressTenantChunk][kCompressWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int words = K >> 5;
+    if (threadIdx.x == 0) grid_launch_dependents();   // (the finishing kernel may become resident; it waits for this grid's end)
     for (int b0 = 0; b0 < B; b0 += kCompressTenantChunk) {
         const int nb = min(kCompressTenantChunk, B - b0);
         for (int bb = lane; bb < nb; bb += 32) warp_sum[bb][warp] = 0.0;
@@ -327,6 +329,9 @@ compress_kernel(const uint4* __restrict__ Wf, const uint4* __restrict__ Wb, uint
 // alpha[b] = (sum of the tenant's block partials, in a fixed order) / (N K), rounded to fp32.
 __global__ void compress_finish_kernel(const double* __restrict__ partial, float* __restrict__ alpha, int nblocks,
                                        double inv_count) {
+    // Launched with an early start behind compress_kernel (which releases it at once): resident and waiting when the
+    // partials are complete, instead of a launch gap later.
+    grid_dependency_wait();
     const int b = blockIdx.x, lane = threadIdx.x;
     double t = 0.0;
     for (int i = lane; i < nblocks; i += 32) t += partial[(size_t)b * nblocks + i];
@@ -354,8 +359,18 @@ cudaError_t launch_compress(const void* Wf, const void* Wb, uint32_t* bits, floa
         reinterpret_cast<const uint4*>(Wf), reinterpret_cast<const uint4*>(Wb), bits, partial, B, N, K, kchunks, tiles);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    compress_finish_kernel<<<(unsigned)B, 32, 0, stream>>>(partial, alpha, (int)blocks, 1.0 / ((double)N * (double)K));
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)B);
+    cfg.blockDim = dim3(32u);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, compress_finish_kernel, const_cast<const double*>(partial), alpha, (int)blocks,
+                              1.0 / ((double)N * (double)K));
 }
 
 cudaError_t launch_pack(const int8_t* S, uint32_t* bits, long long words, cudaStream_t stream) {
