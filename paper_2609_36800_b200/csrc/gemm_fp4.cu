@@ -524,15 +524,19 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         if (lane == 0) grid_launch_dependents();
     } else if (warp == kFWarpMma) {
         // -------------------------------------------------------------- MMA issuer
-        grid_dependency_wait();
-        FT_STAMP(1);   // dependency resolved
-        named_bar_arrive(kFBarDep, kFThreads - 32);   // wakes the decode and epilogue warps
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));   // ... and the producer
+        // Tensor memory is taken while the launch before this one may still be running (a block of this kernel fills a
+        // multiprocessor: whatever ran here before has left, and only this library's kernels let a dependent start
+        // early, after all their blocks hold what they need), so that nothing of it is left to do once the
+        // dependency has resolved.
         tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
         tmem_relinquish();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tmemready);
+        grid_dependency_wait();
+        FT_STAMP(1);   // dependency resolved
+        named_bar_arrive(kFBarDep, kFThreads - 32);   // wakes the decode and epilogue warps
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->depready));   // ... and the producer
         (void)wait_bar(tmemready, 0, abort_flag, 20);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
@@ -606,8 +610,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // issuing threads (this pair and the base issuer) are what keeps the per-step instruction count off the
         // critical path.
         const int h = warp - kFWarpDelta0;
-        named_bar_sync(kFBarDep, kFThreads - 32);
         bool ok = warp_all(wait_bar(tmemready, 0, abort_flag, 20));
+        named_bar_sync(kFBarDep, kFThreads - 32);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
         if (a.resident) {
@@ -687,8 +691,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int h = (warp - kFWarpDecode0) >> 2;
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
-        named_bar_sync(kFBarDep, kFThreads - 32);   // (sleeps while the launch before this one is still running)
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);
+        named_bar_sync(kFBarDep, kFThreads - 32);   // (sleeps while the launch before this one is still running)
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
         if (a.resident) {
@@ -786,8 +790,6 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int first_unit = (int)((unsigned)lo / (unsigned)a.P);
         uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
         uint32_t accphase = 0;
-        named_bar_sync(kFBarDep, kFThreads - 32);   // nothing to do before the grid dependency is resolved; sleep until then
-        grid_dependency_wait();                     // (returns at once: orders this thread's accesses behind the previous kernel's)
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
@@ -801,6 +803,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             for (int c = 0; c < 8; ++c) sf[c] = 0x7F7F7F7Fu;
             tmem_st8(lane_taddr + a.col_sf, sf);
         }
+        named_bar_sync(kFBarDep, kFThreads - 32);   // nothing else to do before the grid dependency is resolved; sleep until then
+        grid_dependency_wait();                     // (returns at once: orders this thread's accesses behind the previous kernel's)
         if (a.resident) write_resident_images();
         if (warp == kFWarpEpi0) FT_STAMP(11);   // epilogue warps awake, tensor memory ready
         if (a.coop) {
