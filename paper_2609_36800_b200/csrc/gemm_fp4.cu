@@ -236,7 +236,7 @@ cudaError_t launch_x_split_fp4(const void* X, uint8_t* img, const Plan& p, bool 
 // column 8M*j, digit q of token t in column q*M + t (already weighted by its scale factors).
 //   out(j*M + t) = base + (alpha_j * 2^-14) * sum_q D[q*M + t]
 template <int M, class Out>
-__device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out, const float* alv) {
+__device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out, float al_lane) {
     constexpr int ND = kFp4Pieces * M;
     constexpr int MB = (M <= 1) ? 1 : (M <= 2) ? 2 : (M <= 4) ? 4 : 8;   // base columns read per tenant (a power of two >= M)
 #pragma unroll 1
@@ -254,7 +254,7 @@ __device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, u
         if constexpr (ND % 32 >= 16) tmem_ld16(col + ND / 32 * 32, rd + ND / 32 * 32);
         if constexpr (ND % 16 >= 8) tmem_ld8(col + ND / 16 * 16, rd + ND / 16 * 16);
         tc_wait_ld();
-        const float al = alv[j] * 6.103515625e-05f;   // 2^-14
+        const float al = __shfl_sync(0xFFFFFFFFu, al_lane, j) * 6.103515625e-05f;   // tenant j's scale (held by lane j) x 2^-14
 #pragma unroll
         for (int t = 0; t < M; ++t) {
             float d = 0.f;
@@ -267,16 +267,16 @@ __device__ __forceinline__ void epilogue_fp4(const GemmArgs& a, const Unit& u, u
 
 template <class Out>
 __device__ __forceinline__ void epilogue_fp4_any_m(const GemmArgs& a, const Unit& u, uint32_t lane_taddr, const Out& out,
-                                                   const float* alv, int am) {
+                                                   float al_lane, int am) {
     switch (am) {
-        case 1: epilogue_fp4<1>(a, u, lane_taddr, out, alv); break;
-        case 2: epilogue_fp4<2>(a, u, lane_taddr, out, alv); break;
-        case 3: epilogue_fp4<3>(a, u, lane_taddr, out, alv); break;
-        case 4: epilogue_fp4<4>(a, u, lane_taddr, out, alv); break;
-        case 5: epilogue_fp4<5>(a, u, lane_taddr, out, alv); break;
-        case 6: epilogue_fp4<6>(a, u, lane_taddr, out, alv); break;
-        case 7: epilogue_fp4<7>(a, u, lane_taddr, out, alv); break;
-        default: epilogue_fp4<8>(a, u, lane_taddr, out, alv); break;
+        case 1: epilogue_fp4<1>(a, u, lane_taddr, out, al_lane); break;
+        case 2: epilogue_fp4<2>(a, u, lane_taddr, out, al_lane); break;
+        case 3: epilogue_fp4<3>(a, u, lane_taddr, out, al_lane); break;
+        case 4: epilogue_fp4<4>(a, u, lane_taddr, out, al_lane); break;
+        case 5: epilogue_fp4<5>(a, u, lane_taddr, out, al_lane); break;
+        case 6: epilogue_fp4<6>(a, u, lane_taddr, out, al_lane); break;
+        case 7: epilogue_fp4<7>(a, u, lane_taddr, out, al_lane); break;
+        default: epilogue_fp4<8>(a, u, lane_taddr, out, al_lane); break;
     }
 }
 
@@ -918,9 +918,10 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             const Unit u = unit_info(a, unit);
             const int n = u.n0 + row;
             const bool whole = (p0 == 0 && p1 == a.P);
-            float alv[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) alv[j] = (j < u.nten) ? __ldg(a.alpha + u.tenant0 + j) : 0.f;
+            // Lane j holds tenant j's scale.  ONE register, first read in the drain: an array indexed by the drain's tenant
+            // loop would live in local memory, and storing it there would make this warp wait for the load (DRAM latency
+            // when alpha is cold) right here, before it has handed the first step's scale factors to the issuers.
+            const float al_lane = (lane < u.nten) ? __ldg(a.alpha + u.tenant0 + lane) : 0.f;
             seg_end += p1 - p0;
             while (ok && n_split < seg_end) ok = split_next(true);
             if (!ok) break;
@@ -945,12 +946,12 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 // into it has landed and every MMA that read it has completed), token-major, one float per weight
                 // row; the cluster's leader adds the blocks' partials up at the end of the kernel.
                 const FClusterPartOut out{reinterpret_cast<float*>(smem) + row};
-                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, am);
+                epilogue_fp4_any_m(a, u, lane_taddr, out, al_lane, am);
                 break;   // (one segment per block)
             }
             {
                 const EpiOut<false, false> out{Y, slotp, a.N, n, row, u.xrow0, 0.f, a};
-                epilogue_fp4_any_m(a, u, lane_taddr, out, alv, am);
+                epilogue_fp4_any_m(a, u, lane_taddr, out, al_lane, am);
             }
             // this warp's arrival on the "accumulators drained" barrier
             tc_fence_before();
