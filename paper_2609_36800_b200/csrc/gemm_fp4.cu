@@ -289,12 +289,18 @@ struct FClusterPartOut {
 // kTB8: units of up to eight tenants (m <= 4): two operand sets per 128-k step, a set = all tenants x 64 k; else up to
 // four tenants (m <= 8): one set per step, a set = all tenants x 128 k.  Either way a decode warp stores 32 columns per
 // set: warp (quad, h) owns the weight rows of lane quadrant `quad` and the tenants j = 2i + h.
-template <bool kTB8>
+template <bool kTB8, bool kVariants>
 __global__ void __launch_bounds__(kFThreads, 1)
 bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmBits, const GemmArgs a) {
     constexpr int kSetsPerStep = kTB8 ? 2 : 1;
     constexpr int kTenPerWarp = kTB8 ? 4 : 2;
     constexpr int kTenCols = kTB8 ? 8 : 16;            // columns of one tenant in a set
+    // The opt-in variants (images written in the kernel: by the epilogue warps per step, by all warps up front, or by
+    // the launch's blocks together) have an instantiation of their own: the default one carries none of their code
+    // (the kernel's code is several times the instruction cache as it is).
+    const int v_resident = kVariants ? a.resident : 0;
+    const int v_coop = kVariants ? a.coop : 0;
+    const int v_convert = kVariants ? a.convert : 0;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -303,7 +309,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     const uint32_t bits_off = a.n_w * a.w_stage_bytes;                     // sign-word slots (two steps each)
     const uint32_t bits_addr = base + bits_off;
     const uint32_t img_off = bits_off + a.n_bits * a.bslot_bytes;          // ring of activation images
-    const int n_ring = a.resident ? a.n_sf : a.n_img;                      // ... its slots (resident images: the scale-factor slots)
+    const int n_ring = v_resident ? a.n_sf : a.n_img;                      // ... its slots (resident images: the scale-factor slots)
     const uint32_t img_addr = base + img_off;
     FCtl* ctl = reinterpret_cast<FCtl*>(smem + img_off + a.n_img * a.img_bytes);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
@@ -444,7 +450,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         ItemIter wi(it), bi(it), xi(it);
         Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, n_ring};
         Unit uw{}, ub{}, ux{};
-        bool more_w = wi.next(), more_b = bi.next(), more_x = !a.convert && xi.next();   // (convert: the epilogue warps write the images)
+        bool more_w = wi.next(), more_b = bi.next(), more_x = !v_convert && xi.next();   // (convert: the epilogue warps write the images)
         if (more_w) { uw = unit_info(a, wi.unit); ub = uw; ux = uw; }
         long long t_idle = 0;
         int idle = 0;
@@ -485,7 +491,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             if (!dep_done) {
                 // the weight rings are full and stay full until the grid dependency resolves: sleep until then
                 dep_done = warp_all(mbar_try_wait_hint(smem_u32(&ctl->depready), 0u, 20000u));
-                if (dep_done && a.coop) {
+                if (dep_done && v_coop) {
                     // Cooperative image pass: every block of the launch writes its share of the activation images to
                     // the workspace and counts itself; the images may be fetched once all have (all blocks of a
                     // cluster-form launch are resident together, one per multiprocessor).  Bounded like every wait.
@@ -541,7 +547,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
         bool ok = true;
-        if (a.resident) {
+        if (v_resident) {
             grid_dependency_wait();   // (returns at once: orders this thread's reads of X behind the previous kernel)
             write_resident_images();
         }
@@ -568,7 +574,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (p == p0) FT_STAMP(3);   // first image ready (base issuer)
                 FT_EV(3, ev_n);
                 if (!ok) break;
-                const uint32_t img_s = img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes;
+                const uint32_t img_s = img_addr + (v_resident ? (p - p0) : pr.idx) * a.img_bytes;
                 const uint64_t xdesc = desc128 + (img_s >> 4);
                 ok = warp_all(wait_bar(smem_u32(&ctl->wfull[wr.idx]), wr.par, abort_flag, 4));
                 FT_ADD(3);
@@ -614,7 +620,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         named_bar_sync(kFBarDep, kFThreads - 32);
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
-        if (a.resident) {
+        if (v_resident) {
             grid_dependency_wait();
             write_resident_images();
         }
@@ -642,7 +648,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sfb0 = sfa + 4u + (uint32_t)(fr.idx * (kTB8 ? 32 : 16));   // this step's scale factors (four columns per tenant)
-                const uint64_t x4desc = desc64 + ((img_addr + (a.resident ? (p - p0) : pr.idx) * a.img_bytes + a.x_tile_bytes) >> 4);
+                const uint64_t x4desc = desc64 + ((img_addr + (v_resident ? (p - p0) : pr.idx) * a.img_bytes + a.x_tile_bytes) >> 4);
 #pragma unroll
                 for (int s = 0; s < kSetsPerStep; ++s, sr.step()) {
                     // The 128 decode threads of this half arrive here once their columns of the set are filled (or when
@@ -695,7 +701,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         named_bar_sync(kFBarDep, kFThreads - 32);   // (sleeps while the launch before this one is still running)
         tc_fence_after();
         const uint32_t tmem_base = ctl->tmem_base;
-        if (a.resident) {
+        if (v_resident) {
             grid_dependency_wait();
             write_resident_images();
         }
@@ -805,9 +811,9 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         }
         named_bar_sync(kFBarDep, kFThreads - 32);   // nothing else to do before the grid dependency is resolved; sleep until then
         grid_dependency_wait();                     // (returns at once: orders this thread's accesses behind the previous kernel's)
-        if (a.resident) write_resident_images();
+        if (v_resident) write_resident_images();
         if (warp == kFWarpEpi0) FT_STAMP(11);   // epilogue warps awake, tensor memory ready
-        if (a.coop) {
+        if (v_coop) {
             // This block's share of the launch's activation images (one tenant group): task = (step, token row, chunk).
             const Unit u0 = unit_info(a, 0);
             const uint32_t sf_off0 = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
@@ -851,8 +857,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const bool sf_v0 = lane < a.Nd, sf_v1 = lane + 32 < a.Nd;
         auto split_next = [&](bool block) -> bool {
             // convert: the slot must be free (its step's MMAs complete); else: its image must have landed
-            const uint32_t bar = a.convert ? smem_u32(&ctl->pempty[xr.idx]) : smem_u32(&ctl->pfull[xr.idx]);
-            const uint32_t par = a.convert ? (xr.par ^ 1) : xr.par;
+            const uint32_t bar = v_convert ? smem_u32(&ctl->pempty[xr.idx]) : smem_u32(&ctl->pfull[xr.idx]);
+            const uint32_t par = v_convert ? (xr.par ^ 1) : xr.par;
             if (block) {
                 if (!wait_bar(bar, par, abort_flag, 14)) return false;
             } else if (!warp_all(mbar_test_wait(bar, par))) {
@@ -873,7 +879,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             }
             if (warp == kFWarpEpi0) FT_EV(13, n_split);
             if (si.first) us = unit_info(a, si.unit);
-            uint8_t* im = smem + img_off + (a.resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
+            uint8_t* im = smem + img_off + (v_resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
             if (a.convert == 1) {
                 const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
                 for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
@@ -1063,14 +1069,19 @@ extern "C" int bitdelta_debug_set_trace_fp4(long long* buf) {
 }
 #endif
 
-static void* fp4_kernel(int tb8) {
-    return tb8 ? reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true>) : reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false>);
+static void* fp4_kernel(int mode) {   // mode: bit 0 = units of up to eight tenants, bit 1 = one of the opt-in variants
+    switch (mode) {
+        case 0: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, false>);
+        case 1: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, false>);
+        case 2: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, true>);
+        default: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, true>);
+    }
 }
 
 cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                             bool early_start, cudaStream_t stream) {
-    const int mode = args.sets_per_step == 2 ? 1 : 0;
-    static std::atomic<unsigned char> attr_done[64][2];
+    const int mode = (args.sets_per_step == 2 ? 1 : 0) | ((args.resident || args.coop || args.convert) ? 2 : 0);
+    static std::atomic<unsigned char> attr_done[64][4];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1101,8 +1112,12 @@ cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, c
     }
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
-    if (mode) return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true>, tmW, tmBits, args);
-    return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false>, tmW, tmBits, args);
+    switch (mode) {
+        case 0: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, false>, tmW, tmBits, args);
+        case 1: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, false>, tmW, tmBits, args);
+        case 2: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, true>, tmW, tmBits, args);
+        default: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, true>, tmW, tmBits, args);
+    }
 }
 
 int fp4_max_active_clusters(uint32_t smem_bytes, int cluster) {
@@ -1119,7 +1134,7 @@ int fp4_max_active_clusters(uint32_t smem_bytes, int cluster) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, bitdelta_gemm_fp4_kernel<true>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, bitdelta_gemm_fp4_kernel<true, false>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
