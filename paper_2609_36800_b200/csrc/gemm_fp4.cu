@@ -289,7 +289,7 @@ struct FClusterPartOut {
 // kTB8: units of up to eight tenants (m <= 4): two operand sets per 128-k step, a set = all tenants x 64 k; else up to
 // four tenants (m <= 8): one set per step, a set = all tenants x 128 k.  Either way a decode warp stores 32 columns per
 // set: warp (quad, h) owns the weight rows of lane quadrant `quad` and the tenants j = 2i + h.
-template <bool kTB8, bool kVariants>
+template <bool kTB8, bool kVariants, int kForm>
 __global__ void __launch_bounds__(kFThreads, 1)
 bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmBits, const GemmArgs a) {
     constexpr int kSetsPerStep = kTB8 ? 2 : 1;
@@ -298,6 +298,8 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     // The opt-in variants (images written in the kernel: by the epilogue warps per step, by all warps up front, or by
     // the launch's blocks together) have an instantiation of their own: the default one carries none of their code
     // (the kernel's code is several times the instruction cache as it is).
+    // kForm: 0 = the flat work list only, 1 = the cluster form only, 2 = whichever the launch says (the variants).
+    const bool is_cluster = (kForm == 2) ? (a.cluster > 1) : (kForm == 1);
     const int v_resident = kVariants ? a.resident : 0;
     const int v_coop = kVariants ? a.coop : 0;
     const int v_convert = kVariants ? a.convert : 0;
@@ -326,9 +328,9 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
 
     // Work: an even share of the flat (unit, k-step) list (or whole units round-robin), or, in the cluster form,
     // this block's share of the k-steps of its cluster's unit.
-    const int crank = (a.cluster > 1) ? (int)cluster_ctarank() : 0;
+    const int crank = is_cluster ? (int)cluster_ctarank() : 0;
     int lo, hi;
-    if (a.cluster > 1) {
+    if (is_cluster) {
         const int cunit = (int)blockIdx.x / a.cluster;
         lo = cunit * a.P + (crank * a.P) / a.cluster;
         hi = cunit * a.P + ((crank + 1) * a.P) / a.cluster;
@@ -336,7 +338,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
         hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
     }
-    SegIter it{lo, hi, a.P, (a.whole_units && a.cluster <= 1) ? (int)gridDim.x : 0};
+    SegIter it{lo, hi, a.P, (a.whole_units && !is_cluster) ? (int)gridDim.x : 0};
     int unit, p0, p1;
 
     // The W_base tile of a step (128 rows x 128 k: both 64-k atoms) in one bulk-tensor copy.  One thread.
@@ -936,7 +938,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 if (!split_next(false)) break;
             }
             float* slotp = nullptr;
-            if (!whole && a.cluster <= 1) {
+            if (!whole && !is_cluster) {
                 const int slot = (unit == first_unit) ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1;
                 slotp = a.partials + (size_t)slot * a.slot_floats;
             }
@@ -947,7 +949,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             if (!ok) break;
             tc_fence_after();
             accphase ^= 1;
-            if (a.cluster > 1) {
+            if (is_cluster) {
                 // Cluster form: this block's partial sums go to its own shared memory (the W_base ring: every load
                 // into it has landed and every MMA that read it has completed), token-major, one float per weight
                 // row; the cluster's leader adds the blocks' partials up at the end of the kernel.
@@ -1024,7 +1026,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     }
     tc_fence_after();
     if (warp == kFWarpMma) tmem_dealloc(ctl->tmem_base, kTmemCols);
-    if (a.cluster > 1) {
+    if (is_cluster) {
         // Cluster form: after a cluster barrier the leader's epilogue threads (one weight row each) add the blocks'
         // partial sums in block order, i.e. in k order, through the distributed shared memory window and write Y; a
         // second barrier keeps the other blocks' shared memory alive until it has read them.
@@ -1069,19 +1071,21 @@ extern "C" int bitdelta_debug_set_trace_fp4(long long* buf) {
 }
 #endif
 
-static void* fp4_kernel(int mode) {   // mode: bit 0 = units of up to eight tenants, bit 1 = one of the opt-in variants
+static void* fp4_kernel(int mode) {   // mode: bit 0 = units of up to eight tenants; + 2 = one of the opt-in variants (either form), + 4 = cluster form
     switch (mode) {
-        case 0: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, false>);
-        case 1: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, false>);
-        case 2: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, true>);
-        default: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, true>);
+        case 0: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, false, 0>);
+        case 1: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, false, 0>);
+        case 2: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, true, 2>);
+        case 3: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, true, 2>);
+        case 4: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<false, false, 1>);
+        default: return reinterpret_cast<void*>(bitdelta_gemm_fp4_kernel<true, false, 1>);
     }
 }
 
 cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                             bool early_start, cudaStream_t stream) {
-    const int mode = (args.sets_per_step == 2 ? 1 : 0) | ((args.resident || args.coop || args.convert) ? 2 : 0);
-    static std::atomic<unsigned char> attr_done[64][4];
+    const int mode = (args.sets_per_step == 2 ? 1 : 0) + ((args.resident || args.coop || args.convert) ? 2 : (args.cluster > 1 ? 4 : 0));
+    static std::atomic<unsigned char> attr_done[64][6];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1113,15 +1117,17 @@ cudaError_t launch_gemm_fp4(const CUtensorMap& tmW, const CUtensorMap& tmBits, c
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
     switch (mode) {
-        case 0: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, false>, tmW, tmBits, args);
-        case 1: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, false>, tmW, tmBits, args);
-        case 2: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, true>, tmW, tmBits, args);
-        default: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, true>, tmW, tmBits, args);
+        case 0: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, false, 0>, tmW, tmBits, args);
+        case 1: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, false, 0>, tmW, tmBits, args);
+        case 2: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, true, 2>, tmW, tmBits, args);
+        case 3: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, true, 2>, tmW, tmBits, args);
+        case 4: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<false, false, 1>, tmW, tmBits, args);
+        default: return cudaLaunchKernelEx(&cfg, bitdelta_gemm_fp4_kernel<true, false, 1>, tmW, tmBits, args);
     }
 }
 
 int fp4_max_active_clusters(uint32_t smem_bytes, int cluster) {
-    if (cudaFuncSetAttribute(fp4_kernel(1), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
+    if (cudaFuncSetAttribute(fp4_kernel(5), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(cluster * 16));
     cfg.blockDim = dim3((unsigned)kFThreads);
@@ -1134,7 +1140,7 @@ int fp4_max_active_clusters(uint32_t smem_bytes, int cluster) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, bitdelta_gemm_fp4_kernel<true, false>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, bitdelta_gemm_fp4_kernel<true, false, 1>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
