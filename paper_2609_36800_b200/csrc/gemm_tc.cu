@@ -60,8 +60,8 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= kSmemCtrlBytes, "control block too large");
 
 
-// kMode 0: tiled schedule; 1..4: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any m;
-// 6: tiled schedule with several tenants per unit.
+// kMode 0: tiled schedule; 1..4 and 8: decode schedule with m = kMode tokens per tenant; 5: decode schedule, any other m;
+// 6: tiled schedule with several tenants per unit; 7: tiled schedule on CTA pairs.
 // One instantiation per mode keeps each launched kernel's code small (the roles' loops then stay in the
 // instruction caches) and turns the schedule switches into compile-time constants.
 // kGen: the general form (binary16 I/O, bias, activation); false compiles the plain bf16 product alone, whose
@@ -88,12 +88,12 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
     constexpr bool kGrouped = kMode == 6;   // tiled schedule with several tenants per unit (16 < m <= 64)
     constexpr bool kPair = kMode == 7;      // tiled schedule on CTA pairs (cluster of two, 256-row MMAs)
-    constexpr bool kDec = kMode >= 1 && kMode <= 5;
+    constexpr bool kDec = (kMode >= 1 && kMode <= 5) || kMode == 8;
     // Pair schedule: this CTA's rank in its cluster (0 = leader, issues the MMAs), the leader's view of
     // the barriers both CTAs signal, and the work share of the CLUSTER.
     const uint32_t rank = kPair ? cluster_ctarank() : 0u;
     const int cta_id = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // index into the work split
-    const int am = (kMode >= 1 && kMode <= 4) ? kMode : a.m;
+    const int am = ((kMode >= 1 && kMode <= 4) || kMode == 8) ? kMode : a.m;
     const bool convert = kDec && a.convert != 0;
     const bool io_f16 = kGen && a.f16 != 0;
     auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<kDec, kGrouped, kPair>(aa, un, am, (int)rank); };
@@ -818,7 +818,7 @@ bitdelta_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
             auto drain = [&](auto gate) {
                 constexpr bool kGate = decltype(gate)::value;
                 const EpiOut<kGen, kGate> out{Y, slotp, a.N, n, row, u.xrow0, bias_n, a};
-                if constexpr (kMode >= 1 && kMode <= 4) {
+                if constexpr ((kMode >= 1 && kMode <= 4) || kMode == 8) {
                     epilogue_decode<kMode, kGen>(a, u, lane_taddr, out, alv, al_lane);
                 } else if constexpr (kMode == 5) {
                     switch (am) {
@@ -922,20 +922,20 @@ cudaError_t launch_gemm_tc(const CUtensorMap& tmW, const CUtensorMap& tmX, const
                            const CUtensorMap& tmBits, const GemmArgs& args, int grid, uint32_t smem_bytes,
                            bool early_start, cudaStream_t stream) {
     // the general form only where something beyond the plain bf16 product is asked for
-    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 8 : 0;
-    // 0 tiled, 1..4 decode with that many tokens per tenant, 5 decode with 5..16, 6 tiled with several tenants per unit,
-    // 7 tiled on CTA pairs
-    const int mode = gen + (!args.decode ? (args.pair ? 7 : (args.win_rows > 0 ? 6 : 0)) : (args.m <= 4 ? args.m : 5));
+    const int gen = (args.f16 || args.act || args.bias != nullptr) ? 9 : 0;
+    // 0 tiled, 1..4 and 8 decode with that many tokens per tenant, 5 decode with any other number up to 16, 6 tiled with
+    // several tenants per unit, 7 tiled on CTA pairs
+    const int mode = gen + (!args.decode ? (args.pair ? 7 : (args.win_rows > 0 ? 6 : 0)) : (args.m <= 4 ? args.m : (args.m == 8 ? 8 : 5)));
     using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmArgs);
-    static const KernelFn kernels[16] = {
+    static const KernelFn kernels[18] = {
         bitdelta_gemm_tc_kernel<0, false>, bitdelta_gemm_tc_kernel<1, false>, bitdelta_gemm_tc_kernel<2, false>,
         bitdelta_gemm_tc_kernel<3, false>, bitdelta_gemm_tc_kernel<4, false>, bitdelta_gemm_tc_kernel<5, false>,
-        bitdelta_gemm_tc_kernel<6, false>, bitdelta_gemm_tc_kernel<7, false>,
+        bitdelta_gemm_tc_kernel<6, false>, bitdelta_gemm_tc_kernel<7, false>, bitdelta_gemm_tc_kernel<8, false>,
         bitdelta_gemm_tc_kernel<0, true>,  bitdelta_gemm_tc_kernel<1, true>,  bitdelta_gemm_tc_kernel<2, true>,
         bitdelta_gemm_tc_kernel<3, true>,  bitdelta_gemm_tc_kernel<4, true>,  bitdelta_gemm_tc_kernel<5, true>,
-        bitdelta_gemm_tc_kernel<6, true>,  bitdelta_gemm_tc_kernel<7, true>};
+        bitdelta_gemm_tc_kernel<6, true>,  bitdelta_gemm_tc_kernel<7, true>,  bitdelta_gemm_tc_kernel<8, true>};
     // (per device and instantiation, once; setting it twice from two threads is harmless)
-    static std::atomic<unsigned char> attr_done[64][16];
+    static std::atomic<unsigned char> attr_done[64][18];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;

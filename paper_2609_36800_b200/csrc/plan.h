@@ -94,8 +94,10 @@ inline bool pair_enabled() {
 }
 
 // The 4-bit decode kernel (gemm_fp4.cu; m <= 8, plain bf16 calls).  By default it is taken where it measures faster than
-// the 8-bit decode kernels: where its cluster form applies (one tenant group, clusters of 2-8 blocks per W_base tile).
-// BITDELTA_FP4=1: wherever it applies (also the flat work list); BITDELTA_FP4=0: never.
+// the 8-bit decode kernels: where its cluster form applies (one tenant group, clusters of 2-8 blocks per W_base tile),
+// and on the flat work list with up to four token rows per tenant (5-20 % faster on fifteen shapes from 8 x 2 x 11008 x
+// 4096 to 64 x 1 x 4096 x 4096; with 5-8 rows per tenant its activation images take the room of the W_base stages and the
+// 8-bit kernel stays ahead).  BITDELTA_FP4=1: wherever it applies; BITDELTA_FP4=0: never.
 inline int fp4_mode() {
     const char* e = getenv("BITDELTA_FP4");
     return (e && e[0] == '1') ? 1 : (e && e[0] == '0') ? 0 : 2;
@@ -251,8 +253,8 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             }
         }
     }
-    // (default: the 4-bit kernel only in its cluster form)
-    if (p.fp4 && fp4_mode() == 2 && p.cluster <= 1) return make_plan(B, m, N, K, num_sms, tb_override, whole_override, allow_pair, force_tiled, false);
+    // (default: the flat list of the 4-bit kernel only with up to four token rows per tenant)
+    if (p.fp4 && fp4_mode() == 2 && p.cluster <= 1 && m > 4) return make_plan(B, m, N, K, num_sms, tb_override, whole_override, allow_pair, force_tiled, false);
 
     p.w_atom_bytes = kTileN * 128;
     p.x_atom_bytes = (uint32_t)p.x_rows * 128;

@@ -51,7 +51,9 @@ def test_fp4_kernel_matches_oracle(shape, schedule, inkernel, monkeypatch):
     assert rel_fro > 1e-5 or max_abs == 0.0   # (a bf16 result cannot sit closer to the fp64 one: guards against comparing a thing with itself)
 
 
-@pytest.mark.parametrize("shape", [(8, 1, 1024, 1024), (3, 2, 384, 640), (1, 1, 2048, 1024), (8, 1, 4096, 4096)], ids=str)
+# (shapes whose clusters are of two or four blocks: a B200 holds all of them at once; clusters of eight that do not all
+# fit are planned as the flat list by the library, where this variant does not apply)
+@pytest.mark.parametrize("shape", [(8, 1, 1024, 1024), (3, 2, 384, 640), (1, 1, 4096, 1024), (8, 1, 4096, 4096)], ids=str)
 def test_fp4_kernel_resident_images_variant(shape, monkeypatch):
     # BITDELTA_FP4_RESIDENT=1: every block writes the images of all its steps into shared memory itself (no pre-pass kernel)
     monkeypatch.setenv("BITDELTA_FP4_RESIDENT", "1")

@@ -80,7 +80,10 @@ def test_schedules_and_work_orders_of_the_measured_workloads():
     # one tenant group, eight tokens per unit: the 4-bit decode kernel in clusters of four blocks per W_base tile
     assert got["decode_attn"]["schedule"] == 8 and got["decode_attn"]["order"] == 3 and got["decode_attn"]["blocks"] == 128
     assert got["tiny"]["schedule"] == 2
-    assert got["decode_mlp_up"]["schedule"] == 1 and got["decode_mlp_up"]["order"] == 2 and got["decode_mlp_up"]["teams"] == 2
+    # two tenant groups of four token rows per tenant: the 4-bit decode kernel on the flat list, one team per group
+    assert got["decode_mlp_up"]["schedule"] == 7 and got["decode_mlp_up"]["order"] == 2 and got["decode_mlp_up"]["teams"] == 2
+    # eight token rows per tenant, eight groups: the 8-bit decode kernel
+    assert got["many_tenant_down"]["schedule"] == 1
     assert got["many_tenant_down"]["order"] == 2 and got["many_tenant_down"]["teams"] == 8 and got["many_tenant_down"]["blocks"] == 144
     assert got["prefill"]["schedule"] == 4 and got["prefill"]["order"] == 0 and got["prefill"]["blocks"] == 148
     for g in got.values():
@@ -88,9 +91,11 @@ def test_schedules_and_work_orders_of_the_measured_workloads():
 
 
 def test_four_bit_decode_kernel_plans(monkeypatch):
-    # default: only where its cluster form applies; BITDELTA_FP4=0 never; BITDELTA_FP4=1 also on the flat work list
+    # default: where its cluster form applies, and on the flat work list with up to four token rows per tenant;
+    # BITDELTA_FP4=0 never; BITDELTA_FP4=1 wherever it applies
     assert bd.gemm_plan(8, 1, 4096, 4096)["schedule"] == 8 and bd.gemm_plan(4, 8, 4096, 4096)["schedule"] == 8
-    assert bd.gemm_plan(16, 1, 4096, 4096)["schedule"] == 2          # two tenant groups: no clusters
+    assert bd.gemm_plan(16, 1, 4096, 4096)["schedule"] == 7          # two tenant groups: no clusters, the flat list
+    assert bd.gemm_plan(16, 8, 4096, 4096)["schedule"] in (1, 2)     # ... with more than four token rows per tenant: the 8-bit kernel
     assert bd.gemm_plan(8, 9, 4096, 4096)["schedule"] == 1           # more than eight tokens per tenant
     one = bd.gemm_plan(8, 1, 4096, 4096)
     assert one["smem_bytes"] <= 227 * 1024 and one["w_ring"] >= 3
