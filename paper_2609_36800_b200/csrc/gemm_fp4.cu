@@ -286,6 +286,56 @@ struct FClusterPartOut {
     __device__ __forceinline__ void put(int tok, float v) const { part_row[tok * kTileN] = v; }
 };
 
+// The walk over a block's (unit, step) items.  Cluster form (kForm 1): one segment of one unit per block, known without a
+// division; the other forms walk the flat list like the 8-bit kernels (gemm_common.cuh).  Every role holds a copy of this
+// code and the kernel's speed depends on its length.
+template <int kForm>
+struct FSeg {
+    int cur, hi;
+    int P;
+    int stride;   // flat list, whole units: > 0 = units cur/P, cur/P + stride, ...
+    int unit1;    // cluster form: the cluster's unit
+    __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
+        if (cur >= hi) return false;
+        if constexpr (kForm == 1) {
+            unit = unit1;
+            p0 = cur - unit1 * P;
+            p1 = hi - unit1 * P;
+            cur = hi;
+            return true;
+        } else {
+            unit = (int)((unsigned)cur / (unsigned)P);
+            if (stride > 0) {
+                p0 = 0;
+                p1 = P;
+                cur += stride * P;
+                return true;
+            }
+            p0 = cur - unit * P;
+            const int rem = hi - cur;
+            const int len = (rem < P - p0) ? rem : (P - p0);
+            p1 = p0 + len;
+            cur += len;
+            return true;
+        }
+    }
+};
+template <int kForm>
+struct FItem {
+    FSeg<kForm> seg;
+    int unit, p, p1;
+    bool first;   // first item of its segment
+    __device__ __forceinline__ explicit FItem(const FSeg<kForm>& s) : seg(s), unit(0), p(0), p1(0), first(false) {}
+    __device__ __forceinline__ bool next() {
+        if (p + 1 < p1) { ++p; first = false; return true; }
+        int p0;
+        if (!seg.next(unit, p0, p1)) { p = 0; p1 = 0; return false; }
+        p = p0;
+        first = true;
+        return true;
+    }
+};
+
 // kTB8: units of up to eight tenants (m <= 4): two operand sets per 128-k step, a set = all tenants x 64 k; else up to
 // four tenants (m <= 8): one set per step, a set = all tenants x 128 k.  Either way a decode warp stores 32 columns per
 // set: warp (quad, h) owns the weight rows of lane quadrant `quad` and the tenants j = 2i + h.
@@ -317,7 +367,19 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     volatile uint32_t* abort_flag = &ctl->abort_flag;
 
     const int am = a.m;
-    auto unit_info = [&](const GemmArgs& aa, int un) { return unit_info_t<true, false, false>(aa, un, am, 0); };
+    auto unit_info = [&](const GemmArgs& aa, int un) {
+        if constexpr (kForm == 1) {   // (cluster form: one tenant group, no teams)
+            Unit u;
+            u.n0 = un * kTileN;
+            u.tenant0 = 0;
+            u.nten = min(aa.TB, aa.B);
+            u.xrow0 = 0;
+            u.ntok = u.nten * am;
+            return u;
+        } else {
+            return unit_info_t<true, false, false>(aa, un, am, 0);
+        }
+    };
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     if (warp == 0) FT_STAMP(0);   // block start
@@ -329,16 +391,17 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     // Work: an even share of the flat (unit, k-step) list (or whole units round-robin), or, in the cluster form,
     // this block's share of the k-steps of its cluster's unit.
     const int crank = is_cluster ? (int)cluster_ctarank() : 0;
-    int lo, hi;
+    int lo, hi, cunit = 0;
     if (is_cluster) {
-        const int cunit = (int)blockIdx.x / a.cluster;
-        lo = cunit * a.P + (crank * a.P) / a.cluster;
-        hi = cunit * a.P + ((crank + 1) * a.P) / a.cluster;
+        const int cshift = 31 - __clz(a.cluster);   // (clusters of 2, 4 or 8 blocks)
+        cunit = (int)(blockIdx.x >> cshift);
+        lo = cunit * a.P + ((crank * a.P) >> cshift);
+        hi = cunit * a.P + (((crank + 1) * a.P) >> cshift);
     } else {
         lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
         hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
     }
-    SegIter it{lo, hi, a.P, (a.whole_units && !is_cluster) ? (int)gridDim.x : 0};
+    FSeg<kForm> it{lo, hi, a.P, (a.whole_units && !is_cluster) ? (int)gridDim.x : 0, cunit};
     int unit, p0, p1;
 
     // The W_base tile of a step (128 rows x 128 k: both 64-k atoms) in one bulk-tensor copy.  One thread.
@@ -392,7 +455,6 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     // Resident form (cluster form, one segment per block): once the grid dependency has resolved, all warps but the
     // producer write the images of all the block's steps, one task per thread and (token row, 16-byte chunk, step).
     auto write_resident_images = [&]() {
-        const int cunit = (int)blockIdx.x / a.cluster;
         const Unit u = unit_info(a, cunit);
         const int q0 = lo - cunit * a.P, nsteps = hi - lo;
         const int tid = (int)threadIdx.x - 32;
@@ -449,7 +511,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // Walks the block's steps three times over, once per stream: W_base tiles and sign words (never written by
         // another kernel: queued before the grid dependency is resolved, as far as their rings allow) and activation
         // images (written by the pre-pass kernel queued before this one: only afterwards).
-        ItemIter wi(it), bi(it), xi(it);
+        FItem<kForm> wi(it), bi(it), xi(it);
         Ring wr{0, 0u, a.n_w}, br{0, 0u, a.n_bits}, xr{0, 0u, n_ring};
         Unit uw{}, ub{}, ux{};
         bool more_w = wi.next(), more_b = bi.next(), more_x = !v_convert && xi.next();   // (convert: the epilogue warps write the images)
@@ -795,7 +857,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int etid = threadIdx.x - kFWarpEpi0 * 32;
-        const int first_unit = (int)((unsigned)lo / (unsigned)a.P);
+        const int first_unit = (kForm == 1) ? cunit : (int)((unsigned)lo / (unsigned)a.P);
         uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
         uint32_t accphase = 0;
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);
@@ -846,11 +908,11 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         // column 4 TB slot + 4 j + n / 32, one byte per 32-k group of the step: the group's exponent + 2q.
         // Steps of the current tile are served with blocking waits (the tile cannot complete without them), later
         // ones whenever their image slot is ready.
-        ItemIter si(it);
+        FItem<kForm> si(it);
         bool more_s = si.next();
         Ring xr{0, 0u, n_ring}, fr{0, 0u, a.n_sf};
         int n_split = 0, seg_end = 0;
-        const int p_first = lo - (int)((unsigned)lo / (unsigned)a.P) * a.P;   // (resident form: the block's first step)
+        const int p_first = is_cluster ? lo - cunit * a.P : lo - (int)((unsigned)lo / (unsigned)a.P) * a.P;   // (resident form: the block's first step)
         Unit us{};
         const uint32_t sf_off = a.x_tile_bytes + (uint32_t)(a.TB * a.Nd) * 64u;
         // (digit row n = q*m + t of a tenant: this lane serves n = lane and n = lane + 32)
@@ -1033,7 +1095,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         cluster_sync_all();
         if (warp == 0) FT_STAMP(8);   // cluster barrier passed
         if (crank == 0 && warp >= kFWarpEpi0 && lo < hi && !*abort_flag) {
-            const Unit u = unit_info(a, (int)blockIdx.x / a.cluster);
+            const Unit u = unit_info(a, cunit);
             const int row = (warp & 3) * 32 + lane;
             const int n = u.n0 + row;
             const uint32_t part = base + (uint32_t)row * 4u;   // this block's part[0][row]; same offset in every block
