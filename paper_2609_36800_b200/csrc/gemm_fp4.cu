@@ -996,8 +996,11 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             while (ok && n_split < seg_end) ok = split_next(true);
             if (!ok) break;
             // until this tile's accumulators are complete: serve ahead whatever image slot is ready
-            while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
-                if (!split_next(false)) break;
+            // (cluster form: the block has no other segment, and the kernel is better off without a second copy of that code)
+            if constexpr (kForm != 1) {
+                while (more_s && !warp_all(mbar_test_wait(smem_u32(&ctl->accfull), accphase))) {
+                    if (!split_next(false)) break;
+                }
             }
             float* slotp = nullptr;
             if (!whole && !is_cluster) {
