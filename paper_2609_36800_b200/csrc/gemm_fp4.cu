@@ -289,12 +289,16 @@ struct FClusterPartOut {
 // The walk over a block's (unit, step) items.  Cluster form (kForm 1): one segment of one unit per block, known without a
 // division; the other forms walk the flat list like the 8-bit kernels (gemm_common.cuh).  Every role holds a copy of this
 // code and the kernel's speed depends on its length.
+// x / d by the multiplier of d (ceil(2^32 / d), 0 for d = 1; exact while x * d < 2^32: the plan sees to that).
+__device__ __forceinline__ int fdiv(int x, uint32_t mg) { return mg ? (int)__umulhi((unsigned)x, mg) : x; }
+
 template <int kForm>
 struct FSeg {
     int cur, hi;
     int P;
     int stride;   // flat list, whole units: > 0 = units cur/P, cur/P + stride, ...
     int unit1;    // cluster form: the cluster's unit
+    uint32_t mg_P;   // flat list: the multiplier of P (fdiv)
     __device__ __forceinline__ bool next(int& unit, int& p0, int& p1) {
         if (cur >= hi) return false;
         if constexpr (kForm == 1) {
@@ -304,7 +308,7 @@ struct FSeg {
             cur = hi;
             return true;
         } else {
-            unit = (int)((unsigned)cur / (unsigned)P);
+            unit = fdiv(cur, mg_P);
             if (stride > 0) {
                 p0 = 0;
                 p1 = P;
@@ -376,8 +380,22 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             u.xrow0 = 0;
             u.ntok = u.nten * am;
             return u;
-        } else {
-            return unit_info_t<true, false, false>(aa, un, am, 0);
+        } else {   // (the look-up of gemm_common.cuh for the decode schedules, its divisions by multipliers)
+            Unit u;
+            int nt, g;
+            if (aa.teams > 1) {   // group-major
+                g = fdiv(un, aa.mg_tiles);
+                nt = un - g * aa.n_tiles;
+            } else {
+                nt = fdiv(un, aa.mg_groups);
+                g = un - nt * aa.groups;
+            }
+            u.n0 = nt * kTileN;
+            u.tenant0 = g * aa.TB;
+            u.nten = min(aa.TB, aa.B - u.tenant0);
+            u.xrow0 = u.tenant0 * am;
+            u.ntok = u.nten * am;
+            return u;
         }
     };
     const int warp = threadIdx.x >> 5;
@@ -401,7 +419,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         lo = a.whole_units ? (int)blockIdx.x * a.P : cta_first_item(a, (int)blockIdx.x);
         hi = a.whole_units ? (int)a.T : cta_first_item(a, (int)blockIdx.x + 1);
     }
-    FSeg<kForm> it{lo, hi, a.P, (a.whole_units && !is_cluster) ? (int)gridDim.x : 0, cunit};
+    FSeg<kForm> it{lo, hi, a.P, (a.whole_units && !is_cluster) ? (int)gridDim.x : 0, cunit, a.mg_P};
     int unit, p0, p1;
 
     // The W_base tile of a step (128 rows x 128 k: both 64-k atoms) in one bulk-tensor copy.  One thread.
@@ -421,7 +439,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
     auto issue_img = [&](const Unit& u, int p, int slot) {
         const uint32_t bar = smem_u32(&ctl->pfull[slot]);
         mbar_arrive_expect_tx(bar, a.img_bytes);
-        const int g = (int)((unsigned)u.tenant0 / (unsigned)a.TB);
+        const int g = fdiv(u.tenant0, a.mg_TB);
         bulk_load(img_addr + slot * a.img_bytes, a.img + ((size_t)g * a.P + p) * a.img_bytes, a.img_bytes, bar);
     };
     if (threadIdx.x == 0) {
@@ -857,7 +875,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int etid = threadIdx.x - kFWarpEpi0 * 32;
-        const int first_unit = (kForm == 1) ? cunit : (int)((unsigned)lo / (unsigned)a.P);
+        const int first_unit = (kForm == 1) ? cunit : fdiv(lo, a.mg_P);
         uint16_t* Y = reinterpret_cast<uint16_t*>(a.Y);
         uint32_t accphase = 0;
         bool ok = wait_bar(tmemready, 0, abort_flag, 20);

@@ -31,6 +31,7 @@ struct GemmArgs {
     int coop;            // ... the launch's blocks write the images together into the workspace (no pre-pass kernel)
     unsigned int* img_counter;   // ... and count themselves here when their share is written
     int sets_per_step;   // ... operand sets per 128-k step
+    uint32_t mg_P, mg_tiles, mg_groups, mg_TB;   // ... ceil(2^32 / d) for d = P, n_tiles, groups, TB (0 for d = 1): x / d = umulhi(x, mg) while x * d < 2^32
     int bits_row;        // ... bytes per row of a sign-word slot: 32 (a slot per two steps) or 16 (a slot per step)
     uint32_t img_bytes;  // ... bytes of one image (16-bit activation tile, then the e2m1 piece tile)
     uint32_t col_sf;     // ... first scale-factor column in tensor memory
@@ -46,6 +47,8 @@ struct GemmArgs {
     float* partials;
 };
 
+// ceil(2^32 / d) (0 for d <= 1): x / d = umulhi(x, magic) as long as x * d < 2^32.
+inline uint32_t magic_u32(int d) { return d <= 1 ? 0u : (uint32_t)((0x100000000ull + (unsigned long long)d - 1ull) / (unsigned long long)d); }
 inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* workspace) {
     GemmArgs a{};
     a.B = p.B; a.m = p.m; a.N = p.N; a.K = p.K;
@@ -67,7 +70,8 @@ inline GemmArgs make_args(const Plan& p, const float* alpha, void* Y, void* work
     char* ws = reinterpret_cast<char*>(workspace);
     a.partials = reinterpret_cast<float*>(ws + p.ws_header_bytes);
     a.fp4 = p.fp4; a.n_img = p.n_img; a.n_sf = p.n_sf; a.resident = p.resident; a.coop = p.coop;
-    a.img_counter = reinterpret_cast<unsigned int*>(ws + p.ws_header_bytes) - 1; a.sets_per_step = p.sets_per_step; a.bits_row = p.bits_row; a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
+    a.img_counter = reinterpret_cast<unsigned int*>(ws + p.ws_header_bytes) - 1; a.sets_per_step = p.sets_per_step; a.bits_row = p.bits_row;
+    a.mg_P = magic_u32(p.P); a.mg_tiles = magic_u32(p.n_tiles); a.mg_groups = magic_u32(p.groups); a.mg_TB = magic_u32(p.TB); a.img_bytes = p.img_bytes; a.col_sf = p.col_sf;
     a.img = reinterpret_cast<uint8_t*>(ws + p.ws_header_bytes + p.ws_partials_bytes);
     return a;
 }

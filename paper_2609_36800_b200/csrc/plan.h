@@ -253,6 +253,13 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             }
         }
     }
+    // (the 4-bit kernel divides item and unit numbers by multipliers that are exact while the product stays below 2^32)
+    if (p.fp4) {
+        int dmax = p.P > p.n_tiles ? p.P : p.n_tiles;
+        if (p.groups > dmax) dmax = p.groups;
+        if ((unsigned long long)p.T * (unsigned long long)dmax >= 0x100000000ull)
+            return make_plan(B, m, N, K, num_sms, tb_override, whole_override, allow_pair, force_tiled, false);
+    }
     // (default: the flat list of the 4-bit kernel only with up to four token rows per tenant)
     if (p.fp4 && fp4_mode() == 2 && p.cluster <= 1 && m > 4) return make_plan(B, m, N, K, num_sms, tb_override, whole_override, allow_pair, force_tiled, false);
 
