@@ -962,7 +962,7 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
             if (warp == kFWarpEpi0) FT_EV(13, n_split);
             if (si.first) us = unit_info(a, si.unit);
             uint8_t* im = smem + img_off + (v_resident ? (si.p - p_first) : xr.idx) * a.img_bytes;
-            if (a.convert == 1) {
+            if (v_convert == 1) {
                 const uint16_t* xstep = reinterpret_cast<const uint16_t*>(a.X) + (size_t)us.xrow0 * a.K + (size_t)si.p * kPairK;
                 for (int task = etid; task < us.ntok * 16; task += kFEpiWarps * 32) {
                     const int r = task >> 4;
