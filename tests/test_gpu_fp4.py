@@ -204,13 +204,16 @@ def test_calls_with_options_keep_the_eight_bit_kernels():
     assert np.max(np.abs(d)) <= 2e-2
 
 
-@pytest.mark.parametrize("fp4", ["default", "0"], ids=["4bit_kernel", "8bit_kernel"])
-def test_three_hundred_back_to_back_launches_are_bit_identical(fp4, monkeypatch):
+@pytest.mark.parametrize("fp4,workload", [("default", "decode_attn"), ("0", "decode_attn"), ("default", "flat")],
+                         ids=["4bit_kernel_clusters", "8bit_kernel", "4bit_kernel_flat_list"])
+def test_three_hundred_back_to_back_launches_are_bit_identical(fp4, workload, monkeypatch):
     # A stress run of this kind (outputs of every launch compared bit for bit with the first) is what exposed an
     # intermittent fault in an earlier experimental kernel that single-launch parity tests passed: keep it.
     if fp4 != "default":
         monkeypatch.setenv("BITDELTA_FP4", fp4)
-    wl = synth.WORKLOADS_BY_NAME["decode_attn"]
+    # (flat: two tenant groups of four token rows per tenant, several cut tiles per block: the 4-bit kernel's flat list)
+    wl = synth.WORKLOADS_BY_NAME["decode_attn"] if workload == "decode_attn" else synth.Workload("flat", B=16, m=4, K=2048, N=2176, seed=5)
+    assert bd.gemm_plan(wl.B, wl.m, wl.N, wl.K)["schedule"] == {"default": 8 if workload == "decode_attn" else 7, "0": 2}[fp4]
     X, W, bits, alpha = synth.make_inputs(wl)
     dX, dW, dbits, dalpha = to_device(X, W, bits, alpha)
     ws = bd.make_workspace(wl.B, wl.m, wl.N, wl.K)
@@ -226,4 +229,4 @@ def test_three_hundred_back_to_back_launches_are_bit_identical(fp4, monkeypatch)
                 assert torch.equal(h, first), f"{int((h != first).sum())} outputs differ from the first launch"
     st, site = bd.last_device_status()
     assert st == 0, (st, site)
-    assert_parity(y_to_f64(first.view(torch.bfloat16)), oracle.gemm(X, W, bits, alpha), "decode_attn")
+    assert_parity(y_to_f64(first.view(torch.bfloat16)), oracle.gemm(X, W, bits, alpha), wl.name)
