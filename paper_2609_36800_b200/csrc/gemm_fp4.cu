@@ -571,8 +571,23 @@ bitdelta_gemm_fp4_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_c
                 continue;
             }
             if (!dep_done) {
-                // the weight rings are full and stay full until the grid dependency resolves: sleep until then
+                // The weight rings are full and stay full until the grid dependency resolves: sleep until then.  The first
+                // image's source is worked out before, and requested right behind the wait (a few instructions next
+                // to the ones this warp has been executing, instead of another trip around the loop).
+                const uint8_t* first_src = nullptr;
+                if (more_x && !v_coop) first_src = a.img + ((size_t)fdiv(ux.tenant0, a.mg_TB) * a.P + xi.p) * a.img_bytes;
                 dep_done = warp_all(mbar_try_wait_hint(smem_u32(&ctl->depready), 0u, 20000u));
+                if (dep_done && first_src != nullptr) {
+                    if (elect_one()) {   // (the image ring is empty: slot 0, first use)
+                        const uint32_t bar = smem_u32(&ctl->pfull[0]);
+                        mbar_arrive_expect_tx(bar, a.img_bytes);
+                        bulk_load(img_addr, first_src, a.img_bytes, bar);
+                    }
+                    __syncwarp();
+                    xr.step();
+                    more_x = xi.next();
+                    if (more_x && xi.first) ux = unit_info(a, xi.unit);
+                }
                 if (dep_done && v_coop) {
                     // Cooperative image pass: every block of the launch writes its share of the activation images to
                     // the workspace and counts itself; the images may be fetched once all have (all blocks of a
