@@ -311,6 +311,10 @@ inline Plan make_plan(int B, int m, int N, int K, int num_sms, int tb_override =
             p.n_w = (kSmemBudget - fixed - p.n_img * (int)p.img_bytes) / (int)p.w_stage_bytes;
         }
         if (p.n_w > 4) p.n_w = 4;
+        // (eight tenants of one token row: a fourth W_base stage measured SLOWER than three: 8 x 1 x 4096 x 4096 14.85 vs 14.45
+        // us, K = 8192 24.7 vs 23.8, 16 x 1 x 4096 x 4096 25.5 vs 24.7, 8 x 1 x 4096 x 11008 31.1 vs 29.7; with fewer tenants per
+        // unit or more token rows per tenant the two are level or the fourth stage is ahead by 0.1-0.2 us)
+        if (p.n_w > 3 && p.TB > 4 && m == 1) p.n_w = 3;
         p.n_sf = p.n_img;
         p.resident = 0;
         if (p.cluster > 1 && p.TB * m <= 16 && p.convert == 0 && getenv("BITDELTA_FP4_RESIDENT") != nullptr) {
